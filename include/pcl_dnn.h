@@ -1,0 +1,157 @@
+/*
+ * pcl_dnn.h -- C ABI of the B200 (sm_100a) compute library for the training
+ * hot path of synchronous SGD: convolution forward / backward-data /
+ * weight-gradient, the fully-connected GEMMs, and the SGD weight update,
+ * over a whole minibatch.
+ *
+ * Conventions that hold for every entry point
+ * -------------------------------------------
+ *  - All tensor pointers are DEVICE pointers to fp32 data, contiguous, and at
+ *    least 16-byte aligned.  The caller owns every buffer, including the
+ *    workspace; the library allocates no device memory.
+ *  - Layouts: activations and their gradients are NHWC (N minibatch, H x W
+ *    feature map, C feature maps innermost); convolution weights and their
+ *    gradients are KRSC (K output maps, R x S kernel, C input maps innermost);
+ *    fully-connected weights are [K][C]; outputs of a convolution are NPQK
+ *    with P = floor((H + 2*pad_h - R)/stride_h) + 1 (same for Q).
+ *  - Outputs are overwritten, never accumulated into.
+ *  - `cuda_stream` is a cudaStream_t passed as void* (NULL = default stream).
+ *    Every call only enqueues work on that stream and returns; none
+ *    synchronises except pcl_last_device_status().
+ *  - Return value: PCL_OK or an error code; nothing throws or aborts.  On any
+ *    error other than PCL_ERR_DEVICE_TIMEOUT no kernel has been launched.
+ *  - Arithmetic: contractions multiply in TF32 (fp32 operands, 10-bit mantissa
+ *    inside the tensor core, or full fp32 on the generic kernels) and
+ *    accumulate in fp32; elementwise work is fp32.
+ *  - Device-side waits are bounded.  A wait that runs out makes the kernel set
+ *    a device status word and return early (outputs then undefined);
+ *    pcl_last_device_status() reports it as PCL_ERR_DEVICE_TIMEOUT.
+ */
+#ifndef PCL_DNN_H
+#define PCL_DNN_H
+
+#include <stddef.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+/* Layer parameters of a 2-D convolution: minibatch, input feature maps,
+ * output feature maps, input height/width, kernel height/width, strides and
+ * zero padding (the parameters of Algorithm 1, with the printed "- 1" offset
+ * generalised to "- pad"). */
+typedef struct {
+    int N, C, K, H, W, R, S, stride_h, stride_w, pad_h, pad_w;
+} pcl_conv_desc;
+
+enum { PCL_ACT_NONE = 0, PCL_ACT_RELU = 1, PCL_ACT_SIGMOID = 2 };
+
+enum {
+    PCL_OK = 0,
+    PCL_ERR_BAD_ARG = 1,           /* null pointer, non-positive size, unknown enum   */
+    PCL_ERR_UNSUPPORTED_SHAPE = 2, /* shape outside what the kernels cover            */
+    PCL_ERR_MISALIGNED = 3,        /* a pointer is not 16-byte aligned                */
+    PCL_ERR_WORKSPACE = 4,         /* workspace smaller than pcl_*_workspace_bytes()  */
+    PCL_ERR_CUDA = 5,              /* a CUDA runtime/driver call failed               */
+    PCL_ERR_DEVICE_TIMEOUT = 6     /* a bounded device-side wait ran out              */
+};
+
+enum { PCL_PASS_FWD = 0, PCL_PASS_BWD_DATA = 1, PCL_PASS_BWD_WEIGHTS = 2 };
+
+/* Which kernel family the conv / fc calls use.  PCL_PATH_AUTO picks the tensor
+ * core (tcgen05 TF32) kernels whenever the shape is eligible and the generic
+ * CUDA-core kernels otherwise; the other two values force one family (a forced
+ * tensor-core path returns PCL_ERR_UNSUPPORTED_SHAPE on ineligible shapes).
+ * Process-wide setting, intended for tests. */
+enum { PCL_PATH_AUTO = 0, PCL_PATH_TENSOR = 1, PCL_PATH_GENERIC = 2 };
+int pcl_set_path(int path);
+
+/* Output spatial size of a convolution.  Returns PCL_ERR_BAD_ARG if the
+ * kernel does not fit in the padded input. */
+int pcl_conv_out_dims(const pcl_conv_desc* d, int* P, int* Q);
+
+/* Bytes of workspace the given pass needs (0 is possible).  The workspace
+ * pointer handed to the pass must be 256-byte aligned. */
+size_t pcl_conv_workspace_bytes(const pcl_conv_desc* d, int pass);
+size_t pcl_fc_workspace_bytes(int N, int C, int K, int pass);
+
+/* Forward propagation (Algorithm 1):
+ *   y[n,p,q,k] = act(bias[k] + sum_{c,r,s} x[n, p*stride_h + r - pad_h,
+ *                                            q*stride_w + s - pad_w, c] * w[k,r,s,c])
+ * with zero contribution outside the image (cross-correlation, no kernel
+ * flip).  x: NHWC in, w: KRSC in, bias: [K] in or NULL, y: NPQK out.
+ * act: PCL_ACT_NONE or PCL_ACT_RELU (fused into the epilogue). */
+int pcl_conv_fwd(const pcl_conv_desc* d, const float* x, const float* w, const float* bias,
+                 float* y, int act, void* ws, size_t ws_bytes, void* cuda_stream);
+
+/* Backpropagation (the "Backpropagation" update rule of Sec. 2.1, gather form):
+ *   dx[n,h,w,c] = sum over (k,r,s) such that p = (h + pad_h - r)/stride_h and
+ *                 q = (w + pad_w - s)/stride_w are integers inside the output
+ *                 of dy[n,p,q,k] * w[k,r,s,c]
+ * dy: NPQK in, w: KRSC in, dx: NHWC out (every element written; positions no
+ * tap reaches get 0).  relu_mask_src: NULL, or an NHWC tensor of dx's shape
+ * (the layer's input, i.e. a ReLU output): dx is zeroed where it is <= 0. */
+int pcl_conv_bwd_data(const pcl_conv_desc* d, const float* dy, const float* w,
+                      const float* relu_mask_src, float* dx,
+                      void* ws, size_t ws_bytes, void* cuda_stream);
+
+/* Weight-gradient update (Sec. 2.1):
+ *   dw[k,r,s,c] = sum_{n,p,q} dy[n,p,q,k] * x[n, p*stride_h + r - pad_h, q*stride_w + s - pad_w, c]
+ *   dbias[k]    = sum_{n,p,q} dy[n,p,q,k]                  (if dbias != NULL)
+ * x: NHWC in, dy: NPQK in, dw: KRSC out, dbias: [K] out or NULL.
+ * The minibatch/pixel reduction is split across thread blocks ("privatise and
+ * reduce", Sec. 2.5).  deterministic != 0: partial sums go to the workspace and
+ * a second pass adds them in a fixed order (bitwise reproducible);
+ * deterministic == 0: partial sums are added with fp32 atomics (order varies). */
+int pcl_conv_bwd_weights(const pcl_conv_desc* d, const float* x, const float* dy,
+                         float* dw, float* dbias, int deterministic,
+                         void* ws, size_t ws_bytes, void* cuda_stream);
+
+/* Fully-connected forward: the k_h = k_w = out_h = out_w = 1 case of Algorithm 1
+ * (Sec. 2.1):  y[n,k] = act(bias[k] + sum_c x[n,c] * w[k,c]).
+ * x: [N][C], w: [K][C], bias: [K] or NULL, y: [N][K].
+ * act: NONE, RELU or SIGMOID. */
+int pcl_fc_fwd(int N, int C, int K, const float* x, const float* w, const float* bias,
+               float* y, int act, void* ws, size_t ws_bytes, void* cuda_stream);
+
+/* Fully-connected backward (same special case of the two update rules):
+ *   dz = dy * act'(y)   (ReLU: [y > 0]; sigmoid: y(1-y); written back into dy)
+ *   dx[n,c] = sum_k dz[n,k] * w[k,c]      (skipped if dx == NULL: first layer)
+ *   dw[k,c] = sum_n dz[n,k] * x[n,c]
+ *   dbias[k] = sum_n dz[n,k]              (skipped if dbias == NULL)
+ * y is only read when act != NONE (may be NULL otherwise).  Workspace size:
+ * pcl_fc_workspace_bytes(N, C, K, PCL_PASS_BWD_DATA). */
+int pcl_fc_bwd(int N, int C, int K, const float* x, const float* w, const float* y, int act,
+               float* dy, float* dx, float* dw, float* dbias,
+               void* ws, size_t ws_bytes, void* cuda_stream);
+
+/* Vanilla SGD (Sec. 1: algorithm and hyper-parameters untouched):
+ *   w[i] <- w[i] - lr * dw[i],  i < n.   w, dw only need 4-byte alignment. */
+int pcl_sgd_update(float* w, const float* dw, size_t n, float lr, void* cuda_stream);
+
+/* Glue the VGG-A / DNN topologies of Sec. 5 need between the passes above. */
+/* 2x2 window, stride 2, no padding; H and W even.  x: NHWC, y: N,H/2,W/2,C. */
+int pcl_maxpool2x2_fwd(int N, int H, int W, int C, const float* x, float* y, void* cuda_stream);
+/* dx gets dy at the first maximum of each window (row-major window order) and 0
+ * elsewhere; then, if relu_mask_src != NULL (NHWC, x's shape), dx is zeroed
+ * where relu_mask_src <= 0. */
+int pcl_maxpool2x2_bwd(int N, int H, int W, int C, const float* x, const float* dy,
+                       const float* relu_mask_src, float* dx, void* cuda_stream);
+/* loss = -(1/N) sum_n log softmax(logits[n,:])[labels[n]]  (device scalar, overwritten)
+ * dlogits = (softmax(logits) - onehot(labels)) / N.  labels: device int32 [N]. */
+int pcl_softmax_xent(int N, int K, const float* logits, const int* labels,
+                     float* loss, float* dlogits, void* cuda_stream);
+
+/* Synchronises the stream, then reads and clears the device status word of the
+ * current device.  PCL_OK, PCL_ERR_DEVICE_TIMEOUT or PCL_ERR_CUDA. */
+int pcl_last_device_status(void* cuda_stream);
+
+/* Number of kernels this library has launched since it was loaded. */
+unsigned long long pcl_launch_count(void);
+
+const char* pcl_status_string(int status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* PCL_DNN_H */

@@ -1,0 +1,186 @@
+"""ctypes binding of libpcl_dnn.so: same names as the C ABI, argument
+marshalling only.  Tensors are torch CUDA tensors (device memory and streams
+are all torch is used for); every step of the path runs in the library's
+kernels.  There is no CPU or library fallback: if the shared library is missing
+or a call fails, an exception is raised.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libpcl_dnn.so")
+
+ACT_NONE, ACT_RELU, ACT_SIGMOID = 0, 1, 2
+PASS_FWD, PASS_BWD_DATA, PASS_BWD_WEIGHTS = 0, 1, 2
+PATH_AUTO, PATH_TENSOR, PATH_GENERIC = 0, 1, 2
+OK = 0
+ERR_BAD_ARG, ERR_UNSUPPORTED_SHAPE, ERR_MISALIGNED, ERR_WORKSPACE, ERR_CUDA, ERR_DEVICE_TIMEOUT = 1, 2, 3, 4, 5, 6
+
+EXPORTS = [
+    "pcl_set_path", "pcl_conv_out_dims", "pcl_conv_workspace_bytes", "pcl_fc_workspace_bytes",
+    "pcl_conv_fwd", "pcl_conv_bwd_data", "pcl_conv_bwd_weights", "pcl_fc_fwd", "pcl_fc_bwd",
+    "pcl_sgd_update", "pcl_maxpool2x2_fwd", "pcl_maxpool2x2_bwd", "pcl_softmax_xent",
+    "pcl_last_device_status", "pcl_launch_count", "pcl_status_string",
+]
+
+
+class PclError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        self.code = code
+        super().__init__(f"{where}: {status_string(code)} (status {code})")
+
+
+class ConvDesc(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_int) for n in
+                ("N", "C", "K", "H", "W", "R", "S", "stride_h", "stride_w", "pad_h", "pad_w")]
+
+
+_lib = None
+
+
+def lib() -> ctypes.CDLL:
+    """Loads the CUDA library; fails loudly if it has not been built."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError(f"{LIB_PATH} is missing: run `python -m paper_1602_06709_b200.build` "
+                               "(there is no fallback path)")
+        L = ctypes.CDLL(LIB_PATH)
+        vp, sz, ci, cf = ctypes.c_void_p, ctypes.c_size_t, ctypes.c_int, ctypes.c_float
+        dp = ctypes.POINTER(ConvDesc)
+        L.pcl_set_path.argtypes = [ci]
+        L.pcl_conv_out_dims.argtypes = [dp, ctypes.POINTER(ci), ctypes.POINTER(ci)]
+        L.pcl_conv_workspace_bytes.argtypes = [dp, ci]
+        L.pcl_conv_workspace_bytes.restype = sz
+        L.pcl_fc_workspace_bytes.argtypes = [ci, ci, ci, ci]
+        L.pcl_fc_workspace_bytes.restype = sz
+        L.pcl_conv_fwd.argtypes = [dp, vp, vp, vp, vp, ci, vp, sz, vp]
+        L.pcl_conv_bwd_data.argtypes = [dp, vp, vp, vp, vp, vp, sz, vp]
+        L.pcl_conv_bwd_weights.argtypes = [dp, vp, vp, vp, vp, ci, vp, sz, vp]
+        L.pcl_fc_fwd.argtypes = [ci, ci, ci, vp, vp, vp, vp, ci, vp, sz, vp]
+        L.pcl_fc_bwd.argtypes = [ci, ci, ci, vp, vp, vp, ci, vp, vp, vp, vp, vp, sz, vp]
+        L.pcl_sgd_update.argtypes = [vp, vp, sz, cf, vp]
+        L.pcl_maxpool2x2_fwd.argtypes = [ci, ci, ci, ci, vp, vp, vp]
+        L.pcl_maxpool2x2_bwd.argtypes = [ci, ci, ci, ci, vp, vp, vp, vp, vp]
+        L.pcl_softmax_xent.argtypes = [ci, ci, vp, vp, vp, vp, vp]
+        L.pcl_last_device_status.argtypes = [vp]
+        L.pcl_launch_count.restype = ctypes.c_ulonglong
+        L.pcl_status_string.argtypes = [ci]
+        L.pcl_status_string.restype = ctypes.c_char_p
+        _lib = L
+    return _lib
+
+
+def status_string(code: int) -> str:
+    return lib().pcl_status_string(code).decode()
+
+
+def _check(code: int, where: str):
+    if code != OK:
+        raise PclError(code, where)
+
+
+def _ptr(t):
+    if t is None:
+        return None
+    assert t.is_cuda and t.is_contiguous(), "tensors must be contiguous CUDA tensors"
+    return ctypes.c_void_p(t.data_ptr())
+
+
+def _stream(stream=None):
+    s = stream if stream is not None else torch.cuda.current_stream()
+    return ctypes.c_void_p(s.cuda_stream)
+
+
+def conv_desc(N, C, K, H, W, R, S, stride=1, pad=0, stride_w=None, pad_w=None) -> ConvDesc:
+    return ConvDesc(N, C, K, H, W, R, S, stride, stride if stride_w is None else stride_w,
+                    pad, pad if pad_w is None else pad_w)
+
+
+def set_path(path: int):
+    _check(lib().pcl_set_path(path), "pcl_set_path")
+
+
+def conv_out_dims(d: ConvDesc):
+    P, Q = ctypes.c_int(), ctypes.c_int()
+    _check(lib().pcl_conv_out_dims(ctypes.byref(d), ctypes.byref(P), ctypes.byref(Q)), "pcl_conv_out_dims")
+    return P.value, Q.value
+
+
+def conv_workspace_bytes(d: ConvDesc, which: int) -> int:
+    return int(lib().pcl_conv_workspace_bytes(ctypes.byref(d), which))
+
+
+def fc_workspace_bytes(N, C, K, which: int) -> int:
+    return int(lib().pcl_fc_workspace_bytes(N, C, K, which))
+
+
+def _ws(ws):
+    if ws is None:
+        return None, 0
+    return _ptr(ws), ws.numel() * ws.element_size()
+
+
+def conv_fwd(d, x, w, bias, y, act=ACT_NONE, ws=None, stream=None):
+    wp, wb = _ws(ws)
+    _check(lib().pcl_conv_fwd(ctypes.byref(d), _ptr(x), _ptr(w), _ptr(bias), _ptr(y), act, wp, wb, _stream(stream)),
+           "pcl_conv_fwd")
+
+
+def conv_bwd_data(d, dy, w, relu_mask_src, dx, ws=None, stream=None):
+    wp, wb = _ws(ws)
+    _check(lib().pcl_conv_bwd_data(ctypes.byref(d), _ptr(dy), _ptr(w), _ptr(relu_mask_src), _ptr(dx), wp, wb,
+                                   _stream(stream)), "pcl_conv_bwd_data")
+
+
+def conv_bwd_weights(d, x, dy, dw, dbias=None, deterministic=True, ws=None, stream=None):
+    wp, wb = _ws(ws)
+    _check(lib().pcl_conv_bwd_weights(ctypes.byref(d), _ptr(x), _ptr(dy), _ptr(dw), _ptr(dbias),
+                                      1 if deterministic else 0, wp, wb, _stream(stream)), "pcl_conv_bwd_weights")
+
+
+def fc_fwd(N, C, K, x, w, bias, y, act=ACT_NONE, ws=None, stream=None):
+    wp, wb = _ws(ws)
+    _check(lib().pcl_fc_fwd(N, C, K, _ptr(x), _ptr(w), _ptr(bias), _ptr(y), act, wp, wb, _stream(stream)),
+           "pcl_fc_fwd")
+
+
+def fc_bwd(N, C, K, x, w, y, act, dy, dx, dw, dbias, ws=None, stream=None):
+    wp, wb = _ws(ws)
+    _check(lib().pcl_fc_bwd(N, C, K, _ptr(x), _ptr(w), _ptr(y), act, _ptr(dy), _ptr(dx), _ptr(dw), _ptr(dbias),
+                            wp, wb, _stream(stream)), "pcl_fc_bwd")
+
+
+def sgd_update(w, dw, lr, stream=None):
+    _check(lib().pcl_sgd_update(_ptr(w), _ptr(dw), w.numel(), ctypes.c_float(lr), _stream(stream)), "pcl_sgd_update")
+
+
+def maxpool2x2_fwd(N, H, W, C, x, y, stream=None):
+    _check(lib().pcl_maxpool2x2_fwd(N, H, W, C, _ptr(x), _ptr(y), _stream(stream)), "pcl_maxpool2x2_fwd")
+
+
+def maxpool2x2_bwd(N, H, W, C, x, dy, relu_mask_src, dx, stream=None):
+    _check(lib().pcl_maxpool2x2_bwd(N, H, W, C, _ptr(x), _ptr(dy), _ptr(relu_mask_src), _ptr(dx), _stream(stream)),
+           "pcl_maxpool2x2_bwd")
+
+
+def softmax_xent(N, K, logits, labels, loss, dlogits, stream=None):
+    assert labels.dtype == torch.int32
+    _check(lib().pcl_softmax_xent(N, K, _ptr(logits), _ptr(labels), _ptr(loss), _ptr(dlogits), _stream(stream)),
+           "pcl_softmax_xent")
+
+
+def last_device_status(stream=None) -> int:
+    return int(lib().pcl_last_device_status(_stream(stream)))
+
+
+def check_device_status(stream=None):
+    _check(last_device_status(stream), "device status")
+
+
+def launch_count() -> int:
+    return int(lib().pcl_launch_count())

@@ -1,0 +1,318 @@
+// HBM-bound kernels: SGD update, split reduction, weight transpose, activation
+// gradient, column sums, 2x2 max-pool, softmax cross-entropy.  All are plain
+// coalesced, vectorised (float4 where alignment allows) grid-stride kernels;
+// their roofline is memory bandwidth.
+#include <math.h>
+
+#include "pcl_internal.h"
+
+namespace pcl {
+
+namespace {
+
+int grid_for(size_t work_items, int block, int per_sm = 8) {
+    size_t blocks = (work_items + block - 1) / block;
+    const size_t cap = size_t(148) * per_sm;
+    if (blocks > cap) blocks = cap;
+    if (blocks < 1) blocks = 1;
+    return int(blocks);
+}
+
+// w <- w - lr * dw.  12 bytes of traffic per parameter.
+__global__ void __launch_bounds__(256) sgd_kernel(float* __restrict__ w, const float* __restrict__ dw, size_t n,
+                                                  float lr, int vec) {
+    const size_t tid = size_t(blockIdx.x) * blockDim.x + threadIdx.x;
+    const size_t stride = size_t(gridDim.x) * blockDim.x;
+    if (vec) {
+        const size_t n4 = n >> 2;
+        float4* w4 = reinterpret_cast<float4*>(w);
+        const float4* d4 = reinterpret_cast<const float4*>(dw);
+        for (size_t i = tid; i < n4; i += stride) {
+            float4 a = w4[i];
+            const float4 g = __ldcs(d4 + i);
+            a.x = fmaf(-lr, g.x, a.x); a.y = fmaf(-lr, g.y, a.y);
+            a.z = fmaf(-lr, g.z, a.z); a.w = fmaf(-lr, g.w, a.w);
+            w4[i] = a;
+        }
+        for (size_t i = (n4 << 2) + tid; i < n; i += stride) w[i] = fmaf(-lr, dw[i], w[i]);
+    } else {
+        for (size_t i = tid; i < n; i += stride) w[i] = fmaf(-lr, dw[i], w[i]);
+    }
+}
+
+__global__ void __launch_bounds__(256) zero_kernel(float* __restrict__ p, size_t n) {
+    const size_t stride = size_t(gridDim.x) * blockDim.x;
+    for (size_t i = size_t(blockIdx.x) * blockDim.x + threadIdx.x; i < n; i += stride) p[i] = 0.f;
+}
+
+// out[i] = partial[0][i] + partial[1][i] + ... in that order (fixed => reproducible)
+__global__ void __launch_bounds__(256) reduce_splits_kernel(const float* __restrict__ partial, float* __restrict__ out,
+                                                            size_t n, int splits) {
+    const size_t stride = size_t(gridDim.x) * blockDim.x;
+    for (size_t i = size_t(blockIdx.x) * blockDim.x + threadIdx.x; i < n; i += stride) {
+        float acc = partial[i];
+        for (int s = 1; s < splits; ++s) acc += partial[size_t(s) * n + i];
+        out[i] = acc;
+    }
+}
+
+// wt_t[c][R-1-r][S-1-s][k] = w[k][r][s][c]: the "transpose-weights" copy the
+// backward-data pass contracts against (Sec. 2.3 keeps such a copy too).
+__global__ void __launch_bounds__(256) transpose_flip_kernel(const float* __restrict__ w, float* __restrict__ out,
+                                                             int K, int RS, int C) {
+    __shared__ float tile[32][33];
+    const int tap = blockIdx.z;
+    const int k0 = blockIdx.y * 32, c0 = blockIdx.x * 32;
+    const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;   // 32 x 8
+    for (int j = ty; j < 32; j += 8) {
+        const int k = k0 + j, c = c0 + tx;
+        tile[j][tx] = (k < K && c < C) ? w[(size_t(k) * RS + tap) * C + c] : 0.f;
+    }
+    __syncthreads();
+    const int tap_f = RS - 1 - tap;   // flipping r and s together reverses the flat tap index
+    for (int j = ty; j < 32; j += 8) {
+        const int c = c0 + j, k = k0 + tx;
+        if (k < K && c < C) out[(size_t(c) * RS + tap_f) * K + k] = tile[tx][j];
+    }
+}
+
+__global__ void __launch_bounds__(256) act_grad_kernel(float* __restrict__ dy, const float* __restrict__ y, size_t n,
+                                                       int act) {
+    const size_t stride = size_t(gridDim.x) * blockDim.x;
+    for (size_t i = size_t(blockIdx.x) * blockDim.x + threadIdx.x; i < n; i += stride) {
+        const float yv = y[i];
+        const float g = dy[i];
+        dy[i] = act == PCL_ACT_RELU ? (yv > 0.f ? g : 0.f) : g * yv * (1.f - yv);
+    }
+}
+
+// partial[split][k] = sum over the split's rows of m[row][k]
+constexpr int kColsumRows = 4096;
+__global__ void __launch_bounds__(256) colsum_kernel(const float* __restrict__ m, size_t rows, int K,
+                                                     float* __restrict__ partial) {
+    const int k = blockIdx.x * 32 + (threadIdx.x & 31);
+    const int ty = threadIdx.x >> 5;
+    const size_t r0 = size_t(blockIdx.y) * kColsumRows;
+    size_t r1 = r0 + kColsumRows;
+    if (r1 > rows) r1 = rows;
+    float acc = 0.f;
+    if (k < K)
+        for (size_t r = r0 + ty; r < r1; r += 8) acc += m[r * K + k];
+    __shared__ float red[8][32];
+    red[ty][threadIdx.x & 31] = acc;
+    __syncthreads();
+    if (ty == 0 && k < K) {
+        float s = 0.f;
+        for (int j = 0; j < 8; ++j) s += red[j][threadIdx.x];
+        partial[size_t(blockIdx.y) * K + k] = s;
+    }
+}
+
+// 2x2 / stride-2 max pooling, NHWC, one thread per (output pixel, 4 channels)
+template <int VEC>
+__global__ void __launch_bounds__(256) maxpool_fwd_kernel(const float* __restrict__ x, float* __restrict__ y, int N,
+                                                          int H, int W, int C) {
+    const int Po = H / 2, Qo = W / 2, Cv = C / VEC;
+    const size_t total = size_t(N) * Po * Qo * Cv;
+    const size_t stride = size_t(gridDim.x) * blockDim.x;
+    for (size_t i = size_t(blockIdx.x) * blockDim.x + threadIdx.x; i < total; i += stride) {
+        const int cv = int(i % Cv); size_t t = i / Cv;
+        const int q = int(t % Qo); t /= Qo;
+        const int p = int(t % Po); const size_t n = t / Po;
+        const float* src = x + ((n * H + 2 * p) * W + 2 * q) * C + cv * VEC;
+        float* dst = y + ((n * Po + p) * Qo + q) * C + cv * VEC;
+        if (VEC == 4) {
+            const float4 a = *reinterpret_cast<const float4*>(src);
+            const float4 b = *reinterpret_cast<const float4*>(src + C);
+            const float4 c = *reinterpret_cast<const float4*>(src + size_t(W) * C);
+            const float4 d = *reinterpret_cast<const float4*>(src + size_t(W) * C + C);
+            float4 o;
+            o.x = fmaxf(fmaxf(a.x, b.x), fmaxf(c.x, d.x)); o.y = fmaxf(fmaxf(a.y, b.y), fmaxf(c.y, d.y));
+            o.z = fmaxf(fmaxf(a.z, b.z), fmaxf(c.z, d.z)); o.w = fmaxf(fmaxf(a.w, b.w), fmaxf(c.w, d.w));
+            *reinterpret_cast<float4*>(dst) = o;
+        } else {
+            dst[0] = fmaxf(fmaxf(src[0], src[C]), fmaxf(src[size_t(W) * C], src[size_t(W) * C + C]));
+        }
+    }
+}
+
+__device__ __forceinline__ void pool_route(float a, float b, float c, float d, float g, float& oa, float& ob,
+                                           float& oc, float& od) {
+    // first maximum in row-major window order
+    int arg = 0; float best = a;
+    if (b > best) { best = b; arg = 1; }
+    if (c > best) { best = c; arg = 2; }
+    if (d > best) { best = d; arg = 3; }
+    oa = arg == 0 ? g : 0.f; ob = arg == 1 ? g : 0.f; oc = arg == 2 ? g : 0.f; od = arg == 3 ? g : 0.f;
+}
+
+template <int VEC>
+__global__ void __launch_bounds__(256) maxpool_bwd_kernel(const float* __restrict__ x, const float* __restrict__ dy,
+                                                          const float* __restrict__ mask, float* __restrict__ dx,
+                                                          int N, int H, int W, int C) {
+    const int Po = H / 2, Qo = W / 2, Cv = C / VEC;
+    const size_t total = size_t(N) * Po * Qo * Cv;
+    const size_t stride = size_t(gridDim.x) * blockDim.x;
+    const size_t rowp = size_t(W) * C;
+    for (size_t i = size_t(blockIdx.x) * blockDim.x + threadIdx.x; i < total; i += stride) {
+        const int cv = int(i % Cv); size_t t = i / Cv;
+        const int q = int(t % Qo); t /= Qo;
+        const int p = int(t % Po); const size_t n = t / Po;
+        const size_t off = ((n * H + 2 * p) * W + 2 * q) * C + cv * VEC;
+        const float* g = dy + ((n * Po + p) * Qo + q) * C + cv * VEC;
+        float xa[VEC], xb[VEC], xc[VEC], xd[VEC], oa[VEC], ob[VEC], oc[VEC], od[VEC], gv[VEC];
+#pragma unroll
+        for (int j = 0; j < VEC; ++j) {
+            xa[j] = x[off + j]; xb[j] = x[off + C + j]; xc[j] = x[off + rowp + j]; xd[j] = x[off + rowp + C + j];
+            gv[j] = g[j];
+        }
+#pragma unroll
+        for (int j = 0; j < VEC; ++j) pool_route(xa[j], xb[j], xc[j], xd[j], gv[j], oa[j], ob[j], oc[j], od[j]);
+        if (mask) {
+#pragma unroll
+            for (int j = 0; j < VEC; ++j) {
+                if (!(mask[off + j] > 0.f)) oa[j] = 0.f;
+                if (!(mask[off + C + j] > 0.f)) ob[j] = 0.f;
+                if (!(mask[off + rowp + j] > 0.f)) oc[j] = 0.f;
+                if (!(mask[off + rowp + C + j] > 0.f)) od[j] = 0.f;
+            }
+        }
+#pragma unroll
+        for (int j = 0; j < VEC; ++j) {
+            dx[off + j] = oa[j]; dx[off + C + j] = ob[j]; dx[off + rowp + j] = oc[j]; dx[off + rowp + C + j] = od[j];
+        }
+    }
+}
+
+// One CTA per row: max, sum of exponentials, loss term, gradient.
+__global__ void __launch_bounds__(256) softmax_xent_kernel(const float* __restrict__ logits,
+                                                           const int* __restrict__ labels, float* __restrict__ loss,
+                                                           float* __restrict__ dlogits, int N, int K) {
+    __shared__ float red[32];
+    __shared__ float bcast;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    for (int n = blockIdx.x; n < N; n += gridDim.x) {
+        const float* z = logits + size_t(n) * K;
+        float mx = -INFINITY;
+        for (int k = threadIdx.x; k < K; k += blockDim.x) mx = fmaxf(mx, z[k]);
+        for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+        if (lane == 0) red[warp] = mx;
+        __syncthreads();
+        if (warp == 0) {
+            float v = lane < (blockDim.x >> 5) ? red[lane] : -INFINITY;
+            for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+            if (lane == 0) bcast = v;
+        }
+        __syncthreads();
+        mx = bcast;
+        float sum = 0.f;
+        for (int k = threadIdx.x; k < K; k += blockDim.x) sum += expf(z[k] - mx);
+        for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
+        __syncthreads();
+        if (lane == 0) red[warp] = sum;
+        __syncthreads();
+        if (warp == 0) {
+            float v = lane < (blockDim.x >> 5) ? red[lane] : 0.f;
+            for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+            if (lane == 0) bcast = v;
+        }
+        __syncthreads();
+        sum = bcast;
+        const int lab = labels[n];
+        const float inv_n = 1.f / float(N);
+        const float inv_sum = 1.f / sum;
+        for (int k = threadIdx.x; k < K; k += blockDim.x) {
+            const float pk = expf(z[k] - mx) * inv_sum;
+            dlogits[size_t(n) * K + k] = (pk - (k == lab ? 1.f : 0.f)) * inv_n;
+        }
+        if (threadIdx.x == 0) atomicAdd(loss, -(z[lab] - mx - logf(sum)) * inv_n);
+        __syncthreads();
+    }
+}
+
+#define PCL_CHECK_LAUNCH() (cudaGetLastError() == cudaSuccess ? PCL_OK : PCL_ERR_CUDA)
+
+}  // namespace
+
+int launch_sgd(float* w, const float* dw, size_t n, float lr, cudaStream_t st) {
+    if (n == 0) return PCL_OK;
+    const int vec = ((reinterpret_cast<uintptr_t>(w) | reinterpret_cast<uintptr_t>(dw)) & 15) == 0;
+    sgd_kernel<<<grid_for(vec ? (n + 3) / 4 : n, 256), 256, 0, st>>>(w, dw, n, lr, vec);
+    count_launch();
+    return PCL_CHECK_LAUNCH();
+}
+
+int launch_zero(float* p, size_t n, cudaStream_t st) {
+    if (n == 0) return PCL_OK;
+    zero_kernel<<<grid_for(n, 256), 256, 0, st>>>(p, n);
+    count_launch();
+    return PCL_CHECK_LAUNCH();
+}
+
+int launch_reduce_splits(const float* partial, float* out, size_t n, int splits, cudaStream_t st) {
+    if (n == 0) return PCL_OK;
+    reduce_splits_kernel<<<grid_for(n, 256), 256, 0, st>>>(partial, out, n, splits);
+    count_launch();
+    return PCL_CHECK_LAUNCH();
+}
+
+int launch_transpose_flip(const float* w, float* wt_t, int K, int R, int S, int C, cudaStream_t st) {
+    if (R * S > 65535) return PCL_ERR_UNSUPPORTED_SHAPE;
+    dim3 grid((C + 31) / 32, (K + 31) / 32, R * S);
+    if (grid.y > 65535) return PCL_ERR_UNSUPPORTED_SHAPE;
+    transpose_flip_kernel<<<grid, 256, 0, st>>>(w, wt_t, K, R * S, C);
+    count_launch();
+    return PCL_CHECK_LAUNCH();
+}
+
+int launch_act_grad(float* dy, const float* y, size_t n, int act, cudaStream_t st) {
+    if (n == 0 || act == PCL_ACT_NONE) return PCL_OK;
+    act_grad_kernel<<<grid_for(n, 256), 256, 0, st>>>(dy, y, n, act);
+    count_launch();
+    return PCL_CHECK_LAUNCH();
+}
+
+int colsum_splits(size_t rows) { return int((rows + kColsumRows - 1) / kColsumRows); }
+
+int launch_colsum(const float* m, size_t rows, int K, float* partial, float* out, cudaStream_t st) {
+    const int splits = colsum_splits(rows);
+    if (splits > 65535) return PCL_ERR_UNSUPPORTED_SHAPE;
+    dim3 grid((K + 31) / 32, splits);
+    colsum_kernel<<<grid, 256, 0, st>>>(m, rows, K, splits == 1 ? out : partial);
+    count_launch();
+    if (cudaGetLastError() != cudaSuccess) return PCL_ERR_CUDA;
+    if (splits > 1) return launch_reduce_splits(partial, out, size_t(K), splits, st);
+    return PCL_OK;
+}
+
+int launch_maxpool_fwd(int N, int H, int W, int C, const float* x, float* y, cudaStream_t st) {
+    const size_t outs = size_t(N) * (H / 2) * (W / 2);
+    if (C % 4 == 0)
+        maxpool_fwd_kernel<4><<<grid_for(outs * (C / 4), 256), 256, 0, st>>>(x, y, N, H, W, C);
+    else
+        maxpool_fwd_kernel<1><<<grid_for(outs * C, 256), 256, 0, st>>>(x, y, N, H, W, C);
+    count_launch();
+    return PCL_CHECK_LAUNCH();
+}
+
+int launch_maxpool_bwd(int N, int H, int W, int C, const float* x, const float* dy, const float* mask, float* dx,
+                       cudaStream_t st) {
+    const size_t outs = size_t(N) * (H / 2) * (W / 2);
+    if (C % 4 == 0)
+        maxpool_bwd_kernel<4><<<grid_for(outs * (C / 4), 256), 256, 0, st>>>(x, dy, mask, dx, N, H, W, C);
+    else
+        maxpool_bwd_kernel<1><<<grid_for(outs * C, 256), 256, 0, st>>>(x, dy, mask, dx, N, H, W, C);
+    count_launch();
+    return PCL_CHECK_LAUNCH();
+}
+
+int launch_softmax_xent(int N, int K, const float* logits, const int* labels, float* loss, float* dlogits,
+                        cudaStream_t st) {
+    int rc = launch_zero(loss, 1, st);
+    if (rc != PCL_OK) return rc;
+    softmax_xent_kernel<<<N < 1184 ? N : 1184, 256, 0, st>>>(logits, labels, loss, dlogits, N, K);
+    count_launch();
+    return PCL_CHECK_LAUNCH();
+}
+
+}  // namespace pcl

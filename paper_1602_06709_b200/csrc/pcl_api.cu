@@ -1,0 +1,321 @@
+// C ABI of the library: argument checks, kernel-family selection, workspace
+// carving, tensor-map construction.  Every entry point only enqueues kernels on
+// the caller's stream.
+#include <atomic>
+#include <mutex>
+
+#include "pcl_internal.h"
+#include "pcl_ptx.cuh"
+
+namespace pcl {
+
+__device__ unsigned int g_device_status = 0;
+
+unsigned int* device_status_ptr() {
+    // one copy of the symbol per device: look the address up per device, once
+    static unsigned int* cache[64] = {};
+    static std::mutex mu;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+    std::lock_guard<std::mutex> lock(mu);
+    if (!cache[dev]) {
+        void* p = nullptr;
+        if (cudaGetSymbolAddress(&p, g_device_status) != cudaSuccess) return nullptr;
+        cache[dev] = static_cast<unsigned int*>(p);
+    }
+    return cache[dev];
+}
+
+static std::atomic<unsigned long long> g_launches{0};
+void count_launch(unsigned n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
+
+static std::atomic<int> g_path{PCL_PATH_AUTO};
+
+encode_tiled_fn get_encode_tiled() {
+    static encode_tiled_fn fn = nullptr;
+    static std::once_flag once;
+    std::call_once(once, [] {
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<encode_tiled_fn>(p);
+    });
+    return fn;
+}
+
+int make_tmap(CUtensorMap* out, const void* base, int rank, const uint64_t* dims, const uint64_t* strides_bytes,
+              const uint32_t* box) {
+    encode_tiled_fn enc = get_encode_tiled();
+    if (!enc) return PCL_ERR_CUDA;
+    cuuint64_t gdim[5];
+    cuuint64_t gstr[4];
+    cuuint32_t gbox[5], estr[5];
+    for (int i = 0; i < rank; ++i) {
+        gdim[i] = dims[i];
+        gbox[i] = box[i];
+        estr[i] = 1;
+        if (box[i] == 0 || box[i] > 256) return PCL_ERR_UNSUPPORTED_SHAPE;
+    }
+    for (int i = 0; i + 1 < rank; ++i) {
+        gstr[i] = strides_bytes[i];
+        if (strides_bytes[i] % 16 != 0 || strides_bytes[i] >= (1ull << 40)) return PCL_ERR_UNSUPPORTED_SHAPE;
+    }
+    if (reinterpret_cast<uintptr_t>(base) & 15) return PCL_ERR_MISALIGNED;
+    const CUresult r = enc(out, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, cuuint32_t(rank), const_cast<void*>(base), gdim, gstr,
+                           gbox, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                           CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS ? PCL_OK : PCL_ERR_CUDA;
+}
+
+namespace {
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
+
+int check_desc(const pcl_conv_desc* d, int* P, int* Q) {
+    if (!d) return PCL_ERR_BAD_ARG;
+    if (d->N <= 0 || d->C <= 0 || d->K <= 0 || d->H <= 0 || d->W <= 0 || d->R <= 0 || d->S <= 0 || d->stride_h <= 0 ||
+        d->stride_w <= 0 || d->pad_h < 0 || d->pad_w < 0)
+        return PCL_ERR_BAD_ARG;
+    const long sh = long(d->H) + 2L * d->pad_h - d->R, sw = long(d->W) + 2L * d->pad_w - d->S;
+    if (sh < 0 || sw < 0) return PCL_ERR_BAD_ARG;
+    *P = int(sh / d->stride_h) + 1;
+    *Q = int(sw / d->stride_w) + 1;
+    // element counts must stay addressable with 63-bit offsets and per-dimension 31-bit indices
+    const double big = 9e18;
+    if (double(d->N) * d->H * d->W * d->C > big || double(d->N) * (*P) * (*Q) * d->K > big) return PCL_ERR_UNSUPPORTED_SHAPE;
+    return PCL_OK;
+}
+
+bool unit_stride(const pcl_conv_desc& d) { return d.stride_h == 1 && d.stride_w == 1; }
+
+// Which family a pass would use for this descriptor (pointer alignment is
+// checked separately; all pointers are required to be 16-byte aligned anyway).
+bool tensor_path_for(const pcl_conv_desc& d, int pass) {
+    if (g_path.load() == PCL_PATH_GENERIC) return false;
+    if (!unit_stride(d)) return false;
+    switch (pass) {
+        case PCL_PASS_FWD: return d.C % 4 == 0;
+        case PCL_PASS_BWD_DATA: return d.K % 4 == 0 && d.pad_h <= d.R - 1 && d.pad_w <= d.S - 1;
+        case PCL_PASS_BWD_WEIGHTS: return d.C % 4 == 0 && d.K % 4 == 0;
+    }
+    return false;
+}
+
+size_t dw_bytes(const pcl_conv_desc& d) { return align_up(size_t(d.K) * d.R * d.S * d.C * 4, 256); }
+
+struct WgradPlan {
+    bool tensor;
+    int splits;          // pixel splits of the main kernel
+    size_t partial_bytes;
+    size_t colsum_bytes;
+};
+
+WgradPlan plan_wgrad(const pcl_conv_desc& d, int P, int Q) {
+    WgradPlan pl{};
+    pl.tensor = tensor_path_for(d, PCL_PASS_BWD_WEIGHTS);
+    pl.splits = pl.tensor ? tc_wgrad_splits(d.N, P, Q, d.C, d.K, d.R, d.S) : generic_wgrad_splits(d, P, Q);
+    pl.partial_bytes = pl.splits > 1 ? size_t(pl.splits) * dw_bytes(d) : 0;
+    const int cs = colsum_splits(size_t(d.N) * P * Q);
+    pl.colsum_bytes = cs > 1 ? align_up(size_t(cs) * d.K * 4, 256) : 0;
+    return pl;
+}
+
+}  // namespace
+}  // namespace pcl
+
+using namespace pcl;
+
+extern "C" {
+
+int pcl_set_path(int path) {
+    if (path != PCL_PATH_AUTO && path != PCL_PATH_TENSOR && path != PCL_PATH_GENERIC) return PCL_ERR_BAD_ARG;
+    g_path.store(path);
+    return PCL_OK;
+}
+
+int pcl_conv_out_dims(const pcl_conv_desc* d, int* P, int* Q) {
+    if (!P || !Q) return PCL_ERR_BAD_ARG;
+    return check_desc(d, P, Q);
+}
+
+size_t pcl_conv_workspace_bytes(const pcl_conv_desc* d, int pass) {
+    int P, Q;
+    if (check_desc(d, &P, &Q) != PCL_OK) return 0;
+    switch (pass) {
+        case PCL_PASS_FWD: return 0;
+        case PCL_PASS_BWD_DATA: return tensor_path_for(*d, pass) ? dw_bytes(*d) : 0;
+        case PCL_PASS_BWD_WEIGHTS: {
+            const WgradPlan pl = plan_wgrad(*d, P, Q);
+            return pl.partial_bytes + pl.colsum_bytes;
+        }
+    }
+    return 0;
+}
+
+size_t pcl_fc_workspace_bytes(int N, int C, int K, int pass) {
+    if (N <= 0 || C <= 0 || K <= 0) return 0;
+    const pcl_conv_desc d{N, C, K, 1, 1, 1, 1, 1, 1, 0, 0};
+    if (pass == PCL_PASS_FWD) return 0;
+    // fc_bwd runs both backward contractions; either pass value returns the total
+    return pcl_conv_workspace_bytes(&d, PCL_PASS_BWD_DATA) + pcl_conv_workspace_bytes(&d, PCL_PASS_BWD_WEIGHTS);
+}
+
+int pcl_conv_fwd(const pcl_conv_desc* d, const float* x, const float* w, const float* bias, float* y, int act,
+                 void* ws, size_t ws_bytes, void* cuda_stream) {
+    (void)ws; (void)ws_bytes;
+    int P, Q;
+    int rc = check_desc(d, &P, &Q);
+    if (rc != PCL_OK) return rc;
+    if (!x || !w || !y) return PCL_ERR_BAD_ARG;
+    if (act != PCL_ACT_NONE && act != PCL_ACT_RELU && act != PCL_ACT_SIGMOID) return PCL_ERR_BAD_ARG;
+    if (!aligned16(x) || !aligned16(w) || !aligned16(y) || !aligned16(bias)) return PCL_ERR_MISALIGNED;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    if (tensor_path_for(*d, PCL_PASS_FWD)) {
+        TcFpropArgs a{x, w, bias, nullptr, y, d->N, d->H, d->W, d->C, d->K, d->R, d->S, d->pad_h, d->pad_w, P, Q, act};
+        return launch_tc_fprop(a, st);
+    }
+    if (g_path.load() == PCL_PATH_TENSOR) return PCL_ERR_UNSUPPORTED_SHAPE;
+    return launch_generic_fwd(*d, P, Q, x, w, bias, y, act, st);
+}
+
+int pcl_conv_bwd_data(const pcl_conv_desc* d, const float* dy, const float* w, const float* relu_mask_src, float* dx,
+                      void* ws, size_t ws_bytes, void* cuda_stream) {
+    int P, Q;
+    int rc = check_desc(d, &P, &Q);
+    if (rc != PCL_OK) return rc;
+    if (!dy || !w || !dx) return PCL_ERR_BAD_ARG;
+    if (!aligned16(dy) || !aligned16(w) || !aligned16(dx) || !aligned16(relu_mask_src)) return PCL_ERR_MISALIGNED;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    if (tensor_path_for(*d, PCL_PASS_BWD_DATA)) {
+        const size_t need = dw_bytes(*d);
+        if (!ws || ws_bytes < need) return PCL_ERR_WORKSPACE;
+        if (reinterpret_cast<uintptr_t>(ws) & 255) return PCL_ERR_MISALIGNED;
+        float* wt_t = static_cast<float*>(ws);
+        rc = launch_transpose_flip(w, wt_t, d->K, d->R, d->S, d->C, st);
+        if (rc != PCL_OK) return rc;
+        // dx = "forward" convolution of dy with the flipped, transposed weights, pad' = R-1-pad
+        TcFpropArgs a{dy, wt_t, nullptr, relu_mask_src, dx, d->N, P, Q, d->K, d->C, d->R, d->S,
+                      d->R - 1 - d->pad_h, d->S - 1 - d->pad_w, d->H, d->W, PCL_ACT_NONE};
+        return launch_tc_fprop(a, st);
+    }
+    if (g_path.load() == PCL_PATH_TENSOR) return PCL_ERR_UNSUPPORTED_SHAPE;
+    return launch_generic_bwd_data(*d, P, Q, dy, w, relu_mask_src, dx, st);
+}
+
+int pcl_conv_bwd_weights(const pcl_conv_desc* d, const float* x, const float* dy, float* dw, float* dbias,
+                         int deterministic, void* ws, size_t ws_bytes, void* cuda_stream) {
+    int P, Q;
+    int rc = check_desc(d, &P, &Q);
+    if (rc != PCL_OK) return rc;
+    if (!x || !dy || !dw) return PCL_ERR_BAD_ARG;
+    if (!aligned16(x) || !aligned16(dy) || !aligned16(dw) || !aligned16(dbias)) return PCL_ERR_MISALIGNED;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    const WgradPlan pl = plan_wgrad(*d, P, Q);
+    if (!pl.tensor && g_path.load() == PCL_PATH_TENSOR) return PCL_ERR_UNSUPPORTED_SHAPE;
+    const bool need_partial = pl.splits > 1 && (deterministic || !pl.tensor);
+    size_t need = (need_partial ? pl.partial_bytes : 0) + (dbias ? pl.colsum_bytes : 0);
+    if (need > 0) {
+        if (!ws || ws_bytes < need) return PCL_ERR_WORKSPACE;
+        if (reinterpret_cast<uintptr_t>(ws) & 255) return PCL_ERR_MISALIGNED;
+    }
+    float* partial = need_partial ? static_cast<float*>(ws) : nullptr;
+    float* cs_partial = reinterpret_cast<float*>(static_cast<char*>(ws) + (need_partial ? pl.partial_bytes : 0));
+    if (pl.tensor) {
+        TcWgradArgs a{x, dy, dw, partial, d->N, d->H, d->W, d->C, d->K, d->R, d->S, d->pad_h, d->pad_w, P, Q, pl.splits};
+        rc = launch_tc_wgrad(a, st);
+    } else {
+        rc = launch_generic_bwd_weights(*d, P, Q, x, dy, dw, partial, pl.splits, st);
+    }
+    if (rc != PCL_OK) return rc;
+    if (dbias) rc = launch_colsum(dy, size_t(d->N) * P * Q, d->K, cs_partial, dbias, st);
+    return rc;
+}
+
+int pcl_fc_fwd(int N, int C, int K, const float* x, const float* w, const float* bias, float* y, int act, void* ws,
+               size_t ws_bytes, void* cuda_stream) {
+    const pcl_conv_desc d{N, C, K, 1, 1, 1, 1, 1, 1, 0, 0};
+    return pcl_conv_fwd(&d, x, w, bias, y, act, ws, ws_bytes, cuda_stream);
+}
+
+int pcl_fc_bwd(int N, int C, int K, const float* x, const float* w, const float* y, int act, float* dy, float* dx,
+               float* dw, float* dbias, void* ws, size_t ws_bytes, void* cuda_stream) {
+    if (N <= 0 || C <= 0 || K <= 0) return PCL_ERR_BAD_ARG;
+    if (!x || !w || !dy || !dw) return PCL_ERR_BAD_ARG;
+    if (act != PCL_ACT_NONE && act != PCL_ACT_RELU && act != PCL_ACT_SIGMOID) return PCL_ERR_BAD_ARG;
+    if (act != PCL_ACT_NONE && !y) return PCL_ERR_BAD_ARG;
+    if (!aligned16(x) || !aligned16(w) || !aligned16(y) || !aligned16(dy) || !aligned16(dx) || !aligned16(dw) ||
+        !aligned16(dbias))
+        return PCL_ERR_MISALIGNED;
+    const pcl_conv_desc d{N, C, K, 1, 1, 1, 1, 1, 1, 0, 0};
+    const size_t need_w = pcl_conv_workspace_bytes(&d, PCL_PASS_BWD_WEIGHTS);
+    const size_t need_d = dx ? pcl_conv_workspace_bytes(&d, PCL_PASS_BWD_DATA) : 0;
+    if (need_w + need_d > 0) {
+        if (!ws || ws_bytes < need_w + need_d) return PCL_ERR_WORKSPACE;
+        if (reinterpret_cast<uintptr_t>(ws) & 255) return PCL_ERR_MISALIGNED;
+    }
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    int rc = launch_act_grad(dy, y, size_t(N) * K, act, st);
+    if (rc != PCL_OK) return rc;
+    // weight gradient first, then backpropagation (the order Sec. 3.1 schedules them in)
+    rc = pcl_conv_bwd_weights(&d, x, dy, dw, dbias, 1, ws, need_w, cuda_stream);
+    if (rc != PCL_OK) return rc;
+    if (dx) rc = pcl_conv_bwd_data(&d, dy, w, nullptr, dx, static_cast<char*>(ws) + need_w, need_d, cuda_stream);
+    return rc;
+}
+
+int pcl_sgd_update(float* w, const float* dw, size_t n, float lr, void* cuda_stream) {
+    if (!w || !dw) return n == 0 ? PCL_OK : PCL_ERR_BAD_ARG;
+    if ((reinterpret_cast<uintptr_t>(w) | reinterpret_cast<uintptr_t>(dw)) & 3) return PCL_ERR_MISALIGNED;
+    return launch_sgd(w, dw, n, lr, static_cast<cudaStream_t>(cuda_stream));
+}
+
+int pcl_maxpool2x2_fwd(int N, int H, int W, int C, const float* x, float* y, void* cuda_stream) {
+    if (N <= 0 || H <= 0 || W <= 0 || C <= 0 || !x || !y) return PCL_ERR_BAD_ARG;
+    if ((H | W) & 1) return PCL_ERR_UNSUPPORTED_SHAPE;
+    if (!aligned16(x) || !aligned16(y)) return PCL_ERR_MISALIGNED;
+    return launch_maxpool_fwd(N, H, W, C, x, y, static_cast<cudaStream_t>(cuda_stream));
+}
+
+int pcl_maxpool2x2_bwd(int N, int H, int W, int C, const float* x, const float* dy, const float* relu_mask_src,
+                       float* dx, void* cuda_stream) {
+    if (N <= 0 || H <= 0 || W <= 0 || C <= 0 || !x || !dy || !dx) return PCL_ERR_BAD_ARG;
+    if ((H | W) & 1) return PCL_ERR_UNSUPPORTED_SHAPE;
+    if (!aligned16(x) || !aligned16(dy) || !aligned16(dx) || !aligned16(relu_mask_src)) return PCL_ERR_MISALIGNED;
+    return launch_maxpool_bwd(N, H, W, C, x, dy, relu_mask_src, dx, static_cast<cudaStream_t>(cuda_stream));
+}
+
+int pcl_softmax_xent(int N, int K, const float* logits, const int* labels, float* loss, float* dlogits,
+                     void* cuda_stream) {
+    if (N <= 0 || K <= 0 || !logits || !labels || !loss || !dlogits) return PCL_ERR_BAD_ARG;
+    return launch_softmax_xent(N, K, logits, labels, loss, dlogits, static_cast<cudaStream_t>(cuda_stream));
+}
+
+int pcl_last_device_status(void* cuda_stream) {
+    if (cudaStreamSynchronize(static_cast<cudaStream_t>(cuda_stream)) != cudaSuccess) return PCL_ERR_CUDA;
+    unsigned int v = 0;
+    if (cudaMemcpyFromSymbol(&v, g_device_status, sizeof(v)) != cudaSuccess) return PCL_ERR_CUDA;
+    if (v != 0) {
+        const unsigned int zero = 0;
+        if (cudaMemcpyToSymbol(g_device_status, &zero, sizeof(zero)) != cudaSuccess) return PCL_ERR_CUDA;
+        return PCL_ERR_DEVICE_TIMEOUT;
+    }
+    return PCL_OK;
+}
+
+unsigned long long pcl_launch_count(void) { return g_launches.load(); }
+
+const char* pcl_status_string(int status) {
+    switch (status) {
+        case PCL_OK: return "ok";
+        case PCL_ERR_BAD_ARG: return "bad argument";
+        case PCL_ERR_UNSUPPORTED_SHAPE: return "unsupported shape";
+        case PCL_ERR_MISALIGNED: return "misaligned pointer";
+        case PCL_ERR_WORKSPACE: return "workspace too small";
+        case PCL_ERR_CUDA: return "CUDA call failed";
+        case PCL_ERR_DEVICE_TIMEOUT: return "device-side wait timed out";
+    }
+    return "unknown status";
+}
+
+}  // extern "C"

@@ -1,0 +1,86 @@
+// Internal launcher interfaces shared by the .cu files of the library.
+#pragma once
+#include <cuda.h>
+#include <cuda_runtime.h>
+#include <stddef.h>
+#include <stdint.h>
+
+#include "../../include/pcl_dnn.h"
+
+namespace pcl {
+
+void count_launch(unsigned n = 1);
+
+// Address of the current device's status word (0 = fine, else the code of the
+// first bounded wait that ran out).  nullptr if the address cannot be obtained.
+unsigned int* device_status_ptr();
+
+// Driver entry point for cuTensorMapEncodeTiled, fetched at run time so that the
+// library has no link-time dependency on libcuda.  Returns nullptr on failure.
+typedef CUresult (*encode_tiled_fn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                    const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                    CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+encode_tiled_fn get_encode_tiled();
+
+// fp32 tensor map with a 128-byte swizzle.  dims/box innermost first;
+// strides_bytes has rank-1 entries (dims 1..rank-1).
+int make_tmap(CUtensorMap* out, const void* base, int rank, const uint64_t* dims, const uint64_t* strides_bytes,
+              const uint32_t* box);
+
+// ---- forward-type implicit GEMM on tcgen05 (stride-1 convolution) ----------
+// out[n,p,q,k] = epi( sum_{r,s,c} in[n, p + r - pad_h, q + s - pad_w, c] * wt[k, r*S+s, c] )
+// epi: + bias[k], activation, optional zeroing where mask_src[n,p,q,k] <= 0.
+struct TcFpropArgs {
+    const float* in;   // [N][H][W][Cin]
+    const float* wt;   // [Kout][R*S][Cin]
+    const float* bias; // [Kout] or null
+    const float* mask_src; // [N][P][Q][Kout] or null
+    float* out;        // [N][P][Q][Kout]
+    int N, H, W, Cin, Kout, R, S, pad_h, pad_w, P, Q, act;
+};
+bool tc_fprop_eligible(const TcFpropArgs& a);
+int launch_tc_fprop(const TcFpropArgs& a, cudaStream_t st);
+
+// ---- weight-gradient-type GEMM on tcgen05 (stride-1 convolution) -----------
+// dw[k, r, s, c] = sum_{n,p,q} dy[n,p,q,k] * x[n, p + r - pad_h, q + s - pad_w, c]
+struct TcWgradArgs {
+    const float* x;   // [N][H][W][C]
+    const float* dy;  // [N][P][Q][K]
+    float* dw;        // [K][R][S][C]
+    float* partial;   // workspace for the two-pass variant ([splits][K*R*S*C]) or null (atomics)
+    int N, H, W, C, K, R, S, pad_h, pad_w, P, Q;
+    int splits;
+};
+bool tc_wgrad_eligible(const TcWgradArgs& a);
+int tc_wgrad_splits(int N, int P, int Q, int C, int K, int R, int S);
+int launch_tc_wgrad(const TcWgradArgs& a, cudaStream_t st);
+
+// ---- generic CUDA-core kernels (any stride / pad / channel count) ----------
+int launch_generic_fwd(const pcl_conv_desc& d, int P, int Q, const float* x, const float* w, const float* bias,
+                       float* y, int act, cudaStream_t st);
+int launch_generic_bwd_data(const pcl_conv_desc& d, int P, int Q, const float* dy, const float* w,
+                            const float* mask_src, float* dx, cudaStream_t st);
+int generic_wgrad_splits(const pcl_conv_desc& d, int P, int Q);
+int launch_generic_bwd_weights(const pcl_conv_desc& d, int P, int Q, const float* x, const float* dy, float* dw,
+                               float* partial, int splits, cudaStream_t st);
+
+// ---- HBM-bound helpers ------------------------------------------------------
+int launch_sgd(float* w, const float* dw, size_t n, float lr, cudaStream_t st);
+int launch_reduce_splits(const float* partial, float* out, size_t n, int splits, cudaStream_t st);
+int launch_zero(float* p, size_t n, cudaStream_t st);
+// wt_t[c][R-1-r][S-1-s][k] = w[k][r][s][c]
+int launch_transpose_flip(const float* w, float* wt_t, int K, int R, int S, int C, cudaStream_t st);
+// dz = dy * act'(y), in place on dy
+int launch_act_grad(float* dy, const float* y, size_t n, int act, cudaStream_t st);
+// out[k] = sum_rows m[row][k]; partial: [colsum_splits(rows)][K] workspace
+int colsum_splits(size_t rows);
+int launch_colsum(const float* m, size_t rows, int K, float* partial, float* out, cudaStream_t st);
+int launch_maxpool_fwd(int N, int H, int W, int C, const float* x, float* y, cudaStream_t st);
+int launch_maxpool_bwd(int N, int H, int W, int C, const float* x, const float* dy, const float* mask, float* dx,
+                       cudaStream_t st);
+int launch_softmax_xent(int N, int K, const float* logits, const int* labels, float* loss, float* dlogits,
+                        cudaStream_t st);
+
+inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+}  // namespace pcl

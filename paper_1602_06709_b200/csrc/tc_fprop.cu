@@ -1,0 +1,351 @@
+// Forward-type implicit-GEMM convolution on the 5th-generation tensor cores.
+//
+//   out[n,p,q,k] = epi( sum_{r,s,c} in[n, p+r-pad_h, q+s-pad_w, c] * wt[k, r*S+s, c] )
+//
+// (Algorithm 1 with stride 1; the same kernel computes the backward-data pass of
+// a stride-1 layer when it is handed dy as `in` and the flipped, transposed
+// weights, and the fully-connected GEMMs as the 1x1 / 1x1-map special case.)
+//
+// GEMM view: M = N*P*Q output pixels, N = Kout, reduction over (r, s, c).
+// One CTA tile is 128 output pixels x BN output maps.  The 128 pixels are a
+// box bw x bh x bn of the (q, p, n) index space, so that for a fixed tap (r, s)
+// the A operand is one 4-D TMA box of the NHWC input shifted by the tap: the
+// im2col matrix is never materialised and zero padding is TMA's out-of-bounds
+// fill.  B is a 3-D TMA box {32 c, 1 tap, BN k} of the weights.
+//
+// Warp roles (192 threads, persistent over tiles):
+//   warp 0     TMA producer, fills a ring of `stages` {A 16 KB, B BN*128 B} slots
+//   warp 1     allocates TMEM, issues tcgen05.mma kind::tf32 (4 per slot, K = 8 each)
+//   warps 2-5  epilogue: TMEM -> registers -> bias/activation/mask -> global
+// Two TMEM accumulators (2 x BN columns) let the epilogue of tile i overlap the
+// main loop of tile i+1.
+#include "pcl_internal.h"
+#include "pcl_ptx.cuh"
+
+namespace pcl {
+
+namespace {
+
+constexpr int kTileM = 128;
+constexpr int kBlockC = 32;                      // fp32 elements per 128-byte swizzle row
+constexpr int kABytes = kTileM * kBlockC * 4;    // 16 KB
+constexpr int kMaxStages = 8;
+constexpr int kSmemBudget = 224 * 1024;
+
+struct FpropParams {
+    int bw_log2, bh_log2;       // box of output pixels: bw x bh x (128 / (bw*bh))
+    int tiles_q, tiles_p, tiles_n, tiles_k;
+    int BN;                     // output maps per tile, multiple of 32, <= 256
+    int R, S, pad_h, pad_w, cblocks;
+    int N, P, Q, Kout;
+    int act;
+    int stages;
+    int tmem_cols;
+    const float* bias;
+    const float* mask_src;
+    float* out;
+    unsigned int* status;       // device status word
+};
+
+__global__ void __launch_bounds__(192, 1)
+tc_fprop_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, FpropParams p) {
+    extern __shared__ uint8_t smem_raw[];
+    __shared__ uint64_t full_bar[kMaxStages];
+    __shared__ uint64_t empty_bar[kMaxStages];
+    __shared__ uint64_t tmem_full_bar[2];
+    __shared__ uint64_t tmem_empty_bar[2];
+    __shared__ uint32_t tmem_base_slot;
+    __shared__ uint32_t abort_flag;
+
+    const int warp = threadIdx.x >> 5;
+    const int lane = threadIdx.x & 31;
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    const uint32_t stage_bytes = kABytes + p.BN * 128;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < p.stages; ++s) {
+            mbar_init(&full_bar[s], 1);
+            mbar_init(&empty_bar[s], 1);
+        }
+        for (int a = 0; a < 2; ++a) {
+            mbar_init(&tmem_full_bar[a], 1);
+            mbar_init(&tmem_empty_bar[a], 4);
+        }
+        abort_flag = 0;
+        mbar_fence_init();
+        prefetch_tmap(&tmA);
+        prefetch_tmap(&tmB);
+    }
+    if (warp == 1) {
+        tmem_alloc(&tmem_base_slot, p.tmem_cols);
+        tmem_relinquish();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = tmem_base_slot;
+
+    const int bw = 1 << p.bw_log2, bh = 1 << p.bh_log2;
+    const int bn = kTileM >> (p.bw_log2 + p.bh_log2);
+    const int m_tiles = p.tiles_q * p.tiles_p * p.tiles_n;
+    const int total_tiles = m_tiles * p.tiles_k;
+    const int kiters = p.R * p.S * p.cblocks;
+
+    if (warp == 0) {
+        // ------------------------------------------------------------ producer
+        if (lane == 0) {
+            int stage = 0;
+            uint32_t phase = 0;
+            int issued = 0;
+            bool ok = true;
+            for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
+                const int kt = t % p.tiles_k;
+                int m = t / p.tiles_k;
+                const int q0 = (m % p.tiles_q) * bw;  m /= p.tiles_q;
+                const int p0 = (m % p.tiles_p) * bh;
+                const int n0 = (m / p.tiles_p) * bn;
+                for (int r = 0; r < p.R && ok; ++r)
+                    for (int s = 0; s < p.S && ok; ++s)
+                        for (int cb = 0; cb < p.cblocks; ++cb) {
+                            if (!bounded_wait(&empty_bar[stage], phase ^ 1u, &abort_flag, p.status, WAIT_PRODUCER_EMPTY)) {
+                                ok = false;
+                                break;
+                            }
+                            uint8_t* a_dst = smem + stage * stage_bytes;
+                            mbar_expect_tx(&full_bar[stage], stage_bytes);
+                            tma_load_4d(a_dst, &tmA, &full_bar[stage], cb * kBlockC, q0 + s - p.pad_w,
+                                        p0 + r - p.pad_h, n0);
+                            tma_load_3d(a_dst + kABytes, &tmB, &full_bar[stage], cb * kBlockC, r * p.S + s,
+                                        kt * p.BN);
+                            ++issued;
+                            if (++stage == p.stages) { stage = 0; phase ^= 1u; }
+                        }
+            }
+            if (!ok) {
+                // Gave up: the copies already issued still land in this CTA's shared
+                // memory, so wait (bounded) for each armed slot before leaving.
+                const int pending = issued < p.stages ? issued : p.stages;
+                for (int j = 0; j < pending; ++j) {
+                    if (--stage < 0) { stage = p.stages - 1; phase ^= 1u; }
+                    for (uint32_t spin = 0; spin < (1u << 20); ++spin)
+                        if (mbar_try_wait(&full_bar[stage], phase)) break;
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ---------------------------------------------------------- MMA issuer
+        const uint32_t idesc = make_idesc_tf32(p.BN, false, false);
+        int stage = 0;
+        uint32_t phase = 0;
+        int tile_cnt = 0;
+        bool ok = true;
+        for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x, ++tile_cnt) {
+            const int acc = tile_cnt & 1;
+            const uint32_t acc_phase = (tile_cnt >> 1) & 1;
+            if (!bounded_wait(&tmem_empty_bar[acc], acc_phase ^ 1u, &abort_flag, p.status, WAIT_MMA_TMEM_EMPTY)) break;
+            tc_fence_after();
+            const uint32_t d_tmem = tmem_base + acc * p.BN;
+            for (int kit = 0; kit < kiters; ++kit) {
+                if (!bounded_wait(&full_bar[stage], phase, &abort_flag, p.status, WAIT_MMA_FULL)) { ok = false; break; }
+                tc_fence_after();
+                if (lane == 0) {
+                    const uint32_t a_addr = smem_u32(smem + stage * stage_bytes);
+                    const uint32_t b_addr = a_addr + kABytes;
+#pragma unroll
+                    for (int kk = 0; kk < 4; ++kk) {
+                        const uint64_t da = make_sw128_desc(a_addr + kk * 32, 16, 1024);
+                        const uint64_t db = make_sw128_desc(b_addr + kk * 32, 16, 1024);
+                        umma_tf32(d_tmem, da, db, idesc, (kit | kk) != 0);
+                    }
+                    umma_commit(&empty_bar[stage]);
+                }
+                __syncwarp();
+                if (++stage == p.stages) { stage = 0; phase ^= 1u; }
+            }
+            if (ok && lane == 0) umma_commit(&tmem_full_bar[acc]);
+            __syncwarp();
+        }
+    } else {
+        // ------------------------------------------------------------ epilogue
+        const int quarter = warp & 3;           // TMEM lanes 32*quarter .. +31
+        const int row = quarter * 32 + lane;    // row of the tile = pixel of the box
+        const int iw = row & (bw - 1);
+        const int ih = (row >> p.bw_log2) & (bh - 1);
+        const int in_ = row >> (p.bw_log2 + p.bh_log2);
+        const bool vec_ok = (p.Kout & 3) == 0;
+        int tile_cnt = 0;
+        for (int t = blockIdx.x; t < total_tiles; t += gridDim.x, ++tile_cnt) {
+            const int acc = tile_cnt & 1;
+            const uint32_t acc_phase = (tile_cnt >> 1) & 1;
+            const int kt = t % p.tiles_k;
+            int m = t / p.tiles_k;
+            const int q = (m % p.tiles_q) * bw + iw;  m /= p.tiles_q;
+            const int pp = (m % p.tiles_p) * bh + ih;
+            const int n = (m / p.tiles_p) * bn + in_;
+            const bool valid = (q < p.Q) && (pp < p.P) && (n < p.N);
+            const size_t pix = (static_cast<size_t>(n) * p.P + pp) * p.Q + q;
+            if (!bounded_wait(&tmem_full_bar[acc], acc_phase, &abort_flag, p.status, WAIT_EPI_TMEM_FULL)) break;
+            tc_fence_after();
+            const uint32_t t_row = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + acc * p.BN;
+            for (int ch = 0; ch < p.BN / 32; ++ch) {
+                uint32_t v[32];
+                tmem_ld_32x32(t_row + ch * 32, v);
+                tmem_ld_wait();
+                const int col0 = kt * p.BN + ch * 32;
+                if (valid && col0 < p.Kout) {
+                    float* dst = p.out + pix * p.Kout + col0;
+                    const float* msk = p.mask_src ? p.mask_src + pix * p.Kout + col0 : nullptr;
+                    if (vec_ok) {
+#pragma unroll
+                        for (int j = 0; j < 32; j += 4) {
+                            if (col0 + j < p.Kout) {
+                                float4 o = make_float4(__uint_as_float(v[j]), __uint_as_float(v[j + 1]),
+                                                       __uint_as_float(v[j + 2]), __uint_as_float(v[j + 3]));
+                                if (p.bias) {
+                                    const float4 b = __ldg(reinterpret_cast<const float4*>(p.bias + col0 + j));
+                                    o.x += b.x; o.y += b.y; o.z += b.z; o.w += b.w;
+                                }
+                                if (p.act == PCL_ACT_RELU) {
+                                    o.x = fmaxf(o.x, 0.f); o.y = fmaxf(o.y, 0.f);
+                                    o.z = fmaxf(o.z, 0.f); o.w = fmaxf(o.w, 0.f);
+                                } else if (p.act == PCL_ACT_SIGMOID) {
+                                    o.x = 1.f / (1.f + __expf(-o.x)); o.y = 1.f / (1.f + __expf(-o.y));
+                                    o.z = 1.f / (1.f + __expf(-o.z)); o.w = 1.f / (1.f + __expf(-o.w));
+                                }
+                                if (msk) {
+                                    const float4 mk = __ldg(reinterpret_cast<const float4*>(msk + j));
+                                    o.x = mk.x > 0.f ? o.x : 0.f; o.y = mk.y > 0.f ? o.y : 0.f;
+                                    o.z = mk.z > 0.f ? o.z : 0.f; o.w = mk.w > 0.f ? o.w : 0.f;
+                                }
+                                *reinterpret_cast<float4*>(dst + j) = o;
+                            }
+                        }
+                    } else {
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) {
+                            if (col0 + j < p.Kout) {
+                                float o = __uint_as_float(v[j]);
+                                if (p.bias) o += __ldg(p.bias + col0 + j);
+                                if (p.act == PCL_ACT_RELU) o = fmaxf(o, 0.f);
+                                else if (p.act == PCL_ACT_SIGMOID) o = 1.f / (1.f + __expf(-o));
+                                if (msk && !(__ldg(msk + j) > 0.f)) o = 0.f;
+                                dst[j] = o;
+                            }
+                        }
+                    }
+                }
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&tmem_empty_bar[acc]);
+        }
+    }
+
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        tmem_dealloc(tmem_base, p.tmem_cols);
+    }
+}
+
+// Pick the 128-pixel box bw x bh x bn (powers of two) that wastes the least
+// work on ragged edges; ties go to the widest box.
+void choose_box(int P, int Q, int N, int* bw_log2, int* bh_log2) {
+    double best = 1e300;
+    int best_w = 0, best_h = 0;
+    for (int lw = 7; lw >= 0; --lw)
+        for (int lh = 7 - lw; lh >= 0; --lh) {
+            const long bw = 1L << lw, bh = 1L << lh, bn = 128 / (bw * bh);
+            const double covered = double((Q + bw - 1) / bw * bw) * double((P + bh - 1) / bh * bh) *
+                                   double((N + bn - 1) / bn * bn);
+            if (covered < best) { best = covered; best_w = lw; best_h = lh; }
+        }
+    *bw_log2 = best_w;
+    *bh_log2 = best_h;
+}
+
+int choose_bn(int Kout, long m_tiles, int sm_count) {
+    // Widest tile that still gives every SM a tile; otherwise the narrowest
+    // width that keeps the tile count from growing further.
+    const int k32 = (Kout + 31) / 32 * 32;
+    int bn = k32 < 256 ? k32 : 256;
+    {   // balance the last tile: Kout = 1000 -> 4 x 256 rather than 3 x 256 + 232
+        const int tiles = (Kout + bn - 1) / bn;
+        bn = ((Kout + tiles - 1) / tiles + 31) / 32 * 32;
+    }
+    while (bn > 64 && m_tiles * ((Kout + bn - 1) / bn) < sm_count) {
+        const int half = (bn / 2 + 31) / 32 * 32;
+        bn = half;
+    }
+    return bn;
+}
+
+int g_sm_count = 0;
+
+}  // namespace
+
+bool tc_fprop_eligible(const TcFpropArgs& a) {
+    if (a.Cin % 4 != 0) return false;                       // TMA strides are multiples of 16 bytes
+    if ((reinterpret_cast<uintptr_t>(a.in) | reinterpret_cast<uintptr_t>(a.wt)) & 15) return false;
+    if (a.R * a.S > 65535) return false;
+    return true;
+}
+
+int launch_tc_fprop(const TcFpropArgs& a, cudaStream_t st) {
+    if (!tc_fprop_eligible(a)) return PCL_ERR_UNSUPPORTED_SHAPE;
+    if (g_sm_count == 0) {
+        int dev = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess) return PCL_ERR_CUDA;
+        if (cudaDeviceGetAttribute(&g_sm_count, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return PCL_ERR_CUDA;
+        if (cudaFuncSetAttribute(tc_fprop_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget + 1024) !=
+            cudaSuccess)
+            return PCL_ERR_CUDA;
+    }
+    FpropParams p{};
+    choose_box(a.P, a.Q, a.N, &p.bw_log2, &p.bh_log2);
+    const int bw = 1 << p.bw_log2, bh = 1 << p.bh_log2, bn = kTileM / (bw * bh);
+    p.tiles_q = (a.Q + bw - 1) / bw;
+    p.tiles_p = (a.P + bh - 1) / bh;
+    p.tiles_n = (a.N + bn - 1) / bn;
+    const long m_tiles = long(p.tiles_q) * p.tiles_p * p.tiles_n;
+    p.BN = choose_bn(a.Kout, m_tiles, g_sm_count);
+    p.tiles_k = (a.Kout + p.BN - 1) / p.BN;
+    if (m_tiles * p.tiles_k > 0x7fffffffL) return PCL_ERR_UNSUPPORTED_SHAPE;
+    p.R = a.R; p.S = a.S; p.pad_h = a.pad_h; p.pad_w = a.pad_w;
+    p.cblocks = (a.Cin + kBlockC - 1) / kBlockC;
+    p.N = a.N; p.P = a.P; p.Q = a.Q; p.Kout = a.Kout;
+    p.act = a.act;
+    const int stage_bytes = kABytes + p.BN * 128;
+    p.stages = kSmemBudget / stage_bytes;
+    if (p.stages > kMaxStages) p.stages = kMaxStages;
+    p.tmem_cols = 32;
+    while (p.tmem_cols < 2 * p.BN) p.tmem_cols *= 2;
+    p.bias = a.bias; p.mask_src = a.mask_src; p.out = a.out;
+    p.status = device_status_ptr();
+    if (!p.status) return PCL_ERR_CUDA;
+
+    CUtensorMap tmA, tmB;
+    {
+        const uint64_t dims[4] = {uint64_t(a.Cin), uint64_t(a.W), uint64_t(a.H), uint64_t(a.N)};
+        const uint64_t strides[3] = {uint64_t(a.Cin) * 4, uint64_t(a.W) * a.Cin * 4, uint64_t(a.H) * a.W * a.Cin * 4};
+        const uint32_t box[4] = {kBlockC, uint32_t(bw), uint32_t(bh), uint32_t(bn)};
+        int rc = make_tmap(&tmA, a.in, 4, dims, strides, box);
+        if (rc != PCL_OK) return rc;
+    }
+    {
+        const uint64_t dims[3] = {uint64_t(a.Cin), uint64_t(a.R) * a.S, uint64_t(a.Kout)};
+        const uint64_t strides[2] = {uint64_t(a.Cin) * 4, uint64_t(a.R) * a.S * a.Cin * 4};
+        const uint32_t box[3] = {kBlockC, 1, uint32_t(p.BN)};
+        int rc = make_tmap(&tmB, a.wt, 3, dims, strides, box);
+        if (rc != PCL_OK) return rc;
+    }
+    const long total = m_tiles * p.tiles_k;
+    const int grid = int(total < g_sm_count ? total : g_sm_count);
+    const size_t smem = size_t(p.stages) * stage_bytes + 1024;
+    tc_fprop_kernel<<<grid, 192, smem, st>>>(tmA, tmB, p);
+    count_launch();
+    return cudaGetLastError() == cudaSuccess ? PCL_OK : PCL_ERR_CUDA;
+}
+
+}  // namespace pcl

@@ -1,0 +1,331 @@
+// Weight-gradient pass on the 5th-generation tensor cores (stride-1 layers).
+//
+//   dw[k, r, s, c] = sum_{n,p,q} dy[n,p,q,k] * x[n, p+r-pad_h, q+s-pad_w, c]
+//
+// GEMM view per tap (r, s): M = K output maps, N = C input maps, reduction over
+// the N*P*Q output pixels.  The reduction index is the OUTER dimension of both
+// NHWC tensors, so both operands are "MN-major": a TMA box {32 maps, 32 pixels}
+// lands in shared memory as 32 rows (one per pixel) of 128 bytes, which is the
+// 128-byte-swizzled MN-major operand layout of tcgen05.mma.  The x box is the
+// dy box shifted by the tap, with zero padding supplied by TMA's out-of-bounds
+// fill.
+//
+// The output is tiny compared with the reduction (Sec. 2.4/2.5 make the same
+// observation), so the pixel range is split across CTAs ("privatise and
+// reduce"): a work item is (128-row k tile, tap, c tile, pixel split); each CTA
+// accumulates its item in TMEM and either writes a partial tile to the
+// workspace (second pass adds the splits in a fixed order) or adds it to dw with
+// fp32 atomics.
+#include "pcl_internal.h"
+#include "pcl_ptx.cuh"
+
+namespace pcl {
+
+namespace {
+
+constexpr int kPix = 32;              // pixels (reduction indices) per pipeline slot
+constexpr int kGroupBytes = kPix * 128;   // one {32 maps x 32 pixels} box
+constexpr int kABytes = 4 * kGroupBytes;  // 128 output maps
+constexpr int kMaxStages = 8;
+constexpr int kSmemBudget = 224 * 1024;
+
+struct WgradParams {
+    int bw_log2, bh_log2;     // pixel box bw x bh x (32/(bw*bh))
+    int boxes_q, boxes_p, boxes_n;
+    int k_tiles, c_tiles, BNc;
+    int R, S, pad_h, pad_w;
+    int K, C;
+    int splits, boxes_per_split;
+    int stages, tmem_cols;
+    int use_atomics;
+    float* out;               // dw, or the partial-sum workspace [splits][K*R*S*C]
+    size_t split_stride;      // K*R*S*C (0 when writing straight to dw)
+    unsigned int* status;     // device status word
+};
+
+__global__ void __launch_bounds__(192, 1)
+tc_wgrad_kernel(const __grid_constant__ CUtensorMap tmDy, const __grid_constant__ CUtensorMap tmX, WgradParams p) {
+    extern __shared__ uint8_t smem_raw[];
+    __shared__ uint64_t full_bar[kMaxStages];
+    __shared__ uint64_t empty_bar[kMaxStages];
+    __shared__ uint64_t tmem_full_bar;
+    __shared__ uint32_t tmem_base_slot;
+    __shared__ uint32_t abort_flag;
+
+    const int warp = threadIdx.x >> 5;
+    const int lane = threadIdx.x & 31;
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    const int b_groups = p.BNc / 32;
+    const uint32_t stage_bytes = kABytes + b_groups * kGroupBytes;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < p.stages; ++s) {
+            mbar_init(&full_bar[s], 1);
+            mbar_init(&empty_bar[s], 1);
+        }
+        mbar_init(&tmem_full_bar, 1);
+        abort_flag = 0;
+        mbar_fence_init();
+        prefetch_tmap(&tmDy);
+        prefetch_tmap(&tmX);
+    }
+    if (warp == 1) {
+        tmem_alloc(&tmem_base_slot, p.tmem_cols);
+        tmem_relinquish();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = tmem_base_slot;
+
+    // work item of this CTA
+    int item = blockIdx.x;
+    const int split = item % p.splits;   item /= p.splits;
+    const int ct = item % p.c_tiles;     item /= p.c_tiles;
+    const int tap = item % (p.R * p.S);
+    const int kt = item / (p.R * p.S);
+    const int r = tap / p.S, s = tap % p.S;
+    const int total_boxes = p.boxes_q * p.boxes_p * p.boxes_n;
+    const int box_begin = split * p.boxes_per_split;
+    int box_end = box_begin + p.boxes_per_split;
+    if (box_end > total_boxes) box_end = total_boxes;
+    const int kiters = box_end > box_begin ? box_end - box_begin : 0;
+    const int bw = 1 << p.bw_log2, bh = 1 << p.bh_log2, bn = kPix >> (p.bw_log2 + p.bh_log2);
+
+    if (warp == 0) {
+        if (lane == 0) {
+            int stage = 0;
+            uint32_t phase = 0;
+            int issued = 0;
+            bool ok = true;
+            for (int b = box_begin; b < box_end; ++b) {
+                int m = b;
+                const int q0 = (m % p.boxes_q) * bw;  m /= p.boxes_q;
+                const int p0 = (m % p.boxes_p) * bh;
+                const int n0 = (m / p.boxes_p) * bn;
+                if (!bounded_wait(&empty_bar[stage], phase ^ 1u, &abort_flag, p.status, WAIT_PRODUCER_EMPTY)) { ok = false; break; }
+                uint8_t* dst = smem + stage * stage_bytes;
+                mbar_expect_tx(&full_bar[stage], stage_bytes);
+#pragma unroll
+                for (int g = 0; g < 4; ++g)
+                    tma_load_4d(dst + g * kGroupBytes, &tmDy, &full_bar[stage], kt * 128 + g * 32, q0, p0, n0);
+                for (int g = 0; g < b_groups; ++g)
+                    tma_load_4d(dst + kABytes + g * kGroupBytes, &tmX, &full_bar[stage], ct * p.BNc + g * 32,
+                                q0 + s - p.pad_w, p0 + r - p.pad_h, n0);
+                ++issued;
+                if (++stage == p.stages) { stage = 0; phase ^= 1u; }
+            }
+            if (!ok) {
+                const int pending = issued < p.stages ? issued : p.stages;
+                for (int j = 0; j < pending; ++j) {
+                    if (--stage < 0) { stage = p.stages - 1; phase ^= 1u; }
+                    for (uint32_t spin = 0; spin < (1u << 20); ++spin)
+                        if (mbar_try_wait(&full_bar[stage], phase)) break;
+                }
+            }
+        }
+    } else if (warp == 1) {
+        const uint32_t idesc = make_idesc_tf32(p.BNc, true, true);
+        int stage = 0;
+        uint32_t phase = 0;
+        bool ok = true;
+        for (int kit = 0; kit < kiters; ++kit) {
+            if (!bounded_wait(&full_bar[stage], phase, &abort_flag, p.status, WAIT_MMA_FULL)) { ok = false; break; }
+            tc_fence_after();
+            if (lane == 0) {
+                const uint32_t a_addr = smem_u32(smem + stage * stage_bytes);
+                const uint32_t b_addr = a_addr + kABytes;
+#pragma unroll
+                for (int kk = 0; kk < kPix / 8; ++kk) {
+                    // 8 pixels per instruction = one 1024-byte group of 8 rows
+                    const uint64_t da = make_sw128_desc(a_addr + kk * 1024, kGroupBytes, 1024);
+                    const uint64_t db = make_sw128_desc(b_addr + kk * 1024, kGroupBytes, 1024);
+                    umma_tf32(tmem_base, da, db, idesc, (kit | kk) != 0);
+                }
+                umma_commit(&empty_bar[stage]);
+            }
+            __syncwarp();
+            if (++stage == p.stages) { stage = 0; phase ^= 1u; }
+        }
+        if (ok && lane == 0) umma_commit(&tmem_full_bar);
+        __syncwarp();
+    } else {
+        const int quarter = warp & 3;
+        const int k = kt * 128 + quarter * 32 + lane;
+        const bool valid = k < p.K;
+        const bool vec_ok = (p.C & 3) == 0;
+        if (bounded_wait(&tmem_full_bar, 0, &abort_flag, p.status, WAIT_EPI_TMEM_FULL)) {
+            tc_fence_after();
+            const uint32_t t_row = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16);
+            float* base = p.out + static_cast<size_t>(split) * p.split_stride +
+                          ((static_cast<size_t>(valid ? k : 0) * p.R + r) * p.S + s) * p.C;
+            for (int ch = 0; ch < b_groups; ++ch) {
+                uint32_t v[32];
+                if (kiters > 0) {
+                    tmem_ld_32x32(t_row + ch * 32, v);
+                    tmem_ld_wait();
+                } else {
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) v[j] = 0u;
+                }
+                const int c0 = ct * p.BNc + ch * 32;
+                if (valid && c0 < p.C) {
+                    float* dst = base + c0;
+                    if (p.use_atomics) {
+#pragma unroll
+                        for (int j = 0; j < 32; ++j)
+                            if (c0 + j < p.C) atomicAdd(dst + j, __uint_as_float(v[j]));
+                    } else if (vec_ok) {
+#pragma unroll
+                        for (int j = 0; j < 32; j += 4)
+                            if (c0 + j < p.C)
+                                *reinterpret_cast<float4*>(dst + j) =
+                                    make_float4(__uint_as_float(v[j]), __uint_as_float(v[j + 1]),
+                                                __uint_as_float(v[j + 2]), __uint_as_float(v[j + 3]));
+                    } else {
+#pragma unroll
+                        for (int j = 0; j < 32; ++j)
+                            if (c0 + j < p.C) dst[j] = __uint_as_float(v[j]);
+                    }
+                }
+            }
+        }
+    }
+
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        tmem_dealloc(tmem_base, p.tmem_cols);
+    }
+}
+
+void choose_pixel_box(int P, int Q, int N, int* bw_log2, int* bh_log2) {
+    double best = 1e300;
+    int best_w = 0, best_h = 0;
+    for (int lw = 5; lw >= 0; --lw)
+        for (int lh = 5 - lw; lh >= 0; --lh) {
+            const long bw = 1L << lw, bh = 1L << lh, bn = kPix / (bw * bh);
+            const double covered = double((Q + bw - 1) / bw * bw) * double((P + bh - 1) / bh * bh) *
+                                   double((N + bn - 1) / bn * bn);
+            if (covered < best) { best = covered; best_w = lw; best_h = lh; }
+        }
+    *bw_log2 = best_w;
+    *bh_log2 = best_h;
+}
+
+int choose_bnc(int C) {
+    const int c32 = (C + 31) / 32 * 32;
+    int bn = c32 < 256 ? c32 : 256;
+    const int tiles = (C + bn - 1) / bn;
+    return ((C + tiles - 1) / tiles + 31) / 32 * 32;
+}
+
+long total_pixel_boxes(int N, int P, int Q) {
+    int lw, lh;
+    choose_pixel_box(P, Q, N, &lw, &lh);
+    const long bw = 1L << lw, bh = 1L << lh, bn = kPix / (bw * bh);
+    return ((Q + bw - 1) / bw) * ((P + bh - 1) / bh) * ((N + bn - 1) / bn);
+}
+
+int g_sm_count = 0;
+int sm_count() {
+    if (g_sm_count == 0) {
+        int dev = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess ||
+            cudaDeviceGetAttribute(&g_sm_count, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || g_sm_count <= 0)
+            g_sm_count = 148;   // sizing only; a launch would fail anyway without a device
+    }
+    return g_sm_count;
+}
+bool g_attr_set = false;
+
+}  // namespace
+
+bool tc_wgrad_eligible(const TcWgradArgs& a) {
+    if (a.C % 4 != 0 || a.K % 4 != 0) return false;
+    if ((reinterpret_cast<uintptr_t>(a.x) | reinterpret_cast<uintptr_t>(a.dy)) & 15) return false;
+    return true;
+}
+
+int tc_wgrad_splits(int N, int P, int Q, int C, int K, int R, int S) {
+    const int bnc = choose_bnc(C);
+    const long items = long((K + 127) / 128) * R * S * ((C + bnc - 1) / bnc);
+    const long boxes = total_pixel_boxes(N, P, Q);
+    long splits = sm_count() / items;
+    if (splits < 1) splits = 1;
+    if (splits > 64) splits = 64;
+    if (splits > boxes) splits = boxes;
+    // drop splits that would be empty
+    const long per = (boxes + splits - 1) / splits;
+    splits = (boxes + per - 1) / per;
+    return int(splits);
+}
+
+int launch_tc_wgrad(const TcWgradArgs& a, cudaStream_t st) {
+    if (!tc_wgrad_eligible(a)) return PCL_ERR_UNSUPPORTED_SHAPE;
+    if (!g_attr_set) {
+        if (cudaFuncSetAttribute(tc_wgrad_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget + 1024) !=
+            cudaSuccess)
+            return PCL_ERR_CUDA;
+        g_attr_set = true;
+    }
+    WgradParams p{};
+    choose_pixel_box(a.P, a.Q, a.N, &p.bw_log2, &p.bh_log2);
+    const int bw = 1 << p.bw_log2, bh = 1 << p.bh_log2, bn = kPix / (bw * bh);
+    p.boxes_q = (a.Q + bw - 1) / bw;
+    p.boxes_p = (a.P + bh - 1) / bh;
+    p.boxes_n = (a.N + bn - 1) / bn;
+    const long boxes = long(p.boxes_q) * p.boxes_p * p.boxes_n;
+    if (boxes > 0x7fffffffL) return PCL_ERR_UNSUPPORTED_SHAPE;
+    p.BNc = choose_bnc(a.C);
+    p.c_tiles = (a.C + p.BNc - 1) / p.BNc;
+    p.k_tiles = (a.K + 127) / 128;
+    p.R = a.R; p.S = a.S; p.pad_h = a.pad_h; p.pad_w = a.pad_w;
+    p.K = a.K; p.C = a.C;
+    p.splits = a.splits;
+    p.boxes_per_split = int((boxes + p.splits - 1) / p.splits);
+    const int stage_bytes = kABytes + (p.BNc / 32) * kGroupBytes;
+    p.stages = kSmemBudget / stage_bytes;
+    if (p.stages > kMaxStages) p.stages = kMaxStages;
+    p.tmem_cols = 32;
+    while (p.tmem_cols < p.BNc) p.tmem_cols *= 2;
+    p.status = device_status_ptr();
+    if (!p.status) return PCL_ERR_CUDA;
+    const size_t dw_elems = size_t(a.K) * a.R * a.S * a.C;
+    if (p.splits == 1) {
+        p.out = a.dw; p.split_stride = 0; p.use_atomics = 0;
+    } else if (a.partial) {
+        p.out = a.partial; p.split_stride = dw_elems; p.use_atomics = 0;
+    } else {
+        p.out = a.dw; p.split_stride = 0; p.use_atomics = 1;
+        int rc = launch_zero(a.dw, dw_elems, st);
+        if (rc != PCL_OK) return rc;
+    }
+
+    CUtensorMap tmDy, tmX;
+    {
+        const uint64_t dims[4] = {uint64_t(a.K), uint64_t(a.Q), uint64_t(a.P), uint64_t(a.N)};
+        const uint64_t strides[3] = {uint64_t(a.K) * 4, uint64_t(a.Q) * a.K * 4, uint64_t(a.P) * a.Q * a.K * 4};
+        const uint32_t box[4] = {32, uint32_t(bw), uint32_t(bh), uint32_t(bn)};
+        int rc = make_tmap(&tmDy, a.dy, 4, dims, strides, box);
+        if (rc != PCL_OK) return rc;
+    }
+    {
+        const uint64_t dims[4] = {uint64_t(a.C), uint64_t(a.W), uint64_t(a.H), uint64_t(a.N)};
+        const uint64_t strides[3] = {uint64_t(a.C) * 4, uint64_t(a.W) * a.C * 4, uint64_t(a.H) * a.W * a.C * 4};
+        const uint32_t box[4] = {32, uint32_t(bw), uint32_t(bh), uint32_t(bn)};
+        int rc = make_tmap(&tmX, a.x, 4, dims, strides, box);
+        if (rc != PCL_OK) return rc;
+    }
+    const long items = long(p.k_tiles) * a.R * a.S * p.c_tiles * p.splits;
+    if (items > 0x7fffffffL) return PCL_ERR_UNSUPPORTED_SHAPE;
+    const size_t smem = size_t(p.stages) * stage_bytes + 1024;
+    tc_wgrad_kernel<<<int(items), 192, smem, st>>>(tmDy, tmX, p);
+    count_launch();
+    if (cudaGetLastError() != cudaSuccess) return PCL_ERR_CUDA;
+    if (p.splits > 1 && a.partial) return launch_reduce_splits(a.partial, a.dw, dw_elems, p.splits, st);
+    return PCL_OK;
+}
+
+}  // namespace pcl

@@ -1,0 +1,100 @@
+"""GPU parity: the three convolution passes through the C ABI against the fp64
+oracle, element by element, on seeded inputs.  Shapes span several tiles and
+ragged tails in every tiled dimension; both kernel families are exercised."""
+import numpy as np
+import pytest
+
+import oracle
+from oracle import ConvShape
+
+pytestmark = pytest.mark.gpu
+
+TENSOR_SHAPES = {
+    "cfg1": ConvShape(N=4, C=16, K=32, H=16, W=16, R=3, S=3, pad_h=1, pad_w=1),
+    "ragged": ConvShape(N=3, C=40, K=72, H=19, W=23, R=3, S=3, pad_h=1, pad_w=1),
+    "k5_nopad": ConvShape(N=2, C=32, K=64, H=24, W=24, R=5, S=5),
+    "one_by_one": ConvShape(N=5, C=64, K=128, H=9, W=9, R=1, S=1),
+    "wide_k": ConvShape(N=4, C=64, K=320, H=12, W=12, R=3, S=3, pad_h=1, pad_w=1),
+    "deep_c": ConvShape(N=2, C=288, K=48, H=14, W=14, R=3, S=3, pad_h=1, pad_w=1),
+    "rect_kernel": ConvShape(N=2, C=24, K=40, H=10, W=17, R=2, S=3, pad_h=1, pad_w=0),
+    "many_pixels": ConvShape(N=6, C=32, K=32, H=56, W=56, R=3, S=3, pad_h=1, pad_w=1),
+}
+GENERIC_SHAPES = {
+    "rgb": ConvShape(N=2, C=3, K=16, H=20, W=20, R=3, S=3, pad_h=1, pad_w=1),
+    "rgb_stride4": ConvShape(N=2, C=3, K=24, H=47, W=47, R=11, S=11, stride_h=4, stride_w=4),
+    "stride2": ConvShape(N=3, C=20, K=36, H=15, W=18, R=3, S=3, stride_h=2, stride_w=2, pad_h=1, pad_w=1),
+    "odd_channels": ConvShape(N=2, C=7, K=9, H=11, W=13, R=3, S=3, pad_h=1, pad_w=1),
+    "mixed_stride": ConvShape(N=2, C=8, K=12, H=16, W=16, R=3, S=5, stride_h=1, stride_w=2, pad_h=0, pad_w=2),
+}
+
+
+def _cases():
+    from paper_1602_06709_b200 import binding as B
+    out = []
+    for tag, s in TENSOR_SHAPES.items():
+        out.append(pytest.param(tag, s, B.PATH_TENSOR, id=f"tensor-{tag}"))
+        out.append(pytest.param(tag, s, B.PATH_GENERIC, id=f"generic-{tag}"))
+    for tag, s in GENERIC_SHAPES.items():
+        out.append(pytest.param(tag, s, B.PATH_AUTO, id=f"auto-{tag}"))
+    return out
+
+
+@pytest.fixture
+def path_guard():
+    from paper_1602_06709_b200 import binding as B
+    yield
+    B.set_path(B.PATH_AUTO)
+
+
+@pytest.mark.parametrize("tag,s,path", _cases())
+def test_conv_three_passes(tag, s, path, path_guard):
+    import gpu_helpers as G
+    from paper_1602_06709_b200 import binding as B
+    B.set_path(path)
+    x, w, dy, bias = G.make_inputs(s, tag)
+    # forward, fused bias + ReLU
+    y = G.run_conv_fwd(s, x, w, bias, B.ACT_RELU)
+    G.assert_parity(y, oracle.conv_fwd(s, x, w, bias, oracle.ACT_RELU), "fwd relu")
+    y = G.run_conv_fwd(s, x, w, None, B.ACT_NONE)
+    G.assert_parity(y, oracle.conv_fwd(s, x, w), "fwd plain")
+    # backward data, with and without the fused ReLU mask
+    dx = G.run_conv_bwd_data(s, dy, w, None)
+    G.assert_parity(dx, oracle.conv_bwd_data(s, dy, w), "bwd_data")
+    dx = G.run_conv_bwd_data(s, dy, w, x)
+    ref = oracle.conv_bwd_data(s, dy, w, x)
+    G.assert_parity(dx, ref, "bwd_data masked")
+    assert np.array_equal(dx == 0, ref == 0) or np.count_nonzero((dx == 0) != (ref == 0)) < 1e-4 * dx.size
+    # weight gradient: deterministic two-pass and atomic variants, with bias gradient
+    dw_ref, db_ref = oracle.conv_bwd_weights(s, x, dy, want_db=True)
+    dw, db = G.run_conv_bwd_weights(s, x, dy, True, deterministic=True)
+    G.assert_parity(dw, dw_ref, "bwd_weights")
+    G.assert_parity(db, db_ref, "dbias")
+    dw2, _ = G.run_conv_bwd_weights(s, x, dy, True, deterministic=True)
+    assert np.array_equal(dw, dw2), "two-pass weight gradient must be bitwise reproducible"
+    dw3, _ = G.run_conv_bwd_weights(s, x, dy, False, deterministic=False)
+    G.assert_parity(dw3, dw_ref, "bwd_weights atomics")
+
+
+def test_cfg1_with_sgd_update():
+    """Config 1 end to end: fwd, bwd_data, bwd_weights, then w <- w - 0.01*dw."""
+    import torch
+    import gpu_helpers as G
+    from paper_1602_06709_b200 import binding as B
+    from paper_1602_06709_b200 import inputs
+    c = inputs.CFG1
+    s = ConvShape(N=c["N"], C=c["C"], K=c["K"], H=c["H"], W=c["W"], R=c["R"], S=c["S"], pad_h=c["pad"], pad_w=c["pad"])
+    x, w, dy = inputs.conv_inputs("cfg1", "conv", s.N, s.C, s.H, s.W, s.K, s.R, s.S, s.P, s.Q, "unit")
+    bias = np.zeros(s.K, dtype=np.float32)
+    y = G.run_conv_fwd(s, x, w, bias, B.ACT_NONE)
+    G.assert_parity(y, oracle.conv_fwd(s, x, w, bias), "fwd")
+    dx = G.run_conv_bwd_data(s, dy, w, None)
+    G.assert_parity(dx, oracle.conv_bwd_data(s, dy, w), "bwd_data")
+    dw, _ = G.run_conv_bwd_weights(s, x, dy, False)
+    dw_ref = oracle.conv_bwd_weights(s, x, dy)
+    G.assert_parity(dw, dw_ref, "bwd_weights")
+    wt = G.dev(w)
+    B.sgd_update(wt, G.dev(dw), 0.01)
+    # the update itself is exact fp32 arithmetic on the GPU's own dw
+    ref = oracle.sgd_update(w, dw, 0.01)
+    np.testing.assert_allclose(wt.cpu().numpy(), ref, rtol=0, atol=1e-7)
+    G.assert_parity(wt.cpu().numpy(), oracle.sgd_update(w, dw_ref, 0.01), "updated weights")
