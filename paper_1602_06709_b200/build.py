@@ -12,7 +12,7 @@ SOURCES = ["pcl_api.cu", "tc_fprop.cu", "tc_wgrad.cu", "generic_conv.cu", "eleme
 HEADERS = ["pcl_internal.h", "pcl_ptx.cuh", os.path.join("..", "..", "include", "pcl_dnn.h")]
 NVCC = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
 FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
-         "-Xcompiler", "-fPIC", "--use_fast_math"]
+         "-Xcompiler", "-fPIC"]
 
 
 def needs_build() -> bool:

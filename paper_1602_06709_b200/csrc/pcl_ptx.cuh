@@ -70,6 +70,15 @@ __device__ __forceinline__ bool bounded_wait(uint64_t* bar, uint32_t parity, vol
     return false;
 }
 
+// Warp-uniform form: every lane polls, and the warp proceeds only if all lanes
+// saw the barrier complete (keeps .sync.aligned instructions convergent even on
+// the give-up path).
+__device__ __forceinline__ bool bounded_wait_warp(uint64_t* bar, uint32_t parity, volatile uint32_t* abort_flag,
+                                                  unsigned int* status_word, uint32_t code) {
+    const bool ok = bounded_wait(bar, parity, abort_flag, status_word, code);
+    return __all_sync(0xffffffffu, ok);
+}
+
 // ---------------------------------------------------------------------- TMA
 __device__ __forceinline__ void prefetch_tmap(const CUtensorMap* m) {
     asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(m)) : "memory");
@@ -140,21 +149,26 @@ __device__ __forceinline__ void tmem_ld_32x32(uint32_t taddr, uint32_t (&v)[32])
 }
 __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 
-// Shared-memory matrix descriptor (64-bit) for a 128-byte-swizzled operand tile.
+// Shared-memory matrix descriptor (64-bit) for a swizzled operand tile.
 //   bits  0-13 start address >> 4      bits 16-29 leading byte offset >> 4
 //   bits 32-45 stride byte offset >> 4 bits 46-47 descriptor version (1 on sm_100)
-//   bits 61-63 swizzle mode (2 = 128-byte)
-// K-major tile (rows of 128 B = 32 fp32 along the reduction): 8-row groups are
-// `sbo` bytes apart, the leading offset is unused.  MN-major tile (rows of 128 B
-// = 32 fp32 along M or N, one row per reduction index): 32-element column
-// groups are `lbo` bytes apart, 8-row reduction groups are `sbo` bytes apart.
-__device__ __forceinline__ uint64_t make_sw128_desc(uint32_t smem_addr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
+//   bits 61-63 swizzle mode: 2 = 128-byte rows swizzled in 16-byte chunks,
+//                            1 = 128-byte rows swizzled in 32-byte chunks
+// K-major tile (mode 2; rows of 128 B = 32 fp32 along the reduction): 8-row groups
+// are `sbo` bytes apart, the leading offset is unused.
+// MN-major tile of 32-bit elements (mode 1 is the only one the hardware takes for
+// tf32; rows of 128 B = 32 fp32 along M or N, one row per reduction index, the
+// swizzle pattern repeats every 4 rows): 32-element column groups are `lbo` bytes
+// apart, 4-row reduction groups are `sbo` bytes apart.
+constexpr uint32_t kSwizzle128B = 2, kSwizzle128B_Atom32B = 1;
+__device__ __forceinline__ uint64_t make_smem_desc(uint32_t smem_addr, uint32_t lbo_bytes, uint32_t sbo_bytes,
+                                                   uint32_t swizzle_mode) {
     uint64_t d = 0;
     d |= static_cast<uint64_t>((smem_addr & 0x3FFFFu) >> 4);
     d |= static_cast<uint64_t>((lbo_bytes >> 4) & 0x3FFFu) << 16;
     d |= static_cast<uint64_t>((sbo_bytes >> 4) & 0x3FFFu) << 32;
     d |= 1ull << 46;
-    d |= 2ull << 61;
+    d |= static_cast<uint64_t>(swizzle_mode) << 61;
     return d;
 }
 

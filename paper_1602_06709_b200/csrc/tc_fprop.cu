@@ -142,19 +142,19 @@ tc_fprop_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
         for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x, ++tile_cnt) {
             const int acc = tile_cnt & 1;
             const uint32_t acc_phase = (tile_cnt >> 1) & 1;
-            if (!bounded_wait(&tmem_empty_bar[acc], acc_phase ^ 1u, &abort_flag, p.status, WAIT_MMA_TMEM_EMPTY)) break;
+            if (!bounded_wait_warp(&tmem_empty_bar[acc], acc_phase ^ 1u, &abort_flag, p.status, WAIT_MMA_TMEM_EMPTY)) break;
             tc_fence_after();
             const uint32_t d_tmem = tmem_base + acc * p.BN;
             for (int kit = 0; kit < kiters; ++kit) {
-                if (!bounded_wait(&full_bar[stage], phase, &abort_flag, p.status, WAIT_MMA_FULL)) { ok = false; break; }
+                if (!bounded_wait_warp(&full_bar[stage], phase, &abort_flag, p.status, WAIT_MMA_FULL)) { ok = false; break; }
                 tc_fence_after();
                 if (lane == 0) {
                     const uint32_t a_addr = smem_u32(smem + stage * stage_bytes);
                     const uint32_t b_addr = a_addr + kABytes;
 #pragma unroll
                     for (int kk = 0; kk < 4; ++kk) {
-                        const uint64_t da = make_sw128_desc(a_addr + kk * 32, 16, 1024);
-                        const uint64_t db = make_sw128_desc(b_addr + kk * 32, 16, 1024);
+                        const uint64_t da = make_smem_desc(a_addr + kk * 32, 16, 1024, kSwizzle128B);
+                        const uint64_t db = make_smem_desc(b_addr + kk * 32, 16, 1024, kSwizzle128B);
                         umma_tf32(d_tmem, da, db, idesc, (kit | kk) != 0);
                     }
                     umma_commit(&empty_bar[stage]);
@@ -184,7 +184,7 @@ tc_fprop_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
             const int n = (m / p.tiles_p) * bn + in_;
             const bool valid = (q < p.Q) && (pp < p.P) && (n < p.N);
             const size_t pix = (static_cast<size_t>(n) * p.P + pp) * p.Q + q;
-            if (!bounded_wait(&tmem_full_bar[acc], acc_phase, &abort_flag, p.status, WAIT_EPI_TMEM_FULL)) break;
+            if (!bounded_wait_warp(&tmem_full_bar[acc], acc_phase, &abort_flag, p.status, WAIT_EPI_TMEM_FULL)) break;
             tc_fence_after();
             const uint32_t t_row = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + acc * p.BN;
             for (int ch = 0; ch < p.BN / 32; ++ch) {
@@ -330,14 +330,14 @@ int launch_tc_fprop(const TcFpropArgs& a, cudaStream_t st) {
         const uint64_t dims[4] = {uint64_t(a.Cin), uint64_t(a.W), uint64_t(a.H), uint64_t(a.N)};
         const uint64_t strides[3] = {uint64_t(a.Cin) * 4, uint64_t(a.W) * a.Cin * 4, uint64_t(a.H) * a.W * a.Cin * 4};
         const uint32_t box[4] = {kBlockC, uint32_t(bw), uint32_t(bh), uint32_t(bn)};
-        int rc = make_tmap(&tmA, a.in, 4, dims, strides, box);
+        int rc = make_tmap(&tmA, a.in, 4, dims, strides, box, false);
         if (rc != PCL_OK) return rc;
     }
     {
         const uint64_t dims[3] = {uint64_t(a.Cin), uint64_t(a.R) * a.S, uint64_t(a.Kout)};
         const uint64_t strides[2] = {uint64_t(a.Cin) * 4, uint64_t(a.R) * a.S * a.Cin * 4};
         const uint32_t box[3] = {kBlockC, 1, uint32_t(p.BN)};
-        int rc = make_tmap(&tmB, a.wt, 3, dims, strides, box);
+        int rc = make_tmap(&tmB, a.wt, 3, dims, strides, box, false);
         if (rc != PCL_OK) return rc;
     }
     const long total = m_tiles * p.tiles_k;

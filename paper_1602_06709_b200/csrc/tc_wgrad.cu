@@ -5,8 +5,9 @@
 // GEMM view per tap (r, s): M = K output maps, N = C input maps, reduction over
 // the N*P*Q output pixels.  The reduction index is the OUTER dimension of both
 // NHWC tensors, so both operands are "MN-major": a TMA box {32 maps, 32 pixels}
-// lands in shared memory as 32 rows (one per pixel) of 128 bytes, which is the
-// 128-byte-swizzled MN-major operand layout of tcgen05.mma.  The x box is the
+// lands in shared memory as 32 rows (one per pixel) of 128 bytes, swizzled in
+// 32-byte chunks, which is the MN-major operand layout tcgen05.mma takes for
+// 32-bit elements.  The x box is the
 // dy box shifted by the tap, with zero padding supplied by TMA's out-of-bounds
 // fill.
 //
@@ -130,16 +131,16 @@ tc_wgrad_kernel(const __grid_constant__ CUtensorMap tmDy, const __grid_constant_
         uint32_t phase = 0;
         bool ok = true;
         for (int kit = 0; kit < kiters; ++kit) {
-            if (!bounded_wait(&full_bar[stage], phase, &abort_flag, p.status, WAIT_MMA_FULL)) { ok = false; break; }
+            if (!bounded_wait_warp(&full_bar[stage], phase, &abort_flag, p.status, WAIT_MMA_FULL)) { ok = false; break; }
             tc_fence_after();
             if (lane == 0) {
                 const uint32_t a_addr = smem_u32(smem + stage * stage_bytes);
                 const uint32_t b_addr = a_addr + kABytes;
 #pragma unroll
                 for (int kk = 0; kk < kPix / 8; ++kk) {
-                    // 8 pixels per instruction = one 1024-byte group of 8 rows
-                    const uint64_t da = make_sw128_desc(a_addr + kk * 1024, kGroupBytes, 1024);
-                    const uint64_t db = make_sw128_desc(b_addr + kk * 1024, kGroupBytes, 1024);
+                    // 8 pixels per instruction = two 512-byte groups of 4 rows
+                    const uint64_t da = make_smem_desc(a_addr + kk * 1024, kGroupBytes, 512, kSwizzle128B_Atom32B);
+                    const uint64_t db = make_smem_desc(b_addr + kk * 1024, kGroupBytes, 512, kSwizzle128B_Atom32B);
                     umma_tf32(tmem_base, da, db, idesc, (kit | kk) != 0);
                 }
                 umma_commit(&empty_bar[stage]);
@@ -154,7 +155,7 @@ tc_wgrad_kernel(const __grid_constant__ CUtensorMap tmDy, const __grid_constant_
         const int k = kt * 128 + quarter * 32 + lane;
         const bool valid = k < p.K;
         const bool vec_ok = (p.C & 3) == 0;
-        if (bounded_wait(&tmem_full_bar, 0, &abort_flag, p.status, WAIT_EPI_TMEM_FULL)) {
+        if (bounded_wait_warp(&tmem_full_bar, 0, &abort_flag, p.status, WAIT_EPI_TMEM_FULL)) {
             tc_fence_after();
             const uint32_t t_row = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16);
             float* base = p.out + static_cast<size_t>(split) * p.split_stride +
@@ -308,14 +309,14 @@ int launch_tc_wgrad(const TcWgradArgs& a, cudaStream_t st) {
         const uint64_t dims[4] = {uint64_t(a.K), uint64_t(a.Q), uint64_t(a.P), uint64_t(a.N)};
         const uint64_t strides[3] = {uint64_t(a.K) * 4, uint64_t(a.Q) * a.K * 4, uint64_t(a.P) * a.Q * a.K * 4};
         const uint32_t box[4] = {32, uint32_t(bw), uint32_t(bh), uint32_t(bn)};
-        int rc = make_tmap(&tmDy, a.dy, 4, dims, strides, box);
+        int rc = make_tmap(&tmDy, a.dy, 4, dims, strides, box, true);
         if (rc != PCL_OK) return rc;
     }
     {
         const uint64_t dims[4] = {uint64_t(a.C), uint64_t(a.W), uint64_t(a.H), uint64_t(a.N)};
         const uint64_t strides[3] = {uint64_t(a.C) * 4, uint64_t(a.W) * a.C * 4, uint64_t(a.H) * a.W * a.C * 4};
         const uint32_t box[4] = {32, uint32_t(bw), uint32_t(bh), uint32_t(bn)};
-        int rc = make_tmap(&tmX, a.x, 4, dims, strides, box);
+        int rc = make_tmap(&tmX, a.x, 4, dims, strides, box, true);
         if (rc != PCL_OK) return rc;
     }
     const long items = long(p.k_tiles) * a.R * a.S * p.c_tiles * p.splits;
