@@ -62,7 +62,7 @@ int make_tmap(CUtensorMap* out, const void* base, int rank, const uint64_t* dims
         if (strides_bytes[i] % 16 != 0 || strides_bytes[i] >= (1ull << 40)) return PCL_ERR_UNSUPPORTED_SHAPE;
     }
     if (reinterpret_cast<uintptr_t>(base) & 15) return PCL_ERR_MISALIGNED;
-    const CUresult r = enc(out, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, cuuint32_t(rank), const_cast<void*>(base), gdim, gstr,
+    const CUresult r = enc(out, CU_TENSOR_MAP_DATA_TYPE_TFLOAT32, cuuint32_t(rank), const_cast<void*>(base), gdim, gstr,
                            gbox, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
                            atom32 ? CU_TENSOR_MAP_SWIZZLE_128B_ATOM_32B : CU_TENSOR_MAP_SWIZZLE_128B,
                            CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);

@@ -1,0 +1,246 @@
+"""Step drivers for the two topologies the workloads name: the VGG-A CNN and
+the 7-layer fully-connected DNN (Sec. 5).  A driver only owns device buffers
+and calls the C ABI in order; all arithmetic happens in the library's kernels.
+
+Per layer the backward pass computes the weight gradient first and the
+backpropagated gradient second, and the first layer skips backpropagation
+(Sec. 3.1).  Parameters and their gradients live in two flat buffers so that
+the SGD update of the whole model is one kernel launch.
+"""
+from __future__ import annotations
+
+from dataclasses import dataclass
+from typing import List, Optional
+
+import numpy as np
+import torch
+
+from . import binding as B
+from . import inputs
+
+
+def _align(n: int, a: int = 64) -> int:
+    return (n + a - 1) // a * a
+
+
+class _ParamStore:
+    """Flat fp32 parameter and gradient buffers with 256-byte aligned views."""
+
+    def __init__(self, shapes: List[tuple]):
+        self.offsets = []
+        off = 0
+        for shp in shapes:
+            self.offsets.append(off)
+            off += _align(int(np.prod(shp)))
+        self.total = off
+        self.shapes = shapes
+        self.params = torch.zeros(off, device="cuda")
+        self.grads = torch.zeros(off, device="cuda")
+
+    def view(self, buf, i):
+        n = int(np.prod(self.shapes[i]))
+        return buf[self.offsets[i]:self.offsets[i] + n].view(self.shapes[i])
+
+    def p(self, i):
+        return self.view(self.params, i)
+
+    def g(self, i):
+        return self.view(self.grads, i)
+
+    def n_real(self) -> int:
+        return sum(int(np.prod(s)) for s in self.shapes)
+
+
+@dataclass
+class _ConvLayer:
+    name: str
+    C: int
+    K: int
+    H: int
+    W: int
+    pool: bool
+    desc: object = None
+
+
+class VggA:
+    """VGG configuration A: eight 3x3 pad-1 convolutions (64,128,256,256,512,512,
+    512,512) each followed by ReLU, 2x2 max-pool after conv 1,2,4,6,8, then
+    FC 25088-4096-4096-1000 and softmax cross-entropy."""
+
+    def __init__(self, N: int, hw: int = inputs.VGGA_HW, conv=None, fc=None, classes: int = inputs.VGGA_CLASSES,
+                 lr: float = 0.01, cfg: str = "cfg5"):
+        self.N, self.lr, self.classes = N, lr, classes
+        conv = conv if conv is not None else inputs.VGGA_CONV
+        self.convs: List[_ConvLayer] = []
+        h = hw
+        for name, C, K, pool in conv:
+            L = _ConvLayer(name, C, K, h, h, pool)
+            L.desc = B.conv_desc(N, C, K, h, h, 3, 3, 1, 1)
+            self.convs.append(L)
+            if pool:
+                h //= 2
+        self.flat = self.convs[-1].K * h * h
+        if fc is None:
+            fc = [(self.flat, 4096), (4096, 4096), (4096, classes)]
+        assert fc[0][0] == self.flat and fc[-1][1] == classes
+        self.fcs = fc
+        shapes = []
+        for L in self.convs:
+            shapes += [(L.K, 3, 3, L.C), (L.K,)]
+        for C, K in fc:
+            shapes += [(K, C), (K,)]
+        self.store = _ParamStore(shapes)
+        nconv = len(self.convs)
+        for i, L in enumerate(self.convs):
+            w = inputs.he_normal_conv(inputs.tensor_id(cfg, L.name, "w"), L.K, 3, 3, L.C)
+            self.store.p(2 * i).copy_(torch.from_numpy(w))
+        for j, (C, K) in enumerate(fc):
+            w = inputs.he_normal_fc(inputs.tensor_id(cfg, f"fc{j + 1}", "w"), K, C)
+            self.store.p(2 * (nconv + j)).copy_(torch.from_numpy(w))
+        # activations and gradients
+        dev = "cuda"
+        self.x = torch.empty(N, hw, hw, self.convs[0].C, device=dev)
+        self.y = [torch.empty(N, L.H, L.W, L.K, device=dev) for L in self.convs]           # post-ReLU
+        self.pooled = [torch.empty(N, L.H // 2, L.W // 2, L.K, device=dev) if L.pool else None for L in self.convs]
+        self.dy = [torch.empty(N, L.H, L.W, L.K, device=dev) for L in self.convs]           # grad wrt pre-activation
+        self.dpooled = [torch.empty(N, L.H // 2, L.W // 2, L.K, device=dev) if L.pool else None for L in self.convs]
+        self.fc_out = [torch.empty(N, K, device=dev) for _, K in fc]
+        self.fc_dout = [torch.empty(N, K, device=dev) for _, K in fc]
+        self.labels = torch.zeros(N, dtype=torch.int32, device=dev)
+        self.loss = torch.zeros(1, device=dev)
+        ws = 0
+        for L in self.convs:
+            ws = max(ws, B.conv_workspace_bytes(L.desc, B.PASS_BWD_DATA), B.conv_workspace_bytes(L.desc, B.PASS_BWD_WEIGHTS))
+        for C, K in fc:
+            ws = max(ws, B.fc_workspace_bytes(N, C, K, B.PASS_BWD_DATA))
+        self.ws = torch.empty(max(ws, 256), dtype=torch.uint8, device=dev)
+        self.conv_flops_fwd = [2 * N * L.K * L.H * L.W * L.C * 9 for L in self.convs]
+        self.fc_flops_fwd = [2 * N * C * K for C, K in fc]
+
+    # -- parameters ---------------------------------------------------------
+    def conv_w(self, i): return self.store.p(2 * i)
+    def conv_b(self, i): return self.store.p(2 * i + 1)
+    def conv_dw(self, i): return self.store.g(2 * i)
+    def conv_db(self, i): return self.store.g(2 * i + 1)
+    def fc_w(self, j): return self.store.p(2 * (len(self.convs) + j))
+    def fc_b(self, j): return self.store.p(2 * (len(self.convs) + j) + 1)
+    def fc_dw(self, j): return self.store.g(2 * (len(self.convs) + j))
+    def fc_db(self, j): return self.store.g(2 * (len(self.convs) + j) + 1)
+
+    def layer_input(self, i):
+        if i == 0:
+            return self.x
+        prev = self.convs[i - 1]
+        return self.pooled[i - 1] if prev.pool else self.y[i - 1]
+
+    # -- one training step --------------------------------------------------
+    def forward(self):
+        for i, L in enumerate(self.convs):
+            B.conv_fwd(L.desc, self.layer_input(i), self.conv_w(i), self.conv_b(i), self.y[i], B.ACT_RELU, self.ws)
+            if L.pool:
+                B.maxpool2x2_fwd(self.N, L.H, L.W, L.K, self.y[i], self.pooled[i])
+        a = self.pooled[-1].view(self.N, self.flat)
+        for j, (C, K) in enumerate(self.fcs):
+            act = B.ACT_RELU if j + 1 < len(self.fcs) else B.ACT_NONE
+            B.fc_fwd(self.N, C, K, a, self.fc_w(j), self.fc_b(j), self.fc_out[j], act)
+            a = self.fc_out[j]
+        B.softmax_xent(self.N, self.classes, self.fc_out[-1], self.labels, self.loss, self.fc_dout[-1])
+
+    def backward(self):
+        nfc = len(self.fcs)
+        for j in reversed(range(nfc)):
+            C, K = self.fcs[j]
+            a = self.fc_out[j - 1] if j > 0 else self.pooled[-1].view(self.N, self.flat)
+            dx = self.fc_dout[j - 1] if j > 0 else self.dpooled[-1].view(self.N, self.flat)
+            act = B.ACT_RELU if j + 1 < nfc else B.ACT_NONE
+            B.fc_bwd(self.N, C, K, a, self.fc_w(j), self.fc_out[j], act, self.fc_dout[j], dx, self.fc_dw(j),
+                     self.fc_db(j), self.ws)
+        for i in reversed(range(len(self.convs))):
+            L = self.convs[i]
+            if L.pool:   # gradient through the pool, then through the ReLU (fused mask)
+                B.maxpool2x2_bwd(self.N, L.H, L.W, L.K, self.y[i], self.dpooled[i], self.y[i], self.dy[i])
+            B.conv_bwd_weights(L.desc, self.layer_input(i), self.dy[i], self.conv_dw(i), self.conv_db(i), True, self.ws)
+            if i > 0:
+                prev = self.convs[i - 1]
+                if prev.pool:
+                    B.conv_bwd_data(L.desc, self.dy[i], self.conv_w(i), None, self.dpooled[i - 1], self.ws)
+                else:   # the layer's input is the previous ReLU output: fuse its mask
+                    B.conv_bwd_data(L.desc, self.dy[i], self.conv_w(i), self.y[i - 1], self.dy[i - 1], self.ws)
+
+    def update(self):
+        B.sgd_update(self.store.params, self.store.grads, self.lr)
+
+    def step(self):
+        self.forward()
+        self.backward()
+        self.update()
+
+    def step_from_host(self, x_host: torch.Tensor, labels_host: torch.Tensor) -> float:
+        """The call a user makes: pinned host minibatch in, loss out."""
+        self.x.copy_(x_host, non_blocking=True)
+        self.labels.copy_(labels_host, non_blocking=True)
+        self.step()
+        return float(self.loss.cpu().item())
+
+
+class Dnn:
+    """Fully-connected DNN: dims[0] inputs, sigmoid hidden layers, linear output
+    layer with softmax cross-entropy (the 7-layer ASR network shape of Sec. 5.4)."""
+
+    def __init__(self, N: int, dims=None, lr: float = 0.01, cfg: str = "cfg4"):
+        dims = dims if dims is not None else inputs.CFG4_DIMS
+        self.N, self.dims, self.lr = N, dims, lr
+        self.layers = list(zip(dims[:-1], dims[1:]))
+        shapes = []
+        for C, K in self.layers:
+            shapes += [(K, C), (K,)]
+        self.store = _ParamStore(shapes)
+        for j, (C, K) in enumerate(self.layers):
+            w = inputs.xavier_uniform_fc(inputs.tensor_id(cfg, f"fc{j + 1}", "w"), K, C)
+            self.store.p(2 * j).copy_(torch.from_numpy(w))
+        dev = "cuda"
+        self.x = torch.empty(N, dims[0], device=dev)
+        self.out = [torch.empty(N, K, device=dev) for _, K in self.layers]
+        self.dout = [torch.empty(N, K, device=dev) for _, K in self.layers]
+        self.labels = torch.zeros(N, dtype=torch.int32, device=dev)
+        self.loss = torch.zeros(1, device=dev)
+        ws = max(B.fc_workspace_bytes(N, C, K, B.PASS_BWD_DATA) for C, K in self.layers)
+        self.ws = torch.empty(max(ws, 256), dtype=torch.uint8, device=dev)
+        self.fc_flops_fwd = [2 * N * C * K for C, K in self.layers]
+
+    def w(self, j): return self.store.p(2 * j)
+    def b(self, j): return self.store.p(2 * j + 1)
+    def dw(self, j): return self.store.g(2 * j)
+    def db(self, j): return self.store.g(2 * j + 1)
+
+    def forward(self):
+        a = self.x
+        n = len(self.layers)
+        for j, (C, K) in enumerate(self.layers):
+            act = B.ACT_SIGMOID if j + 1 < n else B.ACT_NONE
+            B.fc_fwd(self.N, C, K, a, self.w(j), self.b(j), self.out[j], act)
+            a = self.out[j]
+        B.softmax_xent(self.N, self.dims[-1], self.out[-1], self.labels, self.loss, self.dout[-1])
+
+    def backward(self):
+        n = len(self.layers)
+        for j in reversed(range(n)):
+            C, K = self.layers[j]
+            a = self.out[j - 1] if j > 0 else self.x
+            dx = self.dout[j - 1] if j > 0 else None          # first layer: no backpropagation
+            act = B.ACT_SIGMOID if j + 1 < n else B.ACT_NONE
+            B.fc_bwd(self.N, C, K, a, self.w(j), self.out[j], act, self.dout[j], dx, self.dw(j), self.db(j), self.ws)
+
+    def update(self):
+        B.sgd_update(self.store.params, self.store.grads, self.lr)
+
+    def step(self):
+        self.forward()
+        self.backward()
+        self.update()
+
+    def step_from_host(self, x_host, labels_host) -> float:
+        self.x.copy_(x_host, non_blocking=True)
+        self.labels.copy_(labels_host, non_blocking=True)
+        self.step()
+        return float(self.loss.cpu().item())

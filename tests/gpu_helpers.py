@@ -63,3 +63,165 @@ def run_conv_bwd_weights(s, x, dy, want_db, deterministic=True):
                        workspace(B.conv_workspace_bytes(d, B.PASS_BWD_WEIGHTS)))
     B.check_device_status()
     return dw.cpu().numpy(), (db.cpu().numpy() if want_db else None)
+
+
+# ---------------------------------------------------------------------------
+# Per-call verification of a whole training step: every library call of the
+# step is re-computed by the oracle from the inputs the GPU call actually
+# received (copied back from the device) and compared with what the GPU call
+# wrote.  `samples` > 0 checks that many randomly chosen output elements per
+# tensor (for sizes where the full oracle would take too long); 0 checks all.
+# ---------------------------------------------------------------------------
+def _cmp(got_t, ref_fn, size, samples, rng, what, report):
+    got = got_t.detach().cpu().numpy().reshape(-1)
+    if samples and size > samples:
+        idx = np.sort(rng.choice(size, size=samples, replace=False)).astype(np.int64)
+        ref = ref_fn(idx)
+        g = got[idx]
+    else:
+        ref = ref_fn(None).reshape(-1)
+        g = got
+    rel, mx = oracle.parity_errors(g, ref)
+    report.append((what, rel, mx))
+    assert rel <= REL_L2_TOL and mx <= MAX_OVER_RMS_TOL, f"{what}: rel_l2={rel:.3e} max/rms={mx:.3e}"
+
+
+def verify_vgg_step(net, params_before, samples=0, seed=0):
+    """net: VggA after exactly one step(); params_before: flat params (numpy) before the step."""
+    rng = np.random.default_rng(seed)
+    report = []
+    N = net.N
+    st = net.store
+
+    def pview(i):
+        n = int(np.prod(st.shapes[i]))
+        return params_before[st.offsets[i]:st.offsets[i] + n].reshape(st.shapes[i])
+
+    host = lambda t: t.detach().cpu().numpy()
+    nconv = len(net.convs)
+    # forward convolutions and pools
+    for i, L in enumerate(net.convs):
+        s = ConvShape(N=N, C=L.C, K=L.K, H=L.H, W=L.W, R=3, S=3, pad_h=1, pad_w=1)
+        xin = host(net.layer_input(i)); w = pview(2 * i); b = pview(2 * i + 1)
+        _cmp(net.y[i], lambda at: oracle.conv_fwd(s, xin, w, b, oracle.ACT_RELU, at=at), net.y[i].numel(), samples,
+             rng, f"{L.name} fwd", report)
+        if L.pool:
+            y = host(net.y[i])
+            assert np.array_equal(host(net.pooled[i]), oracle.maxpool2x2_fwd(y).astype(np.float32)), f"{L.name} pool"
+    # forward FC
+    a = host(net.pooled[-1]).reshape(N, net.flat)
+    for j, (C, K) in enumerate(net.fcs):
+        act = oracle.ACT_RELU if j + 1 < len(net.fcs) else oracle.ACT_NONE
+        w = pview(2 * (nconv + j)); b = pview(2 * (nconv + j) + 1)
+        s = ConvShape(N=N, C=C, K=K, H=1, W=1, R=1, S=1)
+        a_in = a
+        _cmp(net.fc_out[j], lambda at: oracle.conv_fwd(s, a_in, w, b, act, at=at), N * K, samples, rng,
+             f"fc{j + 1} fwd", report)
+        a = host(net.fc_out[j])
+    # loss
+    loss_ref, dlog_ref = oracle.softmax_xent(a, host(net.labels))
+    assert abs(net.loss.item() - loss_ref) <= 1e-5 * max(1.0, abs(loss_ref))
+    # backward FC (fc_dout[j] now holds dz_j; the incoming dy is not kept, so check dz of the last layer only
+    # against the loss gradient and the contractions against the GPU's own dz)
+    rel, mx = oracle.parity_errors(host(net.fc_dout[-1]), dlog_ref)
+    assert rel <= REL_L2_TOL and mx <= MAX_OVER_RMS_TOL
+    for j in reversed(range(len(net.fcs))):
+        C, K = net.fcs[j]
+        s = ConvShape(N=N, C=C, K=K, H=1, W=1, R=1, S=1)
+        dz = host(net.fc_dout[j])
+        a_in = host(net.fc_out[j - 1]) if j > 0 else host(net.pooled[-1]).reshape(N, net.flat)
+        w = pview(2 * (nconv + j))
+        _cmp(net.fc_dw(j), lambda at: oracle.conv_bwd_weights(s, a_in, dz, at=at), K * C, samples, rng,
+             f"fc{j + 1} dw", report)
+        db_ref = dz.astype(np.float64).sum(axis=0)
+        rel, mx = oracle.parity_errors(host(net.fc_db(j)), db_ref)
+        assert rel <= REL_L2_TOL and mx <= MAX_OVER_RMS_TOL, f"fc{j + 1} db"
+        # dx of layer j is the dy of layer j-1 before its activation gradient was applied in place; for j == 0 it
+        # is kept in dpooled[-1]
+        if j == 0:
+            _cmp(net.dpooled[-1], lambda at: oracle.conv_bwd_data(s, dz, w, at=at), N * C, samples, rng,
+                 "fc1 dx", report)
+        else:
+            # fc_dout[j-1] = dx_j * act'(out_{j-1}): re-apply the activation gradient to the oracle's dx
+            out_prev = host(net.fc_out[j - 1]).reshape(-1)
+
+            def ref_fn(at, s=s, dz=dz, w=w, out_prev=out_prev):
+                if at is None:
+                    dx = oracle.conv_bwd_data(s, dz, w).reshape(-1)
+                    return np.where(out_prev > 0, dx, 0.0)
+                dx = oracle.conv_bwd_data(s, dz, w, at=at)
+                return np.where(out_prev[at] > 0, dx, 0.0)
+            _cmp(net.fc_dout[j - 1], ref_fn, N * C, samples, rng, f"fc{j + 1} dx (masked)", report)
+    # backward convolutions
+    for i in reversed(range(nconv)):
+        L = net.convs[i]
+        s = ConvShape(N=N, C=L.C, K=L.K, H=L.H, W=L.W, R=3, S=3, pad_h=1, pad_w=1)
+        if L.pool:
+            y = host(net.y[i]); dp = host(net.dpooled[i])
+            assert np.array_equal(host(net.dy[i]), oracle.maxpool2x2_bwd(y, dp, y).astype(np.float32)), f"{L.name} pool bwd"
+        dz = host(net.dy[i]); xin = host(net.layer_input(i)); w = pview(2 * i)
+        _cmp(net.conv_dw(i), lambda at: oracle.conv_bwd_weights(s, xin, dz, at=at), net.conv_dw(i).numel(), samples,
+             rng, f"{L.name} dw", report)
+        db_ref = dz.reshape(-1, L.K).astype(np.float64).sum(axis=0)
+        rel, mx = oracle.parity_errors(host(net.conv_db(i)), db_ref)
+        assert rel <= REL_L2_TOL and mx <= MAX_OVER_RMS_TOL, f"{L.name} db"
+        if i > 0:
+            prev = net.convs[i - 1]
+            if prev.pool:
+                _cmp(net.dpooled[i - 1], lambda at: oracle.conv_bwd_data(s, dz, w, None, at=at),
+                     net.dpooled[i - 1].numel(), samples, rng, f"{L.name} dx", report)
+            else:
+                mask = host(net.y[i - 1])
+                _cmp(net.dy[i - 1], lambda at: oracle.conv_bwd_data(s, dz, w, mask, at=at), net.dy[i - 1].numel(),
+                     samples, rng, f"{L.name} dx (masked)", report)
+    # SGD update of every parameter, against the GPU's own gradients
+    grads = host(st.grads); after = host(st.params)
+    ref = oracle.sgd_update(params_before, grads, net.lr)
+    np.testing.assert_allclose(after, ref, rtol=0, atol=1e-6 * max(1.0, float(np.abs(ref).max())))
+    return report
+
+
+def verify_dnn_step(net, params_before, samples=0, seed=0):
+    rng = np.random.default_rng(seed)
+    report = []
+    N = net.N
+    st = net.store
+    host = lambda t: t.detach().cpu().numpy()
+
+    def pview(i):
+        n = int(np.prod(st.shapes[i]))
+        return params_before[st.offsets[i]:st.offsets[i] + n].reshape(st.shapes[i])
+
+    n = len(net.layers)
+    a = host(net.x)
+    for j, (C, K) in enumerate(net.layers):
+        act = oracle.ACT_SIGMOID if j + 1 < n else oracle.ACT_NONE
+        s = ConvShape(N=N, C=C, K=K, H=1, W=1, R=1, S=1)
+        w = pview(2 * j); b = pview(2 * j + 1); a_in = a
+        _cmp(net.out[j], lambda at: oracle.conv_fwd(s, a_in, w, b, act, at=at), N * K, samples, rng, f"fc{j + 1} fwd",
+             report)
+        a = host(net.out[j])
+    loss_ref, dlog_ref = oracle.softmax_xent(a, host(net.labels))
+    assert abs(net.loss.item() - loss_ref) <= 1e-5 * max(1.0, abs(loss_ref))
+    rel, mx = oracle.parity_errors(host(net.dout[-1]), dlog_ref)
+    assert rel <= REL_L2_TOL and mx <= MAX_OVER_RMS_TOL
+    for j in reversed(range(n)):
+        C, K = net.layers[j]
+        s = ConvShape(N=N, C=C, K=K, H=1, W=1, R=1, S=1)
+        dz = host(net.dout[j]); a_in = host(net.out[j - 1]) if j > 0 else host(net.x); w = pview(2 * j)
+        _cmp(net.dw(j), lambda at: oracle.conv_bwd_weights(s, a_in, dz, at=at), K * C, samples, rng, f"fc{j + 1} dw",
+             report)
+        rel, mx = oracle.parity_errors(host(net.db(j)), dz.astype(np.float64).sum(axis=0))
+        assert rel <= REL_L2_TOL and mx <= MAX_OVER_RMS_TOL, f"fc{j + 1} db"
+        if j > 0:
+            out_prev = host(net.out[j - 1]).reshape(-1).astype(np.float64)
+
+            def ref_fn(at, s=s, dz=dz, w=w, out_prev=out_prev):
+                if at is None:
+                    return oracle.conv_bwd_data(s, dz, w).reshape(-1) * out_prev * (1.0 - out_prev)
+                return oracle.conv_bwd_data(s, dz, w, at=at) * out_prev[at] * (1.0 - out_prev[at])
+            _cmp(net.dout[j - 1], ref_fn, N * C, samples, rng, f"fc{j + 1} dx (times sigmoid')", report)
+    grads = host(st.grads); after = host(st.params)
+    ref = oracle.sgd_update(params_before, grads, net.lr)
+    np.testing.assert_allclose(after, ref, rtol=0, atol=1e-6 * max(1.0, float(np.abs(ref).max())))
+    return report

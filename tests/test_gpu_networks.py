@@ -1,0 +1,83 @@
+"""GPU parity of whole training steps (VGG-A-shaped CNN, sigmoid DNN): every
+library call inside the step is checked against the oracle on the inputs that
+call received.  Small versions are checked element by element; the full-size
+workloads are checked on sampled outputs."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import oracle.networks as ON
+
+pytestmark = pytest.mark.gpu
+
+SMALL_CONV = [("conv1", 3, 8, True), ("conv2", 8, 16, True), ("conv3", 16, 32, False), ("conv4", 32, 32, True),
+              ("conv5", 32, 64, False), ("conv6", 64, 64, True), ("conv7", 64, 64, False), ("conv8", 64, 64, True)]
+
+
+def _randomise_biases(net, scale=0.1):
+    from paper_1602_06709_b200 import inputs
+    for i, shp in enumerate(net.store.shapes):
+        if len(shp) == 1:
+            b = inputs.uniform(inputs.tensor_id("bias", i), shp, -scale, scale)
+            net.store.p(i).copy_(torch.from_numpy(b))
+
+
+def _small_vgg(N=4, hw=32):
+    from paper_1602_06709_b200 import inputs, networks
+    net = networks.VggA(N, hw=hw, conv=SMALL_CONV, fc=[(64, 128), (128, 128), (128, 10)], classes=10, cfg="small")
+    _randomise_biases(net)
+    x = inputs.uniform(inputs.tensor_id("small", "x"), (N, hw, hw, 3), 0.0, 1.0)
+    lab = inputs.labels(inputs.tensor_id("small", "labels"), N, 10)
+    net.x.copy_(torch.from_numpy(x)); net.labels.copy_(torch.from_numpy(lab))
+    return net, x, lab
+
+
+def test_small_vgg_step_per_call():
+    import gpu_helpers as G
+    from paper_1602_06709_b200 import binding as B
+    net, x, lab = _small_vgg()
+    before = net.store.params.cpu().numpy().copy()
+    net.step()
+    B.check_device_status()
+    report = G.verify_vgg_step(net, before, samples=0)
+    assert len(report) >= 8 + 3 + 3 + 3 + 8 + 7
+
+
+def test_small_vgg_step_end_to_end_against_chained_oracle():
+    """Information-level check of the whole chain (TF32 truncation compounds over
+    11 layers, so the bound is looser than the per-call bar)."""
+    from paper_1602_06709_b200 import binding as B
+    net, x, lab = _small_vgg()
+    st = net.store
+    conv_params = [(net.conv_w(i).cpu().numpy(), net.conv_b(i).cpu().numpy()) for i in range(8)]
+    fc_params = [(net.fc_w(j).cpu().numpy(), net.fc_b(j).cpu().numpy()) for j in range(3)]
+    net.step()
+    B.check_device_status()
+    ref = ON.vgga_step(x, lab, conv_params, fc_params, [(c, k, p) for _, c, k, p in SMALL_CONV], net.lr)
+    assert abs(net.loss.item() - ref["loss"]) <= 2e-2 * abs(ref["loss"])
+    rel, _ = oracle.parity_errors(net.fc_out[-1].cpu().numpy(), ref["logits"])
+    assert rel < 3e-2
+    rel, _ = oracle.parity_errors(net.conv_dw(0).cpu().numpy(), ref["conv_grads"][0][0])
+    assert rel < 1e-1
+    rel, _ = oracle.parity_errors(net.conv_w(7).cpu().numpy(), ref["conv_params"][7][0])
+    assert rel < 1e-3
+
+
+def test_small_dnn_step_per_call():
+    import gpu_helpers as G
+    from paper_1602_06709_b200 import binding as B
+    from paper_1602_06709_b200 import inputs, networks
+    N, dims = 96, [44, 160, 160, 72]
+    net = networks.Dnn(N, dims=dims, cfg="small_dnn")
+    _randomise_biases(net)
+    x = inputs.normal(inputs.tensor_id("small_dnn", "x"), (N, dims[0]), 1.0)
+    lab = inputs.labels(inputs.tensor_id("small_dnn", "labels"), N, dims[-1])
+    net.x.copy_(torch.from_numpy(x)); net.labels.copy_(torch.from_numpy(lab))
+    params = [(net.w(j).cpu().numpy(), net.b(j).cpu().numpy()) for j in range(3)]
+    before = net.store.params.cpu().numpy().copy()
+    net.step()
+    B.check_device_status()
+    G.verify_dnn_step(net, before, samples=0)
+    ref = ON.dnn_step(x, lab, params, net.lr)
+    assert abs(net.loss.item() - ref["loss"]) <= 1e-2 * abs(ref["loss"])
