@@ -149,6 +149,23 @@ int pcl_last_device_status(void* cuda_stream);
 /* Number of kernels this library has launched since it was loaded. */
 unsigned long long pcl_launch_count(void);
 
+/* Optional per-kernel timing (the paper has no counterpart; measurement aid).
+ * Between pcl_profile_begin() and pcl_profile_end() every kernel launch of the
+ * library is bracketed by two CUDA events on its launching stream.
+ * pcl_profile_end() waits for those events, stops the bracketing and returns, per
+ * kernel family that ran, the number of launches, the summed event time and the
+ * summed algorithmic work (flops for the contraction kernels, bytes for the
+ * memory-bound ones).  stats: HOST array of max_stats entries; *n_stats entries
+ * are filled.  Event objects are created on first use and reused. */
+typedef struct {
+    char name[32];
+    unsigned long long launches;
+    double total_ms;
+    double work;
+} pcl_kernel_stat;
+int pcl_profile_begin(void);
+int pcl_profile_end(pcl_kernel_stat* stats, int max_stats, int* n_stats);
+
 const char* pcl_status_string(int status);
 
 #ifdef __cplusplus

@@ -24,7 +24,7 @@ EXPORTS = [
     "pcl_set_path", "pcl_conv_out_dims", "pcl_conv_workspace_bytes", "pcl_fc_workspace_bytes",
     "pcl_conv_fwd", "pcl_conv_bwd_data", "pcl_conv_bwd_weights", "pcl_fc_fwd", "pcl_fc_bwd",
     "pcl_sgd_update", "pcl_maxpool2x2_fwd", "pcl_maxpool2x2_bwd", "pcl_softmax_xent",
-    "pcl_last_device_status", "pcl_launch_count", "pcl_status_string",
+    "pcl_last_device_status", "pcl_launch_count", "pcl_status_string", "pcl_profile_begin", "pcl_profile_end",
 ]
 
 
@@ -32,6 +32,11 @@ class PclError(RuntimeError):
     def __init__(self, code: int, where: str):
         self.code = code
         super().__init__(f"{where}: {status_string(code)} (status {code})")
+
+
+class KernelStat(ctypes.Structure):
+    _fields_ = [("name", ctypes.c_char * 32), ("launches", ctypes.c_ulonglong), ("total_ms", ctypes.c_double),
+                ("work", ctypes.c_double)]
 
 
 class ConvDesc(ctypes.Structure):
@@ -69,6 +74,7 @@ def lib() -> ctypes.CDLL:
         L.pcl_softmax_xent.argtypes = [ci, ci, vp, vp, vp, vp, vp]
         L.pcl_last_device_status.argtypes = [vp]
         L.pcl_launch_count.restype = ctypes.c_ulonglong
+        L.pcl_profile_end.argtypes = [ctypes.POINTER(KernelStat), ci, ctypes.POINTER(ci)]
         L.pcl_status_string.argtypes = [ci]
         L.pcl_status_string.restype = ctypes.c_char_p
         _lib = L
@@ -184,3 +190,16 @@ def check_device_status(stream=None):
 
 def launch_count() -> int:
     return int(lib().pcl_launch_count())
+
+
+def profile_begin():
+    _check(lib().pcl_profile_begin(), "pcl_profile_begin")
+
+
+def profile_end():
+    """Returns {kernel name: dict(launches, total_ms, work)} for the kernels that ran since profile_begin()."""
+    arr = (KernelStat * 32)()
+    n = ctypes.c_int(0)
+    _check(lib().pcl_profile_end(arr, 32, ctypes.byref(n)), "pcl_profile_end")
+    return {arr[i].name.decode(): dict(launches=int(arr[i].launches), total_ms=float(arr[i].total_ms),
+                                       work=float(arr[i].work)) for i in range(n.value)}

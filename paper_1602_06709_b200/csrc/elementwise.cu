@@ -237,22 +237,28 @@ __global__ void __launch_bounds__(256) softmax_xent_kernel(const float* __restri
 int launch_sgd(float* w, const float* dw, size_t n, float lr, cudaStream_t st) {
     if (n == 0) return PCL_OK;
     const int vec = ((reinterpret_cast<uintptr_t>(w) | reinterpret_cast<uintptr_t>(dw)) & 15) == 0;
-    sgd_kernel<<<grid_for(vec ? (n + 3) / 4 : n, 256), 256, 0, st>>>(w, dw, n, lr, vec);
-    count_launch();
+    {
+        LaunchScope scope(KID_SGD, 12.0 * double(n), st);
+        sgd_kernel<<<grid_for(vec ? (n + 3) / 4 : n, 256), 256, 0, st>>>(w, dw, n, lr, vec);
+    }
     return PCL_CHECK_LAUNCH();
 }
 
 int launch_zero(float* p, size_t n, cudaStream_t st) {
     if (n == 0) return PCL_OK;
-    zero_kernel<<<grid_for(n, 256), 256, 0, st>>>(p, n);
-    count_launch();
+    {
+        LaunchScope scope(KID_ZERO, 4.0 * double(n), st);
+        zero_kernel<<<grid_for(n, 256), 256, 0, st>>>(p, n);
+    }
     return PCL_CHECK_LAUNCH();
 }
 
 int launch_reduce_splits(const float* partial, float* out, size_t n, int splits, cudaStream_t st) {
     if (n == 0) return PCL_OK;
-    reduce_splits_kernel<<<grid_for(n, 256), 256, 0, st>>>(partial, out, n, splits);
-    count_launch();
+    {
+        LaunchScope scope(KID_REDUCE_SPLITS, 4.0 * double(n) * (splits + 1), st);
+        reduce_splits_kernel<<<grid_for(n, 256), 256, 0, st>>>(partial, out, n, splits);
+    }
     return PCL_CHECK_LAUNCH();
 }
 
@@ -260,15 +266,19 @@ int launch_transpose_flip(const float* w, float* wt_t, int K, int R, int S, int 
     if (R * S > 65535) return PCL_ERR_UNSUPPORTED_SHAPE;
     dim3 grid((C + 31) / 32, (K + 31) / 32, R * S);
     if (grid.y > 65535) return PCL_ERR_UNSUPPORTED_SHAPE;
-    transpose_flip_kernel<<<grid, 256, 0, st>>>(w, wt_t, K, R * S, C);
-    count_launch();
+    {
+        LaunchScope scope(KID_TRANSPOSE_FLIP, 8.0 * double(K) * R * S * C, st);
+        transpose_flip_kernel<<<grid, 256, 0, st>>>(w, wt_t, K, R * S, C);
+    }
     return PCL_CHECK_LAUNCH();
 }
 
 int launch_act_grad(float* dy, const float* y, size_t n, int act, cudaStream_t st) {
     if (n == 0 || act == PCL_ACT_NONE) return PCL_OK;
-    act_grad_kernel<<<grid_for(n, 256), 256, 0, st>>>(dy, y, n, act);
-    count_launch();
+    {
+        LaunchScope scope(KID_ACT_GRAD, 12.0 * double(n), st);
+        act_grad_kernel<<<grid_for(n, 256), 256, 0, st>>>(dy, y, n, act);
+    }
     return PCL_CHECK_LAUNCH();
 }
 
@@ -278,8 +288,10 @@ int launch_colsum(const float* m, size_t rows, int K, float* partial, float* out
     const int splits = colsum_splits(rows);
     if (splits > 65535) return PCL_ERR_UNSUPPORTED_SHAPE;
     dim3 grid((K + 31) / 32, splits);
-    colsum_kernel<<<grid, 256, 0, st>>>(m, rows, K, splits == 1 ? out : partial);
-    count_launch();
+    {
+        LaunchScope scope(KID_COLSUM, 4.0 * double(rows) * K, st);
+        colsum_kernel<<<grid, 256, 0, st>>>(m, rows, K, splits == 1 ? out : partial);
+    }
     if (cudaGetLastError() != cudaSuccess) return PCL_ERR_CUDA;
     if (splits > 1) return launch_reduce_splits(partial, out, size_t(K), splits, st);
     return PCL_OK;
@@ -287,22 +299,27 @@ int launch_colsum(const float* m, size_t rows, int K, float* partial, float* out
 
 int launch_maxpool_fwd(int N, int H, int W, int C, const float* x, float* y, cudaStream_t st) {
     const size_t outs = size_t(N) * (H / 2) * (W / 2);
-    if (C % 4 == 0)
-        maxpool_fwd_kernel<4><<<grid_for(outs * (C / 4), 256), 256, 0, st>>>(x, y, N, H, W, C);
-    else
-        maxpool_fwd_kernel<1><<<grid_for(outs * C, 256), 256, 0, st>>>(x, y, N, H, W, C);
-    count_launch();
+    {
+        LaunchScope scope(KID_MAXPOOL_FWD, 20.0 * double(outs) * C, st);
+        if (C % 4 == 0)
+            maxpool_fwd_kernel<4><<<grid_for(outs * (C / 4), 256), 256, 0, st>>>(x, y, N, H, W, C);
+        else
+            maxpool_fwd_kernel<1><<<grid_for(outs * C, 256), 256, 0, st>>>(x, y, N, H, W, C);
+    }
     return PCL_CHECK_LAUNCH();
 }
 
 int launch_maxpool_bwd(int N, int H, int W, int C, const float* x, const float* dy, const float* mask, float* dx,
                        cudaStream_t st) {
     const size_t outs = size_t(N) * (H / 2) * (W / 2);
-    if (C % 4 == 0)
-        maxpool_bwd_kernel<4><<<grid_for(outs * (C / 4), 256), 256, 0, st>>>(x, dy, mask, dx, N, H, W, C);
-    else
-        maxpool_bwd_kernel<1><<<grid_for(outs * C, 256), 256, 0, st>>>(x, dy, mask, dx, N, H, W, C);
-    count_launch();
+    {
+        // per output: 4 x read + 1 dy read + 4 dx written (the mask source is x itself in the step)
+        LaunchScope scope(KID_MAXPOOL_BWD, 36.0 * double(outs) * C, st);
+        if (C % 4 == 0)
+            maxpool_bwd_kernel<4><<<grid_for(outs * (C / 4), 256), 256, 0, st>>>(x, dy, mask, dx, N, H, W, C);
+        else
+            maxpool_bwd_kernel<1><<<grid_for(outs * C, 256), 256, 0, st>>>(x, dy, mask, dx, N, H, W, C);
+    }
     return PCL_CHECK_LAUNCH();
 }
 
@@ -310,8 +327,10 @@ int launch_softmax_xent(int N, int K, const float* logits, const int* labels, fl
                         cudaStream_t st) {
     int rc = launch_zero(loss, 1, st);
     if (rc != PCL_OK) return rc;
-    softmax_xent_kernel<<<N < 1184 ? N : 1184, 256, 0, st>>>(logits, labels, loss, dlogits, N, K);
-    count_launch();
+    {
+        LaunchScope scope(KID_SOFTMAX_XENT, 8.0 * double(N) * K, st);
+        softmax_xent_kernel<<<N < 1184 ? N : 1184, 256, 0, st>>>(logits, labels, loss, dlogits, N, K);
+    }
     return PCL_CHECK_LAUNCH();
 }
 

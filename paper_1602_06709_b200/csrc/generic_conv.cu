@@ -150,13 +150,15 @@ ConvGeom geom(const pcl_conv_desc& d, int P, int Q) {
 }
 
 template <class Problem>
-int launch(const Problem& pr, long rows, long cols, long depth, int splits, cudaStream_t st) {
+int launch(const Problem& pr, int kid, long rows, long cols, long depth, int splits, cudaStream_t st) {
     const long gx = (rows + BM - 1) / BM, gy = (cols + BN - 1) / BN;
     if (gx > 0x7fffffffL || gy > 65535 || splits > 65535) return PCL_ERR_UNSUPPORTED_SHAPE;
     long per = (depth + splits - 1) / splits;
     per = (per + BK - 1) / BK * BK;
-    generic_gemm_kernel<Problem><<<dim3(unsigned(gx), unsigned(gy), unsigned(splits)), 256, 0, st>>>(pr, per);
-    count_launch();
+    {
+        LaunchScope scope(kid, 2.0 * double(rows) * double(cols) * double(depth), st);
+        generic_gemm_kernel<Problem><<<dim3(unsigned(gx), unsigned(gy), unsigned(splits)), 256, 0, st>>>(pr, per);
+    }
     return cudaGetLastError() == cudaSuccess ? PCL_OK : PCL_ERR_CUDA;
 }
 
@@ -165,13 +167,13 @@ int launch(const Problem& pr, long rows, long cols, long depth, int splits, cuda
 int launch_generic_fwd(const pcl_conv_desc& d, int P, int Q, const float* x, const float* w, const float* bias,
                        float* y, int act, cudaStream_t st) {
     FwdProblem pr{geom(d, P, Q), x, w, bias, y, act};
-    return launch(pr, long(d.N) * P * Q, d.K, long(d.R) * d.S * d.C, 1, st);
+    return launch(pr, KID_GENERIC_FWD, long(d.N) * P * Q, d.K, long(d.R) * d.S * d.C, 1, st);
 }
 
 int launch_generic_bwd_data(const pcl_conv_desc& d, int P, int Q, const float* dy, const float* w,
                             const float* mask_src, float* dx, cudaStream_t st) {
     DgradProblem pr{geom(d, P, Q), dy, w, mask_src, dx};
-    return launch(pr, long(d.N) * d.H * d.W, d.C, long(d.R) * d.S * d.K, 1, st);
+    return launch(pr, KID_GENERIC_DGRAD, long(d.N) * d.H * d.W, d.C, long(d.R) * d.S * d.K, 1, st);
 }
 
 int generic_wgrad_splits(const pcl_conv_desc& d, int P, int Q) {
@@ -193,7 +195,7 @@ int launch_generic_bwd_weights(const pcl_conv_desc& d, int P, int Q, const float
     const size_t dw_elems = size_t(d.K) * d.R * d.S * d.C;
     if (splits > 1 && !partial) return PCL_ERR_WORKSPACE;
     WgradProblem pr{geom(d, P, Q), x, dy, splits > 1 ? partial : dw, splits > 1 ? dw_elems : 0};
-    int rc = launch(pr, d.K, long(d.R) * d.S * d.C, long(d.N) * P * Q, splits, st);
+    int rc = launch(pr, KID_GENERIC_WGRAD, d.K, long(d.R) * d.S * d.C, long(d.N) * P * Q, splits, st);
     if (rc != PCL_OK) return rc;
     if (splits > 1) return launch_reduce_splits(partial, dw, dw_elems, splits, st);
     return PCL_OK;

@@ -3,6 +3,8 @@
 // the caller's stream.
 #include <atomic>
 #include <mutex>
+#include <string.h>
+#include <vector>
 
 #include "pcl_internal.h"
 #include "pcl_ptx.cuh"
@@ -27,7 +29,45 @@ unsigned int* device_status_ptr() {
 }
 
 static std::atomic<unsigned long long> g_launches{0};
-void count_launch(unsigned n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
+
+namespace {
+struct ProfEntry { int kid; double work; cudaEvent_t e0, e1; };
+std::mutex g_prof_mu;
+bool g_prof_on = false;
+std::vector<ProfEntry> g_prof_entries;       // entries of the current profiling window
+std::vector<cudaEvent_t> g_prof_pool;        // events created so far, reused across windows
+size_t g_prof_pool_used = 0;
+const char* const kKernelNames[KID_COUNT] = {
+    "tc_fprop_kernel", "tc_wgrad_kernel", "generic_fwd", "generic_bwd_data", "generic_bwd_weights", "sgd_kernel",
+    "reduce_splits_kernel", "zero_kernel", "transpose_flip_kernel", "act_grad_kernel", "colsum_kernel",
+    "maxpool_fwd_kernel", "maxpool_bwd_kernel", "softmax_xent_kernel"};
+
+cudaEvent_t prof_event() {
+    if (g_prof_pool_used == g_prof_pool.size()) {
+        cudaEvent_t e = nullptr;
+        if (cudaEventCreate(&e) != cudaSuccess) return nullptr;
+        g_prof_pool.push_back(e);
+    }
+    return g_prof_pool[g_prof_pool_used++];
+}
+}  // namespace
+
+LaunchScope::LaunchScope(int kid, double work, cudaStream_t stream) : slot(-1), st(stream) {
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    std::lock_guard<std::mutex> lock(g_prof_mu);
+    if (!g_prof_on) return;
+    ProfEntry e{kid, work, prof_event(), prof_event()};
+    if (!e.e0 || !e.e1) return;
+    cudaEventRecord(e.e0, st);
+    slot = int(g_prof_entries.size());
+    g_prof_entries.push_back(e);
+}
+
+LaunchScope::~LaunchScope() {
+    if (slot < 0) return;
+    std::lock_guard<std::mutex> lock(g_prof_mu);
+    if (slot < int(g_prof_entries.size())) cudaEventRecord(g_prof_entries[slot].e1, st);
+}
 
 static std::atomic<int> g_path{PCL_PATH_AUTO};
 
@@ -305,6 +345,43 @@ int pcl_last_device_status(void* cuda_stream) {
 }
 
 unsigned long long pcl_launch_count(void) { return g_launches.load(); }
+
+int pcl_profile_begin(void) {
+    std::lock_guard<std::mutex> lock(g_prof_mu);
+    g_prof_entries.clear();
+    g_prof_pool_used = 0;
+    g_prof_on = true;
+    return PCL_OK;
+}
+
+int pcl_profile_end(pcl_kernel_stat* stats, int max_stats, int* n_stats) {
+    if (!stats || !n_stats || max_stats < 0) return PCL_ERR_BAD_ARG;
+    std::lock_guard<std::mutex> lock(g_prof_mu);
+    g_prof_on = false;
+    pcl_kernel_stat agg[KID_COUNT];
+    memset(agg, 0, sizeof(agg));
+    int rc = PCL_OK;
+    for (const ProfEntry& e : g_prof_entries) {
+        float ms = 0.f;
+        if (cudaEventSynchronize(e.e1) != cudaSuccess || cudaEventElapsedTime(&ms, e.e0, e.e1) != cudaSuccess) {
+            rc = PCL_ERR_CUDA;
+            break;
+        }
+        agg[e.kid].launches += 1;
+        agg[e.kid].total_ms += ms;
+        agg[e.kid].work += e.work;
+    }
+    g_prof_entries.clear();
+    g_prof_pool_used = 0;
+    int n = 0;
+    for (int k = 0; k < KID_COUNT && n < max_stats; ++k) {
+        if (agg[k].launches == 0) continue;
+        strncpy(agg[k].name, kKernelNames[k], sizeof(agg[k].name) - 1);
+        stats[n++] = agg[k];
+    }
+    *n_stats = n;
+    return rc;
+}
 
 const char* pcl_status_string(int status) {
     switch (status) {

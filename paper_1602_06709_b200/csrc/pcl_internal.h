@@ -9,7 +9,25 @@
 
 namespace pcl {
 
-void count_launch(unsigned n = 1);
+// Kernel families, for launch counting and the optional per-kernel timing.
+enum KernelId {
+    KID_TC_FPROP = 0, KID_TC_WGRAD, KID_GENERIC_FWD, KID_GENERIC_DGRAD, KID_GENERIC_WGRAD, KID_SGD, KID_REDUCE_SPLITS,
+    KID_ZERO, KID_TRANSPOSE_FLIP, KID_ACT_GRAD, KID_COLSUM, KID_MAXPOOL_FWD, KID_MAXPOOL_BWD, KID_SOFTMAX_XENT,
+    KID_COUNT
+};
+
+// Brackets one kernel launch: counts it and, while profiling is switched on
+// (pcl_profile_begin), records a CUDA event on the launching stream before and
+// after it.  `work` is the launch's algorithmic work: flops for the contraction
+// kernels, bytes for the memory-bound ones.
+struct LaunchScope {
+    LaunchScope(int kid, double work, cudaStream_t st);
+    ~LaunchScope();
+    LaunchScope(const LaunchScope&) = delete;
+    LaunchScope& operator=(const LaunchScope&) = delete;
+    int slot;
+    cudaStream_t st;
+};
 
 // Address of the current device's status word (0 = fine, else the code of the
 // first bounded wait that ran out).  nullptr if the address cannot be obtained.

@@ -343,8 +343,10 @@ int launch_tc_fprop(const TcFpropArgs& a, cudaStream_t st) {
     const long total = m_tiles * p.tiles_k;
     const int grid = int(total < g_sm_count ? total : g_sm_count);
     const size_t smem = size_t(p.stages) * stage_bytes + 1024;
-    tc_fprop_kernel<<<grid, 192, smem, st>>>(tmA, tmB, p);
-    count_launch();
+    {
+        LaunchScope scope(KID_TC_FPROP, 2.0 * a.N * a.P * a.Q * double(a.Kout) * a.Cin * a.R * a.S, st);
+        tc_fprop_kernel<<<grid, 192, smem, st>>>(tmA, tmB, p);
+    }
     return cudaGetLastError() == cudaSuccess ? PCL_OK : PCL_ERR_CUDA;
 }
 

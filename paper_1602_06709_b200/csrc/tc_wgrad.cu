@@ -322,8 +322,10 @@ int launch_tc_wgrad(const TcWgradArgs& a, cudaStream_t st) {
     const long items = long(p.k_tiles) * a.R * a.S * p.c_tiles * p.splits;
     if (items > 0x7fffffffL) return PCL_ERR_UNSUPPORTED_SHAPE;
     const size_t smem = size_t(p.stages) * stage_bytes + 1024;
-    tc_wgrad_kernel<<<int(items), 192, smem, st>>>(tmDy, tmX, p);
-    count_launch();
+    {
+        LaunchScope scope(KID_TC_WGRAD, 2.0 * a.N * a.P * a.Q * double(a.K) * a.C * a.R * a.S, st);
+        tc_wgrad_kernel<<<int(items), 192, smem, st>>>(tmDy, tmX, p);
+    }
     if (cudaGetLastError() != cudaSuccess) return PCL_ERR_CUDA;
     if (p.splits > 1 && a.partial) return launch_reduce_splits(a.partial, a.dw, dw_elems, p.splits, st);
     return PCL_OK;
