@@ -112,11 +112,11 @@ class VggWorkload:
     name = "configs[4]: full VGG-A training step (fwd+bwd+SGD), N=256, 3x224x224, He-normal weights, 1000 classes"
     unit = "images/s"
 
-    def __init__(self, rank: int):
+    def __init__(self, rank: int, minibatch: int = 0):
         import torch
         from paper_1602_06709_b200 import inputs, networks
         self.torch = torch
-        self.N = 256
+        self.N = minibatch or 256
         self.net = networks.VggA(self.N)
         x = inputs.uniform(inputs.tensor_id("cfg5", "x", rank), (self.N, 224, 224, 3), 0.0, 1.0)
         lab = inputs.labels(inputs.tensor_id("cfg5", "labels", rank), self.N, 1000)
@@ -145,12 +145,14 @@ class ConvWorkload:
     name = "configs[1]: VGG-A mid conv layer 3x3 s1 p1, N=256 C=K=256 56x56: fwd + bwd_data + bwd_weights + SGD update"
     unit = "TFLOP/s"
 
-    def __init__(self, rank: int):
+    def __init__(self, rank: int, minibatch: int = 0):
         import torch
         from paper_1602_06709_b200 import binding as B
         from paper_1602_06709_b200 import inputs
         self.torch, self.B = torch, B
-        c = inputs.CFG2
+        c = dict(inputs.CFG2)
+        if minibatch:
+            c["N"] = minibatch
         self.N = c["N"]
         self.d = B.conv_desc(c["N"], c["C"], c["K"], c["H"], c["W"], c["R"], c["S"], 1, 1)
         x, w, dy = inputs.conv_inputs("cfg2", f"conv{rank}", c["N"], c["C"], c["H"], c["W"], c["K"], 3, 3, 56, 56, "train")
@@ -191,11 +193,11 @@ class DnnWorkload:
     name = "configs[3]: 7-layer DNN 440-5x2048-8192, sigmoid, minibatch 1024: fwd + bwd + SGD update"
     unit = "frames/s"
 
-    def __init__(self, rank: int):
+    def __init__(self, rank: int, minibatch: int = 0):
         import torch
         from paper_1602_06709_b200 import inputs, networks
         self.torch = torch
-        self.N = inputs.CFG4_N
+        self.N = minibatch or inputs.CFG4_N
         self.net = networks.Dnn(self.N)
         x = inputs.normal(inputs.tensor_id("cfg4", "x", rank), (self.N, 440), 1.0)
         lab = inputs.labels(inputs.tensor_id("cfg4", "labels", rank), self.N, 8192)
@@ -310,6 +312,8 @@ def run_ours(args):
     torch.cuda.set_device(local_rank)
     if world > 1:
         dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    if args.minibatch and not args.kernels_only:
+        raise SystemExit("--minibatch changes the workload: only allowed with --kernels-only")
     B.lib()      # fail loudly here if the extension is missing
 
     def barrier():
@@ -324,7 +328,7 @@ def run_ours(args):
         dist.all_reduce(t, op=dist.ReduceOp.MAX)
         return float(t.item())
 
-    wl = WORKLOADS[args.workload](rank)
+    wl = WORKLOADS[args.workload](rank, args.minibatch)
     peaks = load_peaks()
 
     def timed(fn, steps, warmup, sample_clocks=False):
@@ -348,11 +352,17 @@ def run_ours(args):
         clocks = sampler.stop() if sampler else None
         return ms, launches, clocks
 
-    ms, launches, clocks = timed(wl.step, args.steps, max(args.warmup, 3), sample_clocks=True)
+    ms, launches, clocks = timed(wl.step, args.steps, max(args.warmup, 3), sample_clocks=not args.kernels_only)
     status = B.last_device_status()
     if status != B.OK:
         raise SystemExit(f"device status {status}: {B.status_string(status)}")
     value = wl.units_per_step * args.steps * world / (ms / 1e3)
+
+    if args.kernels_only:      # for profiler captures: just the steps, one short line
+        if rank == 0:
+            print(json.dumps({"workload": wl.name, "minibatch": wl.N, "ms_per_step": ms / args.steps,
+                              "gpu_launches": launches}), flush=True)
+        return
 
     # end to end through the user-level call: pinned host minibatch in, result out, every step
     e2e_steps = max(3, min(args.steps, 10))
@@ -446,6 +456,9 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="vgga", choices=sorted(WORKLOADS))
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--minibatch", type=int, default=0, help="override the workload's minibatch (profiling only)")
+    ap.add_argument("--kernels-only", action="store_true",
+                    help="run warm-up + timed steps only and print a short line (for profiler captures)")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
