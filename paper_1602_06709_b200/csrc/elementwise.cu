@@ -230,6 +230,48 @@ __global__ void __launch_bounds__(256) softmax_xent_kernel(const float* __restri
     }
 }
 
+// xs[n][hh][ww][0..3]: channel-padded copy of x with a zero halo of (pad_h, pad_w)
+__global__ void __launch_bounds__(256) stage_pad_c4_kernel(const float* __restrict__ x, float4* __restrict__ xs, int N,
+                                                           int H, int W, int C, int pad_h, int pad_w) {
+    const int Hp = H + 2 * pad_h, Wp = W + 2 * pad_w;
+    const size_t total = size_t(N) * Hp * Wp;
+    const size_t stride = size_t(gridDim.x) * blockDim.x;
+    for (size_t i = size_t(blockIdx.x) * blockDim.x + threadIdx.x; i < total; i += stride) {
+        const int ww = int(i % Wp) - pad_w; size_t t = i / Wp;
+        const int hh = int(t % Hp) - pad_h; const size_t n = t / Hp;
+        float v[4] = {0.f, 0.f, 0.f, 0.f};
+        if (hh >= 0 && hh < H && ww >= 0 && ww < W) {
+            const float* src = x + ((n * H + hh) * W + ww) * C;
+            for (int c = 0; c < C; ++c) v[c] = __ldg(src + c);
+        }
+        xs[i] = make_float4(v[0], v[1], v[2], v[3]);
+    }
+}
+
+// w4[tap][0..3] = w[tap][0..C-1] padded with zeros (tap = flat (k,r,s))
+__global__ void __launch_bounds__(256) stage_w4_kernel(const float* __restrict__ w, float4* __restrict__ w4,
+                                                       size_t taps, int C) {
+    const size_t stride = size_t(gridDim.x) * blockDim.x;
+    for (size_t i = size_t(blockIdx.x) * blockDim.x + threadIdx.x; i < taps; i += stride) {
+        float v[4] = {0.f, 0.f, 0.f, 0.f};
+        for (int c = 0; c < C; ++c) v[c] = w[i * C + c];
+        w4[i] = make_float4(v[0], v[1], v[2], v[3]);
+    }
+}
+
+// dw[tap][c] = sum_s dw4[s][tap][c], c < C  (fixed order)
+__global__ void __launch_bounds__(256) unpad_reduce_kernel(const float* __restrict__ dw4, float* __restrict__ dw,
+                                                           size_t taps, int C, int splits, size_t split_stride) {
+    const size_t total = taps * C;
+    const size_t stride = size_t(gridDim.x) * blockDim.x;
+    for (size_t i = size_t(blockIdx.x) * blockDim.x + threadIdx.x; i < total; i += stride) {
+        const size_t tap = i / C; const int c = int(i % C);
+        float acc = 0.f;
+        for (int s = 0; s < splits; ++s) acc += dw4[size_t(s) * split_stride + tap * 4 + c];
+        dw[i] = acc;
+    }
+}
+
 #define PCL_CHECK_LAUNCH() (cudaGetLastError() == cudaSuccess ? PCL_OK : PCL_ERR_CUDA)
 
 }  // namespace
@@ -269,6 +311,33 @@ int launch_transpose_flip(const float* w, float* wt_t, int K, int R, int S, int 
     {
         LaunchScope scope(KID_TRANSPOSE_FLIP, 8.0 * double(K) * R * S * C, st);
         transpose_flip_kernel<<<grid, 256, 0, st>>>(w, wt_t, K, R * S, C);
+    }
+    return PCL_CHECK_LAUNCH();
+}
+
+int launch_stage_pad_c4(const float* x, float* xs, int N, int H, int W, int C, int pad_h, int pad_w, cudaStream_t st) {
+    const size_t total = size_t(N) * (H + 2 * pad_h) * (W + 2 * pad_w);
+    {
+        LaunchScope scope(KID_STAGE_PAD_C4, 4.0 * double(N) * H * W * C + 16.0 * double(total), st);
+        stage_pad_c4_kernel<<<grid_for(total, 256), 256, 0, st>>>(x, reinterpret_cast<float4*>(xs), N, H, W, C, pad_h,
+                                                                    pad_w);
+    }
+    return PCL_CHECK_LAUNCH();
+}
+
+int launch_stage_w4(const float* w, float* w4, size_t taps, int C, cudaStream_t st) {
+    {
+        LaunchScope scope(KID_STAGE_W4, double(taps) * (4.0 * C + 16.0), st);
+        stage_w4_kernel<<<grid_for(taps, 256), 256, 0, st>>>(w, reinterpret_cast<float4*>(w4), taps, C);
+    }
+    return PCL_CHECK_LAUNCH();
+}
+
+int launch_unpad_reduce(const float* dw4, float* dw, size_t taps, int C, int splits, size_t split_stride,
+                        cudaStream_t st) {
+    {
+        LaunchScope scope(KID_UNPAD_REDUCE, 4.0 * double(taps) * C * (splits + 1), st);
+        unpad_reduce_kernel<<<grid_for(taps * C, 256), 256, 0, st>>>(dw4, dw, taps, C, splits, split_stride);
     }
     return PCL_CHECK_LAUNCH();
 }

@@ -40,7 +40,8 @@ size_t g_prof_pool_used = 0;
 const char* const kKernelNames[KID_COUNT] = {
     "tc_fprop_kernel", "tc_wgrad_kernel", "generic_fwd", "generic_bwd_data", "generic_bwd_weights", "sgd_kernel",
     "reduce_splits_kernel", "zero_kernel", "transpose_flip_kernel", "act_grad_kernel", "colsum_kernel",
-    "maxpool_fwd_kernel", "maxpool_bwd_kernel", "softmax_xent_kernel"};
+    "maxpool_fwd_kernel", "maxpool_bwd_kernel", "softmax_xent_kernel", "stage_pad_c4_kernel", "stage_w4_kernel",
+    "unpad_reduce_kernel"};
 
 cudaEvent_t prof_event() {
     if (g_prof_pool_used == g_prof_pool.size()) {
@@ -143,9 +144,26 @@ bool tensor_path_for(const pcl_conv_desc& d, int pass) {
     return false;
 }
 
+// Few-channel first layers (C < 4, stride 1): the input is staged once as a
+// 4-channel, halo-padded copy; a row of S taps x 4 channels is then contiguous
+// (S*4 <= 32 floats), so the tensor-core kernels see a layer with S*4 "channels",
+// an R x 1 kernel and no padding, read through overlapping TMA windows.
+bool few_channel_path_for(const pcl_conv_desc& d, int pass) {
+    if (g_path.load() == PCL_PATH_GENERIC) return false;
+    if (!unit_stride(d) || d.C >= 4 || d.S * 4 > 32 || d.R > 8) return false;
+    if (pass == PCL_PASS_FWD) return true;
+    if (pass == PCL_PASS_BWD_WEIGHTS) return d.K % 4 == 0;
+    return false;
+}
+size_t staged_x_bytes(const pcl_conv_desc& d) {
+    return align_up(size_t(d.N) * (d.H + 2 * d.pad_h) * (d.W + 2 * d.pad_w) * 16, 256);
+}
+size_t staged_w_bytes(const pcl_conv_desc& d) { return align_up(size_t(d.K) * d.R * d.S * 16, 256); }
+
 size_t dw_bytes(const pcl_conv_desc& d) { return align_up(size_t(d.K) * d.R * d.S * d.C * 4, 256); }
 
 struct WgradPlan {
+    bool few;            // few-channel staged path
     bool tensor;
     int splits;          // pixel splits of the main kernel
     size_t partial_bytes;
@@ -154,9 +172,16 @@ struct WgradPlan {
 
 WgradPlan plan_wgrad(const pcl_conv_desc& d, int P, int Q) {
     WgradPlan pl{};
-    pl.tensor = tensor_path_for(d, PCL_PASS_BWD_WEIGHTS);
-    pl.splits = pl.tensor ? tc_wgrad_splits(d.N, P, Q, d.C, d.K, d.R, d.S) : generic_wgrad_splits(d, P, Q);
-    pl.partial_bytes = pl.splits > 1 ? size_t(pl.splits) * dw_bytes(d) : 0;
+    pl.few = few_channel_path_for(d, PCL_PASS_BWD_WEIGHTS);
+    pl.tensor = pl.few || tensor_path_for(d, PCL_PASS_BWD_WEIGHTS);
+    if (pl.few) {
+        pl.splits = tc_wgrad_splits(d.N, P, Q, d.S * 4, d.K, d.R, 1, 1);
+        // staged x + per-split dw4 tiles (always two-pass: the un-padding pass is needed anyway)
+        pl.partial_bytes = staged_x_bytes(d) + size_t(pl.splits) * staged_w_bytes(d);
+    } else {
+        pl.splits = pl.tensor ? tc_wgrad_splits(d.N, P, Q, d.C, d.K, d.R, d.S) : generic_wgrad_splits(d, P, Q);
+        pl.partial_bytes = pl.splits > 1 ? size_t(pl.splits) * dw_bytes(d) : 0;
+    }
     const int cs = colsum_splits(size_t(d.N) * P * Q);
     pl.colsum_bytes = cs > 1 ? align_up(size_t(cs) * d.K * 4, 256) : 0;
     return pl;
@@ -184,7 +209,7 @@ size_t pcl_conv_workspace_bytes(const pcl_conv_desc* d, int pass) {
     int P, Q;
     if (check_desc(d, &P, &Q) != PCL_OK) return 0;
     switch (pass) {
-        case PCL_PASS_FWD: return 0;
+        case PCL_PASS_FWD: return few_channel_path_for(*d, pass) ? staged_x_bytes(*d) + staged_w_bytes(*d) : 0;
         case PCL_PASS_BWD_DATA: return tensor_path_for(*d, pass) ? dw_bytes(*d) : 0;
         case PCL_PASS_BWD_WEIGHTS: {
             const WgradPlan pl = plan_wgrad(*d, P, Q);
@@ -204,7 +229,6 @@ size_t pcl_fc_workspace_bytes(int N, int C, int K, int pass) {
 
 int pcl_conv_fwd(const pcl_conv_desc* d, const float* x, const float* w, const float* bias, float* y, int act,
                  void* ws, size_t ws_bytes, void* cuda_stream) {
-    (void)ws; (void)ws_bytes;
     int P, Q;
     int rc = check_desc(d, &P, &Q);
     if (rc != PCL_OK) return rc;
@@ -212,6 +236,21 @@ int pcl_conv_fwd(const pcl_conv_desc* d, const float* x, const float* w, const f
     if (act != PCL_ACT_NONE && act != PCL_ACT_RELU && act != PCL_ACT_SIGMOID) return PCL_ERR_BAD_ARG;
     if (!aligned16(x) || !aligned16(w) || !aligned16(y) || !aligned16(bias)) return PCL_ERR_MISALIGNED;
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    if (few_channel_path_for(*d, PCL_PASS_FWD)) {
+        const size_t xs_bytes = staged_x_bytes(*d), need = xs_bytes + staged_w_bytes(*d);
+        if (!ws || ws_bytes < need) return PCL_ERR_WORKSPACE;
+        if (reinterpret_cast<uintptr_t>(ws) & 255) return PCL_ERR_MISALIGNED;
+        float* xs = static_cast<float*>(ws);
+        float* w4 = reinterpret_cast<float*>(static_cast<char*>(ws) + xs_bytes);
+        rc = launch_stage_pad_c4(x, xs, d->N, d->H, d->W, d->C, d->pad_h, d->pad_w, st);
+        if (rc != PCL_OK) return rc;
+        rc = launch_stage_w4(w, w4, size_t(d->K) * d->R * d->S, d->C, st);
+        if (rc != PCL_OK) return rc;
+        const int Hp = d->H + 2 * d->pad_h, Wp = d->W + 2 * d->pad_w;
+        TcFpropArgs a{xs, w4, bias, nullptr, y, d->N, Hp, Q, d->S * 4, d->K, d->R, 1, 0, 0, P, Q, act};
+        a.in_stride_w = 4; a.in_stride_h = long(Wp) * 4; a.in_stride_n = long(Hp) * Wp * 4;
+        return launch_tc_fprop(a, st);
+    }
     if (tensor_path_for(*d, PCL_PASS_FWD)) {
         TcFpropArgs a{x, w, bias, nullptr, y, d->N, d->H, d->W, d->C, d->K, d->R, d->S, d->pad_h, d->pad_w, P, Q, act};
         return launch_tc_fprop(a, st);
@@ -254,6 +293,31 @@ int pcl_conv_bwd_weights(const pcl_conv_desc* d, const float* x, const float* dy
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
     const WgradPlan pl = plan_wgrad(*d, P, Q);
     if (!pl.tensor && g_path.load() == PCL_PATH_TENSOR) return PCL_ERR_UNSUPPORTED_SHAPE;
+    if (pl.few) {
+        const size_t xs_bytes = staged_x_bytes(*d);
+        const size_t need_few = pl.partial_bytes + (dbias ? pl.colsum_bytes : 0);
+        if (!ws || ws_bytes < need_few) return PCL_ERR_WORKSPACE;
+        if (reinterpret_cast<uintptr_t>(ws) & 255) return PCL_ERR_MISALIGNED;
+        float* xs = static_cast<float*>(ws);
+        float* dw4 = reinterpret_cast<float*>(static_cast<char*>(ws) + xs_bytes);
+        float* cs = reinterpret_cast<float*>(static_cast<char*>(ws) + pl.partial_bytes);
+        rc = launch_stage_pad_c4(x, xs, d->N, d->H, d->W, d->C, d->pad_h, d->pad_w, st);
+        if (rc != PCL_OK) return rc;
+        const int Hp = d->H + 2 * d->pad_h, Wp = d->W + 2 * d->pad_w;
+        const size_t taps = size_t(d->K) * d->R * d->S;
+        // partial tiles always go to the workspace (splits == 1 included): dw4 is [split][K][R][S*4]
+        TcWgradArgs a{xs, dy, dw4, pl.splits > 1 ? dw4 : nullptr, d->N, Hp, Q, d->S * 4, d->K, d->R, 1, 0, 0, P, Q,
+                      pl.splits};
+        a.x_stride_w = 4; a.x_stride_h = long(Wp) * 4; a.x_stride_n = long(Hp) * Wp * 4;
+        a.tap_groups = 1;
+        a.skip_reduce = 1;
+        rc = launch_tc_wgrad(a, st);
+        if (rc != PCL_OK) return rc;
+        rc = launch_unpad_reduce(dw4, dw, taps, d->C, pl.splits, taps * 4, st);
+        if (rc != PCL_OK) return rc;
+        if (dbias) rc = launch_colsum(dy, size_t(d->N) * P * Q, d->K, cs, dbias, st);
+        return rc;
+    }
     const bool need_partial = pl.splits > 1 && (deterministic || !pl.tensor);
     size_t need = (need_partial ? pl.partial_bytes : 0) + (dbias ? pl.colsum_bytes : 0);
     if (need > 0) {

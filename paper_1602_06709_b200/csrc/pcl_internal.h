@@ -13,7 +13,7 @@ namespace pcl {
 enum KernelId {
     KID_TC_FPROP = 0, KID_TC_WGRAD, KID_GENERIC_FWD, KID_GENERIC_DGRAD, KID_GENERIC_WGRAD, KID_SGD, KID_REDUCE_SPLITS,
     KID_ZERO, KID_TRANSPOSE_FLIP, KID_ACT_GRAD, KID_COLSUM, KID_MAXPOOL_FWD, KID_MAXPOOL_BWD, KID_SOFTMAX_XENT,
-    KID_COUNT
+    KID_STAGE_PAD_C4, KID_STAGE_W4, KID_UNPAD_REDUCE, KID_COUNT
 };
 
 // Brackets one kernel launch: counts it and, while profiling is switched on
@@ -56,6 +56,10 @@ struct TcFpropArgs {
     const float* mask_src; // [N][P][Q][Kout] or null
     float* out;        // [N][P][Q][Kout]
     int N, H, W, Cin, Kout, R, S, pad_h, pad_w, P, Q, act;
+    // Element strides of `in` between adjacent w, h and n positions; 0 = packed
+    // NHWC (Cin, W*Cin, H*W*Cin).  A w stride smaller than Cin gives overlapping
+    // windows (used by the few-channel first-layer path).
+    long in_stride_w = 0, in_stride_h = 0, in_stride_n = 0;
 };
 bool tc_fprop_eligible(const TcFpropArgs& a);
 int launch_tc_fprop(const TcFpropArgs& a, cudaStream_t st);
@@ -69,9 +73,17 @@ struct TcWgradArgs {
     float* partial;   // workspace for the two-pass variant ([splits][K*R*S*C]) or null (atomics)
     int N, H, W, C, K, R, S, pad_h, pad_w, P, Q;
     int splits;
+    // Element strides of x (0 = packed NHWC), as in TcFpropArgs.
+    long x_stride_w = 0, x_stride_h = 0, x_stride_n = 0;
+    // tap_groups != 0: S must be 1 and C <= 32; one CTA handles all R taps of a k
+    // tile at once, the MMA N dimension being R groups of 32 columns (group g =
+    // tap row g).  dw then has the layout [K][R][C].
+    int tap_groups = 0;
+    // skip_reduce != 0: leave the per-split partial tiles in `partial` (the caller reduces them).
+    int skip_reduce = 0;
 };
 bool tc_wgrad_eligible(const TcWgradArgs& a);
-int tc_wgrad_splits(int N, int P, int Q, int C, int K, int R, int S);
+int tc_wgrad_splits(int N, int P, int Q, int C, int K, int R, int S, int tap_groups = 0);
 int launch_tc_wgrad(const TcWgradArgs& a, cudaStream_t st);
 
 // ---- generic CUDA-core kernels (any stride / pad / channel count) ----------
@@ -89,6 +101,13 @@ int launch_reduce_splits(const float* partial, float* out, size_t n, int splits,
 int launch_zero(float* p, size_t n, cudaStream_t st);
 // wt_t[c][R-1-r][S-1-s][k] = w[k][r][s][c]
 int launch_transpose_flip(const float* w, float* wt_t, int K, int R, int S, int C, cudaStream_t st);
+// Few-channel staging (C < 4): xs[n][h+pad_h][w+pad_w][0..3] = x[n][h][w][0..C-1] padded with zeros (channel
+// padding and a spatial halo of pad_h / pad_w); w4[k][r][s*4 + c] = w[k][r][s][c];
+// dw[k][r][s][c] = sum over splits of dw4[split][k][r][s*4 + c].
+int launch_stage_pad_c4(const float* x, float* xs, int N, int H, int W, int C, int pad_h, int pad_w, cudaStream_t st);
+int launch_stage_w4(const float* w, float* w4, size_t taps, int C, cudaStream_t st);
+int launch_unpad_reduce(const float* dw4, float* dw, size_t taps, int C, int splits, size_t split_stride,
+                        cudaStream_t st);
 // dz = dy * act'(y), in place on dy
 int launch_act_grad(float* dy, const float* y, size_t n, int act, cudaStream_t st);
 // out[k] = sum_rows m[row][k]; partial: [colsum_splits(rows)][K] workspace

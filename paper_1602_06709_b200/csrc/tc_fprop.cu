@@ -328,7 +328,10 @@ int launch_tc_fprop(const TcFpropArgs& a, cudaStream_t st) {
     CUtensorMap tmA, tmB;
     {
         const uint64_t dims[4] = {uint64_t(a.Cin), uint64_t(a.W), uint64_t(a.H), uint64_t(a.N)};
-        const uint64_t strides[3] = {uint64_t(a.Cin) * 4, uint64_t(a.W) * a.Cin * 4, uint64_t(a.H) * a.W * a.Cin * 4};
+        const uint64_t sw = a.in_stride_w ? uint64_t(a.in_stride_w) : uint64_t(a.Cin);
+        const uint64_t sh = a.in_stride_h ? uint64_t(a.in_stride_h) : uint64_t(a.W) * a.Cin;
+        const uint64_t sn = a.in_stride_n ? uint64_t(a.in_stride_n) : uint64_t(a.H) * a.W * a.Cin;
+        const uint64_t strides[3] = {sw * 4, sh * 4, sn * 4};
         const uint32_t box[4] = {kBlockC, uint32_t(bw), uint32_t(bh), uint32_t(bn)};
         int rc = make_tmap(&tmA, a.in, 4, dims, strides, box, false);
         if (rc != PCL_OK) return rc;

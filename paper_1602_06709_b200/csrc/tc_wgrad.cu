@@ -39,6 +39,7 @@ struct WgradParams {
     int splits, boxes_per_split;
     int stages, tmem_cols;
     int use_atomics;
+    int tap_groups;           // column group g of the MMA = tap row g (few-channel first layers)
     float* out;               // dw, or the partial-sum workspace [splits][K*R*S*C]
     size_t split_stride;      // K*R*S*C (0 when writing straight to dw)
     unsigned int* status;     // device status word
@@ -83,8 +84,9 @@ tc_wgrad_kernel(const __grid_constant__ CUtensorMap tmDy, const __grid_constant_
     int item = blockIdx.x;
     const int split = item % p.splits;   item /= p.splits;
     const int ct = item % p.c_tiles;     item /= p.c_tiles;
-    const int tap = item % (p.R * p.S);
-    const int kt = item / (p.R * p.S);
+    const int taps = p.tap_groups ? 1 : p.R * p.S;
+    const int tap = item % taps;
+    const int kt = item / taps;
     const int r = tap / p.S, s = tap % p.S;
     const int total_boxes = p.boxes_q * p.boxes_p * p.boxes_n;
     const int box_begin = split * p.boxes_per_split;
@@ -110,9 +112,12 @@ tc_wgrad_kernel(const __grid_constant__ CUtensorMap tmDy, const __grid_constant_
 #pragma unroll
                 for (int g = 0; g < 4; ++g)
                     tma_load_4d(dst + g * kGroupBytes, &tmDy, &full_bar[stage], kt * 128 + g * 32, q0, p0, n0);
-                for (int g = 0; g < b_groups; ++g)
-                    tma_load_4d(dst + kABytes + g * kGroupBytes, &tmX, &full_bar[stage], ct * p.BNc + g * 32,
-                                q0 + s - p.pad_w, p0 + r - p.pad_h, n0);
+                for (int g = 0; g < b_groups; ++g) {
+                    const int cc = p.tap_groups ? 0 : ct * p.BNc + g * 32;
+                    const int rr = p.tap_groups ? g : r;
+                    tma_load_4d(dst + kABytes + g * kGroupBytes, &tmX, &full_bar[stage], cc, q0 + s - p.pad_w,
+                                p0 + rr - p.pad_h, n0);
+                }
                 ++issued;
                 if (++stage == p.stages) { stage = 0; phase ^= 1u; }
             }
@@ -158,9 +163,10 @@ tc_wgrad_kernel(const __grid_constant__ CUtensorMap tmDy, const __grid_constant_
         if (bounded_wait_warp(&tmem_full_bar, 0, &abort_flag, p.status, WAIT_EPI_TMEM_FULL)) {
             tc_fence_after();
             const uint32_t t_row = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16);
-            float* base = p.out + static_cast<size_t>(split) * p.split_stride +
-                          ((static_cast<size_t>(valid ? k : 0) * p.R + r) * p.S + s) * p.C;
+            const size_t krow = static_cast<size_t>(valid ? k : 0) * p.R;
             for (int ch = 0; ch < b_groups; ++ch) {
+                const int rr = p.tap_groups ? ch : r;
+                float* base = p.out + static_cast<size_t>(split) * p.split_stride + ((krow + rr) * p.S + s) * p.C;
                 uint32_t v[32];
                 if (kiters > 0) {
                     tmem_ld_32x32(t_row + ch * 32, v);
@@ -169,7 +175,7 @@ tc_wgrad_kernel(const __grid_constant__ CUtensorMap tmDy, const __grid_constant_
 #pragma unroll
                     for (int j = 0; j < 32; ++j) v[j] = 0u;
                 }
-                const int c0 = ct * p.BNc + ch * 32;
+                const int c0 = p.tap_groups ? 0 : ct * p.BNc + ch * 32;
                 if (valid && c0 < p.C) {
                     float* dst = base + c0;
                     if (p.use_atomics) {
@@ -245,17 +251,18 @@ bool g_attr_set = false;
 
 bool tc_wgrad_eligible(const TcWgradArgs& a) {
     if (a.C % 4 != 0 || a.K % 4 != 0) return false;
+    if (a.tap_groups && (a.S != 1 || a.C > 32 || a.R * 32 > 256)) return false;
     if ((reinterpret_cast<uintptr_t>(a.x) | reinterpret_cast<uintptr_t>(a.dy)) & 15) return false;
     return true;
 }
 
-int tc_wgrad_splits(int N, int P, int Q, int C, int K, int R, int S) {
+int tc_wgrad_splits(int N, int P, int Q, int C, int K, int R, int S, int tap_groups) {
     const int bnc = choose_bnc(C);
-    const long items = long((K + 127) / 128) * R * S * ((C + bnc - 1) / bnc);
+    const long items = tap_groups ? long((K + 127) / 128) : long((K + 127) / 128) * R * S * ((C + bnc - 1) / bnc);
     const long boxes = total_pixel_boxes(N, P, Q);
     long splits = sm_count() / items;
     if (splits < 1) splits = 1;
-    if (splits > 64) splits = 64;
+    if (splits > 64 && !tap_groups) splits = 64;
     if (splits > boxes) splits = boxes;
     // drop splits that would be empty
     const long per = (boxes + splits - 1) / splits;
@@ -279,8 +286,9 @@ int launch_tc_wgrad(const TcWgradArgs& a, cudaStream_t st) {
     p.boxes_n = (a.N + bn - 1) / bn;
     const long boxes = long(p.boxes_q) * p.boxes_p * p.boxes_n;
     if (boxes > 0x7fffffffL) return PCL_ERR_UNSUPPORTED_SHAPE;
-    p.BNc = choose_bnc(a.C);
-    p.c_tiles = (a.C + p.BNc - 1) / p.BNc;
+    p.tap_groups = a.tap_groups;
+    p.BNc = a.tap_groups ? a.R * 32 : choose_bnc(a.C);
+    p.c_tiles = a.tap_groups ? 1 : (a.C + p.BNc - 1) / p.BNc;
     p.k_tiles = (a.K + 127) / 128;
     p.R = a.R; p.S = a.S; p.pad_h = a.pad_h; p.pad_w = a.pad_w;
     p.K = a.K; p.C = a.C;
@@ -314,12 +322,15 @@ int launch_tc_wgrad(const TcWgradArgs& a, cudaStream_t st) {
     }
     {
         const uint64_t dims[4] = {uint64_t(a.C), uint64_t(a.W), uint64_t(a.H), uint64_t(a.N)};
-        const uint64_t strides[3] = {uint64_t(a.C) * 4, uint64_t(a.W) * a.C * 4, uint64_t(a.H) * a.W * a.C * 4};
+        const uint64_t sw = a.x_stride_w ? uint64_t(a.x_stride_w) : uint64_t(a.C);
+        const uint64_t sh = a.x_stride_h ? uint64_t(a.x_stride_h) : uint64_t(a.W) * a.C;
+        const uint64_t sn = a.x_stride_n ? uint64_t(a.x_stride_n) : uint64_t(a.H) * a.W * a.C;
+        const uint64_t strides[3] = {sw * 4, sh * 4, sn * 4};
         const uint32_t box[4] = {32, uint32_t(bw), uint32_t(bh), uint32_t(bn)};
         int rc = make_tmap(&tmX, a.x, 4, dims, strides, box, true);
         if (rc != PCL_OK) return rc;
     }
-    const long items = long(p.k_tiles) * a.R * a.S * p.c_tiles * p.splits;
+    const long items = long(p.k_tiles) * (a.tap_groups ? 1 : a.R * a.S) * p.c_tiles * p.splits;
     if (items > 0x7fffffffL) return PCL_ERR_UNSUPPORTED_SHAPE;
     const size_t smem = size_t(p.stages) * stage_bytes + 1024;
     {
@@ -327,7 +338,7 @@ int launch_tc_wgrad(const TcWgradArgs& a, cudaStream_t st) {
         tc_wgrad_kernel<<<int(items), 192, smem, st>>>(tmDy, tmX, p);
     }
     if (cudaGetLastError() != cudaSuccess) return PCL_ERR_CUDA;
-    if (p.splits > 1 && a.partial) return launch_reduce_splits(a.partial, a.dw, dw_elems, p.splits, st);
+    if (p.splits > 1 && a.partial && !a.skip_reduce) return launch_reduce_splits(a.partial, a.dw, dw_elems, p.splits, st);
     return PCL_OK;
 }
 

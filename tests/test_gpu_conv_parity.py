@@ -19,8 +19,14 @@ TENSOR_SHAPES = {
     "rect_kernel": ConvShape(N=2, C=24, K=40, H=10, W=17, R=2, S=3, pad_h=1, pad_w=0),
     "many_pixels": ConvShape(N=6, C=32, K=32, H=56, W=56, R=3, S=3, pad_h=1, pad_w=1),
 }
-GENERIC_SHAPES = {
+FEW_CHANNEL_SHAPES = {   # C < 4, stride 1: staged 4-channel copy + overlapping TMA windows
     "rgb": ConvShape(N=2, C=3, K=16, H=20, W=20, R=3, S=3, pad_h=1, pad_w=1),
+    "rgb_big": ConvShape(N=3, C=3, K=64, H=40, W=36, R=3, S=3, pad_h=1, pad_w=1),
+    "gray_5x5": ConvShape(N=2, C=1, K=24, H=17, W=19, R=5, S=5, pad_h=2, pad_w=2),
+    "two_ch_nopad": ConvShape(N=2, C=2, K=36, H=12, W=15, R=3, S=2),
+    "rgb_7x7_pad": ConvShape(N=1, C=3, K=8, H=14, W=14, R=7, S=7, pad_h=3, pad_w=1),
+}
+GENERIC_SHAPES = {
     "rgb_stride4": ConvShape(N=2, C=3, K=24, H=47, W=47, R=11, S=11, stride_h=4, stride_w=4),
     "stride2": ConvShape(N=3, C=20, K=36, H=15, W=18, R=3, S=3, stride_h=2, stride_w=2, pad_h=1, pad_w=1),
     "odd_channels": ConvShape(N=2, C=7, K=9, H=11, W=13, R=3, S=3, pad_h=1, pad_w=1),
@@ -33,6 +39,9 @@ def _cases():
     out = []
     for tag, s in TENSOR_SHAPES.items():
         out.append(pytest.param(tag, s, B.PATH_TENSOR, id=f"tensor-{tag}"))
+        out.append(pytest.param(tag, s, B.PATH_GENERIC, id=f"generic-{tag}"))
+    for tag, s in FEW_CHANNEL_SHAPES.items():
+        out.append(pytest.param(tag, s, B.PATH_AUTO, id=f"few-{tag}"))
         out.append(pytest.param(tag, s, B.PATH_GENERIC, id=f"generic-{tag}"))
     for tag, s in GENERIC_SHAPES.items():
         out.append(pytest.param(tag, s, B.PATH_AUTO, id=f"auto-{tag}"))
