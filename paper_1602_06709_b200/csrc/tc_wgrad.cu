@@ -40,6 +40,7 @@ struct WgradParams {
     int stages, tmem_cols;
     int use_atomics;
     int tap_groups;           // column group g of the MMA = tap row g (few-channel first layers)
+    int grouped;              // 5-D tensor maps: all 32-map groups of an operand arrive with one TMA instruction
     float* out;               // dw, or the partial-sum workspace [splits][K*R*S*C]
     size_t split_stride;      // K*R*S*C (0 when writing straight to dw)
     unsigned int* status;     // device status word
@@ -109,6 +110,11 @@ tc_wgrad_kernel(const __grid_constant__ CUtensorMap tmDy, const __grid_constant_
                 if (!bounded_wait(&empty_bar[stage], phase ^ 1u, &abort_flag, p.status, WAIT_PRODUCER_EMPTY)) { ok = false; break; }
                 uint8_t* dst = smem + stage * stage_bytes;
                 mbar_expect_tx(&full_bar[stage], stage_bytes);
+                if (p.grouped) {
+                    tma_load_5d(dst, &tmDy, &full_bar[stage], 0, q0, p0, n0, kt * 4);
+                    tma_load_5d(dst + kABytes, &tmX, &full_bar[stage], 0, q0 + s - p.pad_w, p0 + r - p.pad_h, n0,
+                                ct * b_groups);
+                } else {
 #pragma unroll
                 for (int g = 0; g < 4; ++g)
                     tma_load_4d(dst + g * kGroupBytes, &tmDy, &full_bar[stage], kt * 128 + g * 32, q0, p0, n0);
@@ -117,6 +123,7 @@ tc_wgrad_kernel(const __grid_constant__ CUtensorMap tmDy, const __grid_constant_
                     const int rr = p.tap_groups ? g : r;
                     tma_load_4d(dst + kABytes + g * kGroupBytes, &tmX, &full_bar[stage], cc, q0 + s - p.pad_w,
                                 p0 + rr - p.pad_h, n0);
+                }
                 }
                 ++issued;
                 if (++stage == p.stages) { stage = 0; phase ^= 1u; }
@@ -312,23 +319,44 @@ int launch_tc_wgrad(const TcWgradArgs& a, cudaStream_t st) {
         if (rc != PCL_OK) return rc;
     }
 
+    // When both map counts are multiples of 32, view each tensor as 5-D {32 maps, w, h, n, group} (the group
+    // dimension has a 128-byte stride) so that one TMA instruction brings all groups of an operand, laid out
+    // [group][pixel][32 maps] in shared memory exactly as the per-group boxes would be.
+    p.grouped = (!a.tap_groups && a.C % 32 == 0 && a.K % 32 == 0) ? 1 : 0;
     CUtensorMap tmDy, tmX;
     {
-        const uint64_t dims[4] = {uint64_t(a.K), uint64_t(a.Q), uint64_t(a.P), uint64_t(a.N)};
-        const uint64_t strides[3] = {uint64_t(a.K) * 4, uint64_t(a.Q) * a.K * 4, uint64_t(a.P) * a.Q * a.K * 4};
-        const uint32_t box[4] = {32, uint32_t(bw), uint32_t(bh), uint32_t(bn)};
-        int rc = make_tmap(&tmDy, a.dy, 4, dims, strides, box, true);
-        if (rc != PCL_OK) return rc;
+        const uint64_t sw = uint64_t(a.K), sh = uint64_t(a.Q) * a.K, sn = uint64_t(a.P) * a.Q * a.K;
+        if (p.grouped) {
+            const uint64_t dims[5] = {32, uint64_t(a.Q), uint64_t(a.P), uint64_t(a.N), uint64_t(a.K / 32)};
+            const uint64_t strides[4] = {sw * 4, sh * 4, sn * 4, 128};
+            const uint32_t box[5] = {32, uint32_t(bw), uint32_t(bh), uint32_t(bn), 4};
+            int rc = make_tmap(&tmDy, a.dy, 5, dims, strides, box, true);
+            if (rc != PCL_OK) return rc;
+        } else {
+            const uint64_t dims[4] = {uint64_t(a.K), uint64_t(a.Q), uint64_t(a.P), uint64_t(a.N)};
+            const uint64_t strides[3] = {sw * 4, sh * 4, sn * 4};
+            const uint32_t box[4] = {32, uint32_t(bw), uint32_t(bh), uint32_t(bn)};
+            int rc = make_tmap(&tmDy, a.dy, 4, dims, strides, box, true);
+            if (rc != PCL_OK) return rc;
+        }
     }
     {
-        const uint64_t dims[4] = {uint64_t(a.C), uint64_t(a.W), uint64_t(a.H), uint64_t(a.N)};
         const uint64_t sw = a.x_stride_w ? uint64_t(a.x_stride_w) : uint64_t(a.C);
         const uint64_t sh = a.x_stride_h ? uint64_t(a.x_stride_h) : uint64_t(a.W) * a.C;
         const uint64_t sn = a.x_stride_n ? uint64_t(a.x_stride_n) : uint64_t(a.H) * a.W * a.C;
-        const uint64_t strides[3] = {sw * 4, sh * 4, sn * 4};
-        const uint32_t box[4] = {32, uint32_t(bw), uint32_t(bh), uint32_t(bn)};
-        int rc = make_tmap(&tmX, a.x, 4, dims, strides, box, true);
-        if (rc != PCL_OK) return rc;
+        if (p.grouped) {
+            const uint64_t dims[5] = {32, uint64_t(a.W), uint64_t(a.H), uint64_t(a.N), uint64_t(a.C / 32)};
+            const uint64_t strides[4] = {sw * 4, sh * 4, sn * 4, 128};
+            const uint32_t box[5] = {32, uint32_t(bw), uint32_t(bh), uint32_t(bn), uint32_t(p.BNc / 32)};
+            int rc = make_tmap(&tmX, a.x, 5, dims, strides, box, true);
+            if (rc != PCL_OK) return rc;
+        } else {
+            const uint64_t dims[4] = {uint64_t(a.C), uint64_t(a.W), uint64_t(a.H), uint64_t(a.N)};
+            const uint64_t strides[3] = {sw * 4, sh * 4, sn * 4};
+            const uint32_t box[4] = {32, uint32_t(bw), uint32_t(bh), uint32_t(bn)};
+            int rc = make_tmap(&tmX, a.x, 4, dims, strides, box, true);
+            if (rc != PCL_OK) return rc;
+        }
     }
     const long items = long(p.k_tiles) * (a.tap_groups ? 1 : a.R * a.S) * p.c_tiles * p.splits;
     if (items > 0x7fffffffL) return PCL_ERR_UNSUPPORTED_SHAPE;
