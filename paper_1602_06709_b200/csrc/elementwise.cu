@@ -234,13 +234,13 @@ __global__ void __launch_bounds__(256) softmax_xent_kernel(const float* __restri
 __global__ void __launch_bounds__(256) stage_pad_c4_kernel(const float* __restrict__ x, float4* __restrict__ xs, int N,
                                                            int H, int W, int C, int pad_h, int pad_w) {
     const int Hp = H + 2 * pad_h, Wp = W + 2 * pad_w;
-    const size_t total = size_t(N) * Hp * Wp;
+    const size_t total = size_t(N) * Hp * Wp + 8;   // 8 trailing zero pixels: windows are read 32 floats wide
     const size_t stride = size_t(gridDim.x) * blockDim.x;
     for (size_t i = size_t(blockIdx.x) * blockDim.x + threadIdx.x; i < total; i += stride) {
         const int ww = int(i % Wp) - pad_w; size_t t = i / Wp;
         const int hh = int(t % Hp) - pad_h; const size_t n = t / Hp;
         float v[4] = {0.f, 0.f, 0.f, 0.f};
-        if (hh >= 0 && hh < H && ww >= 0 && ww < W) {
+        if (n < size_t(N) && hh >= 0 && hh < H && ww >= 0 && ww < W) {
             const float* src = x + ((n * H + hh) * W + ww) * C;
             for (int c = 0; c < C; ++c) v[c] = __ldg(src + c);
         }
@@ -248,14 +248,15 @@ __global__ void __launch_bounds__(256) stage_pad_c4_kernel(const float* __restri
     }
 }
 
-// w4[tap][0..3] = w[tap][0..C-1] padded with zeros (tap = flat (k,r,s))
-__global__ void __launch_bounds__(256) stage_w4_kernel(const float* __restrict__ w, float4* __restrict__ w4,
-                                                       size_t taps, int C) {
+// w32[k*R + r][s*4 + c] = w[k][r][s][c] for c < C, s < S; every other element of the 32-float row is zero
+__global__ void __launch_bounds__(256) stage_w4_kernel(const float* __restrict__ w, float* __restrict__ w32,
+                                                       size_t rows, int S, int C) {
+    const size_t total = rows * 32;
     const size_t stride = size_t(gridDim.x) * blockDim.x;
-    for (size_t i = size_t(blockIdx.x) * blockDim.x + threadIdx.x; i < taps; i += stride) {
-        float v[4] = {0.f, 0.f, 0.f, 0.f};
-        for (int c = 0; c < C; ++c) v[c] = w[i * C + c];
-        w4[i] = make_float4(v[0], v[1], v[2], v[3]);
+    for (size_t i = size_t(blockIdx.x) * blockDim.x + threadIdx.x; i < total; i += stride) {
+        const int j = int(i & 31); const size_t row = i >> 5;
+        const int s = j >> 2, c = j & 3;
+        w32[i] = (s < S && c < C) ? w[(row * S + s) * C + c] : 0.f;
     }
 }
 
@@ -316,7 +317,7 @@ int launch_transpose_flip(const float* w, float* wt_t, int K, int R, int S, int 
 }
 
 int launch_stage_pad_c4(const float* x, float* xs, int N, int H, int W, int C, int pad_h, int pad_w, cudaStream_t st) {
-    const size_t total = size_t(N) * (H + 2 * pad_h) * (W + 2 * pad_w);
+    const size_t total = size_t(N) * (H + 2 * pad_h) * (W + 2 * pad_w) + 8;
     {
         LaunchScope scope(KID_STAGE_PAD_C4, 4.0 * double(N) * H * W * C + 16.0 * double(total), st);
         stage_pad_c4_kernel<<<grid_for(total, 256), 256, 0, st>>>(x, reinterpret_cast<float4*>(xs), N, H, W, C, pad_h,
@@ -325,10 +326,10 @@ int launch_stage_pad_c4(const float* x, float* xs, int N, int H, int W, int C, i
     return PCL_CHECK_LAUNCH();
 }
 
-int launch_stage_w4(const float* w, float* w4, size_t taps, int C, cudaStream_t st) {
+int launch_stage_w4(const float* w, float* w32, size_t rows, int S, int C, cudaStream_t st) {
     {
-        LaunchScope scope(KID_STAGE_W4, double(taps) * (4.0 * C + 16.0), st);
-        stage_w4_kernel<<<grid_for(taps, 256), 256, 0, st>>>(w, reinterpret_cast<float4*>(w4), taps, C);
+        LaunchScope scope(KID_STAGE_W4, double(rows) * (4.0 * S * C + 128.0), st);
+        stage_w4_kernel<<<grid_for(rows * 32, 256), 256, 0, st>>>(w, w32, rows, S, C);
     }
     return PCL_CHECK_LAUNCH();
 }

@@ -155,10 +155,10 @@ bool few_channel_path_for(const pcl_conv_desc& d, int pass) {
     if (pass == PCL_PASS_BWD_WEIGHTS) return d.K % 4 == 0;
     return false;
 }
-size_t staged_x_bytes(const pcl_conv_desc& d) {
-    return align_up(size_t(d.N) * (d.H + 2 * d.pad_h) * (d.W + 2 * d.pad_w) * 16, 256);
+size_t staged_x_bytes(const pcl_conv_desc& d) {   // + 8 zero pixels of slack: windows are read 32 floats wide
+    return align_up((size_t(d.N) * (d.H + 2 * d.pad_h) * (d.W + 2 * d.pad_w) + 8) * 16, 256);
 }
-size_t staged_w_bytes(const pcl_conv_desc& d) { return align_up(size_t(d.K) * d.R * d.S * 16, 256); }
+size_t staged_w_bytes(const pcl_conv_desc& d) { return align_up(size_t(d.K) * d.R * 128, 256); }
 
 size_t dw_bytes(const pcl_conv_desc& d) { return align_up(size_t(d.K) * d.R * d.S * d.C * 4, 256); }
 
@@ -244,10 +244,11 @@ int pcl_conv_fwd(const pcl_conv_desc* d, const float* x, const float* w, const f
         float* w4 = reinterpret_cast<float*>(static_cast<char*>(ws) + xs_bytes);
         rc = launch_stage_pad_c4(x, xs, d->N, d->H, d->W, d->C, d->pad_h, d->pad_w, st);
         if (rc != PCL_OK) return rc;
-        rc = launch_stage_w4(w, w4, size_t(d->K) * d->R * d->S, d->C, st);
+        rc = launch_stage_w4(w, w4, size_t(d->K) * d->R, d->S, d->C, st);
         if (rc != PCL_OK) return rc;
         const int Hp = d->H + 2 * d->pad_h, Wp = d->W + 2 * d->pad_w;
-        TcFpropArgs a{xs, w4, bias, nullptr, y, d->N, Hp, Q, d->S * 4, d->K, d->R, 1, 0, 0, P, Q, act};
+        // the staged layer: 32 "channels" per pixel window (S*4 carry weight, the rest meets zero weights)
+        TcFpropArgs a{xs, w4, bias, nullptr, y, d->N, Hp, Q, 32, d->K, d->R, 1, 0, 0, P, Q, act};
         a.in_stride_w = 4; a.in_stride_h = long(Wp) * 4; a.in_stride_n = long(Hp) * Wp * 4;
         return launch_tc_fprop(a, st);
     }
@@ -309,6 +310,7 @@ int pcl_conv_bwd_weights(const pcl_conv_desc* d, const float* x, const float* dy
         TcWgradArgs a{xs, dy, dw4, pl.splits > 1 ? dw4 : nullptr, d->N, Hp, Q, d->S * 4, d->K, d->R, 1, 0, 0, P, Q,
                       pl.splits};
         a.x_stride_w = 4; a.x_stride_h = long(Wp) * 4; a.x_stride_n = long(Hp) * Wp * 4;
+        a.x_inner = 32;
         a.tap_groups = 1;
         a.skip_reduce = 1;
         rc = launch_tc_wgrad(a, st);

@@ -60,6 +60,10 @@ struct TcFpropArgs {
     // NHWC (Cin, W*Cin, H*W*Cin).  A w stride smaller than Cin gives overlapping
     // windows (used by the few-channel first-layer path).
     long in_stride_w = 0, in_stride_h = 0, in_stride_n = 0;
+    // Innermost extent the tensor map declares (0 = Cin).  The few-channel path declares 32 although only Cin
+    // elements carry weight: the rest of the window is real neighbouring data that meets zero weights, which
+    // avoids TMA's slower partial-row zero fill.
+    int in_inner = 0;
 };
 bool tc_fprop_eligible(const TcFpropArgs& a);
 int launch_tc_fprop(const TcFpropArgs& a, cudaStream_t st);
@@ -75,6 +79,7 @@ struct TcWgradArgs {
     int splits;
     // Element strides of x (0 = packed NHWC), as in TcFpropArgs.
     long x_stride_w = 0, x_stride_h = 0, x_stride_n = 0;
+    int x_inner = 0;   // innermost extent declared for x (0 = C); see TcFpropArgs::in_inner
     // tap_groups != 0: S must be 1 and C <= 32; one CTA handles all R taps of a k
     // tile at once, the MMA N dimension being R groups of 32 columns (group g =
     // tap row g).  dw then has the layout [K][R][C].
@@ -102,10 +107,10 @@ int launch_zero(float* p, size_t n, cudaStream_t st);
 // wt_t[c][R-1-r][S-1-s][k] = w[k][r][s][c]
 int launch_transpose_flip(const float* w, float* wt_t, int K, int R, int S, int C, cudaStream_t st);
 // Few-channel staging (C < 4): xs[n][h+pad_h][w+pad_w][0..3] = x[n][h][w][0..C-1] padded with zeros (channel
-// padding and a spatial halo of pad_h / pad_w); w4[k][r][s*4 + c] = w[k][r][s][c];
+// padding and a spatial halo of pad_h / pad_w); w32[k][r][s*4 + c] = w[k][r][s][c] in zero-padded 32-float rows;
 // dw[k][r][s][c] = sum over splits of dw4[split][k][r][s*4 + c].
 int launch_stage_pad_c4(const float* x, float* xs, int N, int H, int W, int C, int pad_h, int pad_w, cudaStream_t st);
-int launch_stage_w4(const float* w, float* w4, size_t taps, int C, cudaStream_t st);
+int launch_stage_w4(const float* w, float* w32, size_t rows, int S, int C, cudaStream_t st);
 int launch_unpad_reduce(const float* dw4, float* dw, size_t taps, int C, int splits, size_t split_stride,
                         cudaStream_t st);
 // dz = dy * act'(y), in place on dy

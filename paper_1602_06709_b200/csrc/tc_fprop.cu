@@ -31,6 +31,7 @@ constexpr int kBlockC = 32;                      // fp32 elements per 128-byte s
 constexpr int kABytes = kTileM * kBlockC * 4;    // 16 KB
 constexpr int kMaxStages = 8;
 constexpr int kSmemBudget = 224 * 1024;
+constexpr int kEpiStageBytes = 4 * 4096;
 
 struct FpropParams {
     int bw_log2, bh_log2;       // box of output pixels: bw x bh x (128 / (bw*bh))
@@ -61,6 +62,7 @@ tc_fprop_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
     const int lane = threadIdx.x & 31;
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     const uint32_t stage_bytes = kABytes + p.BN * 128;
+    uint8_t* epi_stage = smem + p.stages * stage_bytes;     // 4 warps x 4 KB epilogue transposition tiles
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < p.stages; ++s) {
@@ -187,24 +189,53 @@ tc_fprop_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
             if (!bounded_wait_warp(&tmem_full_bar[acc], acc_phase, &abort_flag, p.status, WAIT_EPI_TMEM_FULL)) break;
             tc_fence_after();
             const uint32_t t_row = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + acc * p.BN;
-            for (int ch = 0; ch < p.BN / 32; ++ch) {
-                uint32_t v[32];
-                tmem_ld_32x32(t_row + ch * 32, v);
-                tmem_ld_wait();
-                const int col0 = kt * p.BN + ch * 32;
-                if (valid && col0 < p.Kout) {
-                    float* dst = p.out + pix * p.Kout + col0;
-                    const float* msk = p.mask_src ? p.mask_src + pix * p.Kout + col0 : nullptr;
-                    if (vec_ok) {
+            if (vec_ok) {
+                // Coalesced path.  Each lane owns one row (pixel) of the accumulator, but a row's 32 columns
+                // are 128 contiguous bytes in global memory, so the chunk is first transposed through a
+                // 4 KB per-warp staging tile (XOR-swizzled 16-byte slots: conflict-free both ways) and then
+                // written 4 rows x 128 bytes per instruction: lane l handles columns 4*(l&7).. of rows
+                // (l>>3) + 4*i.  Bias, activation and the ReLU mask are applied on the way out.
+                size_t roff[8];
+                uint32_t vmask = 0;
 #pragma unroll
-                        for (int j = 0; j < 32; j += 4) {
-                            if (col0 + j < p.Kout) {
-                                float4 o = make_float4(__uint_as_float(v[j]), __uint_as_float(v[j + 1]),
-                                                       __uint_as_float(v[j + 2]), __uint_as_float(v[j + 3]));
-                                if (p.bias) {
-                                    const float4 b = __ldg(reinterpret_cast<const float4*>(p.bias + col0 + j));
-                                    o.x += b.x; o.y += b.y; o.z += b.z; o.w += b.w;
-                                }
+                for (int i = 0; i < 8; ++i) {
+                    const int src = (lane >> 3) + 4 * i;
+                    roff[i] = __shfl_sync(0xffffffffu, static_cast<unsigned long long>(pix * p.Kout), src);
+                    vmask |= (__shfl_sync(0xffffffffu, static_cast<int>(valid), src) ? 1u : 0u) << i;
+                }
+                uint8_t* stg = epi_stage + (warp - 2) * 4096;
+                const int cg = (lane & 7) * 4;
+                for (int ch = 0; ch < p.BN / 32; ++ch) {
+                    uint32_t v[32];
+                    tmem_ld_32x32(t_row + ch * 32, v);
+                    tmem_ld_wait();
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) {
+                        const int slot = j ^ (lane & 7);
+                        *reinterpret_cast<float4*>(stg + lane * 128 + slot * 16) =
+                            make_float4(__uint_as_float(v[4 * j]), __uint_as_float(v[4 * j + 1]),
+                                        __uint_as_float(v[4 * j + 2]), __uint_as_float(v[4 * j + 3]));
+                    }
+                    __syncwarp();
+                    const int col = kt * p.BN + ch * 32 + cg;
+                    if (col < p.Kout) {
+                        float4 b = make_float4(0.f, 0.f, 0.f, 0.f);
+                        if (p.bias) b = __ldg(reinterpret_cast<const float4*>(p.bias + col));
+                        float4 mk[8];
+                        if (p.mask_src) {
+#pragma unroll
+                            for (int i = 0; i < 8; ++i)
+                                mk[i] = ((vmask >> i) & 1u)
+                                            ? __ldg(reinterpret_cast<const float4*>(p.mask_src + roff[i] + col))
+                                            : make_float4(0.f, 0.f, 0.f, 0.f);
+                        }
+#pragma unroll
+                        for (int i = 0; i < 8; ++i) {
+                            const int rr = (lane >> 3) + 4 * i;
+                            const int slot = (lane & 7) ^ (rr & 7);
+                            float4 o = *reinterpret_cast<const float4*>(stg + rr * 128 + slot * 16);
+                            if ((vmask >> i) & 1u) {
+                                o.x += b.x; o.y += b.y; o.z += b.z; o.w += b.w;
                                 if (p.act == PCL_ACT_RELU) {
                                     o.x = fmaxf(o.x, 0.f); o.y = fmaxf(o.y, 0.f);
                                     o.z = fmaxf(o.z, 0.f); o.w = fmaxf(o.w, 0.f);
@@ -212,15 +243,25 @@ tc_fprop_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                                     o.x = 1.f / (1.f + __expf(-o.x)); o.y = 1.f / (1.f + __expf(-o.y));
                                     o.z = 1.f / (1.f + __expf(-o.z)); o.w = 1.f / (1.f + __expf(-o.w));
                                 }
-                                if (msk) {
-                                    const float4 mk = __ldg(reinterpret_cast<const float4*>(msk + j));
-                                    o.x = mk.x > 0.f ? o.x : 0.f; o.y = mk.y > 0.f ? o.y : 0.f;
-                                    o.z = mk.z > 0.f ? o.z : 0.f; o.w = mk.w > 0.f ? o.w : 0.f;
+                                if (p.mask_src) {
+                                    o.x = mk[i].x > 0.f ? o.x : 0.f; o.y = mk[i].y > 0.f ? o.y : 0.f;
+                                    o.z = mk[i].z > 0.f ? o.z : 0.f; o.w = mk[i].w > 0.f ? o.w : 0.f;
                                 }
-                                *reinterpret_cast<float4*>(dst + j) = o;
+                                *reinterpret_cast<float4*>(p.out + roff[i] + col) = o;
                             }
                         }
-                    } else {
+                    }
+                    __syncwarp();
+                }
+            } else {
+                for (int ch = 0; ch < p.BN / 32; ++ch) {
+                    uint32_t v[32];
+                    tmem_ld_32x32(t_row + ch * 32, v);
+                    tmem_ld_wait();
+                    const int col0 = kt * p.BN + ch * 32;
+                    if (valid && col0 < p.Kout) {
+                        float* dst = p.out + pix * p.Kout + col0;
+                        const float* msk = p.mask_src ? p.mask_src + pix * p.Kout + col0 : nullptr;
 #pragma unroll
                         for (int j = 0; j < 32; ++j) {
                             if (col0 + j < p.Kout) {
@@ -317,7 +358,7 @@ int launch_tc_fprop(const TcFpropArgs& a, cudaStream_t st) {
     p.N = a.N; p.P = a.P; p.Q = a.Q; p.Kout = a.Kout;
     p.act = a.act;
     const int stage_bytes = kABytes + p.BN * 128;
-    p.stages = kSmemBudget / stage_bytes;
+    p.stages = (kSmemBudget - kEpiStageBytes) / stage_bytes;
     if (p.stages > kMaxStages) p.stages = kMaxStages;
     p.tmem_cols = 32;
     while (p.tmem_cols < 2 * p.BN) p.tmem_cols *= 2;
@@ -327,7 +368,8 @@ int launch_tc_fprop(const TcFpropArgs& a, cudaStream_t st) {
 
     CUtensorMap tmA, tmB;
     {
-        const uint64_t dims[4] = {uint64_t(a.Cin), uint64_t(a.W), uint64_t(a.H), uint64_t(a.N)};
+        const uint64_t dims[4] = {uint64_t(a.in_inner ? a.in_inner : a.Cin), uint64_t(a.W), uint64_t(a.H),
+                                  uint64_t(a.N)};
         const uint64_t sw = a.in_stride_w ? uint64_t(a.in_stride_w) : uint64_t(a.Cin);
         const uint64_t sh = a.in_stride_h ? uint64_t(a.in_stride_h) : uint64_t(a.W) * a.Cin;
         const uint64_t sn = a.in_stride_n ? uint64_t(a.in_stride_n) : uint64_t(a.H) * a.W * a.Cin;
@@ -345,7 +387,7 @@ int launch_tc_fprop(const TcFpropArgs& a, cudaStream_t st) {
     }
     const long total = m_tiles * p.tiles_k;
     const int grid = int(total < g_sm_count ? total : g_sm_count);
-    const size_t smem = size_t(p.stages) * stage_bytes + 1024;
+    const size_t smem = size_t(p.stages) * stage_bytes + kEpiStageBytes + 1024;
     {
         LaunchScope scope(KID_TC_FPROP, 2.0 * a.N * a.P * a.Q * double(a.Kout) * a.Cin * a.R * a.S, st);
         tc_fprop_kernel<<<grid, 192, smem, st>>>(tmA, tmB, p);

@@ -351,7 +351,8 @@ int launch_tc_wgrad(const TcWgradArgs& a, cudaStream_t st) {
             int rc = make_tmap(&tmX, a.x, 5, dims, strides, box, true);
             if (rc != PCL_OK) return rc;
         } else {
-            const uint64_t dims[4] = {uint64_t(a.C), uint64_t(a.W), uint64_t(a.H), uint64_t(a.N)};
+            const uint64_t dims[4] = {uint64_t(a.x_inner ? a.x_inner : a.C), uint64_t(a.W), uint64_t(a.H),
+                                      uint64_t(a.N)};
             const uint64_t strides[3] = {sw * 4, sh * 4, sn * 4};
             const uint32_t box[4] = {32, uint32_t(bw), uint32_t(bh), uint32_t(bn)};
             int rc = make_tmap(&tmX, a.x, 4, dims, strides, box, true);
