@@ -86,25 +86,60 @@ __global__ void __launch_bounds__(256) act_grad_kernel(float* __restrict__ dy, c
     }
 }
 
-// partial[split][k] = sum over the split's rows of m[row][k]
-constexpr int kColsumRows = 4096;
+// partial[split][k] = sum over the split's rows of m[row][k].
+// A block covers a strip of up to 1024 columns (256 threads x float4 when K is a
+// multiple of 4) so that consecutive rows are read as whole contiguous runs; the
+// threads that share a column group are summed through shared memory in a fixed order.
+constexpr int kColsumRows = 2048;
+template <int VEC>
 __global__ void __launch_bounds__(256) colsum_kernel(const float* __restrict__ m, size_t rows, int K,
                                                      float* __restrict__ partial) {
-    const int k = blockIdx.x * 32 + (threadIdx.x & 31);
-    const int ty = threadIdx.x >> 5;
+    const int kv = K / VEC;                                  // column groups per row
+    const int strip = kv < 256 ? kv : 256;                   // column groups this block covers per row
+    const int lanes = 256 / strip;                           // rows handled concurrently
+    const int cg = blockIdx.x * strip + threadIdx.x % strip; // this thread's column group
+    const int rl = threadIdx.x / strip;
     const size_t r0 = size_t(blockIdx.y) * kColsumRows;
     size_t r1 = r0 + kColsumRows;
     if (r1 > rows) r1 = rows;
-    float acc = 0.f;
-    if (k < K)
-        for (size_t r = r0 + ty; r < r1; r += 8) acc += m[r * K + k];
-    __shared__ float red[8][32];
-    red[ty][threadIdx.x & 31] = acc;
+    float acc[VEC];
+#pragma unroll
+    for (int v = 0; v < VEC; ++v) acc[v] = 0.f;
+    if (cg < kv && rl < lanes) {
+        size_t r = r0 + rl;
+        for (; r + 3 * size_t(lanes) < r1; r += 4 * size_t(lanes)) {      // 4 independent loads in flight
+            float t[4][VEC];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const float* src = m + (r + u * size_t(lanes)) * K + size_t(cg) * VEC;
+                if (VEC == 4) {
+                    const float4 q = __ldcs(reinterpret_cast<const float4*>(src));
+                    t[u][0] = q.x; t[u][1 % VEC] = q.y; t[u][2 % VEC] = q.z; t[u][3 % VEC] = q.w;
+                } else {
+                    t[u][0] = __ldcs(src);
+                }
+            }
+#pragma unroll
+            for (int u = 0; u < 4; ++u)
+#pragma unroll
+                for (int v = 0; v < VEC; ++v) acc[v] += t[u][v];
+        }
+        for (; r < r1; r += lanes) {
+            const float* src = m + r * K + size_t(cg) * VEC;
+#pragma unroll
+            for (int v = 0; v < VEC; ++v) acc[v] += src[v];
+        }
+    }
+    __shared__ float red[256][VEC];
+#pragma unroll
+    for (int v = 0; v < VEC; ++v) red[threadIdx.x][v] = acc[v];
     __syncthreads();
-    if (ty == 0 && k < K) {
-        float s = 0.f;
-        for (int j = 0; j < 8; ++j) s += red[j][threadIdx.x];
-        partial[size_t(blockIdx.y) * K + k] = s;
+    if (rl == 0 && cg < kv) {
+        for (int l = 1; l < lanes; ++l)
+#pragma unroll
+            for (int v = 0; v < VEC; ++v) acc[v] += red[threadIdx.x + l * strip][v];
+#pragma unroll
+        for (int v = 0; v < VEC; ++v) partial[size_t(blockIdx.y) * K + size_t(cg) * VEC + v] = acc[v];
     }
 }
 
@@ -146,6 +181,13 @@ __device__ __forceinline__ void pool_route(float a, float b, float c, float d, f
     oa = arg == 0 ? g : 0.f; ob = arg == 1 ? g : 0.f; oc = arg == 2 ? g : 0.f; od = arg == 3 ? g : 0.f;
 }
 
+__device__ __forceinline__ float4 ld4(const float* p) { return *reinterpret_cast<const float4*>(p); }
+__device__ __forceinline__ float4 mask4(float4 v, float4 m) {
+    return make_float4(m.x > 0.f ? v.x : 0.f, m.y > 0.f ? v.y : 0.f, m.z > 0.f ? v.z : 0.f, m.w > 0.f ? v.w : 0.f);
+}
+
+// One thread per (pooled pixel, VEC channels): reads the 2x2 window of x and one dy, writes the 2x2 window of
+// dx.  When the ReLU mask source is x itself (the usual case: x is a ReLU output) it is not read again.
 template <int VEC>
 __global__ void __launch_bounds__(256) maxpool_bwd_kernel(const float* __restrict__ x, const float* __restrict__ dy,
                                                           const float* __restrict__ mask, float* __restrict__ dx,
@@ -154,32 +196,44 @@ __global__ void __launch_bounds__(256) maxpool_bwd_kernel(const float* __restric
     const size_t total = size_t(N) * Po * Qo * Cv;
     const size_t stride = size_t(gridDim.x) * blockDim.x;
     const size_t rowp = size_t(W) * C;
+    const bool mask_is_x = (mask == x);
     for (size_t i = size_t(blockIdx.x) * blockDim.x + threadIdx.x; i < total; i += stride) {
         const int cv = int(i % Cv); size_t t = i / Cv;
         const int q = int(t % Qo); t /= Qo;
         const int p = int(t % Po); const size_t n = t / Po;
         const size_t off = ((n * H + 2 * p) * W + 2 * q) * C + cv * VEC;
         const float* g = dy + ((n * Po + p) * Qo + q) * C + cv * VEC;
-        float xa[VEC], xb[VEC], xc[VEC], xd[VEC], oa[VEC], ob[VEC], oc[VEC], od[VEC], gv[VEC];
-#pragma unroll
-        for (int j = 0; j < VEC; ++j) {
-            xa[j] = x[off + j]; xb[j] = x[off + C + j]; xc[j] = x[off + rowp + j]; xd[j] = x[off + rowp + C + j];
-            gv[j] = g[j];
-        }
-#pragma unroll
-        for (int j = 0; j < VEC; ++j) pool_route(xa[j], xb[j], xc[j], xd[j], gv[j], oa[j], ob[j], oc[j], od[j]);
-        if (mask) {
-#pragma unroll
-            for (int j = 0; j < VEC; ++j) {
-                if (!(mask[off + j] > 0.f)) oa[j] = 0.f;
-                if (!(mask[off + C + j] > 0.f)) ob[j] = 0.f;
-                if (!(mask[off + rowp + j] > 0.f)) oc[j] = 0.f;
-                if (!(mask[off + rowp + C + j] > 0.f)) od[j] = 0.f;
+        if (VEC == 4) {
+            const float4 a = ld4(x + off), b = ld4(x + off + C), c = ld4(x + off + rowp), d = ld4(x + off + rowp + C);
+            const float4 gv = __ldcs(reinterpret_cast<const float4*>(g));
+            float4 oa, ob, oc, od;
+            pool_route(a.x, b.x, c.x, d.x, gv.x, oa.x, ob.x, oc.x, od.x);
+            pool_route(a.y, b.y, c.y, d.y, gv.y, oa.y, ob.y, oc.y, od.y);
+            pool_route(a.z, b.z, c.z, d.z, gv.z, oa.z, ob.z, oc.z, od.z);
+            pool_route(a.w, b.w, c.w, d.w, gv.w, oa.w, ob.w, oc.w, od.w);
+            if (mask) {
+                if (mask_is_x) {
+                    oa = mask4(oa, a); ob = mask4(ob, b); oc = mask4(oc, c); od = mask4(od, d);
+                } else {
+                    oa = mask4(oa, ld4(mask + off)); ob = mask4(ob, ld4(mask + off + C));
+                    oc = mask4(oc, ld4(mask + off + rowp)); od = mask4(od, ld4(mask + off + rowp + C));
+                }
             }
-        }
-#pragma unroll
-        for (int j = 0; j < VEC; ++j) {
-            dx[off + j] = oa[j]; dx[off + C + j] = ob[j]; dx[off + rowp + j] = oc[j]; dx[off + rowp + C + j] = od[j];
+            __stcs(reinterpret_cast<float4*>(dx + off), oa);
+            __stcs(reinterpret_cast<float4*>(dx + off + C), ob);
+            __stcs(reinterpret_cast<float4*>(dx + off + rowp), oc);
+            __stcs(reinterpret_cast<float4*>(dx + off + rowp + C), od);
+        } else {
+            const float a = x[off], b = x[off + C], c = x[off + rowp], d = x[off + rowp + C];
+            float oa, ob, oc, od;
+            pool_route(a, b, c, d, g[0], oa, ob, oc, od);
+            if (mask) {
+                if (!(mask[off] > 0.f)) oa = 0.f;
+                if (!(mask[off + C] > 0.f)) ob = 0.f;
+                if (!(mask[off + rowp] > 0.f)) oc = 0.f;
+                if (!(mask[off + rowp + C] > 0.f)) od = 0.f;
+            }
+            dx[off] = oa; dx[off + C] = ob; dx[off + rowp] = oc; dx[off + rowp + C] = od;
         }
     }
 }
@@ -357,10 +411,17 @@ int colsum_splits(size_t rows) { return int((rows + kColsumRows - 1) / kColsumRo
 int launch_colsum(const float* m, size_t rows, int K, float* partial, float* out, cudaStream_t st) {
     const int splits = colsum_splits(rows);
     if (splits > 65535) return PCL_ERR_UNSUPPORTED_SHAPE;
-    dim3 grid((K + 31) / 32, splits);
     {
         LaunchScope scope(KID_COLSUM, 4.0 * double(rows) * K, st);
-        colsum_kernel<<<grid, 256, 0, st>>>(m, rows, K, splits == 1 ? out : partial);
+        if (K % 4 == 0 && (reinterpret_cast<uintptr_t>(m) & 15) == 0) {
+            const int kv = K / 4, strip = kv < 256 ? kv : 256;
+            colsum_kernel<4><<<dim3((kv + strip - 1) / strip, splits), 256, 0, st>>>(m, rows, K,
+                                                                                     splits == 1 ? out : partial);
+        } else {
+            const int strip = K < 256 ? K : 256;
+            colsum_kernel<1><<<dim3((K + strip - 1) / strip, splits), 256, 0, st>>>(m, rows, K,
+                                                                                    splits == 1 ? out : partial);
+        }
     }
     if (cudaGetLastError() != cudaSuccess) return PCL_ERR_CUDA;
     if (splits > 1) return launch_reduce_splits(partial, out, size_t(K), splits, st);
@@ -386,7 +447,7 @@ int launch_maxpool_bwd(int N, int H, int W, int C, const float* x, const float* 
         // per output: 4 x read + 1 dy read + 4 dx written (the mask source is x itself in the step)
         LaunchScope scope(KID_MAXPOOL_BWD, 36.0 * double(outs) * C, st);
         if (C % 4 == 0)
-            maxpool_bwd_kernel<4><<<grid_for(outs * (C / 4), 256), 256, 0, st>>>(x, dy, mask, dx, N, H, W, C);
+            maxpool_bwd_kernel<4><<<grid_for(outs * (C / 4), 256, 16), 256, 0, st>>>(x, dy, mask, dx, N, H, W, C);
         else
             maxpool_bwd_kernel<1><<<grid_for(outs * C, 256), 256, 0, st>>>(x, dy, mask, dx, N, H, W, C);
     }
