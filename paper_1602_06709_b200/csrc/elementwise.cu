@@ -90,17 +90,17 @@ __global__ void __launch_bounds__(256) act_grad_kernel(float* __restrict__ dy, c
 // A block covers a strip of up to 1024 columns (256 threads x float4 when K is a
 // multiple of 4) so that consecutive rows are read as whole contiguous runs; the
 // threads that share a column group are summed through shared memory in a fixed order.
-constexpr int kColsumRows = 2048;
+constexpr int kColsumMinRows = 2048;   // rows per split, at least; grown so that there are at most ~1200 splits
 template <int VEC>
 __global__ void __launch_bounds__(256) colsum_kernel(const float* __restrict__ m, size_t rows, int K,
-                                                     float* __restrict__ partial) {
+                                                     float* __restrict__ partial, size_t rows_per_split) {
     const int kv = K / VEC;                                  // column groups per row
     const int strip = kv < 256 ? kv : 256;                   // column groups this block covers per row
     const int lanes = 256 / strip;                           // rows handled concurrently
     const int cg = blockIdx.x * strip + threadIdx.x % strip; // this thread's column group
     const int rl = threadIdx.x / strip;
-    const size_t r0 = size_t(blockIdx.y) * kColsumRows;
-    size_t r1 = r0 + kColsumRows;
+    const size_t r0 = size_t(blockIdx.y) * rows_per_split;
+    size_t r1 = r0 + rows_per_split;
     if (r1 > rows) r1 = rows;
     float acc[VEC];
 #pragma unroll
@@ -406,21 +406,30 @@ int launch_act_grad(float* dy, const float* y, size_t n, int act, cudaStream_t s
     return PCL_CHECK_LAUNCH();
 }
 
-int colsum_splits(size_t rows) { return int((rows + kColsumRows - 1) / kColsumRows); }
+static size_t colsum_rows_per_split(size_t rows) {
+    size_t per = (rows + 1183) / 1184;
+    if (per < size_t(kColsumMinRows)) per = kColsumMinRows;
+    return per;
+}
+int colsum_splits(size_t rows) {
+    const size_t per = colsum_rows_per_split(rows);
+    return int((rows + per - 1) / per);
+}
 
 int launch_colsum(const float* m, size_t rows, int K, float* partial, float* out, cudaStream_t st) {
     const int splits = colsum_splits(rows);
+    const size_t per = colsum_rows_per_split(rows);
     if (splits > 65535) return PCL_ERR_UNSUPPORTED_SHAPE;
     {
         LaunchScope scope(KID_COLSUM, 4.0 * double(rows) * K, st);
         if (K % 4 == 0 && (reinterpret_cast<uintptr_t>(m) & 15) == 0) {
             const int kv = K / 4, strip = kv < 256 ? kv : 256;
             colsum_kernel<4><<<dim3((kv + strip - 1) / strip, splits), 256, 0, st>>>(m, rows, K,
-                                                                                     splits == 1 ? out : partial);
+                                                                                     splits == 1 ? out : partial, per);
         } else {
             const int strip = K < 256 ? K : 256;
             colsum_kernel<1><<<dim3((K + strip - 1) / strip, splits), 256, 0, st>>>(m, rows, K,
-                                                                                    splits == 1 ? out : partial);
+                                                                                    splits == 1 ? out : partial, per);
         }
     }
     if (cudaGetLastError() != cudaSuccess) return PCL_ERR_CUDA;

@@ -7,13 +7,19 @@
 // NHWC tensors, so both operands are "MN-major": a TMA box {32 maps, 32 pixels}
 // lands in shared memory as 32 rows (one per pixel) of 128 bytes, swizzled in
 // 32-byte chunks, which is the MN-major operand layout tcgen05.mma takes for
-// 32-bit elements.  The x box is the
-// dy box shifted by the tap, with zero padding supplied by TMA's out-of-bounds
-// fill.
+// 32-bit elements.  The x box is the dy box shifted by the tap, with zero
+// padding supplied by TMA's out-of-bounds fill.
+//
+// Columns of the MMA are organised in "runs": a run is L consecutive 32-map
+// groups of x for one tap (L <= 8), fetched by one TMA instruction through a
+// 5-D view {32 maps, w, h, n, group} of the tensor.  A CTA accumulates up to 8
+// groups (N <= 256) = several runs, which may belong to different taps: layers
+// with few input maps (C = 64: 2 groups per tap) then still fill a 128 x 192 or
+// 128 x 256 tile and read dy once for 3-4 taps instead of once per tap.
 //
 // The output is tiny compared with the reduction (Sec. 2.4/2.5 make the same
 // observation), so the pixel range is split across CTAs ("privatise and
-// reduce"): a work item is (128-row k tile, tap, c tile, pixel split); each CTA
+// reduce"): a work item is (128-row k tile, block of runs, pixel split); each CTA
 // accumulates its item in TMEM and either writes a partial tile to the
 // workspace (second pass adds the splits in a fixed order) or adds it to dw with
 // fp32 atomics.
@@ -33,14 +39,18 @@ constexpr int kSmemBudget = 224 * 1024;
 struct WgradParams {
     int bw_log2, bh_log2;     // pixel box bw x bh x (32/(bw*bh))
     int boxes_q, boxes_p, boxes_n;
-    int k_tiles, c_tiles, BNc;
+    int k_tiles;
+    int L;                    // 32-map groups per run
+    int runs_per_tap;         // ceil(C/32) / L
+    int total_runs;           // R*S*runs_per_tap
+    int rpi;                  // runs per work item (rpi*L <= 8)
+    int run_blocks;           // ceil(total_runs / rpi)
     int R, S, pad_h, pad_w;
     int K, C;
     int splits, boxes_per_split;
     int stages, tmem_cols;
     int use_atomics;
-    int tap_groups;           // column group g of the MMA = tap row g (few-channel first layers)
-    int grouped;              // 5-D tensor maps: all 32-map groups of an operand arrive with one TMA instruction
+    int grouped;              // 5-D tensor maps (one TMA instruction per operand run) or 4-D per-group boxes (L == 1)
     float* out;               // dw, or the partial-sum workspace [splits][K*R*S*C]
     size_t split_stride;      // K*R*S*C (0 when writing straight to dw)
     unsigned int* status;     // device status word
@@ -58,8 +68,17 @@ tc_wgrad_kernel(const __grid_constant__ CUtensorMap tmDy, const __grid_constant_
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-    const int b_groups = p.BNc / 32;
-    const uint32_t stage_bytes = kABytes + b_groups * kGroupBytes;
+
+    // work item of this CTA
+    int item = blockIdx.x;
+    const int split = item % p.splits;   item /= p.splits;
+    const int rb = item % p.run_blocks;
+    const int kt = item / p.run_blocks;
+    const int run0 = rb * p.rpi;
+    const int nruns = (run0 + p.rpi <= p.total_runs) ? p.rpi : p.total_runs - run0;
+    const int n_groups = nruns * p.L;                 // 32-column groups of this item's MMA
+    const uint32_t stage_bytes = kABytes + p.rpi * p.L * kGroupBytes;   // slot size (same for every item)
+    const uint32_t tx_bytes = kABytes + n_groups * kGroupBytes;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < p.stages; ++s) {
@@ -81,14 +100,6 @@ tc_wgrad_kernel(const __grid_constant__ CUtensorMap tmDy, const __grid_constant_
     tc_fence_after();
     const uint32_t tmem_base = tmem_base_slot;
 
-    // work item of this CTA
-    int item = blockIdx.x;
-    const int split = item % p.splits;   item /= p.splits;
-    const int ct = item % p.c_tiles;     item /= p.c_tiles;
-    const int taps = p.tap_groups ? 1 : p.R * p.S;
-    const int tap = item % taps;
-    const int kt = item / taps;
-    const int r = tap / p.S, s = tap % p.S;
     const int total_boxes = p.boxes_q * p.boxes_p * p.boxes_n;
     const int box_begin = split * p.boxes_per_split;
     int box_end = box_begin + p.boxes_per_split;
@@ -102,33 +113,51 @@ tc_wgrad_kernel(const __grid_constant__ CUtensorMap tmDy, const __grid_constant_
             uint32_t phase = 0;
             int issued = 0;
             bool ok = true;
+            // Per-run TMA coordinates are fixed for the item: decode them once (the k loop must stay
+            // free of integer divisions, this thread paces the whole pipeline).
+            int run_dw[8], run_dh[8], run_c[8];
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+                const int run = run0 + (j < nruns ? j : 0);
+                const int tap = run / p.runs_per_tap;
+                const int cg0 = (run - tap * p.runs_per_tap) * p.L;
+                const int r = tap / p.S, s = tap - r * p.S;
+                run_dw[j] = s - p.pad_w;
+                run_dh[j] = r - p.pad_h;
+                run_c[j] = p.grouped ? cg0 : cg0 * 32;
+            }
+            int qi = box_begin % p.boxes_q;
+            int pi = (box_begin / p.boxes_q) % p.boxes_p;
+            int ni = box_begin / (p.boxes_q * p.boxes_p);
+            const uint32_t run_bytes = p.L * kGroupBytes;
             for (int b = box_begin; b < box_end; ++b) {
-                int m = b;
-                const int q0 = (m % p.boxes_q) * bw;  m /= p.boxes_q;
-                const int p0 = (m % p.boxes_p) * bh;
-                const int n0 = (m / p.boxes_p) * bn;
+                const int q0 = qi * bw, p0 = pi * bh, n0 = ni * bn;
+                if (++qi == p.boxes_q) { qi = 0; if (++pi == p.boxes_p) { pi = 0; ++ni; } }
                 if (!bounded_wait(&empty_bar[stage], phase ^ 1u, &abort_flag, p.status, WAIT_PRODUCER_EMPTY)) { ok = false; break; }
                 uint8_t* dst = smem + stage * stage_bytes;
-                mbar_expect_tx(&full_bar[stage], stage_bytes);
+                mbar_expect_tx(&full_bar[stage], tx_bytes);
                 if (p.grouped) {
                     tma_load_5d(dst, &tmDy, &full_bar[stage], 0, q0, p0, n0, kt * 4);
-                    tma_load_5d(dst + kABytes, &tmX, &full_bar[stage], 0, q0 + s - p.pad_w, p0 + r - p.pad_h, n0,
-                                ct * b_groups);
+#pragma unroll
+                    for (int j = 0; j < 8; ++j)
+                        if (j < nruns)
+                            tma_load_5d(dst + kABytes + j * run_bytes, &tmX, &full_bar[stage], 0, q0 + run_dw[j],
+                                        p0 + run_dh[j], n0, run_c[j]);
                 } else {
 #pragma unroll
-                for (int g = 0; g < 4; ++g)
-                    tma_load_4d(dst + g * kGroupBytes, &tmDy, &full_bar[stage], kt * 128 + g * 32, q0, p0, n0);
-                for (int g = 0; g < b_groups; ++g) {
-                    const int cc = p.tap_groups ? 0 : ct * p.BNc + g * 32;
-                    const int rr = p.tap_groups ? g : r;
-                    tma_load_4d(dst + kABytes + g * kGroupBytes, &tmX, &full_bar[stage], cc, q0 + s - p.pad_w,
-                                p0 + rr - p.pad_h, n0);
-                }
+                    for (int g = 0; g < 4; ++g)
+                        tma_load_4d(dst + g * kGroupBytes, &tmDy, &full_bar[stage], kt * 128 + g * 32, q0, p0, n0);
+#pragma unroll
+                    for (int j = 0; j < 8; ++j)
+                        if (j < nruns)
+                            tma_load_4d(dst + kABytes + j * run_bytes, &tmX, &full_bar[stage], run_c[j],
+                                        q0 + run_dw[j], p0 + run_dh[j], n0);
                 }
                 ++issued;
                 if (++stage == p.stages) { stage = 0; phase ^= 1u; }
             }
             if (!ok) {
+                // Gave up: copies already issued still land in this CTA's shared memory; wait (bounded) for them.
                 const int pending = issued < p.stages ? issued : p.stages;
                 for (int j = 0; j < pending; ++j) {
                     if (--stage < 0) { stage = p.stages - 1; phase ^= 1u; }
@@ -138,7 +167,7 @@ tc_wgrad_kernel(const __grid_constant__ CUtensorMap tmDy, const __grid_constant_
             }
         }
     } else if (warp == 1) {
-        const uint32_t idesc = make_idesc_tf32(p.BNc, true, true);
+        const uint32_t idesc = make_idesc_tf32(n_groups * 32, true, true);
         int stage = 0;
         uint32_t phase = 0;
         bool ok = true;
@@ -170,10 +199,12 @@ tc_wgrad_kernel(const __grid_constant__ CUtensorMap tmDy, const __grid_constant_
         if (bounded_wait_warp(&tmem_full_bar, 0, &abort_flag, p.status, WAIT_EPI_TMEM_FULL)) {
             tc_fence_after();
             const uint32_t t_row = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16);
-            const size_t krow = static_cast<size_t>(valid ? k : 0) * p.R;
-            for (int ch = 0; ch < b_groups; ++ch) {
-                const int rr = p.tap_groups ? ch : r;
-                float* base = p.out + static_cast<size_t>(split) * p.split_stride + ((krow + rr) * p.S + s) * p.C;
+            const size_t krow = static_cast<size_t>(valid ? k : 0) * p.R * p.S;
+            for (int ch = 0; ch < n_groups; ++ch) {
+                const int run = run0 + ch / p.L;
+                const int tap = run / p.runs_per_tap;
+                const int c0 = ((run - tap * p.runs_per_tap) * p.L + ch % p.L) * 32;
+                float* dst = p.out + static_cast<size_t>(split) * p.split_stride + (krow + tap) * p.C + c0;
                 uint32_t v[32];
                 if (kiters > 0) {
                     tmem_ld_32x32(t_row + ch * 32, v);
@@ -182,9 +213,7 @@ tc_wgrad_kernel(const __grid_constant__ CUtensorMap tmDy, const __grid_constant_
 #pragma unroll
                     for (int j = 0; j < 32; ++j) v[j] = 0u;
                 }
-                const int c0 = p.tap_groups ? 0 : ct * p.BNc + ch * 32;
                 if (valid && c0 < p.C) {
-                    float* dst = base + c0;
                     if (p.use_atomics) {
 #pragma unroll
                         for (int j = 0; j < 32; ++j)
@@ -228,18 +257,37 @@ void choose_pixel_box(int P, int Q, int N, int* bw_log2, int* bh_log2) {
     *bh_log2 = best_h;
 }
 
-int choose_bnc(int C) {
-    const int c32 = (C + 31) / 32 * 32;
-    int bn = c32 < 256 ? c32 : 256;
-    const int tiles = (C + bn - 1) / bn;
-    return ((C + tiles - 1) / tiles + 31) / 32 * 32;
-}
-
 long total_pixel_boxes(int N, int P, int Q) {
     int lw, lh;
     choose_pixel_box(P, Q, N, &lw, &lh);
     const long bw = 1L << lw, bh = 1L << lh, bn = kPix / (bw * bh);
     return ((Q + bw - 1) / bw) * ((P + bh - 1) / bh) * ((N + bn - 1) / bn);
+}
+
+// How the columns of a layer are cut into runs and work items.
+struct RunPlan {
+    int grouped, L, runs_per_tap, total_runs, rpi, run_blocks;
+};
+
+RunPlan plan_runs(int C, int K, int R, int S, int tap_groups) {
+    RunPlan r{};
+    const int cgroups = (C + 31) / 32;
+    r.grouped = (!tap_groups && C % 32 == 0 && K % 32 == 0) ? 1 : 0;
+    r.L = 1;
+    if (r.grouped)
+        for (int l = 8; l >= 1; --l)
+            if (cgroups % l == 0) { r.L = l; break; }
+    r.runs_per_tap = cgroups / r.L;
+    r.total_runs = R * S * r.runs_per_tap;
+    const int rpi_max = 8 / r.L;
+    if (tap_groups) {
+        r.rpi = r.total_runs;                        // all tap rows of a k tile in one item
+    } else {
+        const int blocks = (r.total_runs + rpi_max - 1) / rpi_max;
+        r.rpi = (r.total_runs + blocks - 1) / blocks;   // balanced: 18 runs -> 3 x 6 rather than 8 + 8 + 2
+    }
+    r.run_blocks = (r.total_runs + r.rpi - 1) / r.rpi;
+    return r;
 }
 
 int g_sm_count = 0;
@@ -264,8 +312,8 @@ bool tc_wgrad_eligible(const TcWgradArgs& a) {
 }
 
 int tc_wgrad_splits(int N, int P, int Q, int C, int K, int R, int S, int tap_groups) {
-    const int bnc = choose_bnc(C);
-    const long items = tap_groups ? long((K + 127) / 128) : long((K + 127) / 128) * R * S * ((C + bnc - 1) / bnc);
+    const RunPlan rp = plan_runs(C, K, R, S, tap_groups);
+    const long items = long((K + 127) / 128) * rp.run_blocks;
     const long boxes = total_pixel_boxes(N, P, Q);
     long splits = sm_count() / items;
     if (splits < 1) splits = 1;
@@ -293,19 +341,20 @@ int launch_tc_wgrad(const TcWgradArgs& a, cudaStream_t st) {
     p.boxes_n = (a.N + bn - 1) / bn;
     const long boxes = long(p.boxes_q) * p.boxes_p * p.boxes_n;
     if (boxes > 0x7fffffffL) return PCL_ERR_UNSUPPORTED_SHAPE;
-    p.tap_groups = a.tap_groups;
-    p.BNc = a.tap_groups ? a.R * 32 : choose_bnc(a.C);
-    p.c_tiles = a.tap_groups ? 1 : (a.C + p.BNc - 1) / p.BNc;
+    const RunPlan rp = plan_runs(a.C, a.K, a.R, a.S, a.tap_groups);
+    p.grouped = rp.grouped; p.L = rp.L; p.runs_per_tap = rp.runs_per_tap; p.total_runs = rp.total_runs;
+    p.rpi = rp.rpi; p.run_blocks = rp.run_blocks;
     p.k_tiles = (a.K + 127) / 128;
     p.R = a.R; p.S = a.S; p.pad_h = a.pad_h; p.pad_w = a.pad_w;
     p.K = a.K; p.C = a.C;
     p.splits = a.splits;
     p.boxes_per_split = int((boxes + p.splits - 1) / p.splits);
-    const int stage_bytes = kABytes + (p.BNc / 32) * kGroupBytes;
+    const int max_groups = p.rpi * p.L;
+    const int stage_bytes = kABytes + max_groups * kGroupBytes;
     p.stages = kSmemBudget / stage_bytes;
     if (p.stages > kMaxStages) p.stages = kMaxStages;
     p.tmem_cols = 32;
-    while (p.tmem_cols < p.BNc) p.tmem_cols *= 2;
+    while (p.tmem_cols < max_groups * 32) p.tmem_cols *= 2;
     p.status = device_status_ptr();
     if (!p.status) return PCL_ERR_CUDA;
     const size_t dw_elems = size_t(a.K) * a.R * a.S * a.C;
@@ -319,10 +368,9 @@ int launch_tc_wgrad(const TcWgradArgs& a, cudaStream_t st) {
         if (rc != PCL_OK) return rc;
     }
 
-    // When both map counts are multiples of 32, view each tensor as 5-D {32 maps, w, h, n, group} (the group
-    // dimension has a 128-byte stride) so that one TMA instruction brings all groups of an operand, laid out
-    // [group][pixel][32 maps] in shared memory exactly as the per-group boxes would be.
-    p.grouped = (!a.tap_groups && a.C % 32 == 0 && a.K % 32 == 0) ? 1 : 0;
+    // When both map counts are multiples of 32, each tensor is viewed as 5-D {32 maps, w, h, n, group} (the
+    // group dimension has a 128-byte stride) so that one TMA instruction brings a whole run of groups, laid
+    // out [group][pixel][32 maps] in shared memory exactly as per-group boxes would be.
     CUtensorMap tmDy, tmX;
     {
         const uint64_t sw = uint64_t(a.K), sh = uint64_t(a.Q) * a.K, sn = uint64_t(a.P) * a.Q * a.K;
@@ -347,7 +395,7 @@ int launch_tc_wgrad(const TcWgradArgs& a, cudaStream_t st) {
         if (p.grouped) {
             const uint64_t dims[5] = {32, uint64_t(a.W), uint64_t(a.H), uint64_t(a.N), uint64_t(a.C / 32)};
             const uint64_t strides[4] = {sw * 4, sh * 4, sn * 4, 128};
-            const uint32_t box[5] = {32, uint32_t(bw), uint32_t(bh), uint32_t(bn), uint32_t(p.BNc / 32)};
+            const uint32_t box[5] = {32, uint32_t(bw), uint32_t(bh), uint32_t(bn), uint32_t(p.L)};
             int rc = make_tmap(&tmX, a.x, 5, dims, strides, box, true);
             if (rc != PCL_OK) return rc;
         } else {
@@ -359,7 +407,7 @@ int launch_tc_wgrad(const TcWgradArgs& a, cudaStream_t st) {
             if (rc != PCL_OK) return rc;
         }
     }
-    const long items = long(p.k_tiles) * (a.tap_groups ? 1 : a.R * a.S) * p.c_tiles * p.splits;
+    const long items = long(p.k_tiles) * p.run_blocks * p.splits;
     if (items > 0x7fffffffL) return PCL_ERR_UNSUPPORTED_SHAPE;
     const size_t smem = size_t(p.stages) * stage_bytes + 1024;
     {
