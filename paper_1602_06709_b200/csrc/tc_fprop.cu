@@ -13,10 +13,11 @@
 // im2col matrix is never materialised and zero padding is TMA's out-of-bounds
 // fill.  B is a 3-D TMA box {32 c, 1 tap, BN k} of the weights.
 //
-// Warp roles (192 threads, persistent over tiles):
+// Warp roles (320 threads, persistent over tiles):
 //   warp 0     TMA producer, fills a ring of `stages` {A 16 KB, B BN*128 B} slots
 //   warp 1     allocates TMEM, issues tcgen05.mma kind::tf32 (4 per slot, K = 8 each)
-//   warps 2-5  epilogue: TMEM -> registers -> bias/activation/mask -> global
+//   warps 2-9  epilogue: TMEM -> registers -> bias/activation/mask -> global (two warps per TMEM
+//              lane quarter; a lone warp per scheduler is latency-bound on narrow layers)
 // Two TMEM accumulators (2 x BN columns) let the epilogue of tile i overlap the
 // main loop of tile i+1.
 #include "pcl_internal.h"
@@ -31,7 +32,9 @@ constexpr int kBlockC = 32;                      // fp32 elements per 128-byte s
 constexpr int kABytes = kTileM * kBlockC * 4;    // 16 KB
 constexpr int kMaxStages = 8;
 constexpr int kSmemBudget = 224 * 1024;
-constexpr int kEpiStageBytes = 4 * 4096;
+constexpr int kEpiWarps = 8;                    // two per TMEM lane quarter, splitting the column chunks
+constexpr int kEpiStageBytes = kEpiWarps * 4096;
+constexpr int kThreads = (2 + kEpiWarps) * 32;
 
 struct FpropParams {
     int bw_log2, bh_log2;       // box of output pixels: bw x bh x (128 / (bw*bh))
@@ -48,7 +51,33 @@ struct FpropParams {
     unsigned int* status;       // device status word
 };
 
-__global__ void __launch_bounds__(192, 1)
+// Walks the persistent tile sequence t = blockIdx.x, blockIdx.x + gridDim.x, ... and keeps the tile's
+// coordinates (k tile, q tile, p tile, n tile) in mixed-radix counters, so that no role pays integer
+// divisions per tile.
+struct TileIter {
+    int t, kt, qi, pi, ni;
+    int step, dk, dq, dp, dn;
+    __device__ void init(const FpropParams& p, int first, int stride) {
+        t = first; step = stride;
+        int m = first;
+        kt = m % p.tiles_k; m /= p.tiles_k;
+        qi = m % p.tiles_q; m /= p.tiles_q;
+        pi = m % p.tiles_p; ni = m / p.tiles_p;
+        m = stride;
+        dk = m % p.tiles_k; m /= p.tiles_k;
+        dq = m % p.tiles_q; m /= p.tiles_q;
+        dp = m % p.tiles_p; dn = m / p.tiles_p;
+    }
+    __device__ void next(const FpropParams& p) {
+        t += step;
+        kt += dk; int c = kt >= p.tiles_k; kt -= c ? p.tiles_k : 0;
+        qi += dq + c; c = qi >= p.tiles_q; qi -= c ? p.tiles_q : 0;
+        pi += dp + c; c = pi >= p.tiles_p; pi -= c ? p.tiles_p : 0;
+        ni += dn + c;
+    }
+};
+
+__global__ void __launch_bounds__(kThreads, 1)
 tc_fprop_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, FpropParams p) {
     extern __shared__ uint8_t smem_raw[];
     __shared__ uint64_t full_bar[kMaxStages];
@@ -71,7 +100,7 @@ tc_fprop_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
         }
         for (int a = 0; a < 2; ++a) {
             mbar_init(&tmem_full_bar[a], 1);
-            mbar_init(&tmem_empty_bar[a], 4);
+            mbar_init(&tmem_empty_bar[a], kEpiWarps);
         }
         abort_flag = 0;
         mbar_fence_init();
@@ -100,12 +129,10 @@ tc_fprop_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
             uint32_t phase = 0;
             int issued = 0;
             bool ok = true;
-            for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
-                const int kt = t % p.tiles_k;
-                int m = t / p.tiles_k;
-                const int q0 = (m % p.tiles_q) * bw;  m /= p.tiles_q;
-                const int p0 = (m % p.tiles_p) * bh;
-                const int n0 = (m / p.tiles_p) * bn;
+            TileIter it;
+            for (it.init(p, blockIdx.x, gridDim.x); it.t < total_tiles && ok; it.next(p)) {
+                const int kt = it.kt;
+                const int q0 = it.qi * bw, p0 = it.pi * bh, n0 = it.ni * bn;
                 for (int r = 0; r < p.R && ok; ++r)
                     for (int s = 0; s < p.S && ok; ++s)
                         for (int cb = 0; cb < p.cblocks; ++cb) {
@@ -170,20 +197,21 @@ tc_fprop_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
     } else {
         // ------------------------------------------------------------ epilogue
         const int quarter = warp & 3;           // TMEM lanes 32*quarter .. +31
+        const int chalf = (warp - 2) >> 2;      // which half of the 32-column chunks this warp takes
         const int row = quarter * 32 + lane;    // row of the tile = pixel of the box
         const int iw = row & (bw - 1);
         const int ih = (row >> p.bw_log2) & (bh - 1);
         const int in_ = row >> (p.bw_log2 + p.bh_log2);
         const bool vec_ok = (p.Kout & 3) == 0;
         int tile_cnt = 0;
-        for (int t = blockIdx.x; t < total_tiles; t += gridDim.x, ++tile_cnt) {
+        TileIter it;
+        for (it.init(p, blockIdx.x, gridDim.x); it.t < total_tiles; it.next(p), ++tile_cnt) {
             const int acc = tile_cnt & 1;
             const uint32_t acc_phase = (tile_cnt >> 1) & 1;
-            const int kt = t % p.tiles_k;
-            int m = t / p.tiles_k;
-            const int q = (m % p.tiles_q) * bw + iw;  m /= p.tiles_q;
-            const int pp = (m % p.tiles_p) * bh + ih;
-            const int n = (m / p.tiles_p) * bn + in_;
+            const int kt = it.kt;
+            const int q = it.qi * bw + iw;
+            const int pp = it.pi * bh + ih;
+            const int n = it.ni * bn + in_;
             const bool valid = (q < p.Q) && (pp < p.P) && (n < p.N);
             const size_t pix = (static_cast<size_t>(n) * p.P + pp) * p.Q + q;
             if (!bounded_wait_warp(&tmem_full_bar[acc], acc_phase, &abort_flag, p.status, WAIT_EPI_TMEM_FULL)) break;
@@ -205,7 +233,7 @@ tc_fprop_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                 }
                 uint8_t* stg = epi_stage + (warp - 2) * 4096;
                 const int cg = (lane & 7) * 4;
-                for (int ch = 0; ch < p.BN / 32; ++ch) {
+                for (int ch = chalf; ch < p.BN / 32; ch += 2) {
                     uint32_t v[32];
                     tmem_ld_32x32(t_row + ch * 32, v);
                     tmem_ld_wait();
@@ -254,7 +282,7 @@ tc_fprop_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                     __syncwarp();
                 }
             } else {
-                for (int ch = 0; ch < p.BN / 32; ++ch) {
+                for (int ch = chalf; ch < p.BN / 32; ch += 2) {
                     uint32_t v[32];
                     tmem_ld_32x32(t_row + ch * 32, v);
                     tmem_ld_wait();
@@ -390,7 +418,7 @@ int launch_tc_fprop(const TcFpropArgs& a, cudaStream_t st) {
     const size_t smem = size_t(p.stages) * stage_bytes + kEpiStageBytes + 1024;
     {
         LaunchScope scope(KID_TC_FPROP, 2.0 * a.N * a.P * a.Q * double(a.Kout) * a.Cin * a.R * a.S, st);
-        tc_fprop_kernel<<<grid, 192, smem, st>>>(tmA, tmB, p);
+        tc_fprop_kernel<<<grid, kThreads, smem, st>>>(tmA, tmB, p);
     }
     return cudaGetLastError() == cudaSuccess ? PCL_OK : PCL_ERR_CUDA;
 }
