@@ -20,6 +20,8 @@
 //              lane quarter; a lone warp per scheduler is latency-bound on narrow layers)
 // Two TMEM accumulators (2 x BN columns) let the epilogue of tile i overlap the
 // main loop of tile i+1.
+#include <stdlib.h>
+
 #include "pcl_internal.h"
 #include "pcl_ptx.cuh"
 
@@ -45,6 +47,15 @@ struct FpropParams {
     int act;
     int stages;
     int tmem_cols;
+    int tw, th, tn;             // pixels a tile spans in q, p, n (= the box, or 2 x the box in one direction when MT = 2)
+    // Halo mode (R*S > 1): the A operand of ALL taps of a channel block comes from one haloed input patch
+    // of (th + R - 1) x (tw + S - 1) pixels, loaded once; a tap is a row-shifted view of it.  A tile is MT
+    // (1 or 2) boxes of 8 x 16 pixels that share every weight tile.
+    int halo, MT;
+    int PW;                     // patch width in pixels
+    int patch_bytes, a_buf_bytes, NA;
+    int half_off_bytes;         // offset of the second box inside the patch
+    int half_dq, half_dp;       // pixel offset of the second box inside the tile
     const float* bias;
     const float* mask_src;
     float* out;
@@ -82,6 +93,8 @@ tc_fprop_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
     extern __shared__ uint8_t smem_raw[];
     __shared__ uint64_t full_bar[kMaxStages];
     __shared__ uint64_t empty_bar[kMaxStages];
+    __shared__ uint64_t fullA_bar[4];
+    __shared__ uint64_t emptyA_bar[4];
     __shared__ uint64_t tmem_full_bar[2];
     __shared__ uint64_t tmem_empty_bar[2];
     __shared__ uint32_t tmem_base_slot;
@@ -90,13 +103,20 @@ tc_fprop_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-    const uint32_t stage_bytes = kABytes + p.BN * 128;
-    uint8_t* epi_stage = smem + p.stages * stage_bytes;     // 4 warps x 4 KB epilogue transposition tiles
+    // plain mode: ring of {A 16 KB, B BN*128 B} slots.  halo mode: NA patch buffers, then a ring of B slots.
+    const uint32_t b_bytes = p.BN * 128;
+    const uint32_t stage_bytes = p.halo ? b_bytes : kABytes + b_bytes;
+    uint8_t* b_ring = smem + (p.halo ? p.NA * p.a_buf_bytes : kABytes);
+    uint8_t* epi_stage = smem + (p.halo ? p.NA * p.a_buf_bytes : 0) + p.stages * stage_bytes;   // 8 x 4 KB
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < p.stages; ++s) {
             mbar_init(&full_bar[s], 1);
             mbar_init(&empty_bar[s], 1);
+        }
+        for (int a = 0; a < 4; ++a) {
+            mbar_init(&fullA_bar[a], 1);
+            mbar_init(&emptyA_bar[a], 1);
         }
         for (int a = 0; a < 2; ++a) {
             mbar_init(&tmem_full_bar[a], 1);
@@ -117,7 +137,6 @@ tc_fprop_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
     const uint32_t tmem_base = tmem_base_slot;
 
     const int bw = 1 << p.bw_log2, bh = 1 << p.bh_log2;
-    const int bn = kTileM >> (p.bw_log2 + p.bh_log2);
     const int m_tiles = p.tiles_q * p.tiles_p * p.tiles_n;
     const int total_tiles = m_tiles * p.tiles_k;
     const int kiters = p.R * p.S * p.cblocks;
@@ -125,39 +144,71 @@ tc_fprop_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
     if (warp == 0) {
         // ------------------------------------------------------------ producer
         if (lane == 0) {
-            int stage = 0;
+            int stage = 0, issued = 0;
             uint32_t phase = 0;
-            int issued = 0;
+            int a_slot = 0, issuedA = 0;
+            uint32_t phaseA = 0;
             bool ok = true;
             TileIter it;
             for (it.init(p, blockIdx.x, gridDim.x); it.t < total_tiles && ok; it.next(p)) {
                 const int kt = it.kt;
-                const int q0 = it.qi * bw, p0 = it.pi * bh, n0 = it.ni * bn;
-                for (int r = 0; r < p.R && ok; ++r)
-                    for (int s = 0; s < p.S && ok; ++s)
-                        for (int cb = 0; cb < p.cblocks; ++cb) {
+                const int q0 = it.qi * p.tw, p0 = it.pi * p.th, n0 = it.ni * p.tn;
+                if (p.halo) {
+                    for (int cb = 0; cb < p.cblocks && ok; ++cb) {
+                        if (!bounded_wait(&emptyA_bar[a_slot], phaseA ^ 1u, &abort_flag, p.status, WAIT_PRODUCER_EMPTY)) {
+                            ok = false;
+                            break;
+                        }
+                        mbar_expect_tx(&fullA_bar[a_slot], p.patch_bytes);
+                        tma_load_4d(smem + a_slot * p.a_buf_bytes, &tmA, &fullA_bar[a_slot], cb * kBlockC,
+                                    q0 - p.pad_w, p0 - p.pad_h, n0);
+                        ++issuedA;
+                        if (++a_slot == p.NA) { a_slot = 0; phaseA ^= 1u; }
+                        for (int tap = 0; tap < p.R * p.S; ++tap) {
                             if (!bounded_wait(&empty_bar[stage], phase ^ 1u, &abort_flag, p.status, WAIT_PRODUCER_EMPTY)) {
                                 ok = false;
                                 break;
                             }
-                            uint8_t* a_dst = smem + stage * stage_bytes;
-                            mbar_expect_tx(&full_bar[stage], stage_bytes);
-                            tma_load_4d(a_dst, &tmA, &full_bar[stage], cb * kBlockC, q0 + s - p.pad_w,
-                                        p0 + r - p.pad_h, n0);
-                            tma_load_3d(a_dst + kABytes, &tmB, &full_bar[stage], cb * kBlockC, r * p.S + s,
+                            mbar_expect_tx(&full_bar[stage], b_bytes);
+                            tma_load_3d(b_ring + stage * stage_bytes, &tmB, &full_bar[stage], cb * kBlockC, tap,
                                         kt * p.BN);
                             ++issued;
                             if (++stage == p.stages) { stage = 0; phase ^= 1u; }
                         }
+                    }
+                } else {
+                    for (int r = 0; r < p.R && ok; ++r)
+                        for (int s = 0; s < p.S && ok; ++s)
+                            for (int cb = 0; cb < p.cblocks; ++cb) {
+                                if (!bounded_wait(&empty_bar[stage], phase ^ 1u, &abort_flag, p.status, WAIT_PRODUCER_EMPTY)) {
+                                    ok = false;
+                                    break;
+                                }
+                                uint8_t* a_dst = smem + stage * stage_bytes;
+                                mbar_expect_tx(&full_bar[stage], stage_bytes);
+                                tma_load_4d(a_dst, &tmA, &full_bar[stage], cb * kBlockC, q0 + s - p.pad_w,
+                                            p0 + r - p.pad_h, n0);
+                                tma_load_3d(a_dst + kABytes, &tmB, &full_bar[stage], cb * kBlockC, r * p.S + s,
+                                            kt * p.BN);
+                                ++issued;
+                                if (++stage == p.stages) { stage = 0; phase ^= 1u; }
+                            }
+                }
             }
             if (!ok) {
                 // Gave up: the copies already issued still land in this CTA's shared
                 // memory, so wait (bounded) for each armed slot before leaving.
-                const int pending = issued < p.stages ? issued : p.stages;
+                int pending = issued < p.stages ? issued : p.stages;
                 for (int j = 0; j < pending; ++j) {
                     if (--stage < 0) { stage = p.stages - 1; phase ^= 1u; }
                     for (uint32_t spin = 0; spin < (1u << 20); ++spin)
                         if (mbar_try_wait(&full_bar[stage], phase)) break;
+                }
+                pending = issuedA < p.NA ? issuedA : p.NA;
+                for (int j = 0; j < pending; ++j) {
+                    if (--a_slot < 0) { a_slot = p.NA - 1; phaseA ^= 1u; }
+                    for (uint32_t spin = 0; spin < (1u << 20); ++spin)
+                        if (mbar_try_wait(&fullA_bar[a_slot], phaseA)) break;
                 }
             }
         }
@@ -166,6 +217,8 @@ tc_fprop_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
         const uint32_t idesc = make_idesc_tf32(p.BN, false, false);
         int stage = 0;
         uint32_t phase = 0;
+        int a_slot = 0;
+        uint32_t phaseA = 0;
         int tile_cnt = 0;
         bool ok = true;
         for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x, ++tile_cnt) {
@@ -173,23 +226,56 @@ tc_fprop_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
             const uint32_t acc_phase = (tile_cnt >> 1) & 1;
             if (!bounded_wait_warp(&tmem_empty_bar[acc], acc_phase ^ 1u, &abort_flag, p.status, WAIT_MMA_TMEM_EMPTY)) break;
             tc_fence_after();
-            const uint32_t d_tmem = tmem_base + acc * p.BN;
-            for (int kit = 0; kit < kiters; ++kit) {
-                if (!bounded_wait_warp(&full_bar[stage], phase, &abort_flag, p.status, WAIT_MMA_FULL)) { ok = false; break; }
-                tc_fence_after();
-                if (lane == 0) {
-                    const uint32_t a_addr = smem_u32(smem + stage * stage_bytes);
-                    const uint32_t b_addr = a_addr + kABytes;
+            const uint32_t d_tmem = tmem_base + acc * p.MT * p.BN;
+            if (p.halo) {
+                const uint32_t sbo = p.PW * 128;     // one patch row of pixels between the 8-pixel groups
+                for (int cb = 0; cb < p.cblocks && ok; ++cb) {
+                    if (!bounded_wait_warp(&fullA_bar[a_slot], phaseA, &abort_flag, p.status, WAIT_MMA_FULL)) { ok = false; break; }
+                    const uint32_t a_base = smem_u32(smem + a_slot * p.a_buf_bytes);
+                    int tap = 0;
+                    for (int r = 0; r < p.R && ok; ++r)
+                        for (int s = 0; s < p.S; ++s, ++tap) {
+                            if (!bounded_wait_warp(&full_bar[stage], phase, &abort_flag, p.status, WAIT_MMA_FULL)) { ok = false; break; }
+                            tc_fence_after();
+                            if (lane == 0) {
+                                const uint32_t b_addr = smem_u32(b_ring + stage * stage_bytes);
+                                const uint32_t a_tap = a_base + (r * p.PW + s) * 128;   // the tap = a row shift
+                                for (int h = 0; h < p.MT; ++h) {
 #pragma unroll
-                    for (int kk = 0; kk < 4; ++kk) {
-                        const uint64_t da = make_smem_desc(a_addr + kk * 32, 16, 1024, kSwizzle128B);
-                        const uint64_t db = make_smem_desc(b_addr + kk * 32, 16, 1024, kSwizzle128B);
-                        umma_tf32(d_tmem, da, db, idesc, (kit | kk) != 0);
-                    }
-                    umma_commit(&empty_bar[stage]);
+                                    for (int kk = 0; kk < 4; ++kk) {
+                                        const uint64_t da = make_smem_desc(a_tap + h * p.half_off_bytes + kk * 32, 16, sbo,
+                                                                           kSwizzle128B);
+                                        const uint64_t db = make_smem_desc(b_addr + kk * 32, 16, 1024, kSwizzle128B);
+                                        umma_tf32(d_tmem + h * p.BN, da, db, idesc, (cb | tap | kk) != 0);
+                                    }
+                                }
+                                umma_commit(&empty_bar[stage]);
+                            }
+                            __syncwarp();
+                            if (++stage == p.stages) { stage = 0; phase ^= 1u; }
+                        }
+                    if (ok && lane == 0) umma_commit(&emptyA_bar[a_slot]);
+                    __syncwarp();
+                    if (++a_slot == p.NA) { a_slot = 0; phaseA ^= 1u; }
                 }
-                __syncwarp();
-                if (++stage == p.stages) { stage = 0; phase ^= 1u; }
+            } else {
+                for (int kit = 0; kit < kiters; ++kit) {
+                    if (!bounded_wait_warp(&full_bar[stage], phase, &abort_flag, p.status, WAIT_MMA_FULL)) { ok = false; break; }
+                    tc_fence_after();
+                    if (lane == 0) {
+                        const uint32_t a_addr = smem_u32(smem + stage * stage_bytes);
+                        const uint32_t b_addr = a_addr + kABytes;
+#pragma unroll
+                        for (int kk = 0; kk < 4; ++kk) {
+                            const uint64_t da = make_smem_desc(a_addr + kk * 32, 16, 1024, kSwizzle128B);
+                            const uint64_t db = make_smem_desc(b_addr + kk * 32, 16, 1024, kSwizzle128B);
+                            umma_tf32(d_tmem, da, db, idesc, (kit | kk) != 0);
+                        }
+                        umma_commit(&empty_bar[stage]);
+                    }
+                    __syncwarp();
+                    if (++stage == p.stages) { stage = 0; phase ^= 1u; }
+                }
             }
             if (ok && lane == 0) umma_commit(&tmem_full_bar[acc]);
             __syncwarp();
@@ -201,7 +287,7 @@ tc_fprop_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
         const int row = quarter * 32 + lane;    // row of the tile = pixel of the box
         const int iw = row & (bw - 1);
         const int ih = (row >> p.bw_log2) & (bh - 1);
-        const int in_ = row >> (p.bw_log2 + p.bh_log2);
+        const int in_ = row >> (p.bw_log2 + p.bh_log2);      // halo mode: the box is 8 x 16 x 1, so in_ = 0
         const bool vec_ok = (p.Kout & 3) == 0;
         int tile_cnt = 0;
         TileIter it;
@@ -209,14 +295,15 @@ tc_fprop_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
             const int acc = tile_cnt & 1;
             const uint32_t acc_phase = (tile_cnt >> 1) & 1;
             const int kt = it.kt;
-            const int q = it.qi * bw + iw;
-            const int pp = it.pi * bh + ih;
-            const int n = it.ni * bn + in_;
-            const bool valid = (q < p.Q) && (pp < p.P) && (n < p.N);
-            const size_t pix = (static_cast<size_t>(n) * p.P + pp) * p.Q + q;
             if (!bounded_wait_warp(&tmem_full_bar[acc], acc_phase, &abort_flag, p.status, WAIT_EPI_TMEM_FULL)) break;
             tc_fence_after();
-            const uint32_t t_row = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + acc * p.BN;
+            for (int h = 0; h < p.MT; ++h) {
+            const int q = it.qi * p.tw + iw + h * p.half_dq;
+            const int pp = it.pi * p.th + ih + h * p.half_dp;
+            const int n = it.ni * p.tn + in_;
+            const bool valid = (q < p.Q) && (pp < p.P) && (n < p.N);
+            const size_t pix = (static_cast<size_t>(n) * p.P + pp) * p.Q + q;
+            const uint32_t t_row = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + (acc * p.MT + h) * p.BN;
             if (vec_ok) {
                 // Coalesced path.  Each lane owns one row (pixel) of the accumulator, but a row's 32 columns
                 // are 128 contiguous bytes in global memory, so the chunk is first transposed through a
@@ -304,6 +391,7 @@ tc_fprop_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                     }
                 }
             }
+            }   // halves
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(&tmem_empty_bar[acc]);
@@ -361,6 +449,64 @@ bool tc_fprop_eligible(const TcFpropArgs& a) {
     return true;
 }
 
+namespace {
+
+// One way of tiling a layer: plain (a box of 128 pixels, one TMA box per tap) or halo (MT boxes of 8 x 16
+// pixels cut from one haloed patch per channel block).
+struct TileCfg {
+    bool ok = false;
+    int halo = 0, MT = 1, bw_log2 = 0, bh_log2 = 0, tw = 0, th = 0, tn = 0, half_dq = 0, half_dp = 0;
+    int tiles_q = 0, tiles_p = 0, tiles_n = 0, tiles_k = 0, BN = 0;
+    int PW = 0, patch_bytes = 0, a_buf_bytes = 0, NA = 0, half_off_bytes = 0, stages = 0;
+};
+
+TileCfg plain_cfg(const TcFpropArgs& a, int cblocks, int sm_count) {
+    TileCfg c;
+    choose_box(a.P, a.Q, a.N, &c.bw_log2, &c.bh_log2);
+    c.tw = 1 << c.bw_log2; c.th = 1 << c.bh_log2; c.tn = kTileM / (c.tw * c.th);
+    c.tiles_q = (a.Q + c.tw - 1) / c.tw; c.tiles_p = (a.P + c.th - 1) / c.th; c.tiles_n = (a.N + c.tn - 1) / c.tn;
+    const long m_tiles = long(c.tiles_q) * c.tiles_p * c.tiles_n;
+    c.BN = choose_bn(a.Kout, m_tiles, sm_count);
+    c.tiles_k = (a.Kout + c.BN - 1) / c.BN;
+    c.stages = (kSmemBudget - kEpiStageBytes) / (kABytes + c.BN * 128);
+    if (c.stages > kMaxStages) c.stages = kMaxStages;
+    c.ok = c.stages >= 2;
+    return c;
+}
+
+// layout: 0 = one box (8 x 16), 1 = two boxes side by side (16 x 16), 2 = two boxes stacked (8 x 32)
+TileCfg halo_cfg(const TcFpropArgs& a, int cblocks, int sm_count, int layout) {
+    TileCfg c;
+    c.halo = 1; c.MT = layout == 0 ? 1 : 2;
+    c.bw_log2 = 3; c.bh_log2 = 4;
+    c.tw = layout == 1 ? 16 : 8; c.th = layout == 2 ? 32 : 16; c.tn = 1;
+    c.half_dq = layout == 1 ? 8 : 0; c.half_dp = layout == 2 ? 16 : 0;
+    c.PW = c.tw + a.S - 1;
+    const int PH = c.th + a.R - 1;
+    if (a.R * a.S <= 1 || c.PW > 256 || PH > 256) return c;
+    c.patch_bytes = c.PW * PH * 128;
+    c.a_buf_bytes = (c.patch_bytes + 1023) / 1024 * 1024;
+    c.half_off_bytes = layout == 1 ? 8 * 128 : (layout == 2 ? 16 * c.PW * 128 : 0);
+    c.tiles_q = (a.Q + c.tw - 1) / c.tw; c.tiles_p = (a.P + c.th - 1) / c.th; c.tiles_n = a.N;
+    const long m_tiles = long(c.tiles_q) * c.tiles_p * c.tiles_n;
+    c.BN = choose_bn(a.Kout, m_tiles, sm_count);
+    if (2 * c.MT * c.BN > 512) return c;          // two accumulator sets must fit the 512 TMEM columns
+    c.tiles_k = (a.Kout + c.BN - 1) / c.BN;
+    const int room = kSmemBudget - kEpiStageBytes;
+    c.NA = 2;
+    c.stages = (room - c.NA * c.a_buf_bytes) / (c.BN * 128);
+    if (c.stages >= 9 && (room - 3 * c.a_buf_bytes) / (c.BN * 128) >= 6) {
+        c.NA = 3;
+        c.stages = (room - 3 * c.a_buf_bytes) / (c.BN * 128);
+    }
+    if (c.stages > kMaxStages) c.stages = kMaxStages;
+    if (c.stages < 3) return c;
+    c.ok = true;
+    return c;
+}
+
+}  // namespace
+
 int launch_tc_fprop(const TcFpropArgs& a, cudaStream_t st) {
     if (!tc_fprop_eligible(a)) return PCL_ERR_UNSUPPORTED_SHAPE;
     if (g_sm_count == 0) {
@@ -372,24 +518,34 @@ int launch_tc_fprop(const TcFpropArgs& a, cudaStream_t st) {
             return PCL_ERR_CUDA;
     }
     FpropParams p{};
-    choose_box(a.P, a.Q, a.N, &p.bw_log2, &p.bh_log2);
+    p.cblocks = (a.Cin + kBlockC - 1) / kBlockC;
+    TileCfg cfg = plain_cfg(a, p.cblocks, g_sm_count);
+    if (!cfg.ok) return PCL_ERR_UNSUPPORTED_SHAPE;
+    // Test hook: PCL_TILING = plain | halo0 | halo1 | halo2 pins the tiling (when that tiling is possible).
+    const char* pin = getenv("PCL_TILING");
+    const int pinned = !pin ? -2 : (pin[0] == 'p' ? -1 : (pin[0] == 'h' && pin[4] >= '0' && pin[4] <= '2' ? pin[4] - '0' : -2));
+    for (int layout = 0; layout < 3; ++layout) {
+        const TileCfg h = halo_cfg(a, p.cblocks, g_sm_count, layout);
+        if (!h.ok) continue;
+        if (pinned == layout) { cfg = h; break; }
+        // Measured on B200: a row-shifted (not 1024-byte aligned) A view costs the tensor core extra shared
+        // memory cycles, so the haloed tiling only pays where the plain one is starved by operand traffic:
+        // narrow layers (BN <= 128) tiled without ragged edges by two boxes that share every weight tile.
+        if (pinned == -2 && layout > 0 && h.BN <= 128 && a.Q % h.tw == 0 && a.P % h.th == 0) { cfg = h; break; }
+    }
+    p.halo = cfg.halo; p.MT = cfg.MT; p.bw_log2 = cfg.bw_log2; p.bh_log2 = cfg.bh_log2;
+    p.tw = cfg.tw; p.th = cfg.th; p.tn = cfg.tn; p.half_dq = cfg.half_dq; p.half_dp = cfg.half_dp;
+    p.tiles_q = cfg.tiles_q; p.tiles_p = cfg.tiles_p; p.tiles_n = cfg.tiles_n; p.tiles_k = cfg.tiles_k;
+    p.BN = cfg.BN; p.PW = cfg.PW; p.patch_bytes = cfg.patch_bytes; p.a_buf_bytes = cfg.a_buf_bytes; p.NA = cfg.NA;
+    p.half_off_bytes = cfg.half_off_bytes; p.stages = cfg.stages;
     const int bw = 1 << p.bw_log2, bh = 1 << p.bh_log2, bn = kTileM / (bw * bh);
-    p.tiles_q = (a.Q + bw - 1) / bw;
-    p.tiles_p = (a.P + bh - 1) / bh;
-    p.tiles_n = (a.N + bn - 1) / bn;
     const long m_tiles = long(p.tiles_q) * p.tiles_p * p.tiles_n;
-    p.BN = choose_bn(a.Kout, m_tiles, g_sm_count);
-    p.tiles_k = (a.Kout + p.BN - 1) / p.BN;
     if (m_tiles * p.tiles_k > 0x7fffffffL) return PCL_ERR_UNSUPPORTED_SHAPE;
     p.R = a.R; p.S = a.S; p.pad_h = a.pad_h; p.pad_w = a.pad_w;
-    p.cblocks = (a.Cin + kBlockC - 1) / kBlockC;
     p.N = a.N; p.P = a.P; p.Q = a.Q; p.Kout = a.Kout;
     p.act = a.act;
-    const int stage_bytes = kABytes + p.BN * 128;
-    p.stages = (kSmemBudget - kEpiStageBytes) / stage_bytes;
-    if (p.stages > kMaxStages) p.stages = kMaxStages;
     p.tmem_cols = 32;
-    while (p.tmem_cols < 2 * p.BN) p.tmem_cols *= 2;
+    while (p.tmem_cols < 2 * p.MT * p.BN) p.tmem_cols *= 2;
     p.bias = a.bias; p.mask_src = a.mask_src; p.out = a.out;
     p.status = device_status_ptr();
     if (!p.status) return PCL_ERR_CUDA;
@@ -402,8 +558,9 @@ int launch_tc_fprop(const TcFpropArgs& a, cudaStream_t st) {
         const uint64_t sh = a.in_stride_h ? uint64_t(a.in_stride_h) : uint64_t(a.W) * a.Cin;
         const uint64_t sn = a.in_stride_n ? uint64_t(a.in_stride_n) : uint64_t(a.H) * a.W * a.Cin;
         const uint64_t strides[3] = {sw * 4, sh * 4, sn * 4};
-        const uint32_t box[4] = {kBlockC, uint32_t(bw), uint32_t(bh), uint32_t(bn)};
-        int rc = make_tmap(&tmA, a.in, 4, dims, strides, box, false);
+        const uint32_t box_plain[4] = {kBlockC, uint32_t(bw), uint32_t(bh), uint32_t(bn)};
+        const uint32_t box_halo[4] = {kBlockC, uint32_t(p.PW), uint32_t(p.th + a.R - 1), 1};
+        int rc = make_tmap(&tmA, a.in, 4, dims, strides, p.halo ? box_halo : box_plain, false);
         if (rc != PCL_OK) return rc;
     }
     {
@@ -415,7 +572,8 @@ int launch_tc_fprop(const TcFpropArgs& a, cudaStream_t st) {
     }
     const long total = m_tiles * p.tiles_k;
     const int grid = int(total < g_sm_count ? total : g_sm_count);
-    const size_t smem = size_t(p.stages) * stage_bytes + kEpiStageBytes + 1024;
+    const size_t smem = (p.halo ? size_t(p.NA) * p.a_buf_bytes + size_t(p.stages) * p.BN * 128
+                                : size_t(p.stages) * (kABytes + p.BN * 128)) + kEpiStageBytes + 1024;
     {
         LaunchScope scope(KID_TC_FPROP, 2.0 * a.N * a.P * a.Q * double(a.Kout) * a.Cin * a.R * a.S, st);
         tc_fprop_kernel<<<grid, kThreads, smem, st>>>(tmA, tmB, p);
