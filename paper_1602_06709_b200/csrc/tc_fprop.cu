@@ -228,7 +228,11 @@ tc_fprop_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
             tc_fence_after();
             const uint32_t d_tmem = tmem_base + acc * p.MT * p.BN;
             if (p.halo) {
-                const uint32_t sbo = p.PW * 128;     // one patch row of pixels between the 8-pixel groups
+                // Descriptors differ only in their 14-bit address field (address >> 4): build the constant part
+                // once and add offsets, so that the issuing thread spends a few instructions per MMA.
+                const uint64_t a_desc0 = make_smem_desc(0, 16, p.PW * 128, kSwizzle128B);   // 8-pixel groups are one patch row apart
+                const uint64_t b_desc0 = make_smem_desc(0, 16, 1024, kSwizzle128B);
+                const uint32_t half_off16 = p.half_off_bytes >> 4;
                 for (int cb = 0; cb < p.cblocks && ok; ++cb) {
                     if (!bounded_wait_warp(&fullA_bar[a_slot], phaseA, &abort_flag, p.status, WAIT_MMA_FULL)) { ok = false; break; }
                     const uint32_t a_base = smem_u32(smem + a_slot * p.a_buf_bytes);
@@ -238,16 +242,14 @@ tc_fprop_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                             if (!bounded_wait_warp(&full_bar[stage], phase, &abort_flag, p.status, WAIT_MMA_FULL)) { ok = false; break; }
                             tc_fence_after();
                             if (lane == 0) {
-                                const uint32_t b_addr = smem_u32(b_ring + stage * stage_bytes);
-                                const uint32_t a_tap = a_base + (r * p.PW + s) * 128;   // the tap = a row shift
+                                const uint64_t db = b_desc0 + ((smem_u32(b_ring + stage * stage_bytes) & 0x3FFFFu) >> 4);
+                                // the tap = a row shift inside the patch
+                                const uint64_t da = a_desc0 + (((a_base + (r * p.PW + s) * 128) & 0x3FFFFu) >> 4);
                                 for (int h = 0; h < p.MT; ++h) {
 #pragma unroll
-                                    for (int kk = 0; kk < 4; ++kk) {
-                                        const uint64_t da = make_smem_desc(a_tap + h * p.half_off_bytes + kk * 32, 16, sbo,
-                                                                           kSwizzle128B);
-                                        const uint64_t db = make_smem_desc(b_addr + kk * 32, 16, 1024, kSwizzle128B);
-                                        umma_tf32(d_tmem + h * p.BN, da, db, idesc, (cb | tap | kk) != 0);
-                                    }
+                                    for (int kk = 0; kk < 4; ++kk)
+                                        umma_tf32(d_tmem + h * p.BN, da + h * half_off16 + kk * 2, db + kk * 2, idesc,
+                                                  (cb | tap | kk) != 0);
                                 }
                                 umma_commit(&empty_bar[stage]);
                             }
@@ -259,18 +261,15 @@ tc_fprop_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                     if (++a_slot == p.NA) { a_slot = 0; phaseA ^= 1u; }
                 }
             } else {
+                const uint64_t desc0 = make_smem_desc(0, 16, 1024, kSwizzle128B);
                 for (int kit = 0; kit < kiters; ++kit) {
                     if (!bounded_wait_warp(&full_bar[stage], phase, &abort_flag, p.status, WAIT_MMA_FULL)) { ok = false; break; }
                     tc_fence_after();
                     if (lane == 0) {
-                        const uint32_t a_addr = smem_u32(smem + stage * stage_bytes);
-                        const uint32_t b_addr = a_addr + kABytes;
+                        const uint64_t da = desc0 + ((smem_u32(smem + stage * stage_bytes) & 0x3FFFFu) >> 4);
+                        const uint64_t db = da + (kABytes >> 4);
 #pragma unroll
-                        for (int kk = 0; kk < 4; ++kk) {
-                            const uint64_t da = make_smem_desc(a_addr + kk * 32, 16, 1024, kSwizzle128B);
-                            const uint64_t db = make_smem_desc(b_addr + kk * 32, 16, 1024, kSwizzle128B);
-                            umma_tf32(d_tmem, da, db, idesc, (kit | kk) != 0);
-                        }
+                        for (int kk = 0; kk < 4; ++kk) umma_tf32(d_tmem, da + kk * 2, db + kk * 2, idesc, (kit | kk) != 0);
                         umma_commit(&empty_bar[stage]);
                     }
                     __syncwarp();

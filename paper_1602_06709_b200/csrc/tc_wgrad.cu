@@ -168,6 +168,7 @@ tc_wgrad_kernel(const __grid_constant__ CUtensorMap tmDy, const __grid_constant_
         }
     } else if (warp == 1) {
         const uint32_t idesc = make_idesc_tf32(n_groups * 32, true, true);
+        const uint64_t desc0 = make_smem_desc(0, kGroupBytes, 512, kSwizzle128B_Atom32B);
         int stage = 0;
         uint32_t phase = 0;
         bool ok = true;
@@ -175,15 +176,13 @@ tc_wgrad_kernel(const __grid_constant__ CUtensorMap tmDy, const __grid_constant_
             if (!bounded_wait_warp(&full_bar[stage], phase, &abort_flag, p.status, WAIT_MMA_FULL)) { ok = false; break; }
             tc_fence_after();
             if (lane == 0) {
-                const uint32_t a_addr = smem_u32(smem + stage * stage_bytes);
-                const uint32_t b_addr = a_addr + kABytes;
+                // 8 pixels per instruction = two 512-byte groups of 4 rows; descriptors differ only in the
+                // address field, so add offsets to a constant part
+                const uint64_t da = desc0 + ((smem_u32(smem + stage * stage_bytes) & 0x3FFFFu) >> 4);
+                const uint64_t db = da + (kABytes >> 4);
 #pragma unroll
-                for (int kk = 0; kk < kPix / 8; ++kk) {
-                    // 8 pixels per instruction = two 512-byte groups of 4 rows
-                    const uint64_t da = make_smem_desc(a_addr + kk * 1024, kGroupBytes, 512, kSwizzle128B_Atom32B);
-                    const uint64_t db = make_smem_desc(b_addr + kk * 1024, kGroupBytes, 512, kSwizzle128B_Atom32B);
-                    umma_tf32(tmem_base, da, db, idesc, (kit | kk) != 0);
-                }
+                for (int kk = 0; kk < kPix / 8; ++kk)
+                    umma_tf32(tmem_base, da + kk * (1024 >> 4), db + kk * (1024 >> 4), idesc, (kit | kk) != 0);
                 umma_commit(&empty_bar[stage]);
             }
             __syncwarp();
