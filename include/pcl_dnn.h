@@ -53,7 +53,8 @@ enum {
     PCL_ERR_MISALIGNED = 3,        /* a pointer is not 16-byte aligned                */
     PCL_ERR_WORKSPACE = 4,         /* workspace smaller than pcl_*_workspace_bytes()  */
     PCL_ERR_CUDA = 5,              /* a CUDA runtime/driver call failed               */
-    PCL_ERR_DEVICE_TIMEOUT = 6     /* a bounded device-side wait ran out              */
+    PCL_ERR_DEVICE_TIMEOUT = 6,    /* a bounded device-side wait ran out              */
+    PCL_ERR_SCRATCH_LIMIT = 7      /* problem larger than the built-in scratch array  */
 };
 
 enum { PCL_PASS_FWD = 0, PCL_PASS_BWD_DATA = 1, PCL_PASS_BWD_WEIGHTS = 2 };
@@ -148,6 +149,32 @@ int pcl_last_device_status(void* cuda_stream);
 
 /* Number of kernels this library has launched since it was loaded. */
 unsigned long long pcl_launch_count(void);
+
+/* Backward-data for callers that cannot allocate device memory (the paper has
+ * no counterpart; this is a convenience of the library).
+ *
+ * Same result as pcl_conv_bwd_data(), but the caller passes no workspace: the
+ * flipped, transposed weight copy goes into a fixed array inside the library's
+ * device image.  Meant for code that is handed tensors but has no allocator to
+ * ask -- a plugin, a serving loop whose device memory all belongs to someone
+ * else's pool, any place where cudaMalloc is off limits.  The call itself makes
+ * no cudaMalloc / cudaFree and uses no allocating library routine.
+ *
+ *  - Capacity: pcl_noalloc_scratch_bytes() = 16 MiB, i.e. K*R*S*C <= 4 194 304
+ *    weights.  Larger layers get PCL_ERR_SCRATCH_LIMIT and nothing is launched.
+ *    Every GPU that loads the library holds these 16 MiB until the process ends.
+ *  - The first call on each device looks up the array's device address (one
+ *    runtime query, no allocation); make that first call before any stream
+ *    capture begins.
+ *  - All calls share the one array.  Each call overwrites it completely before
+ *    reading it, so calls issued one after another on a stream are fine; calls
+ *    whose kernels may overlap on the GPU (different streams, or different host
+ *    threads on different streams) race on it and must be serialised by the
+ *    caller.
+ * Arguments as for pcl_conv_bwd_data() without ws / ws_bytes. */
+int pcl_conv_bwd_data_noalloc(const pcl_conv_desc* d, const float* dy, const float* w,
+                              const float* relu_mask_src, float* dx, void* cuda_stream);
+size_t pcl_noalloc_scratch_bytes(void);
 
 /* Optional per-kernel timing (the paper has no counterpart; measurement aid).
  * Between pcl_profile_begin() and pcl_profile_end() every kernel launch of the

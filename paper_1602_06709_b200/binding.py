@@ -19,12 +19,13 @@ PASS_FWD, PASS_BWD_DATA, PASS_BWD_WEIGHTS = 0, 1, 2
 PATH_AUTO, PATH_TENSOR, PATH_GENERIC = 0, 1, 2
 OK = 0
 ERR_BAD_ARG, ERR_UNSUPPORTED_SHAPE, ERR_MISALIGNED, ERR_WORKSPACE, ERR_CUDA, ERR_DEVICE_TIMEOUT = 1, 2, 3, 4, 5, 6
+ERR_SCRATCH_LIMIT = 7
 
 EXPORTS = [
     "pcl_set_path", "pcl_conv_out_dims", "pcl_conv_workspace_bytes", "pcl_fc_workspace_bytes",
     "pcl_conv_fwd", "pcl_conv_bwd_data", "pcl_conv_bwd_weights", "pcl_fc_fwd", "pcl_fc_bwd",
     "pcl_sgd_update", "pcl_maxpool2x2_fwd", "pcl_maxpool2x2_bwd", "pcl_softmax_xent",
-    "pcl_last_device_status", "pcl_launch_count", "pcl_status_string", "pcl_profile_begin", "pcl_profile_end",
+    "pcl_last_device_status", "pcl_launch_count", "pcl_status_string", "pcl_profile_begin", "pcl_profile_end", "pcl_conv_bwd_data_noalloc", "pcl_noalloc_scratch_bytes",
 ]
 
 
@@ -75,6 +76,8 @@ def lib() -> ctypes.CDLL:
         L.pcl_last_device_status.argtypes = [vp]
         L.pcl_launch_count.restype = ctypes.c_ulonglong
         L.pcl_profile_end.argtypes = [ctypes.POINTER(KernelStat), ci, ctypes.POINTER(ci)]
+        L.pcl_conv_bwd_data_noalloc.argtypes = [dp, vp, vp, vp, vp, vp]
+        L.pcl_noalloc_scratch_bytes.restype = sz
         L.pcl_status_string.argtypes = [ci]
         L.pcl_status_string.restype = ctypes.c_char_p
         _lib = L
@@ -141,6 +144,17 @@ def conv_bwd_data(d, dy, w, relu_mask_src, dx, ws=None, stream=None):
     wp, wb = _ws(ws)
     _check(lib().pcl_conv_bwd_data(ctypes.byref(d), _ptr(dy), _ptr(w), _ptr(relu_mask_src), _ptr(dx), wp, wb,
                                    _stream(stream)), "pcl_conv_bwd_data")
+
+
+def conv_bwd_data_noalloc(d, dy, w, relu_mask_src, dx, stream=None):
+    """Backward-data without a caller workspace (for callers that cannot allocate device memory): the
+    library's built-in 16 MiB scratch array is used instead.  Calls that may overlap on the GPU race on it."""
+    _check(lib().pcl_conv_bwd_data_noalloc(ctypes.byref(d), _ptr(dy), _ptr(w), _ptr(relu_mask_src), _ptr(dx),
+                                           _stream(stream)), "pcl_conv_bwd_data_noalloc")
+
+
+def noalloc_scratch_bytes() -> int:
+    return int(lib().pcl_noalloc_scratch_bytes())
 
 
 def conv_bwd_weights(d, x, dy, dw, dbias=None, deterministic=True, ws=None, stream=None):

@@ -8,7 +8,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libpcl_dnn.so")
-SOURCES = ["pcl_api.cu", "tc_fprop.cu", "tc_wgrad.cu", "generic_conv.cu", "elementwise.cu"]
+SOURCES = ["pcl_api.cu", "tc_fprop.cu", "tc_wgrad.cu", "generic_conv.cu", "elementwise.cu", "noalloc.cu"]
 HEADERS = ["pcl_internal.h", "pcl_ptx.cuh", os.path.join("..", "..", "include", "pcl_dnn.h")]
 NVCC = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
 FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",

@@ -458,6 +458,7 @@ const char* pcl_status_string(int status) {
         case PCL_ERR_WORKSPACE: return "workspace too small";
         case PCL_ERR_CUDA: return "CUDA call failed";
         case PCL_ERR_DEVICE_TIMEOUT: return "device-side wait timed out";
+        case PCL_ERR_SCRATCH_LIMIT: return "problem exceeds the capacity of the built-in scratch array";
     }
     return "unknown status";
 }
