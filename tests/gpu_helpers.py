@@ -106,8 +106,9 @@ def verify_vgg_step(net, params_before, samples=0, seed=0):
         _cmp(net.y[i], lambda at: oracle.conv_fwd(s, xin, w, b, oracle.ACT_RELU, at=at), net.y[i].numel(), samples,
              rng, f"{L.name} fwd", report)
         if L.pool:
-            y = host(net.y[i])
-            assert np.array_equal(host(net.pooled[i]), oracle.maxpool2x2_fwd(y).astype(np.float32)), f"{L.name} pool"
+            nchk = N if not samples else min(N, 2)       # sampled runs check the pooling on the first images only
+            y = host(net.y[i][:nchk])
+            assert np.array_equal(host(net.pooled[i][:nchk]), oracle.maxpool2x2_fwd(y).astype(np.float32)), f"{L.name} pool"
     # forward FC
     a = host(net.pooled[-1]).reshape(N, net.flat)
     for j, (C, K) in enumerate(net.fcs):
@@ -157,8 +158,9 @@ def verify_vgg_step(net, params_before, samples=0, seed=0):
         L = net.convs[i]
         s = ConvShape(N=N, C=L.C, K=L.K, H=L.H, W=L.W, R=3, S=3, pad_h=1, pad_w=1)
         if L.pool:
-            y = host(net.y[i]); dp = host(net.dpooled[i])
-            assert np.array_equal(host(net.dy[i]), oracle.maxpool2x2_bwd(y, dp, y).astype(np.float32)), f"{L.name} pool bwd"
+            nchk = N if not samples else min(N, 2)
+            y = host(net.y[i][:nchk]); dp = host(net.dpooled[i][:nchk])
+            assert np.array_equal(host(net.dy[i][:nchk]), oracle.maxpool2x2_bwd(y, dp, y).astype(np.float32)), f"{L.name} pool bwd"
         dz = host(net.dy[i]); xin = host(net.layer_input(i)); w = pview(2 * i)
         _cmp(net.conv_dw(i), lambda at: oracle.conv_bwd_weights(s, xin, dz, at=at), net.conv_dw(i).numel(), samples,
              rng, f"{L.name} dw", report)

@@ -107,3 +107,29 @@ def test_cfg1_with_sgd_update():
     ref = oracle.sgd_update(w, dw, 0.01)
     np.testing.assert_allclose(wt.cpu().numpy(), ref, rtol=0, atol=1e-7)
     G.assert_parity(wt.cpu().numpy(), oracle.sgd_update(w, dw_ref, 0.01), "updated weights")
+
+
+HALO_SHAPES = {
+    "fits_16x16": ConvShape(N=3, C=64, K=64, H=32, W=48, R=3, S=3, pad_h=1, pad_w=1),       # two boxes side by side
+    "fits_8x32": ConvShape(N=2, C=32, K=128, H=64, W=24, R=3, S=3, pad_h=1, pad_w=1),
+    "ragged": ConvShape(N=2, C=96, K=40, H=21, W=19, R=3, S=3, pad_h=1, pad_w=1),
+    "k5": ConvShape(N=2, C=32, K=32, H=20, W=20, R=5, S=5, pad_h=2, pad_w=2),
+    "wide": ConvShape(N=2, C=64, K=256, H=16, W=16, R=3, S=3, pad_h=1, pad_w=1),              # BN = 256: one box only
+}
+
+
+@pytest.mark.parametrize("tiling", ["plain", "halo0", "halo1", "halo2"])
+@pytest.mark.parametrize("tag", sorted(HALO_SHAPES))
+def test_forward_type_kernel_every_tiling(tag, tiling, path_guard, monkeypatch):
+    """The forward-type kernel has a plain tiling and three haloed ones (taps as row-shifted views of one
+    input patch); PCL_TILING pins one.  All must agree with the oracle for forward and backward-data."""
+    import gpu_helpers as G
+    from paper_1602_06709_b200 import binding as B
+    monkeypatch.setenv("PCL_TILING", tiling)
+    B.set_path(B.PATH_TENSOR)
+    s = HALO_SHAPES[tag]
+    x, w, dy, bias = G.make_inputs(s, "halo_" + tag)
+    y = G.run_conv_fwd(s, x, w, bias, B.ACT_RELU)
+    G.assert_parity(y, oracle.conv_fwd(s, x, w, bias, oracle.ACT_RELU), f"fwd {tiling}")
+    dx = G.run_conv_bwd_data(s, dy, w, x)
+    G.assert_parity(dx, oracle.conv_bwd_data(s, dy, w, x), f"bwd_data {tiling}")
