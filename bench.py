@@ -301,32 +301,23 @@ def run_reference(args):
 # ---------------------------------------------------------------------------
 def run_ours(args):
     import torch
-    import torch.distributed as dist
     from paper_1602_06709_b200 import binding as B
+    from paper_1602_06709_b200 import replicas
 
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    rank = int(os.environ.get("RANK", "0"))
-    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world, rank, local_rank = replicas.world()
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device: the product path has no CPU fallback")
     torch.cuda.set_device(local_rank)
-    if world > 1:
-        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    replicas.init("nccl", torch.device("cuda", local_rank))
     if args.minibatch and not args.kernels_only:
         raise SystemExit("--minibatch changes the workload: only allowed with --kernels-only")
     B.lib()      # fail loudly here if the extension is missing
 
     def barrier():
-        if world > 1:
-            dist.barrier()
-        torch.cuda.synchronize()
+        replicas.barrier(cuda=True)
 
     def max_over_ranks(v: float) -> float:
-        if world == 1:
-            return v
-        t = torch.tensor([v], device="cuda", dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        return float(t.item())
+        return replicas.max_over_ranks(v, device="cuda")
 
     wl = WORKLOADS[args.workload](rank, args.minibatch)
     peaks = load_peaks()
@@ -356,7 +347,7 @@ def run_ours(args):
     status = B.last_device_status()
     if status != B.OK:
         raise SystemExit(f"device status {status}: {B.status_string(status)}")
-    value = wl.units_per_step * args.steps * world / (ms / 1e3)
+    value = replicas.whole_job_throughput(wl.units_per_step, args.steps, world, ms)
 
     if args.kernels_only:      # for profiler captures: just the steps, one short line
         if rank == 0:
@@ -367,7 +358,7 @@ def run_ours(args):
     # end to end through the user-level call: pinned host minibatch in, result out, every step
     e2e_steps = max(3, min(args.steps, 10))
     ms_e2e, _, _ = timed(wl.e2e_step, e2e_steps, 1)
-    e2e_value = wl.units_per_step * e2e_steps * world / (ms_e2e / 1e3)
+    e2e_value = replicas.whole_job_throughput(wl.units_per_step, e2e_steps, world, ms_e2e)
 
     # instrumented repeat of the same steps: CUDA events around every kernel launch on the launching stream
     prof_steps = max(1, min(args.steps, 5))
@@ -444,8 +435,7 @@ def run_ours(args):
             **extra,
         }
         print(json.dumps(line), flush=True)
-    if world > 1:
-        dist.destroy_process_group()
+    replicas.shutdown()
 
 
 def main():
