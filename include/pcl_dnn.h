@@ -96,6 +96,18 @@ int pcl_conv_bwd_data(const pcl_conv_desc* d, const float* dy, const float* w,
                       const float* relu_mask_src, float* dx,
                       void* ws, size_t ws_bytes, void* cuda_stream);
 
+/* Backpropagation that also returns the per-map sums of what it wrote:
+ *   dx as pcl_conv_bwd_data();  dx_colsum[c] = sum_{n,h,w} dx[n,h,w,c]   (after the mask).
+ * With the ReLU mask fused, dx is the gradient w.r.t. the pre-activation of the
+ * layer below, so dx_colsum is that layer's bias gradient: the sums are formed
+ * in the epilogue while the tile is on chip instead of re-reading dx from
+ * memory.  Deterministic (fixed summation order).  dx_colsum: [C] out.
+ * Workspace: pcl_conv_bwd_data_colsum_workspace_bytes(d). */
+size_t pcl_conv_bwd_data_colsum_workspace_bytes(const pcl_conv_desc* d);
+int pcl_conv_bwd_data_colsum(const pcl_conv_desc* d, const float* dy, const float* w,
+                             const float* relu_mask_src, float* dx, float* dx_colsum,
+                             void* ws, size_t ws_bytes, void* cuda_stream);
+
 /* Weight-gradient update (Sec. 2.1):
  *   dw[k,r,s,c] = sum_{n,p,q} dy[n,p,q,k] * x[n, p*stride_h + r - pad_h, q*stride_w + s - pad_w, c]
  *   dbias[k]    = sum_{n,p,q} dy[n,p,q,k]                  (if dbias != NULL)
@@ -138,6 +150,13 @@ int pcl_maxpool2x2_fwd(int N, int H, int W, int C, const float* x, float* y, voi
  * where relu_mask_src <= 0. */
 int pcl_maxpool2x2_bwd(int N, int H, int W, int C, const float* x, const float* dy,
                        const float* relu_mask_src, float* dx, void* cuda_stream);
+/* pcl_maxpool2x2_bwd() plus dx_colsum[c] = sum_{n,h,w} dx[n,h,w,c] (the bias gradient of the
+ * convolution whose ReLU output was pooled).  Deterministic.  Workspace:
+ * pcl_maxpool2x2_bwd_colsum_workspace_bytes(N, H, W, C). */
+size_t pcl_maxpool2x2_bwd_colsum_workspace_bytes(int N, int H, int W, int C);
+int pcl_maxpool2x2_bwd_colsum(int N, int H, int W, int C, const float* x, const float* dy,
+                              const float* relu_mask_src, float* dx, float* dx_colsum,
+                              void* ws, size_t ws_bytes, void* cuda_stream);
 /* loss = -(1/N) sum_n log softmax(logits[n,:])[labels[n]]  (device scalar, overwritten)
  * dlogits = (softmax(logits) - onehot(labels)) / N.  labels: device int32 [N]. */
 int pcl_softmax_xent(int N, int K, const float* logits, const int* labels,

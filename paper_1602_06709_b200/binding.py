@@ -26,6 +26,8 @@ EXPORTS = [
     "pcl_conv_fwd", "pcl_conv_bwd_data", "pcl_conv_bwd_weights", "pcl_fc_fwd", "pcl_fc_bwd",
     "pcl_sgd_update", "pcl_maxpool2x2_fwd", "pcl_maxpool2x2_bwd", "pcl_softmax_xent",
     "pcl_last_device_status", "pcl_launch_count", "pcl_status_string", "pcl_profile_begin", "pcl_profile_end", "pcl_conv_bwd_data_noalloc", "pcl_noalloc_scratch_bytes",
+    "pcl_conv_bwd_data_colsum_workspace_bytes", "pcl_conv_bwd_data_colsum",
+    "pcl_maxpool2x2_bwd_colsum_workspace_bytes", "pcl_maxpool2x2_bwd_colsum",
 ]
 
 
@@ -76,6 +78,12 @@ def lib() -> ctypes.CDLL:
         L.pcl_last_device_status.argtypes = [vp]
         L.pcl_launch_count.restype = ctypes.c_ulonglong
         L.pcl_profile_end.argtypes = [ctypes.POINTER(KernelStat), ci, ctypes.POINTER(ci)]
+        L.pcl_conv_bwd_data_colsum_workspace_bytes.argtypes = [dp]
+        L.pcl_conv_bwd_data_colsum_workspace_bytes.restype = sz
+        L.pcl_conv_bwd_data_colsum.argtypes = [dp, vp, vp, vp, vp, vp, vp, sz, vp]
+        L.pcl_maxpool2x2_bwd_colsum_workspace_bytes.argtypes = [ci, ci, ci, ci]
+        L.pcl_maxpool2x2_bwd_colsum_workspace_bytes.restype = sz
+        L.pcl_maxpool2x2_bwd_colsum.argtypes = [ci, ci, ci, ci, vp, vp, vp, vp, vp, vp, sz, vp]
         L.pcl_conv_bwd_data_noalloc.argtypes = [dp, vp, vp, vp, vp, vp]
         L.pcl_noalloc_scratch_bytes.restype = sz
         L.pcl_status_string.argtypes = [ci]
@@ -144,6 +152,26 @@ def conv_bwd_data(d, dy, w, relu_mask_src, dx, ws=None, stream=None):
     wp, wb = _ws(ws)
     _check(lib().pcl_conv_bwd_data(ctypes.byref(d), _ptr(dy), _ptr(w), _ptr(relu_mask_src), _ptr(dx), wp, wb,
                                    _stream(stream)), "pcl_conv_bwd_data")
+
+
+def conv_bwd_data_colsum_workspace_bytes(d: ConvDesc) -> int:
+    return int(lib().pcl_conv_bwd_data_colsum_workspace_bytes(ctypes.byref(d)))
+
+
+def conv_bwd_data_colsum(d, dy, w, relu_mask_src, dx, dx_colsum, ws=None, stream=None):
+    wp, wb = _ws(ws)
+    _check(lib().pcl_conv_bwd_data_colsum(ctypes.byref(d), _ptr(dy), _ptr(w), _ptr(relu_mask_src), _ptr(dx),
+                                          _ptr(dx_colsum), wp, wb, _stream(stream)), "pcl_conv_bwd_data_colsum")
+
+
+def maxpool2x2_bwd_colsum_workspace_bytes(N, H, W, C) -> int:
+    return int(lib().pcl_maxpool2x2_bwd_colsum_workspace_bytes(N, H, W, C))
+
+
+def maxpool2x2_bwd_colsum(N, H, W, C, x, dy, relu_mask_src, dx, dx_colsum, ws=None, stream=None):
+    wp, wb = _ws(ws)
+    _check(lib().pcl_maxpool2x2_bwd_colsum(N, H, W, C, _ptr(x), _ptr(dy), _ptr(relu_mask_src), _ptr(dx),
+                                           _ptr(dx_colsum), wp, wb, _stream(stream)), "pcl_maxpool2x2_bwd_colsum")
 
 
 def conv_bwd_data_noalloc(d, dy, w, relu_mask_src, dx, stream=None):

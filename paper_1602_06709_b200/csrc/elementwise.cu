@@ -90,7 +90,7 @@ __global__ void __launch_bounds__(256) act_grad_kernel(float* __restrict__ dy, c
 // A block covers a strip of up to 1024 columns (256 threads x float4 when K is a
 // multiple of 4) so that consecutive rows are read as whole contiguous runs; the
 // threads that share a column group are summed through shared memory in a fixed order.
-constexpr int kColsumMinRows = 2048;   // rows per split, at least; grown so that there are at most ~1200 splits
+constexpr int kColsumMinRows = 64;     // rows per split, at least; grown so that there are at most ~1200 splits
 template <int VEC>
 __global__ void __launch_bounds__(256) colsum_kernel(const float* __restrict__ m, size_t rows, int K,
                                                      float* __restrict__ partial, size_t rows_per_split) {
@@ -188,15 +188,20 @@ __device__ __forceinline__ float4 mask4(float4 v, float4 m) {
 
 // One thread per (pooled pixel, VEC channels): reads the 2x2 window of x and one dy, writes the 2x2 window of
 // dx.  When the ReLU mask source is x itself (the usual case: x is a ReLU output) it is not read again.
+// colsum_rows (VEC == 4 only, C/4 must divide 256): row blockIdx.x receives the per-channel sums of everything this
+// block wrote to dx.  Every thread keeps the same 4 channels for the whole grid-stride loop, so it sums privately;
+// the threads of a block that share channels are then added in a fixed order.
 template <int VEC>
 __global__ void __launch_bounds__(256) maxpool_bwd_kernel(const float* __restrict__ x, const float* __restrict__ dy,
                                                           const float* __restrict__ mask, float* __restrict__ dx,
-                                                          int N, int H, int W, int C) {
+                                                          int N, int H, int W, int C,
+                                                          float* __restrict__ colsum_rows = nullptr) {
     const int Po = H / 2, Qo = W / 2, Cv = C / VEC;
     const size_t total = size_t(N) * Po * Qo * Cv;
     const size_t stride = size_t(gridDim.x) * blockDim.x;
     const size_t rowp = size_t(W) * C;
     const bool mask_is_x = (mask == x);
+    float4 csum = make_float4(0.f, 0.f, 0.f, 0.f);
     for (size_t i = size_t(blockIdx.x) * blockDim.x + threadIdx.x; i < total; i += stride) {
         const int cv = int(i % Cv); size_t t = i / Cv;
         const int q = int(t % Qo); t /= Qo;
@@ -223,6 +228,8 @@ __global__ void __launch_bounds__(256) maxpool_bwd_kernel(const float* __restric
             __stcs(reinterpret_cast<float4*>(dx + off + C), ob);
             __stcs(reinterpret_cast<float4*>(dx + off + rowp), oc);
             __stcs(reinterpret_cast<float4*>(dx + off + rowp + C), od);
+            csum.x += (oa.x + ob.x) + (oc.x + od.x); csum.y += (oa.y + ob.y) + (oc.y + od.y);
+            csum.z += (oa.z + ob.z) + (oc.z + od.z); csum.w += (oa.w + ob.w) + (oc.w + od.w);
         } else {
             const float a = x[off], b = x[off + C], c = x[off + rowp], d = x[off + rowp + C];
             float oa, ob, oc, od;
@@ -234,6 +241,19 @@ __global__ void __launch_bounds__(256) maxpool_bwd_kernel(const float* __restric
                 if (!(mask[off + rowp + C] > 0.f)) od = 0.f;
             }
             dx[off] = oa; dx[off + C] = ob; dx[off + rowp] = oc; dx[off + rowp + C] = od;
+        }
+    }
+    if (VEC == 4 && colsum_rows) {
+        __shared__ float4 red[256];
+        red[threadIdx.x] = csum;
+        __syncthreads();
+        const int Cv4 = C / 4;
+        if (threadIdx.x < Cv4) {
+            float4 a = red[threadIdx.x];
+            for (int t = threadIdx.x + Cv4; t < 256; t += Cv4) {
+                a.x += red[t].x; a.y += red[t].y; a.z += red[t].z; a.w += red[t].w;
+            }
+            *reinterpret_cast<float4*>(colsum_rows + size_t(blockIdx.x) * C + threadIdx.x * 4) = a;
         }
     }
 }
@@ -459,6 +479,24 @@ int launch_maxpool_bwd(int N, int H, int W, int C, const float* x, const float* 
             maxpool_bwd_kernel<4><<<grid_for(outs * (C / 4), 256, 16), 256, 0, st>>>(x, dy, mask, dx, N, H, W, C);
         else
             maxpool_bwd_kernel<1><<<grid_for(outs * C, 256), 256, 0, st>>>(x, dy, mask, dx, N, H, W, C);
+    }
+    return PCL_CHECK_LAUNCH();
+}
+
+long maxpool_bwd_colsum_rows(int N, int H, int W, int C) {
+    if (C % 4 != 0 || 256 % (C / 4) != 0) return 0;
+    const size_t outs = size_t(N) * (H / 2) * (W / 2);
+    return grid_for(outs * (C / 4), 256, 16);
+}
+
+int launch_maxpool_bwd_colsum(int N, int H, int W, int C, const float* x, const float* dy, const float* mask,
+                              float* dx, float* colsum_rows, cudaStream_t st) {
+    if (maxpool_bwd_colsum_rows(N, H, W, C) == 0) return PCL_ERR_UNSUPPORTED_SHAPE;
+    const size_t outs = size_t(N) * (H / 2) * (W / 2);
+    {
+        LaunchScope scope(KID_MAXPOOL_BWD, 36.0 * double(outs) * C, st);
+        maxpool_bwd_kernel<4><<<grid_for(outs * (C / 4), 256, 16), 256, 0, st>>>(x, dy, mask, dx, N, H, W, C,
+                                                                                  colsum_rows);
     }
     return PCL_CHECK_LAUNCH();
 }

@@ -284,6 +284,105 @@ int pcl_conv_bwd_data(const pcl_conv_desc* d, const float* dy, const float* w, c
     return launch_generic_bwd_data(*d, P, Q, dy, w, relu_mask_src, dx, st);
 }
 
+namespace {
+// Workspace layout of the fused "dx + column sums of dx" calls: [main pass scratch][per-tile / per-block sum rows]
+// [second-stage partials of the column sum over those rows].
+size_t colsum_stage_bytes(long rows, int cols) {
+    if (rows <= 0) return 0;
+    const int cs = colsum_splits(size_t(rows));
+    return align_up(size_t(rows) * cols * 4, 256) + (cs > 1 ? align_up(size_t(cs) * cols * 4, 256) : 0);
+}
+TcFpropArgs bwd_data_args(const pcl_conv_desc& d, int P, int Q, const float* dy, const float* wt_t,
+                          const float* mask, float* dx) {
+    return TcFpropArgs{dy, wt_t, nullptr, mask, dx, d.N, P, Q, d.K, d.C, d.R, d.S,
+                       d.R - 1 - d.pad_h, d.S - 1 - d.pad_w, d.H, d.W, PCL_ACT_NONE};
+}
+}  // namespace
+
+size_t pcl_conv_bwd_data_colsum_workspace_bytes(const pcl_conv_desc* d) {
+    int P, Q;
+    if (check_desc(d, &P, &Q) != PCL_OK) return 0;
+    const size_t base = pcl_conv_workspace_bytes(d, PCL_PASS_BWD_DATA);
+    long rows = 0;
+    if (tensor_path_for(*d, PCL_PASS_BWD_DATA) && d->C % 4 == 0)
+        rows = tc_fprop_colsum_rows(bwd_data_args(*d, P, Q, nullptr, nullptr, nullptr, nullptr));
+    if (rows > 0) return base + colsum_stage_bytes(rows, d->C);
+    const int cs = colsum_splits(size_t(d->N) * d->H * d->W);          // unfused: column sum of dx itself
+    return base + (cs > 1 ? align_up(size_t(cs) * d->C * 4, 256) : 0);
+}
+
+int pcl_conv_bwd_data_colsum(const pcl_conv_desc* d, const float* dy, const float* w, const float* relu_mask_src,
+                             float* dx, float* dx_colsum, void* ws, size_t ws_bytes, void* cuda_stream) {
+    int P, Q;
+    int rc = check_desc(d, &P, &Q);
+    if (rc != PCL_OK) return rc;
+    if (!dy || !w || !dx || !dx_colsum) return PCL_ERR_BAD_ARG;
+    if (!aligned16(dy) || !aligned16(w) || !aligned16(dx) || !aligned16(relu_mask_src) || !aligned16(dx_colsum))
+        return PCL_ERR_MISALIGNED;
+    const size_t need = pcl_conv_bwd_data_colsum_workspace_bytes(d);
+    if (need > 0) {
+        if (!ws || ws_bytes < need) return PCL_ERR_WORKSPACE;
+        if (reinterpret_cast<uintptr_t>(ws) & 255) return PCL_ERR_MISALIGNED;
+    }
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    const size_t base = pcl_conv_workspace_bytes(d, PCL_PASS_BWD_DATA);
+    char* extra = static_cast<char*>(ws) + base;
+    long rows = 0;
+    if (tensor_path_for(*d, PCL_PASS_BWD_DATA) && d->C % 4 == 0)
+        rows = tc_fprop_colsum_rows(bwd_data_args(*d, P, Q, nullptr, nullptr, nullptr, nullptr));
+    if (rows > 0) {
+        float* wt_t = static_cast<float*>(ws);
+        rc = launch_transpose_flip(w, wt_t, d->K, d->R, d->S, d->C, st);
+        if (rc != PCL_OK) return rc;
+        TcFpropArgs a = bwd_data_args(*d, P, Q, dy, wt_t, relu_mask_src, dx);
+        float* sum_rows = reinterpret_cast<float*>(extra);
+        a.colsum_rows = sum_rows;
+        // rows the chosen tiling does not write must not contribute: the sizing took the largest tiling
+        rc = launch_zero(sum_rows, size_t(rows) * d->C, st);
+        if (rc != PCL_OK) return rc;
+        rc = launch_tc_fprop(a, st);
+        if (rc != PCL_OK) return rc;
+        float* partial = reinterpret_cast<float*>(extra + align_up(size_t(rows) * d->C * 4, 256));
+        return launch_colsum(sum_rows, size_t(rows), d->C, partial, dx_colsum, st);
+    }
+    rc = pcl_conv_bwd_data(d, dy, w, relu_mask_src, dx, ws, base, cuda_stream);
+    if (rc != PCL_OK) return rc;
+    return launch_colsum(dx, size_t(d->N) * d->H * d->W, d->C, reinterpret_cast<float*>(extra), dx_colsum, st);
+}
+
+size_t pcl_maxpool2x2_bwd_colsum_workspace_bytes(int N, int H, int W, int C) {
+    if (N <= 0 || H <= 0 || W <= 0 || C <= 0) return 0;
+    const long rows = maxpool_bwd_colsum_rows(N, H, W, C);
+    if (rows > 0) return colsum_stage_bytes(rows, C);
+    const int cs = colsum_splits(size_t(N) * H * W);
+    return cs > 1 ? align_up(size_t(cs) * C * 4, 256) : 0;
+}
+
+int pcl_maxpool2x2_bwd_colsum(int N, int H, int W, int C, const float* x, const float* dy, const float* relu_mask_src,
+                              float* dx, float* dx_colsum, void* ws, size_t ws_bytes, void* cuda_stream) {
+    if (N <= 0 || H <= 0 || W <= 0 || C <= 0 || !x || !dy || !dx || !dx_colsum) return PCL_ERR_BAD_ARG;
+    if ((H | W) & 1) return PCL_ERR_UNSUPPORTED_SHAPE;
+    if (!aligned16(x) || !aligned16(dy) || !aligned16(dx) || !aligned16(relu_mask_src) || !aligned16(dx_colsum))
+        return PCL_ERR_MISALIGNED;
+    const size_t need = pcl_maxpool2x2_bwd_colsum_workspace_bytes(N, H, W, C);
+    if (need > 0) {
+        if (!ws || ws_bytes < need) return PCL_ERR_WORKSPACE;
+        if (reinterpret_cast<uintptr_t>(ws) & 255) return PCL_ERR_MISALIGNED;
+    }
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    const long rows = maxpool_bwd_colsum_rows(N, H, W, C);
+    if (rows > 0) {
+        float* sum_rows = static_cast<float*>(ws);
+        int rc = launch_maxpool_bwd_colsum(N, H, W, C, x, dy, relu_mask_src, dx, sum_rows, st);
+        if (rc != PCL_OK) return rc;
+        float* partial = reinterpret_cast<float*>(static_cast<char*>(ws) + align_up(size_t(rows) * C * 4, 256));
+        return launch_colsum(sum_rows, size_t(rows), C, partial, dx_colsum, st);
+    }
+    int rc = launch_maxpool_bwd(N, H, W, C, x, dy, relu_mask_src, dx, st);
+    if (rc != PCL_OK) return rc;
+    return launch_colsum(dx, size_t(N) * H * W, C, static_cast<float*>(ws), dx_colsum, st);
+}
+
 int pcl_conv_bwd_weights(const pcl_conv_desc* d, const float* x, const float* dy, float* dw, float* dbias,
                          int deterministic, void* ws, size_t ws_bytes, void* cuda_stream) {
     int P, Q;

@@ -64,8 +64,13 @@ struct TcFpropArgs {
     // elements carry weight: the rest of the window is real neighbouring data that meets zero weights, which
     // avoids TMA's slower partial-row zero fill.
     int in_inner = 0;
+    // Optional fused column sums of the output (after bias / activation / mask): every (tile box, 32-row
+    // quarter) writes one row of per-column sums to `colsum_rows` ([tc_fprop_colsum_rows(a)][Kout], fully
+    // written when Kout % 4 == 0); the caller adds the rows up in a fixed order.
+    float* colsum_rows = nullptr;
 };
 bool tc_fprop_eligible(const TcFpropArgs& a);
+long tc_fprop_colsum_rows(const TcFpropArgs& a);
 int launch_tc_fprop(const TcFpropArgs& a, cudaStream_t st);
 
 // ---- weight-gradient-type GEMM on tcgen05 (stride-1 convolution) -----------
@@ -121,6 +126,11 @@ int launch_colsum(const float* m, size_t rows, int K, float* partial, float* out
 int launch_maxpool_fwd(int N, int H, int W, int C, const float* x, float* y, cudaStream_t st);
 int launch_maxpool_bwd(int N, int H, int W, int C, const float* x, const float* dy, const float* mask, float* dx,
                        cudaStream_t st);
+// The same with fused per-block column sums of dx: colsum_rows is [maxpool_bwd_colsum_rows(N,H,W,C)][C]; returns 0
+// rows when the shape cannot take the fused form (then use launch_colsum on dx).
+long maxpool_bwd_colsum_rows(int N, int H, int W, int C);
+int launch_maxpool_bwd_colsum(int N, int H, int W, int C, const float* x, const float* dy, const float* mask,
+                              float* dx, float* colsum_rows, cudaStream_t st);
 int launch_softmax_xent(int N, int K, const float* logits, const int* labels, float* loss, float* dlogits,
                         cudaStream_t st);
 

@@ -59,6 +59,7 @@ struct FpropParams {
     const float* bias;
     const float* mask_src;
     float* out;
+    float* colsum_rows;         // optional [m_tiles * MT * 4][Kout] per-(box, quarter) column sums of the output
     unsigned int* status;       // device status word
 };
 
@@ -303,6 +304,11 @@ tc_fprop_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
             const bool valid = (q < p.Q) && (pp < p.P) && (n < p.N);
             const size_t pix = (static_cast<size_t>(n) * p.P + pp) * p.Q + q;
             const uint32_t t_row = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + (acc * p.MT + h) * p.BN;
+            float* cs_row = nullptr;
+            if (p.colsum_rows) {
+                const size_t m_index = (static_cast<size_t>(it.ni) * p.tiles_p + it.pi) * p.tiles_q + it.qi;
+                cs_row = p.colsum_rows + ((m_index * p.MT + h) * 4 + quarter) * p.Kout;
+            }
             if (vec_ok) {
                 // Coalesced path.  Each lane owns one row (pixel) of the accumulator, but a row's 32 columns
                 // are 128 contiguous bytes in global memory, so the chunk is first transposed through a
@@ -332,9 +338,11 @@ tc_fprop_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                     }
                     __syncwarp();
                     const int col = kt * p.BN + ch * 32 + cg;
+                    const unsigned live = __ballot_sync(0xffffffffu, col < p.Kout);   // lanes l, l^8, l^16 agree
                     if (col < p.Kout) {
                         float4 b = make_float4(0.f, 0.f, 0.f, 0.f);
                         if (p.bias) b = __ldg(reinterpret_cast<const float4*>(p.bias + col));
+                        float4 csum = make_float4(0.f, 0.f, 0.f, 0.f);
                         float4 mk[8];
                         if (p.mask_src) {
 #pragma unroll
@@ -362,7 +370,16 @@ tc_fprop_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                                     o.z = mk[i].z > 0.f ? o.z : 0.f; o.w = mk[i].w > 0.f ? o.w : 0.f;
                                 }
                                 *reinterpret_cast<float4*>(p.out + roff[i] + col) = o;
+                                csum.x += o.x; csum.y += o.y; csum.z += o.z; csum.w += o.w;
                             }
+                        }
+                        if (cs_row) {
+                            // rows (lane>>3) + 4i were summed per lane; add the four lane groups in a fixed order
+                            csum.x += __shfl_xor_sync(live, csum.x, 8);  csum.y += __shfl_xor_sync(live, csum.y, 8);
+                            csum.z += __shfl_xor_sync(live, csum.z, 8);  csum.w += __shfl_xor_sync(live, csum.w, 8);
+                            csum.x += __shfl_xor_sync(live, csum.x, 16); csum.y += __shfl_xor_sync(live, csum.y, 16);
+                            csum.z += __shfl_xor_sync(live, csum.z, 16); csum.w += __shfl_xor_sync(live, csum.w, 16);
+                            if (lane < 8) *reinterpret_cast<float4*>(cs_row + col) = csum;
                         }
                     }
                     __syncwarp();
@@ -504,34 +521,73 @@ TileCfg halo_cfg(const TcFpropArgs& a, int cblocks, int sm_count, int layout) {
     return c;
 }
 
-}  // namespace
-
-int launch_tc_fprop(const TcFpropArgs& a, cudaStream_t st) {
-    if (!tc_fprop_eligible(a)) return PCL_ERR_UNSUPPORTED_SHAPE;
-    if (g_sm_count == 0) {
-        int dev = 0;
-        if (cudaGetDevice(&dev) != cudaSuccess) return PCL_ERR_CUDA;
-        if (cudaDeviceGetAttribute(&g_sm_count, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return PCL_ERR_CUDA;
-        if (cudaFuncSetAttribute(tc_fprop_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget + 1024) !=
-            cudaSuccess)
-            return PCL_ERR_CUDA;
-    }
-    FpropParams p{};
-    p.cblocks = (a.Cin + kBlockC - 1) / kBlockC;
-    TileCfg cfg = plain_cfg(a, p.cblocks, g_sm_count);
-    if (!cfg.ok) return PCL_ERR_UNSUPPORTED_SHAPE;
+// The tiling a launch will use (also needed to size the fused column-sum rows).
+TileCfg select_cfg(const TcFpropArgs& a, int sm_count) {
+    const int cblocks = (a.Cin + kBlockC - 1) / kBlockC;
+    TileCfg cfg = plain_cfg(a, cblocks, sm_count);
+    if (!cfg.ok) return cfg;
     // Test hook: PCL_TILING = plain | halo0 | halo1 | halo2 pins the tiling (when that tiling is possible).
     const char* pin = getenv("PCL_TILING");
     const int pinned = !pin ? -2 : (pin[0] == 'p' ? -1 : (pin[0] == 'h' && pin[4] >= '0' && pin[4] <= '2' ? pin[4] - '0' : -2));
     for (int layout = 0; layout < 3; ++layout) {
-        const TileCfg h = halo_cfg(a, p.cblocks, g_sm_count, layout);
+        const TileCfg h = halo_cfg(a, cblocks, sm_count, layout);
         if (!h.ok) continue;
         if (pinned == layout) { cfg = h; break; }
-        // Measured on B200: a row-shifted (not 1024-byte aligned) A view costs the tensor core extra shared
-        // memory cycles, so the haloed tiling only pays where the plain one is starved by operand traffic:
-        // narrow layers (BN <= 128) tiled without ragged edges by two boxes that share every weight tile.
+        // Measured on B200: the haloed tiling only pays where the plain one is starved by operand traffic,
+        // i.e. narrow layers (BN <= 128) tiled without ragged edges by two boxes that share every weight tile;
+        // wide layers already run at the power-limited tensor rate with the plain tiling.
         if (pinned == -2 && layout > 0 && h.BN <= 128 && a.Q % h.tw == 0 && a.P % h.th == 0) { cfg = h; break; }
     }
+    return cfg;
+}
+
+}  // namespace
+
+static int ensure_device_setup() {
+    if (g_sm_count == 0) {
+        int dev = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess) return PCL_ERR_CUDA;
+        if (cudaDeviceGetAttribute(&g_sm_count, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return PCL_ERR_CUDA;
+    }
+    return PCL_OK;
+}
+
+long tc_fprop_colsum_rows(const TcFpropArgs& a) {
+    int sm = g_sm_count;
+    if (sm == 0) {      // sizing query before any launch (possibly without a device): use the B200 SM count
+        int dev = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess ||
+            cudaDeviceGetAttribute(&sm, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sm <= 0)
+            sm = 148;
+    }
+    if (a.Kout % 4 != 0) return 0;
+    // rows are independent of BN, but the haloed / plain choice depends on it: take the larger of all tilings
+    long rows = 0;
+    const int cblocks = (a.Cin + kBlockC - 1) / kBlockC;
+    const TileCfg pc = plain_cfg(a, cblocks, sm);
+    if (pc.ok) rows = long(pc.tiles_q) * pc.tiles_p * pc.tiles_n * 4;
+    for (int layout = 0; layout < 3; ++layout) {
+        const TileCfg h = halo_cfg(a, cblocks, sm, layout);
+        const long r = h.ok ? long(h.tiles_q) * h.tiles_p * h.tiles_n * h.MT * 4 : 0;
+        if (r > rows) rows = r;
+    }
+    return rows;
+}
+
+int launch_tc_fprop(const TcFpropArgs& a, cudaStream_t st) {
+    if (!tc_fprop_eligible(a)) return PCL_ERR_UNSUPPORTED_SHAPE;
+    static bool attr_set = false;
+    if (!attr_set) {
+        if (ensure_device_setup() != PCL_OK) return PCL_ERR_CUDA;
+        if (cudaFuncSetAttribute(tc_fprop_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget + 1024) !=
+            cudaSuccess)
+            return PCL_ERR_CUDA;
+        attr_set = true;
+    }
+    FpropParams p{};
+    p.cblocks = (a.Cin + kBlockC - 1) / kBlockC;
+    const TileCfg cfg = select_cfg(a, g_sm_count);
+    if (!cfg.ok) return PCL_ERR_UNSUPPORTED_SHAPE;
     p.halo = cfg.halo; p.MT = cfg.MT; p.bw_log2 = cfg.bw_log2; p.bh_log2 = cfg.bh_log2;
     p.tw = cfg.tw; p.th = cfg.th; p.tn = cfg.tn; p.half_dq = cfg.half_dq; p.half_dp = cfg.half_dp;
     p.tiles_q = cfg.tiles_q; p.tiles_p = cfg.tiles_p; p.tiles_n = cfg.tiles_n; p.tiles_k = cfg.tiles_k;
@@ -546,6 +602,8 @@ int launch_tc_fprop(const TcFpropArgs& a, cudaStream_t st) {
     p.tmem_cols = 32;
     while (p.tmem_cols < 2 * p.MT * p.BN) p.tmem_cols *= 2;
     p.bias = a.bias; p.mask_src = a.mask_src; p.out = a.out;
+    p.colsum_rows = (a.Kout % 4 == 0) ? a.colsum_rows : nullptr;
+    if (a.colsum_rows && !p.colsum_rows) return PCL_ERR_UNSUPPORTED_SHAPE;
     p.status = device_status_ptr();
     if (!p.status) return PCL_ERR_CUDA;
 

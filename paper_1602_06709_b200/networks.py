@@ -110,7 +110,9 @@ class VggA:
         self.loss = torch.zeros(1, device=dev)
         ws = 0
         for L in self.convs:
-            ws = max(ws, B.conv_workspace_bytes(L.desc, B.PASS_BWD_DATA), B.conv_workspace_bytes(L.desc, B.PASS_BWD_WEIGHTS))
+            ws = max(ws, B.conv_workspace_bytes(L.desc, B.PASS_FWD), B.conv_workspace_bytes(L.desc, B.PASS_BWD_DATA),
+                     B.conv_workspace_bytes(L.desc, B.PASS_BWD_WEIGHTS), B.conv_bwd_data_colsum_workspace_bytes(L.desc),
+                     B.maxpool2x2_bwd_colsum_workspace_bytes(N, L.H, L.W, L.K))
         for C, K in fc:
             ws = max(ws, B.fc_workspace_bytes(N, C, K, B.PASS_BWD_DATA))
         self.ws = torch.empty(max(ws, 256), dtype=torch.uint8, device=dev)
@@ -157,15 +159,19 @@ class VggA:
                      self.fc_db(j), self.ws)
         for i in reversed(range(len(self.convs))):
             L = self.convs[i]
+            # The bias gradient of layer i is the per-map sum of dy[i]; it is formed by whichever kernel writes
+            # dy[i] (the pool backward here, or the backward-data pass of layer i+1 below), not by a separate pass.
             if L.pool:   # gradient through the pool, then through the ReLU (fused mask)
-                B.maxpool2x2_bwd(self.N, L.H, L.W, L.K, self.y[i], self.dpooled[i], self.y[i], self.dy[i])
-            B.conv_bwd_weights(L.desc, self.layer_input(i), self.dy[i], self.conv_dw(i), self.conv_db(i), True, self.ws)
+                B.maxpool2x2_bwd_colsum(self.N, L.H, L.W, L.K, self.y[i], self.dpooled[i], self.y[i], self.dy[i],
+                                        self.conv_db(i), self.ws)
+            B.conv_bwd_weights(L.desc, self.layer_input(i), self.dy[i], self.conv_dw(i), None, True, self.ws)
             if i > 0:
                 prev = self.convs[i - 1]
                 if prev.pool:
                     B.conv_bwd_data(L.desc, self.dy[i], self.conv_w(i), None, self.dpooled[i - 1], self.ws)
-                else:   # the layer's input is the previous ReLU output: fuse its mask
-                    B.conv_bwd_data(L.desc, self.dy[i], self.conv_w(i), self.y[i - 1], self.dy[i - 1], self.ws)
+                else:   # the layer's input is the previous ReLU output: fuse its mask (and its bias gradient)
+                    B.conv_bwd_data_colsum(L.desc, self.dy[i], self.conv_w(i), self.y[i - 1], self.dy[i - 1],
+                                           self.conv_db(i - 1), self.ws)
 
     def update(self):
         B.sgd_update(self.store.params, self.store.grads, self.lr)

@@ -128,3 +128,49 @@ def test_softmax_xent(N, K):
     assert abs(loss.item() - loss_ref) <= 1e-5 * max(1.0, abs(loss_ref))
     G.assert_parity(dz.cpu().numpy(), dz_ref, "dlogits")
     np.testing.assert_allclose(dz.cpu().numpy(), dz_ref, rtol=1e-4, atol=1e-8)
+
+
+@pytest.mark.parametrize("N,H,W,C", [(2, 8, 6, 8), (3, 14, 14, 20), (2, 28, 28, 64), (1, 4, 4, 1024)])
+def test_maxpool_bwd_with_fused_column_sums(N, H, W, C):
+    import gpu_helpers as G
+    from paper_1602_06709_b200 import binding as B
+    from paper_1602_06709_b200 import inputs
+    x = np.maximum(inputs.normal(inputs.tensor_id("poolcs", N, H, W, C, "x"), (N, H, W, C), 1.0), 0.0)
+    dy = inputs.normal(inputs.tensor_id("poolcs", N, H, W, C, "dy"), (N, H // 2, W // 2, C), 1.0)
+    xt, dyt = G.dev(x), G.dev(dy)
+    dxt = torch.full((N, H, W, C), float("nan"), device="cuda")
+    cs = torch.full((C,), float("nan"), device="cuda")
+    ws = G.workspace(B.maxpool2x2_bwd_colsum_workspace_bytes(N, H, W, C))
+    B.maxpool2x2_bwd_colsum(N, H, W, C, xt, dyt, xt, dxt, cs, ws)
+    ref = oracle.maxpool2x2_bwd(x, dy, x)
+    assert np.array_equal(dxt.cpu().numpy(), ref.astype(np.float32))
+    G.assert_parity(cs.cpu().numpy(), ref.reshape(-1, C).sum(axis=0), "pool dx column sums")
+    cs2 = torch.empty_like(cs)
+    B.maxpool2x2_bwd_colsum(N, H, W, C, xt, dyt, xt, dxt, cs2, ws)
+    assert torch.equal(cs, cs2)
+
+
+@pytest.mark.parametrize("tiling", ["auto", "plain", "halo1"])
+@pytest.mark.parametrize("shape", [(3, 40, 72, 19, 23), (2, 64, 64, 32, 32), (2, 128, 320, 12, 12), (2, 7, 9, 11, 13)])
+def test_conv_bwd_data_with_fused_column_sums(shape, tiling, monkeypatch):
+    import gpu_helpers as G
+    from oracle import ConvShape
+    from paper_1602_06709_b200 import binding as B
+    if tiling != "auto":
+        monkeypatch.setenv("PCL_TILING", tiling)
+    N, C, K, H, W = shape
+    s = ConvShape(N=N, C=C, K=K, H=H, W=W, R=3, S=3, pad_h=1, pad_w=1)
+    x, w, dy, _ = G.make_inputs(s, f"dgradcs{C}")
+    d = G.shape_to_desc(s)
+    dx = torch.full((N, H, W, C), float("nan"), device="cuda")
+    cs = torch.full((C,), float("nan"), device="cuda")
+    ws = G.workspace(B.conv_bwd_data_colsum_workspace_bytes(d))
+    B.conv_bwd_data_colsum(d, G.dev(dy), G.dev(w), G.dev(x), dx, cs, ws)
+    B.check_device_status()
+    ref = oracle.conv_bwd_data(s, dy, w, x)
+    G.assert_parity(dx.cpu().numpy(), ref, "dx")
+    # the sums are of the GPU's own dx (per-call parity), formed in fp32 in a fixed order
+    G.assert_parity(cs.cpu().numpy(), dx.cpu().numpy().astype(np.float64).reshape(-1, C).sum(axis=0), "dx column sums")
+    cs2 = torch.empty_like(cs)
+    B.conv_bwd_data_colsum(d, G.dev(dy), G.dev(w), G.dev(x), dx, cs2, ws)
+    assert torch.equal(cs, cs2)
