@@ -46,6 +46,7 @@ struct FpropParams {
     int N, P, Q, Kout;
     int act;
     int stages;
+    int KS;                     // k-steps (plain: {A,B} pairs; halo: weight tiles of consecutive taps) per pipeline slot
     int tmem_cols;
     int tw, th, tn;             // pixels a tile spans in q, p, n (= the box, or 2 x the box in one direction when MT = 2)
     // Halo mode (R*S > 1): the A operand of ALL taps of a channel block comes from one haloed input patch
@@ -105,8 +106,11 @@ tc_fprop_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
     const int lane = threadIdx.x & 31;
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     // plain mode: ring of {A 16 KB, B BN*128 B} slots.  halo mode: NA patch buffers, then a ring of B slots.
+    // A slot holds KS k-steps: the issuing thread pays one barrier round trip and one commit per slot, which
+    // is what bounds narrow tiles (their MMAs are short), so narrow tiles batch several k-steps per slot.
     const uint32_t b_bytes = p.BN * 128;
-    const uint32_t stage_bytes = p.halo ? b_bytes : kABytes + b_bytes;
+    const uint32_t step_bytes = p.halo ? b_bytes : kABytes + b_bytes;
+    const uint32_t stage_bytes = p.KS * step_bytes;
     uint8_t* b_ring = smem + (p.halo ? p.NA * p.a_buf_bytes : kABytes);
     uint8_t* epi_stage = smem + (p.halo ? p.NA * p.a_buf_bytes : 0) + p.stages * stage_bytes;   // 8 x 4 KB
 
@@ -165,35 +169,40 @@ tc_fprop_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                                     q0 - p.pad_w, p0 - p.pad_h, n0);
                         ++issuedA;
                         if (++a_slot == p.NA) { a_slot = 0; phaseA ^= 1u; }
-                        for (int tap = 0; tap < p.R * p.S; ++tap) {
+                        for (int tap = 0; tap < p.R * p.S; tap += p.KS) {
                             if (!bounded_wait(&empty_bar[stage], phase ^ 1u, &abort_flag, p.status, WAIT_PRODUCER_EMPTY)) {
                                 ok = false;
                                 break;
                             }
-                            mbar_expect_tx(&full_bar[stage], b_bytes);
-                            tma_load_3d(b_ring + stage * stage_bytes, &tmB, &full_bar[stage], cb * kBlockC, tap,
-                                        kt * p.BN);
+                            const int nst = p.R * p.S - tap < p.KS ? p.R * p.S - tap : p.KS;
+                            mbar_expect_tx(&full_bar[stage], nst * b_bytes);
+                            for (int j = 0; j < nst; ++j)
+                                tma_load_3d(b_ring + stage * stage_bytes + j * b_bytes, &tmB, &full_bar[stage],
+                                            cb * kBlockC, tap + j, kt * p.BN);
                             ++issued;
                             if (++stage == p.stages) { stage = 0; phase ^= 1u; }
                         }
                     }
                 } else {
-                    for (int r = 0; r < p.R && ok; ++r)
-                        for (int s = 0; s < p.S && ok; ++s)
-                            for (int cb = 0; cb < p.cblocks; ++cb) {
-                                if (!bounded_wait(&empty_bar[stage], phase ^ 1u, &abort_flag, p.status, WAIT_PRODUCER_EMPTY)) {
-                                    ok = false;
-                                    break;
-                                }
-                                uint8_t* a_dst = smem + stage * stage_bytes;
-                                mbar_expect_tx(&full_bar[stage], stage_bytes);
-                                tma_load_4d(a_dst, &tmA, &full_bar[stage], cb * kBlockC, q0 + s - p.pad_w,
-                                            p0 + r - p.pad_h, n0);
-                                tma_load_3d(a_dst + kABytes, &tmB, &full_bar[stage], cb * kBlockC, r * p.S + s,
-                                            kt * p.BN);
-                                ++issued;
-                                if (++stage == p.stages) { stage = 0; phase ^= 1u; }
-                            }
+                    int r = 0, s = 0, cb = 0;        // k-step order: r, then s, then channel block
+                    for (int kit = 0; kit < kiters; kit += p.KS) {
+                        if (!bounded_wait(&empty_bar[stage], phase ^ 1u, &abort_flag, p.status, WAIT_PRODUCER_EMPTY)) {
+                            ok = false;
+                            break;
+                        }
+                        const int nst = kiters - kit < p.KS ? kiters - kit : p.KS;
+                        mbar_expect_tx(&full_bar[stage], nst * step_bytes);
+                        for (int j = 0; j < nst; ++j) {
+                            uint8_t* a_dst = smem + stage * stage_bytes + j * step_bytes;
+                            tma_load_4d(a_dst, &tmA, &full_bar[stage], cb * kBlockC, q0 + s - p.pad_w,
+                                        p0 + r - p.pad_h, n0);
+                            tma_load_3d(a_dst + kABytes, &tmB, &full_bar[stage], cb * kBlockC, r * p.S + s,
+                                        kt * p.BN);
+                            if (++cb == p.cblocks) { cb = 0; if (++s == p.S) { s = 0; ++r; } }
+                        }
+                        ++issued;
+                        if (++stage == p.stages) { stage = 0; phase ^= 1u; }
+                    }
                 }
             }
             if (!ok) {
@@ -237,40 +246,49 @@ tc_fprop_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                 for (int cb = 0; cb < p.cblocks && ok; ++cb) {
                     if (!bounded_wait_warp(&fullA_bar[a_slot], phaseA, &abort_flag, p.status, WAIT_MMA_FULL)) { ok = false; break; }
                     const uint32_t a_base = smem_u32(smem + a_slot * p.a_buf_bytes);
-                    int tap = 0;
-                    for (int r = 0; r < p.R && ok; ++r)
-                        for (int s = 0; s < p.S; ++s, ++tap) {
-                            if (!bounded_wait_warp(&full_bar[stage], phase, &abort_flag, p.status, WAIT_MMA_FULL)) { ok = false; break; }
-                            tc_fence_after();
-                            if (lane == 0) {
-                                const uint64_t db = b_desc0 + ((smem_u32(b_ring + stage * stage_bytes) & 0x3FFFFu) >> 4);
+                    int r = 0, s = 0;
+                    for (int tap = 0; tap < p.R * p.S && ok; tap += p.KS) {
+                        if (!bounded_wait_warp(&full_bar[stage], phase, &abort_flag, p.status, WAIT_MMA_FULL)) { ok = false; break; }
+                        tc_fence_after();
+                        const int nst = p.R * p.S - tap < p.KS ? p.R * p.S - tap : p.KS;
+                        if (lane == 0) {
+                            uint64_t db = b_desc0 + ((smem_u32(b_ring + stage * stage_bytes) & 0x3FFFFu) >> 4);
+                            for (int j = 0; j < nst; ++j) {
                                 // the tap = a row shift inside the patch
                                 const uint64_t da = a_desc0 + (((a_base + (r * p.PW + s) * 128) & 0x3FFFFu) >> 4);
                                 for (int h = 0; h < p.MT; ++h) {
 #pragma unroll
                                     for (int kk = 0; kk < 4; ++kk)
                                         umma_tf32(d_tmem + h * p.BN, da + h * half_off16 + kk * 2, db + kk * 2, idesc,
-                                                  (cb | tap | kk) != 0);
+                                                  (cb | tap | j | kk) != 0);
                                 }
-                                umma_commit(&empty_bar[stage]);
+                                db += b_bytes >> 4;
+                                if (++s == p.S) { s = 0; ++r; }
                             }
-                            __syncwarp();
-                            if (++stage == p.stages) { stage = 0; phase ^= 1u; }
+                            umma_commit(&empty_bar[stage]);
                         }
+                        __syncwarp();
+                        if (++stage == p.stages) { stage = 0; phase ^= 1u; }
+                    }
                     if (ok && lane == 0) umma_commit(&emptyA_bar[a_slot]);
                     __syncwarp();
                     if (++a_slot == p.NA) { a_slot = 0; phaseA ^= 1u; }
                 }
             } else {
                 const uint64_t desc0 = make_smem_desc(0, 16, 1024, kSwizzle128B);
-                for (int kit = 0; kit < kiters; ++kit) {
+                for (int kit = 0; kit < kiters; kit += p.KS) {
                     if (!bounded_wait_warp(&full_bar[stage], phase, &abort_flag, p.status, WAIT_MMA_FULL)) { ok = false; break; }
                     tc_fence_after();
+                    const int nst = kiters - kit < p.KS ? kiters - kit : p.KS;
                     if (lane == 0) {
-                        const uint64_t da = desc0 + ((smem_u32(smem + stage * stage_bytes) & 0x3FFFFu) >> 4);
-                        const uint64_t db = da + (kABytes >> 4);
+                        uint64_t da = desc0 + ((smem_u32(smem + stage * stage_bytes) & 0x3FFFFu) >> 4);
+                        for (int j = 0; j < nst; ++j) {
+                            const uint64_t db = da + (kABytes >> 4);
 #pragma unroll
-                        for (int kk = 0; kk < 4; ++kk) umma_tf32(d_tmem, da + kk * 2, db + kk * 2, idesc, (kit | kk) != 0);
+                            for (int kk = 0; kk < 4; ++kk)
+                                umma_tf32(d_tmem, da + kk * 2, db + kk * 2, idesc, (kit | j | kk) != 0);
+                            da += step_bytes >> 4;
+                        }
                         umma_commit(&empty_bar[stage]);
                     }
                     __syncwarp();
@@ -469,11 +487,16 @@ namespace {
 
 // One way of tiling a layer: plain (a box of 128 pixels, one TMA box per tap) or halo (MT boxes of 8 x 16
 // pixels cut from one haloed patch per channel block).
+int env_int(const char* name, int dflt) {       // test / tuning hook
+    const char* v = getenv(name);
+    return v ? atoi(v) : dflt;
+}
+
 struct TileCfg {
     bool ok = false;
     int halo = 0, MT = 1, bw_log2 = 0, bh_log2 = 0, tw = 0, th = 0, tn = 0, half_dq = 0, half_dp = 0;
     int tiles_q = 0, tiles_p = 0, tiles_n = 0, tiles_k = 0, BN = 0;
-    int PW = 0, patch_bytes = 0, a_buf_bytes = 0, NA = 0, half_off_bytes = 0, stages = 0;
+    int PW = 0, patch_bytes = 0, a_buf_bytes = 0, NA = 0, half_off_bytes = 0, stages = 0, KS = 1;
 };
 
 TileCfg plain_cfg(const TcFpropArgs& a, int cblocks, int sm_count) {
@@ -484,7 +507,12 @@ TileCfg plain_cfg(const TcFpropArgs& a, int cblocks, int sm_count) {
     const long m_tiles = long(c.tiles_q) * c.tiles_p * c.tiles_n;
     c.BN = choose_bn(a.Kout, m_tiles, sm_count);
     c.tiles_k = (a.Kout + c.BN - 1) / c.BN;
-    c.stages = (kSmemBudget - kEpiStageBytes) / (kABytes + c.BN * 128);
+    // narrow tiles: several k-steps per slot (see the kernel), as long as 4 slots still fit
+    c.KS = env_int("PCL_KS", c.BN <= 128 ? 2 : 1);
+    const int kiters = a.R * a.S * cblocks;
+    if (c.KS > kiters) c.KS = kiters;
+    while (c.KS > 1 && (kSmemBudget - kEpiStageBytes) / (c.KS * (kABytes + c.BN * 128)) < 3) --c.KS;
+    c.stages = (kSmemBudget - kEpiStageBytes) / (c.KS * (kABytes + c.BN * 128));
     if (c.stages > kMaxStages) c.stages = kMaxStages;
     c.ok = c.stages >= 2;
     return c;
@@ -510,10 +538,14 @@ TileCfg halo_cfg(const TcFpropArgs& a, int cblocks, int sm_count, int layout) {
     c.tiles_k = (a.Kout + c.BN - 1) / c.BN;
     const int room = kSmemBudget - kEpiStageBytes;
     c.NA = 2;
-    c.stages = (room - c.NA * c.a_buf_bytes) / (c.BN * 128);
-    if (c.stages >= 9 && (room - 3 * c.a_buf_bytes) / (c.BN * 128) >= 6) {
+    c.KS = env_int("PCL_KS_HALO", c.BN <= 64 ? 3 : (c.BN <= 128 ? 2 : 1));
+    if (c.KS > a.R * a.S) c.KS = a.R * a.S;
+    while (c.KS > 1 && (room - c.NA * c.a_buf_bytes) / (c.KS * c.BN * 128) < 3) --c.KS;
+    const int slot = c.KS * c.BN * 128;
+    c.stages = (room - c.NA * c.a_buf_bytes) / slot;
+    if (c.stages >= 9 && (room - 3 * c.a_buf_bytes) / slot >= 6) {
         c.NA = 3;
-        c.stages = (room - 3 * c.a_buf_bytes) / (c.BN * 128);
+        c.stages = (room - 3 * c.a_buf_bytes) / slot;
     }
     if (c.stages > kMaxStages) c.stages = kMaxStages;
     if (c.stages < 3) return c;
@@ -592,7 +624,7 @@ int launch_tc_fprop(const TcFpropArgs& a, cudaStream_t st) {
     p.tw = cfg.tw; p.th = cfg.th; p.tn = cfg.tn; p.half_dq = cfg.half_dq; p.half_dp = cfg.half_dp;
     p.tiles_q = cfg.tiles_q; p.tiles_p = cfg.tiles_p; p.tiles_n = cfg.tiles_n; p.tiles_k = cfg.tiles_k;
     p.BN = cfg.BN; p.PW = cfg.PW; p.patch_bytes = cfg.patch_bytes; p.a_buf_bytes = cfg.a_buf_bytes; p.NA = cfg.NA;
-    p.half_off_bytes = cfg.half_off_bytes; p.stages = cfg.stages;
+    p.half_off_bytes = cfg.half_off_bytes; p.stages = cfg.stages; p.KS = cfg.KS;
     const int bw = 1 << p.bw_log2, bh = 1 << p.bh_log2, bn = kTileM / (bw * bh);
     const long m_tiles = long(p.tiles_q) * p.tiles_p * p.tiles_n;
     if (m_tiles * p.tiles_k > 0x7fffffffL) return PCL_ERR_UNSUPPORTED_SHAPE;
@@ -629,8 +661,8 @@ int launch_tc_fprop(const TcFpropArgs& a, cudaStream_t st) {
     }
     const long total = m_tiles * p.tiles_k;
     const int grid = int(total < g_sm_count ? total : g_sm_count);
-    const size_t smem = (p.halo ? size_t(p.NA) * p.a_buf_bytes + size_t(p.stages) * p.BN * 128
-                                : size_t(p.stages) * (kABytes + p.BN * 128)) + kEpiStageBytes + 1024;
+    const size_t smem = (p.halo ? size_t(p.NA) * p.a_buf_bytes + size_t(p.stages) * p.KS * p.BN * 128
+                                : size_t(p.stages) * p.KS * (kABytes + p.BN * 128)) + kEpiStageBytes + 1024;
     {
         LaunchScope scope(KID_TC_FPROP, 2.0 * a.N * a.P * a.Q * double(a.Kout) * a.Cin * a.R * a.S, st);
         tc_fprop_kernel<<<grid, kThreads, smem, st>>>(tmA, tmB, p);
