@@ -23,6 +23,8 @@
 // accumulates its item in TMEM and either writes a partial tile to the
 // workspace (second pass adds the splits in a fixed order) or adds it to dw with
 // fp32 atomics.
+#include <stdlib.h>
+
 #include "pcl_internal.h"
 #include "pcl_ptx.cuh"
 
@@ -49,8 +51,11 @@ struct WgradParams {
     int K, C;
     int splits, boxes_per_split;
     int stages, tmem_cols;
+    int KS;                   // pixel boxes (k-steps of 32 pixels) per pipeline slot; > 1 for narrow column blocks
     int use_atomics;
-    int grouped;              // 5-D tensor maps (one TMA instruction per operand run) or 4-D per-group boxes (L == 1)
+    int grouped;              // x: 5-D tensor map (one TMA instruction per run) or 4-D per-group boxes (L == 1)
+    int grouped_dy;           // dy: 5-D tensor map (all four 32-map groups in one instruction)
+    int x_taprows;            // x: 5-D map whose 5th dimension is the tap row (few-channel path): one instruction per k-step
     float* out;               // dw, or the partial-sum workspace [splits][K*R*S*C]
     size_t split_stride;      // K*R*S*C (0 when writing straight to dw)
     unsigned int* status;     // device status word
@@ -77,7 +82,8 @@ tc_wgrad_kernel(const __grid_constant__ CUtensorMap tmDy, const __grid_constant_
     const int run0 = rb * p.rpi;
     const int nruns = (run0 + p.rpi <= p.total_runs) ? p.rpi : p.total_runs - run0;
     const int n_groups = nruns * p.L;                 // 32-column groups of this item's MMA
-    const uint32_t stage_bytes = kABytes + p.rpi * p.L * kGroupBytes;   // slot size (same for every item)
+    const uint32_t step_bytes = kABytes + p.rpi * p.L * kGroupBytes;    // one k-step (same for every item)
+    const uint32_t stage_bytes = p.KS * step_bytes;                     // a slot holds KS k-steps
     const uint32_t tx_bytes = kABytes + n_groups * kGroupBytes;
 
     if (threadIdx.x == 0) {
@@ -130,14 +136,26 @@ tc_wgrad_kernel(const __grid_constant__ CUtensorMap tmDy, const __grid_constant_
             int pi = (box_begin / p.boxes_q) % p.boxes_p;
             int ni = box_begin / (p.boxes_q * p.boxes_p);
             const uint32_t run_bytes = p.L * kGroupBytes;
+            int sub = 0;                                         // position of the k-step inside its slot
             for (int b = box_begin; b < box_end; ++b) {
                 const int q0 = qi * bw, p0 = pi * bh, n0 = ni * bn;
                 if (++qi == p.boxes_q) { qi = 0; if (++pi == p.boxes_p) { pi = 0; ++ni; } }
-                if (!bounded_wait(&empty_bar[stage], phase ^ 1u, &abort_flag, p.status, WAIT_PRODUCER_EMPTY)) { ok = false; break; }
-                uint8_t* dst = smem + stage * stage_bytes;
-                mbar_expect_tx(&full_bar[stage], tx_bytes);
-                if (p.grouped) {
+                if (sub == 0) {
+                    if (!bounded_wait(&empty_bar[stage], phase ^ 1u, &abort_flag, p.status, WAIT_PRODUCER_EMPTY)) { ok = false; break; }
+                    const int nst = box_end - b < p.KS ? box_end - b : p.KS;
+                    mbar_expect_tx(&full_bar[stage], nst * tx_bytes);
+                }
+                uint8_t* dst = smem + stage * stage_bytes + sub * step_bytes;
+                if (p.grouped_dy) {
                     tma_load_5d(dst, &tmDy, &full_bar[stage], 0, q0, p0, n0, kt * 4);
+                } else {
+#pragma unroll
+                    for (int g = 0; g < 4; ++g)
+                        tma_load_4d(dst + g * kGroupBytes, &tmDy, &full_bar[stage], kt * 128 + g * 32, q0, p0, n0);
+                }
+                if (p.x_taprows) {
+                    tma_load_5d(dst + kABytes, &tmX, &full_bar[stage], 0, q0 + run_dw[0], p0 + run_dh[0], n0, 0);
+                } else if (p.grouped) {
 #pragma unroll
                     for (int j = 0; j < 8; ++j)
                         if (j < nruns)
@@ -145,16 +163,16 @@ tc_wgrad_kernel(const __grid_constant__ CUtensorMap tmDy, const __grid_constant_
                                         p0 + run_dh[j], n0, run_c[j]);
                 } else {
 #pragma unroll
-                    for (int g = 0; g < 4; ++g)
-                        tma_load_4d(dst + g * kGroupBytes, &tmDy, &full_bar[stage], kt * 128 + g * 32, q0, p0, n0);
-#pragma unroll
                     for (int j = 0; j < 8; ++j)
                         if (j < nruns)
                             tma_load_4d(dst + kABytes + j * run_bytes, &tmX, &full_bar[stage], run_c[j],
                                         q0 + run_dw[j], p0 + run_dh[j], n0);
                 }
-                ++issued;
-                if (++stage == p.stages) { stage = 0; phase ^= 1u; }
+                if (++sub == p.KS || b == box_end - 1) {
+                    sub = 0;
+                    ++issued;
+                    if (++stage == p.stages) { stage = 0; phase ^= 1u; }
+                }
             }
             if (!ok) {
                 // Gave up: copies already issued still land in this CTA's shared memory; wait (bounded) for them.
@@ -172,17 +190,20 @@ tc_wgrad_kernel(const __grid_constant__ CUtensorMap tmDy, const __grid_constant_
         int stage = 0;
         uint32_t phase = 0;
         bool ok = true;
-        for (int kit = 0; kit < kiters; ++kit) {
+        for (int kit = 0; kit < kiters; kit += p.KS) {
             if (!bounded_wait_warp(&full_bar[stage], phase, &abort_flag, p.status, WAIT_MMA_FULL)) { ok = false; break; }
             tc_fence_after();
+            const int nst = kiters - kit < p.KS ? kiters - kit : p.KS;
             if (lane == 0) {
+              for (int j = 0; j < nst; ++j) {
                 // 8 pixels per instruction = two 512-byte groups of 4 rows; descriptors differ only in the
                 // address field, so add offsets to a constant part
-                const uint64_t da = desc0 + ((smem_u32(smem + stage * stage_bytes) & 0x3FFFFu) >> 4);
+                const uint64_t da = desc0 + ((smem_u32(smem + stage * stage_bytes + j * step_bytes) & 0x3FFFFu) >> 4);
                 const uint64_t db = da + (kABytes >> 4);
 #pragma unroll
                 for (int kk = 0; kk < kPix / 8; ++kk)
-                    umma_tf32(tmem_base, da + kk * (1024 >> 4), db + kk * (1024 >> 4), idesc, (kit | kk) != 0);
+                    umma_tf32(tmem_base, da + kk * (1024 >> 4), db + kk * (1024 >> 4), idesc, (kit | j | kk) != 0);
+              }
                 umma_commit(&empty_bar[stage]);
             }
             __syncwarp();
@@ -341,7 +362,7 @@ int launch_tc_wgrad(const TcWgradArgs& a, cudaStream_t st) {
     const long boxes = long(p.boxes_q) * p.boxes_p * p.boxes_n;
     if (boxes > 0x7fffffffL) return PCL_ERR_UNSUPPORTED_SHAPE;
     const RunPlan rp = plan_runs(a.C, a.K, a.R, a.S, a.tap_groups);
-    p.grouped = rp.grouped; p.L = rp.L; p.runs_per_tap = rp.runs_per_tap; p.total_runs = rp.total_runs;
+    p.grouped = rp.grouped; p.grouped_dy = (a.K % 32 == 0) ? 1 : 0; p.x_taprows = a.tap_groups ? 1 : 0; p.L = rp.L; p.runs_per_tap = rp.runs_per_tap; p.total_runs = rp.total_runs;
     p.rpi = rp.rpi; p.run_blocks = rp.run_blocks;
     p.k_tiles = (a.K + 127) / 128;
     p.R = a.R; p.S = a.S; p.pad_h = a.pad_h; p.pad_w = a.pad_w;
@@ -349,7 +370,15 @@ int launch_tc_wgrad(const TcWgradArgs& a, cudaStream_t st) {
     p.splits = a.splits;
     p.boxes_per_split = int((boxes + p.splits - 1) / p.splits);
     const int max_groups = p.rpi * p.L;
-    const int stage_bytes = kABytes + max_groups * kGroupBytes;
+    const int step_bytes = kABytes + max_groups * kGroupBytes;
+    // A k-step of a narrow column block is 4 short MMAs; the issuing thread's per-slot round trip (~600
+    // cycles) then dominates, so such blocks get several k-steps per slot while at least 3 slots fit.
+    const int mma_clk = 4 * (max_groups * 16 > 52 ? max_groups * 16 : 52);
+    p.KS = (600 + mma_clk - 1) / mma_clk;
+    if (getenv("PCL_KS_WGRAD")) p.KS = atoi(getenv("PCL_KS_WGRAD"));
+    while (p.KS > 1 && kSmemBudget / (p.KS * step_bytes) < 3) --p.KS;
+    if (p.KS < 1) p.KS = 1;
+    const int stage_bytes = p.KS * step_bytes;
     p.stages = kSmemBudget / stage_bytes;
     if (p.stages > kMaxStages) p.stages = kMaxStages;
     p.tmem_cols = 32;
@@ -373,7 +402,7 @@ int launch_tc_wgrad(const TcWgradArgs& a, cudaStream_t st) {
     CUtensorMap tmDy, tmX;
     {
         const uint64_t sw = uint64_t(a.K), sh = uint64_t(a.Q) * a.K, sn = uint64_t(a.P) * a.Q * a.K;
-        if (p.grouped) {
+        if (p.grouped_dy) {
             const uint64_t dims[5] = {32, uint64_t(a.Q), uint64_t(a.P), uint64_t(a.N), uint64_t(a.K / 32)};
             const uint64_t strides[4] = {sw * 4, sh * 4, sn * 4, 128};
             const uint32_t box[5] = {32, uint32_t(bw), uint32_t(bh), uint32_t(bn), 4};
@@ -391,7 +420,17 @@ int launch_tc_wgrad(const TcWgradArgs& a, cudaStream_t st) {
         const uint64_t sw = a.x_stride_w ? uint64_t(a.x_stride_w) : uint64_t(a.C);
         const uint64_t sh = a.x_stride_h ? uint64_t(a.x_stride_h) : uint64_t(a.W) * a.C;
         const uint64_t sn = a.x_stride_n ? uint64_t(a.x_stride_n) : uint64_t(a.H) * a.W * a.C;
-        if (p.grouped) {
+        if (p.x_taprows) {
+            // few-channel path: the R tap rows of a pixel window are R boxes one image row apart; a 5th
+            // dimension with the row stride fetches them with one instruction (H extent shrinks by R-1 so
+            // that row + tap stays inside the staged image)
+            const uint64_t dims[5] = {uint64_t(a.x_inner ? a.x_inner : a.C), uint64_t(a.W), uint64_t(a.H - a.R + 1),
+                                      uint64_t(a.N), uint64_t(a.R)};
+            const uint64_t strides[4] = {sw * 4, sh * 4, sn * 4, sh * 4};
+            const uint32_t box[5] = {32, uint32_t(bw), uint32_t(bh), uint32_t(bn), uint32_t(a.R)};
+            int rc = make_tmap(&tmX, a.x, 5, dims, strides, box, true);
+            if (rc != PCL_OK) return rc;
+        } else if (p.grouped) {
             const uint64_t dims[5] = {32, uint64_t(a.W), uint64_t(a.H), uint64_t(a.N), uint64_t(a.C / 32)};
             const uint64_t strides[4] = {sw * 4, sh * 4, sn * 4, 128};
             const uint32_t box[5] = {32, uint32_t(bw), uint32_t(bh), uint32_t(bn), uint32_t(p.L)};
