@@ -41,6 +41,13 @@ METRIC = "conv fwd/bwd-data/bwd-wgt TFLOP/s and VGG-A images/sec at 1 B200 (% TF
 TF32_OVER_BF16_NOMINAL = 1.1 / 2.25      # nominal dense TF32 / bf16 tensor peaks
 FALLBACK_BF16_TFLOPS = 1590.0
 FALLBACK_HBM_GBS = 6650.0
+# dram__bytes_read.sum + dram__bytes_write.sum per launch from ncu (captured at minibatch 32 and scaled to the
+# full minibatch: weight bytes once, activation bytes x 8); source: profiles/vgga_step_n256_launch_list.md and
+# profiles/tc_fprop_tc_wgrad_conv256_56x56_n32.md
+NCU_DRAM_BYTES_PER_LAUNCH = {
+    "vgga": {"tc_fprop_kernel": 773.2e6, "tc_wgrad_kernel": 910.1e6},
+    "conv": {"tc_fprop_kernel": (164e6 + 284e6) / 2 * 8, "tc_wgrad_kernel": 209.5e6 * 8},
+}
 
 
 def load_peaks():
@@ -390,11 +397,7 @@ def run_ours(args):
         roofline = dict(bound="hbm", kernel=dom, achieved=achieved, peak=peaks["hbm_gbs"], unit="GB/s",
                         frac=achieved / peaks["hbm_gbs"], traffic=None, peak_source=f"{peaks['source']} copy bandwidth",
                         launches_per_step=ds["launches"] // prof_steps)
-    traffic_path = os.path.join(ROOT, "profiles", "traffic.json")
-    if os.path.exists(traffic_path):
-        with open(traffic_path) as f:
-            tr = json.load(f)
-        roofline["traffic"] = tr.get(args.workload, {}).get(dom)
+    roofline["traffic"] = NCU_DRAM_BYTES_PER_LAUNCH.get(args.workload, {}).get(dom)
 
     extra = {}
     tc = [stats[k] for k in ("tc_fprop_kernel", "tc_wgrad_kernel") if k in stats]
