@@ -224,6 +224,9 @@ tc_fprop_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
         }
     } else if (warp == 1) {
         // ---------------------------------------------------------- MMA issuer
+        // One thread runs the whole loop (waits included): a warp-wide wait + re-convergence per slot would
+        // add to the per-slot cost that bounds narrow tiles.
+        if (lane == 0) {
         const uint32_t idesc = make_idesc_tf32(p.BN, false, false);
         int stage = 0;
         uint32_t phase = 0;
@@ -234,7 +237,7 @@ tc_fprop_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
         for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x, ++tile_cnt) {
             const int acc = tile_cnt & 1;
             const uint32_t acc_phase = (tile_cnt >> 1) & 1;
-            if (!bounded_wait_warp(&tmem_empty_bar[acc], acc_phase ^ 1u, &abort_flag, p.status, WAIT_MMA_TMEM_EMPTY)) break;
+            if (!bounded_wait(&tmem_empty_bar[acc], acc_phase ^ 1u, &abort_flag, p.status, WAIT_MMA_TMEM_EMPTY)) break;
             tc_fence_after();
             const uint32_t d_tmem = tmem_base + acc * p.MT * p.BN;
             if (p.halo) {
@@ -244,14 +247,14 @@ tc_fprop_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                 const uint64_t b_desc0 = make_smem_desc(0, 16, 1024, kSwizzle128B);
                 const uint32_t half_off16 = p.half_off_bytes >> 4;
                 for (int cb = 0; cb < p.cblocks && ok; ++cb) {
-                    if (!bounded_wait_warp(&fullA_bar[a_slot], phaseA, &abort_flag, p.status, WAIT_MMA_FULL)) { ok = false; break; }
+                    if (!bounded_wait(&fullA_bar[a_slot], phaseA, &abort_flag, p.status, WAIT_MMA_FULL)) { ok = false; break; }
                     const uint32_t a_base = smem_u32(smem + a_slot * p.a_buf_bytes);
                     int r = 0, s = 0;
                     for (int tap = 0; tap < p.R * p.S && ok; tap += p.KS) {
-                        if (!bounded_wait_warp(&full_bar[stage], phase, &abort_flag, p.status, WAIT_MMA_FULL)) { ok = false; break; }
+                        if (!bounded_wait(&full_bar[stage], phase, &abort_flag, p.status, WAIT_MMA_FULL)) { ok = false; break; }
                         tc_fence_after();
                         const int nst = p.R * p.S - tap < p.KS ? p.R * p.S - tap : p.KS;
-                        if (lane == 0) {
+                        {
                             uint64_t db = b_desc0 + ((smem_u32(b_ring + stage * stage_bytes) & 0x3FFFFu) >> 4);
                             for (int j = 0; j < nst; ++j) {
                                 // the tap = a row shift inside the patch
@@ -267,20 +270,18 @@ tc_fprop_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                             }
                             umma_commit(&empty_bar[stage]);
                         }
-                        __syncwarp();
                         if (++stage == p.stages) { stage = 0; phase ^= 1u; }
                     }
-                    if (ok && lane == 0) umma_commit(&emptyA_bar[a_slot]);
-                    __syncwarp();
+                    if (ok) umma_commit(&emptyA_bar[a_slot]);
                     if (++a_slot == p.NA) { a_slot = 0; phaseA ^= 1u; }
                 }
             } else {
                 const uint64_t desc0 = make_smem_desc(0, 16, 1024, kSwizzle128B);
                 for (int kit = 0; kit < kiters; kit += p.KS) {
-                    if (!bounded_wait_warp(&full_bar[stage], phase, &abort_flag, p.status, WAIT_MMA_FULL)) { ok = false; break; }
+                    if (!bounded_wait(&full_bar[stage], phase, &abort_flag, p.status, WAIT_MMA_FULL)) { ok = false; break; }
                     tc_fence_after();
                     const int nst = kiters - kit < p.KS ? kiters - kit : p.KS;
-                    if (lane == 0) {
+                    {
                         uint64_t da = desc0 + ((smem_u32(smem + stage * stage_bytes) & 0x3FFFFu) >> 4);
                         for (int j = 0; j < nst; ++j) {
                             const uint64_t db = da + (kABytes >> 4);
@@ -291,13 +292,13 @@ tc_fprop_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                         }
                         umma_commit(&empty_bar[stage]);
                     }
-                    __syncwarp();
                     if (++stage == p.stages) { stage = 0; phase ^= 1u; }
                 }
             }
-            if (ok && lane == 0) umma_commit(&tmem_full_bar[acc]);
-            __syncwarp();
+            if (ok) umma_commit(&tmem_full_bar[acc]);
         }
+        }
+        __syncwarp();
     } else {
         // ------------------------------------------------------------ epilogue
         const int quarter = warp & 3;           // TMEM lanes 32*quarter .. +31

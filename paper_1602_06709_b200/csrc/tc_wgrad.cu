@@ -185,16 +185,17 @@ tc_wgrad_kernel(const __grid_constant__ CUtensorMap tmDy, const __grid_constant_
             }
         }
     } else if (warp == 1) {
+        if (lane == 0) {     // one thread runs the whole issue loop, waits included
         const uint32_t idesc = make_idesc_tf32(n_groups * 32, true, true);
         const uint64_t desc0 = make_smem_desc(0, kGroupBytes, 512, kSwizzle128B_Atom32B);
         int stage = 0;
         uint32_t phase = 0;
         bool ok = true;
         for (int kit = 0; kit < kiters; kit += p.KS) {
-            if (!bounded_wait_warp(&full_bar[stage], phase, &abort_flag, p.status, WAIT_MMA_FULL)) { ok = false; break; }
+            if (!bounded_wait(&full_bar[stage], phase, &abort_flag, p.status, WAIT_MMA_FULL)) { ok = false; break; }
             tc_fence_after();
             const int nst = kiters - kit < p.KS ? kiters - kit : p.KS;
-            if (lane == 0) {
+            {
               for (int j = 0; j < nst; ++j) {
                 // 8 pixels per instruction = two 512-byte groups of 4 rows; descriptors differ only in the
                 // address field, so add offsets to a constant part
@@ -206,10 +207,10 @@ tc_wgrad_kernel(const __grid_constant__ CUtensorMap tmDy, const __grid_constant_
               }
                 umma_commit(&empty_bar[stage]);
             }
-            __syncwarp();
             if (++stage == p.stages) { stage = 0; phase ^= 1u; }
         }
-        if (ok && lane == 0) umma_commit(&tmem_full_bar);
+        if (ok) umma_commit(&tmem_full_bar);
+        }
         __syncwarp();
     } else {
         const int quarter = warp & 3;
