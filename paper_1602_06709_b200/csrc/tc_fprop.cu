@@ -458,19 +458,27 @@ void choose_box(int P, int Q, int N, int* bw_log2, int* bh_log2) {
 }
 
 int choose_bn(int Kout, long m_tiles, int sm_count) {
-    // Widest tile that still gives every SM a tile; otherwise the narrowest
-    // width that keeps the tile count from growing further.
+    // Score = (fraction of SM-slots the tiles fill, counting whole waves) x (tensor efficiency of the width):
+    // an MMA costs max(N/2, ~52) cycles, so N < 128 wastes the pipe, and wider tiles re-read A less often.
     const int k32 = (Kout + 31) / 32 * 32;
-    int bn = k32 < 256 ? k32 : 256;
-    {   // balance the last tile: Kout = 1000 -> 4 x 256 rather than 3 x 256 + 232
-        const int tiles = (Kout + bn - 1) / bn;
-        bn = ((Kout + tiles - 1) / tiles + 31) / 32 * 32;
+    int best = 32;
+    double best_score = -1.0;
+    for (int bn = 256; bn >= 32; bn -= 32) {
+        if (bn > k32 && bn != 32) continue;
+        const long n_tiles = (Kout + bn - 1) / bn;
+        if ((n_tiles - 1) * bn >= Kout) continue;
+        // balance the last tile: Kout = 1000 -> 4 x 256 rather than 3 x 256 + 232
+        const int bal = int(((Kout + n_tiles - 1) / n_tiles + 31) / 32 * 32);
+        if (bal != bn && bal < bn) continue;       // the balanced width is tried on its own
+        const long tiles = m_tiles * n_tiles;
+        const long waves = (tiles + sm_count - 1) / sm_count;
+        const double fill = double(tiles) / double(waves * sm_count);
+        const double useful = double(Kout) / double(n_tiles * bn);           // ragged last columns
+        const double eff = (bn >= 128 ? 0.88 + 0.12 * (bn - 128) / 128.0 : 0.88 * bn / 128.0);
+        const double score = fill * useful * eff;
+        if (score > best_score + 1e-9) { best_score = score; best = bn; }
     }
-    while (bn > 64 && m_tiles * ((Kout + bn - 1) / bn) < sm_count) {
-        const int half = (bn / 2 + 31) / 32 * 32;
-        bn = half;
-    }
-    return bn;
+    return best;
 }
 
 int g_sm_count = 0;
