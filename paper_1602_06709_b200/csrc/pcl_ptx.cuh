@@ -157,6 +157,203 @@ __device__ __forceinline__ void tmem_ld_32x32(uint32_t taddr, uint32_t (&v)[32])
 }
 __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 
+// ------------------------------------------------------- CTA pairs (cta_group::2)
+// Two CTAs of a cluster (ranks 2i, 2i+1) run one M = 256 MMA: each holds its own 128 rows of A and half
+// of the B rows at the same shared-memory offsets, the even CTA (the leader) issues.  Loads of either
+// CTA may complete on the leader's barrier; a commit can arrive on the same barrier of both CTAs.
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+__device__ __forceinline__ uint32_t cluster_id_x() {
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%clusterid.x;" : "=r"(r));
+    return r;
+}
+__device__ __forceinline__ uint32_t nclusters_x() {
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%nclusterid.x;" : "=r"(r));
+    return r;
+}
+// shared::cluster address of `p` (a shared-memory object of this CTA) in the CTA of rank `rank`
+__device__ __forceinline__ uint32_t map_to_cta(const void* p, uint32_t rank) {
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(smem_u32(p)), "r"(rank));
+    return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+    asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t bar_cluster_addr) {
+    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(bar_cluster_addr) : "memory");
+}
+__device__ __forceinline__ void tma_load_3d_pair(void* dst, const CUtensorMap* m, uint32_t bar_cluster_addr, int c0,
+                                                 int c1, int c2) {
+    asm volatile(
+        "cp.async.bulk.tensor.3d.cta_group::2.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
+        ::"r"(smem_u32(dst)), "l"(reinterpret_cast<uint64_t>(m)), "r"(bar_cluster_addr), "r"(c0), "r"(c1), "r"(c2)
+        : "memory");
+}
+__device__ __forceinline__ void tma_load_4d_pair(void* dst, const CUtensorMap* m, uint32_t bar_cluster_addr, int c0,
+                                                 int c1, int c2, int c3) {
+    asm volatile(
+        "cp.async.bulk.tensor.4d.cta_group::2.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
+        ::"r"(smem_u32(dst)), "l"(reinterpret_cast<uint64_t>(m)), "r"(bar_cluster_addr), "r"(c0), "r"(c1), "r"(c2),
+        "r"(c3)
+        : "memory");
+}
+__device__ __forceinline__ void tma_load_5d_pair(void* dst, const CUtensorMap* m, uint32_t bar_cluster_addr, int c0,
+                                                 int c1, int c2, int c3, int c4) {
+    asm volatile(
+        "cp.async.bulk.tensor.5d.cta_group::2.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6, %7}], [%2];"
+        ::"r"(smem_u32(dst)), "l"(reinterpret_cast<uint64_t>(m)), "r"(bar_cluster_addr), "r"(c0), "r"(c1), "r"(c2),
+        "r"(c3), "r"(c4)
+        : "memory");
+}
+__device__ __forceinline__ void tmem_alloc_pair(uint32_t* smem_result, uint32_t ncols) {
+    asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(smem_result)),
+                 "r"(ncols)
+                 : "memory");
+}
+__device__ __forceinline__ void tmem_relinquish_pair() {
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc_pair(uint32_t taddr, uint32_t ncols) {
+    asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void umma_tf32_pair(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                               uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::2.kind::tf32 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+// One arrival on `bar` (same offset) in both CTAs of the pair once the issued pair MMAs are done.
+__device__ __forceinline__ void umma_commit_pair(uint64_t* bar) {
+    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+                 ::"r"(smem_u32(bar)), "h"(static_cast<uint16_t>(3))
+                 : "memory");
+}
+
+// ------------------------------------------------- lean forms for the single-thread pipeline loops
+// The producer and the MMA-issuing thread each run alone in their warp, so every instruction they execute costs
+// several cycles of the k-step budget (a 128 x 256 x 32 k-step is 512 tensor cycles; measured: a loop of ~100
+// instructions per k-step held the tensor pipe at 63 %).  These forms take shared-memory addresses as 32-bit
+// registers that the loops advance by addition, and issue the four K = 8 MMAs of a k-step from one asm block.
+__device__ __forceinline__ bool mbar_try_wait_addr(uint32_t bar_addr, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar_addr), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+static __device__ __noinline__ bool bounded_wait_slow(uint32_t bar_addr, uint32_t parity, volatile uint32_t* abort_flag,
+                                               unsigned int* status_word, uint32_t code) {
+    unsigned long long t0 = 0;
+    for (uint32_t spin = 0;; ++spin) {
+        if (mbar_try_wait_addr(bar_addr, parity)) return true;
+        if ((spin & 63u) == 63u) {
+            if (*abort_flag) return false;
+            const unsigned long long now = global_nanos();
+            if (t0 == 0) t0 = now;
+            else if (now - t0 > kWaitNanos) break;
+            __nanosleep(64);
+        }
+    }
+    *abort_flag = 1u;
+    atomicCAS(status_word, 0u, code);
+    return false;
+}
+// One poll inline (the common case); the bounded polling loop is out of line.
+__device__ __forceinline__ bool bounded_wait_addr(uint32_t bar_addr, uint32_t parity, volatile uint32_t* abort_flag,
+                                                  unsigned int* status_word, uint32_t code) {
+    if (mbar_try_wait_addr(bar_addr, parity)) return true;
+    return bounded_wait_slow(bar_addr, parity, abort_flag, status_word, code);
+}
+__device__ __forceinline__ void mbar_expect_tx_addr(uint32_t bar_addr, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar_addr), "r"(bytes) : "memory");
+}
+template <bool kPair>
+__device__ __forceinline__ void umma_commit_addr(uint32_t bar_addr) {
+    if constexpr (kPair)
+        asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+                     ::"r"(bar_addr), "h"(static_cast<uint16_t>(3))
+                     : "memory");
+    else
+        asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar_addr)
+                     : "memory");
+}
+// TMA loads with 32-bit shared addresses; kPair: the barrier is a shared::cluster address (the leader's).
+template <bool kPair>
+__device__ __forceinline__ void tma_load_3d_addr(uint32_t dst, const CUtensorMap* m, uint32_t bar, int c0, int c1, int c2) {
+    if constexpr (kPair)
+        asm volatile(
+            "cp.async.bulk.tensor.3d.cta_group::2.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
+            ::"r"(dst), "l"(reinterpret_cast<uint64_t>(m)), "r"(bar), "r"(c0), "r"(c1), "r"(c2) : "memory");
+    else
+        asm volatile(
+            "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
+            ::"r"(dst), "l"(reinterpret_cast<uint64_t>(m)), "r"(bar), "r"(c0), "r"(c1), "r"(c2) : "memory");
+}
+template <bool kPair>
+__device__ __forceinline__ void tma_load_4d_addr(uint32_t dst, const CUtensorMap* m, uint32_t bar, int c0, int c1, int c2,
+                                                 int c3) {
+    if constexpr (kPair)
+        asm volatile(
+            "cp.async.bulk.tensor.4d.cta_group::2.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
+            ::"r"(dst), "l"(reinterpret_cast<uint64_t>(m)), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3) : "memory");
+    else
+        asm volatile(
+            "cp.async.bulk.tensor.4d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
+            ::"r"(dst), "l"(reinterpret_cast<uint64_t>(m)), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3) : "memory");
+}
+template <bool kPair>
+__device__ __forceinline__ void tma_load_5d_addr(uint32_t dst, const CUtensorMap* m, uint32_t bar, int c0, int c1, int c2,
+                                                 int c3, int c4) {
+    if constexpr (kPair)
+        asm volatile(
+            "cp.async.bulk.tensor.5d.cta_group::2.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6, %7}], [%2];"
+            ::"r"(dst), "l"(reinterpret_cast<uint64_t>(m)), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(c4) : "memory");
+    else
+        asm volatile(
+            "cp.async.bulk.tensor.5d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6, %7}], [%2];"
+            ::"r"(dst), "l"(reinterpret_cast<uint64_t>(m)), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(c4) : "memory");
+}
+// The four K = 8 MMAs of one k-step (32 reduction elements).  Descriptors are given as their low words (the
+// address field lives there) plus the constant high words; k-block kk is kAStep / kBStep sixteen-byte units
+// further (2 for a K-major 128-byte row, 64 for an MN-major tile whose 8-deep reduction groups are 1 KB apart).
+// `acc_first` = 0 makes the first MMA overwrite the accumulator.
+#define PCL_UMMA_KSTEP_BODY(CG)                                                                                   \
+    asm volatile(                                                                                                 \
+        "{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\t.reg .b32 al, bl;\n\t"                                        \
+        "setp.ne.b32 p, %6, 0;\n\t"                                                                               \
+        "mov.b64 da, {%1, %3};\n\tmov.b64 db, {%2, %4};\n\t"                                                      \
+        "tcgen05.mma.cta_group::" CG ".kind::tf32 [%0], da, db, %5, p;\n\t"                                        \
+        "setp.ne.b32 p, 1, 0;\n\t"                                                                                \
+        "add.u32 al, %1, %7;\n\tadd.u32 bl, %2, %8;\n\tmov.b64 da, {al, %3};\n\tmov.b64 db, {bl, %4};\n\t"          \
+        "tcgen05.mma.cta_group::" CG ".kind::tf32 [%0], da, db, %5, p;\n\t"                                        \
+        "add.u32 al, al, %7;\n\tadd.u32 bl, bl, %8;\n\tmov.b64 da, {al, %3};\n\tmov.b64 db, {bl, %4};\n\t"          \
+        "tcgen05.mma.cta_group::" CG ".kind::tf32 [%0], da, db, %5, p;\n\t"                                        \
+        "add.u32 al, al, %7;\n\tadd.u32 bl, bl, %8;\n\tmov.b64 da, {al, %3};\n\tmov.b64 db, {bl, %4};\n\t"          \
+        "tcgen05.mma.cta_group::" CG ".kind::tf32 [%0], da, db, %5, p;\n\t}"                                       \
+        ::"r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(a_hi), "r"(b_hi), "r"(idesc), "r"(acc_first), "n"(kAStep),       \
+        "n"(kBStep)                                                                                               \
+        : "memory")
+template <bool kPair, int kAStep, int kBStep>
+__device__ __forceinline__ void umma_kstep_tf32(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t a_hi,
+                                                uint32_t b_hi, uint32_t idesc, uint32_t acc_first) {
+    if constexpr (kPair) PCL_UMMA_KSTEP_BODY("2");
+    else PCL_UMMA_KSTEP_BODY("1");
+}
+#undef PCL_UMMA_KSTEP_BODY
+
 // Shared-memory matrix descriptor (64-bit) for a swizzled operand tile.
 //   bits  0-13 start address >> 4      bits 16-29 leading byte offset >> 4
 //   bits 32-45 stride byte offset >> 4 bits 46-47 descriptor version (1 on sm_100)
@@ -180,13 +377,14 @@ __device__ __forceinline__ uint64_t make_smem_desc(uint32_t smem_addr, uint32_t 
     return d;
 }
 
-// Instruction descriptor for kind::tf32, fp32 accumulator, M = 128.
+// Instruction descriptor for kind::tf32, fp32 accumulator, M = 128 (256 for a CTA pair).
 //   bits 4-5 D format (1 = f32)   bits 7-9 A format (2 = tf32)   bits 10-12 B format
 //   bit 15 A is MN-major          bit 16 B is MN-major
 //   bits 17-22 N >> 3             bits 24-28 M >> 4
-__host__ __device__ constexpr uint32_t make_idesc_tf32(uint32_t n, bool a_mn_major, bool b_mn_major) {
+__host__ __device__ constexpr uint32_t make_idesc_tf32(uint32_t n, bool a_mn_major, bool b_mn_major,
+                                                       uint32_t m = 128u) {
     return (1u << 4) | (2u << 7) | (2u << 10) | (static_cast<uint32_t>(a_mn_major) << 15) |
-           (static_cast<uint32_t>(b_mn_major) << 16) | ((n >> 3) << 17) | ((128u >> 4) << 24);
+           (static_cast<uint32_t>(b_mn_major) << 16) | ((n >> 3) << 17) | ((m >> 4) << 24);
 }
 
 // Wait codes recorded in the device status word (which role gave up).

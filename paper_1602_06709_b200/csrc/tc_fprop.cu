@@ -47,6 +47,8 @@ struct FpropParams {
     int act;
     int stages;
     int KS;                     // k-steps (plain: {A,B} pairs; halo: weight tiles of consecutive taps) per pipeline slot
+    int grp;                    // plain tiling: a slot's KS k-steps are KS consecutive channel blocks of one tap, fetched by
+                                // ONE copy of A and one of B (slot layout: KS A tiles, then KS B tiles)
     int tmem_cols;
     int tw, th, tn;             // pixels a tile spans in q, p, n (= the box, or 2 x the box in one direction when MT = 2)
     // Halo mode (R*S > 1): the A operand of ALL taps of a channel block comes from one haloed input patch
@@ -90,6 +92,10 @@ struct TileIter {
     }
 };
 
+// kPair: two CTAs of a cluster (ranks 0 and 1) compute two M tiles (consecutive image groups) against the
+// same BN = 256 weight tile with M = 256 MMAs issued by rank 0; each CTA loads its own A tile and only half
+// of the weight rows, which cuts the shared-memory fill traffic per MMA by a third (plain tiling only).
+template <bool kPair>
 __global__ void __launch_bounds__(kThreads, 1)
 tc_fprop_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, FpropParams p) {
     extern __shared__ uint8_t smem_raw[];
@@ -108,7 +114,18 @@ tc_fprop_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
     // plain mode: ring of {A 16 KB, B BN*128 B} slots.  halo mode: NA patch buffers, then a ring of B slots.
     // A slot holds KS k-steps: the issuing thread pays one barrier round trip and one commit per slot, which
     // is what bounds narrow tiles (their MMAs are short), so narrow tiles batch several k-steps per slot.
-    const uint32_t b_bytes = p.BN * 128;
+    const uint32_t b_bytes = kPair ? p.BN * 64 : p.BN * 128;
+    const uint32_t pair_rank = kPair ? cluster_ctarank() : 0u;
+    const int first_tile = kPair ? int(cluster_id_x()) : int(blockIdx.x);
+    const int tile_stride = kPair ? int(nclusters_x()) : int(gridDim.x);
+    auto issue_mma = [](uint32_t d, uint64_t da, uint64_t db, uint32_t idesc, uint32_t accumulate) {
+        if constexpr (kPair) umma_tf32_pair(d, da, db, idesc, accumulate);
+        else umma_tf32(d, da, db, idesc, accumulate);
+    };
+    auto commit = [](uint64_t* bar) {
+        if constexpr (kPair) umma_commit_pair(bar);
+        else umma_commit(bar);
+    };
     const uint32_t step_bytes = p.halo ? b_bytes : kABytes + b_bytes;
     const uint32_t stage_bytes = p.KS * step_bytes;
     uint8_t* b_ring = smem + (p.halo ? p.NA * p.a_buf_bytes : kABytes);
@@ -125,7 +142,7 @@ tc_fprop_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
         }
         for (int a = 0; a < 2; ++a) {
             mbar_init(&tmem_full_bar[a], 1);
-            mbar_init(&tmem_empty_bar[a], kEpiWarps);
+            mbar_init(&tmem_empty_bar[a], kPair ? 2 * kEpiWarps : kEpiWarps);
         }
         abort_flag = 0;
         mbar_fence_init();
@@ -133,11 +150,12 @@ tc_fprop_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
         prefetch_tmap(&tmB);
     }
     if (warp == 1) {
-        tmem_alloc(&tmem_base_slot, p.tmem_cols);
-        tmem_relinquish();
+        if constexpr (kPair) { tmem_alloc_pair(&tmem_base_slot, p.tmem_cols); tmem_relinquish_pair(); }
+        else { tmem_alloc(&tmem_base_slot, p.tmem_cols); tmem_relinquish(); }
     }
     tc_fence_before();
     __syncthreads();
+    if constexpr (kPair) cluster_sync_all();     // the peer's barriers exist before anything signals them
     tc_fence_after();
     const uint32_t tmem_base = tmem_base_slot;
 
@@ -148,60 +166,91 @@ tc_fprop_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
 
     if (warp == 0) {
         // ------------------------------------------------------------ producer
+        // One thread; its loop is kept to a few instructions per copy (addresses and coordinates advance by
+        // addition), because at one thread per warp every instruction costs cycles of the k-step budget.
         if (lane == 0) {
             int stage = 0, issued = 0;
             uint32_t phase = 0;
             int a_slot = 0, issuedA = 0;
             uint32_t phaseA = 0;
             bool ok = true;
+            const uint32_t full0 = smem_u32(&full_bar[0]), empty0 = smem_u32(&empty_bar[0]);
+            const uint32_t ring0 = smem_u32(p.halo ? b_ring : smem);
+            uint32_t full_a = full0, empty_a = empty0, slot_a = ring0;
+            const uint32_t full_dst0 = kPair ? map_to_cta(&full_bar[0], 0) : full0;   // where the copies complete
+            uint32_t full_dst = full_dst0;
+            const int c_end = p.cblocks * kBlockC;
+            const int taps = p.R * p.S;
             TileIter it;
-            for (it.init(p, blockIdx.x, gridDim.x); it.t < total_tiles && ok; it.next(p)) {
-                const int kt = it.kt;
-                const int q0 = it.qi * p.tw, p0 = it.pi * p.th, n0 = it.ni * p.tn;
+            for (it.init(p, first_tile, tile_stride); it.t < total_tiles && ok; it.next(p)) {
+                const int q0 = it.qi * p.tw, p0 = it.pi * p.th;
+                const int n0 = (kPair ? 2 * it.ni + int(pair_rank) : it.ni) * p.tn;
+                const int kcol = it.kt * p.BN + (kPair ? int(pair_rank) * (p.BN >> 1) : 0);
                 if (p.halo) {
-                    for (int cb = 0; cb < p.cblocks && ok; ++cb) {
+                    for (int c0 = 0; c0 < c_end && ok; c0 += kBlockC) {
                         if (!bounded_wait(&emptyA_bar[a_slot], phaseA ^ 1u, &abort_flag, p.status, WAIT_PRODUCER_EMPTY)) {
                             ok = false;
                             break;
                         }
                         mbar_expect_tx(&fullA_bar[a_slot], p.patch_bytes);
-                        tma_load_4d(smem + a_slot * p.a_buf_bytes, &tmA, &fullA_bar[a_slot], cb * kBlockC,
-                                    q0 - p.pad_w, p0 - p.pad_h, n0);
+                        tma_load_4d(smem + a_slot * p.a_buf_bytes, &tmA, &fullA_bar[a_slot], c0, q0 - p.pad_w,
+                                    p0 - p.pad_h, n0);
                         ++issuedA;
                         if (++a_slot == p.NA) { a_slot = 0; phaseA ^= 1u; }
-                        for (int tap = 0; tap < p.R * p.S; tap += p.KS) {
-                            if (!bounded_wait(&empty_bar[stage], phase ^ 1u, &abort_flag, p.status, WAIT_PRODUCER_EMPTY)) {
+                        for (int tap = 0; tap < taps; tap += p.KS) {
+                            if (!bounded_wait_addr(empty_a, phase ^ 1u, &abort_flag, p.status, WAIT_PRODUCER_EMPTY)) {
                                 ok = false;
                                 break;
                             }
-                            const int nst = p.R * p.S - tap < p.KS ? p.R * p.S - tap : p.KS;
-                            mbar_expect_tx(&full_bar[stage], nst * b_bytes);
-                            for (int j = 0; j < nst; ++j)
-                                tma_load_3d(b_ring + stage * stage_bytes + j * b_bytes, &tmB, &full_bar[stage],
-                                            cb * kBlockC, tap + j, kt * p.BN);
+                            const int nst = taps - tap < p.KS ? taps - tap : p.KS;
+                            mbar_expect_tx_addr(full_a, nst * b_bytes);
+                            uint32_t dst = slot_a;
+                            for (int j = 0; j < nst; ++j, dst += b_bytes)
+                                tma_load_3d_addr<false>(dst, &tmB, full_a, c0, tap + j, kcol);
                             ++issued;
-                            if (++stage == p.stages) { stage = 0; phase ^= 1u; }
+                            full_a += 8; empty_a += 8; slot_a += stage_bytes;
+                            if (++stage == p.stages) { stage = 0; phase ^= 1u; full_a = full0; empty_a = empty0; slot_a = ring0; }
                         }
                     }
                 } else {
-                    int r = 0, s = 0, cb = 0;        // k-step order: r, then s, then channel block
+                    // k-step order: r, then s, then channel block
+                    int c0 = 0, s = 0, tap = 0;
+                    int cq = q0 - p.pad_w, cp = p0 - p.pad_h;
                     for (int kit = 0; kit < kiters; kit += p.KS) {
-                        if (!bounded_wait(&empty_bar[stage], phase ^ 1u, &abort_flag, p.status, WAIT_PRODUCER_EMPTY)) {
+                        if (!bounded_wait_addr(empty_a, phase ^ 1u, &abort_flag, p.status, WAIT_PRODUCER_EMPTY)) {
                             ok = false;
                             break;
                         }
                         const int nst = kiters - kit < p.KS ? kiters - kit : p.KS;
-                        mbar_expect_tx(&full_bar[stage], nst * step_bytes);
-                        for (int j = 0; j < nst; ++j) {
-                            uint8_t* a_dst = smem + stage * stage_bytes + j * step_bytes;
-                            tma_load_4d(a_dst, &tmA, &full_bar[stage], cb * kBlockC, q0 + s - p.pad_w,
-                                        p0 + r - p.pad_h, n0);
-                            tma_load_3d(a_dst + kABytes, &tmB, &full_bar[stage], cb * kBlockC, r * p.S + s,
-                                        kt * p.BN);
-                            if (++cb == p.cblocks) { cb = 0; if (++s == p.S) { s = 0; ++r; } }
+                        // pair: both CTAs' copies complete on the leader's barrier, which its producer arms
+                        if (!kPair) mbar_expect_tx_addr(full_a, nst * step_bytes);
+                        else if (pair_rank == 0) mbar_expect_tx_addr(full_a, 2 * nst * step_bytes);
+                        uint32_t dst = slot_a;
+                        if (p.grp) {
+                            // (cblocks is a multiple of KS here, so nst = KS and a slot never straddles two taps)
+                            tma_load_5d_addr<kPair>(dst, &tmA, full_dst, 0, cq, cp, n0, c0 >> 5);
+                            tma_load_4d_addr<kPair>(dst + p.KS * kABytes, &tmB, full_dst, 0, kcol, c0 >> 5, tap);
+                            c0 += p.KS * kBlockC;
+                            if (c0 == c_end) {
+                                c0 = 0; ++tap; ++cq;
+                                if (++s == p.S) { s = 0; cq -= p.S; ++cp; }
+                            }
+                        } else
+                        for (int j = 0; j < nst; ++j, dst += step_bytes) {
+                            tma_load_4d_addr<kPair>(dst, &tmA, full_dst, c0, cq, cp, n0);
+                            tma_load_3d_addr<kPair>(dst + kABytes, &tmB, full_dst, c0, tap, kcol);
+                            c0 += kBlockC;
+                            if (c0 == c_end) {
+                                c0 = 0; ++tap; ++cq;
+                                if (++s == p.S) { s = 0; cq -= p.S; ++cp; }
+                            }
                         }
                         ++issued;
-                        if (++stage == p.stages) { stage = 0; phase ^= 1u; }
+                        full_a += 8; empty_a += 8; full_dst += 8; slot_a += stage_bytes;
+                        if (++stage == p.stages) {
+                            stage = 0; phase ^= 1u;
+                            full_a = full0; empty_a = empty0; full_dst = full_dst0; slot_a = ring0;
+                        }
                     }
                 }
             }
@@ -226,76 +275,103 @@ tc_fprop_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
         // ---------------------------------------------------------- MMA issuer
         // One thread runs the whole loop (waits included): a warp-wide wait + re-convergence per slot would
         // add to the per-slot cost that bounds narrow tiles.
-        if (lane == 0) {
-        const uint32_t idesc = make_idesc_tf32(p.BN, false, false);
+        if (lane == 0 && pair_rank == 0) {
+        const uint32_t idesc = make_idesc_tf32(p.BN, false, false, kPair ? 256u : 128u);
         int stage = 0;
         uint32_t phase = 0;
         int a_slot = 0;
         uint32_t phaseA = 0;
         int tile_cnt = 0;
         bool ok = true;
-        for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x, ++tile_cnt) {
+        // Descriptors differ only in the 14-bit address field (address >> 4) of their low word: the loop keeps
+        // low words in registers and advances them by addition.
+        const uint64_t b_desc0 = make_smem_desc(smem_u32(p.halo ? b_ring : smem), 16, 1024, kSwizzle128B);
+        const uint32_t b_hi = uint32_t(b_desc0 >> 32), ring_lo0 = uint32_t(b_desc0);
+        const uint32_t full0 = smem_u32(&full_bar[0]), empty0 = smem_u32(&empty_bar[0]);
+        uint32_t full_a = full0, empty_a = empty0, slot_lo = ring_lo0;
+        const uint32_t stage16 = stage_bytes >> 4, step16 = step_bytes >> 4;
+        // where k-step j of a slot finds its operands (16-byte units from the slot start)
+        const uint32_t a_step16 = p.grp ? (kABytes >> 4) : step16;
+        const uint32_t b_off16 = p.grp ? p.KS * (kABytes >> 4) : (kABytes >> 4);
+        const uint32_t b_step16 = p.grp ? (b_bytes >> 4) : step16;
+        for (int t = first_tile; t < total_tiles && ok; t += tile_stride, ++tile_cnt) {
             const int acc = tile_cnt & 1;
             const uint32_t acc_phase = (tile_cnt >> 1) & 1;
             if (!bounded_wait(&tmem_empty_bar[acc], acc_phase ^ 1u, &abort_flag, p.status, WAIT_MMA_TMEM_EMPTY)) break;
             tc_fence_after();
             const uint32_t d_tmem = tmem_base + acc * p.MT * p.BN;
+            uint32_t accum = 0;         // the tile's first MMA overwrites the accumulator
             if (p.halo) {
-                // Descriptors differ only in their 14-bit address field (address >> 4): build the constant part
-                // once and add offsets, so that the issuing thread spends a few instructions per MMA.
                 const uint64_t a_desc0 = make_smem_desc(0, 16, p.PW * 128, kSwizzle128B);   // 8-pixel groups are one patch row apart
-                const uint64_t b_desc0 = make_smem_desc(0, 16, 1024, kSwizzle128B);
+                const uint32_t a_hi = uint32_t(a_desc0 >> 32);
                 const uint32_t half_off16 = p.half_off_bytes >> 4;
+                const uint32_t row16 = (p.PW - p.S) * 8;        // from the end of a tap row to the start of the next
+                const int taps = p.R * p.S;
                 for (int cb = 0; cb < p.cblocks && ok; ++cb) {
                     if (!bounded_wait(&fullA_bar[a_slot], phaseA, &abort_flag, p.status, WAIT_MMA_FULL)) { ok = false; break; }
-                    const uint32_t a_base = smem_u32(smem + a_slot * p.a_buf_bytes);
-                    int r = 0, s = 0;
-                    for (int tap = 0; tap < p.R * p.S && ok; tap += p.KS) {
-                        if (!bounded_wait(&full_bar[stage], phase, &abort_flag, p.status, WAIT_MMA_FULL)) { ok = false; break; }
+                    // the tap (r, s) = a shift by (r * PW + s) pixels of 128 bytes inside the patch
+                    uint32_t a_lo = uint32_t(a_desc0) + ((smem_u32(smem + a_slot * p.a_buf_bytes) & 0x3FFFFu) >> 4);
+                    int s = 0;
+                    for (int tap = 0; tap < taps; tap += p.KS) {
+                        if (!bounded_wait_addr(full_a, phase, &abort_flag, p.status, WAIT_MMA_FULL)) { ok = false; break; }
                         tc_fence_after();
-                        const int nst = p.R * p.S - tap < p.KS ? p.R * p.S - tap : p.KS;
-                        {
-                            uint64_t db = b_desc0 + ((smem_u32(b_ring + stage * stage_bytes) & 0x3FFFFu) >> 4);
-                            for (int j = 0; j < nst; ++j) {
-                                // the tap = a row shift inside the patch
-                                const uint64_t da = a_desc0 + (((a_base + (r * p.PW + s) * 128) & 0x3FFFFu) >> 4);
-                                for (int h = 0; h < p.MT; ++h) {
-#pragma unroll
-                                    for (int kk = 0; kk < 4; ++kk)
-                                        umma_tf32(d_tmem + h * p.BN, da + h * half_off16 + kk * 2, db + kk * 2, idesc,
-                                                  (cb | tap | j | kk) != 0);
-                                }
-                                db += b_bytes >> 4;
-                                if (++s == p.S) { s = 0; ++r; }
-                            }
-                            umma_commit(&empty_bar[stage]);
+                        const int nst = taps - tap < p.KS ? taps - tap : p.KS;
+                        uint32_t b_lo = slot_lo;
+                        for (int j = 0; j < nst; ++j) {
+                            umma_kstep_tf32<kPair, 2, 2>(d_tmem, a_lo, b_lo, a_hi, b_hi, idesc, accum);
+                            accum = 1;
+                            if (p.MT == 2) umma_kstep_tf32<kPair, 2, 2>(d_tmem + p.BN, a_lo + half_off16, b_lo, a_hi, b_hi, idesc, tap | j | cb);
+                            b_lo += b_bytes >> 4;
+                            a_lo += 8;
+                            if (++s == p.S) { s = 0; a_lo += row16; }
                         }
-                        if (++stage == p.stages) { stage = 0; phase ^= 1u; }
+                        umma_commit_addr<kPair>(empty_a);
+                        full_a += 8; empty_a += 8; slot_lo += stage16;
+                        if (++stage == p.stages) { stage = 0; phase ^= 1u; full_a = full0; empty_a = empty0; slot_lo = ring_lo0; }
                     }
-                    if (ok) umma_commit(&emptyA_bar[a_slot]);
+                    if (ok) commit(&emptyA_bar[a_slot]);
                     if (++a_slot == p.NA) { a_slot = 0; phaseA ^= 1u; }
                 }
+            } else if (p.KS == 1) {
+                // the hot loop of the wide layers: one k-step per slot, nothing but the wait, four MMAs, the commit
+                // and the ring advance
+                for (int kit = 0; kit < kiters; ++kit) {
+                    if (!bounded_wait_addr(full_a, phase, &abort_flag, p.status, WAIT_MMA_FULL)) { ok = false; break; }
+                    tc_fence_after();
+                    umma_kstep_tf32<kPair, 2, 2>(d_tmem, slot_lo, slot_lo + (kABytes >> 4), b_hi, b_hi, idesc, accum);
+                    accum = 1;
+                    umma_commit_addr<kPair>(empty_a);
+                    full_a += 8; empty_a += 8; slot_lo += stage16;
+                    if (++stage == p.stages) { stage = 0; phase ^= 1u; full_a = full0; empty_a = empty0; slot_lo = ring_lo0; }
+                }
+            } else if (p.KS == 2 && p.grp) {
+                // two k-steps per slot, fetched by one copy per operand
+                for (int kit = 0; kit < kiters; kit += 2) {
+                    if (!bounded_wait_addr(full_a, phase, &abort_flag, p.status, WAIT_MMA_FULL)) { ok = false; break; }
+                    tc_fence_after();
+                    umma_kstep_tf32<kPair, 2, 2>(d_tmem, slot_lo, slot_lo + b_off16, b_hi, b_hi, idesc, accum);
+                    umma_kstep_tf32<kPair, 2, 2>(d_tmem, slot_lo + a_step16, slot_lo + b_off16 + b_step16, b_hi, b_hi, idesc, 1);
+                    accum = 1;
+                    umma_commit_addr<kPair>(empty_a);
+                    full_a += 8; empty_a += 8; slot_lo += stage16;
+                    if (++stage == p.stages) { stage = 0; phase ^= 1u; full_a = full0; empty_a = empty0; slot_lo = ring_lo0; }
+                }
             } else {
-                const uint64_t desc0 = make_smem_desc(0, 16, 1024, kSwizzle128B);
                 for (int kit = 0; kit < kiters; kit += p.KS) {
-                    if (!bounded_wait(&full_bar[stage], phase, &abort_flag, p.status, WAIT_MMA_FULL)) { ok = false; break; }
+                    if (!bounded_wait_addr(full_a, phase, &abort_flag, p.status, WAIT_MMA_FULL)) { ok = false; break; }
                     tc_fence_after();
                     const int nst = kiters - kit < p.KS ? kiters - kit : p.KS;
-                    {
-                        uint64_t da = desc0 + ((smem_u32(smem + stage * stage_bytes) & 0x3FFFFu) >> 4);
-                        for (int j = 0; j < nst; ++j) {
-                            const uint64_t db = da + (kABytes >> 4);
-#pragma unroll
-                            for (int kk = 0; kk < 4; ++kk)
-                                umma_tf32(d_tmem, da + kk * 2, db + kk * 2, idesc, (kit | j | kk) != 0);
-                            da += step_bytes >> 4;
-                        }
-                        umma_commit(&empty_bar[stage]);
+                    uint32_t a_lo = slot_lo, b_lo = slot_lo + b_off16;
+                    for (int j = 0; j < nst; ++j, a_lo += a_step16, b_lo += b_step16) {
+                        umma_kstep_tf32<kPair, 2, 2>(d_tmem, a_lo, b_lo, b_hi, b_hi, idesc, accum);
+                        accum = 1;
                     }
-                    if (++stage == p.stages) { stage = 0; phase ^= 1u; }
+                    umma_commit_addr<kPair>(empty_a);
+                    full_a += 8; empty_a += 8; slot_lo += stage16;
+                    if (++stage == p.stages) { stage = 0; phase ^= 1u; full_a = full0; empty_a = empty0; slot_lo = ring_lo0; }
                 }
             }
-            if (ok) umma_commit(&tmem_full_bar[acc]);
+            if (ok) commit(&tmem_full_bar[acc]);
         }
         }
         __syncwarp();
@@ -310,8 +386,9 @@ tc_fprop_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
         const bool vec_ok = (p.Kout & 3) == 0;
         int tile_cnt = 0;
         TileIter it;
-        for (it.init(p, blockIdx.x, gridDim.x); it.t < total_tiles; it.next(p), ++tile_cnt) {
+        for (it.init(p, first_tile, tile_stride); it.t < total_tiles; it.next(p), ++tile_cnt) {
             const int acc = tile_cnt & 1;
+            const int ni = kPair ? 2 * it.ni + int(pair_rank) : it.ni;
             const uint32_t acc_phase = (tile_cnt >> 1) & 1;
             const int kt = it.kt;
             if (!bounded_wait_warp(&tmem_full_bar[acc], acc_phase, &abort_flag, p.status, WAIT_EPI_TMEM_FULL)) break;
@@ -319,13 +396,13 @@ tc_fprop_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
             for (int h = 0; h < p.MT; ++h) {
             const int q = it.qi * p.tw + iw + h * p.half_dq;
             const int pp = it.pi * p.th + ih + h * p.half_dp;
-            const int n = it.ni * p.tn + in_;
+            const int n = ni * p.tn + in_;
             const bool valid = (q < p.Q) && (pp < p.P) && (n < p.N);
             const size_t pix = (static_cast<size_t>(n) * p.P + pp) * p.Q + q;
             const uint32_t t_row = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + (acc * p.MT + h) * p.BN;
             float* cs_row = nullptr;
-            if (p.colsum_rows) {
-                const size_t m_index = (static_cast<size_t>(it.ni) * p.tiles_p + it.pi) * p.tiles_q + it.qi;
+            if (p.colsum_rows && ni * p.tn < p.N) {      // (an odd image-group count leaves the pair's last tile empty)
+                const size_t m_index = (static_cast<size_t>(ni) * p.tiles_p + it.pi) * p.tiles_q + it.qi;
                 cs_row = p.colsum_rows + ((m_index * p.MT + h) * 4 + quarter) * p.Kout;
             }
             if (vec_ok) {
@@ -429,15 +506,20 @@ tc_fprop_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
             }   // halves
             tc_fence_before();
             __syncwarp();
-            if (lane == 0) mbar_arrive(&tmem_empty_bar[acc]);
+            if (lane == 0) {
+                if (kPair && pair_rank != 0) mbar_arrive_cluster(map_to_cta(&tmem_empty_bar[acc], 0));
+                else mbar_arrive(&tmem_empty_bar[acc]);
+            }
         }
     }
 
     tc_fence_before();
     __syncthreads();
+    if constexpr (kPair) cluster_sync_all();     // neither CTA leaves while the pair's MMAs or arrivals may touch it
     if (warp == 1) {
         tc_fence_after();
-        tmem_dealloc(tmem_base, p.tmem_cols);
+        if constexpr (kPair) tmem_dealloc_pair(tmem_base, p.tmem_cols);
+        else tmem_dealloc(tmem_base, p.tmem_cols);
     }
 }
 
@@ -506,6 +588,8 @@ struct TileCfg {
     int halo = 0, MT = 1, bw_log2 = 0, bh_log2 = 0, tw = 0, th = 0, tn = 0, half_dq = 0, half_dp = 0;
     int tiles_q = 0, tiles_p = 0, tiles_n = 0, tiles_k = 0, BN = 0;
     int PW = 0, patch_bytes = 0, a_buf_bytes = 0, NA = 0, half_off_bytes = 0, stages = 0, KS = 1;
+    int grp = 0;        // one copy per operand and slot (KS channel blocks of one tap)
+    int pair = 0;       // CTA pairs: two image-group tiles share one 256-wide weight tile (see the kernel)
 };
 
 TileCfg plain_cfg(const TcFpropArgs& a, int cblocks, int sm_count) {
@@ -517,11 +601,14 @@ TileCfg plain_cfg(const TcFpropArgs& a, int cblocks, int sm_count) {
     c.BN = choose_bn(a.Kout, m_tiles, sm_count);
     c.tiles_k = (a.Kout + c.BN - 1) / c.BN;
     // narrow tiles: several k-steps per slot (see the kernel), as long as 4 slots still fit
-    c.KS = env_int("PCL_KS", c.BN <= 128 ? 2 : 1);
+    c.pair = env_int("PCL_PAIR", 1) && c.tiles_n >= 2 && sm_count >= 2;
+    const int step_bytes = kABytes + (c.pair ? c.BN * 64 : c.BN * 128);
+    c.KS = env_int("PCL_KS", 2);
     const int kiters = a.R * a.S * cblocks;
     if (c.KS > kiters) c.KS = kiters;
-    while (c.KS > 1 && (kSmemBudget - kEpiStageBytes) / (c.KS * (kABytes + c.BN * 128)) < 3) --c.KS;
-    c.stages = (kSmemBudget - kEpiStageBytes) / (c.KS * (kABytes + c.BN * 128));
+    while (c.KS > 1 && (kSmemBudget - kEpiStageBytes) / (c.KS * step_bytes) < 3) --c.KS;
+    c.stages = (kSmemBudget - kEpiStageBytes) / (c.KS * step_bytes);
+    c.grp = env_int("PCL_GRP", 1) && c.KS > 1 && a.Cin % kBlockC == 0 && cblocks % c.KS == 0 && a.in_inner == 0;
     if (c.stages > kMaxStages) c.stages = kMaxStages;
     c.ok = c.stages >= 2;
     return c;
@@ -620,8 +707,10 @@ int launch_tc_fprop(const TcFpropArgs& a, cudaStream_t st) {
     static bool attr_set = false;
     if (!attr_set) {
         if (ensure_device_setup() != PCL_OK) return PCL_ERR_CUDA;
-        if (cudaFuncSetAttribute(tc_fprop_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget + 1024) !=
-            cudaSuccess)
+        if (cudaFuncSetAttribute(tc_fprop_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 kSmemBudget + 1024) != cudaSuccess ||
+            cudaFuncSetAttribute(tc_fprop_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 kSmemBudget + 1024) != cudaSuccess)
             return PCL_ERR_CUDA;
         attr_set = true;
     }
@@ -631,9 +720,10 @@ int launch_tc_fprop(const TcFpropArgs& a, cudaStream_t st) {
     if (!cfg.ok) return PCL_ERR_UNSUPPORTED_SHAPE;
     p.halo = cfg.halo; p.MT = cfg.MT; p.bw_log2 = cfg.bw_log2; p.bh_log2 = cfg.bh_log2;
     p.tw = cfg.tw; p.th = cfg.th; p.tn = cfg.tn; p.half_dq = cfg.half_dq; p.half_dp = cfg.half_dp;
-    p.tiles_q = cfg.tiles_q; p.tiles_p = cfg.tiles_p; p.tiles_n = cfg.tiles_n; p.tiles_k = cfg.tiles_k;
+    p.tiles_q = cfg.tiles_q; p.tiles_p = cfg.tiles_p; p.tiles_k = cfg.tiles_k;
+    p.tiles_n = cfg.pair ? (cfg.tiles_n + 1) / 2 : cfg.tiles_n;      // pair mode iterates over pairs of image groups
     p.BN = cfg.BN; p.PW = cfg.PW; p.patch_bytes = cfg.patch_bytes; p.a_buf_bytes = cfg.a_buf_bytes; p.NA = cfg.NA;
-    p.half_off_bytes = cfg.half_off_bytes; p.stages = cfg.stages; p.KS = cfg.KS;
+    p.half_off_bytes = cfg.half_off_bytes; p.stages = cfg.stages; p.KS = cfg.KS; p.grp = cfg.grp;
     const int bw = 1 << p.bw_log2, bh = 1 << p.bh_log2, bn = kTileM / (bw * bh);
     const long m_tiles = long(p.tiles_q) * p.tiles_p * p.tiles_n;
     if (m_tiles * p.tiles_k > 0x7fffffffL) return PCL_ERR_UNSUPPORTED_SHAPE;
@@ -658,23 +748,64 @@ int launch_tc_fprop(const TcFpropArgs& a, cudaStream_t st) {
         const uint64_t strides[3] = {sw * 4, sh * 4, sn * 4};
         const uint32_t box_plain[4] = {kBlockC, uint32_t(bw), uint32_t(bh), uint32_t(bn)};
         const uint32_t box_halo[4] = {kBlockC, uint32_t(p.PW), uint32_t(p.th + a.R - 1), 1};
-        int rc = make_tmap(&tmA, a.in, 4, dims, strides, p.halo ? box_halo : box_plain, false);
+        int rc;
+        if (cfg.grp) {
+            // channel blocks as a fifth dimension (128 bytes apart), so that one box spans KS of them
+            const uint64_t dims5[5] = {kBlockC, uint64_t(a.W), uint64_t(a.H), uint64_t(a.N), uint64_t(p.cblocks)};
+            const uint64_t strides5[4] = {sw * 4, sh * 4, sn * 4, kBlockC * 4};
+            const uint32_t box5[5] = {kBlockC, uint32_t(bw), uint32_t(bh), uint32_t(bn), uint32_t(p.KS)};
+            rc = make_tmap(&tmA, a.in, 5, dims5, strides5, box5, false);
+        } else {
+            rc = make_tmap(&tmA, a.in, 4, dims, strides, p.halo ? box_halo : box_plain, false);
+        }
         if (rc != PCL_OK) return rc;
     }
     {
         const uint64_t dims[3] = {uint64_t(a.Cin), uint64_t(a.R) * a.S, uint64_t(a.Kout)};
         const uint64_t strides[2] = {uint64_t(a.Cin) * 4, uint64_t(a.R) * a.S * a.Cin * 4};
-        const uint32_t box[3] = {kBlockC, 1, uint32_t(p.BN)};
-        int rc = make_tmap(&tmB, a.wt, 3, dims, strides, box, false);
+        const uint32_t box[3] = {kBlockC, 1, uint32_t(cfg.pair ? p.BN / 2 : p.BN)};
+        int rc;
+        if (cfg.grp) {
+            // {channel in block, output map, channel block, tap}: a box of KS channel blocks lands as KS weight tiles
+            const uint64_t dims4[4] = {kBlockC, uint64_t(a.Kout), uint64_t(p.cblocks), uint64_t(a.R) * a.S};
+            const uint64_t strides4[3] = {uint64_t(a.R) * a.S * a.Cin * 4, kBlockC * 4, uint64_t(a.Cin) * 4};
+            const uint32_t box4[4] = {kBlockC, uint32_t(cfg.pair ? p.BN / 2 : p.BN), uint32_t(p.KS), 1};
+            rc = make_tmap(&tmB, a.wt, 4, dims4, strides4, box4, false);
+        } else {
+            rc = make_tmap(&tmB, a.wt, 3, dims, strides, box, false);
+        }
         if (rc != PCL_OK) return rc;
     }
     const long total = m_tiles * p.tiles_k;
-    const int grid = int(total < g_sm_count ? total : g_sm_count);
     const size_t smem = (p.halo ? size_t(p.NA) * p.a_buf_bytes + size_t(p.stages) * p.KS * p.BN * 128
-                                : size_t(p.stages) * p.KS * (kABytes + p.BN * 128)) + kEpiStageBytes + 1024;
-    {
+                                : size_t(p.stages) * p.KS * (kABytes + (cfg.pair ? p.BN * 64 : p.BN * 128))) +
+                        kEpiStageBytes + 1024;
+    if (cfg.pair) {
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeClusterDimension;
+        attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+        cudaLaunchConfig_t lc{};
+        lc.blockDim = dim3(kThreads); lc.dynamicSmemBytes = smem; lc.stream = st;
+        lc.attrs = attr; lc.numAttrs = 1;
+        // how many pairs the device holds at once with this much shared memory (cached per size)
+        static size_t cached_smem = 0;
+        static int cached_clusters = 0;
+        if (cached_smem != smem) {
+            lc.gridDim = dim3(unsigned(g_sm_count / 2 * 2));
+            int n = 0;
+            if (cudaOccupancyMaxActiveClusters(&n, tc_fprop_kernel<true>, &lc) != cudaSuccess || n <= 0) return PCL_ERR_CUDA;
+            cached_clusters = n < g_sm_count / 2 ? n : g_sm_count / 2;
+            cached_smem = smem;
+        }
+        const long pair_tiles = long(p.tiles_q) * p.tiles_p * p.tiles_n * p.tiles_k;
+        long nclus = pair_tiles < cached_clusters ? pair_tiles : cached_clusters;
+        lc.gridDim = dim3(unsigned(2 * nclus));
         LaunchScope scope(KID_TC_FPROP, 2.0 * a.N * a.P * a.Q * double(a.Kout) * a.Cin * a.R * a.S, st);
-        tc_fprop_kernel<<<grid, kThreads, smem, st>>>(tmA, tmB, p);
+        if (cudaLaunchKernelEx(&lc, tc_fprop_kernel<true>, tmA, tmB, p) != cudaSuccess) return PCL_ERR_CUDA;
+    } else {
+        const int grid = int(total < g_sm_count ? total : g_sm_count);
+        LaunchScope scope(KID_TC_FPROP, 2.0 * a.N * a.P * a.Q * double(a.Kout) * a.Cin * a.R * a.S, st);
+        tc_fprop_kernel<false><<<grid, kThreads, smem, st>>>(tmA, tmB, p);
     }
     return cudaGetLastError() == cudaSuccess ? PCL_OK : PCL_ERR_CUDA;
 }

@@ -133,3 +133,38 @@ def test_forward_type_kernel_every_tiling(tag, tiling, path_guard, monkeypatch):
     G.assert_parity(y, oracle.conv_fwd(s, x, w, bias, oracle.ACT_RELU), f"fwd {tiling}")
     dx = G.run_conv_bwd_data(s, dy, w, x)
     G.assert_parity(dx, oracle.conv_bwd_data(s, dy, w, x), f"bwd_data {tiling}")
+
+
+PIPELINE_SHAPES = {
+    # several image groups per tile row, so that CTA pairs form; an odd group count leaves one pair half empty
+    "odd_groups": ConvShape(N=6, C=64, K=96, H=28, W=28, R=3, S=3, pad_h=1, pad_w=1),
+    "even_groups_wide": ConvShape(N=8, C=128, K=256, H=14, W=14, R=3, S=3, pad_h=1, pad_w=1),
+    "fc_like": ConvShape(N=384, C=192, K=320, H=1, W=1, R=1, S=1),
+    "ragged_c": ConvShape(N=5, C=72, K=48, H=20, W=20, R=3, S=3, pad_h=1, pad_w=1),     # C % 32 != 0: no grouped copies
+}
+
+
+@pytest.mark.parametrize("variant", ["pair0", "pair1_ks1", "pair1_ks2_nogroup", "pair1_ks2_group", "pair0_ks2_group"])
+@pytest.mark.parametrize("tag", sorted(PIPELINE_SHAPES))
+def test_forward_type_kernel_pipeline_variants(tag, variant, path_guard, monkeypatch):
+    """The plain tiling runs as single CTAs or CTA pairs (one M = 256 MMA over two tiles), with one or
+    two k-steps per pipeline slot fetched by one copy per k-step or one per slot.  Every combination
+    must agree with the oracle (forward with the fused epilogue, backward-data with mask and fused
+    bias gradient path left to the network tests)."""
+    import gpu_helpers as G
+    from paper_1602_06709_b200 import binding as B
+    env = {"pair0": dict(PCL_PAIR="0", PCL_KS="1"), "pair1_ks1": dict(PCL_PAIR="1", PCL_KS="1"),
+           "pair1_ks2_nogroup": dict(PCL_PAIR="1", PCL_KS="2", PCL_GRP="0"),
+           "pair1_ks2_group": dict(PCL_PAIR="1", PCL_KS="2", PCL_GRP="1"),
+           "pair0_ks2_group": dict(PCL_PAIR="0", PCL_KS="2", PCL_GRP="1")}[variant]
+    for k, v in env.items():
+        monkeypatch.setenv(k, v)
+    monkeypatch.setenv("PCL_TILING", "plain")
+    B.set_path(B.PATH_TENSOR)
+    s = PIPELINE_SHAPES[tag]
+    x, w, dy, bias = G.make_inputs(s, "pipe_" + tag)
+    y = G.run_conv_fwd(s, x, w, bias, B.ACT_RELU)
+    G.assert_parity(y, oracle.conv_fwd(s, x, w, bias, oracle.ACT_RELU), f"fwd {variant}")
+    dx = G.run_conv_bwd_data(s, dy, w, x)
+    G.assert_parity(dx, oracle.conv_bwd_data(s, dy, w, x), f"bwd_data {variant}")
+    assert B.last_device_status() == 0
