@@ -23,6 +23,11 @@
 // accumulates its item in TMEM and either writes a partial tile to the
 // workspace (second pass adds the splits in a fixed order) or adds it to dw with
 // fp32 atomics.
+//
+// A k-step is one pixel box of 32 or 64 pixels (4 or 8 MMAs of 8 pixels).  With an
+// even number of k tiles, two CTAs of a cluster take k tiles 2i and 2i+1 of the
+// same run block and pixel split: each loads its own dy tile and half of the x
+// runs, and the even CTA issues M = 256 MMAs for both (cta_group::2).
 #include <stdlib.h>
 
 #include "pcl_internal.h"
@@ -32,26 +37,24 @@ namespace pcl {
 
 namespace {
 
-constexpr int kPix = 32;              // pixels (reduction indices) per pipeline slot
-constexpr int kGroupBytes = kPix * 128;   // one {32 maps x 32 pixels} box
-constexpr int kABytes = 4 * kGroupBytes;  // 128 output maps
 constexpr int kMaxStages = 8;
 constexpr int kSmemBudget = 224 * 1024;
 
 struct WgradParams {
-    int bw_log2, bh_log2;     // pixel box bw x bh x (32/(bw*bh))
+    int bw_log2, bh_log2;     // pixel box bw x bh x (pix/(bw*bh))
+    int pix;                  // pixels (reduction indices) per k-step: 32 or 64
     int boxes_q, boxes_p, boxes_n;
     int k_tiles;
     int L;                    // 32-map groups per run
     int runs_per_tap;         // ceil(C/32) / L
     int total_runs;           // R*S*runs_per_tap
-    int rpi;                  // runs per work item (rpi*L <= 8)
+    int rpi;                  // runs per work item (rpi*L <= 8); even in pair mode
     int run_blocks;           // ceil(total_runs / rpi)
     int R, S, pad_h, pad_w;
     int K, C;
     int splits, boxes_per_split;
     int stages, tmem_cols;
-    int KS;                   // pixel boxes (k-steps of 32 pixels) per pipeline slot; > 1 for narrow column blocks
+    int KS;                   // k-steps per pipeline slot; > 1 for narrow column blocks
     int use_atomics;
     int grouped;              // x: 5-D tensor map (one TMA instruction per run) or 4-D per-group boxes (L == 1)
     int grouped_dy;           // dy: 5-D tensor map (all four 32-map groups in one instruction)
@@ -61,6 +64,9 @@ struct WgradParams {
     unsigned int* status;     // device status word
 };
 
+// kPair: see the header.  Pair mode needs grouped x and dy maps; every item then has rpi runs (runs past the
+// last tap read zeros through the out-of-bounds fill and are not stored).
+template <bool kPair>
 __global__ void __launch_bounds__(192, 1)
 tc_wgrad_kernel(const __grid_constant__ CUtensorMap tmDy, const __grid_constant__ CUtensorMap tmX, WgradParams p) {
     extern __shared__ uint8_t smem_raw[];
@@ -73,18 +79,23 @@ tc_wgrad_kernel(const __grid_constant__ CUtensorMap tmDy, const __grid_constant_
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    const uint32_t pair_rank = kPair ? cluster_ctarank() : 0u;
 
-    // work item of this CTA
-    int item = blockIdx.x;
+    // work item of this CTA (pair: of this cluster; the two CTAs take k tiles 2i and 2i + 1)
+    int item = kPair ? int(cluster_id_x()) : int(blockIdx.x);
     const int split = item % p.splits;   item /= p.splits;
     const int rb = item % p.run_blocks;
-    const int kt = item / p.run_blocks;
+    const int kt = kPair ? 2 * (item / p.run_blocks) + int(pair_rank) : item / p.run_blocks;
     const int run0 = rb * p.rpi;
-    const int nruns = (run0 + p.rpi <= p.total_runs) ? p.rpi : p.total_runs - run0;
+    const int nruns = kPair ? p.rpi : ((run0 + p.rpi <= p.total_runs) ? p.rpi : p.total_runs - run0);
     const int n_groups = nruns * p.L;                 // 32-column groups of this item's MMA
-    const uint32_t step_bytes = kABytes + p.rpi * p.L * kGroupBytes;    // one k-step (same for every item)
+    const int my_runs = kPair ? nruns >> 1 : nruns;   // runs this CTA loads (pair: its half of the columns)
+    const int my_run0 = run0 + int(pair_rank) * my_runs;
+    const uint32_t group_bytes = p.pix * 128;         // one {32 maps x pix pixels} box
+    const uint32_t a_bytes = 4 * group_bytes;         // 128 output maps
+    const uint32_t step_bytes = a_bytes + (kPair ? (p.rpi >> 1) : p.rpi) * p.L * group_bytes;   // one k-step (same for every item)
     const uint32_t stage_bytes = p.KS * step_bytes;                     // a slot holds KS k-steps
-    const uint32_t tx_bytes = kABytes + n_groups * kGroupBytes;
+    const uint32_t tx_bytes = a_bytes + my_runs * p.L * group_bytes;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < p.stages; ++s) {
@@ -98,11 +109,12 @@ tc_wgrad_kernel(const __grid_constant__ CUtensorMap tmDy, const __grid_constant_
         prefetch_tmap(&tmX);
     }
     if (warp == 1) {
-        tmem_alloc(&tmem_base_slot, p.tmem_cols);
-        tmem_relinquish();
+        if constexpr (kPair) { tmem_alloc_pair(&tmem_base_slot, p.tmem_cols); tmem_relinquish_pair(); }
+        else { tmem_alloc(&tmem_base_slot, p.tmem_cols); tmem_relinquish(); }
     }
     tc_fence_before();
     __syncthreads();
+    if constexpr (kPair) cluster_sync_all();     // the peer's barriers exist before anything signals them
     tc_fence_after();
     const uint32_t tmem_base = tmem_base_slot;
 
@@ -111,67 +123,89 @@ tc_wgrad_kernel(const __grid_constant__ CUtensorMap tmDy, const __grid_constant_
     int box_end = box_begin + p.boxes_per_split;
     if (box_end > total_boxes) box_end = total_boxes;
     const int kiters = box_end > box_begin ? box_end - box_begin : 0;
-    const int bw = 1 << p.bw_log2, bh = 1 << p.bh_log2, bn = kPix >> (p.bw_log2 + p.bh_log2);
+    const int bw = 1 << p.bw_log2, bh = 1 << p.bh_log2, bn = p.pix >> (p.bw_log2 + p.bh_log2);
 
     if (warp == 0) {
+        // One thread; the loop is kept to a few instructions per copy (every instruction of a lone thread
+        // costs cycles of the k-step budget): addresses advance by addition, run coordinates are decoded once.
         if (lane == 0) {
             int stage = 0;
             uint32_t phase = 0;
             int issued = 0;
             bool ok = true;
-            // Per-run TMA coordinates are fixed for the item: decode them once (the k loop must stay
-            // free of integer divisions, this thread paces the whole pipeline).
             int run_dw[8], run_dh[8], run_c[8];
 #pragma unroll
             for (int j = 0; j < 8; ++j) {
-                const int run = run0 + (j < nruns ? j : 0);
-                const int tap = run / p.runs_per_tap;
-                const int cg0 = (run - tap * p.runs_per_tap) * p.L;
-                const int r = tap / p.S, s = tap - r * p.S;
-                run_dw[j] = s - p.pad_w;
-                run_dh[j] = r - p.pad_h;
-                run_c[j] = p.grouped ? cg0 : cg0 * 32;
+                const int run = my_run0 + (j < my_runs ? j : 0);
+                if (run < p.total_runs) {
+                    const int tap = run / p.runs_per_tap;
+                    const int cg0 = (run - tap * p.runs_per_tap) * p.L;
+                    const int r = tap / p.S, s = tap - r * p.S;
+                    run_dw[j] = s - p.pad_w;
+                    run_dh[j] = r - p.pad_h;
+                    run_c[j] = p.grouped ? cg0 : cg0 * 32;
+                } else {
+                    // (pair mode only) a run past the last tap: a group coordinate outside the tensor reads zeros
+                    run_dw[j] = 0; run_dh[j] = 0; run_c[j] = (p.C + 31) / 32;
+                }
             }
             int qi = box_begin % p.boxes_q;
             int pi = (box_begin / p.boxes_q) % p.boxes_p;
             int ni = box_begin / (p.boxes_q * p.boxes_p);
-            const uint32_t run_bytes = p.L * kGroupBytes;
+            const uint32_t run_bytes = p.L * group_bytes;
+            const uint32_t full0 = smem_u32(&full_bar[0]), empty0 = smem_u32(&empty_bar[0]), ring0 = smem_u32(smem);
+            const uint32_t full_dst0 = kPair ? map_to_cta(&full_bar[0], 0) : full0;     // where the copies complete
+            uint32_t full_a = full0, empty_a = empty0, full_dst = full_dst0, slot_a = ring0;
+            uint32_t dst = ring0;
             int sub = 0;                                         // position of the k-step inside its slot
+            int q0 = qi * bw, p0 = pi * bh, n0 = ni * bn;
             for (int b = box_begin; b < box_end; ++b) {
-                const int q0 = qi * bw, p0 = pi * bh, n0 = ni * bn;
-                if (++qi == p.boxes_q) { qi = 0; if (++pi == p.boxes_p) { pi = 0; ++ni; } }
                 if (sub == 0) {
-                    if (!bounded_wait(&empty_bar[stage], phase ^ 1u, &abort_flag, p.status, WAIT_PRODUCER_EMPTY)) { ok = false; break; }
+                    if (!bounded_wait_addr(empty_a, phase ^ 1u, &abort_flag, p.status, WAIT_PRODUCER_EMPTY)) { ok = false; break; }
                     const int nst = box_end - b < p.KS ? box_end - b : p.KS;
-                    mbar_expect_tx(&full_bar[stage], nst * tx_bytes);
+                    // pair: both CTAs' copies complete on the leader's barrier, which its producer arms
+                    if (!kPair) mbar_expect_tx_addr(full_a, nst * tx_bytes);
+                    else if (pair_rank == 0) mbar_expect_tx_addr(full_a, 2 * nst * tx_bytes);
+                    dst = slot_a;
                 }
-                uint8_t* dst = smem + stage * stage_bytes + sub * step_bytes;
                 if (p.grouped_dy) {
-                    tma_load_5d(dst, &tmDy, &full_bar[stage], 0, q0, p0, n0, kt * 4);
+                    tma_load_5d_addr<kPair>(dst, &tmDy, full_dst, 0, q0, p0, n0, kt * 4);
                 } else {
 #pragma unroll
                     for (int g = 0; g < 4; ++g)
-                        tma_load_4d(dst + g * kGroupBytes, &tmDy, &full_bar[stage], kt * 128 + g * 32, q0, p0, n0);
+                        tma_load_4d_addr<kPair>(dst + g * group_bytes, &tmDy, full_dst, kt * 128 + g * 32, q0, p0, n0);
                 }
+                const uint32_t xdst = dst + a_bytes;
                 if (p.x_taprows) {
-                    tma_load_5d(dst + kABytes, &tmX, &full_bar[stage], 0, q0 + run_dw[0], p0 + run_dh[0], n0, 0);
+                    tma_load_5d_addr<kPair>(xdst, &tmX, full_dst, 0, q0 + run_dw[0], p0 + run_dh[0], n0, 0);
                 } else if (p.grouped) {
 #pragma unroll
                     for (int j = 0; j < 8; ++j)
-                        if (j < nruns)
-                            tma_load_5d(dst + kABytes + j * run_bytes, &tmX, &full_bar[stage], 0, q0 + run_dw[j],
-                                        p0 + run_dh[j], n0, run_c[j]);
+                        if (j < my_runs)
+                            tma_load_5d_addr<kPair>(xdst + j * run_bytes, &tmX, full_dst, 0, q0 + run_dw[j], p0 + run_dh[j],
+                                                    n0, run_c[j]);
                 } else {
 #pragma unroll
                     for (int j = 0; j < 8; ++j)
-                        if (j < nruns)
-                            tma_load_4d(dst + kABytes + j * run_bytes, &tmX, &full_bar[stage], run_c[j],
-                                        q0 + run_dw[j], p0 + run_dh[j], n0);
+                        if (j < my_runs)
+                            tma_load_4d_addr<kPair>(xdst + j * run_bytes, &tmX, full_dst, run_c[j], q0 + run_dw[j],
+                                                    p0 + run_dh[j], n0);
                 }
+                // next pixel box
+                q0 += bw;
+                if (++qi == p.boxes_q) {
+                    qi = 0; q0 = 0; p0 += bh;
+                    if (++pi == p.boxes_p) { pi = 0; p0 = 0; n0 += bn; }
+                }
+                dst += step_bytes;
                 if (++sub == p.KS || b == box_end - 1) {
                     sub = 0;
                     ++issued;
-                    if (++stage == p.stages) { stage = 0; phase ^= 1u; }
+                    full_a += 8; empty_a += 8; full_dst += 8; slot_a += stage_bytes;
+                    if (++stage == p.stages) {
+                        stage = 0; phase ^= 1u;
+                        full_a = full0; empty_a = empty0; full_dst = full_dst0; slot_a = ring0;
+                    }
                 }
             }
             if (!ok) {
@@ -185,31 +219,34 @@ tc_wgrad_kernel(const __grid_constant__ CUtensorMap tmDy, const __grid_constant_
             }
         }
     } else if (warp == 1) {
-        if (lane == 0) {     // one thread runs the whole issue loop, waits included
-        const uint32_t idesc = make_idesc_tf32(n_groups * 32, true, true);
-        const uint64_t desc0 = make_smem_desc(0, kGroupBytes, 512, kSwizzle128B_Atom32B);
+        if (lane == 0 && pair_rank == 0) {     // one thread runs the whole issue loop, waits included
+        const uint32_t idesc = make_idesc_tf32(n_groups * 32, true, true, kPair ? 256u : 128u);
+        // 8 pixels per MMA = two 512-byte groups of 4 rows (1 KB, 64 sixteen-byte units, per MMA); descriptors differ
+        // only in the address field of their low word
+        const uint64_t desc0 = make_smem_desc(smem_u32(smem), group_bytes, 512, kSwizzle128B_Atom32B);
+        const uint32_t hi = uint32_t(desc0 >> 32), ring_lo0 = uint32_t(desc0);
+        const uint32_t full0 = smem_u32(&full_bar[0]), empty0 = smem_u32(&empty_bar[0]);
+        uint32_t full_a = full0, empty_a = empty0, slot_lo = ring_lo0;
+        const uint32_t stage16 = stage_bytes >> 4, step16 = step_bytes >> 4, a16 = a_bytes >> 4;
+        const bool wide = p.pix == 64;
         int stage = 0;
-        uint32_t phase = 0;
+        uint32_t phase = 0, accum = 0;
         bool ok = true;
         for (int kit = 0; kit < kiters; kit += p.KS) {
-            if (!bounded_wait(&full_bar[stage], phase, &abort_flag, p.status, WAIT_MMA_FULL)) { ok = false; break; }
+            if (!bounded_wait_addr(full_a, phase, &abort_flag, p.status, WAIT_MMA_FULL)) { ok = false; break; }
             tc_fence_after();
             const int nst = kiters - kit < p.KS ? kiters - kit : p.KS;
-            {
-              for (int j = 0; j < nst; ++j) {
-                // 8 pixels per instruction = two 512-byte groups of 4 rows; descriptors differ only in the
-                // address field, so add offsets to a constant part
-                const uint64_t da = desc0 + ((smem_u32(smem + stage * stage_bytes + j * step_bytes) & 0x3FFFFu) >> 4);
-                const uint64_t db = da + (kABytes >> 4);
-#pragma unroll
-                for (int kk = 0; kk < kPix / 8; ++kk)
-                    umma_tf32(tmem_base, da + kk * (1024 >> 4), db + kk * (1024 >> 4), idesc, (kit | j | kk) != 0);
-              }
-                umma_commit(&empty_bar[stage]);
+            uint32_t a_lo = slot_lo;
+            for (int j = 0; j < nst; ++j, a_lo += step16) {
+                umma_kstep_tf32<kPair, 64, 64>(tmem_base, a_lo, a_lo + a16, hi, hi, idesc, accum);
+                accum = 1;
+                if (wide) umma_kstep_tf32<kPair, 64, 64>(tmem_base, a_lo + 256, a_lo + a16 + 256, hi, hi, idesc, 1);
             }
-            if (++stage == p.stages) { stage = 0; phase ^= 1u; }
+            umma_commit_addr<kPair>(empty_a);
+            full_a += 8; empty_a += 8; slot_lo += stage16;
+            if (++stage == p.stages) { stage = 0; phase ^= 1u; full_a = full0; empty_a = empty0; slot_lo = ring_lo0; }
         }
-        if (ok) umma_commit(&tmem_full_bar);
+        if (ok) umma_commit_addr<kPair>(smem_u32(&tmem_full_bar));
         }
         __syncwarp();
     } else {
@@ -223,6 +260,7 @@ tc_wgrad_kernel(const __grid_constant__ CUtensorMap tmDy, const __grid_constant_
             const size_t krow = static_cast<size_t>(valid ? k : 0) * p.R * p.S;
             for (int ch = 0; ch < n_groups; ++ch) {
                 const int run = run0 + ch / p.L;
+                if (run >= p.total_runs) break;         // (pair mode) columns of runs past the last tap
                 const int tap = run / p.runs_per_tap;
                 const int c0 = ((run - tap * p.runs_per_tap) * p.L + ch % p.L) * 32;
                 float* dst = p.out + static_cast<size_t>(split) * p.split_stride + (krow + tap) * p.C + c0;
@@ -258,18 +296,21 @@ tc_wgrad_kernel(const __grid_constant__ CUtensorMap tmDy, const __grid_constant_
 
     tc_fence_before();
     __syncthreads();
+    if constexpr (kPair) cluster_sync_all();     // neither CTA leaves while the pair's MMAs may read its tiles
     if (warp == 1) {
         tc_fence_after();
-        tmem_dealloc(tmem_base, p.tmem_cols);
+        if constexpr (kPair) tmem_dealloc_pair(tmem_base, p.tmem_cols);
+        else tmem_dealloc(tmem_base, p.tmem_cols);
     }
 }
 
-void choose_pixel_box(int P, int Q, int N, int* bw_log2, int* bh_log2) {
+void choose_pixel_box(int pix, int P, int Q, int N, int* bw_log2, int* bh_log2) {
+    const int lp = pix == 64 ? 6 : 5;
     double best = 1e300;
     int best_w = 0, best_h = 0;
-    for (int lw = 5; lw >= 0; --lw)
-        for (int lh = 5 - lw; lh >= 0; --lh) {
-            const long bw = 1L << lw, bh = 1L << lh, bn = kPix / (bw * bh);
+    for (int lw = lp; lw >= 0; --lw)
+        for (int lh = lp - lw; lh >= 0; --lh) {
+            const long bw = 1L << lw, bh = 1L << lh, bn = pix / (bw * bh);
             const double covered = double((Q + bw - 1) / bw * bw) * double((P + bh - 1) / bh * bh) *
                                    double((N + bn - 1) / bn * bn);
             if (covered < best) { best = covered; best_w = lw; best_h = lh; }
@@ -278,25 +319,30 @@ void choose_pixel_box(int P, int Q, int N, int* bw_log2, int* bh_log2) {
     *bh_log2 = best_h;
 }
 
-long total_pixel_boxes(int N, int P, int Q) {
-    int lw, lh;
-    choose_pixel_box(P, Q, N, &lw, &lh);
-    const long bw = 1L << lw, bh = 1L << lh, bn = kPix / (bw * bh);
-    return ((Q + bw - 1) / bw) * ((P + bh - 1) / bh) * ((N + bn - 1) / bn);
+int env_int(const char* name, int dflt) {       // test / tuning hook
+    const char* v = getenv(name);
+    return v ? atoi(v) : dflt;
 }
 
-// How the columns of a layer are cut into runs and work items.
-struct RunPlan {
+// How a layer is cut into work items and k-steps.
+struct WgradPlan {
     int grouped, L, runs_per_tap, total_runs, rpi, run_blocks;
+    int pair;               // CTA pairs over k tiles 2i, 2i + 1
+    int pix;                // pixels per k-step
+    int KS, stages, step_bytes;
+    int bw_log2, bh_log2;
+    long boxes;
 };
 
-RunPlan plan_runs(int C, int K, int R, int S, int tap_groups) {
-    RunPlan r{};
+WgradPlan plan_wgrad(int N, int P, int Q, int C, int K, int R, int S, int tap_groups) {
+    WgradPlan r{};
     const int cgroups = (C + 31) / 32;
+    const int k_tiles = (K + 127) / 128;
     r.grouped = (!tap_groups && C % 32 == 0 && K % 32 == 0) ? 1 : 0;
+    r.pair = env_int("PCL_PAIR_WGRAD", 1) && r.grouped && k_tiles % 2 == 0;
     r.L = 1;
     if (r.grouped)
-        for (int l = 8; l >= 1; --l)
+        for (int l = r.pair ? 4 : 8; l >= 1; --l)        // pair: each CTA loads whole runs, half of the item's
             if (cgroups % l == 0) { r.L = l; break; }
     r.runs_per_tap = cgroups / r.L;
     r.total_runs = R * S * r.runs_per_tap;
@@ -306,8 +352,27 @@ RunPlan plan_runs(int C, int K, int R, int S, int tap_groups) {
     } else {
         const int blocks = (r.total_runs + rpi_max - 1) / rpi_max;
         r.rpi = (r.total_runs + blocks - 1) / blocks;   // balanced: 18 runs -> 3 x 6 rather than 8 + 8 + 2
+        if (r.pair && (r.rpi & 1)) ++r.rpi;             // (8 / L is even for L = 1..4, so this stays <= rpi_max)
     }
     r.run_blocks = (r.total_runs + r.rpi - 1) / r.rpi;
+    // 64-pixel k-steps halve the copies and commits per MMA; taken when three pipeline slots still fit
+    const int cta_groups = 4 + (r.pair ? r.rpi / 2 : r.rpi) * r.L;      // 32-map groups a CTA loads per k-step
+    r.pix = env_int("PCL_PIX_WGRAD", 64);
+    if (r.pix != 64 || kSmemBudget / (cta_groups * 64 * 128) < 3) r.pix = 32;
+    r.step_bytes = cta_groups * r.pix * 128;
+    // A k-step of a narrow column block is a few short MMAs; such blocks get several k-steps per slot (one
+    // barrier round trip and commit per slot) while at least 3 slots fit.
+    const int max_groups = r.rpi * r.L;
+    const int mma_clk = (r.pix / 8) * (max_groups * 16 > 52 ? max_groups * 16 : 52);
+    r.KS = (600 + mma_clk - 1) / mma_clk;
+    r.KS = env_int("PCL_KS_WGRAD", r.KS);
+    while (r.KS > 1 && kSmemBudget / (r.KS * r.step_bytes) < 3) --r.KS;
+    if (r.KS < 1) r.KS = 1;
+    r.stages = kSmemBudget / (r.KS * r.step_bytes);
+    if (r.stages > kMaxStages) r.stages = kMaxStages;
+    choose_pixel_box(r.pix, P, Q, N, &r.bw_log2, &r.bh_log2);
+    const long bw = 1L << r.bw_log2, bh = 1L << r.bh_log2, bn = r.pix / (bw * bh);
+    r.boxes = ((Q + bw - 1) / bw) * ((P + bh - 1) / bh) * ((N + bn - 1) / bn);
     return r;
 }
 
@@ -333,55 +398,48 @@ bool tc_wgrad_eligible(const TcWgradArgs& a) {
 }
 
 int tc_wgrad_splits(int N, int P, int Q, int C, int K, int R, int S, int tap_groups) {
-    const RunPlan rp = plan_runs(C, K, R, S, tap_groups);
+    const WgradPlan rp = plan_wgrad(N, P, Q, C, K, R, S, tap_groups);
     const long items = long((K + 127) / 128) * rp.run_blocks;
-    const long boxes = total_pixel_boxes(N, P, Q);
     long splits = sm_count() / items;
     if (splits < 1) splits = 1;
     if (splits > 64 && !tap_groups) splits = 64;
-    if (splits > boxes) splits = boxes;
+    if (splits > rp.boxes) splits = rp.boxes;
     // drop splits that would be empty
-    const long per = (boxes + splits - 1) / splits;
-    splits = (boxes + per - 1) / per;
+    const long per = (rp.boxes + splits - 1) / splits;
+    splits = (rp.boxes + per - 1) / per;
     return int(splits);
 }
 
 int launch_tc_wgrad(const TcWgradArgs& a, cudaStream_t st) {
     if (!tc_wgrad_eligible(a)) return PCL_ERR_UNSUPPORTED_SHAPE;
     if (!g_attr_set) {
-        if (cudaFuncSetAttribute(tc_wgrad_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget + 1024) !=
-            cudaSuccess)
+        if (cudaFuncSetAttribute(tc_wgrad_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 kSmemBudget + 1024) != cudaSuccess ||
+            cudaFuncSetAttribute(tc_wgrad_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 kSmemBudget + 1024) != cudaSuccess)
             return PCL_ERR_CUDA;
         g_attr_set = true;
     }
     WgradParams p{};
-    choose_pixel_box(a.P, a.Q, a.N, &p.bw_log2, &p.bh_log2);
-    const int bw = 1 << p.bw_log2, bh = 1 << p.bh_log2, bn = kPix / (bw * bh);
+    const WgradPlan rp = plan_wgrad(a.N, a.P, a.Q, a.C, a.K, a.R, a.S, a.tap_groups);
+    p.pix = rp.pix; p.bw_log2 = rp.bw_log2; p.bh_log2 = rp.bh_log2;
+    const int bw = 1 << p.bw_log2, bh = 1 << p.bh_log2, bn = p.pix / (bw * bh);
     p.boxes_q = (a.Q + bw - 1) / bw;
     p.boxes_p = (a.P + bh - 1) / bh;
     p.boxes_n = (a.N + bn - 1) / bn;
-    const long boxes = long(p.boxes_q) * p.boxes_p * p.boxes_n;
+    const long boxes = rp.boxes;
     if (boxes > 0x7fffffffL) return PCL_ERR_UNSUPPORTED_SHAPE;
-    const RunPlan rp = plan_runs(a.C, a.K, a.R, a.S, a.tap_groups);
     p.grouped = rp.grouped; p.grouped_dy = (a.K % 32 == 0) ? 1 : 0; p.x_taprows = a.tap_groups ? 1 : 0; p.L = rp.L; p.runs_per_tap = rp.runs_per_tap; p.total_runs = rp.total_runs;
     p.rpi = rp.rpi; p.run_blocks = rp.run_blocks;
     p.k_tiles = (a.K + 127) / 128;
     p.R = a.R; p.S = a.S; p.pad_h = a.pad_h; p.pad_w = a.pad_w;
     p.K = a.K; p.C = a.C;
     p.splits = a.splits;
+    if (p.splits < 1) return PCL_ERR_BAD_ARG;
     p.boxes_per_split = int((boxes + p.splits - 1) / p.splits);
     const int max_groups = p.rpi * p.L;
-    const int step_bytes = kABytes + max_groups * kGroupBytes;
-    // A k-step of a narrow column block is 4 short MMAs; the issuing thread's per-slot round trip (~600
-    // cycles) then dominates, so such blocks get several k-steps per slot while at least 3 slots fit.
-    const int mma_clk = 4 * (max_groups * 16 > 52 ? max_groups * 16 : 52);
-    p.KS = (600 + mma_clk - 1) / mma_clk;
-    if (getenv("PCL_KS_WGRAD")) p.KS = atoi(getenv("PCL_KS_WGRAD"));
-    while (p.KS > 1 && kSmemBudget / (p.KS * step_bytes) < 3) --p.KS;
-    if (p.KS < 1) p.KS = 1;
-    const int stage_bytes = p.KS * step_bytes;
-    p.stages = kSmemBudget / stage_bytes;
-    if (p.stages > kMaxStages) p.stages = kMaxStages;
+    p.KS = rp.KS; p.stages = rp.stages;
+    const int stage_bytes = p.KS * rp.step_bytes;
     p.tmem_cols = 32;
     while (p.tmem_cols < max_groups * 32) p.tmem_cols *= 2;
     p.status = device_status_ptr();
@@ -451,7 +509,17 @@ int launch_tc_wgrad(const TcWgradArgs& a, cudaStream_t st) {
     const size_t smem = size_t(p.stages) * stage_bytes + 1024;
     {
         LaunchScope scope(KID_TC_WGRAD, 2.0 * a.N * a.P * a.Q * double(a.K) * a.C * a.R * a.S, st);
-        tc_wgrad_kernel<<<int(items), 192, smem, st>>>(tmDy, tmX, p);
+        if (rp.pair) {
+            cudaLaunchAttribute attr[1];
+            attr[0].id = cudaLaunchAttributeClusterDimension;
+            attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+            cudaLaunchConfig_t lc{};
+            lc.gridDim = dim3(unsigned(items)); lc.blockDim = dim3(192); lc.dynamicSmemBytes = smem; lc.stream = st;
+            lc.attrs = attr; lc.numAttrs = 1;
+            if (cudaLaunchKernelEx(&lc, tc_wgrad_kernel<true>, tmDy, tmX, p) != cudaSuccess) return PCL_ERR_CUDA;
+        } else {
+            tc_wgrad_kernel<false><<<int(items), 192, smem, st>>>(tmDy, tmX, p);
+        }
     }
     if (cudaGetLastError() != cudaSuccess) return PCL_ERR_CUDA;
     if (p.splits > 1 && a.partial && !a.skip_reduce) return launch_reduce_splits(a.partial, a.dw, dw_elems, p.splits, st);
