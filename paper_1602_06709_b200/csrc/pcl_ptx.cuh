@@ -79,6 +79,33 @@ __device__ __forceinline__ bool bounded_wait_warp(uint64_t* bar, uint32_t parity
     return __all_sync(0xffffffffu, ok);
 }
 
+// Low-duty form for warps that wait long (an epilogue warp waits for a whole main loop): lane 0 polls and
+// sleeps between polls, so that the wait takes almost no issue slots from the single-thread pipeline loops
+// that share the warp scheduler; the result is broadcast.
+__device__ __forceinline__ bool bounded_wait_warp_relaxed(uint64_t* bar, uint32_t parity, volatile uint32_t* abort_flag,
+                                                          unsigned int* status_word, uint32_t code) {
+    int ok = 1;
+    if ((threadIdx.x & 31) == 0) {
+        unsigned long long t0 = 0;
+        ok = 0;
+        for (uint32_t spin = 0;; ++spin) {
+            if (mbar_try_wait(bar, parity)) { ok = 1; break; }
+            __nanosleep(200);
+            if ((spin & 15u) == 15u) {
+                if (*abort_flag) break;
+                const unsigned long long now = global_nanos();
+                if (t0 == 0) t0 = now;
+                else if (now - t0 > kWaitNanos) {
+                    *abort_flag = 1u;
+                    atomicCAS(status_word, 0u, code);
+                    break;
+                }
+            }
+        }
+    }
+    return __shfl_sync(0xffffffffu, ok, 0) != 0;
+}
+
 // ---------------------------------------------------------------------- TMA
 __device__ __forceinline__ void prefetch_tmap(const CUtensorMap* m) {
     asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(m)) : "memory");
@@ -155,6 +182,16 @@ __device__ __forceinline__ void tmem_ld_32x32(uint32_t taddr, uint32_t (&v)[32])
         : "r"(taddr)
         : "memory");
 }
+// Zero 32 lanes x 32 consecutive fp32 columns (the counterpart of tmem_ld_32x32).
+__device__ __forceinline__ void tmem_st_32x32_zero(uint32_t taddr) {
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
+        "{%1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1, "
+        "%1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1};"
+        ::"r"(taddr), "r"(0u)
+        : "memory");
+}
+__device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 
 // ------------------------------------------------------- CTA pairs (cta_group::2)
@@ -394,6 +431,7 @@ enum : uint32_t {
     WAIT_MMA_TMEM_EMPTY = 0x103,
     WAIT_EPI_TMEM_FULL = 0x104,
     WAIT_DRAIN = 0x105,
+    WAIT_ISSUE_TURN = 0x106,
 };
 
 }  // namespace pcl

@@ -36,7 +36,8 @@ constexpr int kMaxStages = 8;
 constexpr int kSmemBudget = 224 * 1024;
 constexpr int kEpiWarps = 8;                    // two per TMEM lane quarter, splitting the column chunks
 constexpr int kEpiStageBytes = kEpiWarps * 4096;
-constexpr int kThreads = (2 + kEpiWarps) * 32;
+constexpr int kSecondIssuerWarp = 2 + kEpiWarps;        // warp 10
+constexpr int kThreads = (3 + kEpiWarps) * 32;
 
 struct FpropParams {
     int bw_log2, bh_log2;       // box of output pixels: bw x bh x (128 / (bw*bh))
@@ -47,6 +48,7 @@ struct FpropParams {
     int act;
     int stages;
     int KS;                     // k-steps (plain: {A,B} pairs; halo: weight tiles of consecutive taps) per pipeline slot
+    int issuers;                // MMA-issuing threads (1 or 2; see the kernel)
     int grp;                    // plain tiling: a slot's KS k-steps are KS consecutive channel blocks of one tap, fetched by
                                 // ONE copy of A and one of B (slot layout: KS A tiles, then KS B tiles)
     int tmem_cols;
@@ -92,12 +94,209 @@ struct TileIter {
     }
 };
 
+// Two MMA issuers take turns: the thread that owns slot `seq` spins (bounded) until the slots before it have
+// been issued.  The other thread is at most one slot of MMAs away, so the wait is short.
+__device__ __forceinline__ bool wait_issue_turn(volatile uint32_t* issue_seq, uint32_t seq, volatile uint32_t* abort_flag,
+                                                unsigned int* status_word) {
+    if (*issue_seq == seq) return true;
+    unsigned long long t0 = 0;
+    for (uint32_t spin = 0;; ++spin) {
+        if (*issue_seq == seq) return true;
+        if ((spin & 255u) == 255u) {
+            if (*abort_flag) return false;
+            const unsigned long long now = global_nanos();
+            if (t0 == 0) t0 = now;
+            else if (now - t0 > kWaitNanos) break;
+        }
+    }
+    *abort_flag = 1u;
+    atomicCAS(status_word, 0u, static_cast<unsigned int>(WAIT_ISSUE_TURN));
+    return false;
+}
+
+// What the issuing thread needs from the kernel body.
+struct IssuerCtx {
+    uint8_t* smem;
+    uint8_t* b_ring;
+    uint64_t *full_bar, *empty_bar, *fullA_bar, *emptyA_bar, *tmem_full_bar, *tmem_empty_bar;
+    volatile uint32_t* abort_flag;
+    volatile uint32_t* issue_seq;
+    uint32_t tmem_base, b_bytes, step_bytes, stage_bytes;
+    int first_tile, tile_stride, total_tiles, kiters;
+};
+
+// kTaps consecutive taps of a haloed slot, straight-line (a taken branch costs a lone thread tens of cycles).
+template <bool kPair, int kTaps, int kMT>
+__device__ __forceinline__ void halo_taps(uint32_t d_tmem, uint32_t BN, uint32_t& a_lo, uint32_t b_lo, int& s, int S,
+                                          uint32_t row16, uint32_t half_off16, uint32_t b16, uint32_t a_hi,
+                                          uint32_t b_hi, uint32_t idesc, uint32_t& accum) {
+#pragma unroll
+    for (int j = 0; j < kTaps; ++j) {
+        umma_kstep_tf32<kPair, 2, 2>(d_tmem, a_lo, b_lo, a_hi, b_hi, idesc, accum);
+        if (kMT == 2) umma_kstep_tf32<kPair, 2, 2>(d_tmem + BN, a_lo + half_off16, b_lo, a_hi, b_hi, idesc, accum);
+        accum = 1;
+        b_lo += b16;
+        const bool wrap = ++s == S;     // the tap (r, s): next pixel of the patch, or the start of the next patch row
+        a_lo += wrap ? 8 + row16 : 8;
+        s = wrap ? 0 : s;
+    }
+}
+
+// The MMA-issuing role, one thread per issuing warp (waits included), kept out of line and free of anything the
+// loops do not need.  A lone thread executes an instruction every several cycles; a barrier poll or a commit costs
+// it ~80 cycles and every MMA ~45, so per slot it spends 300-400 cycles outside the MMAs, which the MMA queue (4-5
+// deep) hides only behind wide MMAs (N = 256).  kDuo: two issuers take the slots alternately, so that one thread's
+// bookkeeping overlaps the other's MMAs.  MMAs of both accumulate into the same tile (the pipe executes them one
+// after another whichever thread issued them); a sequence number in shared memory makes the threads issue slot g
+// only after slot g-1 has been issued, so the order of the additions, and with it every bit of the result, is
+// that of a single issuer.
+template <bool kPair, bool kDuo>
+__device__ __noinline__ void mma_issuer(const FpropParams& p, const IssuerCtx& c, const uint32_t issuer) {
+    // Everything the loops use is copied into registers first: the asm statements below clobber memory, so
+    // anything left behind a reference would be re-read after each of them.
+    const int BN = p.BN, KS = p.KS, MT = p.MT, NA = p.NA, PW = p.PW, S = p.S, taps = p.R * p.S;
+    const int a_buf_bytes = p.a_buf_bytes, cblocks = p.cblocks, grp = p.grp, halo = p.halo, stages = p.stages;
+    const uint32_t half_off16 = p.half_off_bytes >> 4;
+    unsigned int* const status = p.status;
+    volatile uint32_t* const abort_flag = c.abort_flag;
+    volatile uint32_t* const issue_seq = c.issue_seq;
+    uint8_t* const smem = c.smem;
+    const uint32_t fullA0 = smem_u32(&c.fullA_bar[0]), emptyA0 = smem_u32(&c.emptyA_bar[0]);
+    const uint32_t tfull0 = smem_u32(&c.tmem_full_bar[0]), tempty0 = smem_u32(&c.tmem_empty_bar[0]);
+    const uint32_t tmem_base = c.tmem_base, b16 = c.b_bytes >> 4;
+    const int first_tile = c.first_tile, tile_stride = c.tile_stride, total_tiles = c.total_tiles, kiters = c.kiters;
+
+    const uint32_t idesc = make_idesc_tf32(BN, false, false, kPair ? 256u : 128u);
+    // Descriptors differ only in the 14-bit address field (address >> 4) of their low word: the loops keep low
+    // words in registers and advance them by addition.
+    const uint64_t b_desc0 = make_smem_desc(smem_u32(halo ? c.b_ring : smem), 16, 1024, kSwizzle128B);
+    const uint32_t b_hi = uint32_t(b_desc0 >> 32), ring_lo0 = uint32_t(b_desc0);
+    const uint32_t full0 = smem_u32(&c.full_bar[0]), empty0 = smem_u32(&c.empty_bar[0]);
+    const uint32_t stage16 = c.stage_bytes >> 4, step16 = c.step_bytes >> 4;
+    // where k-step j of a slot finds its operands (16-byte units from the slot start)
+    const uint32_t a_step16 = grp ? (kABytes >> 4) : step16;
+    const uint32_t b_off16 = grp ? KS * (kABytes >> 4) : (kABytes >> 4);
+    const uint32_t b_step16 = grp ? b16 : step16;
+
+    uint32_t full_a = full0, empty_a = empty0, slot_lo = ring_lo0;     // ring position
+    int stage = 0;
+    uint32_t phase = 0;
+    uint32_t turn = 0, seq = 0;     // kDuo: whose slot comes next; slots so far (both threads count alike)
+    int a_slot = 0;
+    uint32_t phaseA = 0;
+    int tile_cnt = 0;
+    bool ok = true;
+
+#define PCL_SLOT_BEGIN()                                                                                          \
+    bool mine = true;                                                                                             \
+    if (kDuo) { mine = turn == issuer; turn ^= 1u; }
+#define PCL_SLOT_ACQUIRE()                                                                                        \
+    if (!bounded_wait_addr(full_a, phase, abort_flag, status, WAIT_MMA_FULL)) { ok = false; break; }             \
+    if (kDuo && !wait_issue_turn(issue_seq, seq, abort_flag, status)) { ok = false; break; }                     \
+    tc_fence_after();
+#define PCL_SLOT_RELEASE()                                                                                        \
+    if (kDuo) *issue_seq = seq + 1;                                                                               \
+    umma_commit_addr<kPair>(empty_a);
+#define PCL_SLOT_END()                                                                                            \
+    if (kDuo) ++seq;                                                                                              \
+    accum = 1;                                                                                                    \
+    full_a += 8; empty_a += 8; slot_lo += stage16;                                                                \
+    if (++stage == stages) { stage = 0; phase ^= 1u; full_a = full0; empty_a = empty0; slot_lo = ring_lo0; }
+
+    for (int t = first_tile; t < total_tiles && ok; t += tile_stride, ++tile_cnt) {
+        const uint32_t acc = tile_cnt & 1;
+        const uint32_t acc_phase = (tile_cnt >> 1) & 1;
+        if (!bounded_wait_addr(tempty0 + acc * 8, acc_phase ^ 1u, abort_flag, status, WAIT_MMA_TMEM_EMPTY)) break;
+        tc_fence_after();
+        const uint32_t d_tmem = tmem_base + acc * MT * BN;
+        uint32_t accum = 0;         // the tile's first MMA (whoever issues it) overwrites the accumulator
+        if (halo) {
+            const uint64_t a_desc0 = make_smem_desc(0, 16, PW * 128, kSwizzle128B);   // 8-pixel groups are one patch row apart
+            const uint32_t a_hi = uint32_t(a_desc0 >> 32);
+            const uint32_t row16 = (PW - S) * 8;        // from the end of a tap row to the start of the next
+            for (int cb = 0; cb < cblocks && ok; ++cb) {
+                if (!bounded_wait_addr(fullA0 + a_slot * 8, phaseA, abort_flag, status, WAIT_MMA_FULL)) { ok = false; break; }
+                // the tap (r, s) = a shift by (r * PW + s) pixels of 128 bytes inside the patch
+                uint32_t a_lo = uint32_t(a_desc0) + ((smem_u32(smem + a_slot * a_buf_bytes) & 0x3FFFFu) >> 4);
+                int s = 0;
+                for (int tap = 0; tap < taps; tap += KS) {
+                    const int nst = taps - tap < KS ? taps - tap : KS;
+                    PCL_SLOT_BEGIN()
+                    if (mine) {
+                        PCL_SLOT_ACQUIRE()
+                        if (MT == 2) {
+                            if (nst == 3) halo_taps<kPair, 3, 2>(d_tmem, BN, a_lo, slot_lo, s, S, row16, half_off16, b16, a_hi, b_hi, idesc, accum);
+                            else if (nst == 2) halo_taps<kPair, 2, 2>(d_tmem, BN, a_lo, slot_lo, s, S, row16, half_off16, b16, a_hi, b_hi, idesc, accum);
+                            else {
+                                uint32_t b_lo = slot_lo;
+                                for (int j = 0; j < nst; ++j, b_lo += b16)
+                                    halo_taps<kPair, 1, 2>(d_tmem, BN, a_lo, b_lo, s, S, row16, half_off16, b16, a_hi, b_hi, idesc, accum);
+                            }
+                        } else {
+                            if (nst == 3) halo_taps<kPair, 3, 1>(d_tmem, BN, a_lo, slot_lo, s, S, row16, half_off16, b16, a_hi, b_hi, idesc, accum);
+                            else if (nst == 2) halo_taps<kPair, 2, 1>(d_tmem, BN, a_lo, slot_lo, s, S, row16, half_off16, b16, a_hi, b_hi, idesc, accum);
+                            else {
+                                uint32_t b_lo = slot_lo;
+                                for (int j = 0; j < nst; ++j, b_lo += b16)
+                                    halo_taps<kPair, 1, 1>(d_tmem, BN, a_lo, b_lo, s, S, row16, half_off16, b16, a_hi, b_hi, idesc, accum);
+                            }
+                        }
+                        PCL_SLOT_RELEASE()
+                    } else {
+                        for (int j = 0; j < nst; ++j) {
+                            const bool wrap = ++s == S;
+                            a_lo += wrap ? 8 + row16 : 8;
+                            s = wrap ? 0 : s;
+                        }
+                    }
+                    PCL_SLOT_END()
+                }
+                if (ok) umma_commit_addr<kPair>(emptyA0 + a_slot * 8);       // one arrival per issuer
+                if (++a_slot == NA) { a_slot = 0; phaseA ^= 1u; }
+            }
+        } else if (KS == 2 && grp) {
+            // two k-steps per slot, fetched by one copy per operand (the hot loop of the wide layers)
+            for (int kit = 0; kit < kiters; kit += 2) {
+                PCL_SLOT_BEGIN()
+                if (mine) {
+                    PCL_SLOT_ACQUIRE()
+                    umma_kstep_tf32<kPair, 2, 2>(d_tmem, slot_lo, slot_lo + b_off16, b_hi, b_hi, idesc, accum);
+                    umma_kstep_tf32<kPair, 2, 2>(d_tmem, slot_lo + a_step16, slot_lo + b_off16 + b_step16, b_hi, b_hi, idesc, 1);
+                    PCL_SLOT_RELEASE()
+                }
+                PCL_SLOT_END()
+            }
+        } else {
+            for (int kit = 0; kit < kiters; kit += KS) {
+                const int nst = kiters - kit < KS ? kiters - kit : KS;
+                PCL_SLOT_BEGIN()
+                if (mine) {
+                    PCL_SLOT_ACQUIRE()
+                    uint32_t a_lo = slot_lo, b_lo = slot_lo + b_off16;
+                    for (int j = 0; j < nst; ++j, a_lo += a_step16, b_lo += b_step16) {
+                        umma_kstep_tf32<kPair, 2, 2>(d_tmem, a_lo, b_lo, b_hi, b_hi, idesc, accum);
+                        accum = 1;
+                    }
+                    PCL_SLOT_RELEASE()
+                }
+                PCL_SLOT_END()
+            }
+        }
+        if (ok) umma_commit_addr<kPair>(tfull0 + acc * 8);       // one arrival per issuer
+    }
+#undef PCL_SLOT_BEGIN
+#undef PCL_SLOT_ACQUIRE
+#undef PCL_SLOT_RELEASE
+#undef PCL_SLOT_END
+}
+
 // kPair: two CTAs of a cluster (ranks 0 and 1) compute two M tiles (consecutive image groups) against the
 // same BN = 256 weight tile with M = 256 MMAs issued by rank 0; each CTA loads its own A tile and only half
 // of the weight rows, which cuts the shared-memory fill traffic per MMA by a third (plain tiling only).
 template <bool kPair>
 __global__ void __launch_bounds__(kThreads, 1)
-tc_fprop_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, FpropParams p) {
+tc_fprop_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+                const __grid_constant__ FpropParams p) {
     extern __shared__ uint8_t smem_raw[];
     __shared__ uint64_t full_bar[kMaxStages];
     __shared__ uint64_t empty_bar[kMaxStages];
@@ -107,6 +306,7 @@ tc_fprop_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
     __shared__ uint64_t tmem_empty_bar[2];
     __shared__ uint32_t tmem_base_slot;
     __shared__ uint32_t abort_flag;
+    __shared__ volatile uint32_t issue_seq;      // two issuers: number of slots whose MMAs have been issued
 
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
@@ -138,13 +338,14 @@ tc_fprop_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
         }
         for (int a = 0; a < 4; ++a) {
             mbar_init(&fullA_bar[a], 1);
-            mbar_init(&emptyA_bar[a], 1);
+            mbar_init(&emptyA_bar[a], p.issuers);
         }
         for (int a = 0; a < 2; ++a) {
-            mbar_init(&tmem_full_bar[a], 1);
+            mbar_init(&tmem_full_bar[a], p.issuers);
             mbar_init(&tmem_empty_bar[a], kPair ? 2 * kEpiWarps : kEpiWarps);
         }
         abort_flag = 0;
+        issue_seq = 0;
         mbar_fence_init();
         prefetch_tmap(&tmA);
         prefetch_tmap(&tmB);
@@ -192,9 +393,11 @@ tc_fprop_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                             ok = false;
                             break;
                         }
-                        mbar_expect_tx(&fullA_bar[a_slot], p.patch_bytes);
-                        tma_load_4d(smem + a_slot * p.a_buf_bytes, &tmA, &fullA_bar[a_slot], c0, q0 - p.pad_w,
-                                    p0 - p.pad_h, n0);
+                        if (!kPair) mbar_expect_tx(&fullA_bar[a_slot], p.patch_bytes);
+                        else if (pair_rank == 0) mbar_expect_tx(&fullA_bar[a_slot], 2 * p.patch_bytes);
+                        tma_load_4d_addr<kPair>(smem_u32(smem + a_slot * p.a_buf_bytes), &tmA,
+                                                kPair ? map_to_cta(&fullA_bar[a_slot], 0) : smem_u32(&fullA_bar[a_slot]),
+                                                c0, q0 - p.pad_w, p0 - p.pad_h, n0);
                         ++issuedA;
                         if (++a_slot == p.NA) { a_slot = 0; phaseA ^= 1u; }
                         for (int tap = 0; tap < taps; tap += p.KS) {
@@ -203,13 +406,24 @@ tc_fprop_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                                 break;
                             }
                             const int nst = taps - tap < p.KS ? taps - tap : p.KS;
-                            mbar_expect_tx_addr(full_a, nst * b_bytes);
-                            uint32_t dst = slot_a;
-                            for (int j = 0; j < nst; ++j, dst += b_bytes)
-                                tma_load_3d_addr<false>(dst, &tmB, full_a, c0, tap + j, kcol);
+                            const int ncp = p.grp ? p.KS : nst;       // a box counts in full, also where it is filled with zeros
+                            if (!kPair) mbar_expect_tx_addr(full_a, ncp * b_bytes);
+                            else if (pair_rank == 0) mbar_expect_tx_addr(full_a, 2 * ncp * b_bytes);
+                            if (p.grp) {
+                                // the slot's taps in one copy (box {32 channels, BN maps, KS taps}; taps past the last
+                                // one are outside the tensor: filled with zeros and not used)
+                                tma_load_3d_addr<kPair>(slot_a, &tmB, full_dst, c0, kcol, tap);
+                            } else {
+                                uint32_t dst = slot_a;
+                                for (int j = 0; j < nst; ++j, dst += b_bytes)
+                                    tma_load_3d_addr<kPair>(dst, &tmB, full_dst, c0, tap + j, kcol);
+                            }
                             ++issued;
-                            full_a += 8; empty_a += 8; slot_a += stage_bytes;
-                            if (++stage == p.stages) { stage = 0; phase ^= 1u; full_a = full0; empty_a = empty0; slot_a = ring0; }
+                            full_a += 8; empty_a += 8; full_dst += 8; slot_a += stage_bytes;
+                            if (++stage == p.stages) {
+                                stage = 0; phase ^= 1u;
+                                full_a = full0; empty_a = empty0; full_dst = full_dst0; slot_a = ring0;
+                            }
                         }
                     }
                 } else {
@@ -271,108 +485,19 @@ tc_fprop_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                 }
             }
         }
-    } else if (warp == 1) {
-        // ---------------------------------------------------------- MMA issuer
-        // One thread runs the whole loop (waits included): a warp-wide wait + re-convergence per slot would
-        // add to the per-slot cost that bounds narrow tiles.
-        if (lane == 0 && pair_rank == 0) {
-        const uint32_t idesc = make_idesc_tf32(p.BN, false, false, kPair ? 256u : 128u);
-        int stage = 0;
-        uint32_t phase = 0;
-        int a_slot = 0;
-        uint32_t phaseA = 0;
-        int tile_cnt = 0;
-        bool ok = true;
-        // Descriptors differ only in the 14-bit address field (address >> 4) of their low word: the loop keeps
-        // low words in registers and advances them by addition.
-        const uint64_t b_desc0 = make_smem_desc(smem_u32(p.halo ? b_ring : smem), 16, 1024, kSwizzle128B);
-        const uint32_t b_hi = uint32_t(b_desc0 >> 32), ring_lo0 = uint32_t(b_desc0);
-        const uint32_t full0 = smem_u32(&full_bar[0]), empty0 = smem_u32(&empty_bar[0]);
-        uint32_t full_a = full0, empty_a = empty0, slot_lo = ring_lo0;
-        const uint32_t stage16 = stage_bytes >> 4, step16 = step_bytes >> 4;
-        // where k-step j of a slot finds its operands (16-byte units from the slot start)
-        const uint32_t a_step16 = p.grp ? (kABytes >> 4) : step16;
-        const uint32_t b_off16 = p.grp ? p.KS * (kABytes >> 4) : (kABytes >> 4);
-        const uint32_t b_step16 = p.grp ? (b_bytes >> 4) : step16;
-        for (int t = first_tile; t < total_tiles && ok; t += tile_stride, ++tile_cnt) {
-            const int acc = tile_cnt & 1;
-            const uint32_t acc_phase = (tile_cnt >> 1) & 1;
-            if (!bounded_wait(&tmem_empty_bar[acc], acc_phase ^ 1u, &abort_flag, p.status, WAIT_MMA_TMEM_EMPTY)) break;
-            tc_fence_after();
-            const uint32_t d_tmem = tmem_base + acc * p.MT * p.BN;
-            uint32_t accum = 0;         // the tile's first MMA overwrites the accumulator
-            if (p.halo) {
-                const uint64_t a_desc0 = make_smem_desc(0, 16, p.PW * 128, kSwizzle128B);   // 8-pixel groups are one patch row apart
-                const uint32_t a_hi = uint32_t(a_desc0 >> 32);
-                const uint32_t half_off16 = p.half_off_bytes >> 4;
-                const uint32_t row16 = (p.PW - p.S) * 8;        // from the end of a tap row to the start of the next
-                const int taps = p.R * p.S;
-                for (int cb = 0; cb < p.cblocks && ok; ++cb) {
-                    if (!bounded_wait(&fullA_bar[a_slot], phaseA, &abort_flag, p.status, WAIT_MMA_FULL)) { ok = false; break; }
-                    // the tap (r, s) = a shift by (r * PW + s) pixels of 128 bytes inside the patch
-                    uint32_t a_lo = uint32_t(a_desc0) + ((smem_u32(smem + a_slot * p.a_buf_bytes) & 0x3FFFFu) >> 4);
-                    int s = 0;
-                    for (int tap = 0; tap < taps; tap += p.KS) {
-                        if (!bounded_wait_addr(full_a, phase, &abort_flag, p.status, WAIT_MMA_FULL)) { ok = false; break; }
-                        tc_fence_after();
-                        const int nst = taps - tap < p.KS ? taps - tap : p.KS;
-                        uint32_t b_lo = slot_lo;
-                        for (int j = 0; j < nst; ++j) {
-                            umma_kstep_tf32<kPair, 2, 2>(d_tmem, a_lo, b_lo, a_hi, b_hi, idesc, accum);
-                            accum = 1;
-                            if (p.MT == 2) umma_kstep_tf32<kPair, 2, 2>(d_tmem + p.BN, a_lo + half_off16, b_lo, a_hi, b_hi, idesc, tap | j | cb);
-                            b_lo += b_bytes >> 4;
-                            a_lo += 8;
-                            if (++s == p.S) { s = 0; a_lo += row16; }
-                        }
-                        umma_commit_addr<kPair>(empty_a);
-                        full_a += 8; empty_a += 8; slot_lo += stage16;
-                        if (++stage == p.stages) { stage = 0; phase ^= 1u; full_a = full0; empty_a = empty0; slot_lo = ring_lo0; }
-                    }
-                    if (ok) commit(&emptyA_bar[a_slot]);
-                    if (++a_slot == p.NA) { a_slot = 0; phaseA ^= 1u; }
-                }
-            } else if (p.KS == 1) {
-                // the hot loop of the wide layers: one k-step per slot, nothing but the wait, four MMAs, the commit
-                // and the ring advance
-                for (int kit = 0; kit < kiters; ++kit) {
-                    if (!bounded_wait_addr(full_a, phase, &abort_flag, p.status, WAIT_MMA_FULL)) { ok = false; break; }
-                    tc_fence_after();
-                    umma_kstep_tf32<kPair, 2, 2>(d_tmem, slot_lo, slot_lo + (kABytes >> 4), b_hi, b_hi, idesc, accum);
-                    accum = 1;
-                    umma_commit_addr<kPair>(empty_a);
-                    full_a += 8; empty_a += 8; slot_lo += stage16;
-                    if (++stage == p.stages) { stage = 0; phase ^= 1u; full_a = full0; empty_a = empty0; slot_lo = ring_lo0; }
-                }
-            } else if (p.KS == 2 && p.grp) {
-                // two k-steps per slot, fetched by one copy per operand
-                for (int kit = 0; kit < kiters; kit += 2) {
-                    if (!bounded_wait_addr(full_a, phase, &abort_flag, p.status, WAIT_MMA_FULL)) { ok = false; break; }
-                    tc_fence_after();
-                    umma_kstep_tf32<kPair, 2, 2>(d_tmem, slot_lo, slot_lo + b_off16, b_hi, b_hi, idesc, accum);
-                    umma_kstep_tf32<kPair, 2, 2>(d_tmem, slot_lo + a_step16, slot_lo + b_off16 + b_step16, b_hi, b_hi, idesc, 1);
-                    accum = 1;
-                    umma_commit_addr<kPair>(empty_a);
-                    full_a += 8; empty_a += 8; slot_lo += stage16;
-                    if (++stage == p.stages) { stage = 0; phase ^= 1u; full_a = full0; empty_a = empty0; slot_lo = ring_lo0; }
-                }
-            } else {
-                for (int kit = 0; kit < kiters; kit += p.KS) {
-                    if (!bounded_wait_addr(full_a, phase, &abort_flag, p.status, WAIT_MMA_FULL)) { ok = false; break; }
-                    tc_fence_after();
-                    const int nst = kiters - kit < p.KS ? kiters - kit : p.KS;
-                    uint32_t a_lo = slot_lo, b_lo = slot_lo + b_off16;
-                    for (int j = 0; j < nst; ++j, a_lo += a_step16, b_lo += b_step16) {
-                        umma_kstep_tf32<kPair, 2, 2>(d_tmem, a_lo, b_lo, b_hi, b_hi, idesc, accum);
-                        accum = 1;
-                    }
-                    umma_commit_addr<kPair>(empty_a);
-                    full_a += 8; empty_a += 8; slot_lo += stage16;
-                    if (++stage == p.stages) { stage = 0; phase ^= 1u; full_a = full0; empty_a = empty0; slot_lo = ring_lo0; }
-                }
-            }
-            if (ok) commit(&tmem_full_bar[acc]);
-        }
+    } else if (warp == 1 || warp == kSecondIssuerWarp) {
+        // --------------------------------------------------------- MMA issuers
+        const uint32_t issuer = warp == 1 ? 0u : 1u;
+        if (lane == 0 && pair_rank == 0 && issuer < uint32_t(p.issuers)) {
+            IssuerCtx c;
+            c.smem = smem; c.b_ring = b_ring;
+            c.full_bar = full_bar; c.empty_bar = empty_bar; c.fullA_bar = fullA_bar; c.emptyA_bar = emptyA_bar;
+            c.tmem_full_bar = tmem_full_bar; c.tmem_empty_bar = tmem_empty_bar;
+            c.abort_flag = &abort_flag; c.issue_seq = &issue_seq;
+            c.tmem_base = tmem_base; c.b_bytes = b_bytes; c.step_bytes = step_bytes; c.stage_bytes = stage_bytes;
+            c.first_tile = first_tile; c.tile_stride = tile_stride; c.total_tiles = total_tiles; c.kiters = kiters;
+            if (p.issuers == 2) mma_issuer<kPair, true>(p, c, issuer);
+            else mma_issuer<kPair, false>(p, c, issuer);
         }
         __syncwarp();
     } else {
@@ -588,6 +713,7 @@ struct TileCfg {
     int halo = 0, MT = 1, bw_log2 = 0, bh_log2 = 0, tw = 0, th = 0, tn = 0, half_dq = 0, half_dp = 0;
     int tiles_q = 0, tiles_p = 0, tiles_n = 0, tiles_k = 0, BN = 0;
     int PW = 0, patch_bytes = 0, a_buf_bytes = 0, NA = 0, half_off_bytes = 0, stages = 0, KS = 1;
+    int issuers = 1;    // MMA-issuing threads
     int grp = 0;        // one copy per operand and slot (KS channel blocks of one tap)
     int pair = 0;       // CTA pairs: two image-group tiles share one 256-wide weight tile (see the kernel)
 };
@@ -601,7 +727,9 @@ TileCfg plain_cfg(const TcFpropArgs& a, int cblocks, int sm_count) {
     c.BN = choose_bn(a.Kout, m_tiles, sm_count);
     c.tiles_k = (a.Kout + c.BN - 1) / c.BN;
     // narrow tiles: several k-steps per slot (see the kernel), as long as 4 slots still fit
-    c.pair = env_int("PCL_PAIR", 1) && c.tiles_n >= 2 && sm_count >= 2;
+    // pairs pay where operand traffic or the issue rate of wide MMAs bounds the tile; narrow tiles are bound by
+    // the issuing thread and run as single CTAs with two issuers instead
+    c.pair = env_int("PCL_PAIR", 1) && c.BN >= 128 && c.tiles_n >= 2 && sm_count >= 2;
     const int step_bytes = kABytes + (c.pair ? c.BN * 64 : c.BN * 128);
     c.KS = env_int("PCL_KS", 2);
     const int kiters = a.R * a.S * cblocks;
@@ -632,12 +760,15 @@ TileCfg halo_cfg(const TcFpropArgs& a, int cblocks, int sm_count, int layout) {
     c.BN = choose_bn(a.Kout, m_tiles, sm_count);
     if (2 * c.MT * c.BN > 512) return c;          // two accumulator sets must fit the 512 TMEM columns
     c.tiles_k = (a.Kout + c.BN - 1) / c.BN;
+    c.pair = env_int("PCL_PAIR_HALO", 0) && c.tiles_n >= 2 && sm_count >= 2;      // pairs of images (no gain measured)
+    const int b_bytes = c.pair ? c.BN * 64 : c.BN * 128;
     const int room = kSmemBudget - kEpiStageBytes;
     c.NA = 2;
     c.KS = env_int("PCL_KS_HALO", c.BN <= 64 ? 3 : (c.BN <= 128 ? 2 : 1));
     if (c.KS > a.R * a.S) c.KS = a.R * a.S;
-    while (c.KS > 1 && (room - c.NA * c.a_buf_bytes) / (c.KS * c.BN * 128) < 3) --c.KS;
-    const int slot = c.KS * c.BN * 128;
+    while (c.KS > 1 && (room - c.NA * c.a_buf_bytes) / (c.KS * b_bytes) < 3) --c.KS;
+    c.grp = env_int("PCL_GRP", 1) && c.KS > 1;
+    const int slot = c.KS * b_bytes;
     c.stages = (room - c.NA * c.a_buf_bytes) / slot;
     if (c.stages >= 9 && (room - 3 * c.a_buf_bytes) / slot >= 6) {
         c.NA = 3;
@@ -724,6 +855,9 @@ int launch_tc_fprop(const TcFpropArgs& a, cudaStream_t st) {
     p.tiles_n = cfg.pair ? (cfg.tiles_n + 1) / 2 : cfg.tiles_n;      // pair mode iterates over pairs of image groups
     p.BN = cfg.BN; p.PW = cfg.PW; p.patch_bytes = cfg.patch_bytes; p.a_buf_bytes = cfg.a_buf_bytes; p.NA = cfg.NA;
     p.half_off_bytes = cfg.half_off_bytes; p.stages = cfg.stages; p.KS = cfg.KS; p.grp = cfg.grp;
+    // Two issuing threads only for single-CTA tiles: pair MMAs (cta_group::2) issued from two warps at once
+    // ended in launch failures on B200, so a pair always has one issuer.
+    p.issuers = (!cfg.pair && env_int("PCL_ISSUERS", 2) >= 2) ? 2 : 1;
     const int bw = 1 << p.bw_log2, bh = 1 << p.bh_log2, bn = kTileM / (bw * bh);
     const long m_tiles = long(p.tiles_q) * p.tiles_p * p.tiles_n;
     if (m_tiles * p.tiles_k > 0x7fffffffL) return PCL_ERR_UNSUPPORTED_SHAPE;
@@ -749,7 +883,7 @@ int launch_tc_fprop(const TcFpropArgs& a, cudaStream_t st) {
         const uint32_t box_plain[4] = {kBlockC, uint32_t(bw), uint32_t(bh), uint32_t(bn)};
         const uint32_t box_halo[4] = {kBlockC, uint32_t(p.PW), uint32_t(p.th + a.R - 1), 1};
         int rc;
-        if (cfg.grp) {
+        if (cfg.grp && !cfg.halo) {
             // channel blocks as a fifth dimension (128 bytes apart), so that one box spans KS of them
             const uint64_t dims5[5] = {kBlockC, uint64_t(a.W), uint64_t(a.H), uint64_t(a.N), uint64_t(p.cblocks)};
             const uint64_t strides5[4] = {sw * 4, sh * 4, sn * 4, kBlockC * 4};
@@ -765,7 +899,13 @@ int launch_tc_fprop(const TcFpropArgs& a, cudaStream_t st) {
         const uint64_t strides[2] = {uint64_t(a.Cin) * 4, uint64_t(a.R) * a.S * a.Cin * 4};
         const uint32_t box[3] = {kBlockC, 1, uint32_t(cfg.pair ? p.BN / 2 : p.BN)};
         int rc;
-        if (cfg.grp) {
+        if (cfg.grp && cfg.halo) {
+            // {channel, output map, tap}: a box of KS taps lands as KS weight tiles
+            const uint64_t dims3[3] = {uint64_t(a.Cin), uint64_t(a.Kout), uint64_t(a.R) * a.S};
+            const uint64_t strides3[2] = {uint64_t(a.R) * a.S * a.Cin * 4, uint64_t(a.Cin) * 4};
+            const uint32_t box3[3] = {kBlockC, uint32_t(cfg.pair ? p.BN / 2 : p.BN), uint32_t(p.KS)};
+            rc = make_tmap(&tmB, a.wt, 3, dims3, strides3, box3, false);
+        } else if (cfg.grp) {
             // {channel in block, output map, channel block, tap}: a box of KS channel blocks lands as KS weight tiles
             const uint64_t dims4[4] = {kBlockC, uint64_t(a.Kout), uint64_t(p.cblocks), uint64_t(a.R) * a.S};
             const uint64_t strides4[3] = {uint64_t(a.R) * a.S * a.Cin * 4, kBlockC * 4, uint64_t(a.Cin) * 4};
@@ -777,7 +917,7 @@ int launch_tc_fprop(const TcFpropArgs& a, cudaStream_t st) {
         if (rc != PCL_OK) return rc;
     }
     const long total = m_tiles * p.tiles_k;
-    const size_t smem = (p.halo ? size_t(p.NA) * p.a_buf_bytes + size_t(p.stages) * p.KS * p.BN * 128
+    const size_t smem = (p.halo ? size_t(p.NA) * p.a_buf_bytes + size_t(p.stages) * p.KS * (cfg.pair ? p.BN * 64 : p.BN * 128)
                                 : size_t(p.stages) * p.KS * (kABytes + (cfg.pair ? p.BN * 64 : p.BN * 128))) +
                         kEpiStageBytes + 1024;
     if (cfg.pair) {
