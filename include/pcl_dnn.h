@@ -85,6 +85,18 @@ size_t pcl_fc_workspace_bytes(int N, int C, int K, int pass);
 int pcl_conv_fwd(const pcl_conv_desc* d, const float* x, const float* w, const float* bias,
                  float* y, int act, void* ws, size_t ws_bytes, void* cuda_stream);
 
+/* Forward propagation followed by the 2x2 / stride-2 max pooling that the conv -> ReLU -> pool
+ * blocks of the VGG-A topology (Sec. 5) apply to it:
+ *   y as pcl_conv_fwd();   y_pool[n,p,q,k] = max_{i,j in {0,1}} y[n, 2p+i, 2q+j, k].
+ * On the tensor-core path the maxima are taken in the epilogue while the tile is on chip (max
+ * commutes with adding the bias and with a monotone activation), which saves re-reading y;
+ * other shapes run the pooling kernel after the convolution.  out_h and out_w must be even
+ * (PCL_ERR_UNSUPPORTED_SHAPE otherwise).  y_pool: [N][out_h/2][out_w/2][K] out, 16-byte aligned.
+ * Workspace as pcl_conv_fwd(). */
+int pcl_conv_fwd_pool(const pcl_conv_desc* d, const float* x, const float* w, const float* bias,
+                      float* y, float* y_pool, int act,
+                      void* ws, size_t ws_bytes, void* cuda_stream);
+
 /* Backpropagation (the "Backpropagation" update rule of Sec. 2.1, gather form):
  *   dx[n,h,w,c] = sum over (k,r,s) such that p = (h + pad_h - r)/stride_h and
  *                 q = (w + pad_w - s)/stride_w are integers inside the output

@@ -227,14 +227,17 @@ size_t pcl_fc_workspace_bytes(int N, int C, int K, int pass) {
     return pcl_conv_workspace_bytes(&d, PCL_PASS_BWD_DATA) + pcl_conv_workspace_bytes(&d, PCL_PASS_BWD_WEIGHTS);
 }
 
-int pcl_conv_fwd(const pcl_conv_desc* d, const float* x, const float* w, const float* bias, float* y, int act,
-                 void* ws, size_t ws_bytes, void* cuda_stream) {
+// Forward pass; y_pool != nullptr: also the 2x2 window maxima of y, fused into the tensor-core epilogue where
+// the shape allows it and computed by the pooling kernel otherwise.
+static int conv_fwd_impl(const pcl_conv_desc* d, const float* x, const float* w, const float* bias, float* y,
+                         float* y_pool, int act, void* ws, size_t ws_bytes, void* cuda_stream) {
     int P, Q;
     int rc = check_desc(d, &P, &Q);
     if (rc != PCL_OK) return rc;
     if (!x || !w || !y) return PCL_ERR_BAD_ARG;
     if (act != PCL_ACT_NONE && act != PCL_ACT_RELU && act != PCL_ACT_SIGMOID) return PCL_ERR_BAD_ARG;
-    if (!aligned16(x) || !aligned16(w) || !aligned16(y) || !aligned16(bias)) return PCL_ERR_MISALIGNED;
+    if (!aligned16(x) || !aligned16(w) || !aligned16(y) || !aligned16(bias) || !aligned16(y_pool)) return PCL_ERR_MISALIGNED;
+    if (y_pool && (P % 2 != 0 || Q % 2 != 0)) return PCL_ERR_UNSUPPORTED_SHAPE;
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
     if (few_channel_path_for(*d, PCL_PASS_FWD)) {
         const size_t xs_bytes = staged_x_bytes(*d), need = xs_bytes + staged_w_bytes(*d);
@@ -250,14 +253,31 @@ int pcl_conv_fwd(const pcl_conv_desc* d, const float* x, const float* w, const f
         // the staged layer: 32 "channels" per pixel window (S*4 carry weight, the rest meets zero weights)
         TcFpropArgs a{xs, w4, bias, nullptr, y, d->N, Hp, Q, 32, d->K, d->R, 1, 0, 0, P, Q, act};
         a.in_stride_w = 4; a.in_stride_h = long(Wp) * 4; a.in_stride_n = long(Hp) * Wp * 4;
-        return launch_tc_fprop(a, st);
-    }
-    if (tensor_path_for(*d, PCL_PASS_FWD)) {
+        if (y_pool && tc_fprop_can_pool(a)) { a.pool_out = y_pool; y_pool = nullptr; }
+        rc = launch_tc_fprop(a, st);
+    } else if (tensor_path_for(*d, PCL_PASS_FWD)) {
         TcFpropArgs a{x, w, bias, nullptr, y, d->N, d->H, d->W, d->C, d->K, d->R, d->S, d->pad_h, d->pad_w, P, Q, act};
-        return launch_tc_fprop(a, st);
+        if (y_pool && tc_fprop_can_pool(a)) { a.pool_out = y_pool; y_pool = nullptr; }
+        rc = launch_tc_fprop(a, st);
+    } else if (g_path.load() == PCL_PATH_TENSOR) {
+        return PCL_ERR_UNSUPPORTED_SHAPE;
+    } else {
+        rc = launch_generic_fwd(*d, P, Q, x, w, bias, y, act, st);
     }
-    if (g_path.load() == PCL_PATH_TENSOR) return PCL_ERR_UNSUPPORTED_SHAPE;
-    return launch_generic_fwd(*d, P, Q, x, w, bias, y, act, st);
+    if (rc != PCL_OK) return rc;
+    if (y_pool) return launch_maxpool_fwd(d->N, P, Q, d->K, y, y_pool, st);     // not fused above
+    return PCL_OK;
+}
+
+int pcl_conv_fwd(const pcl_conv_desc* d, const float* x, const float* w, const float* bias, float* y, int act,
+                 void* ws, size_t ws_bytes, void* cuda_stream) {
+    return conv_fwd_impl(d, x, w, bias, y, nullptr, act, ws, ws_bytes, cuda_stream);
+}
+
+int pcl_conv_fwd_pool(const pcl_conv_desc* d, const float* x, const float* w, const float* bias, float* y,
+                      float* y_pool, int act, void* ws, size_t ws_bytes, void* cuda_stream) {
+    if (!y_pool) return PCL_ERR_BAD_ARG;
+    return conv_fwd_impl(d, x, w, bias, y, y_pool, act, ws, ws_bytes, cuda_stream);
 }
 
 int pcl_conv_bwd_data(const pcl_conv_desc* d, const float* dy, const float* w, const float* relu_mask_src, float* dx,

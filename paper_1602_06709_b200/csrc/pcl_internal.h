@@ -68,7 +68,11 @@ struct TcFpropArgs {
     // quarter) writes one row of per-column sums to `colsum_rows` ([tc_fprop_colsum_rows(a)][Kout], fully
     // written when Kout % 4 == 0); the caller adds the rows up in a fixed order.
     float* colsum_rows = nullptr;
+    // Optional fused 2x2 / stride-2 max pooling of the output: pool_out [N][P/2][Q/2][Kout] gets the window maxima
+    // of `out` (after bias and activation).  Needs even P and Q and Kout % 4 == 0 (tc_fprop_can_pool()).
+    float* pool_out = nullptr;
 };
+bool tc_fprop_can_pool(const TcFpropArgs& a);
 bool tc_fprop_eligible(const TcFpropArgs& a);
 long tc_fprop_colsum_rows(const TcFpropArgs& a);
 int launch_tc_fprop(const TcFpropArgs& a, cudaStream_t st);

@@ -64,6 +64,7 @@ struct FpropParams {
     const float* bias;
     const float* mask_src;
     float* out;
+    float* pool_out;            // optional [N][P/2][Q/2][Kout]: 2x2 window maxima of the output
     float* colsum_rows;         // optional [m_tiles * MT * 4][Kout] per-(box, quarter) column sums of the output
     unsigned int* status;       // device status word
 };
@@ -602,6 +603,39 @@ tc_fprop_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                             csum.z += __shfl_xor_sync(live, csum.z, 16); csum.w += __shfl_xor_sync(live, csum.w, 16);
                             if (lane < 8) *reinterpret_cast<float4*>(cs_row + col) = csum;
                         }
+                        if (p.pool_out) {
+                            // Fused 2x2 max pooling.  The warp's 32 rows are 32 consecutive pixels of the box
+                            // (bit 0 of the row = parity of q, bit log2(bw) = parity of p; the box starts at even
+                            // coordinates), so they hold 8 whole windows; lane l takes windows (l >> 3) and
+                            // (l >> 3) + 4 of its 4 columns.  max commutes with adding the bias and with the
+                            // (monotone) activation, so the maximum of the raw accumulators is finished like `o`.
+                            const int lb = p.bw_log2;
+#pragma unroll
+                            for (int half = 0; half < 2; ++half) {
+                                const int wdx = (lane >> 3) + 4 * half;
+                                const int r0 = ((wdx & ((1 << (lb - 1)) - 1)) << 1) | ((wdx >> (lb - 1)) << (lb + 1));
+                                float4 m = make_float4(-INFINITY, -INFINITY, -INFINITY, -INFINITY);
+#pragma unroll
+                                for (int e = 0; e < 4; ++e) {
+                                    const int rr = r0 | (e & 1) | ((e >> 1) << lb);
+                                    const float4 t4 = *reinterpret_cast<const float4*>(stg + rr * 128 + (((lane & 7) ^ (rr & 7)) * 16));
+                                    m.x = fmaxf(m.x, t4.x); m.y = fmaxf(m.y, t4.y); m.z = fmaxf(m.z, t4.z); m.w = fmaxf(m.w, t4.w);
+                                }
+                                m.x += b.x; m.y += b.y; m.z += b.z; m.w += b.w;
+                                if (p.act == PCL_ACT_RELU) {
+                                    m.x = fmaxf(m.x, 0.f); m.y = fmaxf(m.y, 0.f); m.z = fmaxf(m.z, 0.f); m.w = fmaxf(m.w, 0.f);
+                                } else if (p.act == PCL_ACT_SIGMOID) {
+                                    m.x = 1.f / (1.f + __expf(-m.x)); m.y = 1.f / (1.f + __expf(-m.y));
+                                    m.z = 1.f / (1.f + __expf(-m.z)); m.w = 1.f / (1.f + __expf(-m.w));
+                                }
+                                const int wrow = quarter * 32 + r0;       // the window's first pixel inside the box
+                                const int wq = it.qi * p.tw + (wrow & (bw - 1)) + h * p.half_dq;
+                                const int wp = it.pi * p.th + ((wrow >> p.bw_log2) & (bh - 1)) + h * p.half_dp;
+                                const int wn = ni * p.tn + (wrow >> (p.bw_log2 + p.bh_log2));
+                                if (wq < p.Q && wp < p.P && wn < p.N)
+                                    *reinterpret_cast<float4*>(p.pool_out + ((static_cast<size_t>(wn) * (p.P >> 1) + (wp >> 1)) * (p.Q >> 1) + (wq >> 1)) * p.Kout + col) = m;
+                            }
+                        }
                     }
                     __syncwarp();
                 }
@@ -650,11 +684,12 @@ tc_fprop_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
 
 // Pick the 128-pixel box bw x bh x bn (powers of two) that wastes the least
 // work on ragged edges; ties go to the widest box.
-void choose_box(int P, int Q, int N, int* bw_log2, int* bh_log2) {
+// pool: the box must hold whole 2x2 windows inside each 32-pixel quarter (2 <= bw <= 16, bh >= 2).
+void choose_box(int P, int Q, int N, bool pool, int* bw_log2, int* bh_log2) {
     double best = 1e300;
-    int best_w = 0, best_h = 0;
-    for (int lw = 7; lw >= 0; --lw)
-        for (int lh = 7 - lw; lh >= 0; --lh) {
+    int best_w = pool ? 1 : 0, best_h = pool ? 1 : 0;
+    for (int lw = pool ? 4 : 7; lw >= (pool ? 1 : 0); --lw)
+        for (int lh = 7 - lw; lh >= (pool ? 1 : 0); --lh) {
             const long bw = 1L << lw, bh = 1L << lh, bn = 128 / (bw * bh);
             const double covered = double((Q + bw - 1) / bw * bw) * double((P + bh - 1) / bh * bh) *
                                    double((N + bn - 1) / bn * bn);
@@ -692,6 +727,10 @@ int g_sm_count = 0;
 
 }  // namespace
 
+bool tc_fprop_can_pool(const TcFpropArgs& a) {
+    return a.P % 2 == 0 && a.Q % 2 == 0 && a.P >= 2 && a.Q >= 2 && a.Kout % 4 == 0 && a.mask_src == nullptr;
+}
+
 bool tc_fprop_eligible(const TcFpropArgs& a) {
     if (a.Cin % 4 != 0) return false;                       // TMA strides are multiples of 16 bytes
     if ((reinterpret_cast<uintptr_t>(a.in) | reinterpret_cast<uintptr_t>(a.wt)) & 15) return false;
@@ -720,7 +759,7 @@ struct TileCfg {
 
 TileCfg plain_cfg(const TcFpropArgs& a, int cblocks, int sm_count) {
     TileCfg c;
-    choose_box(a.P, a.Q, a.N, &c.bw_log2, &c.bh_log2);
+    choose_box(a.P, a.Q, a.N, a.pool_out != nullptr, &c.bw_log2, &c.bh_log2);
     c.tw = 1 << c.bw_log2; c.th = 1 << c.bh_log2; c.tn = kTileM / (c.tw * c.th);
     c.tiles_q = (a.Q + c.tw - 1) / c.tw; c.tiles_p = (a.P + c.th - 1) / c.th; c.tiles_n = (a.N + c.tn - 1) / c.tn;
     const long m_tiles = long(c.tiles_q) * c.tiles_p * c.tiles_n;
@@ -867,6 +906,8 @@ int launch_tc_fprop(const TcFpropArgs& a, cudaStream_t st) {
     p.tmem_cols = 32;
     while (p.tmem_cols < 2 * p.MT * p.BN) p.tmem_cols *= 2;
     p.bias = a.bias; p.mask_src = a.mask_src; p.out = a.out;
+    if (a.pool_out && !tc_fprop_can_pool(a)) return PCL_ERR_UNSUPPORTED_SHAPE;
+    p.pool_out = a.pool_out;
     p.colsum_rows = (a.Kout % 4 == 0) ? a.colsum_rows : nullptr;
     if (a.colsum_rows && !p.colsum_rows) return PCL_ERR_UNSUPPORTED_SHAPE;
     p.status = device_status_ptr();

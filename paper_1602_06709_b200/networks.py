@@ -138,9 +138,11 @@ class VggA:
     # -- one training step --------------------------------------------------
     def forward(self):
         for i, L in enumerate(self.convs):
-            B.conv_fwd(L.desc, self.layer_input(i), self.conv_w(i), self.conv_b(i), self.y[i], B.ACT_RELU, self.ws)
-            if L.pool:
-                B.maxpool2x2_fwd(self.N, L.H, L.W, L.K, self.y[i], self.pooled[i])
+            if L.pool:      # conv -> ReLU -> 2x2 pool, the maxima taken in the convolution's epilogue
+                B.conv_fwd_pool(L.desc, self.layer_input(i), self.conv_w(i), self.conv_b(i), self.y[i], self.pooled[i],
+                                B.ACT_RELU, self.ws)
+            else:
+                B.conv_fwd(L.desc, self.layer_input(i), self.conv_w(i), self.conv_b(i), self.y[i], B.ACT_RELU, self.ws)
         a = self.pooled[-1].view(self.N, self.flat)
         for j, (C, K) in enumerate(self.fcs):
             act = B.ACT_RELU if j + 1 < len(self.fcs) else B.ACT_NONE

@@ -174,3 +174,46 @@ def test_conv_bwd_data_with_fused_column_sums(shape, tiling, monkeypatch):
     cs2 = torch.empty_like(cs)
     B.conv_bwd_data_colsum(d, G.dev(dy), G.dev(w), G.dev(x), dx, cs2, ws)
     assert torch.equal(cs, cs2)
+
+
+POOL_FUSED_SHAPES = [
+    # N, C, K, H, W: even outputs; several image groups; ragged in q/p; C < 4 (few-channel path); halo-eligible 16x16 fits
+    (3, 32, 64, 12, 20), (4, 64, 96, 28, 28), (2, 3, 16, 20, 36), (2, 64, 128, 32, 48), (5, 24, 40, 6, 10), (2, 7, 9, 10, 12),
+]
+
+
+@pytest.mark.parametrize("tiling", ["auto", "plain", "halo0", "halo1", "halo2"])
+@pytest.mark.parametrize("shape", POOL_FUSED_SHAPES)
+def test_conv_fwd_with_fused_maxpool(shape, tiling, monkeypatch):
+    """conv -> ReLU -> 2x2 max pool in one call: y must match the oracle's convolution, and the pooled
+    tensor must be bit-for-bit the 2x2 maxima of the y the same call wrote (the epilogue takes the
+    maximum of the raw accumulators, which commutes exactly with the bias add and the ReLU)."""
+    import gpu_helpers as G
+    from oracle import ConvShape
+    from paper_1602_06709_b200 import binding as B
+    if tiling != "auto":
+        monkeypatch.setenv("PCL_TILING", tiling)
+    N, C, K, H, W = shape
+    s = ConvShape(N=N, C=C, K=K, H=H, W=W, R=3, S=3, pad_h=1, pad_w=1)
+    x, w, _, bias = G.make_inputs(s, f"fwdpool{C}_{K}")
+    d = G.shape_to_desc(s)
+    for act, oact in ((B.ACT_RELU, oracle.ACT_RELU), (B.ACT_NONE, oracle.ACT_NONE)):
+        y = torch.full((N, H, W, K), float("nan"), device="cuda")
+        yp = torch.full((N, H // 2, W // 2, K), float("nan"), device="cuda")
+        ws = G.workspace(B.conv_workspace_bytes(d, B.PASS_FWD))
+        B.conv_fwd_pool(d, G.dev(x), G.dev(w), G.dev(bias), y, yp, act, ws)
+        B.check_device_status()
+        G.assert_parity(y.cpu().numpy(), oracle.conv_fwd(s, x, w, bias, oact), "y")
+        assert np.array_equal(yp.cpu().numpy(), oracle.maxpool2x2_fwd(y.cpu().numpy().astype(np.float64)).astype(np.float32))
+
+
+def test_conv_fwd_pool_rejects_odd_output():
+    import gpu_helpers as G
+    from oracle import ConvShape
+    from paper_1602_06709_b200 import binding as B
+    s = ConvShape(N=1, C=8, K=8, H=7, W=8, R=3, S=3, pad_h=1, pad_w=1)
+    d = G.shape_to_desc(s)
+    x = torch.zeros(1, 7, 8, 8, device="cuda"); w = torch.zeros(8, 3, 3, 8, device="cuda")
+    y = torch.zeros(1, 7, 8, 8, device="cuda"); yp = torch.zeros(1, 3, 4, 8, device="cuda")
+    with pytest.raises(B.PclError):
+        B.conv_fwd_pool(d, x, w, None, y, yp, B.ACT_RELU, None)
