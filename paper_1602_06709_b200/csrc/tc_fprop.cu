@@ -294,7 +294,9 @@ __device__ __noinline__ void mma_issuer(const FpropParams& p, const IssuerCtx& c
 // kPair: two CTAs of a cluster (ranks 0 and 1) compute two M tiles (consecutive image groups) against the
 // same BN = 256 weight tile with M = 256 MMAs issued by rank 0; each CTA loads its own A tile and only half
 // of the weight rows, which cuts the shared-memory fill traffic per MMA by a third (plain tiling only).
-template <bool kPair>
+// kPool: the epilogue also writes the 2x2 window maxima (kept out of the other instantiations, whose epilogue it
+// would cost registers).
+template <bool kPair, bool kPool>
 __global__ void __launch_bounds__(kThreads, 1)
 tc_fprop_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                 const __grid_constant__ FpropParams p) {
@@ -603,7 +605,7 @@ tc_fprop_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                             csum.z += __shfl_xor_sync(live, csum.z, 16); csum.w += __shfl_xor_sync(live, csum.w, 16);
                             if (lane < 8) *reinterpret_cast<float4*>(cs_row + col) = csum;
                         }
-                        if (p.pool_out) {
+                        if (kPool) {
                             // Fused 2x2 max pooling.  The warp's 32 rows are 32 consecutive pixels of the box
                             // (bit 0 of the row = parity of q, bit log2(bw) = parity of p; the box starts at even
                             // coordinates), so they hold 8 whole windows; lane l takes windows (l >> 3) and
@@ -877,9 +879,13 @@ int launch_tc_fprop(const TcFpropArgs& a, cudaStream_t st) {
     static bool attr_set = false;
     if (!attr_set) {
         if (ensure_device_setup() != PCL_OK) return PCL_ERR_CUDA;
-        if (cudaFuncSetAttribute(tc_fprop_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        if (cudaFuncSetAttribute(tc_fprop_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  kSmemBudget + 1024) != cudaSuccess ||
-            cudaFuncSetAttribute(tc_fprop_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+            cudaFuncSetAttribute(tc_fprop_kernel<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 kSmemBudget + 1024) != cudaSuccess ||
+            cudaFuncSetAttribute(tc_fprop_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 kSmemBudget + 1024) != cudaSuccess ||
+            cudaFuncSetAttribute(tc_fprop_kernel<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  kSmemBudget + 1024) != cudaSuccess)
             return PCL_ERR_CUDA;
         attr_set = true;
@@ -896,7 +902,11 @@ int launch_tc_fprop(const TcFpropArgs& a, cudaStream_t st) {
     p.half_off_bytes = cfg.half_off_bytes; p.stages = cfg.stages; p.KS = cfg.KS; p.grp = cfg.grp;
     // Two issuing threads only for single-CTA tiles: pair MMAs (cta_group::2) issued from two warps at once
     // ended in launch failures on B200, so a pair always has one issuer.
-    p.issuers = (!cfg.pair && env_int("PCL_ISSUERS", 2) >= 2) ? 2 : 1;
+    // They pay where a tile has many slots; the hand-over between the threads costs more than it hides on
+    // tiles of a few k-steps (the few-channel first layer: 3).
+    const int slots_per_tile = cfg.halo ? p.cblocks * ((a.R * a.S + cfg.KS - 1) / cfg.KS)
+                                        : (a.R * a.S * p.cblocks + cfg.KS - 1) / cfg.KS;
+    p.issuers = (!cfg.pair && slots_per_tile >= 8 && env_int("PCL_ISSUERS", 2) >= 2) ? 2 : 1;
     const int bw = 1 << p.bw_log2, bh = 1 << p.bh_log2, bn = kTileM / (bw * bh);
     const long m_tiles = long(p.tiles_q) * p.tiles_p * p.tiles_n;
     if (m_tiles * p.tiles_k > 0x7fffffffL) return PCL_ERR_UNSUPPORTED_SHAPE;
@@ -974,7 +984,7 @@ int launch_tc_fprop(const TcFpropArgs& a, cudaStream_t st) {
         if (cached_smem != smem) {
             lc.gridDim = dim3(unsigned(g_sm_count / 2 * 2));
             int n = 0;
-            if (cudaOccupancyMaxActiveClusters(&n, tc_fprop_kernel<true>, &lc) != cudaSuccess || n <= 0) return PCL_ERR_CUDA;
+            if (cudaOccupancyMaxActiveClusters(&n, tc_fprop_kernel<true, false>, &lc) != cudaSuccess || n <= 0) return PCL_ERR_CUDA;
             cached_clusters = n < g_sm_count / 2 ? n : g_sm_count / 2;
             cached_smem = smem;
         }
@@ -982,11 +992,14 @@ int launch_tc_fprop(const TcFpropArgs& a, cudaStream_t st) {
         long nclus = pair_tiles < cached_clusters ? pair_tiles : cached_clusters;
         lc.gridDim = dim3(unsigned(2 * nclus));
         LaunchScope scope(KID_TC_FPROP, 2.0 * a.N * a.P * a.Q * double(a.Kout) * a.Cin * a.R * a.S, st);
-        if (cudaLaunchKernelEx(&lc, tc_fprop_kernel<true>, tmA, tmB, p) != cudaSuccess) return PCL_ERR_CUDA;
+        const cudaError_t le = p.pool_out ? cudaLaunchKernelEx(&lc, tc_fprop_kernel<true, true>, tmA, tmB, p)
+                                          : cudaLaunchKernelEx(&lc, tc_fprop_kernel<true, false>, tmA, tmB, p);
+        if (le != cudaSuccess) return PCL_ERR_CUDA;
     } else {
         const int grid = int(total < g_sm_count ? total : g_sm_count);
         LaunchScope scope(KID_TC_FPROP, 2.0 * a.N * a.P * a.Q * double(a.Kout) * a.Cin * a.R * a.S, st);
-        tc_fprop_kernel<false><<<grid, kThreads, smem, st>>>(tmA, tmB, p);
+        if (p.pool_out) tc_fprop_kernel<false, true><<<grid, kThreads, smem, st>>>(tmA, tmB, p);
+        else tc_fprop_kernel<false, false><<<grid, kThreads, smem, st>>>(tmA, tmB, p);
     }
     return cudaGetLastError() == cudaSuccess ? PCL_OK : PCL_ERR_CUDA;
 }
