@@ -141,7 +141,8 @@ class VggWorkload:
         self.net.step()
 
     def e2e_step(self):
-        return self.net.step_from_host(self.x_host, self.lab_host)
+        # the next minibatch (here: the same pinned buffers) is copied while this step computes
+        return self.net.step_from_host(self.x_host, self.lab_host, self.x_host, self.lab_host)
 
     def describe(self):
         return dict(minibatch=self.N, conv_flop_per_step=self.conv_flops, fc_flop_per_step=self.fc_flops,
@@ -218,7 +219,8 @@ class DnnWorkload:
         self.net.step()
 
     def e2e_step(self):
-        return self.net.step_from_host(self.x_host, self.lab_host)
+        # the next minibatch (here: the same pinned buffers) is copied while this step computes
+        return self.net.step_from_host(self.x_host, self.lab_host, self.x_host, self.lab_host)
 
     def describe(self):
         return dict(minibatch=self.N, fc_flop_per_step=3 * sum(self.net.fc_flops_fwd), params=self.net.store.n_real())

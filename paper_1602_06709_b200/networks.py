@@ -61,8 +61,42 @@ class _ConvLayer:
     pool: bool
     desc: object = None
 
+class _HostFeed:
+    """Host-side input feed shared by the step drivers: the minibatch of a step is copied from pinned host
+    memory, and the copy of the NEXT minibatch can run on a second stream while this step computes (two
+    device input buffers that swap).  Buffers and call order only; no arithmetic of the method."""
 
-class VggA:
+    def _feed_init(self):
+        self._alt_x = torch.empty_like(self.x)
+        self._alt_labels = torch.empty_like(self.labels)
+        self._copy_stream = torch.cuda.Stream()
+        self._staged = None          # event: the alternate buffers hold the next minibatch
+
+    def step_from_host(self, x_host, labels_host, next_x_host=None, next_labels_host=None) -> float:
+        """The call a user makes: pinned host minibatch in, loss out.  If the previous call was given this
+        minibatch as its `next_*` arguments, its copy has already been issued and only has to be waited for;
+        `next_*` of this call start the copy of the following minibatch before the step is launched."""
+        cur = torch.cuda.current_stream()
+        if self._staged is not None:
+            cur.wait_event(self._staged)
+            self.x, self._alt_x = self._alt_x, self.x
+            self.labels, self._alt_labels = self._alt_labels, self.labels
+            self._staged = None
+        else:
+            self.x.copy_(x_host, non_blocking=True)
+            self.labels.copy_(labels_host, non_blocking=True)
+        if next_x_host is not None:
+            # the alternate buffers were last read by the previous step, which has finished (its loss was read)
+            with torch.cuda.stream(self._copy_stream):
+                self._alt_x.copy_(next_x_host, non_blocking=True)
+                self._alt_labels.copy_(next_labels_host, non_blocking=True)
+                self._staged = torch.cuda.Event()
+                self._staged.record(self._copy_stream)
+        self.step()
+        return float(self.loss.cpu().item())
+
+
+class VggA(_HostFeed):
     """VGG configuration A: eight 3x3 pad-1 convolutions (64,128,256,256,512,512,
     512,512) each followed by ReLU, 2x2 max-pool after conv 1,2,4,6,8, then
     FC 25088-4096-4096-1000 and softmax cross-entropy."""
@@ -107,6 +141,7 @@ class VggA:
         self.fc_out = [torch.empty(N, K, device=dev) for _, K in fc]
         self.fc_dout = [torch.empty(N, K, device=dev) for _, K in fc]
         self.labels = torch.zeros(N, dtype=torch.int32, device=dev)
+        self._feed_init()
         self.loss = torch.zeros(1, device=dev)
         ws = 0
         for L in self.convs:
@@ -183,15 +218,9 @@ class VggA:
         self.backward()
         self.update()
 
-    def step_from_host(self, x_host: torch.Tensor, labels_host: torch.Tensor) -> float:
-        """The call a user makes: pinned host minibatch in, loss out."""
-        self.x.copy_(x_host, non_blocking=True)
-        self.labels.copy_(labels_host, non_blocking=True)
-        self.step()
-        return float(self.loss.cpu().item())
 
 
-class Dnn:
+class Dnn(_HostFeed):
     """Fully-connected DNN: dims[0] inputs, sigmoid hidden layers, linear output
     layer with softmax cross-entropy (the 7-layer ASR network shape of Sec. 5.4)."""
 
@@ -211,6 +240,7 @@ class Dnn:
         self.out = [torch.empty(N, K, device=dev) for _, K in self.layers]
         self.dout = [torch.empty(N, K, device=dev) for _, K in self.layers]
         self.labels = torch.zeros(N, dtype=torch.int32, device=dev)
+        self._feed_init()
         self.loss = torch.zeros(1, device=dev)
         ws = max(B.fc_workspace_bytes(N, C, K, B.PASS_BWD_DATA) for C, K in self.layers)
         self.ws = torch.empty(max(ws, 256), dtype=torch.uint8, device=dev)
@@ -247,8 +277,3 @@ class Dnn:
         self.backward()
         self.update()
 
-    def step_from_host(self, x_host, labels_host) -> float:
-        self.x.copy_(x_host, non_blocking=True)
-        self.labels.copy_(labels_host, non_blocking=True)
-        self.step()
-        return float(self.loss.cpu().item())
