@@ -114,6 +114,14 @@ namespace {
 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
 
+// Backward-data on the tensor-core path reads the KRSC weights in place (as an MN-major operand) when the layer's
+// input-map count is a multiple of 32; otherwise it goes through a flipped, transposed copy in the workspace.
+// PCL_WEIGHTS_IN_PLACE=0 forces the copy (test hook).
+bool weights_read_in_place(const pcl_conv_desc& d) {
+    const char* v = getenv("PCL_WEIGHTS_IN_PLACE");
+    return d.C % 32 == 0 && !(v && v[0] == '0');
+}
+
 int check_desc(const pcl_conv_desc* d, int* P, int* Q) {
     if (!d) return PCL_ERR_BAD_ARG;
     if (d->N <= 0 || d->C <= 0 || d->K <= 0 || d->H <= 0 || d->W <= 0 || d->R <= 0 || d->S <= 0 || d->stride_h <= 0 ||
@@ -292,12 +300,18 @@ int pcl_conv_bwd_data(const pcl_conv_desc* d, const float* dy, const float* w, c
         const size_t need = dw_bytes(*d);
         if (!ws || ws_bytes < need) return PCL_ERR_WORKSPACE;
         if (reinterpret_cast<uintptr_t>(ws) & 255) return PCL_ERR_MISALIGNED;
-        float* wt_t = static_cast<float*>(ws);
-        rc = launch_transpose_flip(w, wt_t, d->K, d->R, d->S, d->C, st);
-        if (rc != PCL_OK) return rc;
         // dx = "forward" convolution of dy with the flipped, transposed weights, pad' = R-1-pad
-        TcFpropArgs a{dy, wt_t, nullptr, relu_mask_src, dx, d->N, P, Q, d->K, d->C, d->R, d->S,
+        TcFpropArgs a{dy, w, nullptr, relu_mask_src, dx, d->N, P, Q, d->K, d->C, d->R, d->S,
                       d->R - 1 - d->pad_h, d->S - 1 - d->pad_w, d->H, d->W, PCL_ACT_NONE};
+        if (weights_read_in_place(*d)) {
+            // the kernel reads w itself as an MN-major operand (taps flipped by index): no transposed copy
+            a.wt_mn_major = 1; a.flip_taps = 1;
+        } else {
+            float* wt_t = static_cast<float*>(ws);
+            rc = launch_transpose_flip(w, wt_t, d->K, d->R, d->S, d->C, st);
+            if (rc != PCL_OK) return rc;
+            a.wt = wt_t;
+        }
         return launch_tc_fprop(a, st);
     }
     if (g_path.load() == PCL_PATH_TENSOR) return PCL_ERR_UNSUPPORTED_SHAPE;
@@ -312,10 +326,13 @@ size_t colsum_stage_bytes(long rows, int cols) {
     const int cs = colsum_splits(size_t(rows));
     return align_up(size_t(rows) * cols * 4, 256) + (cs > 1 ? align_up(size_t(cs) * cols * 4, 256) : 0);
 }
-TcFpropArgs bwd_data_args(const pcl_conv_desc& d, int P, int Q, const float* dy, const float* wt_t,
+// `w` is the layer's own KRSC tensor when the kernel can read it in place, else the caller puts the transposed copy in.
+TcFpropArgs bwd_data_args(const pcl_conv_desc& d, int P, int Q, const float* dy, const float* w,
                           const float* mask, float* dx) {
-    return TcFpropArgs{dy, wt_t, nullptr, mask, dx, d.N, P, Q, d.K, d.C, d.R, d.S,
-                       d.R - 1 - d.pad_h, d.S - 1 - d.pad_w, d.H, d.W, PCL_ACT_NONE};
+    TcFpropArgs a{dy, w, nullptr, mask, dx, d.N, P, Q, d.K, d.C, d.R, d.S,
+                  d.R - 1 - d.pad_h, d.S - 1 - d.pad_w, d.H, d.W, PCL_ACT_NONE};
+    if (weights_read_in_place(d)) { a.wt_mn_major = 1; a.flip_taps = 1; }
+    return a;
 }
 }  // namespace
 
@@ -351,10 +368,13 @@ int pcl_conv_bwd_data_colsum(const pcl_conv_desc* d, const float* dy, const floa
     if (tensor_path_for(*d, PCL_PASS_BWD_DATA) && d->C % 4 == 0)
         rows = tc_fprop_colsum_rows(bwd_data_args(*d, P, Q, nullptr, nullptr, nullptr, nullptr));
     if (rows > 0) {
-        float* wt_t = static_cast<float*>(ws);
-        rc = launch_transpose_flip(w, wt_t, d->K, d->R, d->S, d->C, st);
-        if (rc != PCL_OK) return rc;
-        TcFpropArgs a = bwd_data_args(*d, P, Q, dy, wt_t, relu_mask_src, dx);
+        TcFpropArgs a = bwd_data_args(*d, P, Q, dy, w, relu_mask_src, dx);
+        if (!a.wt_mn_major) {
+            float* wt_t = static_cast<float*>(ws);
+            rc = launch_transpose_flip(w, wt_t, d->K, d->R, d->S, d->C, st);
+            if (rc != PCL_OK) return rc;
+            a.wt = wt_t;
+        }
         float* sum_rows = reinterpret_cast<float*>(extra);
         a.colsum_rows = sum_rows;
         // rows the chosen tiling does not write must not contribute: the sizing took the largest tiling

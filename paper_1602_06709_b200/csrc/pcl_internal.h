@@ -71,6 +71,11 @@ struct TcFpropArgs {
     // Optional fused 2x2 / stride-2 max pooling of the output: pool_out [N][P/2][Q/2][Kout] gets the window maxima
     // of `out` (after bias and activation).  Needs even P and Q and Kout % 4 == 0 (tc_fprop_can_pool()).
     float* pool_out = nullptr;
+    // wt_mn_major != 0: `wt` is laid out [Cin][R*S][Kout] (output maps innermost), i.e. a layer's own KRSC weights
+    // seen from its backward-data pass (reduction over the layer's K, columns = the layer's C): the kernel then
+    // reads B as an MN-major operand and no transposed copy is needed.  Needs Kout % 32 == 0.
+    // flip_taps != 0: tap t of the loop reads tap R*S-1-t of `wt` (the spatial flip of backward-data).
+    int wt_mn_major = 0, flip_taps = 0;
 };
 bool tc_fprop_can_pool(const TcFpropArgs& a);
 bool tc_fprop_eligible(const TcFpropArgs& a);

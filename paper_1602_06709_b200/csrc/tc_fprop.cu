@@ -48,6 +48,9 @@ struct FpropParams {
     int act;
     int stages;
     int KS;                     // k-steps (plain: {A,B} pairs; halo: weight tiles of consecutive taps) per pipeline slot
+    int bmn;                    // B (weights) is MN-major: laid out [Cin][R*S][Kout], read through {32 maps, reduction rows,
+                                // tap, 32-map group} boxes with the 32-byte-atom swizzle (backward-data without a transposed copy)
+    int flip;                   // tap t reads tap R*S-1-t of the weights
     int issuers;                // MMA-issuing threads (1 or 2; see the kernel)
     int grp;                    // plain tiling: a slot's KS k-steps are KS consecutive channel blocks of one tap, fetched by
                                 // ONE copy of A and one of B (slot layout: KS A tiles, then KS B tiles)
@@ -130,11 +133,11 @@ struct IssuerCtx {
 template <bool kPair, int kTaps, int kMT>
 __device__ __forceinline__ void halo_taps(uint32_t d_tmem, uint32_t BN, uint32_t& a_lo, uint32_t b_lo, int& s, int S,
                                           uint32_t row16, uint32_t half_off16, uint32_t b16, uint32_t a_hi,
-                                          uint32_t b_hi, uint32_t idesc, uint32_t& accum) {
+                                          uint32_t b_hi, uint32_t idesc, uint32_t& accum, uint32_t bks) {
 #pragma unroll
     for (int j = 0; j < kTaps; ++j) {
-        umma_kstep_tf32<kPair, 2, 2>(d_tmem, a_lo, b_lo, a_hi, b_hi, idesc, accum);
-        if (kMT == 2) umma_kstep_tf32<kPair, 2, 2>(d_tmem + BN, a_lo + half_off16, b_lo, a_hi, b_hi, idesc, accum);
+        umma_kstep_tf32_bs<kPair>(d_tmem, a_lo, b_lo, a_hi, b_hi, idesc, accum, bks);
+        if (kMT == 2) umma_kstep_tf32_bs<kPair>(d_tmem + BN, a_lo + half_off16, b_lo, a_hi, b_hi, idesc, accum, bks);
         accum = 1;
         b_lo += b16;
         const bool wrap = ++s == S;     // the tap (r, s): next pixel of the patch, or the start of the next patch row
@@ -167,17 +170,27 @@ __device__ __noinline__ void mma_issuer(const FpropParams& p, const IssuerCtx& c
     const uint32_t tmem_base = c.tmem_base, b16 = c.b_bytes >> 4;
     const int first_tile = c.first_tile, tile_stride = c.tile_stride, total_tiles = c.total_tiles, kiters = c.kiters;
 
-    const uint32_t idesc = make_idesc_tf32(BN, false, false, kPair ? 256u : 128u);
+    const int bmn = p.bmn;
+    const uint32_t idesc = make_idesc_tf32(BN, false, bmn != 0, kPair ? 256u : 128u);
+    const uint32_t bks = bmn ? 64u : 2u;         // k-block stride of B inside a k-step (16-byte units)
     // Descriptors differ only in the 14-bit address field (address >> 4) of their low word: the loops keep low
     // words in registers and advance them by addition.
-    const uint64_t b_desc0 = make_smem_desc(smem_u32(halo ? c.b_ring : smem), 16, 1024, kSwizzle128B);
-    const uint32_t b_hi = uint32_t(b_desc0 >> 32), ring_lo0 = uint32_t(b_desc0);
+    // The ring descriptor is B's in the haloed tiling (the ring holds weight tiles only) and A's in the plain one
+    // (B's low word is then A's plus an offset that also carries the difference of the leading-offset fields).
+    // MN-major B: 32-map groups are `b_group` bytes apart, 4-row reduction groups 512.
+    const uint32_t b_group = (!halo && grp) ? KS * 4096u : 4096u;
+    const uint64_t k_desc0 = make_smem_desc(smem_u32(halo ? c.b_ring : smem), 16, 1024, kSwizzle128B);
+    const uint64_t m_desc0 = make_smem_desc(smem_u32(halo ? c.b_ring : smem), b_group, 512, kSwizzle128B_Atom32B);
+    const uint32_t a_hi_plain = uint32_t(k_desc0 >> 32);
+    const uint32_t b_hi = uint32_t((bmn ? m_desc0 : k_desc0) >> 32);
+    const uint32_t ring_lo0 = uint32_t((halo && bmn) ? m_desc0 : k_desc0);
+    const uint32_t b_lbo_delta = bmn ? uint32_t(m_desc0) - uint32_t(k_desc0) : 0u;
     const uint32_t full0 = smem_u32(&c.full_bar[0]), empty0 = smem_u32(&c.empty_bar[0]);
     const uint32_t stage16 = c.stage_bytes >> 4, step16 = c.step_bytes >> 4;
     // where k-step j of a slot finds its operands (16-byte units from the slot start)
     const uint32_t a_step16 = grp ? (kABytes >> 4) : step16;
-    const uint32_t b_off16 = grp ? KS * (kABytes >> 4) : (kABytes >> 4);
-    const uint32_t b_step16 = grp ? b16 : step16;
+    const uint32_t b_off16 = (grp ? KS * (kABytes >> 4) : (kABytes >> 4)) + b_lbo_delta;
+    const uint32_t b_step16 = grp ? (bmn ? 256u : b16) : step16;
 
     uint32_t full_a = full0, empty_a = empty0, slot_lo = ring_lo0;     // ring position
     int stage = 0;
@@ -226,20 +239,20 @@ __device__ __noinline__ void mma_issuer(const FpropParams& p, const IssuerCtx& c
                     if (mine) {
                         PCL_SLOT_ACQUIRE()
                         if (MT == 2) {
-                            if (nst == 3) halo_taps<kPair, 3, 2>(d_tmem, BN, a_lo, slot_lo, s, S, row16, half_off16, b16, a_hi, b_hi, idesc, accum);
-                            else if (nst == 2) halo_taps<kPair, 2, 2>(d_tmem, BN, a_lo, slot_lo, s, S, row16, half_off16, b16, a_hi, b_hi, idesc, accum);
+                            if (nst == 3) halo_taps<kPair, 3, 2>(d_tmem, BN, a_lo, slot_lo, s, S, row16, half_off16, b16, a_hi, b_hi, idesc, accum, bks);
+                            else if (nst == 2) halo_taps<kPair, 2, 2>(d_tmem, BN, a_lo, slot_lo, s, S, row16, half_off16, b16, a_hi, b_hi, idesc, accum, bks);
                             else {
                                 uint32_t b_lo = slot_lo;
                                 for (int j = 0; j < nst; ++j, b_lo += b16)
-                                    halo_taps<kPair, 1, 2>(d_tmem, BN, a_lo, b_lo, s, S, row16, half_off16, b16, a_hi, b_hi, idesc, accum);
+                                    halo_taps<kPair, 1, 2>(d_tmem, BN, a_lo, b_lo, s, S, row16, half_off16, b16, a_hi, b_hi, idesc, accum, bks);
                             }
                         } else {
-                            if (nst == 3) halo_taps<kPair, 3, 1>(d_tmem, BN, a_lo, slot_lo, s, S, row16, half_off16, b16, a_hi, b_hi, idesc, accum);
-                            else if (nst == 2) halo_taps<kPair, 2, 1>(d_tmem, BN, a_lo, slot_lo, s, S, row16, half_off16, b16, a_hi, b_hi, idesc, accum);
+                            if (nst == 3) halo_taps<kPair, 3, 1>(d_tmem, BN, a_lo, slot_lo, s, S, row16, half_off16, b16, a_hi, b_hi, idesc, accum, bks);
+                            else if (nst == 2) halo_taps<kPair, 2, 1>(d_tmem, BN, a_lo, slot_lo, s, S, row16, half_off16, b16, a_hi, b_hi, idesc, accum, bks);
                             else {
                                 uint32_t b_lo = slot_lo;
                                 for (int j = 0; j < nst; ++j, b_lo += b16)
-                                    halo_taps<kPair, 1, 1>(d_tmem, BN, a_lo, b_lo, s, S, row16, half_off16, b16, a_hi, b_hi, idesc, accum);
+                                    halo_taps<kPair, 1, 1>(d_tmem, BN, a_lo, b_lo, s, S, row16, half_off16, b16, a_hi, b_hi, idesc, accum, bks);
                             }
                         }
                         PCL_SLOT_RELEASE()
@@ -261,8 +274,8 @@ __device__ __noinline__ void mma_issuer(const FpropParams& p, const IssuerCtx& c
                 PCL_SLOT_BEGIN()
                 if (mine) {
                     PCL_SLOT_ACQUIRE()
-                    umma_kstep_tf32<kPair, 2, 2>(d_tmem, slot_lo, slot_lo + b_off16, b_hi, b_hi, idesc, accum);
-                    umma_kstep_tf32<kPair, 2, 2>(d_tmem, slot_lo + a_step16, slot_lo + b_off16 + b_step16, b_hi, b_hi, idesc, 1);
+                    umma_kstep_tf32_bs<kPair>(d_tmem, slot_lo, slot_lo + b_off16, a_hi_plain, b_hi, idesc, accum, bks);
+                    umma_kstep_tf32_bs<kPair>(d_tmem, slot_lo + a_step16, slot_lo + b_off16 + b_step16, a_hi_plain, b_hi, idesc, 1, bks);
                     PCL_SLOT_RELEASE()
                 }
                 PCL_SLOT_END()
@@ -275,7 +288,7 @@ __device__ __noinline__ void mma_issuer(const FpropParams& p, const IssuerCtx& c
                     PCL_SLOT_ACQUIRE()
                     uint32_t a_lo = slot_lo, b_lo = slot_lo + b_off16;
                     for (int j = 0; j < nst; ++j, a_lo += a_step16, b_lo += b_step16) {
-                        umma_kstep_tf32<kPair, 2, 2>(d_tmem, a_lo, b_lo, b_hi, b_hi, idesc, accum);
+                        umma_kstep_tf32_bs<kPair>(d_tmem, a_lo, b_lo, a_hi_plain, b_hi, idesc, accum, bks);
                         accum = 1;
                     }
                     PCL_SLOT_RELEASE()
@@ -419,7 +432,8 @@ tc_fprop_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                             } else {
                                 uint32_t dst = slot_a;
                                 for (int j = 0; j < nst; ++j, dst += b_bytes)
-                                    tma_load_3d_addr<kPair>(dst, &tmB, full_dst, c0, tap + j, kcol);
+                                    if (p.bmn) tma_load_4d_addr<kPair>(dst, &tmB, full_dst, 0, c0, p.flip ? taps - 1 - (tap + j) : tap + j, kcol >> 5);
+                                    else tma_load_3d_addr<kPair>(dst, &tmB, full_dst, c0, tap + j, kcol);
                             }
                             ++issued;
                             full_a += 8; empty_a += 8; full_dst += 8; slot_a += stage_bytes;
@@ -446,7 +460,8 @@ tc_fprop_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                         if (p.grp) {
                             // (cblocks is a multiple of KS here, so nst = KS and a slot never straddles two taps)
                             tma_load_5d_addr<kPair>(dst, &tmA, full_dst, 0, cq, cp, n0, c0 >> 5);
-                            tma_load_4d_addr<kPair>(dst + p.KS * kABytes, &tmB, full_dst, 0, kcol, c0 >> 5, tap);
+                            if (p.bmn) tma_load_4d_addr<kPair>(dst + p.KS * kABytes, &tmB, full_dst, 0, c0, p.flip ? taps - 1 - tap : tap, kcol >> 5);
+                            else tma_load_4d_addr<kPair>(dst + p.KS * kABytes, &tmB, full_dst, 0, kcol, c0 >> 5, tap);
                             c0 += p.KS * kBlockC;
                             if (c0 == c_end) {
                                 c0 = 0; ++tap; ++cq;
@@ -455,7 +470,8 @@ tc_fprop_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                         } else
                         for (int j = 0; j < nst; ++j, dst += step_bytes) {
                             tma_load_4d_addr<kPair>(dst, &tmA, full_dst, c0, cq, cp, n0);
-                            tma_load_3d_addr<kPair>(dst + kABytes, &tmB, full_dst, c0, tap, kcol);
+                            if (p.bmn) tma_load_4d_addr<kPair>(dst + kABytes, &tmB, full_dst, 0, c0, p.flip ? taps - 1 - tap : tap, kcol >> 5);
+                            else tma_load_3d_addr<kPair>(dst + kABytes, &tmB, full_dst, c0, tap, kcol);
                             c0 += kBlockC;
                             if (c0 == c_end) {
                                 c0 = 0; ++tap; ++cq;
@@ -734,6 +750,7 @@ bool tc_fprop_can_pool(const TcFpropArgs& a) {
 }
 
 bool tc_fprop_eligible(const TcFpropArgs& a) {
+    if (a.wt_mn_major && a.Kout % kBlockC != 0) return false;
     if (a.Cin % 4 != 0) return false;                       // TMA strides are multiples of 16 bytes
     if ((reinterpret_cast<uintptr_t>(a.in) | reinterpret_cast<uintptr_t>(a.wt)) & 15) return false;
     if (a.R * a.S > 65535) return false;
@@ -770,7 +787,8 @@ TileCfg plain_cfg(const TcFpropArgs& a, int cblocks, int sm_count) {
     // narrow tiles: several k-steps per slot (see the kernel), as long as 4 slots still fit
     // pairs pay where operand traffic or the issue rate of wide MMAs bounds the tile; narrow tiles are bound by
     // the issuing thread and run as single CTAs with two issuers instead
-    c.pair = env_int("PCL_PAIR", 1) && c.BN >= 128 && c.tiles_n >= 2 && sm_count >= 2;
+    c.pair = env_int("PCL_PAIR", 1) && c.BN >= 128 && c.tiles_n >= 2 && sm_count >= 2 &&
+             (!a.wt_mn_major || c.BN % 64 == 0);        // MN-major weights are fetched in whole 32-map groups per CTA
     const int step_bytes = kABytes + (c.pair ? c.BN * 64 : c.BN * 128);
     c.KS = env_int("PCL_KS", 2);
     const int kiters = a.R * a.S * cblocks;
@@ -808,7 +826,7 @@ TileCfg halo_cfg(const TcFpropArgs& a, int cblocks, int sm_count, int layout) {
     c.KS = env_int("PCL_KS_HALO", c.BN <= 64 ? 3 : (c.BN <= 128 ? 2 : 1));
     if (c.KS > a.R * a.S) c.KS = a.R * a.S;
     while (c.KS > 1 && (room - c.NA * c.a_buf_bytes) / (c.KS * b_bytes) < 3) --c.KS;
-    c.grp = env_int("PCL_GRP", 1) && c.KS > 1;
+    c.grp = env_int("PCL_GRP", 1) && c.KS > 1 && !a.wt_mn_major;      // (MN-major weights: one copy per tap)
     const int slot = c.KS * b_bytes;
     c.stages = (room - c.NA * c.a_buf_bytes) / slot;
     if (c.stages >= 9 && (room - 3 * c.a_buf_bytes) / slot >= 6) {
@@ -900,6 +918,7 @@ int launch_tc_fprop(const TcFpropArgs& a, cudaStream_t st) {
     p.tiles_n = cfg.pair ? (cfg.tiles_n + 1) / 2 : cfg.tiles_n;      // pair mode iterates over pairs of image groups
     p.BN = cfg.BN; p.PW = cfg.PW; p.patch_bytes = cfg.patch_bytes; p.a_buf_bytes = cfg.a_buf_bytes; p.NA = cfg.NA;
     p.half_off_bytes = cfg.half_off_bytes; p.stages = cfg.stages; p.KS = cfg.KS; p.grp = cfg.grp;
+    p.bmn = a.wt_mn_major ? 1 : 0; p.flip = a.flip_taps ? 1 : 0;
     // Two issuing threads only for single-CTA tiles: pair MMAs (cta_group::2) issued from two warps at once
     // ended in launch failures on B200, so a pair always has one issuer.
     // They pay where a tile has many slots; the hand-over between the threads costs more than it hides on
@@ -950,7 +969,15 @@ int launch_tc_fprop(const TcFpropArgs& a, cudaStream_t st) {
         const uint64_t strides[2] = {uint64_t(a.Cin) * 4, uint64_t(a.R) * a.S * a.Cin * 4};
         const uint32_t box[3] = {kBlockC, 1, uint32_t(cfg.pair ? p.BN / 2 : p.BN)};
         int rc;
-        if (cfg.grp && cfg.halo) {
+        if (a.wt_mn_major) {
+            // weights [Cin][R*S][Kout]: {32 maps, reduction rows, tap, 32-map group}; a box lands as
+            // [group][32 (x KS in the plain tiling) reduction rows][32 maps], the MN-major operand layout
+            const uint64_t dims4[4] = {kBlockC, uint64_t(a.Cin), uint64_t(a.R) * a.S, uint64_t(a.Kout / kBlockC)};
+            const uint64_t strides4[3] = {uint64_t(a.R) * a.S * a.Kout * 4, uint64_t(a.Kout) * 4, kBlockC * 4};
+            const uint32_t box4[4] = {kBlockC, uint32_t(kBlockC * ((cfg.grp && !cfg.halo) ? p.KS : 1)), 1,
+                                      uint32_t((cfg.pair ? p.BN / 2 : p.BN) / kBlockC)};
+            rc = make_tmap(&tmB, a.wt, 4, dims4, strides4, box4, true);
+        } else if (cfg.grp && cfg.halo) {
             // {channel, output map, tap}: a box of KS taps lands as KS weight tiles
             const uint64_t dims3[3] = {uint64_t(a.Cin), uint64_t(a.Kout), uint64_t(a.R) * a.S};
             const uint64_t strides3[2] = {uint64_t(a.R) * a.S * a.Cin * 4, uint64_t(a.Cin) * 4};

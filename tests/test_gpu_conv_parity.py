@@ -168,3 +168,24 @@ def test_forward_type_kernel_pipeline_variants(tag, variant, path_guard, monkeyp
     dx = G.run_conv_bwd_data(s, dy, w, x)
     G.assert_parity(dx, oracle.conv_bwd_data(s, dy, w, x), f"bwd_data {variant}")
     assert B.last_device_status() == 0
+
+
+@pytest.mark.parametrize("tiling", ["plain", "halo1", "auto"])
+@pytest.mark.parametrize("tag", ["odd_groups", "even_groups_wide", "fc_like"])
+def test_backward_data_reads_weights_in_place(tag, tiling, path_guard, monkeypatch):
+    """Backward-data takes the KRSC weights as an MN-major operand (taps flipped by index) when the layer's
+    input-map count is a multiple of 32; PCL_WEIGHTS_IN_PLACE=0 forces the flipped, transposed copy.  Same
+    products, same order of additions: the two must agree bit for bit, and with the oracle."""
+    import gpu_helpers as G
+    from paper_1602_06709_b200 import binding as B
+    monkeypatch.setenv("PCL_TILING", tiling)
+    B.set_path(B.PATH_TENSOR)
+    s = PIPELINE_SHAPES[tag]
+    x, w, dy, _ = G.make_inputs(s, "inplace_" + tag)
+    monkeypatch.setenv("PCL_WEIGHTS_IN_PLACE", "1")
+    dx1 = G.run_conv_bwd_data(s, dy, w, x)
+    monkeypatch.setenv("PCL_WEIGHTS_IN_PLACE", "0")
+    dx0 = G.run_conv_bwd_data(s, dy, w, x)
+    G.assert_parity(dx1, oracle.conv_bwd_data(s, dy, w, x), "bwd_data in place")
+    assert np.array_equal(dx0, dx1)
+    assert B.last_device_status() == 0
