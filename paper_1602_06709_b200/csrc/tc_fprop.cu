@@ -309,7 +309,10 @@ __device__ __noinline__ void mma_issuer(const FpropParams& p, const IssuerCtx& c
 // of the weight rows, which cuts the shared-memory fill traffic per MMA by a third (plain tiling only).
 // kPool: the epilogue also writes the 2x2 window maxima (kept out of the other instantiations, whose epilogue it
 // would cost registers).
-template <bool kPair, bool kPool>
+// kMask: the epilogue applies the ReLU mask (backward-data); its eight prefetched mask vectors would cost the other
+// instantiations registers (the epilogue is what the 168-register budget of an 11-warp CTA is short of, and a
+// spilled value that has left L1 costs ~600 cycles per use).
+template <bool kPair, bool kPool, bool kMask>
 __global__ void __launch_bounds__(kThreads, 1)
 tc_fprop_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                 const __grid_constant__ FpropParams p) {
@@ -584,7 +587,7 @@ tc_fprop_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                         if (p.bias) b = __ldg(reinterpret_cast<const float4*>(p.bias + col));
                         float4 csum = make_float4(0.f, 0.f, 0.f, 0.f);
                         float4 mk[8];
-                        if (p.mask_src) {
+                        if (kMask) {
 #pragma unroll
                             for (int i = 0; i < 8; ++i)
                                 mk[i] = ((vmask >> i) & 1u)
@@ -605,7 +608,7 @@ tc_fprop_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                                     o.x = 1.f / (1.f + __expf(-o.x)); o.y = 1.f / (1.f + __expf(-o.y));
                                     o.z = 1.f / (1.f + __expf(-o.z)); o.w = 1.f / (1.f + __expf(-o.w));
                                 }
-                                if (p.mask_src) {
+                                if (kMask) {
                                     o.x = mk[i].x > 0.f ? o.x : 0.f; o.y = mk[i].y > 0.f ? o.y : 0.f;
                                     o.z = mk[i].z > 0.f ? o.z : 0.f; o.w = mk[i].w > 0.f ? o.w : 0.f;
                                 }
@@ -665,7 +668,7 @@ tc_fprop_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                     const int col0 = kt * p.BN + ch * 32;
                     if (valid && col0 < p.Kout) {
                         float* dst = p.out + pix * p.Kout + col0;
-                        const float* msk = p.mask_src ? p.mask_src + pix * p.Kout + col0 : nullptr;
+                        const float* msk = kMask ? p.mask_src + pix * p.Kout + col0 : nullptr;
 #pragma unroll
                         for (int j = 0; j < 32; ++j) {
                             if (col0 + j < p.Kout) {
@@ -897,15 +900,13 @@ int launch_tc_fprop(const TcFpropArgs& a, cudaStream_t st) {
     static bool attr_set = false;
     if (!attr_set) {
         if (ensure_device_setup() != PCL_OK) return PCL_ERR_CUDA;
-        if (cudaFuncSetAttribute(tc_fprop_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 kSmemBudget + 1024) != cudaSuccess ||
-            cudaFuncSetAttribute(tc_fprop_kernel<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 kSmemBudget + 1024) != cudaSuccess ||
-            cudaFuncSetAttribute(tc_fprop_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 kSmemBudget + 1024) != cudaSuccess ||
-            cudaFuncSetAttribute(tc_fprop_kernel<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 kSmemBudget + 1024) != cudaSuccess)
-            return PCL_ERR_CUDA;
+        const void* kernels[6] = {
+            (const void*)tc_fprop_kernel<false, false, false>, (const void*)tc_fprop_kernel<false, true, false>,
+            (const void*)tc_fprop_kernel<false, false, true>,  (const void*)tc_fprop_kernel<true, false, false>,
+            (const void*)tc_fprop_kernel<true, true, false>,   (const void*)tc_fprop_kernel<true, false, true>};
+        for (const void* k : kernels)
+            if (cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget + 1024) != cudaSuccess)
+                return PCL_ERR_CUDA;
         attr_set = true;
     }
     FpropParams p{};
@@ -1011,7 +1012,7 @@ int launch_tc_fprop(const TcFpropArgs& a, cudaStream_t st) {
         if (cached_smem != smem) {
             lc.gridDim = dim3(unsigned(g_sm_count / 2 * 2));
             int n = 0;
-            if (cudaOccupancyMaxActiveClusters(&n, tc_fprop_kernel<true, false>, &lc) != cudaSuccess || n <= 0) return PCL_ERR_CUDA;
+            if (cudaOccupancyMaxActiveClusters(&n, tc_fprop_kernel<true, false, false>, &lc) != cudaSuccess || n <= 0) return PCL_ERR_CUDA;
             cached_clusters = n < g_sm_count / 2 ? n : g_sm_count / 2;
             cached_smem = smem;
         }
@@ -1019,14 +1020,16 @@ int launch_tc_fprop(const TcFpropArgs& a, cudaStream_t st) {
         long nclus = pair_tiles < cached_clusters ? pair_tiles : cached_clusters;
         lc.gridDim = dim3(unsigned(2 * nclus));
         LaunchScope scope(KID_TC_FPROP, 2.0 * a.N * a.P * a.Q * double(a.Kout) * a.Cin * a.R * a.S, st);
-        const cudaError_t le = p.pool_out ? cudaLaunchKernelEx(&lc, tc_fprop_kernel<true, true>, tmA, tmB, p)
-                                          : cudaLaunchKernelEx(&lc, tc_fprop_kernel<true, false>, tmA, tmB, p);
+        const cudaError_t le = p.pool_out   ? cudaLaunchKernelEx(&lc, tc_fprop_kernel<true, true, false>, tmA, tmB, p)
+                               : p.mask_src ? cudaLaunchKernelEx(&lc, tc_fprop_kernel<true, false, true>, tmA, tmB, p)
+                                            : cudaLaunchKernelEx(&lc, tc_fprop_kernel<true, false, false>, tmA, tmB, p);
         if (le != cudaSuccess) return PCL_ERR_CUDA;
     } else {
         const int grid = int(total < g_sm_count ? total : g_sm_count);
         LaunchScope scope(KID_TC_FPROP, 2.0 * a.N * a.P * a.Q * double(a.Kout) * a.Cin * a.R * a.S, st);
-        if (p.pool_out) tc_fprop_kernel<false, true><<<grid, kThreads, smem, st>>>(tmA, tmB, p);
-        else tc_fprop_kernel<false, false><<<grid, kThreads, smem, st>>>(tmA, tmB, p);
+        if (p.pool_out) tc_fprop_kernel<false, true, false><<<grid, kThreads, smem, st>>>(tmA, tmB, p);
+        else if (p.mask_src) tc_fprop_kernel<false, false, true><<<grid, kThreads, smem, st>>>(tmA, tmB, p);
+        else tc_fprop_kernel<false, false, false><<<grid, kThreads, smem, st>>>(tmA, tmB, p);
     }
     return cudaGetLastError() == cudaSuccess ? PCL_OK : PCL_ERR_CUDA;
 }
