@@ -106,6 +106,18 @@ __device__ __forceinline__ bool bounded_wait_warp_relaxed(uint64_t* bar, uint32_
     return __shfl_sync(0xffffffffu, ok, 0) != 0;
 }
 
+// Explicit shared-memory vector accesses (32-bit shared address): the staging tile of the epilogue is reached through
+// a pointer whose address space the compiler cannot see, and generic accesses would be ordered against the global
+// stores around them.
+__device__ __forceinline__ void st_shared_v4(uint32_t addr, float x, float y, float z, float w) {
+    asm volatile("st.shared.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "f"(x), "f"(y), "f"(z), "f"(w) : "memory");
+}
+__device__ __forceinline__ float4 ld_shared_v4(uint32_t addr) {
+    float4 v;
+    asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(addr));
+    return v;
+}
+
 // ---------------------------------------------------------------------- TMA
 __device__ __forceinline__ void prefetch_tmap(const CUtensorMap* m) {
     asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(m)) : "memory");

@@ -566,25 +566,32 @@ tc_fprop_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                     roff[i] = __shfl_sync(0xffffffffu, static_cast<unsigned long long>(pix * p.Kout), src);
                     vmask |= (__shfl_sync(0xffffffffu, static_cast<int>(valid), src) ? 1u : 0u) << i;
                 }
-                uint8_t* stg = epi_stage + (warp - 2) * 4096;
+                const uint32_t stg = smem_u32(epi_stage + (warp - 2) * 4096);
                 const int cg = (lane & 7) * 4;
                 for (int ch = chalf; ch < p.BN / 32; ch += 2) {
+                    const int col = kt * p.BN + ch * 32 + cg;
+                    // (the bias is fetched before the accumulator so that its latency hides behind the staging)
+                    float4 b = make_float4(0.f, 0.f, 0.f, 0.f);
+                    if (p.bias && col < p.Kout) b = __ldg(reinterpret_cast<const float4*>(p.bias + col));
                     uint32_t v[32];
                     tmem_ld_32x32(t_row + ch * 32, v);
                     tmem_ld_wait();
 #pragma unroll
                     for (int j = 0; j < 8; ++j) {
                         const int slot = j ^ (lane & 7);
-                        *reinterpret_cast<float4*>(stg + lane * 128 + slot * 16) =
-                            make_float4(__uint_as_float(v[4 * j]), __uint_as_float(v[4 * j + 1]),
-                                        __uint_as_float(v[4 * j + 2]), __uint_as_float(v[4 * j + 3]));
+                        st_shared_v4(stg + lane * 128 + slot * 16, __uint_as_float(v[4 * j]), __uint_as_float(v[4 * j + 1]),
+                                     __uint_as_float(v[4 * j + 2]), __uint_as_float(v[4 * j + 3]));
                     }
                     __syncwarp();
-                    const int col = kt * p.BN + ch * 32 + cg;
                     const unsigned live = __ballot_sync(0xffffffffu, col < p.Kout);   // lanes l, l^8, l^16 agree
                     if (col < p.Kout) {
-                        float4 b = make_float4(0.f, 0.f, 0.f, 0.f);
-                        if (p.bias) b = __ldg(reinterpret_cast<const float4*>(p.bias + col));
+                        // all eight staged rows first, so that their latencies overlap
+                        float4 ov[8];
+#pragma unroll
+                        for (int i = 0; i < 8; ++i) {
+                            const int rr = (lane >> 3) + 4 * i;
+                            ov[i] = ld_shared_v4(stg + rr * 128 + (((lane & 7) ^ (rr & 7)) * 16));
+                        }
                         float4 csum = make_float4(0.f, 0.f, 0.f, 0.f);
                         float4 mk[8];
                         if (kMask) {
@@ -596,9 +603,7 @@ tc_fprop_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                         }
 #pragma unroll
                         for (int i = 0; i < 8; ++i) {
-                            const int rr = (lane >> 3) + 4 * i;
-                            const int slot = (lane & 7) ^ (rr & 7);
-                            float4 o = *reinterpret_cast<const float4*>(stg + rr * 128 + slot * 16);
+                            float4 o = ov[i];
                             if ((vmask >> i) & 1u) {
                                 o.x += b.x; o.y += b.y; o.z += b.z; o.w += b.w;
                                 if (p.act == PCL_ACT_RELU) {
@@ -639,7 +644,7 @@ tc_fprop_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
 #pragma unroll
                                 for (int e = 0; e < 4; ++e) {
                                     const int rr = r0 | (e & 1) | ((e >> 1) << lb);
-                                    const float4 t4 = *reinterpret_cast<const float4*>(stg + rr * 128 + (((lane & 7) ^ (rr & 7)) * 16));
+                                    const float4 t4 = ld_shared_v4(stg + rr * 128 + (((lane & 7) ^ (rr & 7)) * 16));
                                     m.x = fmaxf(m.x, t4.x); m.y = fmaxf(m.y, t4.y); m.z = fmaxf(m.z, t4.z); m.w = fmaxf(m.w, t4.w);
                                 }
                                 m.x += b.x; m.y += b.y; m.z += b.z; m.w += b.w;
