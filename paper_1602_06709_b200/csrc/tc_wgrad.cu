@@ -258,12 +258,17 @@ tc_wgrad_kernel(const __grid_constant__ CUtensorMap tmDy, const __grid_constant_
             tc_fence_after();
             const uint32_t t_row = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16);
             const size_t krow = static_cast<size_t>(valid ? k : 0) * p.R * p.S;
+            // Each lane owns one output-map row of the accumulator, but 32 columns of a row are 128 contiguous
+            // bytes of dw: a chunk is transposed through a 4 KB staging tile per warp (the pipeline's shared
+            // memory, idle by now: every copy has landed and every MMA has read it) and written 4 rows x 128
+            // bytes per instruction.
+            const uint32_t stg = smem_u32(smem) + (warp - 2) * 4096;
+            const int cg = (lane & 7) * 4;
             for (int ch = 0; ch < n_groups; ++ch) {
                 const int run = run0 + ch / p.L;
                 if (run >= p.total_runs) break;         // (pair mode) columns of runs past the last tap
                 const int tap = run / p.runs_per_tap;
                 const int c0 = ((run - tap * p.runs_per_tap) * p.L + ch % p.L) * 32;
-                float* dst = p.out + static_cast<size_t>(split) * p.split_stride + (krow + tap) * p.C + c0;
                 uint32_t v[32];
                 if (kiters > 0) {
                     tmem_ld_32x32(t_row + ch * 32, v);
@@ -272,18 +277,36 @@ tc_wgrad_kernel(const __grid_constant__ CUtensorMap tmDy, const __grid_constant_
 #pragma unroll
                     for (int j = 0; j < 32; ++j) v[j] = 0u;
                 }
-                if (valid && c0 < p.C) {
+                if (vec_ok) {
+#pragma unroll
+                    for (int j = 0; j < 8; ++j)
+                        st_shared_v4(stg + lane * 128 + ((j ^ (lane & 7)) * 16), __uint_as_float(v[4 * j]),
+                                     __uint_as_float(v[4 * j + 1]), __uint_as_float(v[4 * j + 2]), __uint_as_float(v[4 * j + 3]));
+                    __syncwarp();
+                    if (c0 + cg < p.C) {
+#pragma unroll
+                        for (int i = 0; i < 8; ++i) {
+                            const int rr = (lane >> 3) + 4 * i;
+                            const int kk = kt * 128 + quarter * 32 + rr;
+                            const float4 o = ld_shared_v4(stg + rr * 128 + (((lane & 7) ^ (rr & 7)) * 16));
+                            if (kk < p.K) {
+                                float* dst = p.out + static_cast<size_t>(split) * p.split_stride +
+                                             (static_cast<size_t>(kk) * p.R * p.S + tap) * p.C + c0 + cg;
+                                if (p.use_atomics) {
+                                    atomicAdd(dst, o.x); atomicAdd(dst + 1, o.y); atomicAdd(dst + 2, o.z); atomicAdd(dst + 3, o.w);
+                                } else {
+                                    *reinterpret_cast<float4*>(dst) = o;
+                                }
+                            }
+                        }
+                    }
+                    __syncwarp();
+                } else if (valid && c0 < p.C) {
+                    float* dst = p.out + static_cast<size_t>(split) * p.split_stride + (krow + tap) * p.C + c0;
                     if (p.use_atomics) {
 #pragma unroll
                         for (int j = 0; j < 32; ++j)
                             if (c0 + j < p.C) atomicAdd(dst + j, __uint_as_float(v[j]));
-                    } else if (vec_ok) {
-#pragma unroll
-                        for (int j = 0; j < 32; j += 4)
-                            if (c0 + j < p.C)
-                                *reinterpret_cast<float4*>(dst + j) =
-                                    make_float4(__uint_as_float(v[j]), __uint_as_float(v[j + 1]),
-                                                __uint_as_float(v[j + 2]), __uint_as_float(v[j + 3]));
                     } else {
 #pragma unroll
                         for (int j = 0; j < 32; ++j)
