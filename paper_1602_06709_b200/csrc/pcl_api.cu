@@ -86,7 +86,7 @@ encode_tiled_fn get_encode_tiled() {
 }
 
 int make_tmap(CUtensorMap* out, const void* base, int rank, const uint64_t* dims, const uint64_t* strides_bytes,
-              const uint32_t* box, bool atom32) {
+              const uint32_t* box, bool atom32, bool plain_f32) {
     encode_tiled_fn enc = get_encode_tiled();
     if (!enc) return PCL_ERR_CUDA;
     cuuint64_t gdim[5];
@@ -103,7 +103,7 @@ int make_tmap(CUtensorMap* out, const void* base, int rank, const uint64_t* dims
         if (strides_bytes[i] % 16 != 0 || strides_bytes[i] >= (1ull << 40)) return PCL_ERR_UNSUPPORTED_SHAPE;
     }
     if (reinterpret_cast<uintptr_t>(base) & 15) return PCL_ERR_MISALIGNED;
-    const CUresult r = enc(out, CU_TENSOR_MAP_DATA_TYPE_TFLOAT32, cuuint32_t(rank), const_cast<void*>(base), gdim, gstr,
+    const CUresult r = enc(out, plain_f32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_TFLOAT32, cuuint32_t(rank), const_cast<void*>(base), gdim, gstr,
                            gbox, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
                            atom32 ? CU_TENSOR_MAP_SWIZZLE_128B_ATOM_32B : CU_TENSOR_MAP_SWIZZLE_128B,
                            CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);

@@ -43,8 +43,9 @@ encode_tiled_fn get_encode_tiled();
 // fp32 tensor map with a 128-byte swizzle span, swizzled in 16-byte chunks
 // (K-major operands) or, if atom32, in 32-byte chunks (MN-major operands).
 // dims/box innermost first; strides_bytes has rank-1 entries (dims 1..rank-1).
+// The element type is TFLOAT32 (TMA rounds fp32 to tf32, nearest-even, on load) unless plain_f32 (maps used for stores).
 int make_tmap(CUtensorMap* out, const void* base, int rank, const uint64_t* dims, const uint64_t* strides_bytes,
-              const uint32_t* box, bool atom32);
+              const uint32_t* box, bool atom32, bool plain_f32 = false);
 
 // ---- forward-type implicit GEMM on tcgen05 (stride-1 convolution) ----------
 // out[n,p,q,k] = epi( sum_{r,s,c} in[n, p + r - pad_h, q + s - pad_w, c] * wt[k, r*S+s, c] )

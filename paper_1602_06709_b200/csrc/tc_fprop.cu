@@ -67,6 +67,7 @@ struct FpropParams {
     const float* bias;
     const float* mask_src;
     float* out;
+    int tma_store;              // the epilogue writes `out` with TMA stores from the staging tiles (tmOut is valid)
     float* pool_out;            // optional [N][P/2][Q/2][Kout]: 2x2 window maxima of the output
     float* colsum_rows;         // optional [m_tiles * MT * 4][Kout] per-(box, quarter) column sums of the output
     unsigned int* status;       // device status word
@@ -315,7 +316,7 @@ __device__ __noinline__ void mma_issuer(const FpropParams& p, const IssuerCtx& c
 template <bool kPair, bool kPool, bool kMask>
 __global__ void __launch_bounds__(kThreads, 1)
 tc_fprop_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
-                const __grid_constant__ FpropParams p) {
+                const __grid_constant__ CUtensorMap tmOut, const __grid_constant__ FpropParams p) {
     extern __shared__ uint8_t smem_raw[];
     __shared__ uint64_t full_bar[kMaxStages];
     __shared__ uint64_t empty_bar[kMaxStages];
@@ -552,7 +553,76 @@ tc_fprop_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                 const size_t m_index = (static_cast<size_t>(ni) * p.tiles_p + it.pi) * p.tiles_q + it.qi;
                 cs_row = p.colsum_rows + ((m_index * p.MT + h) * 4 + quarter) * p.Kout;
             }
-            if (vec_ok) {
+            if (!kMask && p.tma_store) {
+                // TMA-store path (no mask, no column sums).  Each lane owns one row (pixel) of the accumulator: it
+                // finishes its 32 columns in registers (bias, activation), puts them into its row of the warp's
+                // 4 KB staging tile in the 128-byte-swizzle layout, and one lane hands the tile to TMA, which writes
+                // the 32 pixels x 128 bytes and clips what lies outside the tensor.  The warp's 32 rows are 32
+                // consecutive pixels of the box, i.e. a sub-box whose first pixel is (sq, sp, sn).
+                const uint32_t stg = smem_u32(epi_stage + (warp - 2) * 4096);
+                const int srow = quarter * 32;
+                const int sq = it.qi * p.tw + (srow & (bw - 1)) + h * p.half_dq;
+                const int sp = it.pi * p.th + ((srow >> p.bw_log2) & (bh - 1)) + h * p.half_dp;
+                const int sn = ni * p.tn + (srow >> (p.bw_log2 + p.bh_log2));
+                const bool in_range = sq < p.Q && sp < p.P && sn < p.N;     // (a store never starts outside the tensor)
+                for (int ch = chalf; ch < p.BN / 32; ch += 2) {
+                    const int col0 = kt * p.BN + ch * 32;
+                    float4 bv[8];
+#pragma unroll
+                    for (int j = 0; j < 8; ++j)
+                        bv[j] = (p.bias && col0 + 4 * j < p.Kout) ? __ldg(reinterpret_cast<const float4*>(p.bias + col0 + 4 * j))
+                                                                   : make_float4(0.f, 0.f, 0.f, 0.f);
+                    uint32_t v[32];
+                    tmem_ld_32x32(t_row + ch * 32, v);
+                    tmem_ld_wait();
+                    // the previous store of this warp must have read the staging tile before it is overwritten
+                    if (lane == 0) bulk_wait_group_read0();
+                    __syncwarp();
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) {
+                        float4 o = make_float4(__uint_as_float(v[4 * j]) + bv[j].x, __uint_as_float(v[4 * j + 1]) + bv[j].y,
+                                               __uint_as_float(v[4 * j + 2]) + bv[j].z, __uint_as_float(v[4 * j + 3]) + bv[j].w);
+                        if (p.act == PCL_ACT_RELU) {
+                            o.x = fmaxf(o.x, 0.f); o.y = fmaxf(o.y, 0.f); o.z = fmaxf(o.z, 0.f); o.w = fmaxf(o.w, 0.f);
+                        } else if (p.act == PCL_ACT_SIGMOID) {
+                            o.x = 1.f / (1.f + __expf(-o.x)); o.y = 1.f / (1.f + __expf(-o.y));
+                            o.z = 1.f / (1.f + __expf(-o.z)); o.w = 1.f / (1.f + __expf(-o.w));
+                        }
+                        st_shared_v4(stg + lane * 128 + ((j ^ (lane & 7)) * 16), o.x, o.y, o.z, o.w);
+                    }
+                    fence_proxy_async_shared();
+                    __syncwarp();
+                    if (lane == 0 && in_range && col0 < p.Kout) {
+                        tma_store_4d(&tmOut, stg, col0, sq, sp, sn);
+                        bulk_commit_group();
+                    }
+                    if (kPool) {
+                        // Fused 2x2 max pooling from the finished values in the staging tile: the 32 rows hold 8 whole
+                        // windows (bit 0 of the row = parity of q, bit log2(bw) = parity of p; boxes start at even
+                        // coordinates); lane l takes windows (l >> 3) and (l >> 3) + 4 of its 4 columns.
+                        const int lb = p.bw_log2;
+                        const int col = col0 + (lane & 7) * 4;
+#pragma unroll
+                        for (int half = 0; half < 2; ++half) {
+                            const int wdx = (lane >> 3) + 4 * half;
+                            const int r0 = ((wdx & ((1 << (lb - 1)) - 1)) << 1) | ((wdx >> (lb - 1)) << (lb + 1));
+                            float4 m = make_float4(-INFINITY, -INFINITY, -INFINITY, -INFINITY);
+#pragma unroll
+                            for (int e = 0; e < 4; ++e) {
+                                const int rr = r0 | (e & 1) | ((e >> 1) << lb);
+                                const float4 t4 = ld_shared_v4(stg + rr * 128 + (((lane & 7) ^ (rr & 7)) * 16));
+                                m.x = fmaxf(m.x, t4.x); m.y = fmaxf(m.y, t4.y); m.z = fmaxf(m.z, t4.z); m.w = fmaxf(m.w, t4.w);
+                            }
+                            const int wrow = srow + r0;
+                            const int wq = it.qi * p.tw + (wrow & (bw - 1)) + h * p.half_dq;
+                            const int wp = it.pi * p.th + ((wrow >> p.bw_log2) & (bh - 1)) + h * p.half_dp;
+                            const int wn = ni * p.tn + (wrow >> (p.bw_log2 + p.bh_log2));
+                            if (col < p.Kout && wq < p.Q && wp < p.P && wn < p.N)
+                                *reinterpret_cast<float4*>(p.pool_out + ((static_cast<size_t>(wn) * (p.P >> 1) + (wp >> 1)) * (p.Q >> 1) + (wq >> 1)) * p.Kout + col) = m;
+                        }
+                    }
+                }
+            } else if (vec_ok) {
                 // Coalesced path.  Each lane owns one row (pixel) of the accumulator, but a row's 32 columns
                 // are 128 contiguous bytes in global memory, so the chunk is first transposed through a
                 // 4 KB per-warp staging tile (XOR-swizzled 16-byte slots: conflict-free both ways) and then
@@ -696,6 +766,7 @@ tc_fprop_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                 else mbar_arrive(&tmem_empty_bar[acc]);
             }
         }
+        if (!kMask && p.tma_store && lane == 0) bulk_wait_group0();     // every store of this warp has completed
     }
 
     tc_fence_before();
@@ -1000,6 +1071,18 @@ int launch_tc_fprop(const TcFpropArgs& a, cudaStream_t st) {
         }
         if (rc != PCL_OK) return rc;
     }
+    // Output map for the TMA-store epilogue: a warp stores the 32 consecutive box pixels it owns, 32 maps at a time.
+    CUtensorMap tmOut = tmA;        // (a valid map is passed in any case; unused unless p.tma_store)
+    p.tma_store = 0;
+    if (env_int("PCL_TMA_STORE", 1) && !a.mask_src && !a.colsum_rows && a.Kout % 4 == 0 &&
+        (reinterpret_cast<uintptr_t>(a.out) & 15) == 0) {
+        const uint32_t bx = bw < 32 ? bw : 32, by = uint32_t(bh) < 32 / bx ? uint32_t(bh) : 32 / bx, bnn = 32 / (bx * by);
+        const uint64_t dims[4] = {uint64_t(a.Kout), uint64_t(a.Q), uint64_t(a.P), uint64_t(a.N)};
+        const uint64_t strides[3] = {uint64_t(a.Kout) * 4, uint64_t(a.Q) * a.Kout * 4, uint64_t(a.P) * a.Q * a.Kout * 4};
+        const uint32_t box[4] = {kBlockC, bx, by, bnn};
+        if (make_tmap(&tmOut, a.out, 4, dims, strides, box, false, true) == PCL_OK) p.tma_store = 1;
+        else tmOut = tmA;
+    }
     const long total = m_tiles * p.tiles_k;
     const size_t smem = (p.halo ? size_t(p.NA) * p.a_buf_bytes + size_t(p.stages) * p.KS * (cfg.pair ? p.BN * 64 : p.BN * 128)
                                 : size_t(p.stages) * p.KS * (kABytes + (cfg.pair ? p.BN * 64 : p.BN * 128))) +
@@ -1025,16 +1108,16 @@ int launch_tc_fprop(const TcFpropArgs& a, cudaStream_t st) {
         long nclus = pair_tiles < cached_clusters ? pair_tiles : cached_clusters;
         lc.gridDim = dim3(unsigned(2 * nclus));
         LaunchScope scope(KID_TC_FPROP, 2.0 * a.N * a.P * a.Q * double(a.Kout) * a.Cin * a.R * a.S, st);
-        const cudaError_t le = p.pool_out   ? cudaLaunchKernelEx(&lc, tc_fprop_kernel<true, true, false>, tmA, tmB, p)
-                               : p.mask_src ? cudaLaunchKernelEx(&lc, tc_fprop_kernel<true, false, true>, tmA, tmB, p)
-                                            : cudaLaunchKernelEx(&lc, tc_fprop_kernel<true, false, false>, tmA, tmB, p);
+        const cudaError_t le = p.pool_out   ? cudaLaunchKernelEx(&lc, tc_fprop_kernel<true, true, false>, tmA, tmB, tmOut, p)
+                               : p.mask_src ? cudaLaunchKernelEx(&lc, tc_fprop_kernel<true, false, true>, tmA, tmB, tmOut, p)
+                                            : cudaLaunchKernelEx(&lc, tc_fprop_kernel<true, false, false>, tmA, tmB, tmOut, p);
         if (le != cudaSuccess) return PCL_ERR_CUDA;
     } else {
         const int grid = int(total < g_sm_count ? total : g_sm_count);
         LaunchScope scope(KID_TC_FPROP, 2.0 * a.N * a.P * a.Q * double(a.Kout) * a.Cin * a.R * a.S, st);
-        if (p.pool_out) tc_fprop_kernel<false, true, false><<<grid, kThreads, smem, st>>>(tmA, tmB, p);
-        else if (p.mask_src) tc_fprop_kernel<false, false, true><<<grid, kThreads, smem, st>>>(tmA, tmB, p);
-        else tc_fprop_kernel<false, false, false><<<grid, kThreads, smem, st>>>(tmA, tmB, p);
+        if (p.pool_out) tc_fprop_kernel<false, true, false><<<grid, kThreads, smem, st>>>(tmA, tmB, tmOut, p);
+        else if (p.mask_src) tc_fprop_kernel<false, false, true><<<grid, kThreads, smem, st>>>(tmA, tmB, tmOut, p);
+        else tc_fprop_kernel<false, false, false><<<grid, kThreads, smem, st>>>(tmA, tmB, tmOut, p);
     }
     return cudaGetLastError() == cudaSuccess ? PCL_OK : PCL_ERR_CUDA;
 }
