@@ -182,9 +182,10 @@ POOL_FUSED_SHAPES = [
 ]
 
 
+@pytest.mark.parametrize("store", ["tma", "direct"])
 @pytest.mark.parametrize("tiling", ["auto", "plain", "halo0", "halo1", "halo2"])
 @pytest.mark.parametrize("shape", POOL_FUSED_SHAPES)
-def test_conv_fwd_with_fused_maxpool(shape, tiling, monkeypatch):
+def test_conv_fwd_with_fused_maxpool(shape, tiling, store, monkeypatch):
     """conv -> ReLU -> 2x2 max pool in one call: y must match the oracle's convolution, and the pooled
     tensor must be bit-for-bit the 2x2 maxima of the y the same call wrote (the epilogue takes the
     maximum of the raw accumulators, which commutes exactly with the bias add and the ReLU)."""
@@ -193,6 +194,8 @@ def test_conv_fwd_with_fused_maxpool(shape, tiling, monkeypatch):
     from paper_1602_06709_b200 import binding as B
     if tiling != "auto":
         monkeypatch.setenv("PCL_TILING", tiling)
+    # the epilogue writes y either with TMA stores from its staging tiles or with per-lane coalesced stores
+    monkeypatch.setenv("PCL_TMA_STORE", "1" if store == "tma" else "0")
     N, C, K, H, W = shape
     s = ConvShape(N=N, C=C, K=K, H=H, W=W, R=3, S=3, pad_h=1, pad_w=1)
     x, w, _, bias = G.make_inputs(s, f"fwdpool{C}_{K}")
