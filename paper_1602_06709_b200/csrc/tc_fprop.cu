@@ -51,6 +51,7 @@ struct FpropParams {
     int bmn;                    // B (weights) is MN-major: laid out [Cin][R*S][Kout], read through {32 maps, reduction rows,
                                 // tap, 32-map group} boxes with the 32-byte-atom swizzle (backward-data without a transposed copy)
     int flip;                   // tap t reads tap R*S-1-t of the weights
+    int split_acc;              // two issuers with an accumulator each (2 x 2 x MT x BN TMEM columns)
     int issuers;                // MMA-issuing threads (1 or 2; see the kernel)
     int grp;                    // plain tiling: a slot's KS k-steps are KS consecutive channel blocks of one tap, fetched by
                                 // ONE copy of A and one of B (slot layout: KS A tiles, then KS B tiles)
@@ -130,6 +131,15 @@ struct IssuerCtx {
     int first_tile, tile_stride, total_tiles, kiters;
 };
 
+// v += the 32 x 32 block at `taddr` (the second issuer's accumulator).
+__device__ __forceinline__ void add_second_accumulator(uint32_t taddr, uint32_t (&v)[32]) {
+    uint32_t w[32];
+    tmem_ld_32x32(taddr, w);
+    tmem_ld_wait();
+#pragma unroll
+    for (int i = 0; i < 32; ++i) v[i] = __float_as_uint(__uint_as_float(v[i]) + __uint_as_float(w[i]));
+}
+
 // kTaps consecutive taps of a haloed slot, straight-line (a taken branch costs a lone thread tens of cycles).
 template <bool kPair, int kTaps, int kMT>
 __device__ __forceinline__ void halo_taps(uint32_t d_tmem, uint32_t BN, uint32_t& a_lo, uint32_t b_lo, int& s, int S,
@@ -171,6 +181,9 @@ __device__ __noinline__ void mma_issuer(const FpropParams& p, const IssuerCtx& c
     const uint32_t tmem_base = c.tmem_base, b16 = c.b_bytes >> 4;
     const int first_tile = c.first_tile, tile_stride = c.tile_stride, total_tiles = c.total_tiles, kiters = c.kiters;
 
+    // kDuo with `split`: each issuer accumulates its slots into an accumulator of its own (the epilogue adds the
+    // two), so the threads need not hand over: no ordering between them can change a bit of the result.
+    const bool split = kDuo && p.split_acc;
     const int bmn = p.bmn;
     const uint32_t idesc = make_idesc_tf32(BN, false, bmn != 0, kPair ? 256u : 128u);
     const uint32_t bks = bmn ? 64u : 2u;         // k-block stride of B inside a k-step (16-byte units)
@@ -207,14 +220,14 @@ __device__ __noinline__ void mma_issuer(const FpropParams& p, const IssuerCtx& c
     if (kDuo) { mine = turn == issuer; turn ^= 1u; }
 #define PCL_SLOT_ACQUIRE()                                                                                        \
     if (!bounded_wait_addr(full_a, phase, abort_flag, status, WAIT_MMA_FULL)) { ok = false; break; }             \
-    if (kDuo && !wait_issue_turn(issue_seq, seq, abort_flag, status)) { ok = false; break; }                     \
+    if (kDuo && !split && !wait_issue_turn(issue_seq, seq, abort_flag, status)) { ok = false; break; }           \
     tc_fence_after();
 #define PCL_SLOT_RELEASE()                                                                                        \
-    if (kDuo) *issue_seq = seq + 1;                                                                               \
+    if (kDuo && !split) *issue_seq = seq + 1;                                                                     \
     umma_commit_addr<kPair>(empty_a);
 #define PCL_SLOT_END()                                                                                            \
     if (kDuo) ++seq;                                                                                              \
-    accum = 1;                                                                                                    \
+    if (!split || mine) accum = 1;      /* split: an issuer's own first slot overwrites its own accumulator */    \
     full_a += 8; empty_a += 8; slot_lo += stage16;                                                                \
     if (++stage == stages) { stage = 0; phase ^= 1u; full_a = full0; empty_a = empty0; slot_lo = ring_lo0; }
 
@@ -223,7 +236,7 @@ __device__ __noinline__ void mma_issuer(const FpropParams& p, const IssuerCtx& c
         const uint32_t acc_phase = (tile_cnt >> 1) & 1;
         if (!bounded_wait_addr(tempty0 + acc * 8, acc_phase ^ 1u, abort_flag, status, WAIT_MMA_TMEM_EMPTY)) break;
         tc_fence_after();
-        const uint32_t d_tmem = tmem_base + acc * MT * BN;
+        const uint32_t d_tmem = tmem_base + (split ? (2 * acc + issuer) * MT * BN : acc * MT * BN);
         uint32_t accum = 0;         // the tile's first MMA (whoever issues it) overwrites the accumulator
         if (halo) {
             const uint64_t a_desc0 = make_smem_desc(0, 16, PW * 128, kSwizzle128B);   // 8-pixel groups are one patch row apart
@@ -547,7 +560,9 @@ tc_fprop_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
             const int n = ni * p.tn + in_;
             const bool valid = (q < p.Q) && (pp < p.P) && (n < p.N);
             const size_t pix = (static_cast<size_t>(n) * p.P + pp) * p.Q + q;
-            const uint32_t t_row = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + (acc * p.MT + h) * p.BN;
+            const uint32_t t_row = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) +
+                                   ((p.split_acc ? 2 * acc : acc) * p.MT + h) * p.BN;
+            const uint32_t t_second = p.MT * p.BN;      // split accumulators: the second issuer's copy of this box
             float* cs_row = nullptr;
             if (p.colsum_rows && ni * p.tn < p.N) {      // (an odd image-group count leaves the pair's last tile empty)
                 const size_t m_index = (static_cast<size_t>(ni) * p.tiles_p + it.pi) * p.tiles_q + it.qi;
@@ -575,6 +590,7 @@ tc_fprop_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                     uint32_t v[32];
                     tmem_ld_32x32(t_row + ch * 32, v);
                     tmem_ld_wait();
+                    if (!kPool && p.split_acc) add_second_accumulator(t_row + t_second + ch * 32, v);
                     // the previous store of this warp must have read the staging tile before it is overwritten
                     if (lane == 0) bulk_wait_group_read0();
                     __syncwarp();
@@ -646,6 +662,7 @@ tc_fprop_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                     uint32_t v[32];
                     tmem_ld_32x32(t_row + ch * 32, v);
                     tmem_ld_wait();
+                    if (!kPool && p.split_acc) add_second_accumulator(t_row + t_second + ch * 32, v);
 #pragma unroll
                     for (int j = 0; j < 8; ++j) {
                         const int slot = j ^ (lane & 7);
@@ -740,6 +757,7 @@ tc_fprop_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                     uint32_t v[32];
                     tmem_ld_32x32(t_row + ch * 32, v);
                     tmem_ld_wait();
+                    if (!kPool && p.split_acc) add_second_accumulator(t_row + t_second + ch * 32, v);
                     const int col0 = kt * p.BN + ch * 32;
                     if (valid && col0 < p.Kout) {
                         float* dst = p.out + pix * p.Kout + col0;
@@ -1009,8 +1027,10 @@ int launch_tc_fprop(const TcFpropArgs& a, cudaStream_t st) {
     p.R = a.R; p.S = a.S; p.pad_h = a.pad_h; p.pad_w = a.pad_w;
     p.N = a.N; p.P = a.P; p.Q = a.Q; p.Kout = a.Kout;
     p.act = a.act;
+    // (not in the pooling instantiation: its epilogue has no registers to spare)
+    p.split_acc = (p.issuers == 2 && 4 * p.MT * p.BN <= 512 && !a.pool_out && env_int("PCL_SPLIT_ACC", 1)) ? 1 : 0;
     p.tmem_cols = 32;
-    while (p.tmem_cols < 2 * p.MT * p.BN) p.tmem_cols *= 2;
+    while (p.tmem_cols < (p.split_acc ? 4 : 2) * p.MT * p.BN) p.tmem_cols *= 2;
     p.bias = a.bias; p.mask_src = a.mask_src; p.out = a.out;
     if (a.pool_out && !tc_fprop_can_pool(a)) return PCL_ERR_UNSUPPORTED_SHAPE;
     p.pool_out = a.pool_out;

@@ -189,3 +189,36 @@ def test_backward_data_reads_weights_in_place(tag, tiling, path_guard, monkeypat
     G.assert_parity(dx1, oracle.conv_bwd_data(s, dy, w, x), "bwd_data in place")
     assert np.array_equal(dx0, dx1)
     assert B.last_device_status() == 0
+
+
+@pytest.mark.parametrize("mode", ["solo", "ordered", "split"])
+@pytest.mark.parametrize("tag", ["fits_16x16", "fits_8x32", "k5"])
+def test_two_issuers_keep_results_reproducible(tag, mode, path_guard, monkeypatch):
+    """Narrow single-CTA tiles may run two MMA-issuing threads: either ordered by a sequence number (the
+    additions then happen in the order of one issuer: bit-identical to it) or with an accumulator each that
+    the epilogue adds (a different, but fixed, order).  Every mode must match the oracle and repeat itself
+    bit for bit; the ordered mode must equal the single issuer exactly."""
+    import gpu_helpers as G
+    from paper_1602_06709_b200 import binding as B
+    env = {"solo": dict(PCL_ISSUERS="1"), "ordered": dict(PCL_ISSUERS="2", PCL_SPLIT_ACC="0"),
+           "split": dict(PCL_ISSUERS="2", PCL_SPLIT_ACC="1")}
+    B.set_path(B.PATH_TENSOR)
+    s = HALO_SHAPES[tag]
+    x, w, dy, bias = G.make_inputs(s, "issuers_" + tag)
+
+    def run(m):
+        for k in ("PCL_ISSUERS", "PCL_SPLIT_ACC"):
+            monkeypatch.delenv(k, raising=False)
+        for k, v in env[m].items():
+            monkeypatch.setenv(k, v)
+        return G.run_conv_fwd(s, x, w, bias, B.ACT_RELU), G.run_conv_bwd_data(s, dy, w, x)
+
+    y, dx = run(mode)
+    G.assert_parity(y, oracle.conv_fwd(s, x, w, bias, oracle.ACT_RELU), f"fwd {mode}")
+    G.assert_parity(dx, oracle.conv_bwd_data(s, dy, w, x), f"bwd_data {mode}")
+    y2, dx2 = run(mode)
+    assert np.array_equal(y, y2) and np.array_equal(dx, dx2)
+    if mode == "ordered":
+        y1, dx1 = run("solo")
+        assert np.array_equal(y, y1) and np.array_equal(dx, dx1)
+    assert B.last_device_status() == 0
