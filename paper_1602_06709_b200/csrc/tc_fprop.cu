@@ -3,23 +3,28 @@
 //   out[n,p,q,k] = epi( sum_{r,s,c} in[n, p+r-pad_h, q+s-pad_w, c] * wt[k, r*S+s, c] )
 //
 // (Algorithm 1 with stride 1; the same kernel computes the backward-data pass of
-// a stride-1 layer when it is handed dy as `in` and the flipped, transposed
-// weights, and the fully-connected GEMMs as the 1x1 / 1x1-map special case.)
+// a stride-1 layer when it is handed dy as `in` and either the layer's own KRSC
+// weights, read in place as an MN-major operand with the taps flipped by index,
+// or a flipped, transposed copy; and the fully-connected GEMMs as the 1x1 /
+// 1x1-map special case.)
 //
 // GEMM view: M = N*P*Q output pixels, N = Kout, reduction over (r, s, c).
 // One CTA tile is 128 output pixels x BN output maps.  The 128 pixels are a
 // box bw x bh x bn of the (q, p, n) index space, so that for a fixed tap (r, s)
-// the A operand is one 4-D TMA box of the NHWC input shifted by the tap: the
-// im2col matrix is never materialised and zero padding is TMA's out-of-bounds
-// fill.  B is a 3-D TMA box {32 c, 1 tap, BN k} of the weights.
+// the A operand is one TMA box of the NHWC input shifted by the tap: the im2col
+// matrix is never materialised and zero padding is TMA's out-of-bounds fill.
+// B is a TMA box of BN weight rows.  Variants, chosen per launch on the host:
+//   plain tiling    one box per tap; a slot holds two channel blocks fetched by one copy per operand
+//   haloed tiling   one input patch per channel block, taps are row-shifted views of it (narrow layers)
+//   CTA pairs       two CTAs of a cluster share a weight tile, the leader issues M = 256 MMAs (cta_group::2)
 //
-// Warp roles (320 threads, persistent over tiles):
-//   warp 0     TMA producer, fills a ring of `stages` {A 16 KB, B BN*128 B} slots
-//   warp 1     allocates TMEM, issues tcgen05.mma kind::tf32 (4 per slot, K = 8 each)
-//   warps 2-9  epilogue: TMEM -> registers -> bias/activation/mask -> global (two warps per TMEM
-//              lane quarter; a lone warp per scheduler is latency-bound on narrow layers)
-// Two TMEM accumulators (2 x BN columns) let the epilogue of tile i overlap the
-// main loop of tile i+1.
+// Warp roles (352 threads, persistent over tiles):
+//   warp 0        TMA producer (one thread), fills the ring of slots
+//   warp 1        allocates TMEM; one thread issues tcgen05.mma kind::tf32 (mma_issuer())
+//   warp 10       second issuing thread for single-CTA tiles with many slots
+//   warps 2-9     epilogue: TMEM -> registers -> bias / activation / mask [/ column sums / 2x2 max pool]
+//                 -> global, through TMA stores or coalesced per-lane stores (two warps per TMEM lane quarter)
+// Two TMEM accumulator sets let the epilogue of tile i overlap the main loop of tile i+1.
 #include <stdlib.h>
 
 #include "pcl_internal.h"
