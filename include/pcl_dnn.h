@@ -103,7 +103,10 @@ int pcl_conv_fwd_pool(const pcl_conv_desc* d, const float* x, const float* w, co
  *                 of dy[n,p,q,k] * w[k,r,s,c]
  * dy: NPQK in, w: KRSC in, dx: NHWC out (every element written; positions no
  * tap reaches get 0).  relu_mask_src: NULL, or an NHWC tensor of dx's shape
- * (the layer's input, i.e. a ReLU output): dx is zeroed where it is <= 0. */
+ * (the layer's input, i.e. a ReLU output): dx is zeroed where it is <= 0.
+ * Workspace: pcl_conv_workspace_bytes(d, PCL_PASS_BWD_DATA) (room for a flipped,
+ * transposed copy of w, the "transpose-weights" of Sec. 2.3; the tensor-core path
+ * reads w in place instead when C is a multiple of 32, the workspace must still be given). */
 int pcl_conv_bwd_data(const pcl_conv_desc* d, const float* dy, const float* w,
                       const float* relu_mask_src, float* dx,
                       void* ws, size_t ws_bytes, void* cuda_stream);
