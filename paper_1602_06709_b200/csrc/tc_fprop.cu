@@ -820,6 +820,10 @@ void choose_box(int P, int Q, int N, bool pool, int* bw_log2, int* bh_log2) {
 }
 
 int choose_bn(int Kout, long m_tiles, int sm_count) {
+    if (const char* v = getenv("PCL_BN")) {          // tuning hook: a multiple of 32 in [32, 256]
+        const int bn = atoi(v);
+        if (bn >= 32 && bn <= 256 && bn % 32 == 0) return bn;
+    }
     // Score = (fraction of SM-slots the tiles fill, counting whole waves) x (tensor efficiency of the width):
     // an MMA costs max(N/2, ~52) cycles, so N < 128 wastes the pipe, and wider tiles re-read A less often.
     const int k32 = (Kout + 31) / 32 * 32;
