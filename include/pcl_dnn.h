@@ -92,9 +92,13 @@ int pcl_conv_fwd(const pcl_conv_desc* d, const float* x, const float* w, const f
  * commutes with adding the bias and with a monotone activation), which saves re-reading y;
  * other shapes run the pooling kernel after the convolution.  out_h and out_w must be even
  * (PCL_ERR_UNSUPPORTED_SHAPE otherwise).  y_pool: [N][out_h/2][out_w/2][K] out, 16-byte aligned.
+ * pool_codes: NULL, or [N][out_h/2][out_w/2][K] bytes out (16-byte aligned): per pooled element the
+ * position code of its window, bits 0-1 = position of the first maximum in row-major window order
+ * (0: 2p,2q  1: 2p,2q+1  2: 2p+1,2q  3: 2p+1,2q+1), bit 2 set where that maximum is <= 0.  With the
+ * codes, pcl_maxpool2x2_bwd_codes() routes the gradient without reading y again.
  * Workspace as pcl_conv_fwd(). */
 int pcl_conv_fwd_pool(const pcl_conv_desc* d, const float* x, const float* w, const float* bias,
-                      float* y, float* y_pool, int act,
+                      float* y, float* y_pool, unsigned char* pool_codes, int act,
                       void* ws, size_t ws_bytes, void* cuda_stream);
 
 /* Backpropagation (the "Backpropagation" update rule of Sec. 2.1, gather form):
@@ -172,6 +176,17 @@ size_t pcl_maxpool2x2_bwd_colsum_workspace_bytes(int N, int H, int W, int C);
 int pcl_maxpool2x2_bwd_colsum(int N, int H, int W, int C, const float* x, const float* dy,
                               const float* relu_mask_src, float* dx, float* dx_colsum,
                               void* ws, size_t ws_bytes, void* cuda_stream);
+/* Pooling with position codes (see pcl_conv_fwd_pool): the forward pass also writes codes[n,p,q,c];
+ * the backward pass takes the codes instead of x:  dx gets dy at the coded position of each window
+ * and 0 elsewhere; relu_mask != 0: windows whose code has bit 2 set (maximum <= 0, i.e. the ReLU
+ * that produced x was inactive there) get 0 everywhere, which equals pcl_maxpool2x2_bwd() with
+ * relu_mask_src = x.  dx_colsum: NULL, or [C] out = sum_{n,h,w} dx[n,h,w,c] (deterministic), then the
+ * workspace of pcl_maxpool2x2_bwd_colsum_workspace_bytes(N, H, W, C) is needed. */
+int pcl_maxpool2x2_fwd_codes(int N, int H, int W, int C, const float* x, float* y, unsigned char* codes,
+                             void* cuda_stream);
+int pcl_maxpool2x2_bwd_codes(int N, int H, int W, int C, const unsigned char* codes, const float* dy,
+                             int relu_mask, float* dx, float* dx_colsum,
+                             void* ws, size_t ws_bytes, void* cuda_stream);
 /* loss = -(1/N) sum_n log softmax(logits[n,:])[labels[n]]  (device scalar, overwritten)
  * dlogits = (softmax(logits) - onehot(labels)) / N.  labels: device int32 [N]. */
 int pcl_softmax_xent(int N, int K, const float* logits, const int* labels,

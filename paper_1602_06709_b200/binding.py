@@ -28,6 +28,7 @@ EXPORTS = [
     "pcl_last_device_status", "pcl_launch_count", "pcl_status_string", "pcl_profile_begin", "pcl_profile_end", "pcl_conv_bwd_data_noalloc", "pcl_noalloc_scratch_bytes",
     "pcl_conv_bwd_data_colsum_workspace_bytes", "pcl_conv_bwd_data_colsum",
     "pcl_maxpool2x2_bwd_colsum_workspace_bytes", "pcl_maxpool2x2_bwd_colsum", "pcl_conv_fwd_pool",
+    "pcl_maxpool2x2_fwd_codes", "pcl_maxpool2x2_bwd_codes",
 ]
 
 
@@ -68,7 +69,9 @@ def lib() -> ctypes.CDLL:
         L.pcl_fc_workspace_bytes.restype = sz
         L.pcl_conv_fwd.argtypes = [dp, vp, vp, vp, vp, ci, vp, sz, vp]
         L.pcl_conv_bwd_data.argtypes = [dp, vp, vp, vp, vp, vp, sz, vp]
-        L.pcl_conv_fwd_pool.argtypes = [dp, vp, vp, vp, vp, vp, ci, vp, sz, vp]
+        L.pcl_conv_fwd_pool.argtypes = [dp, vp, vp, vp, vp, vp, vp, ci, vp, sz, vp]
+        L.pcl_maxpool2x2_fwd_codes.argtypes = [ci, ci, ci, ci, vp, vp, vp, vp]
+        L.pcl_maxpool2x2_bwd_codes.argtypes = [ci, ci, ci, ci, vp, vp, ci, vp, vp, vp, sz, vp]
         L.pcl_conv_bwd_weights.argtypes = [dp, vp, vp, vp, vp, ci, vp, sz, vp]
         L.pcl_fc_fwd.argtypes = [ci, ci, ci, vp, vp, vp, vp, ci, vp, sz, vp]
         L.pcl_fc_bwd.argtypes = [ci, ci, ci, vp, vp, vp, ci, vp, vp, vp, vp, vp, sz, vp]
@@ -149,10 +152,21 @@ def conv_fwd(d, x, w, bias, y, act=ACT_NONE, ws=None, stream=None):
            "pcl_conv_fwd")
 
 
-def conv_fwd_pool(d, x, w, bias, y, y_pool, act=ACT_NONE, ws=None, stream=None):
+def conv_fwd_pool(d, x, w, bias, y, y_pool, act=ACT_NONE, ws=None, stream=None, pool_codes=None):
     wp, wb = _ws(ws)
-    _check(lib().pcl_conv_fwd_pool(ctypes.byref(d), _ptr(x), _ptr(w), _ptr(bias), _ptr(y), _ptr(y_pool), act, wp, wb,
-                                   _stream(stream)), "pcl_conv_fwd_pool")
+    _check(lib().pcl_conv_fwd_pool(ctypes.byref(d), _ptr(x), _ptr(w), _ptr(bias), _ptr(y), _ptr(y_pool),
+                                   _ptr(pool_codes), act, wp, wb, _stream(stream)), "pcl_conv_fwd_pool")
+
+
+def maxpool2x2_fwd_codes(N, H, W, C, x, y, codes, stream=None):
+    _check(lib().pcl_maxpool2x2_fwd_codes(N, H, W, C, _ptr(x), _ptr(y), _ptr(codes), _stream(stream)),
+           "pcl_maxpool2x2_fwd_codes")
+
+
+def maxpool2x2_bwd_codes(N, H, W, C, codes, dy, relu_mask, dx, dx_colsum=None, ws=None, stream=None):
+    wp, wb = _ws(ws)
+    _check(lib().pcl_maxpool2x2_bwd_codes(N, H, W, C, _ptr(codes), _ptr(dy), int(bool(relu_mask)), _ptr(dx),
+                                          _ptr(dx_colsum), wp, wb, _stream(stream)), "pcl_maxpool2x2_bwd_codes")
 
 
 def conv_bwd_data(d, dy, w, relu_mask_src, dx, ws=None, stream=None):

@@ -143,10 +143,20 @@ __global__ void __launch_bounds__(256) colsum_kernel(const float* __restrict__ m
     }
 }
 
+// Position code of a 2x2 window (a b / c d): bits 0-1 = position of the first maximum in row-major order, bit 2 set
+// where that maximum is <= 0 (what a ReLU mask on the pooled layer would zero).
+__device__ __forceinline__ unsigned int pool_code1(float a, float b, float c, float d) {
+    unsigned int arg = 0; float best = a;
+    if (b > best) { best = b; arg = 1; }
+    if (c > best) { best = c; arg = 2; }
+    if (d > best) { best = d; arg = 3; }
+    return arg | (best > 0.f ? 0u : 4u);
+}
+
 // 2x2 / stride-2 max pooling, NHWC, one thread per (output pixel, 4 channels)
 template <int VEC>
 __global__ void __launch_bounds__(256) maxpool_fwd_kernel(const float* __restrict__ x, float* __restrict__ y, int N,
-                                                          int H, int W, int C) {
+                                                          int H, int W, int C, unsigned char* __restrict__ idx = nullptr) {
     const int Po = H / 2, Qo = W / 2, Cv = C / VEC;
     const size_t total = size_t(N) * Po * Qo * Cv;
     const size_t stride = size_t(gridDim.x) * blockDim.x;
@@ -165,8 +175,14 @@ __global__ void __launch_bounds__(256) maxpool_fwd_kernel(const float* __restric
             o.x = fmaxf(fmaxf(a.x, b.x), fmaxf(c.x, d.x)); o.y = fmaxf(fmaxf(a.y, b.y), fmaxf(c.y, d.y));
             o.z = fmaxf(fmaxf(a.z, b.z), fmaxf(c.z, d.z)); o.w = fmaxf(fmaxf(a.w, b.w), fmaxf(c.w, d.w));
             *reinterpret_cast<float4*>(dst) = o;
+            if (idx) {
+                unsigned int code = pool_code1(a.x, b.x, c.x, d.x) | (pool_code1(a.y, b.y, c.y, d.y) << 8) |
+                                    (pool_code1(a.z, b.z, c.z, d.z) << 16) | (pool_code1(a.w, b.w, c.w, d.w) << 24);
+                *reinterpret_cast<unsigned int*>(idx + (dst - y)) = code;
+            }
         } else {
             dst[0] = fmaxf(fmaxf(src[0], src[C]), fmaxf(src[size_t(W) * C], src[size_t(W) * C + C]));
+            if (idx) idx[dst - y] = static_cast<unsigned char>(pool_code1(src[0], src[C], src[size_t(W) * C], src[size_t(W) * C + C]));
         }
     }
 }
@@ -241,6 +257,67 @@ __global__ void __launch_bounds__(256) maxpool_bwd_kernel(const float* __restric
                 if (!(mask[off + rowp + C] > 0.f)) od = 0.f;
             }
             dx[off] = oa; dx[off + C] = ob; dx[off + rowp] = oc; dx[off + rowp + C] = od;
+        }
+    }
+    if (VEC == 4 && colsum_rows) {
+        __shared__ float4 red[256];
+        red[threadIdx.x] = csum;
+        __syncthreads();
+        const int Cv4 = C / 4;
+        if (threadIdx.x < Cv4) {
+            float4 a = red[threadIdx.x];
+            for (int t = threadIdx.x + Cv4; t < 256; t += Cv4) {
+                a.x += red[t].x; a.y += red[t].y; a.z += red[t].z; a.w += red[t].w;
+            }
+            *reinterpret_cast<float4*>(colsum_rows + size_t(blockIdx.x) * C + threadIdx.x * 4) = a;
+        }
+    }
+}
+
+// Pooling backward from the position codes the forward pass recorded (no pass over the pooled layer's input):
+// dx gets dy at the coded position of each window and 0 elsewhere; with `relu`, windows whose code has bit 2 set
+// (maximum <= 0) get 0 everywhere.  Column sums as in maxpool_bwd_kernel.
+template <int VEC>
+__global__ void __launch_bounds__(256) maxpool_bwd_idx_kernel(const unsigned char* __restrict__ idx,
+                                                              const float* __restrict__ dy, int relu,
+                                                              float* __restrict__ dx, int N, int H, int W, int C,
+                                                              float* __restrict__ colsum_rows = nullptr) {
+    const int Po = H / 2, Qo = W / 2, Cv = C / VEC;
+    const size_t total = size_t(N) * Po * Qo * Cv;
+    const size_t stride = size_t(gridDim.x) * blockDim.x;
+    const size_t rowp = size_t(W) * C;
+    const unsigned int kill = relu ? 4u : 0u;
+    float4 csum = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (size_t i = size_t(blockIdx.x) * blockDim.x + threadIdx.x; i < total; i += stride) {
+        const int cv = int(i % Cv); size_t t = i / Cv;
+        const int q = int(t % Qo); t /= Qo;
+        const int p = int(t % Po); const size_t n = t / Po;
+        const size_t off = ((n * H + 2 * p) * W + 2 * q) * C + cv * VEC;
+        const size_t po = ((n * Po + p) * Qo + q) * C + cv * VEC;
+        if (VEC == 4) {
+            const float4 gv = __ldcs(reinterpret_cast<const float4*>(dy + po));
+            const unsigned int code = __ldcs(reinterpret_cast<const unsigned int*>(idx + po));
+            const float g[4] = {gv.x, gv.y, gv.z, gv.w};
+            float o[4][4];      // [position][channel]
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+                const unsigned int cc = (code >> (8 * c)) & 0xffu;
+                const float gg = (cc & kill) ? 0.f : g[c];
+#pragma unroll
+                for (int e = 0; e < 4; ++e) o[e][c] = (cc & 3u) == unsigned(e) ? gg : 0.f;
+                (&csum.x)[c] += gg;
+            }
+            __stcs(reinterpret_cast<float4*>(dx + off), make_float4(o[0][0], o[0][1], o[0][2], o[0][3]));
+            __stcs(reinterpret_cast<float4*>(dx + off + C), make_float4(o[1][0], o[1][1], o[1][2], o[1][3]));
+            __stcs(reinterpret_cast<float4*>(dx + off + rowp), make_float4(o[2][0], o[2][1], o[2][2], o[2][3]));
+            __stcs(reinterpret_cast<float4*>(dx + off + rowp + C), make_float4(o[3][0], o[3][1], o[3][2], o[3][3]));
+        } else {
+            const unsigned int cc = idx[po];
+            const float gg = (cc & kill) ? 0.f : dy[po];
+            dx[off] = (cc & 3u) == 0u ? gg : 0.f;
+            dx[off + C] = (cc & 3u) == 1u ? gg : 0.f;
+            dx[off + rowp] = (cc & 3u) == 2u ? gg : 0.f;
+            dx[off + rowp + C] = (cc & 3u) == 3u ? gg : 0.f;
         }
     }
     if (VEC == 4 && colsum_rows) {
@@ -457,14 +534,31 @@ int launch_colsum(const float* m, size_t rows, int K, float* partial, float* out
     return PCL_OK;
 }
 
-int launch_maxpool_fwd(int N, int H, int W, int C, const float* x, float* y, cudaStream_t st) {
+int launch_maxpool_fwd(int N, int H, int W, int C, const float* x, float* y, cudaStream_t st, unsigned char* idx) {
     const size_t outs = size_t(N) * (H / 2) * (W / 2);
     {
         LaunchScope scope(KID_MAXPOOL_FWD, 20.0 * double(outs) * C, st);
         if (C % 4 == 0)
-            maxpool_fwd_kernel<4><<<grid_for(outs * (C / 4), 256), 256, 0, st>>>(x, y, N, H, W, C);
+            maxpool_fwd_kernel<4><<<grid_for(outs * (C / 4), 256), 256, 0, st>>>(x, y, N, H, W, C, idx);
         else
-            maxpool_fwd_kernel<1><<<grid_for(outs * C, 256), 256, 0, st>>>(x, y, N, H, W, C);
+            maxpool_fwd_kernel<1><<<grid_for(outs * C, 256), 256, 0, st>>>(x, y, N, H, W, C, idx);
+    }
+    return PCL_CHECK_LAUNCH();
+}
+
+// colsum_rows: null, or [maxpool_bwd_colsum_rows()][C] (then C % 4 == 0 and C/4 divides 256)
+int launch_maxpool_bwd_idx(int N, int H, int W, int C, const unsigned char* idx, const float* dy, int relu, float* dx,
+                           float* colsum_rows, cudaStream_t st) {
+    const size_t outs = size_t(N) * (H / 2) * (W / 2);
+    if (colsum_rows && maxpool_bwd_colsum_rows(N, H, W, C) == 0) return PCL_ERR_UNSUPPORTED_SHAPE;
+    {
+        // per output: 1 code byte + 1 dy read + 4 dx written
+        LaunchScope scope(KID_MAXPOOL_BWD, 21.0 * double(outs) * C, st);
+        if (C % 4 == 0)
+            maxpool_bwd_idx_kernel<4><<<grid_for(outs * (C / 4), 256, 16), 256, 0, st>>>(idx, dy, relu, dx, N, H, W, C,
+                                                                                          colsum_rows);
+        else
+            maxpool_bwd_idx_kernel<1><<<grid_for(outs * C, 256), 256, 0, st>>>(idx, dy, relu, dx, N, H, W, C);
     }
     return PCL_CHECK_LAUNCH();
 }

@@ -238,7 +238,8 @@ size_t pcl_fc_workspace_bytes(int N, int C, int K, int pass) {
 // Forward pass; y_pool != nullptr: also the 2x2 window maxima of y, fused into the tensor-core epilogue where
 // the shape allows it and computed by the pooling kernel otherwise.
 static int conv_fwd_impl(const pcl_conv_desc* d, const float* x, const float* w, const float* bias, float* y,
-                         float* y_pool, int act, void* ws, size_t ws_bytes, void* cuda_stream) {
+                         float* y_pool, unsigned char* pool_codes, int act, void* ws, size_t ws_bytes,
+                         void* cuda_stream) {
     int P, Q;
     int rc = check_desc(d, &P, &Q);
     if (rc != PCL_OK) return rc;
@@ -246,6 +247,7 @@ static int conv_fwd_impl(const pcl_conv_desc* d, const float* x, const float* w,
     if (act != PCL_ACT_NONE && act != PCL_ACT_RELU && act != PCL_ACT_SIGMOID) return PCL_ERR_BAD_ARG;
     if (!aligned16(x) || !aligned16(w) || !aligned16(y) || !aligned16(bias) || !aligned16(y_pool)) return PCL_ERR_MISALIGNED;
     if (y_pool && (P % 2 != 0 || Q % 2 != 0)) return PCL_ERR_UNSUPPORTED_SHAPE;
+    if (pool_codes && (!y_pool || !aligned16(pool_codes))) return y_pool ? PCL_ERR_MISALIGNED : PCL_ERR_BAD_ARG;
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
     if (few_channel_path_for(*d, PCL_PASS_FWD)) {
         const size_t xs_bytes = staged_x_bytes(*d), need = xs_bytes + staged_w_bytes(*d);
@@ -261,11 +263,11 @@ static int conv_fwd_impl(const pcl_conv_desc* d, const float* x, const float* w,
         // the staged layer: 32 "channels" per pixel window (S*4 carry weight, the rest meets zero weights)
         TcFpropArgs a{xs, w4, bias, nullptr, y, d->N, Hp, Q, 32, d->K, d->R, 1, 0, 0, P, Q, act};
         a.in_stride_w = 4; a.in_stride_h = long(Wp) * 4; a.in_stride_n = long(Hp) * Wp * 4;
-        if (y_pool && tc_fprop_can_pool(a)) { a.pool_out = y_pool; y_pool = nullptr; }
+        if (y_pool && tc_fprop_can_pool(a)) { a.pool_out = y_pool; a.pool_idx = pool_codes; y_pool = nullptr; }
         rc = launch_tc_fprop(a, st);
     } else if (tensor_path_for(*d, PCL_PASS_FWD)) {
         TcFpropArgs a{x, w, bias, nullptr, y, d->N, d->H, d->W, d->C, d->K, d->R, d->S, d->pad_h, d->pad_w, P, Q, act};
-        if (y_pool && tc_fprop_can_pool(a)) { a.pool_out = y_pool; y_pool = nullptr; }
+        if (y_pool && tc_fprop_can_pool(a)) { a.pool_out = y_pool; a.pool_idx = pool_codes; y_pool = nullptr; }
         rc = launch_tc_fprop(a, st);
     } else if (g_path.load() == PCL_PATH_TENSOR) {
         return PCL_ERR_UNSUPPORTED_SHAPE;
@@ -273,19 +275,20 @@ static int conv_fwd_impl(const pcl_conv_desc* d, const float* x, const float* w,
         rc = launch_generic_fwd(*d, P, Q, x, w, bias, y, act, st);
     }
     if (rc != PCL_OK) return rc;
-    if (y_pool) return launch_maxpool_fwd(d->N, P, Q, d->K, y, y_pool, st);     // not fused above
+    if (y_pool) return launch_maxpool_fwd(d->N, P, Q, d->K, y, y_pool, st, pool_codes);     // not fused above
     return PCL_OK;
 }
 
 int pcl_conv_fwd(const pcl_conv_desc* d, const float* x, const float* w, const float* bias, float* y, int act,
                  void* ws, size_t ws_bytes, void* cuda_stream) {
-    return conv_fwd_impl(d, x, w, bias, y, nullptr, act, ws, ws_bytes, cuda_stream);
+    return conv_fwd_impl(d, x, w, bias, y, nullptr, nullptr, act, ws, ws_bytes, cuda_stream);
 }
 
 int pcl_conv_fwd_pool(const pcl_conv_desc* d, const float* x, const float* w, const float* bias, float* y,
-                      float* y_pool, int act, void* ws, size_t ws_bytes, void* cuda_stream) {
+                      float* y_pool, unsigned char* pool_codes, int act, void* ws, size_t ws_bytes,
+                      void* cuda_stream) {
     if (!y_pool) return PCL_ERR_BAD_ARG;
-    return conv_fwd_impl(d, x, w, bias, y, y_pool, act, ws, ws_bytes, cuda_stream);
+    return conv_fwd_impl(d, x, w, bias, y, y_pool, pool_codes, act, ws, ws_bytes, cuda_stream);
 }
 
 int pcl_conv_bwd_data(const pcl_conv_desc* d, const float* dy, const float* w, const float* relu_mask_src, float* dx,
@@ -419,6 +422,39 @@ int pcl_maxpool2x2_bwd_colsum(int N, int H, int W, int C, const float* x, const 
         return launch_colsum(sum_rows, size_t(rows), C, partial, dx_colsum, st);
     }
     int rc = launch_maxpool_bwd(N, H, W, C, x, dy, relu_mask_src, dx, st);
+    if (rc != PCL_OK) return rc;
+    return launch_colsum(dx, size_t(N) * H * W, C, static_cast<float*>(ws), dx_colsum, st);
+}
+
+int pcl_maxpool2x2_fwd_codes(int N, int H, int W, int C, const float* x, float* y, unsigned char* codes,
+                             void* cuda_stream) {
+    if (N <= 0 || H <= 0 || W <= 0 || C <= 0 || !x || !y || !codes) return PCL_ERR_BAD_ARG;
+    if ((H | W) & 1) return PCL_ERR_UNSUPPORTED_SHAPE;
+    if (!aligned16(x) || !aligned16(y) || !aligned16(codes)) return PCL_ERR_MISALIGNED;
+    return launch_maxpool_fwd(N, H, W, C, x, y, static_cast<cudaStream_t>(cuda_stream), codes);
+}
+
+int pcl_maxpool2x2_bwd_codes(int N, int H, int W, int C, const unsigned char* codes, const float* dy, int relu_mask,
+                             float* dx, float* dx_colsum, void* ws, size_t ws_bytes, void* cuda_stream) {
+    if (N <= 0 || H <= 0 || W <= 0 || C <= 0 || !codes || !dy || !dx) return PCL_ERR_BAD_ARG;
+    if ((H | W) & 1) return PCL_ERR_UNSUPPORTED_SHAPE;
+    if (!aligned16(codes) || !aligned16(dy) || !aligned16(dx) || !aligned16(dx_colsum)) return PCL_ERR_MISALIGNED;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    if (!dx_colsum) return launch_maxpool_bwd_idx(N, H, W, C, codes, dy, relu_mask, dx, nullptr, st);
+    const size_t need = pcl_maxpool2x2_bwd_colsum_workspace_bytes(N, H, W, C);
+    if (need > 0) {
+        if (!ws || ws_bytes < need) return PCL_ERR_WORKSPACE;
+        if (reinterpret_cast<uintptr_t>(ws) & 255) return PCL_ERR_MISALIGNED;
+    }
+    const long rows = maxpool_bwd_colsum_rows(N, H, W, C);
+    if (rows > 0) {
+        float* sum_rows = static_cast<float*>(ws);
+        int rc = launch_maxpool_bwd_idx(N, H, W, C, codes, dy, relu_mask, dx, sum_rows, st);
+        if (rc != PCL_OK) return rc;
+        float* partial = reinterpret_cast<float*>(static_cast<char*>(ws) + align_up(size_t(rows) * C * 4, 256));
+        return launch_colsum(sum_rows, size_t(rows), C, partial, dx_colsum, st);
+    }
+    int rc = launch_maxpool_bwd_idx(N, H, W, C, codes, dy, relu_mask, dx, nullptr, st);
     if (rc != PCL_OK) return rc;
     return launch_colsum(dx, size_t(N) * H * W, C, static_cast<float*>(ws), dx_colsum, st);
 }

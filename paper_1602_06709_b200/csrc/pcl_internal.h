@@ -72,6 +72,9 @@ struct TcFpropArgs {
     // Optional fused 2x2 / stride-2 max pooling of the output: pool_out [N][P/2][Q/2][Kout] gets the window maxima
     // of `out` (after bias and activation).  Needs even P and Q and Kout % 4 == 0 (tc_fprop_can_pool()).
     float* pool_out = nullptr;
+    // with pool_out: [N][P/2][Q/2][Kout] bytes, bits 0-1 = position of the window's first maximum (row-major), bit 2 set
+    // where that maximum is <= 0 (what a ReLU mask would zero); lets the pooling backward pass skip reading `out`
+    unsigned char* pool_idx = nullptr;
     // wt_mn_major != 0: `wt` is laid out [Cin][R*S][Kout] (output maps innermost), i.e. a layer's own KRSC weights
     // seen from its backward-data pass (reduction over the layer's K, columns = the layer's C): the kernel then
     // reads B as an MN-major operand and no transposed copy is needed.  Needs Kout % 32 == 0.
@@ -133,7 +136,10 @@ int launch_act_grad(float* dy, const float* y, size_t n, int act, cudaStream_t s
 // out[k] = sum_rows m[row][k]; partial: [colsum_splits(rows)][K] workspace
 int colsum_splits(size_t rows);
 int launch_colsum(const float* m, size_t rows, int K, float* partial, float* out, cudaStream_t st);
-int launch_maxpool_fwd(int N, int H, int W, int C, const float* x, float* y, cudaStream_t st);
+// idx (optional): per output the position code of its window (bits 0-1 first maximum, bit 2: maximum <= 0)
+int launch_maxpool_fwd(int N, int H, int W, int C, const float* x, float* y, cudaStream_t st, unsigned char* idx = nullptr);
+int launch_maxpool_bwd_idx(int N, int H, int W, int C, const unsigned char* idx, const float* dy, int relu, float* dx,
+                           float* colsum_rows, cudaStream_t st);
 int launch_maxpool_bwd(int N, int H, int W, int C, const float* x, const float* dy, const float* mask, float* dx,
                        cudaStream_t st);
 // The same with fused per-block column sums of dx: colsum_rows is [maxpool_bwd_colsum_rows(N,H,W,C)][C]; returns 0

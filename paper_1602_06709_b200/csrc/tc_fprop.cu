@@ -74,6 +74,8 @@ struct FpropParams {
     const float* mask_src;
     float* out;
     int tma_store;              // the epilogue writes `out` with TMA stores from the staging tiles (tmOut is valid)
+    unsigned char* pool_idx;    // optional, with pool_out: per pooled element the position of the maximum (bits 0-1) and bit 2
+                                // if that maximum is <= 0
     float* pool_out;            // optional [N][P/2][Q/2][Kout]: 2x2 window maxima of the output
     float* colsum_rows;         // optional [m_tiles * MT * 4][Kout] per-(box, quarter) column sums of the output
     unsigned int* status;       // device status word
@@ -135,6 +137,29 @@ struct IssuerCtx {
     uint32_t tmem_base, b_bytes, step_bytes, stage_bytes;
     int first_tile, tile_stride, total_tiles, kiters;
 };
+
+// 2x2 pooling of four channels: running maximum and its position e (0..3, row-major in the window; the FIRST
+// maximum wins, as in the pooling kernels), one position per channel in the bytes of `arg`.
+__device__ __forceinline__ void pool_take(float4& m, uint32_t& arg, const float4 t, const uint32_t e) {
+    if (t.x > m.x) { m.x = t.x; arg = (arg & 0xffffff00u) | e; }
+    if (t.y > m.y) { m.y = t.y; arg = (arg & 0xffff00ffu) | (e << 8); }
+    if (t.z > m.z) { m.z = t.z; arg = (arg & 0xff00ffffu) | (e << 16); }
+    if (t.w > m.w) { m.w = t.w; arg = (arg & 0x00ffffffu) | (e << 24); }
+}
+// position bytes plus bit 2 where the maximum is not positive (what a ReLU mask on the pooled layer would zero)
+__device__ __forceinline__ uint32_t pool_code(const float4 m, const uint32_t arg) {
+    return arg | (m.x > 0.f ? 0u : 4u) | (m.y > 0.f ? 0u : 4u << 8) | (m.z > 0.f ? 0u : 4u << 16) | (m.w > 0.f ? 0u : 4u << 24);
+}
+__device__ __forceinline__ float4 finish4(float4 o, const float4 b, const int act) {
+    o.x += b.x; o.y += b.y; o.z += b.z; o.w += b.w;
+    if (act == PCL_ACT_RELU) {
+        o.x = fmaxf(o.x, 0.f); o.y = fmaxf(o.y, 0.f); o.z = fmaxf(o.z, 0.f); o.w = fmaxf(o.w, 0.f);
+    } else if (act == PCL_ACT_SIGMOID) {
+        o.x = 1.f / (1.f + __expf(-o.x)); o.y = 1.f / (1.f + __expf(-o.y));
+        o.z = 1.f / (1.f + __expf(-o.z)); o.w = 1.f / (1.f + __expf(-o.w));
+    }
+    return o;
+}
 
 // v += the 32 x 32 block at `taddr` (the second issuer's accumulator).
 __device__ __forceinline__ void add_second_accumulator(uint32_t taddr, uint32_t (&v)[32]) {
@@ -627,19 +652,22 @@ tc_fprop_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                         for (int half = 0; half < 2; ++half) {
                             const int wdx = (lane >> 3) + 4 * half;
                             const int r0 = ((wdx & ((1 << (lb - 1)) - 1)) << 1) | ((wdx >> (lb - 1)) << (lb + 1));
-                            float4 m = make_float4(-INFINITY, -INFINITY, -INFINITY, -INFINITY);
+                            float4 m = ld_shared_v4(stg + r0 * 128 + (((lane & 7) ^ (r0 & 7)) * 16));
+                            uint32_t arg = 0;
 #pragma unroll
-                            for (int e = 0; e < 4; ++e) {
+                            for (int e = 1; e < 4; ++e) {
                                 const int rr = r0 | (e & 1) | ((e >> 1) << lb);
-                                const float4 t4 = ld_shared_v4(stg + rr * 128 + (((lane & 7) ^ (rr & 7)) * 16));
-                                m.x = fmaxf(m.x, t4.x); m.y = fmaxf(m.y, t4.y); m.z = fmaxf(m.z, t4.z); m.w = fmaxf(m.w, t4.w);
+                                pool_take(m, arg, ld_shared_v4(stg + rr * 128 + (((lane & 7) ^ (rr & 7)) * 16)), e);
                             }
                             const int wrow = srow + r0;
                             const int wq = it.qi * p.tw + (wrow & (bw - 1)) + h * p.half_dq;
                             const int wp = it.pi * p.th + ((wrow >> p.bw_log2) & (bh - 1)) + h * p.half_dp;
                             const int wn = ni * p.tn + (wrow >> (p.bw_log2 + p.bh_log2));
-                            if (col < p.Kout && wq < p.Q && wp < p.P && wn < p.N)
-                                *reinterpret_cast<float4*>(p.pool_out + ((static_cast<size_t>(wn) * (p.P >> 1) + (wp >> 1)) * (p.Q >> 1) + (wq >> 1)) * p.Kout + col) = m;
+                            if (col < p.Kout && wq < p.Q && wp < p.P && wn < p.N) {
+                                const size_t po = ((static_cast<size_t>(wn) * (p.P >> 1) + (wp >> 1)) * (p.Q >> 1) + (wq >> 1)) * p.Kout + col;
+                                *reinterpret_cast<float4*>(p.pool_out + po) = m;
+                                if (p.pool_idx) *reinterpret_cast<uint32_t*>(p.pool_idx + po) = pool_code(m, arg);
+                            }
                         }
                     }
                 }
@@ -732,26 +760,23 @@ tc_fprop_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                             for (int half = 0; half < 2; ++half) {
                                 const int wdx = (lane >> 3) + 4 * half;
                                 const int r0 = ((wdx & ((1 << (lb - 1)) - 1)) << 1) | ((wdx >> (lb - 1)) << (lb + 1));
-                                float4 m = make_float4(-INFINITY, -INFINITY, -INFINITY, -INFINITY);
+                                // (the staged values are raw accumulators here: each is finished like `o` before it is compared)
+                                float4 m = finish4(ld_shared_v4(stg + r0 * 128 + (((lane & 7) ^ (r0 & 7)) * 16)), b, p.act);
+                                uint32_t arg = 0;
 #pragma unroll
-                                for (int e = 0; e < 4; ++e) {
+                                for (int e = 1; e < 4; ++e) {
                                     const int rr = r0 | (e & 1) | ((e >> 1) << lb);
-                                    const float4 t4 = ld_shared_v4(stg + rr * 128 + (((lane & 7) ^ (rr & 7)) * 16));
-                                    m.x = fmaxf(m.x, t4.x); m.y = fmaxf(m.y, t4.y); m.z = fmaxf(m.z, t4.z); m.w = fmaxf(m.w, t4.w);
-                                }
-                                m.x += b.x; m.y += b.y; m.z += b.z; m.w += b.w;
-                                if (p.act == PCL_ACT_RELU) {
-                                    m.x = fmaxf(m.x, 0.f); m.y = fmaxf(m.y, 0.f); m.z = fmaxf(m.z, 0.f); m.w = fmaxf(m.w, 0.f);
-                                } else if (p.act == PCL_ACT_SIGMOID) {
-                                    m.x = 1.f / (1.f + __expf(-m.x)); m.y = 1.f / (1.f + __expf(-m.y));
-                                    m.z = 1.f / (1.f + __expf(-m.z)); m.w = 1.f / (1.f + __expf(-m.w));
+                                    pool_take(m, arg, finish4(ld_shared_v4(stg + rr * 128 + (((lane & 7) ^ (rr & 7)) * 16)), b, p.act), e);
                                 }
                                 const int wrow = quarter * 32 + r0;       // the window's first pixel inside the box
                                 const int wq = it.qi * p.tw + (wrow & (bw - 1)) + h * p.half_dq;
                                 const int wp = it.pi * p.th + ((wrow >> p.bw_log2) & (bh - 1)) + h * p.half_dp;
                                 const int wn = ni * p.tn + (wrow >> (p.bw_log2 + p.bh_log2));
-                                if (wq < p.Q && wp < p.P && wn < p.N)
-                                    *reinterpret_cast<float4*>(p.pool_out + ((static_cast<size_t>(wn) * (p.P >> 1) + (wp >> 1)) * (p.Q >> 1) + (wq >> 1)) * p.Kout + col) = m;
+                                if (wq < p.Q && wp < p.P && wn < p.N) {
+                                    const size_t po = ((static_cast<size_t>(wn) * (p.P >> 1) + (wp >> 1)) * (p.Q >> 1) + (wq >> 1)) * p.Kout + col;
+                                    *reinterpret_cast<float4*>(p.pool_out + po) = m;
+                                    if (p.pool_idx) *reinterpret_cast<uint32_t*>(p.pool_idx + po) = pool_code(m, arg);
+                                }
                             }
                         }
                     }
@@ -1043,6 +1068,7 @@ int launch_tc_fprop(const TcFpropArgs& a, cudaStream_t st) {
     p.bias = a.bias; p.mask_src = a.mask_src; p.out = a.out;
     if (a.pool_out && !tc_fprop_can_pool(a)) return PCL_ERR_UNSUPPORTED_SHAPE;
     p.pool_out = a.pool_out;
+    p.pool_idx = a.pool_out ? a.pool_idx : nullptr;
     p.colsum_rows = (a.Kout % 4 == 0) ? a.colsum_rows : nullptr;
     if (a.colsum_rows && !p.colsum_rows) return PCL_ERR_UNSUPPORTED_SHAPE;
     p.status = device_status_ptr();

@@ -138,6 +138,9 @@ class VggA(_HostFeed):
         self.pooled = [torch.empty(N, L.H // 2, L.W // 2, L.K, device=dev) if L.pool else None for L in self.convs]
         self.dy = [torch.empty(N, L.H, L.W, L.K, device=dev) for L in self.convs]           # grad wrt pre-activation
         self.dpooled = [torch.empty(N, L.H // 2, L.W // 2, L.K, device=dev) if L.pool else None for L in self.convs]
+        # position codes of the pooling windows (one byte per pooled element), written by the forward epilogue
+        self.pool_codes = [torch.empty(N, L.H // 2, L.W // 2, L.K, dtype=torch.uint8, device=dev) if L.pool else None
+                           for L in self.convs]
         self.fc_out = [torch.empty(N, K, device=dev) for _, K in fc]
         self.fc_dout = [torch.empty(N, K, device=dev) for _, K in fc]
         self.labels = torch.zeros(N, dtype=torch.int32, device=dev)
@@ -175,7 +178,7 @@ class VggA(_HostFeed):
         for i, L in enumerate(self.convs):
             if L.pool:      # conv -> ReLU -> 2x2 pool, the maxima taken in the convolution's epilogue
                 B.conv_fwd_pool(L.desc, self.layer_input(i), self.conv_w(i), self.conv_b(i), self.y[i], self.pooled[i],
-                                B.ACT_RELU, self.ws)
+                                B.ACT_RELU, self.ws, pool_codes=self.pool_codes[i])
             else:
                 B.conv_fwd(L.desc, self.layer_input(i), self.conv_w(i), self.conv_b(i), self.y[i], B.ACT_RELU, self.ws)
         a = self.pooled[-1].view(self.N, self.flat)
@@ -198,9 +201,9 @@ class VggA(_HostFeed):
             L = self.convs[i]
             # The bias gradient of layer i is the per-map sum of dy[i]; it is formed by whichever kernel writes
             # dy[i] (the pool backward here, or the backward-data pass of layer i+1 below), not by a separate pass.
-            if L.pool:   # gradient through the pool, then through the ReLU (fused mask)
-                B.maxpool2x2_bwd_colsum(self.N, L.H, L.W, L.K, self.y[i], self.dpooled[i], self.y[i], self.dy[i],
-                                        self.conv_db(i), self.ws)
+            if L.pool:   # gradient through the pool, then through the ReLU (fused mask), routed by the position codes
+                B.maxpool2x2_bwd_codes(self.N, L.H, L.W, L.K, self.pool_codes[i], self.dpooled[i], True, self.dy[i],
+                                       self.conv_db(i), self.ws)
             B.conv_bwd_weights(L.desc, self.layer_input(i), self.dy[i], self.conv_dw(i), None, True, self.ws)
             if i > 0:
                 prev = self.convs[i - 1]

@@ -176,6 +176,11 @@ def test_conv_bwd_data_with_fused_column_sums(shape, tiling, monkeypatch):
     assert torch.equal(cs, cs2)
 
 
+def inputs_normal(tag, shape):
+    from paper_1602_06709_b200 import inputs
+    return inputs.normal(inputs.tensor_id(*tag), shape, 1.0)
+
+
 POOL_FUSED_SHAPES = [
     # N, C, K, H, W: even outputs; several image groups; ragged in q/p; C < 4 (few-channel path); halo-eligible 16x16 fits
     (3, 32, 64, 12, 20), (4, 64, 96, 28, 28), (2, 3, 16, 20, 36), (2, 64, 128, 32, 48), (5, 24, 40, 6, 10), (2, 7, 9, 10, 12),
@@ -204,10 +209,19 @@ def test_conv_fwd_with_fused_maxpool(shape, tiling, store, monkeypatch):
         y = torch.full((N, H, W, K), float("nan"), device="cuda")
         yp = torch.full((N, H // 2, W // 2, K), float("nan"), device="cuda")
         ws = G.workspace(B.conv_workspace_bytes(d, B.PASS_FWD))
-        B.conv_fwd_pool(d, G.dev(x), G.dev(w), G.dev(bias), y, yp, act, ws)
+        codes = torch.full((N, H // 2, W // 2, K), 255, dtype=torch.uint8, device="cuda")
+        B.conv_fwd_pool(d, G.dev(x), G.dev(w), G.dev(bias), y, yp, act, ws, pool_codes=codes)
         B.check_device_status()
         G.assert_parity(y.cpu().numpy(), oracle.conv_fwd(s, x, w, bias, oact), "y")
-        assert np.array_equal(yp.cpu().numpy(), oracle.maxpool2x2_fwd(y.cpu().numpy().astype(np.float64)).astype(np.float32))
+        yh = y.cpu().numpy()
+        assert np.array_equal(yp.cpu().numpy(), oracle.maxpool2x2_fwd(yh.astype(np.float64)).astype(np.float32))
+        # the position codes route a gradient exactly as the pooling backward pass does from the y this call wrote
+        g = inputs_normal(("fwdpool_g", N, H, W, K), (N, H // 2, W // 2, K))
+        for relu in (False, True):
+            dx = torch.full((N, H, W, K), float("nan"), device="cuda")
+            B.maxpool2x2_bwd_codes(N, H, W, K, codes, G.dev(g), relu, dx)
+            ref = oracle.maxpool2x2_bwd(yh, g, yh if relu else None)
+            assert np.array_equal(dx.cpu().numpy(), ref.astype(np.float32))
 
 
 def test_conv_fwd_pool_rejects_odd_output():
@@ -220,3 +234,36 @@ def test_conv_fwd_pool_rejects_odd_output():
     y = torch.zeros(1, 7, 8, 8, device="cuda"); yp = torch.zeros(1, 3, 4, 8, device="cuda")
     with pytest.raises(B.PclError):
         B.conv_fwd_pool(d, x, w, None, y, yp, B.ACT_RELU, None)
+
+
+@pytest.mark.parametrize("N,H,W,C", [(2, 8, 6, 8), (3, 14, 14, 5), (2, 28, 28, 64), (1, 4, 4, 1024)])
+def test_maxpool_with_position_codes(N, H, W, C):
+    """Forward pooling that records each window's position code, and the backward pass that takes the codes
+    instead of x: bit-exact against the oracle's pooling passes, with and without the ReLU mask and with the
+    fused column sums (equal to the x-based kernel's)."""
+    import gpu_helpers as G
+    from paper_1602_06709_b200 import binding as B
+    from paper_1602_06709_b200 import inputs
+    x = np.maximum(inputs.normal(inputs.tensor_id("poolcodes", N, H, W, C, "x"), (N, H, W, C), 1.0), 0.0)  # ties at 0
+    dy = inputs.normal(inputs.tensor_id("poolcodes", N, H, W, C, "dy"), (N, H // 2, W // 2, C), 1.0)
+    xt, dyt = G.dev(x), G.dev(dy)
+    yt = torch.full((N, H // 2, W // 2, C), float("nan"), device="cuda")
+    codes = torch.full((N, H // 2, W // 2, C), 255, dtype=torch.uint8, device="cuda")
+    B.maxpool2x2_fwd_codes(N, H, W, C, xt, yt, codes)
+    assert np.array_equal(yt.cpu().numpy(), oracle.maxpool2x2_fwd(x).astype(np.float32))
+    assert int(codes.max()) <= 7
+    for relu in (False, True):
+        dxt = torch.full((N, H, W, C), float("nan"), device="cuda")
+        B.maxpool2x2_bwd_codes(N, H, W, C, codes, dyt, relu, dxt)
+        ref = oracle.maxpool2x2_bwd(x, dy, x if relu else None)
+        assert np.array_equal(dxt.cpu().numpy(), ref.astype(np.float32))
+    cs = torch.full((C,), float("nan"), device="cuda")
+    ws = G.workspace(B.maxpool2x2_bwd_colsum_workspace_bytes(N, H, W, C))
+    dxt = torch.full((N, H, W, C), float("nan"), device="cuda")
+    B.maxpool2x2_bwd_codes(N, H, W, C, codes, dyt, True, dxt, cs, ws)
+    ref = oracle.maxpool2x2_bwd(x, dy, x)
+    assert np.array_equal(dxt.cpu().numpy(), ref.astype(np.float32))
+    G.assert_parity(cs.cpu().numpy(), ref.reshape(-1, C).sum(axis=0), "pool dx column sums")
+    cs_x = torch.empty_like(cs)
+    B.maxpool2x2_bwd_colsum(N, H, W, C, xt, dyt, xt, dxt, cs_x, ws)
+    assert torch.equal(cs, cs_x)
