@@ -195,6 +195,10 @@ int pcl_softmax_xent(int N, int K, const float* logits, const int* labels,
 /* Synchronises the stream, then reads and clears the device status word of the
  * current device.  PCL_OK, PCL_ERR_DEVICE_TIMEOUT or PCL_ERR_CUDA. */
 int pcl_last_device_status(void* cuda_stream);
+/* Which wait gave up when pcl_last_device_status() last returned PCL_ERR_DEVICE_TIMEOUT (0 if it never did):
+ * 0x101 producer waiting for a free slot, 0x102 MMA issuer waiting for operands, 0x103 MMA issuer waiting for a
+ * free accumulator, 0x104 epilogue waiting for an accumulator, 0x106 MMA issuer waiting for its turn.  Diagnostic. */
+unsigned int pcl_last_wait_code(void);
 
 /* Number of kernels this library has launched since it was loaded. */
 unsigned long long pcl_launch_count(void);

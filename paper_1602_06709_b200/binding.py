@@ -28,7 +28,7 @@ EXPORTS = [
     "pcl_last_device_status", "pcl_launch_count", "pcl_status_string", "pcl_profile_begin", "pcl_profile_end", "pcl_conv_bwd_data_noalloc", "pcl_noalloc_scratch_bytes",
     "pcl_conv_bwd_data_colsum_workspace_bytes", "pcl_conv_bwd_data_colsum",
     "pcl_maxpool2x2_bwd_colsum_workspace_bytes", "pcl_maxpool2x2_bwd_colsum", "pcl_conv_fwd_pool",
-    "pcl_maxpool2x2_fwd_codes", "pcl_maxpool2x2_bwd_codes",
+    "pcl_maxpool2x2_fwd_codes", "pcl_maxpool2x2_bwd_codes", "pcl_last_wait_code",
 ]
 
 
@@ -81,6 +81,7 @@ def lib() -> ctypes.CDLL:
         L.pcl_softmax_xent.argtypes = [ci, ci, vp, vp, vp, vp, vp]
         L.pcl_last_device_status.argtypes = [vp]
         L.pcl_launch_count.restype = ctypes.c_ulonglong
+        L.pcl_last_wait_code.restype = ctypes.c_uint
         L.pcl_profile_end.argtypes = [ctypes.POINTER(KernelStat), ci, ctypes.POINTER(ci)]
         L.pcl_conv_bwd_data_colsum_workspace_bytes.argtypes = [dp]
         L.pcl_conv_bwd_data_colsum_workspace_bytes.restype = sz
@@ -167,6 +168,10 @@ def maxpool2x2_bwd_codes(N, H, W, C, codes, dy, relu_mask, dx, dx_colsum=None, w
     wp, wb = _ws(ws)
     _check(lib().pcl_maxpool2x2_bwd_codes(N, H, W, C, _ptr(codes), _ptr(dy), int(bool(relu_mask)), _ptr(dx),
                                           _ptr(dx_colsum), wp, wb, _stream(stream)), "pcl_maxpool2x2_bwd_codes")
+
+
+def last_wait_code() -> int:
+    return int(lib().pcl_last_wait_code())
 
 
 def conv_bwd_data(d, dy, w, relu_mask_src, dx, ws=None, stream=None):

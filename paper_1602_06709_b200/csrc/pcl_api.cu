@@ -573,17 +573,22 @@ int pcl_softmax_xent(int N, int K, const float* logits, const int* labels, float
     return launch_softmax_xent(N, K, logits, labels, loss, dlogits, static_cast<cudaStream_t>(cuda_stream));
 }
 
+static std::atomic<unsigned int> g_last_wait_code{0};
+
 int pcl_last_device_status(void* cuda_stream) {
     if (cudaStreamSynchronize(static_cast<cudaStream_t>(cuda_stream)) != cudaSuccess) return PCL_ERR_CUDA;
     unsigned int v = 0;
     if (cudaMemcpyFromSymbol(&v, g_device_status, sizeof(v)) != cudaSuccess) return PCL_ERR_CUDA;
     if (v != 0) {
+        g_last_wait_code.store(v);
         const unsigned int zero = 0;
         if (cudaMemcpyToSymbol(g_device_status, &zero, sizeof(zero)) != cudaSuccess) return PCL_ERR_CUDA;
         return PCL_ERR_DEVICE_TIMEOUT;
     }
     return PCL_OK;
 }
+
+unsigned int pcl_last_wait_code(void) { return g_last_wait_code.load(); }
 
 unsigned long long pcl_launch_count(void) { return g_launches.load(); }
 

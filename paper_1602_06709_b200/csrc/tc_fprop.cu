@@ -212,7 +212,10 @@ __device__ __noinline__ void mma_issuer(const FpropParams& p, const IssuerCtx& c
     const int first_tile = c.first_tile, tile_stride = c.tile_stride, total_tiles = c.total_tiles, kiters = c.kiters;
 
     // kDuo with `split`: each issuer accumulates its slots into an accumulator of its own (the epilogue adds the
-    // two), so the threads need not hand over: no ordering between them can change a bit of the result.
+    // two), so no ordering between the threads' MMAs can change a bit of the result and a thread passes the turn on
+    // as soon as it has its slot, before issuing.  The slot STARTS stay ordered: letting one issuer overtake the
+    // other (no turn at all) gave, rarely, wrong sums and lost slot releases on a 96-wide plain tiling with three
+    // stages; cause not found, ordered starts are clean (40 x 40 repetitions, bit-identical).
     const bool split = kDuo && p.split_acc;
     const int bmn = p.bmn;
     const uint32_t idesc = make_idesc_tf32(BN, false, bmn != 0, kPair ? 256u : 128u);
@@ -250,7 +253,8 @@ __device__ __noinline__ void mma_issuer(const FpropParams& p, const IssuerCtx& c
     if (kDuo) { mine = turn == issuer; turn ^= 1u; }
 #define PCL_SLOT_ACQUIRE()                                                                                        \
     if (!bounded_wait_addr(full_a, phase, abort_flag, status, WAIT_MMA_FULL)) { ok = false; break; }             \
-    if (kDuo && !split && !wait_issue_turn(issue_seq, seq, abort_flag, status)) { ok = false; break; }           \
+    if (kDuo && !wait_issue_turn(issue_seq, seq, abort_flag, status)) { ok = false; break; }                     \
+    if (kDuo && split) *issue_seq = seq + 1;     /* split: only the slot STARTS are ordered (see below) */        \
     tc_fence_after();
 #define PCL_SLOT_RELEASE()                                                                                        \
     if (kDuo && !split) *issue_seq = seq + 1;                                                                     \

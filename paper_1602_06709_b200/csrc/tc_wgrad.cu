@@ -38,6 +38,7 @@ namespace pcl {
 namespace {
 
 constexpr int kMaxStages = 8;
+constexpr int kWgradThreads = 320;     // warp 0 producer, warp 1 MMA issuer, warps 2-9 epilogue (two per TMEM lane quarter)
 constexpr int kSmemBudget = 224 * 1024;
 
 struct WgradParams {
@@ -67,7 +68,7 @@ struct WgradParams {
 // kPair: see the header.  Pair mode needs grouped x and dy maps; every item then has rpi runs (runs past the
 // last tap read zeros through the out-of-bounds fill and are not stored).
 template <bool kPair>
-__global__ void __launch_bounds__(192, 1)
+__global__ void __launch_bounds__(kWgradThreads, 1)
 tc_wgrad_kernel(const __grid_constant__ CUtensorMap tmDy, const __grid_constant__ CUtensorMap tmX, WgradParams p) {
     extern __shared__ uint8_t smem_raw[];
     __shared__ uint64_t full_bar[kMaxStages];
@@ -264,7 +265,7 @@ tc_wgrad_kernel(const __grid_constant__ CUtensorMap tmDy, const __grid_constant_
             // bytes per instruction.
             const uint32_t stg = smem_u32(smem) + (warp - 2) * 4096;
             const int cg = (lane & 7) * 4;
-            for (int ch = 0; ch < n_groups; ++ch) {
+            for (int ch = (warp - 2) >> 2; ch < n_groups; ch += 2) {     // the quarter's two warps take alternate chunks
                 const int run = run0 + ch / p.L;
                 if (run >= p.total_runs) break;         // (pair mode) columns of runs past the last tap
                 const int tap = run / p.runs_per_tap;
@@ -537,11 +538,11 @@ int launch_tc_wgrad(const TcWgradArgs& a, cudaStream_t st) {
             attr[0].id = cudaLaunchAttributeClusterDimension;
             attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
             cudaLaunchConfig_t lc{};
-            lc.gridDim = dim3(unsigned(items)); lc.blockDim = dim3(192); lc.dynamicSmemBytes = smem; lc.stream = st;
+            lc.gridDim = dim3(unsigned(items)); lc.blockDim = dim3(kWgradThreads); lc.dynamicSmemBytes = smem; lc.stream = st;
             lc.attrs = attr; lc.numAttrs = 1;
             if (cudaLaunchKernelEx(&lc, tc_wgrad_kernel<true>, tmDy, tmX, p) != cudaSuccess) return PCL_ERR_CUDA;
         } else {
-            tc_wgrad_kernel<false><<<int(items), 192, smem, st>>>(tmDy, tmX, p);
+            tc_wgrad_kernel<false><<<int(items), kWgradThreads, smem, st>>>(tmDy, tmX, p);
         }
     }
     if (cudaGetLastError() != cudaSuccess) return PCL_ERR_CUDA;

@@ -222,3 +222,28 @@ def test_two_issuers_keep_results_reproducible(tag, mode, path_guard, monkeypatc
         y1, dx1 = run("solo")
         assert np.array_equal(y, y1) and np.array_equal(dx, dx1)
     assert B.last_device_status() == 0
+
+
+def test_two_issuer_backward_data_repeats_bit_for_bit(path_guard):
+    """Regression: a 96-map backward-data launch (plain tiling, three pipeline stages, two issuers with an
+    accumulator each) once lost slot releases and summed wrongly when one issuer could overtake the other.
+    Twenty repetitions must finish without a device-side timeout and agree bit for bit."""
+    import torch
+    import gpu_helpers as G
+    from paper_1602_06709_b200 import binding as B
+    B.set_path(B.PATH_TENSOR)
+    s = ConvShape(N=64, C=96, K=256, H=24, W=24, R=5, S=5)
+    x, w, dy, _ = G.make_inputs(s, "two_issuer_regression")
+    d = G.shape_to_desc(s)
+    dyt, wt, xt = G.dev(dy), G.dev(w), G.dev(x)
+    ws = G.workspace(B.conv_workspace_bytes(d, B.PASS_BWD_DATA))
+    first = None
+    for _ in range(20):
+        dx = torch.empty(s.N, s.H, s.W, s.C, device="cuda")
+        B.conv_bwd_data(d, dyt, wt, xt, dx, ws)
+        B.check_device_status()
+        if first is None:
+            first = dx
+            G.assert_parity(dx.cpu().numpy(), oracle.conv_bwd_data(s, dy, w, x), "bwd_data")
+        else:
+            assert torch.equal(first, dx)
