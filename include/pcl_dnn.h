@@ -96,7 +96,12 @@ int pcl_conv_fwd(const pcl_conv_desc* d, const float* x, const float* w, const f
  * position code of its window, bits 0-1 = position of the first maximum in row-major window order
  * (0: 2p,2q  1: 2p,2q+1  2: 2p+1,2q  3: 2p+1,2q+1), bit 2 set where that maximum is <= 0.  With the
  * codes, pcl_maxpool2x2_bwd_codes() routes the gradient without reading y again.
+ * y may be NULL where pcl_conv_fwd_pool_is_fused(d) != 0: the full-resolution output is then not
+ * stored at all (a training step that holds y_pool and the codes never reads it again: the pooled
+ * layer's backward passes take their ReLU mask from bit 2 of the codes); y_pool and pool_codes are
+ * bit-for-bit what the call with y writes.  Elsewhere a NULL y returns PCL_ERR_UNSUPPORTED_SHAPE.
  * Workspace as pcl_conv_fwd(). */
+int pcl_conv_fwd_pool_is_fused(const pcl_conv_desc* d);
 int pcl_conv_fwd_pool(const pcl_conv_desc* d, const float* x, const float* w, const float* bias,
                       float* y, float* y_pool, unsigned char* pool_codes, int act,
                       void* ws, size_t ws_bytes, void* cuda_stream);

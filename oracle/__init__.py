@@ -278,6 +278,28 @@ def maxpool2x2_bwd(x, dy, relu_mask_src=None) -> np.ndarray:
     return dx
 
 
+def maxpool2x2_codes(x) -> np.ndarray:
+    """Position code of each 2x2 window (one byte per pooled element): bits 0-1 = position of the window's first
+    maximum in row-major window order (0: (0,0), 1: (0,1), 2: (1,0), 3: (1,1)), bit 2 set where that maximum
+    is <= 0 (where a ReLU mask taken from x would zero the routed gradient)."""
+    x = np.asarray(x, dtype=np.float64)
+    N, H, W, C = x.shape
+    v = x.reshape(N, H // 2, 2, W // 2, 2, C).transpose(0, 1, 3, 5, 2, 4).reshape(N, H // 2, W // 2, C, 4)
+    arg = v.argmax(axis=-1)
+    return (arg + 4 * (v.max(axis=-1) <= 0.0)).astype(np.uint8)
+
+
+def maxpool2x2_bwd_codes(codes, dy, relu_mask: bool) -> np.ndarray:
+    """Routes dy by position codes (maxpool2x2_codes): the coded position of each window gets dy, the other three 0;
+    with relu_mask, windows whose code has bit 2 set get 0 everywhere."""
+    codes = np.asarray(codes).astype(np.int64)
+    dy = np.asarray(dy, dtype=np.float64)
+    N, P, Q, C = dy.shape
+    g = dy * (codes < 4) if relu_mask else dy
+    onehot = ((codes & 3)[..., None] == np.arange(4)).astype(np.float64)
+    return (onehot * g[..., None]).reshape(N, P, Q, C, 2, 2).transpose(0, 1, 4, 2, 5, 3).reshape(N, 2 * P, 2 * Q, C)
+
+
 def softmax_xent(logits, labels):
     """loss = -(1/N) sum_n log softmax(z_n)[label_n];  dz = (softmax(z) - onehot)/N."""
     z = np.asarray(logits, dtype=np.float64)

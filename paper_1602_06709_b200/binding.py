@@ -27,7 +27,7 @@ EXPORTS = [
     "pcl_sgd_update", "pcl_maxpool2x2_fwd", "pcl_maxpool2x2_bwd", "pcl_softmax_xent",
     "pcl_last_device_status", "pcl_launch_count", "pcl_status_string", "pcl_profile_begin", "pcl_profile_end", "pcl_conv_bwd_data_noalloc", "pcl_noalloc_scratch_bytes",
     "pcl_conv_bwd_data_colsum_workspace_bytes", "pcl_conv_bwd_data_colsum",
-    "pcl_maxpool2x2_bwd_colsum_workspace_bytes", "pcl_maxpool2x2_bwd_colsum", "pcl_conv_fwd_pool",
+    "pcl_maxpool2x2_bwd_colsum_workspace_bytes", "pcl_maxpool2x2_bwd_colsum", "pcl_conv_fwd_pool", "pcl_conv_fwd_pool_is_fused",
     "pcl_maxpool2x2_fwd_codes", "pcl_maxpool2x2_bwd_codes", "pcl_last_wait_code",
 ]
 
@@ -70,6 +70,7 @@ def lib() -> ctypes.CDLL:
         L.pcl_conv_fwd.argtypes = [dp, vp, vp, vp, vp, ci, vp, sz, vp]
         L.pcl_conv_bwd_data.argtypes = [dp, vp, vp, vp, vp, vp, sz, vp]
         L.pcl_conv_fwd_pool.argtypes = [dp, vp, vp, vp, vp, vp, vp, ci, vp, sz, vp]
+        L.pcl_conv_fwd_pool_is_fused.argtypes = [dp]
         L.pcl_maxpool2x2_fwd_codes.argtypes = [ci, ci, ci, ci, vp, vp, vp, vp]
         L.pcl_maxpool2x2_bwd_codes.argtypes = [ci, ci, ci, ci, vp, vp, ci, vp, vp, vp, sz, vp]
         L.pcl_conv_bwd_weights.argtypes = [dp, vp, vp, vp, vp, ci, vp, sz, vp]
@@ -153,7 +154,12 @@ def conv_fwd(d, x, w, bias, y, act=ACT_NONE, ws=None, stream=None):
            "pcl_conv_fwd")
 
 
+def conv_fwd_pool_is_fused(d) -> bool:
+    return bool(lib().pcl_conv_fwd_pool_is_fused(ctypes.byref(d)))
+
+
 def conv_fwd_pool(d, x, w, bias, y, y_pool, act=ACT_NONE, ws=None, stream=None, pool_codes=None):
+    """y may be None where conv_fwd_pool_is_fused(d): the full-resolution output is then not stored."""
     wp, wb = _ws(ws)
     _check(lib().pcl_conv_fwd_pool(ctypes.byref(d), _ptr(x), _ptr(w), _ptr(bias), _ptr(y), _ptr(y_pool),
                                    _ptr(pool_codes), act, wp, wb, _stream(stream)), "pcl_conv_fwd_pool")

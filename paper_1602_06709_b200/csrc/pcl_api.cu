@@ -243,9 +243,11 @@ static int conv_fwd_impl(const pcl_conv_desc* d, const float* x, const float* w,
     int P, Q;
     int rc = check_desc(d, &P, &Q);
     if (rc != PCL_OK) return rc;
-    if (!x || !w || !y) return PCL_ERR_BAD_ARG;
+    if (!x || !w || (!y && !y_pool)) return PCL_ERR_BAD_ARG;
     if (act != PCL_ACT_NONE && act != PCL_ACT_RELU && act != PCL_ACT_SIGMOID) return PCL_ERR_BAD_ARG;
     if (!aligned16(x) || !aligned16(w) || !aligned16(y) || !aligned16(bias) || !aligned16(y_pool)) return PCL_ERR_MISALIGNED;
+    // without y only the one-kernel form can run (the separate pooling kernel reads y)
+    if (!y && !pcl_conv_fwd_pool_is_fused(d)) return PCL_ERR_UNSUPPORTED_SHAPE;
     if (y_pool && (P % 2 != 0 || Q % 2 != 0)) return PCL_ERR_UNSUPPORTED_SHAPE;
     if (pool_codes && (!y_pool || !aligned16(pool_codes))) return y_pool ? PCL_ERR_MISALIGNED : PCL_ERR_BAD_ARG;
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
@@ -277,6 +279,15 @@ static int conv_fwd_impl(const pcl_conv_desc* d, const float* x, const float* w,
     if (rc != PCL_OK) return rc;
     if (y_pool) return launch_maxpool_fwd(d->N, P, Q, d->K, y, y_pool, st, pool_codes);     // not fused above
     return PCL_OK;
+}
+
+int pcl_conv_fwd_pool_is_fused(const pcl_conv_desc* d) {
+    int P, Q;
+    if (check_desc(d, &P, &Q) != PCL_OK) return 0;
+    if (!few_channel_path_for(*d, PCL_PASS_FWD) && !tensor_path_for(*d, PCL_PASS_FWD)) return 0;
+    TcFpropArgs a{};
+    a.P = P; a.Q = Q; a.Kout = d->K;
+    return tc_fprop_can_pool(a) ? 1 : 0;
 }
 
 int pcl_conv_fwd(const pcl_conv_desc* d, const float* x, const float* w, const float* bias, float* y, int act,

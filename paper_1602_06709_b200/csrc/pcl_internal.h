@@ -55,7 +55,7 @@ struct TcFpropArgs {
     const float* wt;   // [Kout][R*S][Cin]
     const float* bias; // [Kout] or null
     const float* mask_src; // [N][P][Q][Kout] or null
-    float* out;        // [N][P][Q][Kout]
+    float* out;        // [N][P][Q][Kout]; may be null with pool_out (nothing is stored at full resolution)
     int N, H, W, Cin, Kout, R, S, pad_h, pad_w, P, Q, act;
     // Element strides of `in` between adjacent w, h and n positions; 0 = packed
     // NHWC (Cin, W*Cin, H*W*Cin).  A w stride smaller than Cin gives overlapping

@@ -642,7 +642,7 @@ tc_fprop_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                     }
                     fence_proxy_async_shared();
                     __syncwarp();
-                    if (lane == 0 && in_range && col0 < p.Kout) {
+                    if (lane == 0 && in_range && col0 < p.Kout && p.out) {     // (pooling launches may keep y unstored)
                         tma_store_4d(&tmOut, stg, col0, sq, sp, sn);
                         bulk_commit_group();
                     }
@@ -1133,7 +1133,12 @@ int launch_tc_fprop(const TcFpropArgs& a, cudaStream_t st) {
     // Output map for the TMA-store epilogue: a warp stores the 32 consecutive box pixels it owns, 32 maps at a time.
     CUtensorMap tmOut = tmA;        // (a valid map is passed in any case; unused unless p.tma_store)
     p.tma_store = 0;
-    if (env_int("PCL_TMA_STORE", 1) && !a.mask_src && !a.colsum_rows && a.Kout % 4 == 0 &&
+    if (!a.out) {
+        // pooled output only: the epilogue stages each chunk as for a TMA store, takes the maxima from the staging
+        // tile and stores nothing at full resolution
+        if (!a.pool_out || a.colsum_rows) return PCL_ERR_BAD_ARG;
+        p.tma_store = 1;
+    } else if (env_int("PCL_TMA_STORE", 1) && !a.mask_src && !a.colsum_rows && a.Kout % 4 == 0 &&
         (reinterpret_cast<uintptr_t>(a.out) & 15) == 0) {
         const uint32_t bx = bw < 32 ? bw : 32, by = uint32_t(bh) < 32 / bx ? uint32_t(bh) : 32 / bx, bnn = 32 / (bx * by);
         const uint64_t dims[4] = {uint64_t(a.Kout), uint64_t(a.Q), uint64_t(a.P), uint64_t(a.N)};

@@ -102,7 +102,10 @@ class VggA(_HostFeed):
     FC 25088-4096-4096-1000 and softmax cross-entropy."""
 
     def __init__(self, N: int, hw: int = inputs.VGGA_HW, conv=None, fc=None, classes: int = inputs.VGGA_CLASSES,
-                 lr: float = 0.01, cfg: str = "cfg5"):
+                 lr: float = 0.01, cfg: str = "cfg5", keep_unpooled: bool = False):
+        """keep_unpooled: also store the full-resolution output of the pooled layers (self.y[i]).  The step never
+        reads it (pooling backward and the ReLU mask go by the position codes), so by default it is neither
+        allocated nor written where the convolution and the pooling run as one kernel."""
         self.N, self.lr, self.classes = N, lr, classes
         conv = conv if conv is not None else inputs.VGGA_CONV
         self.convs: List[_ConvLayer] = []
@@ -134,7 +137,8 @@ class VggA(_HostFeed):
         # activations and gradients
         dev = "cuda"
         self.x = torch.empty(N, hw, hw, self.convs[0].C, device=dev)
-        self.y = [torch.empty(N, L.H, L.W, L.K, device=dev) for L in self.convs]           # post-ReLU
+        self.y = [None if (L.pool and not keep_unpooled and B.conv_fwd_pool_is_fused(L.desc))
+                  else torch.empty(N, L.H, L.W, L.K, device=dev) for L in self.convs]       # post-ReLU
         self.pooled = [torch.empty(N, L.H // 2, L.W // 2, L.K, device=dev) if L.pool else None for L in self.convs]
         self.dy = [torch.empty(N, L.H, L.W, L.K, device=dev) for L in self.convs]           # grad wrt pre-activation
         self.dpooled = [torch.empty(N, L.H // 2, L.W // 2, L.K, device=dev) if L.pool else None for L in self.convs]

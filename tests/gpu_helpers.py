@@ -86,6 +86,36 @@ def _cmp(got_t, ref_fn, size, samples, rng, what, report):
     assert rel <= REL_L2_TOL and mx <= MAX_OVER_RMS_TOL, f"{what}: rel_l2={rel:.3e} max/rms={mx:.3e}"
 
 
+def _check_pooled_only(net, i, s, xin, w, b, samples, rng, report):
+    """A pooled layer whose full-resolution output was not stored: the pooled tensor against the oracle's
+    pool(relu(conv)), and the position codes against the oracle's own window values -- a code must name a position
+    whose value is the window's maximum up to the parity tolerance (TF32 rounding may reorder near-ties, never
+    more), and bit 2 must say exactly whether the stored maximum is <= 0."""
+    L = net.convs[i]
+    N, P, Q, K = s.N, s.P, s.Q, s.K
+    size = N * (P // 2) * (Q // 2) * K
+    got_p = net.pooled[i].detach().cpu().numpy().reshape(-1)
+    codes = net.pool_codes[i].detach().cpu().numpy().reshape(-1)
+    idx = (np.sort(rng.choice(size, size=samples, replace=False)).astype(np.int64) if samples and size > samples
+           else np.arange(size, dtype=np.int64))
+    k = idx % K; q2 = (idx // K) % (Q // 2); p2 = (idx // (K * (Q // 2))) % (P // 2); n = idx // (K * (Q // 2) * (P // 2))
+    win = np.stack([((n * P + 2 * p2 + e // 2) * Q + 2 * q2 + e % 2) * K + k for e in range(4)], axis=1)   # [len][4]
+    if samples and size > samples:
+        yw = oracle.conv_fwd(s, xin, w, b, oracle.ACT_RELU, at=win.reshape(-1)).reshape(-1, 4)
+    else:
+        yw = oracle.conv_fwd(s, xin, w, b, oracle.ACT_RELU).reshape(-1)[win]
+    ref = yw.max(axis=1)
+    rel, mx = oracle.parity_errors(got_p[idx], ref)
+    report.append((f"{L.name} fwd+pool", rel, mx))
+    assert rel <= REL_L2_TOL and mx <= MAX_OVER_RMS_TOL, f"{L.name} fwd+pool: rel_l2={rel:.3e} max/rms={mx:.3e}"
+    c = codes[idx].astype(np.int64)
+    assert c.max() <= 7, f"{L.name}: position code out of range"
+    assert np.array_equal(c >= 4, got_p[idx] <= 0.0), f"{L.name}: bit 2 of the codes != (stored maximum <= 0)"
+    tol = MAX_OVER_RMS_TOL * float(np.sqrt(np.mean(ref * ref)))
+    chosen = yw[np.arange(len(idx)), c & 3]
+    assert np.all(chosen >= ref - tol), f"{L.name}: a code names a position that is not the window's maximum"
+
+
 def verify_vgg_step(net, params_before, samples=0, seed=0):
     """net: VggA after exactly one step(); params_before: flat params (numpy) before the step."""
     rng = np.random.default_rng(seed)
@@ -103,6 +133,9 @@ def verify_vgg_step(net, params_before, samples=0, seed=0):
     for i, L in enumerate(net.convs):
         s = ConvShape(N=N, C=L.C, K=L.K, H=L.H, W=L.W, R=3, S=3, pad_h=1, pad_w=1)
         xin = host(net.layer_input(i)); w = pview(2 * i); b = pview(2 * i + 1)
+        if net.y[i] is None:
+            _check_pooled_only(net, i, s, xin, w, b, samples, rng, report)
+            continue
         _cmp(net.y[i], lambda at: oracle.conv_fwd(s, xin, w, b, oracle.ACT_RELU, at=at), net.y[i].numel(), samples,
              rng, f"{L.name} fwd", report)
         if L.pool:
@@ -157,7 +190,11 @@ def verify_vgg_step(net, params_before, samples=0, seed=0):
     for i in reversed(range(nconv)):
         L = net.convs[i]
         s = ConvShape(N=N, C=L.C, K=L.K, H=L.H, W=L.W, R=3, S=3, pad_h=1, pad_w=1)
-        if L.pool:
+        if L.pool and net.y[i] is None:      # routed by the position codes the forward call recorded, bit for bit
+            nchk = N if not samples else min(N, 2)
+            ref = oracle.maxpool2x2_bwd_codes(host(net.pool_codes[i][:nchk]), host(net.dpooled[i][:nchk]), True)
+            assert np.array_equal(host(net.dy[i][:nchk]), ref.astype(np.float32)), f"{L.name} pool bwd (codes)"
+        elif L.pool:
             nchk = N if not samples else min(N, 2)
             y = host(net.y[i][:nchk]); dp = host(net.dpooled[i][:nchk])
             assert np.array_equal(host(net.dy[i][:nchk]), oracle.maxpool2x2_bwd(y, dp, y).astype(np.float32)), f"{L.name} pool bwd"

@@ -222,6 +222,17 @@ def test_conv_fwd_with_fused_maxpool(shape, tiling, store, monkeypatch):
             B.maxpool2x2_bwd_codes(N, H, W, K, codes, G.dev(g), relu, dx)
             ref = oracle.maxpool2x2_bwd(yh, g, yh if relu else None)
             assert np.array_equal(dx.cpu().numpy(), ref.astype(np.float32))
+        assert np.array_equal(codes.cpu().numpy(), oracle.maxpool2x2_codes(yh))
+        # without y (where the call runs as one kernel): the same pooled tensor and codes, bit for bit
+        if B.conv_fwd_pool_is_fused(d):
+            yp2 = torch.full_like(yp, float("nan")); codes2 = torch.full_like(codes, 255)
+            B.conv_fwd_pool(d, G.dev(x), G.dev(w), G.dev(bias), None, yp2, act, ws, pool_codes=codes2)
+            B.check_device_status()
+            assert torch.equal(yp2, yp) and torch.equal(codes2, codes)
+            yp3 = torch.full_like(yp, float("nan"))
+            B.conv_fwd_pool(d, G.dev(x), G.dev(w), G.dev(bias), None, yp3, act, ws)     # no codes either
+            B.check_device_status()
+            assert torch.equal(yp3, yp)
 
 
 def test_conv_fwd_pool_rejects_odd_output():
@@ -234,6 +245,23 @@ def test_conv_fwd_pool_rejects_odd_output():
     y = torch.zeros(1, 7, 8, 8, device="cuda"); yp = torch.zeros(1, 3, 4, 8, device="cuda")
     with pytest.raises(B.PclError):
         B.conv_fwd_pool(d, x, w, None, y, yp, B.ACT_RELU, None)
+
+
+def test_conv_fwd_pool_without_y_only_where_fused():
+    """A strided layer runs the generic convolution and a separate pooling kernel, which reads y: y is required."""
+    import gpu_helpers as G
+    from oracle import ConvShape
+    from paper_1602_06709_b200 import binding as B
+    s = ConvShape(N=1, C=8, K=8, H=16, W=16, R=3, S=3, stride_h=2, stride_w=2, pad_h=1, pad_w=1)
+    d = G.shape_to_desc(s)
+    assert not B.conv_fwd_pool_is_fused(d)
+    x = torch.zeros(1, 16, 16, 8, device="cuda"); w = torch.zeros(8, 3, 3, 8, device="cuda")
+    yp = torch.zeros(1, 4, 4, 8, device="cuda")
+    with pytest.raises(B.PclError) as e:
+        B.conv_fwd_pool(d, x, w, None, None, yp, B.ACT_RELU, None)
+    assert e.value.code == B.ERR_UNSUPPORTED_SHAPE
+    s1 = ConvShape(N=1, C=8, K=8, H=16, W=16, R=3, S=3, pad_h=1, pad_w=1)
+    assert B.conv_fwd_pool_is_fused(G.shape_to_desc(s1))
 
 
 @pytest.mark.parametrize("N,H,W,C", [(2, 8, 6, 8), (3, 14, 14, 5), (2, 28, 28, 64), (1, 4, 4, 1024)])

@@ -23,9 +23,10 @@ def _randomise_biases(net, scale=0.1):
             net.store.p(i).copy_(torch.from_numpy(b))
 
 
-def _small_vgg(N=4, hw=32):
+def _small_vgg(N=4, hw=32, keep_unpooled=False):
     from paper_1602_06709_b200 import inputs, networks
-    net = networks.VggA(N, hw=hw, conv=SMALL_CONV, fc=[(64, 128), (128, 128), (128, 10)], classes=10, cfg="small")
+    net = networks.VggA(N, hw=hw, conv=SMALL_CONV, fc=[(64, 128), (128, 128), (128, 10)], classes=10, cfg="small",
+                        keep_unpooled=keep_unpooled)
     _randomise_biases(net)
     x = inputs.uniform(inputs.tensor_id("small", "x"), (N, hw, hw, 3), 0.0, 1.0)
     lab = inputs.labels(inputs.tensor_id("small", "labels"), N, 10)
@@ -33,15 +34,34 @@ def _small_vgg(N=4, hw=32):
     return net, x, lab
 
 
-def test_small_vgg_step_per_call():
+@pytest.mark.parametrize("keep_unpooled", [False, True])
+def test_small_vgg_step_per_call(keep_unpooled):
+    """keep_unpooled=False is the step as benched: pooled layers store only the pooled tensor and the position
+    codes; True also stores their full-resolution outputs, which lets the pooling be checked exactly."""
     import gpu_helpers as G
     from paper_1602_06709_b200 import binding as B
-    net, x, lab = _small_vgg()
+    net, x, lab = _small_vgg(keep_unpooled=keep_unpooled)
+    assert all((net.y[i] is None) == (L.pool and not keep_unpooled) for i, L in enumerate(net.convs))
     before = net.store.params.cpu().numpy().copy()
     net.step()
     B.check_device_status()
     report = G.verify_vgg_step(net, before, samples=0)
     assert len(report) >= 8 + 3 + 3 + 3 + 8 + 7
+
+
+def test_unstored_pooled_layer_outputs_change_nothing():
+    """Two steps with and without the pooled layers' full-resolution outputs stored: identical parameters."""
+    from paper_1602_06709_b200 import binding as B
+    res = []
+    for keep in (False, True):
+        net, x, lab = _small_vgg(N=8, keep_unpooled=keep)
+        net.step(); net.step()
+        B.check_device_status()
+        res.append((net.store.params.cpu().numpy().copy(), [c.cpu().numpy().copy() for c in net.pool_codes if c is not None],
+                    [t.cpu().numpy().copy() for t in net.pooled if t is not None]))
+    assert np.array_equal(res[0][0], res[1][0])
+    for a, b in zip(res[0][1] + res[0][2], res[1][1] + res[1][2]):
+        assert np.array_equal(a, b)
 
 
 def test_small_vgg_step_end_to_end_against_chained_oracle():

@@ -67,6 +67,33 @@ def test_maxpool_backward_ties_go_to_first_and_mask():
     assert oracle.maxpool2x2_bwd(x, dy, relu_mask_src=x).sum() == 0.0
 
 
+def test_maxpool_position_codes_brute_force_and_routing():
+    """Codes by a literal loop over each window (first maximum in row-major order, bit 2 for a maximum <= 0);
+    routing by codes must equal the pooling backward pass from x, with and without the ReLU mask taken from x."""
+    x = np.maximum(RNG.normal(size=(2, 6, 4, 3)), 0.0)        # post-ReLU values: ties among zeros
+    x[0, 0:2, 0:2, 0] = 0.0                                   # an all-zero window
+    x[1, 2:4, 2:4, 1] = 5.0                                   # a positive four-way tie
+    codes = oracle.maxpool2x2_codes(x)
+    assert codes.dtype == np.uint8 and codes.shape == (2, 3, 2, 3)
+    for n in range(2):
+        for p in range(3):
+            for q in range(2):
+                for c in range(3):
+                    win = [x[n, 2 * p + i, 2 * q + j, c] for i in range(2) for j in range(2)]
+                    e = min(k for k in range(4) if win[k] == max(win))
+                    assert codes[n, p, q, c] == e + (4 if max(win) <= 0 else 0)
+    assert codes[0, 0, 0, 0] == 4 and codes[1, 1, 1, 1] == 0
+    dy = RNG.normal(size=(2, 3, 2, 3))
+    np.testing.assert_array_equal(oracle.maxpool2x2_bwd_codes(codes, dy, False), oracle.maxpool2x2_bwd(x, dy))
+    np.testing.assert_array_equal(oracle.maxpool2x2_bwd_codes(codes, dy, True),
+                                  oracle.maxpool2x2_bwd(x, dy, relu_mask_src=x))
+    # a hand-written case: code 3 sends the gradient to the window's last position, code 6 (masked) nowhere
+    g = oracle.maxpool2x2_bwd_codes(np.array([[[[3, 6]]]], dtype=np.uint8), np.array([[[[2.0, 7.0]]]]), True)
+    assert g.shape == (1, 2, 2, 2) and g[0, 1, 1, 0] == 2.0 and g.sum() == 2.0
+    g = oracle.maxpool2x2_bwd_codes(np.array([[[[3, 6]]]], dtype=np.uint8), np.array([[[[2.0, 7.0]]]]), False)
+    assert g[0, 1, 0, 1] == 7.0 and g.sum() == 9.0
+
+
 def test_softmax_xent_closed_forms():
     N, K = 5, 7
     z = RNG.normal(size=(N, K)) * 3
