@@ -43,6 +43,12 @@ constexpr int kEpiWarps = 8;                    // two per TMEM lane quarter, sp
 constexpr int kEpiStageBytes = kEpiWarps * 4096;
 constexpr int kSecondIssuerWarp = 2 + kEpiWarps;        // warp 10
 constexpr int kThreads = (3 + kEpiWarps) * 32;
+// Launches whose tiles have a short reduction (the few-channel first layer: three k-steps) are bound by the
+// epilogue warps, each of which issues an instruction every ~7 cycles: those run sixteen of them (four per TMEM
+// lane quarter, warps 11-18 added behind the second issuer's warp) under a 104-register cap.
+constexpr int kEpiWarpsWide = 16;
+constexpr int kThreadsWide = (3 + kEpiWarpsWide) * 32;
+constexpr int kEpiStageBytesWide = kEpiWarpsWide * (4096 + 128);      // staging tiles, then one 32-float bias slot per warp
 
 struct FpropParams {
     int bw_log2, bh_log2;       // box of output pixels: bw x bh x (128 / (bw*bh))
@@ -360,8 +366,8 @@ __device__ __noinline__ void mma_issuer(const FpropParams& p, const IssuerCtx& c
 // kMask: the epilogue applies the ReLU mask (backward-data); its eight prefetched mask vectors would cost the other
 // instantiations registers (the epilogue is what the 168-register budget of an 11-warp CTA is short of, and a
 // spilled value that has left L1 costs ~600 cycles per use).
-template <bool kPair, bool kPool, bool kMask>
-__global__ void __launch_bounds__(kThreads, 1)
+template <bool kPair, bool kPool, bool kMask, int kEpi = kEpiWarps>
+__global__ void __launch_bounds__((3 + kEpi) * 32, 1)
 tc_fprop_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                 const __grid_constant__ CUtensorMap tmOut, const __grid_constant__ FpropParams p) {
     extern __shared__ uint8_t smem_raw[];
@@ -396,7 +402,7 @@ tc_fprop_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
     const uint32_t step_bytes = p.halo ? b_bytes : kABytes + b_bytes;
     const uint32_t stage_bytes = p.KS * step_bytes;
     uint8_t* b_ring = smem + (p.halo ? p.NA * p.a_buf_bytes : kABytes);
-    uint8_t* epi_stage = smem + (p.halo ? p.NA * p.a_buf_bytes : 0) + p.stages * stage_bytes;   // 8 x 4 KB
+    uint8_t* epi_stage = smem + (p.halo ? p.NA * p.a_buf_bytes : 0) + p.stages * stage_bytes;   // kEpi x 4 KB (+ kEpi x 128 B of bias slots in the 16-warp variant)
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < p.stages; ++s) {
@@ -409,7 +415,7 @@ tc_fprop_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
         }
         for (int a = 0; a < 2; ++a) {
             mbar_init(&tmem_full_bar[a], p.issuers);
-            mbar_init(&tmem_empty_bar[a], kPair ? 2 * kEpiWarps : kEpiWarps);
+            mbar_init(&tmem_empty_bar[a], kPair ? 2 * kEpi : kEpi);
         }
         abort_flag = 0;
         issue_seq = 0;
@@ -573,7 +579,11 @@ tc_fprop_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
     } else {
         // ------------------------------------------------------------ epilogue
         const int quarter = warp & 3;           // TMEM lanes 32*quarter .. +31
-        const int chalf = (warp - 2) >> 2;      // which half of the 32-column chunks this warp takes
+        const int epi = warp < kSecondIssuerWarp ? warp - 2 : warp - 3;     // 0 .. kEpi-1 (warp 10 is an issuer)
+        // the quarter's kEpi/4 warps share its (box, 32-column chunk) items: warp `sub` takes every (kEpi/4)-th
+        constexpr int kSub = kEpi / 4;
+        const int sub = epi >> 2;               // (warps 2-5: 0, 6-9: 1, 11-14: 2, 15-18: 3; one of each per quarter)
+        const int cpb = p.BN / 32;              // chunks per box
         const int row = quarter * 32 + lane;    // row of the tile = pixel of the box
         const int iw = row & (bw - 1);
         const int ih = (row >> p.bw_log2) & (bh - 1);
@@ -589,6 +599,7 @@ tc_fprop_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
             if (!bounded_wait_warp(&tmem_full_bar[acc], acc_phase, &abort_flag, p.status, WAIT_EPI_TMEM_FULL)) break;
             tc_fence_after();
             for (int h = 0; h < p.MT; ++h) {
+            const int ch0 = (sub - h * cpb) & (kSub - 1);       // first chunk of box h that is this warp's
             const int q = it.qi * p.tw + iw + h * p.half_dq;
             const int pp = it.pi * p.th + ih + h * p.half_dp;
             const int n = ni * p.tn + in_;
@@ -602,36 +613,36 @@ tc_fprop_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                 const size_t m_index = (static_cast<size_t>(ni) * p.tiles_p + it.pi) * p.tiles_q + it.qi;
                 cs_row = p.colsum_rows + ((m_index * p.MT + h) * 4 + quarter) * p.Kout;
             }
-            if (!kMask && p.tma_store) {
+            if (kEpi > kEpiWarps || (!kMask && p.tma_store)) {      // (wide-epilogue launches always stage)
                 // TMA-store path (no mask, no column sums).  Each lane owns one row (pixel) of the accumulator: it
                 // finishes its 32 columns in registers (bias, activation), puts them into its row of the warp's
                 // 4 KB staging tile in the 128-byte-swizzle layout, and one lane hands the tile to TMA, which writes
                 // the 32 pixels x 128 bytes and clips what lies outside the tensor.  The warp's 32 rows are 32
                 // consecutive pixels of the box, i.e. a sub-box whose first pixel is (sq, sp, sn).
-                const uint32_t stg = smem_u32(epi_stage + (warp - 2) * 4096);
+                const uint32_t stg = smem_u32(epi_stage + epi * 4096);
                 const int srow = quarter * 32;
-                const int sq = it.qi * p.tw + (srow & (bw - 1)) + h * p.half_dq;
-                const int sp = it.pi * p.th + ((srow >> p.bw_log2) & (bh - 1)) + h * p.half_dp;
-                const int sn = ni * p.tn + (srow >> (p.bw_log2 + p.bh_log2));
-                const bool in_range = sq < p.Q && sp < p.P && sn < p.N;     // (a store never starts outside the tensor)
-                for (int ch = chalf; ch < p.BN / 32; ch += 2) {
+                for (int ch = ch0; ch < cpb; ch += kSub) {
                     const int col0 = kt * p.BN + ch * 32;
-                    float4 bv[8];
+                    // (the 8-warp variant fetches the chunk's bias ahead of the accumulator, eight vectors per lane;
+                    // under the 16-warp variant's register cap each lane fetches one value and the warp shares the
+                    // 32 of them through 128 bytes of shared memory)
+                    constexpr int kBv = kEpi > kEpiWarps ? 1 : 8;
+                    float4 bv[kBv];
+                    float bias_lane = 0.f;
+                    if (kEpi == kEpiWarps) {
 #pragma unroll
-                    for (int j = 0; j < 8; ++j)
-                        bv[j] = (p.bias && col0 + 4 * j < p.Kout) ? __ldg(reinterpret_cast<const float4*>(p.bias + col0 + 4 * j))
-                                                                   : make_float4(0.f, 0.f, 0.f, 0.f);
-                    uint32_t v[32];
-                    tmem_ld_32x32(t_row + ch * 32, v);
-                    tmem_ld_wait();
-                    if (!kPool && p.split_acc) add_second_accumulator(t_row + t_second + ch * 32, v);
-                    // the previous store of this warp must have read the staging tile before it is overwritten
-                    if (lane == 0) bulk_wait_group_read0();
-                    __syncwarp();
-#pragma unroll
-                    for (int j = 0; j < 8; ++j) {
-                        float4 o = make_float4(__uint_as_float(v[4 * j]) + bv[j].x, __uint_as_float(v[4 * j + 1]) + bv[j].y,
-                                               __uint_as_float(v[4 * j + 2]) + bv[j].z, __uint_as_float(v[4 * j + 3]) + bv[j].w);
+                        for (int j = 0; j < kBv; ++j)
+                            bv[j] = (p.bias && col0 + 4 * j < p.Kout) ? __ldg(reinterpret_cast<const float4*>(p.bias + col0 + 4 * j))
+                                                                       : make_float4(0.f, 0.f, 0.f, 0.f);
+                    } else {
+                        // (the previous chunk's reads of the slot lie before the __syncwarp() that ended its staging)
+                        if (p.bias && col0 + lane < p.Kout) bias_lane = __ldg(p.bias + col0 + lane);
+                        reinterpret_cast<float*>(epi_stage + kEpi * 4096 + epi * 128)[lane] = bias_lane;
+                    }
+                    // finishes four columns (bias, activation) and puts them into the lane's row of the staging tile
+                    auto finish_store = [&](const uint32_t* v4, const float4 bj, const int j) {
+                        float4 o = make_float4(__uint_as_float(v4[0]) + bj.x, __uint_as_float(v4[1]) + bj.y,
+                                               __uint_as_float(v4[2]) + bj.z, __uint_as_float(v4[3]) + bj.w);
                         if (p.act == PCL_ACT_RELU) {
                             o.x = fmaxf(o.x, 0.f); o.y = fmaxf(o.y, 0.f); o.z = fmaxf(o.z, 0.f); o.w = fmaxf(o.w, 0.f);
                         } else if (p.act == PCL_ACT_SIGMOID) {
@@ -639,12 +650,42 @@ tc_fprop_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                             o.z = 1.f / (1.f + __expf(-o.z)); o.w = 1.f / (1.f + __expf(-o.w));
                         }
                         st_shared_v4(stg + lane * 128 + ((j ^ (lane & 7)) * 16), o.x, o.y, o.z, o.w);
+                    };
+                    if constexpr (kEpi == kEpiWarps) {
+                        uint32_t v[32];
+                        tmem_ld_32x32(t_row + ch * 32, v);
+                        tmem_ld_wait();
+                        if (!kPool && p.split_acc) add_second_accumulator(t_row + t_second + ch * 32, v);
+                        // the previous store of this warp must have read the staging tile before it is overwritten
+                        if (lane == 0) bulk_wait_group_read0();
+                        __syncwarp();
+#pragma unroll
+                        for (int j = 0; j < 8; ++j) finish_store(&v[4 * j], bv[j], j);
+                    } else {
+                        // two loads of 16 columns: half the registers
+                        if (lane == 0) bulk_wait_group_read0();
+                        __syncwarp();       // (also: every lane's bias value is in the warp's bias slot)
+                        const uint32_t bias_a = smem_u32(epi_stage + kEpi * 4096 + epi * 128);    // behind the staging tiles
+#pragma unroll
+                        for (int hh = 0; hh < 2; ++hh) {
+                            uint32_t v[16];
+                            tmem_ld_32x16(t_row + ch * 32 + hh * 16, v);
+                            tmem_ld_wait();
+#pragma unroll
+                            for (int jj = 0; jj < 4; ++jj)
+                                finish_store(&v[4 * jj], ld_shared_v4(bias_a + 16 * (hh * 4 + jj)), hh * 4 + jj);
+                        }
                     }
                     fence_proxy_async_shared();
                     __syncwarp();
-                    if (lane == 0 && in_range && col0 < p.Kout && p.out) {     // (pooling launches may keep y unstored)
-                        tma_store_4d(&tmOut, stg, col0, sq, sp, sn);
-                        bulk_commit_group();
+                    if (lane == 0 && col0 < p.Kout && p.out) {     // (pooling launches may keep y unstored)
+                        const int sq = it.qi * p.tw + (srow & (bw - 1)) + h * p.half_dq;
+                        const int sp = it.pi * p.th + ((srow >> p.bw_log2) & (bh - 1)) + h * p.half_dp;
+                        const int sn = ni * p.tn + (srow >> (p.bw_log2 + p.bh_log2));
+                        if (sq < p.Q && sp < p.P && sn < p.N) {     // (a store never starts outside the tensor)
+                            tma_store_4d(&tmOut, stg, col0, sq, sp, sn);
+                            bulk_commit_group();
+                        }
                     }
                     if (kPool) {
                         // Fused 2x2 max pooling from the finished values in the staging tile: the 32 rows hold 8 whole
@@ -675,7 +716,7 @@ tc_fprop_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                         }
                     }
                 }
-            } else if (vec_ok) {
+            } else if (kEpi == kEpiWarps && vec_ok) {
                 // Coalesced path.  Each lane owns one row (pixel) of the accumulator, but a row's 32 columns
                 // are 128 contiguous bytes in global memory, so the chunk is first transposed through a
                 // 4 KB per-warp staging tile (XOR-swizzled 16-byte slots: conflict-free both ways) and then
@@ -689,9 +730,9 @@ tc_fprop_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                     roff[i] = __shfl_sync(0xffffffffu, static_cast<unsigned long long>(pix * p.Kout), src);
                     vmask |= (__shfl_sync(0xffffffffu, static_cast<int>(valid), src) ? 1u : 0u) << i;
                 }
-                const uint32_t stg = smem_u32(epi_stage + (warp - 2) * 4096);
+                const uint32_t stg = smem_u32(epi_stage + epi * 4096);
                 const int cg = (lane & 7) * 4;
-                for (int ch = chalf; ch < p.BN / 32; ch += 2) {
+                for (int ch = ch0; ch < cpb; ch += kSub) {
                     const int col = kt * p.BN + ch * 32 + cg;
                     // (the bias is fetched before the accumulator so that its latency hides behind the staging)
                     float4 b = make_float4(0.f, 0.f, 0.f, 0.f);
@@ -699,7 +740,7 @@ tc_fprop_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                     uint32_t v[32];
                     tmem_ld_32x32(t_row + ch * 32, v);
                     tmem_ld_wait();
-                    if (!kPool && p.split_acc) add_second_accumulator(t_row + t_second + ch * 32, v);
+                    if (!kPool && kEpi == kEpiWarps && p.split_acc) add_second_accumulator(t_row + t_second + ch * 32, v);
 #pragma unroll
                     for (int j = 0; j < 8; ++j) {
                         const int slot = j ^ (lane & 7);
@@ -786,12 +827,12 @@ tc_fprop_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                     }
                     __syncwarp();
                 }
-            } else {
-                for (int ch = chalf; ch < p.BN / 32; ch += 2) {
+            } else if (kEpi == kEpiWarps) {
+                for (int ch = ch0; ch < cpb; ch += kSub) {
                     uint32_t v[32];
                     tmem_ld_32x32(t_row + ch * 32, v);
                     tmem_ld_wait();
-                    if (!kPool && p.split_acc) add_second_accumulator(t_row + t_second + ch * 32, v);
+                    if (!kPool && kEpi == kEpiWarps && p.split_acc) add_second_accumulator(t_row + t_second + ch * 32, v);
                     const int col0 = kt * p.BN + ch * 32;
                     if (valid && col0 < p.Kout) {
                         float* dst = p.out + pix * p.Kout + col0;
@@ -1032,10 +1073,12 @@ int launch_tc_fprop(const TcFpropArgs& a, cudaStream_t st) {
     static bool attr_set = false;
     if (!attr_set) {
         if (ensure_device_setup() != PCL_OK) return PCL_ERR_CUDA;
-        const void* kernels[6] = {
+        const void* kernels[8] = {
             (const void*)tc_fprop_kernel<false, false, false>, (const void*)tc_fprop_kernel<false, true, false>,
             (const void*)tc_fprop_kernel<false, false, true>,  (const void*)tc_fprop_kernel<true, false, false>,
-            (const void*)tc_fprop_kernel<true, true, false>,   (const void*)tc_fprop_kernel<true, false, true>};
+            (const void*)tc_fprop_kernel<true, true, false>,   (const void*)tc_fprop_kernel<true, false, true>,
+            (const void*)tc_fprop_kernel<false, false, false, kEpiWarpsWide>,
+            (const void*)tc_fprop_kernel<false, true, false, kEpiWarpsWide>};
         for (const void* k : kernels)
             if (cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget + 1024) != cudaSuccess)
                 return PCL_ERR_CUDA;
@@ -1147,10 +1190,26 @@ int launch_tc_fprop(const TcFpropArgs& a, cudaStream_t st) {
         if (make_tmap(&tmOut, a.out, 4, dims, strides, box, false, true) == PCL_OK) p.tma_store = 1;
         else tmOut = tmA;
     }
+    // Sixteen epilogue warps where the epilogue bounds the tile: estimated cycles of a box's MMAs (a K8 step of
+    // BN <= 64 columns takes ~50 cycles, wider ones BN/2) against ~1600 cycles per 32-column chunk and warp.  Their
+    // staging tiles take 32 KB more; the ring gives up slots for them as long as three remain.
+    bool wide_epi = false;
+    const int epi_hook = env_int("PCL_EPI_WARPS", 16);      // test hook: 8 = never, 32 = wherever the variant can run
+    if (!cfg.pair && p.tma_store && !p.split_acc && epi_hook >= 16) {
+        const long mma_clk = long(a.R) * a.S * p.cblocks * 4 * (p.BN <= 64 ? 50 : p.BN / 2);
+        const long epi_clk = long(p.BN / 32) * 1600 / 2;
+        if (2 * epi_clk > 3 * mma_clk || epi_hook >= 32) {
+            const int slot = p.KS * (p.halo ? p.BN * 128 : kABytes + p.BN * 128);
+            const int fixed = (p.halo ? p.NA * p.a_buf_bytes : 0) + kEpiStageBytesWide;
+            int stages = p.stages;
+            while (stages > 3 && fixed + stages * slot > kSmemBudget) --stages;
+            if (fixed + stages * slot <= kSmemBudget) { p.stages = stages; wide_epi = true; }
+        }
+    }
     const long total = m_tiles * p.tiles_k;
     const size_t smem = (p.halo ? size_t(p.NA) * p.a_buf_bytes + size_t(p.stages) * p.KS * (cfg.pair ? p.BN * 64 : p.BN * 128)
                                 : size_t(p.stages) * p.KS * (kABytes + (cfg.pair ? p.BN * 64 : p.BN * 128))) +
-                        kEpiStageBytes + 1024;
+                        (wide_epi ? kEpiStageBytesWide : kEpiStageBytes) + 1024;
     if (cfg.pair) {
         cudaLaunchAttribute attr[1];
         attr[0].id = cudaLaunchAttributeClusterDimension;
@@ -1179,7 +1238,9 @@ int launch_tc_fprop(const TcFpropArgs& a, cudaStream_t st) {
     } else {
         const int grid = int(total < g_sm_count ? total : g_sm_count);
         LaunchScope scope(KID_TC_FPROP, 2.0 * a.N * a.P * a.Q * double(a.Kout) * a.Cin * a.R * a.S, st);
-        if (p.pool_out) tc_fprop_kernel<false, true, false><<<grid, kThreads, smem, st>>>(tmA, tmB, tmOut, p);
+        if (wide_epi && p.pool_out) tc_fprop_kernel<false, true, false, kEpiWarpsWide><<<grid, kThreadsWide, smem, st>>>(tmA, tmB, tmOut, p);
+        else if (wide_epi) tc_fprop_kernel<false, false, false, kEpiWarpsWide><<<grid, kThreadsWide, smem, st>>>(tmA, tmB, tmOut, p);
+        else if (p.pool_out) tc_fprop_kernel<false, true, false><<<grid, kThreads, smem, st>>>(tmA, tmB, tmOut, p);
         else if (p.mask_src) tc_fprop_kernel<false, false, true><<<grid, kThreads, smem, st>>>(tmA, tmB, tmOut, p);
         else tc_fprop_kernel<false, false, false><<<grid, kThreads, smem, st>>>(tmA, tmB, tmOut, p);
     }

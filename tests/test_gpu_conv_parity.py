@@ -170,6 +170,29 @@ def test_forward_type_kernel_pipeline_variants(tag, variant, path_guard, monkeyp
     assert B.last_device_status() == 0
 
 
+@pytest.mark.parametrize("tiling", ["plain", "halo0", "halo1", "halo2", "auto"])
+@pytest.mark.parametrize("tag", sorted(PIPELINE_SHAPES))
+def test_forward_with_sixteen_epilogue_warps(tag, tiling, path_guard, monkeypatch):
+    """Launches with a very short reduction run sixteen epilogue warps instead of eight (four per TMEM lane
+    quarter share a tile's 32-column chunks).  PCL_EPI_WARPS=32 forces that variant wherever it can run: the
+    result must equal the eight-warp variant's bit for bit (same accumulators, same epilogue arithmetic)."""
+    import gpu_helpers as G
+    from paper_1602_06709_b200 import binding as B
+    monkeypatch.setenv("PCL_TILING", tiling)
+    monkeypatch.setenv("PCL_PAIR", "0")
+    monkeypatch.setenv("PCL_SPLIT_ACC", "0")
+    B.set_path(B.PATH_TENSOR)
+    s = PIPELINE_SHAPES[tag]
+    x, w, dy, bias = G.make_inputs(s, "epi16_" + tag)
+    res = {}
+    for warps in ("8", "32"):
+        monkeypatch.setenv("PCL_EPI_WARPS", warps)
+        res[warps] = G.run_conv_fwd(s, x, w, bias, B.ACT_RELU)
+    G.assert_parity(res["32"], oracle.conv_fwd(s, x, w, bias, oracle.ACT_RELU), f"fwd {tiling}")
+    assert np.array_equal(res["8"], res["32"])
+    assert B.last_device_status() == 0
+
+
 @pytest.mark.parametrize("tiling", ["plain", "halo1", "auto"])
 @pytest.mark.parametrize("tag", ["odd_groups", "even_groups_wide", "fc_like"])
 def test_backward_data_reads_weights_in_place(tag, tiling, path_guard, monkeypatch):

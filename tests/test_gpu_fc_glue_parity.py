@@ -187,7 +187,7 @@ POOL_FUSED_SHAPES = [
 ]
 
 
-@pytest.mark.parametrize("store", ["tma", "direct"])
+@pytest.mark.parametrize("store", ["tma", "direct", "tma_16_epilogue_warps"])
 @pytest.mark.parametrize("tiling", ["auto", "plain", "halo0", "halo1", "halo2"])
 @pytest.mark.parametrize("shape", POOL_FUSED_SHAPES)
 def test_conv_fwd_with_fused_maxpool(shape, tiling, store, monkeypatch):
@@ -200,7 +200,11 @@ def test_conv_fwd_with_fused_maxpool(shape, tiling, store, monkeypatch):
     if tiling != "auto":
         monkeypatch.setenv("PCL_TILING", tiling)
     # the epilogue writes y either with TMA stores from its staging tiles or with per-lane coalesced stores
-    monkeypatch.setenv("PCL_TMA_STORE", "1" if store == "tma" else "0")
+    monkeypatch.setenv("PCL_TMA_STORE", "0" if store == "direct" else "1")
+    # the kernel variant with sixteen epilogue warps (chosen by itself only for very short reductions), single CTAs
+    monkeypatch.setenv("PCL_EPI_WARPS", "32" if store == "tma_16_epilogue_warps" else "8")
+    if store == "tma_16_epilogue_warps":
+        monkeypatch.setenv("PCL_PAIR", "0")
     N, C, K, H, W = shape
     s = ConvShape(N=N, C=C, K=K, H=H, W=W, R=3, S=3, pad_h=1, pad_w=1)
     x, w, _, bias = G.make_inputs(s, f"fwdpool{C}_{K}")
