@@ -61,7 +61,43 @@ class _ConvLayer:
     pool: bool
     desc: object = None
 
-class _HostFeed:
+class _GraphStep:
+    """A step is a fixed sequence of launches on fixed buffers, so it can be captured once into a CUDA graph and
+    replayed with a single launch (the DNN step is ~45 short kernels: issued one by one, the host's launch rate
+    bounds it).  One graph per input buffer: the host feed alternates between two."""
+
+    _graphs = None
+
+    def capture_step(self):
+        """Call once, after construction (or after any eager steps).  The library's one-time setup (function
+        attributes, its device status word) must not fall into the capture, so one eager step runs first, with the
+        parameters put back afterwards."""
+        saved = self.store.params.clone()
+        self.step()
+        torch.cuda.synchronize()
+        self.store.params.copy_(saved)
+        del saved
+        self._graphs = {}
+        for _ in range(2):
+            g = torch.cuda.CUDAGraph()
+            n0 = B.launch_count()
+            with torch.cuda.graph(g):
+                self.step()
+            self.graph_launches = B.launch_count() - n0       # kernels one replay launches
+            self._graphs[self.x.data_ptr()] = g
+            self.x, self._alt_x = self._alt_x, self.x
+            self.labels, self._alt_labels = self._alt_labels, self.labels
+
+    def run_step(self):
+        """step(), through the captured graph when there is one for the current input buffer."""
+        g = self._graphs.get(self.x.data_ptr()) if self._graphs else None
+        if g is None:
+            self.step()
+        else:
+            g.replay()
+
+
+class _HostFeed(_GraphStep):
     """Host-side input feed shared by the step drivers: the minibatch of a step is copied from pinned host
     memory, and the copy of the NEXT minibatch can run on a second stream while this step computes (two
     device input buffers that swap).  Buffers and call order only; no arithmetic of the method."""
@@ -92,7 +128,7 @@ class _HostFeed:
                 self._alt_labels.copy_(next_labels_host, non_blocking=True)
                 self._staged = torch.cuda.Event()
                 self._staged.record(self._copy_stream)
-        self.step()
+        self.run_step()
         return float(self.loss.cpu().item())
 
 

@@ -128,3 +128,45 @@ def test_host_feed_with_overlapped_copy_matches_plain_copies():
     assert np.allclose(l0, l1, rtol=1e-5, atol=0)
     assert np.array_equal(p0, p1)
     assert len(set(l0)) > 1      # the minibatches differ, so a stale buffer would show
+
+
+@pytest.mark.parametrize("kind", ["dnn", "vgg"])
+def test_captured_step_graph_equals_eager_steps(kind):
+    """capture_step() records the step's launches into a CUDA graph (one per input buffer of the host feed);
+    replaying it must leave exactly the parameters that eager steps leave, also with the overlapped host feed
+    that alternates between the two input buffers."""
+    from paper_1602_06709_b200 import inputs, networks
+    if kind == "dnn":
+        N, dims = 64, [40, 96, 64]
+        make = lambda: networks.Dnn(N, dims=dims, cfg="graph_dnn")
+        xshape, classes, normal = (N, dims[0]), dims[-1], True
+    else:
+        N, hw = 4, 32
+        make = lambda: networks.VggA(N, hw=hw, conv=SMALL_CONV, fc=[(64, 128), (128, 128), (128, 10)], classes=10,
+                                     cfg="graph_vgg")
+        xshape, classes, normal = (N, hw, hw, 3), 10, False
+    batches = []
+    for i in range(4):
+        tid = inputs.tensor_id("graph", kind, "x", i)
+        x = inputs.normal(tid, xshape, 1.0) if normal else inputs.uniform(tid, xshape, 0.0, 1.0)
+        lab = inputs.labels(inputs.tensor_id("graph", kind, "labels", i), N, classes)
+        batches.append((torch.from_numpy(x).pin_memory(), torch.from_numpy(lab).pin_memory()))
+
+    def run(graph, overlap):
+        net = make()
+        before = net.store.params.cpu().numpy().copy()
+        if graph:
+            net.capture_step()
+            assert np.array_equal(net.store.params.cpu().numpy(), before)       # capturing changes nothing
+        losses = []
+        for i, (x, lab) in enumerate(batches):
+            nxt = batches[i + 1] if overlap and i + 1 < len(batches) else (None, None)
+            losses.append(net.step_from_host(x, lab, nxt[0], nxt[1]))
+        return losses, net.store.params.cpu().numpy().copy()
+
+    l0, p0 = run(False, False)
+    for overlap in (False, True):
+        l1, p1 = run(True, overlap)
+        assert np.allclose(l0, l1, rtol=1e-5, atol=0)       # (the scalar loss is summed with atomics)
+        assert np.array_equal(p0, p1)
+    assert len(set(l0)) > 1
