@@ -195,6 +195,21 @@ WgradPlan plan_wgrad(const pcl_conv_desc& d, int P, int Q) {
     return pl;
 }
 
+// FC weight gradient dw[K][C] = dz^T[K][N] * x[N][C] through the forward-type kernel: its "pixels" are the K output
+// rows, its reduction the minibatch, and x [N][C] is read in place as an MN-major weight operand; only dz has to be
+// transposed (N*K floats).  The weight-gradient kernel proper is built for long reductions (one tile per CTA,
+// epilogue not overlapped); with a minibatch-long reduction its tiles are mostly epilogue, while the forward-type
+// kernel is persistent, overlaps a tile's epilogue with the next tile's MMAs and stores through TMA.
+bool fc_dw_as_forward(int N, int C, int K) {
+    if (g_path.load() == PCL_PATH_GENERIC) return false;
+    if (N % 4 != 0 || C % 32 != 0 || K % 4 != 0) return false;
+    if (const char* v = getenv("PCL_FC_DW_FORWARD")) return atoi(v) != 0;      // test / tuning hook
+    // measured (B200): it pays for a short reduction and a large dw (VGG-A FC1: 0.26 -> 0.13 ms, FC2: 0.052 -> 0.039
+    // with the transpose); at minibatch 1024 (the DNN layers) and for small dw the weight-gradient kernel is as fast
+    return N <= 512 && size_t(K) * C >= (size_t(1) << 23);
+}
+size_t fc_dzt_bytes(int N, int K) { return align_up(size_t(N) * K * 4, 256); }
+
 }  // namespace
 }  // namespace pcl
 
@@ -231,8 +246,11 @@ size_t pcl_fc_workspace_bytes(int N, int C, int K, int pass) {
     if (N <= 0 || C <= 0 || K <= 0) return 0;
     const pcl_conv_desc d{N, C, K, 1, 1, 1, 1, 1, 1, 0, 0};
     if (pass == PCL_PASS_FWD) return 0;
-    // fc_bwd runs both backward contractions; either pass value returns the total
-    return pcl_conv_workspace_bytes(&d, PCL_PASS_BWD_DATA) + pcl_conv_workspace_bytes(&d, PCL_PASS_BWD_WEIGHTS);
+    // fc_bwd runs both backward contractions; either pass value returns the total (the weight-gradient part is
+    // sized for either of its two forms)
+    const size_t wgrad_form = pcl_conv_workspace_bytes(&d, PCL_PASS_BWD_WEIGHTS);
+    const size_t fwd_form = fc_dzt_bytes(N, K) + plan_wgrad(d, 1, 1).colsum_bytes;
+    return pcl_conv_workspace_bytes(&d, PCL_PASS_BWD_DATA) + (wgrad_form > fwd_form ? wgrad_form : fwd_form);
 }
 
 // Forward pass; y_pool != nullptr: also the 2x2 window maxima of y, fused into the tensor-core epilogue where
@@ -541,7 +559,9 @@ int pcl_fc_bwd(int N, int C, int K, const float* x, const float* w, const float*
         !aligned16(dbias))
         return PCL_ERR_MISALIGNED;
     const pcl_conv_desc d{N, C, K, 1, 1, 1, 1, 1, 1, 0, 0};
-    const size_t need_w = pcl_conv_workspace_bytes(&d, PCL_PASS_BWD_WEIGHTS);
+    const bool dw_fwd = fc_dw_as_forward(N, C, K);
+    const size_t colsum_bytes = plan_wgrad(d, 1, 1).colsum_bytes;
+    const size_t need_w = dw_fwd ? fc_dzt_bytes(N, K) + colsum_bytes : pcl_conv_workspace_bytes(&d, PCL_PASS_BWD_WEIGHTS);
     const size_t need_d = dx ? pcl_conv_workspace_bytes(&d, PCL_PASS_BWD_DATA) : 0;
     if (need_w + need_d > 0) {
         if (!ws || ws_bytes < need_w + need_d) return PCL_ERR_WORKSPACE;
@@ -551,7 +571,18 @@ int pcl_fc_bwd(int N, int C, int K, const float* x, const float* w, const float*
     int rc = launch_act_grad(dy, y, size_t(N) * K, act, st);
     if (rc != PCL_OK) return rc;
     // weight gradient first, then backpropagation (the order Sec. 3.1 schedules them in)
-    rc = pcl_conv_bwd_weights(&d, x, dy, dw, dbias, 1, ws, need_w, cuda_stream);
+    if (dw_fwd) {
+        float* dzt = static_cast<float*>(ws);
+        float* cs = reinterpret_cast<float*>(static_cast<char*>(ws) + fc_dzt_bytes(N, K));
+        rc = launch_transpose_flip(dy, dzt, N, 1, 1, K, st);       // dzt[k][n] = dz[n][k]
+        if (rc != PCL_OK) return rc;
+        TcFpropArgs a{dzt, x, nullptr, nullptr, dw, K, 1, 1, N, C, 1, 1, 0, 0, 1, 1, PCL_ACT_NONE};
+        a.wt_mn_major = 1;
+        rc = launch_tc_fprop(a, st);
+        if (rc == PCL_OK && dbias) rc = launch_colsum(dy, size_t(N), K, cs, dbias, st);
+    } else {
+        rc = pcl_conv_bwd_weights(&d, x, dy, dw, dbias, 1, ws, need_w, cuda_stream);
+    }
     if (rc != PCL_OK) return rc;
     if (dx) rc = pcl_conv_bwd_data(&d, dy, w, nullptr, dx, static_cast<char*>(ws) + need_w, need_d, cuda_stream);
     return rc;

@@ -15,6 +15,7 @@ FC_CASES = [
     (257, 36, 1000, "none"),
     (8, 2052, 64, "sigmoid"),
     (300, 32, 32, "none"),
+    (132, 64, 264, "relu"),     # minibatch not a multiple of 32: ragged reduction of the forward-form weight gradient
 ]
 
 
@@ -26,12 +27,17 @@ def path_guard():
 
 
 @pytest.mark.parametrize("N,C,K,act", FC_CASES)
-@pytest.mark.parametrize("path", ["tensor", "generic"])
-def test_fc_fwd_bwd(N, C, K, act, path, path_guard):
+@pytest.mark.parametrize("path", ["tensor", "tensor_dw_forward_form", "tensor_dw_wgrad_form", "generic"])
+def test_fc_fwd_bwd(N, C, K, act, path, path_guard, monkeypatch):
+    """The FC weight gradient has two forms on the tensor path: the weight-gradient kernel, or (short reductions,
+    C % 32 == 0) the forward-type kernel over dz^T with x read in place as an MN-major operand;
+    PCL_FC_DW_FORWARD pins one."""
     import gpu_helpers as G
     from paper_1602_06709_b200 import binding as B
     from paper_1602_06709_b200 import inputs
-    B.set_path(B.PATH_TENSOR if path == "tensor" else B.PATH_GENERIC)
+    if path.startswith("tensor_dw"):
+        monkeypatch.setenv("PCL_FC_DW_FORWARD", "1" if "forward" in path else "0")
+    B.set_path(B.PATH_GENERIC if path == "generic" else B.PATH_TENSOR)
     code = {"none": B.ACT_NONE, "relu": B.ACT_RELU, "sigmoid": B.ACT_SIGMOID}[act]
     tid = lambda r: inputs.tensor_id("fc", N, C, K, r)
     x = inputs.normal(tid("x"), (N, C), 1.0)
