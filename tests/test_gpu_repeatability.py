@@ -42,3 +42,30 @@ def test_passes_repeat_bit_for_bit(name, N, C, K, H, R, pad):
         else:
             for a, o in zip(ref, outs):
                 assert a is None or torch.equal(a, o)
+
+
+@pytest.mark.parametrize("name,N,C,K,H", [("first", 32, 3, 64, 224), ("narrow", 32, 64, 128, 112), ("wide", 32, 256, 256, 56)])
+def test_forward_with_pool_repeats_bit_for_bit(name, N, C, K, H):
+    """conv -> ReLU -> 2x2 pool in one launch, with and without the full-resolution output stored (the first layer
+    runs the sixteen-epilogue-warp variant): pooled tensor and position codes identical across launches and
+    between the two forms."""
+    from paper_1602_06709_b200 import binding as B
+    d = B.conv_desc(N, C, K, H, H, 3, 3, 1, 1)
+    assert B.conv_fwd_pool_is_fused(d)
+    g = torch.Generator(device="cuda").manual_seed(709)
+    x = torch.rand(N, H, H, C, device="cuda", generator=g)
+    w = torch.randn(K, 3, 3, C, device="cuda", generator=g) * 0.05
+    b = torch.randn(K, device="cuda", generator=g) * 0.1
+    ws = torch.empty(max(256, B.conv_workspace_bytes(d, B.PASS_FWD)), dtype=torch.uint8, device="cuda")
+    ref = None
+    for i in range(8):
+        yp = torch.full((N, H // 2, H // 2, K), float("nan"), device="cuda")
+        codes = torch.full((N, H // 2, H // 2, K), 255, dtype=torch.uint8, device="cuda")
+        y = torch.empty(N, H, H, K, device="cuda") if i % 2 else None
+        B.conv_fwd_pool(d, x, w, b, y, yp, B.ACT_RELU, ws, pool_codes=codes)
+        B.check_device_status()
+        if ref is None:
+            ref = (yp, codes)
+        else:
+            assert torch.equal(ref[0], yp) and torch.equal(ref[1], codes)
+    assert int(ref[1].max()) <= 7 and not torch.isnan(ref[0]).any()
