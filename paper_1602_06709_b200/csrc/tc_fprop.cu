@@ -24,6 +24,7 @@
 //   warp 10       second issuing thread for single-CTA tiles with many slots
 //   warps 2-9     epilogue: TMEM -> registers -> bias / activation / mask [/ column sums / 2x2 max pool]
 //                 -> global, through TMA stores or coalesced per-lane stores (two warps per TMEM lane quarter)
+//   warps 11-18   eight more epilogue warps (608 threads) in the variant for tiles with a very short reduction
 // Two TMEM accumulator sets let the epilogue of tile i overlap the main loop of tile i+1.
 #include <stdlib.h>
 
