@@ -289,16 +289,23 @@ def oracle_sample(workload: str):
     raise ValueError(workload)
 
 
-def time_oracle(workload: str, steps: int, warmup: int):
+def time_oracle(workload: str, steps: int, warmup: int, min_seconds: float = 0.0):
+    """steps > 0: exactly that many timed calls of the bounded sample.  min_seconds > 0 (the cpu_baseline leg): the
+    sample is repeated until about that much CPU time has been measured (at most 16 calls)."""
     import oracle
     fn, units, sample = oracle_sample(workload)
     for _ in range(warmup):
         fn()
     t0 = time.perf_counter()
-    for _ in range(steps):
+    done = 0
+    while done < steps or (min_seconds > 0 and done < 16 and time.perf_counter() - t0 < min_seconds):
         fn()
+        done += 1
     dt = time.perf_counter() - t0
-    return dict(value=units * steps / dt, seconds_per_step=dt / steps, cores=oracle.threads(), sample=sample)
+    if done > 1 and min_seconds > 0:
+        sample += f", {done} calls"
+    return dict(value=units * done / dt, seconds_per_step=dt / done, cores=oracle.threads(), sample=sample,
+                seconds=dt)
 
 
 def run_reference(args):
@@ -442,9 +449,9 @@ def run_ours(args):
 
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
-        r = time_oracle(args.workload, 1, 0)
+        r = time_oracle(args.workload, 1, 0, min_seconds=12.0)
         cpu = dict(value=r["value"], unit=wl.unit, cores=r["cores"], kind="oracle", sample=r["sample"],
-                   seconds=r["seconds_per_step"])
+                   seconds=r["seconds"])
 
     if rank == 0:
         line = {
