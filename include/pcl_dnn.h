@@ -144,6 +144,25 @@ int pcl_conv_bwd_weights(const pcl_conv_desc* d, const float* x, const float* dy
                          float* dw, float* dbias, int deterministic,
                          void* ws, size_t ws_bytes, void* cuda_stream);
 
+/* Weight-gradient update of a layer whose output went through the 2x2 / stride-2 max pool (the
+ * conv -> ReLU -> pool blocks of the VGG-A topology, Sec. 5), taken straight from the POOLED gradient:
+ *   dy[n,p,q,k] = dy_pool[n,p/2,q/2,k]  where (p%2)*2 + q%2 == pool_codes[n,p/2,q/2,k] & 3
+ *                                       (and, if relu_mask != 0, bit 2 of that code is clear), else 0;
+ *   dw, dbias as pcl_conv_bwd_weights() of that dy (two-pass, bitwise reproducible).
+ * I.e. pcl_maxpool2x2_bwd_codes() followed by pcl_conv_bwd_weights(), but dy is never written to or
+ * read from memory: the kernel builds its dy tiles on chip.  For a layer with no backward-data pass of
+ * its own (the first layer: Sec. 3.1 skips its backpropagation) nothing else needs dy.
+ * dy_pool: [N][out_h/2][out_w/2][K] in, pool_codes: same shape, bytes, in (codes as written by
+ * pcl_conv_fwd_pool / pcl_maxpool2x2_fwd_codes), both 16-byte aligned; dbias: [K] out or NULL.
+ * Available where pcl_conv_bwd_weights_pooled_is_fused(d) != 0 (the few-channel first-layer path, even
+ * out_h and out_w, K % 4 == 0); elsewhere PCL_ERR_UNSUPPORTED_SHAPE (run the two calls instead).
+ * Workspace: pcl_conv_bwd_weights_pooled_workspace_bytes(d), 256-byte aligned. */
+int pcl_conv_bwd_weights_pooled_is_fused(const pcl_conv_desc* d);
+size_t pcl_conv_bwd_weights_pooled_workspace_bytes(const pcl_conv_desc* d);
+int pcl_conv_bwd_weights_pooled(const pcl_conv_desc* d, const float* x, const float* dy_pool,
+                                const unsigned char* pool_codes, int relu_mask, float* dw, float* dbias,
+                                void* ws, size_t ws_bytes, void* cuda_stream);
+
 /* Fully-connected forward: the k_h = k_w = out_h = out_w = 1 case of Algorithm 1
  * (Sec. 2.1):  y[n,k] = act(bias[k] + sum_c x[n,c] * w[k,c]).
  * x: [N][C], w: [K][C], bias: [K] or NULL, y: [N][K].

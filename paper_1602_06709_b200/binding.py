@@ -28,6 +28,7 @@ EXPORTS = [
     "pcl_last_device_status", "pcl_launch_count", "pcl_status_string", "pcl_profile_begin", "pcl_profile_end", "pcl_conv_bwd_data_noalloc", "pcl_noalloc_scratch_bytes",
     "pcl_conv_bwd_data_colsum_workspace_bytes", "pcl_conv_bwd_data_colsum",
     "pcl_maxpool2x2_bwd_colsum_workspace_bytes", "pcl_maxpool2x2_bwd_colsum", "pcl_conv_fwd_pool", "pcl_conv_fwd_pool_is_fused",
+    "pcl_conv_bwd_weights_pooled", "pcl_conv_bwd_weights_pooled_is_fused", "pcl_conv_bwd_weights_pooled_workspace_bytes",
     "pcl_maxpool2x2_fwd_codes", "pcl_maxpool2x2_bwd_codes", "pcl_last_wait_code",
 ]
 
@@ -71,6 +72,10 @@ def lib() -> ctypes.CDLL:
         L.pcl_conv_bwd_data.argtypes = [dp, vp, vp, vp, vp, vp, sz, vp]
         L.pcl_conv_fwd_pool.argtypes = [dp, vp, vp, vp, vp, vp, vp, ci, vp, sz, vp]
         L.pcl_conv_fwd_pool_is_fused.argtypes = [dp]
+        L.pcl_conv_bwd_weights_pooled_is_fused.argtypes = [dp]
+        L.pcl_conv_bwd_weights_pooled_workspace_bytes.argtypes = [dp]
+        L.pcl_conv_bwd_weights_pooled_workspace_bytes.restype = sz
+        L.pcl_conv_bwd_weights_pooled.argtypes = [dp, vp, vp, vp, ci, vp, vp, vp, sz, vp]
         L.pcl_maxpool2x2_fwd_codes.argtypes = [ci, ci, ci, ci, vp, vp, vp, vp]
         L.pcl_maxpool2x2_bwd_codes.argtypes = [ci, ci, ci, ci, vp, vp, ci, vp, vp, vp, sz, vp]
         L.pcl_conv_bwd_weights.argtypes = [dp, vp, vp, vp, vp, ci, vp, sz, vp]
@@ -163,6 +168,21 @@ def conv_fwd_pool(d, x, w, bias, y, y_pool, act=ACT_NONE, ws=None, stream=None, 
     wp, wb = _ws(ws)
     _check(lib().pcl_conv_fwd_pool(ctypes.byref(d), _ptr(x), _ptr(w), _ptr(bias), _ptr(y), _ptr(y_pool),
                                    _ptr(pool_codes), act, wp, wb, _stream(stream)), "pcl_conv_fwd_pool")
+
+
+def conv_bwd_weights_pooled_is_fused(d) -> bool:
+    return bool(lib().pcl_conv_bwd_weights_pooled_is_fused(ctypes.byref(d)))
+
+
+def conv_bwd_weights_pooled_workspace_bytes(d) -> int:
+    return int(lib().pcl_conv_bwd_weights_pooled_workspace_bytes(ctypes.byref(d)))
+
+
+def conv_bwd_weights_pooled(d, x, dy_pool, pool_codes, relu_mask, dw, dbias=None, ws=None, stream=None):
+    wp, wb = _ws(ws)
+    _check(lib().pcl_conv_bwd_weights_pooled(ctypes.byref(d), _ptr(x), _ptr(dy_pool), _ptr(pool_codes),
+                                             int(bool(relu_mask)), _ptr(dw), _ptr(dbias), wp, wb, _stream(stream)),
+           "pcl_conv_bwd_weights_pooled")
 
 
 def maxpool2x2_fwd_codes(N, H, W, C, x, y, codes, stream=None):

@@ -488,6 +488,74 @@ int pcl_maxpool2x2_bwd_codes(int N, int H, int W, int C, const unsigned char* co
     return launch_colsum(dx, size_t(N) * H * W, C, static_cast<float*>(ws), dx_colsum, st);
 }
 
+namespace {
+// Pooled-dy form of the few-channel weight gradient: splits and workspace layout [staged x][per-split dw tiles]
+// [per-split bias-gradient rows].
+struct PooledWgradPlan { bool ok; int splits; size_t tiles_off, rows_off, cs_off, total; };
+PooledWgradPlan plan_pooled_wgrad(const pcl_conv_desc& d, int P, int Q) {
+    PooledWgradPlan pl{};
+    if (!few_channel_path_for(d, PCL_PASS_BWD_WEIGHTS)) return pl;
+    if (!tc_wgrad_can_take_pooled_dy(d.N, P, Q, d.S * 4, d.K, d.R, 1, 1)) return pl;
+    pl.ok = true;
+    pl.splits = tc_wgrad_splits(d.N, P, Q, d.S * 4, d.K, d.R, 1, 1, 1);
+    pl.tiles_off = staged_x_bytes(d);
+    pl.rows_off = pl.tiles_off + size_t(pl.splits) * staged_w_bytes(d);
+    pl.cs_off = pl.rows_off + align_up(size_t(pl.splits) * 8 * d.K * 4, 256);      // one row per (split, epilogue warp)
+    const int cs = colsum_splits(size_t(pl.splits) * 8);
+    pl.total = pl.cs_off + (cs > 1 ? align_up(size_t(cs) * d.K * 4, 256) : 0);
+    return pl;
+}
+}  // namespace
+
+int pcl_conv_bwd_weights_pooled_is_fused(const pcl_conv_desc* d) {
+    int P, Q;
+    if (check_desc(d, &P, &Q) != PCL_OK) return 0;
+    return plan_pooled_wgrad(*d, P, Q).ok ? 1 : 0;
+}
+
+size_t pcl_conv_bwd_weights_pooled_workspace_bytes(const pcl_conv_desc* d) {
+    int P, Q;
+    if (check_desc(d, &P, &Q) != PCL_OK) return 0;
+    return plan_pooled_wgrad(*d, P, Q).total;
+}
+
+int pcl_conv_bwd_weights_pooled(const pcl_conv_desc* d, const float* x, const float* dy_pool,
+                                const unsigned char* pool_codes, int relu_mask, float* dw, float* dbias, void* ws,
+                                size_t ws_bytes, void* cuda_stream) {
+    int P, Q;
+    int rc = check_desc(d, &P, &Q);
+    if (rc != PCL_OK) return rc;
+    if (!x || !dy_pool || !pool_codes || !dw) return PCL_ERR_BAD_ARG;
+    if (!aligned16(x) || !aligned16(dy_pool) || !aligned16(pool_codes) || !aligned16(dw) || !aligned16(dbias))
+        return PCL_ERR_MISALIGNED;
+    const PooledWgradPlan pl = plan_pooled_wgrad(*d, P, Q);
+    if (!pl.ok) return PCL_ERR_UNSUPPORTED_SHAPE;
+    if (!ws || ws_bytes < pl.total) return PCL_ERR_WORKSPACE;
+    if (reinterpret_cast<uintptr_t>(ws) & 255) return PCL_ERR_MISALIGNED;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    float* xs = static_cast<float*>(ws);
+    float* dw4 = reinterpret_cast<float*>(static_cast<char*>(ws) + pl.tiles_off);
+    float* rows = reinterpret_cast<float*>(static_cast<char*>(ws) + pl.rows_off);
+    float* cs = reinterpret_cast<float*>(static_cast<char*>(ws) + pl.cs_off);
+    rc = launch_stage_pad_c4(x, xs, d->N, d->H, d->W, d->C, d->pad_h, d->pad_w, st);
+    if (rc != PCL_OK) return rc;
+    const int Hp = d->H + 2 * d->pad_h, Wp = d->W + 2 * d->pad_w;
+    const size_t taps = size_t(d->K) * d->R * d->S;
+    TcWgradArgs a{xs, nullptr, dw4, pl.splits > 1 ? dw4 : nullptr, d->N, Hp, Q, d->S * 4, d->K, d->R, 1, 0, 0, P, Q,
+                  pl.splits};
+    a.x_stride_w = 4; a.x_stride_h = long(Wp) * 4; a.x_stride_n = long(Hp) * Wp * 4;
+    a.x_inner = 32;
+    a.tap_groups = 1;
+    a.skip_reduce = 1;
+    a.dy_pool = dy_pool; a.codes = pool_codes; a.relu_mask = relu_mask ? 1 : 0; a.db_rows = dbias ? rows : nullptr;
+    rc = launch_tc_wgrad(a, st);
+    if (rc != PCL_OK) return rc;
+    rc = launch_unpad_reduce(dw4, dw, taps, d->C, pl.splits, taps * 4, st);
+    if (rc != PCL_OK) return rc;
+    if (dbias) rc = launch_colsum(rows, size_t(pl.splits) * 8, d->K, cs, dbias, st);       // adds the rows, fixed order
+    return rc;
+}
+
 int pcl_conv_bwd_weights(const pcl_conv_desc* d, const float* x, const float* dy, float* dw, float* dbias,
                          int deterministic, void* ws, size_t ws_bytes, void* cuda_stream) {
     int P, Q;

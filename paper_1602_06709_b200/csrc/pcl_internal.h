@@ -104,9 +104,19 @@ struct TcWgradArgs {
     int tap_groups = 0;
     // skip_reduce != 0: leave the per-split partial tiles in `partial` (the caller reduces them).
     int skip_reduce = 0;
+    // Pooled dy: `dy` is null and the kernel builds its dy tiles from dy_pool [N][P/2][Q/2][K] and the pooling
+    // windows' position codes (same shape, bytes): the coded position of each window gets the gradient, the other
+    // three zero; relu_mask: windows whose code has bit 2 set get nothing.  db_rows (optional, [splits * 8][K]) gets
+    // per-(split, epilogue warp) sums of the scattered gradient, i.e. the bias gradient before the rows are added.
+    // Needs even P and Q, K % 4 == 0, single-CTA items (tc_wgrad_can_take_pooled_dy()).
+    const float* dy_pool = nullptr;
+    const unsigned char* codes = nullptr;
+    int relu_mask = 0;
+    float* db_rows = nullptr;
 };
 bool tc_wgrad_eligible(const TcWgradArgs& a);
-int tc_wgrad_splits(int N, int P, int Q, int C, int K, int R, int S, int tap_groups = 0);
+bool tc_wgrad_can_take_pooled_dy(int N, int P, int Q, int C, int K, int R, int S, int tap_groups);
+int tc_wgrad_splits(int N, int P, int Q, int C, int K, int R, int S, int tap_groups = 0, int pooled_dy = 0);
 int launch_tc_wgrad(const TcWgradArgs& a, cudaStream_t st);
 
 // ---- generic CUDA-core kernels (any stride / pad / channel count) ----------

@@ -24,6 +24,14 @@
 // workspace (second pass adds the splits in a fixed order) or adds it to dw with
 // fp32 atomics.
 //
+// Pooled dy ("dy_pool" launches, for a layer whose output went through a 2x2 max pool and that has no
+// backward-data pass of its own, i.e. the first layer): dy is never materialised.  The eight epilogue warps, idle
+// during the main loop, build each k-step's dy tile in shared memory themselves from the pooled gradient and the
+// windows' position codes (one (pooled pixel, 4 maps) item per thread: the gradient goes to the coded position of
+// the window, zeros to the other three, everything rounded to TF32 as a TMA load would), in exactly the layout a
+// TMA load of dy produces (rows of 128 bytes per pixel and 32-map group, 32-byte chunks XOR-ed with row & 3), and
+// arrive on the slot's barrier next to the x copy.  They also sum what they scatter: the bias gradient.
+//
 // A k-step is one pixel box of 32 or 64 pixels (4 or 8 MMAs of 8 pixels).  With an
 // even number of k tiles, two CTAs of a cluster take k tiles 2i and 2i+1 of the
 // same run block and pixel split: each loads its own dy tile and half of the x
@@ -40,6 +48,7 @@ namespace {
 constexpr int kMaxStages = 8;
 constexpr int kWgradThreads = 320;     // warp 0 producer, warp 1 MMA issuer, warps 2-9 epilogue (two per TMEM lane quarter)
 constexpr int kSmemBudget = 224 * 1024;
+constexpr int kExpanderWarps = 8;      // the epilogue warps, which build the dy tiles of pooled-dy launches during the main loop
 
 struct WgradParams {
     int bw_log2, bh_log2;     // pixel box bw x bh x (pix/(bw*bh))
@@ -60,6 +69,13 @@ struct WgradParams {
     int grouped;              // x: 5-D tensor map (one TMA instruction per run) or 4-D per-group boxes (L == 1)
     int grouped_dy;           // dy: 5-D tensor map (all four 32-map groups in one instruction)
     int x_taprows;            // x: 5-D map whose 5th dimension is the tap row (few-channel path): one instruction per k-step
+    // pooled dy (see the header): dy_pool [N][P/2][Q/2][K], codes the same shape in bytes (bits 0-1 position in the
+    // window, bit 2 "maximum <= 0"); relu_mask: windows with bit 2 set contribute nothing; db_rows [splits * 8][K]
+    const float* dy_pool;
+    const unsigned char* codes;
+    int relu_mask;
+    float* db_rows;
+    int N, P, Q;              // output size (for the pooled tile's bounds)
     float* out;               // dw, or the partial-sum workspace [splits][K*R*S*C]
     size_t split_stride;      // K*R*S*C (0 when writing straight to dw)
     unsigned int* status;     // device status word
@@ -96,11 +112,11 @@ tc_wgrad_kernel(const __grid_constant__ CUtensorMap tmDy, const __grid_constant_
     const uint32_t a_bytes = 4 * group_bytes;         // 128 output maps
     const uint32_t step_bytes = a_bytes + (kPair ? (p.rpi >> 1) : p.rpi) * p.L * group_bytes;   // one k-step (same for every item)
     const uint32_t stage_bytes = p.KS * step_bytes;                     // a slot holds KS k-steps
-    const uint32_t tx_bytes = a_bytes + my_runs * p.L * group_bytes;
+    const uint32_t tx_bytes = (p.dy_pool ? 0u : a_bytes) + my_runs * p.L * group_bytes;   // (pooled dy: written by the epilogue warps)
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < p.stages; ++s) {
-            mbar_init(&full_bar[s], 1);
+            mbar_init(&full_bar[s], p.dy_pool ? 1 + kExpanderWarps : 1);     // + one arrival per warp that builds dy
             mbar_init(&empty_bar[s], 1);
         }
         mbar_init(&tmem_full_bar, 1);
@@ -169,7 +185,9 @@ tc_wgrad_kernel(const __grid_constant__ CUtensorMap tmDy, const __grid_constant_
                     else if (pair_rank == 0) mbar_expect_tx_addr(full_a, 2 * nst * tx_bytes);
                     dst = slot_a;
                 }
-                if (p.grouped_dy) {
+                if (p.dy_pool) {
+                    // (no dy copy: the epilogue warps write the tile)
+                } else if (p.grouped_dy) {
                     tma_load_5d_addr<kPair>(dst, &tmDy, full_dst, 0, q0, p0, n0, kt * 4);
                 } else {
 #pragma unroll
@@ -255,8 +273,135 @@ tc_wgrad_kernel(const __grid_constant__ CUtensorMap tmDy, const __grid_constant_
         const int k = kt * 128 + quarter * 32 + lane;
         const bool valid = k < p.K;
         const bool vec_ok = (p.C & 3) == 0;
+        float4 db_acc[2] = {make_float4(0.f, 0.f, 0.f, 0.f), make_float4(0.f, 0.f, 0.f, 0.f)};
+        const int t = int(threadIdx.x) - 64;                 // 0 .. 255 among the epilogue warps
+        int maps_here = p.K - kt * 128;                      // output maps of this k tile
+        if (maps_here > 128) maps_here = 128;
+        const int units = maps_here >> 2;                    // 4-map units of the tile (K % 4 == 0)
+        if (p.dy_pool) {
+            // ---------------------------------------------------- builds the dy tiles (pooled-dy launches)
+            const int hw = bw >> 1, hh = bh >> 1;             // the box in pooled pixels (bw, bh are even)
+            const int ppix = p.pix >> 2;
+            const int items = ppix * units;                   // (pooled pixel, 4-map unit) items per k-step: <= 512
+            const int P2 = p.P >> 1, Q2 = p.Q >> 1;
+            const uint32_t ring0 = smem_u32(smem);
+            int stage = 0, sub = 0;
+            uint32_t phase = 0, dstA = ring0;
+            int qi = box_begin % p.boxes_q;
+            int pi = (box_begin / p.boxes_q) % p.boxes_p;
+            int ni = box_begin / (p.boxes_q * p.boxes_p);
+            bool ok = true;
+            // this thread's (at most two) items: pooled pixel j of the box and 4-map unit u, the same in every k-step
+            int item_w[2], item_h[2], item_n[2];
+            uint32_t rowoff[2];
+#pragma unroll
+            for (int i = 0; i < 2; ++i) {
+                const int item = t + 256 * i;
+                rowoff[i] = 0xFFFFFFFFu; item_w[i] = item_h[i] = item_n[i] = 0;
+                if (item < items) {
+                    const int j = item / units, u = item - j * units;
+                    item_w[i] = j % hw; item_h[i] = (j / hw) % hh; item_n[i] = j / (hw * hh);
+                    // first of the window's four rows in the tile, and the unit's place in it
+                    rowoff[i] = uint32_t(((item_n[i] * bh + 2 * item_h[i]) * bw + 2 * item_w[i]) << 7) | uint32_t(u);
+                }
+            }
+            // byte offsets, inside a k-step's dy tile, of the item's 16 bytes at the window's four positions
+            uint32_t off[2][4];
+#pragma unroll
+            for (int i = 0; i < 2; ++i)
+#pragma unroll
+                for (uint32_t e = 0; e < 4; ++e) {
+                    const uint32_t u = rowoff[i] & 127u, row = (rowoff[i] >> 7) + (e >> 1) * uint32_t(bw) + (e & 1u);
+                    off[i][e] = (u >> 3) * group_bytes + row * 128u + (((u & 7u) ^ ((row & 3u) << 1)) << 4);
+                }
+            // the loads of k-step b + 2 are issued before k-step b is written: their latency (DRAM: the pooled gradient
+            // was written by the previous kernel and is larger than L2) overlaps two whole k-steps
+            auto fetch = [&](int fqi, int fpi, int fni, float4 (&fv)[2], uint32_t (&fc)[2]) {
+#pragma unroll
+                for (int i = 0; i < 2; ++i) {
+                    fv[i] = make_float4(0.f, 0.f, 0.f, 0.f); fc[i] = 0u;
+                    if (rowoff[i] == 0xFFFFFFFFu) continue;
+                    const int qq = fqi * hw + item_w[i], pp = fpi * hh + item_h[i], n = fni * bn + item_n[i];
+                    if (qq < Q2 && pp < P2 && n < p.N) {
+                        const size_t idx = ((static_cast<size_t>(n) * P2 + pp) * Q2 + qq) * p.K + kt * 128 + (rowoff[i] & 127u) * 4;
+                        fv[i] = __ldg(reinterpret_cast<const float4*>(p.dy_pool + idx));
+                        fc[i] = __ldg(reinterpret_cast<const unsigned int*>(p.codes + idx));
+                    }
+                }
+            };
+            float4 v[2], vn[2], vnn[2];
+            uint32_t c[2], cn[2], cnn[2];
+            auto next_box = [&]() {             // the producer's walk over the pixel boxes
+                if (++qi == p.boxes_q) {
+                    qi = 0;
+                    if (++pi == p.boxes_p) { pi = 0; ++ni; }
+                }
+            };
+            if (box_begin < box_end) { fetch(qi, pi, ni, vn, cn); next_box(); }
+            if (box_begin + 1 < box_end) { fetch(qi, pi, ni, vnn, cnn); next_box(); }
+            for (int b = box_begin; b < box_end && ok; ++b) {
+#pragma unroll
+                for (int i = 0; i < 2; ++i) { v[i] = vn[i]; c[i] = cn[i]; vn[i] = vnn[i]; cn[i] = cnn[i]; }
+                if (b + 2 < box_end) { fetch(qi, pi, ni, vnn, cnn); next_box(); }
+                if (sub == 0) {
+                    if (!bounded_wait_warp(&empty_bar[stage], phase ^ 1u, &abort_flag, p.status, WAIT_PRODUCER_EMPTY)) { ok = false; break; }
+                    dstA = ring0 + stage * stage_bytes;
+                }
+#pragma unroll
+                for (int i = 0; i < 2; ++i) {
+                    if (rowoff[i] == 0xFFFFFFFFu) continue;
+                    const float vv[4] = {v[i].x, v[i].y, v[i].z, v[i].w};
+                    float live[4];
+                    uint32_t pos[4];
+#pragma unroll
+                    for (int m = 0; m < 4; ++m) {
+                        const uint32_t code = (c[i] >> (8 * m)) & 7u;
+                        pos[m] = code & 3u;
+                        live[m] = (p.relu_mask && code >= 4u) ? 0.f : vv[m];
+                    }
+                    db_acc[i].x += live[0]; db_acc[i].y += live[1]; db_acc[i].z += live[2]; db_acc[i].w += live[3];
+#pragma unroll
+                    for (int m = 0; m < 4; ++m) live[m] = to_tf32(live[m]);
+#pragma unroll
+                    for (uint32_t e = 0; e < 4; ++e)
+                        st_shared_v4(dstA + off[i][e], pos[0] == e ? live[0] : 0.f, pos[1] == e ? live[1] : 0.f,
+                                     pos[2] == e ? live[2] : 0.f, pos[3] == e ? live[3] : 0.f);
+                }
+                dstA += step_bytes;
+                if (++sub == p.KS || b == box_end - 1) {
+                    sub = 0;
+                    fence_proxy_async_shared();          // the tensor core reads the tile through the async proxy
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(&full_bar[stage]);
+                    if (++stage == p.stages) { stage = 0; phase ^= 1u; }
+                }
+            }
+        }
         if (bounded_wait_warp(&tmem_full_bar, 0, &abort_flag, p.status, WAIT_EPI_TMEM_FULL)) {
             tc_fence_after();
+            if (p.dy_pool && p.db_rows) {
+                // Bias gradient: every warp adds up, per 4-map unit and in a fixed order, what its own lanes
+                // scattered, and writes one row [K] per (split, warp); the caller adds the rows.  (Warp-local on
+                // purpose: no barrier between warps that a timed-out warp could leave the others waiting at.  The
+                // pipeline's shared memory is idle by now; the 1 KB slots lie behind the epilogue's staging tiles.)
+                float4* scratch = reinterpret_cast<float4*>(smem + 32768) + (warp - 2) * 64;
+                scratch[lane] = db_acc[0];
+                scratch[32 + lane] = db_acc[1];
+                __syncwarp();
+                if (lane < units) {
+                    float4 sum = make_float4(0.f, 0.f, 0.f, 0.f);
+                    for (int e = 0; e < 64; ++e) {
+                        const int item = (e < 32 ? 0 : 256 - 32) + (warp - 2) * 32 + e;      // lane e (e - 32) of this warp, slot 0 (1)
+                        if (item % units == lane) {
+                            const float4 a = scratch[e];
+                            sum.x += a.x; sum.y += a.y; sum.z += a.z; sum.w += a.w;
+                        }
+                    }
+                    *reinterpret_cast<float4*>(p.db_rows + (static_cast<size_t>(split) * kExpanderWarps + (warp - 2)) * p.K +
+                                               kt * 128 + lane * 4) = sum;
+                }
+                __syncwarp();
+            }
             const uint32_t t_row = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16);
             const size_t krow = static_cast<size_t>(valid ? k : 0) * p.R * p.S;
             // Each lane owns one output-map row of the accumulator, but 32 columns of a row are 128 contiguous
@@ -328,12 +473,13 @@ tc_wgrad_kernel(const __grid_constant__ CUtensorMap tmDy, const __grid_constant_
     }
 }
 
-void choose_pixel_box(int pix, int P, int Q, int N, int* bw_log2, int* bh_log2) {
+// min_l: smallest log2 of the box width and height (1 for pooled dy: the box must hold whole 2x2 windows)
+void choose_pixel_box(int pix, int P, int Q, int N, int* bw_log2, int* bh_log2, int min_l = 0) {
     const int lp = pix == 64 ? 6 : 5;
     double best = 1e300;
-    int best_w = 0, best_h = 0;
-    for (int lw = lp; lw >= 0; --lw)
-        for (int lh = lp - lw; lh >= 0; --lh) {
+    int best_w = min_l, best_h = min_l;
+    for (int lw = lp - min_l; lw >= min_l; --lw)
+        for (int lh = lp - lw; lh >= min_l; --lh) {
             const long bw = 1L << lw, bh = 1L << lh, bn = pix / (bw * bh);
             const double covered = double((Q + bw - 1) / bw * bw) * double((P + bh - 1) / bh * bh) *
                                    double((N + bn - 1) / bn * bn);
@@ -358,12 +504,12 @@ struct WgradPlan {
     long boxes;
 };
 
-WgradPlan plan_wgrad(int N, int P, int Q, int C, int K, int R, int S, int tap_groups) {
+WgradPlan plan_wgrad(int N, int P, int Q, int C, int K, int R, int S, int tap_groups, int pooled_dy = 0) {
     WgradPlan r{};
     const int cgroups = (C + 31) / 32;
     const int k_tiles = (K + 127) / 128;
     r.grouped = (!tap_groups && C % 32 == 0 && K % 32 == 0) ? 1 : 0;
-    r.pair = env_int("PCL_PAIR_WGRAD", 1) && r.grouped && k_tiles % 2 == 0;
+    r.pair = env_int("PCL_PAIR_WGRAD", 1) && r.grouped && k_tiles % 2 == 0 && !pooled_dy;
     r.L = 1;
     if (r.grouped)
         for (int l = r.pair ? 4 : 8; l >= 1; --l)        // pair: each CTA loads whole runs, half of the item's
@@ -394,7 +540,7 @@ WgradPlan plan_wgrad(int N, int P, int Q, int C, int K, int R, int S, int tap_gr
     if (r.KS < 1) r.KS = 1;
     r.stages = kSmemBudget / (r.KS * r.step_bytes);
     if (r.stages > kMaxStages) r.stages = kMaxStages;
-    choose_pixel_box(r.pix, P, Q, N, &r.bw_log2, &r.bh_log2);
+    choose_pixel_box(r.pix, P, Q, N, &r.bw_log2, &r.bh_log2, pooled_dy ? 1 : 0);
     const long bw = 1L << r.bw_log2, bh = 1L << r.bh_log2, bn = r.pix / (bw * bh);
     r.boxes = ((Q + bw - 1) / bw) * ((P + bh - 1) / bh) * ((N + bn - 1) / bn);
     return r;
@@ -421,8 +567,15 @@ bool tc_wgrad_eligible(const TcWgradArgs& a) {
     return true;
 }
 
-int tc_wgrad_splits(int N, int P, int Q, int C, int K, int R, int S, int tap_groups) {
-    const WgradPlan rp = plan_wgrad(N, P, Q, C, K, R, S, tap_groups);
+bool tc_wgrad_can_take_pooled_dy(int N, int P, int Q, int C, int K, int R, int S, int tap_groups) {
+    if (P % 2 != 0 || Q % 2 != 0 || K % 4 != 0 || N <= 0) return false;
+    const WgradPlan rp = plan_wgrad(N, P, Q, C, K, R, S, tap_groups, 1);
+    // the bias-gradient scratch (8 KB behind the epilogue's 32 KB of staging tiles) lies in the pipeline's memory
+    return !rp.pair && rp.stages * rp.KS * rp.step_bytes >= 40960;
+}
+
+int tc_wgrad_splits(int N, int P, int Q, int C, int K, int R, int S, int tap_groups, int pooled_dy) {
+    const WgradPlan rp = plan_wgrad(N, P, Q, C, K, R, S, tap_groups, pooled_dy);
     const long items = long((K + 127) / 128) * rp.run_blocks;
     long splits = sm_count() / items;
     if (splits < 1) splits = 1;
@@ -445,7 +598,12 @@ int launch_tc_wgrad(const TcWgradArgs& a, cudaStream_t st) {
         g_attr_set = true;
     }
     WgradParams p{};
-    const WgradPlan rp = plan_wgrad(a.N, a.P, a.Q, a.C, a.K, a.R, a.S, a.tap_groups);
+    const int pooled = a.dy_pool ? 1 : 0;
+    if (pooled && (!a.codes || !tc_wgrad_can_take_pooled_dy(a.N, a.P, a.Q, a.C, a.K, a.R, a.S, a.tap_groups)))
+        return PCL_ERR_UNSUPPORTED_SHAPE;
+    const WgradPlan rp = plan_wgrad(a.N, a.P, a.Q, a.C, a.K, a.R, a.S, a.tap_groups, pooled);
+    p.dy_pool = a.dy_pool; p.codes = a.codes; p.relu_mask = a.relu_mask; p.db_rows = pooled ? a.db_rows : nullptr;
+    p.N = a.N; p.P = a.P; p.Q = a.Q;
     p.pix = rp.pix; p.bw_log2 = rp.bw_log2; p.bh_log2 = rp.bh_log2;
     const int bw = 1 << p.bw_log2, bh = 1 << p.bh_log2, bn = p.pix / (bw * bh);
     p.boxes_q = (a.Q + bw - 1) / bw;
@@ -483,7 +641,7 @@ int launch_tc_wgrad(const TcWgradArgs& a, cudaStream_t st) {
     // group dimension has a 128-byte stride) so that one TMA instruction brings a whole run of groups, laid
     // out [group][pixel][32 maps] in shared memory exactly as per-group boxes would be.
     CUtensorMap tmDy, tmX;
-    {
+    if (!pooled) {
         const uint64_t sw = uint64_t(a.K), sh = uint64_t(a.Q) * a.K, sn = uint64_t(a.P) * a.Q * a.K;
         if (p.grouped_dy) {
             const uint64_t dims[5] = {32, uint64_t(a.Q), uint64_t(a.P), uint64_t(a.N), uint64_t(a.K / 32)};
@@ -528,6 +686,7 @@ int launch_tc_wgrad(const TcWgradArgs& a, cudaStream_t st) {
             if (rc != PCL_OK) return rc;
         }
     }
+    if (pooled) tmDy = tmX;      // (a valid map is passed in any case; the kernel does not use it)
     const long items = long(p.k_tiles) * p.run_blocks * p.splits;
     if (items > 0x7fffffffL) return PCL_ERR_UNSUPPORTED_SHAPE;
     const size_t smem = size_t(p.stages) * stage_bytes + 1024;

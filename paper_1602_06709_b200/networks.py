@@ -176,7 +176,12 @@ class VggA(_HostFeed):
         self.y = [None if (L.pool and not keep_unpooled and B.conv_fwd_pool_is_fused(L.desc))
                   else torch.empty(N, L.H, L.W, L.K, device=dev) for L in self.convs]       # post-ReLU
         self.pooled = [torch.empty(N, L.H // 2, L.W // 2, L.K, device=dev) if L.pool else None for L in self.convs]
-        self.dy = [torch.empty(N, L.H, L.W, L.K, device=dev) for L in self.convs]           # grad wrt pre-activation
+        # The first layer has no backward-data pass; where it is pooled and the library can take its weight gradient
+        # straight from the pooled gradient and the position codes, its full-resolution dy is never formed either.
+        self.first_from_pooled = bool(self.convs[0].pool and not keep_unpooled and
+                                      B.conv_bwd_weights_pooled_is_fused(self.convs[0].desc))
+        self.dy = [None if (i == 0 and self.first_from_pooled) else torch.empty(N, L.H, L.W, L.K, device=dev)
+                   for i, L in enumerate(self.convs)]                                          # grad wrt pre-activation
         self.dpooled = [torch.empty(N, L.H // 2, L.W // 2, L.K, device=dev) if L.pool else None for L in self.convs]
         # position codes of the pooling windows (one byte per pooled element), written by the forward epilogue
         self.pool_codes = [torch.empty(N, L.H // 2, L.W // 2, L.K, dtype=torch.uint8, device=dev) if L.pool else None
@@ -187,6 +192,8 @@ class VggA(_HostFeed):
         self._feed_init()
         self.loss = torch.zeros(1, device=dev)
         ws = 0
+        if self.first_from_pooled:
+            ws = B.conv_bwd_weights_pooled_workspace_bytes(self.convs[0].desc)
         for L in self.convs:
             ws = max(ws, B.conv_workspace_bytes(L.desc, B.PASS_FWD), B.conv_workspace_bytes(L.desc, B.PASS_BWD_DATA),
                      B.conv_workspace_bytes(L.desc, B.PASS_BWD_WEIGHTS), B.conv_bwd_data_colsum_workspace_bytes(L.desc),
@@ -241,6 +248,11 @@ class VggA(_HostFeed):
             L = self.convs[i]
             # The bias gradient of layer i is the per-map sum of dy[i]; it is formed by whichever kernel writes
             # dy[i] (the pool backward here, or the backward-data pass of layer i+1 below), not by a separate pass.
+            if i == 0 and self.first_from_pooled:
+                # pooling backward, ReLU mask, bias gradient and weight gradient in one pass over the pooled gradient
+                B.conv_bwd_weights_pooled(L.desc, self.layer_input(0), self.dpooled[0], self.pool_codes[0], True,
+                                          self.conv_dw(0), self.conv_db(0), self.ws)
+                continue
             if L.pool:   # gradient through the pool, then through the ReLU (fused mask), routed by the position codes
                 B.maxpool2x2_bwd_codes(self.N, L.H, L.W, L.K, self.pool_codes[i], self.dpooled[i], True, self.dy[i],
                                        self.conv_db(i), self.ws)

@@ -190,6 +190,20 @@ def verify_vgg_step(net, params_before, samples=0, seed=0):
     for i in reversed(range(nconv)):
         L = net.convs[i]
         s = ConvShape(N=N, C=L.C, K=L.K, H=L.H, W=L.W, R=3, S=3, pad_h=1, pad_w=1)
+        if net.dy[i] is None:
+            # first layer, weight gradient taken straight from the pooled gradient: the reference dy is the oracle's
+            # code-routed pooling backward pass (image by image, to bound the host memory of the full-size run)
+            codes_h, dp_h = host(net.pool_codes[i]), host(net.dpooled[i])
+            dz = np.empty((N, L.H, L.W, L.K), np.float32)
+            for n in range(N):
+                dz[n] = oracle.maxpool2x2_bwd_codes(codes_h[n:n + 1], dp_h[n:n + 1], True)[0]
+            xin = host(net.layer_input(i))
+            _cmp(net.conv_dw(i), lambda at: oracle.conv_bwd_weights(s, xin, dz, at=at), net.conv_dw(i).numel(), samples,
+                 rng, f"{L.name} dw (from pooled dy)", report)
+            db_ref = dz.reshape(-1, L.K).astype(np.float64).sum(axis=0)
+            rel, mx = oracle.parity_errors(host(net.conv_db(i)), db_ref)
+            assert rel <= REL_L2_TOL and mx <= MAX_OVER_RMS_TOL, f"{L.name} db (from pooled dy)"
+            continue
         if L.pool and net.y[i] is None:      # routed by the position codes the forward call recorded, bit for bit
             nchk = N if not samples else min(N, 2)
             ref = oracle.maxpool2x2_bwd_codes(host(net.pool_codes[i][:nchk]), host(net.dpooled[i][:nchk]), True)

@@ -3,6 +3,7 @@ oracle, element by element, on seeded inputs.  Shapes span several tiles and
 ragged tails in every tiled dimension; both kernel families are exercised."""
 import numpy as np
 import pytest
+import torch
 
 import oracle
 from oracle import ConvShape
@@ -270,3 +271,64 @@ def test_two_issuer_backward_data_repeats_bit_for_bit(path_guard):
             G.assert_parity(dx.cpu().numpy(), oracle.conv_bwd_data(s, dy, w, x), "bwd_data")
         else:
             assert torch.equal(first, dx)
+
+
+POOLED_WGRAD_SHAPES = {
+    # few-channel first layers with even outputs: ragged boxes in q and p, several images per box, R != S, K > 128
+    "rgb": ConvShape(N=2, C=3, K=16, H=20, W=36, R=3, S=3, pad_h=1, pad_w=1),
+    "rgb_k64": ConvShape(N=3, C=3, K=64, H=40, W=36, R=3, S=3, pad_h=1, pad_w=1),
+    "gray_5x5": ConvShape(N=2, C=1, K=24, H=18, W=20, R=5, S=5, pad_h=2, pad_w=2),
+    "two_ch_nopad": ConvShape(N=5, C=2, K=36, H=12, W=15, R=3, S=2),
+    "rgb_k160": ConvShape(N=2, C=3, K=160, H=8, W=8, R=3, S=3, pad_h=1, pad_w=1),
+    "tiny_maps": ConvShape(N=9, C=3, K=8, H=4, W=6, R=3, S=3, pad_h=1, pad_w=1),
+}
+
+
+@pytest.mark.parametrize("relu", [True, False])
+@pytest.mark.parametrize("tag", sorted(POOLED_WGRAD_SHAPES))
+def test_weight_gradient_from_pooled_gradient(tag, relu, path_guard):
+    """pcl_conv_bwd_weights_pooled: the weight gradient of a pooled first layer straight from the pooled gradient and
+    the windows' position codes (the kernel builds its dy tiles on chip).  Reference: the oracle's code-routed
+    pooling backward pass followed by the oracle's weight gradient."""
+    import gpu_helpers as G
+    from paper_1602_06709_b200 import binding as B
+    from paper_1602_06709_b200 import inputs
+    s = POOLED_WGRAD_SHAPES[tag]
+    d = G.shape_to_desc(s)
+    assert B.conv_bwd_weights_pooled_is_fused(d)
+    x, _, _, _ = G.make_inputs(s, "pooled_" + tag)
+    P2, Q2 = s.P // 2, s.Q // 2
+    dyp = inputs.normal(inputs.tensor_id("pooled_wgrad", tag, "dyp"), (s.N, P2, Q2, s.K), 1.0)
+    codes = (inputs.uniform(inputs.tensor_id("pooled_wgrad", tag, "codes"), (s.N, P2, Q2, s.K), 0.0, 8.0)
+             .astype(np.int64).clip(0, 7).astype(np.uint8))
+    dy = oracle.maxpool2x2_bwd_codes(codes, dyp, relu).astype(np.float32)
+    dw_ref, db_ref = oracle.conv_bwd_weights(s, x, dy, want_db=True)
+    ws = G.workspace(B.conv_bwd_weights_pooled_workspace_bytes(d))
+    outs = []
+    for _ in range(2):
+        dw = torch.full((s.K, s.R, s.S, s.C), float("nan"), device="cuda")
+        db = torch.full((s.K,), float("nan"), device="cuda")
+        B.conv_bwd_weights_pooled(d, G.dev(x), G.dev(dyp), torch.from_numpy(codes).cuda(), relu, dw, db, ws)
+        B.check_device_status()
+        outs.append((dw.cpu().numpy(), db.cpu().numpy()))
+    G.assert_parity(outs[0][0], dw_ref, "dw from pooled dy")
+    G.assert_parity(outs[0][1], db_ref, "db from pooled dy")
+    assert np.array_equal(outs[0][0], outs[1][0]) and np.array_equal(outs[0][1], outs[1][1])
+    # without the bias gradient
+    dw2 = torch.full((s.K, s.R, s.S, s.C), float("nan"), device="cuda")
+    B.conv_bwd_weights_pooled(d, G.dev(x), G.dev(dyp), torch.from_numpy(codes).cuda(), relu, dw2, None, ws)
+    B.check_device_status()
+    assert np.array_equal(dw2.cpu().numpy(), outs[0][0])
+
+
+def test_weight_gradient_from_pooled_gradient_only_where_fused():
+    import gpu_helpers as G
+    from paper_1602_06709_b200 import binding as B
+    s = ConvShape(N=2, C=32, K=32, H=8, W=8, R=3, S=3, pad_h=1, pad_w=1)       # not a few-channel layer
+    d = G.shape_to_desc(s)
+    assert not B.conv_bwd_weights_pooled_is_fused(d)
+    z = lambda *shape: torch.zeros(*shape, device="cuda")
+    with pytest.raises(B.PclError) as e:
+        B.conv_bwd_weights_pooled(d, z(2, 8, 8, 32), z(2, 4, 4, 32), torch.zeros(2, 4, 4, 32, dtype=torch.uint8, device="cuda"),
+                                  True, z(32, 3, 3, 32), None, G.workspace(1 << 20))
+    assert e.value.code == B.ERR_UNSUPPORTED_SHAPE
