@@ -379,7 +379,7 @@ tc_wgrad_kernel(const __grid_constant__ CUtensorMap tmDy, const __grid_constant_
         }
         if (bounded_wait_warp(&tmem_full_bar, 0, &abort_flag, p.status, WAIT_EPI_TMEM_FULL)) {
             tc_fence_after();
-            if (p.dy_pool && p.db_rows) {
+            if (p.dy_pool && p.db_rows && rb == 0) {        // (every run block would report the same sums)
                 // Bias gradient: every warp adds up, per 4-map unit and in a fixed order, what its own lanes
                 // scattered, and writes one row [K] per (split, warp); the caller adds the rows.  (Warp-local on
                 // purpose: no barrier between warps that a timed-out warp could leave the others waiting at.  The
