@@ -45,7 +45,7 @@ FALLBACK_HBM_GBS = 6650.0
 # full minibatch: weight bytes once, activation bytes x 8); source: profiles/vgga_step_n256_launch_list.md and
 # profiles/tc_fprop_tc_wgrad_conv256_56x56_n32.md
 NCU_DRAM_BYTES_PER_LAUNCH = {
-    "vgga": {"tc_fprop_kernel": 531.4e6, "tc_wgrad_kernel": 1181.3e6},
+    "vgga": {"tc_fprop_kernel": 531.4e6, "tc_wgrad_kernel": 930.7e6},
     "conv": {"tc_fprop_kernel": (163.8e6 + 283.9e6) / 2 * 8, "tc_wgrad_kernel": 209.9e6 * 8},
 }
 
