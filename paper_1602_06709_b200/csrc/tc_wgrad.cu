@@ -24,6 +24,14 @@
 // workspace (second pass adds the splits in a fixed order) or adds it to dw with
 // fp32 atomics.
 //
+// Haloed x ("xhalo", single-CTA items of stride-1 layers with S > 1 and few input maps): the S taps of one kernel
+// row read pixel boxes that overlap in all but S-1 columns, so ONE box of (bw + S - 1) x bh x bn pixels per 32-map
+// group is fetched per k-step and every tap is a view of it shifted by one 128-byte row: an MMA takes the S taps of
+// one map group as S consecutive 32-column groups 128 bytes apart (the descriptor's leading-dimension offset),
+// i.e. N = 32*S columns, one MMA per map group and 8 pixels.  A work item is then (k tile, kernel row, pixel
+// split).  For C = 64, 3x3 this cuts the bytes fetched per 64 pixels from 80 to 50 KB; such layers sit at the
+// L2-to-SM ceiling, not at the tensor pipe's.
+//
 // Pooled dy ("dy_pool" launches, for a layer whose output went through a 2x2 max pool and that has no
 // backward-data pass of its own, i.e. the first layer): dy is never materialised.  The eight epilogue warps, idle
 // during the main loop, build each k-step's dy tile in shared memory themselves from the pooled gradient and the
@@ -37,6 +45,8 @@
 // same run block and pixel split: each loads its own dy tile and half of the x
 // runs, and the even CTA issues M = 256 MMAs for both (cta_group::2).
 #include <stdlib.h>
+
+#include <type_traits>
 
 #include "pcl_internal.h"
 #include "pcl_ptx.cuh"
@@ -69,6 +79,10 @@ struct WgradParams {
     int grouped;              // x: 5-D tensor map (one TMA instruction per run) or 4-D per-group boxes (L == 1)
     int grouped_dy;           // dy: 5-D tensor map (all four 32-map groups in one instruction)
     int x_taprows;            // x: 5-D map whose 5th dimension is the tap row (few-channel path): one instruction per k-step
+    int xhalo;                // haloed x boxes: item = (k tile, kernel row, split), one x copy per k-step (see the header)
+    int cg;                   // xhalo: 32-map groups of x (C / 32)
+    int x_group_bytes;        // xhalo: bytes of one group's haloed box, (bw + S - 1) * bh * bn * 128
+    int x_step_bytes;         // xhalo: bytes of a k-step (dy tile + cg haloed boxes, rounded up to 1 KB)
     // pooled dy (see the header): dy_pool [N][P/2][Q/2][K], codes the same shape in bytes (bits 0-1 position in the
     // window, bit 2 "maximum <= 0"); relu_mask: windows with bit 2 set contribute nothing; db_rows [splits * 8][K]
     const float* dy_pool;
@@ -80,6 +94,19 @@ struct WgradParams {
     size_t split_stride;      // K*R*S*C (0 when writing straight to dw)
     unsigned int* status;     // device status word
 };
+
+// One box row of a haloed-x k-step: kSteps MMA steps of 8 pixels, each one MMA per map group (kCg of them) over the
+// S taps.  Straight-line: every instruction of the lone issuing thread costs cycles of the k-step budget.
+template <int kSteps, int kCg>
+__device__ __forceinline__ void xhalo_row(uint32_t d_tmem, uint32_t xn, uint32_t a_lo, uint32_t b_lo, uint32_t hi,
+                                          uint32_t idesc, uint32_t acc_first, uint32_t xg16) {
+#pragma unroll
+    for (int m = 0; m < kSteps; ++m)
+#pragma unroll
+        for (int g = 0; g < kCg; ++g)
+            umma_tf32(d_tmem + g * xn, (uint64_t(hi) << 32) | (a_lo + 64u * m), (uint64_t(hi) << 32) | (b_lo + 64u * m + g * xg16),
+                      idesc, m == 0 ? acc_first : 1u);
+}
 
 // kPair: see the header.  Pair mode needs grouped x and dy maps; every item then has rpi runs (runs past the
 // last tap read zeros through the out-of-bounds fill and are not stored).
@@ -105,14 +132,15 @@ tc_wgrad_kernel(const __grid_constant__ CUtensorMap tmDy, const __grid_constant_
     const int kt = kPair ? 2 * (item / p.run_blocks) + int(pair_rank) : item / p.run_blocks;
     const int run0 = rb * p.rpi;
     const int nruns = kPair ? p.rpi : ((run0 + p.rpi <= p.total_runs) ? p.rpi : p.total_runs - run0);
-    const int n_groups = nruns * p.L;                 // 32-column groups of this item's MMA
+    const int n_groups = p.xhalo ? p.cg * p.S : nruns * p.L;      // 32-column groups of this item's accumulator
     const int my_runs = kPair ? nruns >> 1 : nruns;   // runs this CTA loads (pair: its half of the columns)
     const int my_run0 = run0 + int(pair_rank) * my_runs;
     const uint32_t group_bytes = p.pix * 128;         // one {32 maps x pix pixels} box
     const uint32_t a_bytes = 4 * group_bytes;         // 128 output maps
-    const uint32_t step_bytes = a_bytes + (kPair ? (p.rpi >> 1) : p.rpi) * p.L * group_bytes;   // one k-step (same for every item)
+    const uint32_t step_bytes = p.xhalo ? uint32_t(p.x_step_bytes)
+                                        : a_bytes + (kPair ? (p.rpi >> 1) : p.rpi) * p.L * group_bytes;   // one k-step (same for every item)
     const uint32_t stage_bytes = p.KS * step_bytes;                     // a slot holds KS k-steps
-    const uint32_t tx_bytes = (p.dy_pool ? 0u : a_bytes) + my_runs * p.L * group_bytes;   // (pooled dy: written by the epilogue warps)
+    const uint32_t tx_bytes = (p.dy_pool ? 0u : a_bytes) + (p.xhalo ? uint32_t(p.cg) * p.x_group_bytes : my_runs * p.L * group_bytes);   // (pooled dy: written by the epilogue warps)
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < p.stages; ++s) {
@@ -195,7 +223,10 @@ tc_wgrad_kernel(const __grid_constant__ CUtensorMap tmDy, const __grid_constant_
                         tma_load_4d_addr<kPair>(dst + g * group_bytes, &tmDy, full_dst, kt * 128 + g * 32, q0, p0, n0);
                 }
                 const uint32_t xdst = dst + a_bytes;
-                if (p.x_taprows) {
+                if (p.xhalo) {
+                    // all map groups of the haloed box of kernel row `rb` (columns q0 - pad_w .. q0 + bw + S - 2 - pad_w)
+                    tma_load_5d_addr<kPair>(xdst, &tmX, full_dst, 0, q0 - p.pad_w, p0 + rb - p.pad_h, n0, 0);
+                } else if (p.x_taprows) {
                     tma_load_5d_addr<kPair>(xdst, &tmX, full_dst, 0, q0 + run_dw[0], p0 + run_dh[0], n0, 0);
                 } else if (p.grouped) {
 #pragma unroll
@@ -248,9 +279,52 @@ tc_wgrad_kernel(const __grid_constant__ CUtensorMap tmDy, const __grid_constant_
         uint32_t full_a = full0, empty_a = empty0, slot_lo = ring_lo0;
         const uint32_t stage16 = stage_bytes >> 4, step16 = step_bytes >> 4, a16 = a_bytes >> 4;
         const bool wide = p.pix == 64;
+        // xhalo: N = 32*S per MMA, B's leading-dimension offset one 128-byte row (8 sixteen-byte units, bits 16-29 of
+        // the low word) = one tap; a box row of bw pixels is bw/8 MMA steps per map group, the next box row starts
+        // bw + S - 1 rows further in the haloed box
+        const uint32_t idesc_x = make_idesc_tf32(p.S * 32, true, true, 128u);
+        const uint32_t xn = p.S * 32, xg16 = uint32_t(p.x_group_bytes) >> 4;
+        const uint32_t xlbo = (8u << 16) - (ring_lo0 & 0x3FFF0000u);      // replaces dy's offset field by 8
+        const int xrows = p.pix >> p.bw_log2, xsteps = bw >> 3;
+        const uint32_t xrow16 = uint32_t(bw + p.S - 1) * 8u;
         int stage = 0;
         uint32_t phase = 0, accum = 0;
         bool ok = true;
+        // haloed x: one k-step per slot (KS = 1); the whole k-step is straight-line for the common box shapes
+        auto xhalo_loop = [&](auto rows_c, auto steps_c, auto cg_c) {
+            constexpr int kRows = decltype(rows_c)::value, kSteps = decltype(steps_c)::value, kCg = decltype(cg_c)::value;
+            const int rows = kRows ? kRows : xrows, steps = kSteps ? kSteps : xsteps, cgs = kCg ? kCg : p.cg;
+            for (int kit = 0; kit < kiters; ++kit) {
+                if (!bounded_wait_addr(full_a, phase, &abort_flag, p.status, WAIT_MMA_FULL)) { ok = false; break; }
+                tc_fence_after();
+                uint32_t ar = slot_lo, br = slot_lo + a16 + xlbo;
+                if constexpr (kRows != 0) {
+#pragma unroll
+                    for (int r = 0; r < kRows; ++r, ar += 64u * kSteps, br += xrow16)
+                        xhalo_row<kSteps, kCg>(tmem_base, xn, ar, br, hi, idesc_x, r == 0 ? accum : 1u, xg16);
+                } else {
+                    for (int r = 0; r < rows; ++r, ar += 64u * steps, br += xrow16)
+                        for (int m = 0; m < steps; ++m)
+                            for (int g = 0; g < cgs; ++g)
+                                umma_tf32(tmem_base + g * xn, (uint64_t(hi) << 32) | (ar + 64u * m),
+                                          (uint64_t(hi) << 32) | (br + 64u * m + g * xg16), idesc_x, (accum | r | m) ? 1u : 0u);
+                }
+                accum = 1;
+                umma_commit_addr<kPair>(empty_a);
+                full_a += 8; empty_a += 8; slot_lo += stage16;
+                if (++stage == p.stages) { stage = 0; phase ^= 1u; full_a = full0; empty_a = empty0; slot_lo = ring_lo0; }
+            }
+        };
+        using std::integral_constant;
+        if (p.xhalo) {
+            const int key = xrows * 100 + xsteps * 10 + p.cg;
+            if (key == 422) xhalo_loop(integral_constant<int, 4>{}, integral_constant<int, 2>{}, integral_constant<int, 2>{});
+            else if (key == 812) xhalo_loop(integral_constant<int, 8>{}, integral_constant<int, 1>{}, integral_constant<int, 2>{});
+            else if (key == 242) xhalo_loop(integral_constant<int, 2>{}, integral_constant<int, 4>{}, integral_constant<int, 2>{});
+            else if (key == 421) xhalo_loop(integral_constant<int, 4>{}, integral_constant<int, 2>{}, integral_constant<int, 1>{});
+            else if (key == 222) xhalo_loop(integral_constant<int, 2>{}, integral_constant<int, 2>{}, integral_constant<int, 2>{});
+            else xhalo_loop(integral_constant<int, 0>{}, integral_constant<int, 0>{}, integral_constant<int, 0>{});
+        } else
         for (int kit = 0; kit < kiters; kit += p.KS) {
             if (!bounded_wait_addr(full_a, phase, &abort_flag, p.status, WAIT_MMA_FULL)) { ok = false; break; }
             tc_fence_after();
@@ -411,10 +485,16 @@ tc_wgrad_kernel(const __grid_constant__ CUtensorMap tmDy, const __grid_constant_
             const uint32_t stg = smem_u32(smem) + (warp - 2) * 4096;
             const int cg = (lane & 7) * 4;
             for (int ch = (warp - 2) >> 2; ch < n_groups; ch += 2) {     // the quarter's two warps take alternate chunks
-                const int run = run0 + ch / p.L;
-                if (run >= p.total_runs) break;         // (pair mode) columns of runs past the last tap
-                const int tap = run / p.runs_per_tap;
-                const int c0 = ((run - tap * p.runs_per_tap) * p.L + ch % p.L) * 32;
+                int tap, c0;
+                if (p.xhalo) {                          // columns: [map group][tap of kernel row rb]
+                    tap = rb * p.S + ch % p.S;
+                    c0 = (ch / p.S) * 32;
+                } else {
+                    const int run = run0 + ch / p.L;
+                    if (run >= p.total_runs) break;     // (pair mode) columns of runs past the last tap
+                    tap = run / p.runs_per_tap;
+                    c0 = ((run - tap * p.runs_per_tap) * p.L + ch % p.L) * 32;
+                }
                 uint32_t v[32];
                 if (kiters > 0) {
                     tmem_ld_32x32(t_row + ch * 32, v);
@@ -474,11 +554,13 @@ tc_wgrad_kernel(const __grid_constant__ CUtensorMap tmDy, const __grid_constant_
 }
 
 // min_l: smallest log2 of the box width and height (1 for pooled dy: the box must hold whole 2x2 windows)
-void choose_pixel_box(int pix, int P, int Q, int N, int* bw_log2, int* bh_log2, int min_l = 0) {
+// min_lw: smallest log2 of the box width alone (3 for haloed x: a box row must hold whole 8-pixel MMA steps)
+void choose_pixel_box(int pix, int P, int Q, int N, int* bw_log2, int* bh_log2, int min_l = 0, int min_lw = 0) {
     const int lp = pix == 64 ? 6 : 5;
     double best = 1e300;
-    int best_w = min_l, best_h = min_l;
-    for (int lw = lp - min_l; lw >= min_l; --lw)
+    if (min_lw < min_l) min_lw = min_l;
+    int best_w = min_lw, best_h = min_l;
+    for (int lw = lp - min_l; lw >= min_lw; --lw)
         for (int lh = lp - lw; lh >= min_l; --lh) {
             const long bw = 1L << lw, bh = 1L << lh, bn = pix / (bw * bh);
             const double covered = double((Q + bw - 1) / bw * bw) * double((P + bh - 1) / bh * bh) *
@@ -502,6 +584,7 @@ struct WgradPlan {
     int KS, stages, step_bytes;
     int bw_log2, bh_log2;
     long boxes;
+    int xhalo, x_group_bytes;     // haloed x boxes (see the header): item = (k tile, kernel row, split)
 };
 
 WgradPlan plan_wgrad(int N, int P, int Q, int C, int K, int R, int S, int tap_groups, int pooled_dy = 0) {
@@ -525,6 +608,26 @@ WgradPlan plan_wgrad(int N, int P, int Q, int C, int K, int R, int S, int tap_gr
         if (r.pair && (r.rpi & 1)) ++r.rpi;             // (8 / L is even for L = 1..4, so this stays <= rpi_max)
     }
     r.run_blocks = (r.total_runs + r.rpi - 1) / r.rpi;
+    // Haloed x boxes for single-CTA items of layers with few input maps (all taps of a kernel row fit one
+    // accumulator): the pixel box must hold whole 8-pixel runs in w.
+    if (r.grouped && !r.pair && !pooled_dy && S >= 2 && cgroups * S * 32 <= 256 && Q >= 8 && env_int("PCL_XHALO_WGRAD", 1)) {
+        for (int pix = env_int("PCL_PIX_WGRAD", 64) == 64 ? 64 : 32; pix >= 32 && !r.xhalo; pix >>= 1) {
+            int lw, lh;
+            choose_pixel_box(pix, P, Q, N, &lw, &lh, 0, 3);
+            const long bw = 1L << lw, bh = 1L << lh, bn = pix / (bw * bh);
+            const int xg = int((bw + S - 1) * bh * bn * 128);
+            const int step = (4 * pix * 128 + cgroups * xg + 1023) / 1024 * 1024;
+            if (kSmemBudget / step < 3) continue;
+            r.xhalo = 1; r.x_group_bytes = xg; r.pix = pix; r.step_bytes = step;
+            r.bw_log2 = lw; r.bh_log2 = lh;
+            r.run_blocks = R;
+            r.KS = 1;
+            r.stages = kSmemBudget / step;
+            if (r.stages > kMaxStages) r.stages = kMaxStages;
+            r.boxes = ((Q + bw - 1) / bw) * ((P + bh - 1) / bh) * ((N + bn - 1) / bn);
+        }
+        if (r.xhalo) return r;
+    }
     // 64-pixel k-steps halve the copies and commits per MMA; taken when three pipeline slots still fit
     const int cta_groups = 4 + (r.pair ? r.rpi / 2 : r.rpi) * r.L;      // 32-map groups a CTA loads per k-step
     r.pix = env_int("PCL_PIX_WGRAD", 64);
@@ -611,6 +714,7 @@ int launch_tc_wgrad(const TcWgradArgs& a, cudaStream_t st) {
     p.boxes_n = (a.N + bn - 1) / bn;
     const long boxes = rp.boxes;
     if (boxes > 0x7fffffffL) return PCL_ERR_UNSUPPORTED_SHAPE;
+    p.xhalo = rp.xhalo; p.cg = (a.C + 31) / 32; p.x_group_bytes = rp.x_group_bytes; p.x_step_bytes = rp.step_bytes;
     p.grouped = rp.grouped; p.grouped_dy = (a.K % 32 == 0) ? 1 : 0; p.x_taprows = a.tap_groups ? 1 : 0; p.L = rp.L; p.runs_per_tap = rp.runs_per_tap; p.total_runs = rp.total_runs;
     p.rpi = rp.rpi; p.run_blocks = rp.run_blocks;
     p.k_tiles = (a.K + 127) / 128;
@@ -619,7 +723,7 @@ int launch_tc_wgrad(const TcWgradArgs& a, cudaStream_t st) {
     p.splits = a.splits;
     if (p.splits < 1) return PCL_ERR_BAD_ARG;
     p.boxes_per_split = int((boxes + p.splits - 1) / p.splits);
-    const int max_groups = p.rpi * p.L;
+    const int max_groups = p.xhalo ? p.cg * a.S : p.rpi * p.L;
     p.KS = rp.KS; p.stages = rp.stages;
     const int stage_bytes = p.KS * rp.step_bytes;
     p.tmem_cols = 32;
@@ -661,7 +765,14 @@ int launch_tc_wgrad(const TcWgradArgs& a, cudaStream_t st) {
         const uint64_t sw = a.x_stride_w ? uint64_t(a.x_stride_w) : uint64_t(a.C);
         const uint64_t sh = a.x_stride_h ? uint64_t(a.x_stride_h) : uint64_t(a.W) * a.C;
         const uint64_t sn = a.x_stride_n ? uint64_t(a.x_stride_n) : uint64_t(a.H) * a.W * a.C;
-        if (p.x_taprows) {
+        if (p.xhalo) {
+            // haloed box: S - 1 more columns than the dy box, all map groups with one instruction
+            const uint64_t dims[5] = {32, uint64_t(a.W), uint64_t(a.H), uint64_t(a.N), uint64_t(a.C / 32)};
+            const uint64_t strides[4] = {sw * 4, sh * 4, sn * 4, 128};
+            const uint32_t box[5] = {32, uint32_t(bw + a.S - 1), uint32_t(bh), uint32_t(bn), uint32_t(p.cg)};
+            int rc = make_tmap(&tmX, a.x, 5, dims, strides, box, true);
+            if (rc != PCL_OK) return rc;
+        } else if (p.x_taprows) {
             // few-channel path: the R tap rows of a pixel window are R boxes one image row apart; a 5th
             // dimension with the row stride fetches them with one instruction (H extent shrinks by R-1 so
             // that row + tap stays inside the staged image)

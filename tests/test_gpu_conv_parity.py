@@ -194,6 +194,43 @@ def test_forward_with_sixteen_epilogue_warps(tag, tiling, path_guard, monkeypatc
     assert B.last_device_status() == 0
 
 
+XHALO_SHAPES = {
+    # single-CTA weight-gradient items (odd number of 128-map tiles), few input maps, S > 1
+    "c64_k128": ConvShape(N=3, C=64, K=128, H=28, W=28, R=3, S=3, pad_h=1, pad_w=1),
+    "ragged_q": ConvShape(N=2, C=64, K=96, H=13, W=21, R=3, S=3, pad_h=1, pad_w=1),
+    "c32_5x5_nopad": ConvShape(N=2, C=32, K=64, H=20, W=24, R=5, S=5),
+    "rect_pad2": ConvShape(N=5, C=32, K=40, H=9, W=16, R=2, S=3, pad_h=0, pad_w=2),
+    "three_k_tiles": ConvShape(N=2, C=64, K=320, H=16, W=16, R=3, S=3, pad_h=1, pad_w=1),
+    "row_kernel": ConvShape(N=4, C=64, K=128, H=10, W=40, R=1, S=3, pad_h=0, pad_w=1),
+    "wide_box": ConvShape(N=2, C=64, K=64, H=6, W=64, R=3, S=3, pad_h=1, pad_w=1),
+}
+
+
+@pytest.mark.parametrize("pix", ["64", "32"])
+@pytest.mark.parametrize("tag", sorted(XHALO_SHAPES))
+def test_weight_gradient_with_haloed_input_boxes(tag, pix, path_guard, monkeypatch):
+    """Layers with few input maps fetch one haloed input box per k-step and take the S taps of a kernel row as
+    row-shifted views of it (one MMA over 32*S columns); PCL_XHALO_WGRAD=0 keeps one box per tap.  Both must agree
+    with the oracle; the two-pass result must repeat bit for bit."""
+    import gpu_helpers as G
+    from paper_1602_06709_b200 import binding as B
+    B.set_path(B.PATH_TENSOR)
+    monkeypatch.setenv("PCL_PIX_WGRAD", pix)
+    s = XHALO_SHAPES[tag]
+    x, w, dy, _ = G.make_inputs(s, "xhalo_" + tag)
+    dw_ref, db_ref = oracle.conv_bwd_weights(s, x, dy, want_db=True)
+    for mode in ("1", "0"):
+        monkeypatch.setenv("PCL_XHALO_WGRAD", mode)
+        dw, db = G.run_conv_bwd_weights(s, x, dy, True, deterministic=True)
+        G.assert_parity(dw, dw_ref, f"bwd_weights xhalo={mode}")
+        G.assert_parity(db, db_ref, "dbias")
+        dw2, _ = G.run_conv_bwd_weights(s, x, dy, False, deterministic=True)
+        assert np.array_equal(dw, dw2)
+        dw3, _ = G.run_conv_bwd_weights(s, x, dy, False, deterministic=False)
+        G.assert_parity(dw3, dw_ref, f"bwd_weights atomics xhalo={mode}")
+    assert B.last_device_status() == 0
+
+
 @pytest.mark.parametrize("tiling", ["plain", "halo1", "auto"])
 @pytest.mark.parametrize("tag", ["odd_groups", "even_groups_wide", "fc_like"])
 def test_backward_data_reads_weights_in_place(tag, tiling, path_guard, monkeypatch):
