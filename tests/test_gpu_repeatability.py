@@ -69,3 +69,28 @@ def test_forward_with_pool_repeats_bit_for_bit(name, N, C, K, H):
         else:
             assert torch.equal(ref[0], yp) and torch.equal(ref[1], codes)
     assert int(ref[1].max()) <= 7 and not torch.isnan(ref[0]).any()
+
+
+def test_first_layer_weight_gradient_from_pooled_gradient_repeats_bit_for_bit():
+    """The weight-gradient kernel whose epilogue warps build the dy tiles in shared memory (generic-proxy stores handed
+    to the tensor core through fence.proxy.async and the slot's barrier): identical results over repeated launches."""
+    from paper_1602_06709_b200 import binding as B
+    N, C, K, H = 32, 3, 64, 224
+    d = B.conv_desc(N, C, K, H, H, 3, 3, 1, 1)
+    assert B.conv_bwd_weights_pooled_is_fused(d)
+    g = torch.Generator(device="cuda").manual_seed(16)
+    x = torch.rand(N, H, H, C, device="cuda", generator=g)
+    dyp = torch.randn(N, H // 2, H // 2, K, device="cuda", generator=g) * 1e-2
+    codes = torch.randint(0, 8, (N, H // 2, H // 2, K), dtype=torch.uint8, device="cuda", generator=g)
+    ws = torch.empty(max(256, B.conv_bwd_weights_pooled_workspace_bytes(d)), dtype=torch.uint8, device="cuda")
+    ref = None
+    for _ in range(10):
+        dw = torch.full((K, 3, 3, C), float("nan"), device="cuda")
+        db = torch.full((K,), float("nan"), device="cuda")
+        B.conv_bwd_weights_pooled(d, x, dyp, codes, True, dw, db, ws)
+        B.check_device_status()
+        if ref is None:
+            ref = (dw, db)
+        else:
+            assert torch.equal(ref[0], dw) and torch.equal(ref[1], db)
+    assert not torch.isnan(ref[0]).any() and not torch.isnan(ref[1]).any()
