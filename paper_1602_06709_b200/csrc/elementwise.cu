@@ -381,21 +381,31 @@ __global__ void __launch_bounds__(256) softmax_xent_kernel(const float* __restri
     }
 }
 
-// xs[n][hh][ww][0..3]: channel-padded copy of x with a zero halo of (pad_h, pad_w)
+// xs[n][hh][ww][0..3]: channel-padded copy of x with a zero halo of (pad_h, pad_w).  One block per padded image row
+// (no per-pixel index divisions: the kernel is otherwise bound by them, not by memory); the block after the last
+// row writes the 8 trailing zero pixels (windows are read 32 floats wide).
 __global__ void __launch_bounds__(256) stage_pad_c4_kernel(const float* __restrict__ x, float4* __restrict__ xs, int N,
                                                            int H, int W, int C, int pad_h, int pad_w) {
     const int Hp = H + 2 * pad_h, Wp = W + 2 * pad_w;
-    const size_t total = size_t(N) * Hp * Wp + 8;   // 8 trailing zero pixels: windows are read 32 floats wide
-    const size_t stride = size_t(gridDim.x) * blockDim.x;
-    for (size_t i = size_t(blockIdx.x) * blockDim.x + threadIdx.x; i < total; i += stride) {
-        const int ww = int(i % Wp) - pad_w; size_t t = i / Wp;
-        const int hh = int(t % Hp) - pad_h; const size_t n = t / Hp;
+    const size_t row = blockIdx.x;                       // n * Hp + hh + pad_h
+    if (row == size_t(N) * Hp) {
+        if (threadIdx.x < 8) xs[row * Wp + threadIdx.x] = make_float4(0.f, 0.f, 0.f, 0.f);
+        return;
+    }
+    const size_t n = row / Hp;
+    const int hh = int(row - n * Hp) - pad_h;
+    float4* dst = xs + row * Wp;
+    if (hh < 0 || hh >= H) {
+        for (int i = threadIdx.x; i < Wp; i += blockDim.x) dst[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+        return;
+    }
+    const float* src = x + (n * H + hh) * size_t(W) * C;
+    for (int i = threadIdx.x; i < Wp; i += blockDim.x) {
+        const int ww = i - pad_w;
         float v[4] = {0.f, 0.f, 0.f, 0.f};
-        if (n < size_t(N) && hh >= 0 && hh < H && ww >= 0 && ww < W) {
-            const float* src = x + ((n * H + hh) * W + ww) * C;
-            for (int c = 0; c < C; ++c) v[c] = __ldg(src + c);
-        }
-        xs[i] = make_float4(v[0], v[1], v[2], v[3]);
+        if (ww >= 0 && ww < W)
+            for (int c = 0; c < C; ++c) v[c] = __ldg(src + size_t(ww) * C + c);
+        dst[i] = make_float4(v[0], v[1], v[2], v[3]);
     }
 }
 
@@ -471,8 +481,9 @@ int launch_stage_pad_c4(const float* x, float* xs, int N, int H, int W, int C, i
     const size_t total = size_t(N) * (H + 2 * pad_h) * (W + 2 * pad_w) + 8;
     {
         LaunchScope scope(KID_STAGE_PAD_C4, 4.0 * double(N) * H * W * C + 16.0 * double(total), st);
-        stage_pad_c4_kernel<<<grid_for(total, 256), 256, 0, st>>>(x, reinterpret_cast<float4*>(xs), N, H, W, C, pad_h,
-                                                                    pad_w);
+        const size_t rows = size_t(N) * (H + 2 * pad_h) + 1;        // + the block that writes the trailing zero pixels
+        if (rows > 0x7fffffffu) return PCL_ERR_UNSUPPORTED_SHAPE;
+        stage_pad_c4_kernel<<<unsigned(rows), 256, 0, st>>>(x, reinterpret_cast<float4*>(xs), N, H, W, C, pad_h, pad_w);
     }
     return PCL_CHECK_LAUNCH();
 }
