@@ -160,7 +160,7 @@ class ConvWorkload:
     name = "configs[1]: VGG-A mid conv layer 3x3 s1 p1, N=256 C=K=256 56x56: fwd + bwd_data + bwd_weights + SGD update"
     unit = "TFLOP/s"
 
-    def __init__(self, rank: int, minibatch: int = 0):
+    def __init__(self, rank: int, minibatch: int = 0, layer=None):
         import torch
         from paper_1602_06709_b200 import binding as B
         from paper_1602_06709_b200 import inputs
@@ -168,9 +168,13 @@ class ConvWorkload:
         c = dict(inputs.CFG2)
         if minibatch:
             c["N"] = minibatch
+        if layer:       # profiler captures of another 3x3 pad-1 layer shape (--layer C,K,H with --kernels-only)
+            c["C"], c["K"], c["H"] = layer
+            c["W"] = c["H"]
         self.N = c["N"]
         self.d = B.conv_desc(c["N"], c["C"], c["K"], c["H"], c["W"], c["R"], c["S"], 1, 1)
-        x, w, dy = inputs.conv_inputs("cfg2", f"conv{rank}", c["N"], c["C"], c["H"], c["W"], c["K"], 3, 3, 56, 56, "train")
+        x, w, dy = inputs.conv_inputs("cfg2", f"conv{rank}", c["N"], c["C"], c["H"], c["W"], c["K"], 3, 3, c["H"], c["W"],
+                                      "train")
         self.x_host = torch.from_numpy(x).pin_memory()
         self.dy_host = torch.from_numpy(dy).pin_memory()
         self.x = torch.empty_like(self.x_host, device="cuda"); self.x.copy_(self.x_host)
@@ -180,7 +184,7 @@ class ConvWorkload:
         self.y = torch.empty_like(self.dy); self.dx = torch.empty_like(self.x); self.dw = torch.empty_like(self.w)
         ws = max(B.conv_workspace_bytes(self.d, i) for i in range(3))
         self.ws = torch.empty(max(ws, 256), dtype=torch.uint8, device="cuda")
-        self.flops_pass = 2 * c["N"] * c["K"] * 56 * 56 * c["C"] * 9
+        self.flops_pass = 2 * c["N"] * c["K"] * c["H"] * c["W"] * c["C"] * 9
         self.units_per_step = 3 * self.flops_pass / 1e12      # TFLOP per step
         self.h2d = (self.x_host.numel() + self.dy_host.numel()) * 4
         self.d2h = self.dw.numel() * 4
@@ -351,7 +355,12 @@ def run_ours(args):
     def max_over_ranks(v: float) -> float:
         return replicas.max_over_ranks(v, device="cuda")
 
-    wl = WORKLOADS[args.workload](rank, args.minibatch)
+    if args.layer and not (args.kernels_only and args.workload == "conv"):
+        raise SystemExit("--layer changes the workload: only allowed with --workload conv --kernels-only")
+    if args.layer:
+        wl = ConvWorkload(rank, args.minibatch, tuple(int(v) for v in args.layer.split(",")))
+    else:
+        wl = WORKLOADS[args.workload](rank, args.minibatch)
     peaks = load_peaks()
     # The DNN step is ~45 short kernels and bound by the host's launch rate when issued one by one: by default it is
     # replayed from a CUDA graph of exactly those launches.  The VGG-A step keeps the GPU busy either way.
@@ -486,6 +495,7 @@ def main():
     ap.add_argument("--graph", default="auto", choices=["auto", "0", "1"],
                     help="replay the step from a CUDA graph of its launches (auto: the DNN step only)")
     ap.add_argument("--minibatch", type=int, default=0, help="override the workload's minibatch (profiling only)")
+    ap.add_argument("--layer", default="", help="C,K,H of another 3x3 pad-1 layer for --workload conv (profiling only)")
     ap.add_argument("--kernels-only", action="store_true",
                     help="run warm-up + timed steps only and print a short line (for profiler captures)")
     args = ap.parse_args()
