@@ -42,8 +42,7 @@ TF32_OVER_BF16_NOMINAL = 1.1 / 2.25      # nominal dense TF32 / bf16 tensor peak
 FALLBACK_BF16_TFLOPS = 1590.0
 FALLBACK_HBM_GBS = 6650.0
 # dram__bytes_read.sum + dram__bytes_write.sum per launch from ncu (captured at minibatch 32 and scaled to the
-# full minibatch: weight bytes once, activation bytes x 8); source: profiles/vgga_step_n256_launch_list.md and
-# profiles/tc_fprop_tc_wgrad_conv256_56x56_n32.md
+# full minibatch: weight bytes once, activation bytes x 8); the captures are summarised under profiles/
 NCU_DRAM_BYTES_PER_LAUNCH = {
     "vgga": {"tc_fprop_kernel": 531.4e6, "tc_wgrad_kernel": 930.7e6},
     "conv": {"tc_fprop_kernel": (163.8e6 + 283.9e6) / 2 * 8, "tc_wgrad_kernel": 209.9e6 * 8},
