@@ -166,7 +166,12 @@ int pcl_conv_bwd_weights_pooled(const pcl_conv_desc* d, const float* x, const fl
 /* Fully-connected forward: the k_h = k_w = out_h = out_w = 1 case of Algorithm 1
  * (Sec. 2.1):  y[n,k] = act(bias[k] + sum_c x[n,c] * w[k,c]).
  * x: [N][C], w: [K][C], bias: [K] or NULL, y: [N][K].
- * act: NONE, RELU or SIGMOID. */
+ * act: NONE, RELU or SIGMOID.
+ * Workspace: optional.  With pcl_fc_workspace_bytes(N, C, K, PCL_PASS_FWD) bytes (256-byte aligned) a
+ * layer with few output tiles and a long reduction splits the reduction over more CTAs and adds the
+ * partial results in a fixed order in a second pass; without it the same result is computed unsplit
+ * (up to the order of the fp32 additions).  pcl_conv_fwd() takes the same optional scratch
+ * (pcl_conv_workspace_bytes(d, PCL_PASS_FWD)). */
 int pcl_fc_fwd(int N, int C, int K, const float* x, const float* w, const float* bias,
                float* y, int act, void* ws, size_t ws_bytes, void* cuda_stream);
 

@@ -457,6 +457,45 @@ int launch_zero(float* p, size_t n, cudaStream_t st) {
     return PCL_CHECK_LAUNCH();
 }
 
+// out[r][k] = act(bias[k] + sum_s partial[s][r][k]): second pass of a split-reduction forward-type launch
+__global__ void __launch_bounds__(256) reduce_splits_bias_act_kernel(const float4* __restrict__ partial, float4* __restrict__ out,
+                                                                      const float* __restrict__ bias, int act, size_t n4,
+                                                                      int K4, int splits) {
+    const size_t stride = size_t(gridDim.x) * blockDim.x;
+    for (size_t i = size_t(blockIdx.x) * blockDim.x + threadIdx.x; i < n4; i += stride) {
+        float4 acc = partial[i];
+        for (int s = 1; s < splits; ++s) {
+            const float4 v = partial[size_t(s) * n4 + i];
+            acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
+        }
+        if (bias) {
+            const float4 b = __ldg(reinterpret_cast<const float4*>(bias) + (i % K4));
+            acc.x += b.x; acc.y += b.y; acc.z += b.z; acc.w += b.w;
+        }
+        if (act == PCL_ACT_RELU) {
+            acc.x = fmaxf(acc.x, 0.f); acc.y = fmaxf(acc.y, 0.f); acc.z = fmaxf(acc.z, 0.f); acc.w = fmaxf(acc.w, 0.f);
+        } else if (act == PCL_ACT_SIGMOID) {
+            acc.x = 1.f / (1.f + __expf(-acc.x)); acc.y = 1.f / (1.f + __expf(-acc.y));
+            acc.z = 1.f / (1.f + __expf(-acc.z)); acc.w = 1.f / (1.f + __expf(-acc.w));
+        }
+        out[i] = acc;
+    }
+}
+
+int launch_reduce_splits_bias_act(const float* partial, float* out, const float* bias, int act, size_t rows, int K,
+                                  int splits, cudaStream_t st) {
+    if (K % 4 != 0) return PCL_ERR_UNSUPPORTED_SHAPE;
+    const size_t n4 = rows * (K / 4);
+    if (n4 == 0) return PCL_OK;
+    {
+        LaunchScope scope(KID_REDUCE_SPLITS, 16.0 * double(n4) * (splits + 1), st);
+        reduce_splits_bias_act_kernel<<<grid_for(n4, 256), 256, 0, st>>>(reinterpret_cast<const float4*>(partial),
+                                                                          reinterpret_cast<float4*>(out), bias, act, n4, K / 4,
+                                                                          splits);
+    }
+    return PCL_CHECK_LAUNCH();
+}
+
 int launch_reduce_splits(const float* partial, float* out, size_t n, int splits, cudaStream_t st) {
     if (n == 0) return PCL_OK;
     {

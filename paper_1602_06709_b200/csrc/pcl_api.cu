@@ -228,12 +228,28 @@ int pcl_conv_out_dims(const pcl_conv_desc* d, int* P, int* Q) {
     return check_desc(d, P, Q);
 }
 
+// Scratch for a split reduction of the forward / backward-data launch (layers with few tiles and a long reduction:
+// the FC layers at small minibatch); 0 where the launcher would not split.
+static size_t fwd_split_bytes(const pcl_conv_desc& d, int P, int Q) {
+    TcFpropArgs a{nullptr, nullptr, nullptr, nullptr, nullptr, d.N, d.H, d.W, d.C, d.K, d.R, d.S, d.pad_h, d.pad_w, P, Q,
+                  PCL_ACT_NONE};
+    return align_up(tc_fprop_split_ws_bytes(a), 256);
+}
+static size_t bwd_data_split_bytes(const pcl_conv_desc& d, int P, int Q) {
+    TcFpropArgs a{nullptr, nullptr, nullptr, nullptr, nullptr, d.N, P, Q, d.K, d.C, d.R, d.S,
+                  d.R - 1 - d.pad_h, d.S - 1 - d.pad_w, d.H, d.W, PCL_ACT_NONE};
+    if (d.C % 32 == 0) a.wt_mn_major = 1;       // (either form of the weights gives the same tiling)
+    return align_up(tc_fprop_split_ws_bytes(a), 256);
+}
+
 size_t pcl_conv_workspace_bytes(const pcl_conv_desc* d, int pass) {
     int P, Q;
     if (check_desc(d, &P, &Q) != PCL_OK) return 0;
     switch (pass) {
-        case PCL_PASS_FWD: return few_channel_path_for(*d, pass) ? staged_x_bytes(*d) + staged_w_bytes(*d) : 0;
-        case PCL_PASS_BWD_DATA: return tensor_path_for(*d, pass) ? dw_bytes(*d) : 0;
+        case PCL_PASS_FWD:
+            if (few_channel_path_for(*d, pass)) return staged_x_bytes(*d) + staged_w_bytes(*d);
+            return tensor_path_for(*d, pass) ? fwd_split_bytes(*d, P, Q) : 0;
+        case PCL_PASS_BWD_DATA: return tensor_path_for(*d, pass) ? dw_bytes(*d) + bwd_data_split_bytes(*d, P, Q) : 0;
         case PCL_PASS_BWD_WEIGHTS: {
             const WgradPlan pl = plan_wgrad(*d, P, Q);
             return pl.partial_bytes + pl.colsum_bytes;
@@ -245,7 +261,7 @@ size_t pcl_conv_workspace_bytes(const pcl_conv_desc* d, int pass) {
 size_t pcl_fc_workspace_bytes(int N, int C, int K, int pass) {
     if (N <= 0 || C <= 0 || K <= 0) return 0;
     const pcl_conv_desc d{N, C, K, 1, 1, 1, 1, 1, 1, 0, 0};
-    if (pass == PCL_PASS_FWD) return 0;
+    if (pass == PCL_PASS_FWD) return pcl_conv_workspace_bytes(&d, PCL_PASS_FWD);
     // fc_bwd runs both backward contractions; either pass value returns the total (the weight-gradient part is
     // sized for either of its two forms)
     const size_t wgrad_form = pcl_conv_workspace_bytes(&d, PCL_PASS_BWD_WEIGHTS);
@@ -288,6 +304,9 @@ static int conv_fwd_impl(const pcl_conv_desc* d, const float* x, const float* w,
     } else if (tensor_path_for(*d, PCL_PASS_FWD)) {
         TcFpropArgs a{x, w, bias, nullptr, y, d->N, d->H, d->W, d->C, d->K, d->R, d->S, d->pad_h, d->pad_w, P, Q, act};
         if (y_pool && tc_fprop_can_pool(a)) { a.pool_out = y_pool; a.pool_idx = pool_codes; y_pool = nullptr; }
+        if (ws && (reinterpret_cast<uintptr_t>(ws) & 255) == 0) {      // scratch for a split reduction, if the caller gave some
+            a.split_ws = static_cast<float*>(ws); a.split_ws_bytes = ws_bytes;
+        }
         rc = launch_tc_fprop(a, st);
     } else if (g_path.load() == PCL_PATH_TENSOR) {
         return PCL_ERR_UNSUPPORTED_SHAPE;
@@ -335,6 +354,8 @@ int pcl_conv_bwd_data(const pcl_conv_desc* d, const float* dy, const float* w, c
         // dx = "forward" convolution of dy with the flipped, transposed weights, pad' = R-1-pad
         TcFpropArgs a{dy, w, nullptr, relu_mask_src, dx, d->N, P, Q, d->K, d->C, d->R, d->S,
                       d->R - 1 - d->pad_h, d->S - 1 - d->pad_w, d->H, d->W, PCL_ACT_NONE};
+        // what follows the transposed-weights area is scratch for a split reduction
+        a.split_ws = reinterpret_cast<float*>(static_cast<char*>(ws) + need); a.split_ws_bytes = ws_bytes - need;
         if (weights_read_in_place(*d)) {
             // the kernel reads w itself as an MN-major operand (taps flipped by index): no transposed copy
             a.wt_mn_major = 1; a.flip_taps = 1;

@@ -75,6 +75,11 @@ struct TcFpropArgs {
     // with pool_out: [N][P/2][Q/2][Kout] bytes, bits 0-1 = position of the window's first maximum (row-major), bit 2 set
     // where that maximum is <= 0 (what a ReLU mask would zero); lets the pooling backward pass skip reading `out`
     unsigned char* pool_idx = nullptr;
+    // Optional scratch for a split reduction (launches with few tiles and a long reduction): if given, and the
+    // launcher finds splits worth while and the scratch large enough (tc_fprop_split_ws_bytes()), every split's raw
+    // partial tile goes there and a second pass adds them in a fixed order and applies bias and activation.
+    float* split_ws = nullptr;
+    size_t split_ws_bytes = 0;
     // wt_mn_major != 0: `wt` is laid out [Cin][R*S][Kout] (output maps innermost), i.e. a layer's own KRSC weights
     // seen from its backward-data pass (reduction over the layer's K, columns = the layer's C): the kernel then
     // reads B as an MN-major operand and no transposed copy is needed.  Needs Kout % 32 == 0.
@@ -82,6 +87,8 @@ struct TcFpropArgs {
     int wt_mn_major = 0, flip_taps = 0;
 };
 bool tc_fprop_can_pool(const TcFpropArgs& a);
+// bytes of split_ws with which launch_tc_fprop(a) would split the reduction (0: it would not)
+size_t tc_fprop_split_ws_bytes(const TcFpropArgs& a);
 bool tc_fprop_eligible(const TcFpropArgs& a);
 long tc_fprop_colsum_rows(const TcFpropArgs& a);
 int launch_tc_fprop(const TcFpropArgs& a, cudaStream_t st);
@@ -131,6 +138,9 @@ int launch_generic_bwd_weights(const pcl_conv_desc& d, int P, int Q, const float
 // ---- HBM-bound helpers ------------------------------------------------------
 int launch_sgd(float* w, const float* dw, size_t n, float lr, cudaStream_t st);
 int launch_reduce_splits(const float* partial, float* out, size_t n, int splits, cudaStream_t st);
+// out[r][k] = act(bias[k] + sum_s partial[s][r][k]), splits added in index order; K % 4 == 0
+int launch_reduce_splits_bias_act(const float* partial, float* out, const float* bias, int act, size_t rows, int K,
+                                  int splits, cudaStream_t st);
 int launch_zero(float* p, size_t n, cudaStream_t st);
 // wt_t[c][R-1-r][S-1-s][k] = w[k][r][s][c]
 int launch_transpose_flip(const float* w, float* wt_t, int K, int R, int S, int C, cudaStream_t st);

@@ -81,6 +81,11 @@ struct FpropParams {
     const float* mask_src;
     float* out;
     int tma_store;              // the epilogue writes `out` with TMA stores from the staging tiles (tmOut is valid)
+    // Split reduction (few tiles, long reduction: the FC layers at small minibatch): ksplit > 1 cuts the k-steps of
+    // every tile into ksplit equal ranges of kps k-steps, each a tile of its own whose raw accumulators go to
+    // out + split * split_stride (the caller adds the splits, then bias and activation).  Plain tiling only.
+    int ksplit, kps;
+    size_t split_stride;
     unsigned char* pool_idx;    // optional, with pool_out: per pooled element the position of the maximum (bits 0-1) and bit 2
                                 // if that maximum is <= 0
     float* pool_out;            // optional [N][P/2][Q/2][Kout]: 2x2 window maxima of the output
@@ -92,25 +97,28 @@ struct FpropParams {
 // coordinates (k tile, q tile, p tile, n tile) in mixed-radix counters, so that no role pays integer
 // divisions per tile.
 struct TileIter {
-    int t, kt, qi, pi, ni;
-    int step, dk, dq, dp, dn;
+    int t, kt, qi, pi, ni, sp;      // sp: reduction split (outermost; 0 unless ksplit > 1)
+    int step, dk, dq, dp, dn, ds;
     __device__ void init(const FpropParams& p, int first, int stride) {
         t = first; step = stride;
         int m = first;
         kt = m % p.tiles_k; m /= p.tiles_k;
         qi = m % p.tiles_q; m /= p.tiles_q;
-        pi = m % p.tiles_p; ni = m / p.tiles_p;
+        pi = m % p.tiles_p; m /= p.tiles_p;
+        ni = m % p.tiles_n; sp = m / p.tiles_n;
         m = stride;
         dk = m % p.tiles_k; m /= p.tiles_k;
         dq = m % p.tiles_q; m /= p.tiles_q;
-        dp = m % p.tiles_p; dn = m / p.tiles_p;
+        dp = m % p.tiles_p; m /= p.tiles_p;
+        dn = m % p.tiles_n; ds = m / p.tiles_n;
     }
     __device__ void next(const FpropParams& p) {
         t += step;
         kt += dk; int c = kt >= p.tiles_k; kt -= c ? p.tiles_k : 0;
         qi += dq + c; c = qi >= p.tiles_q; qi -= c ? p.tiles_q : 0;
         pi += dp + c; c = pi >= p.tiles_p; pi -= c ? p.tiles_p : 0;
-        ni += dn + c;
+        ni += dn + c; c = ni >= p.tiles_n; ni -= c ? p.tiles_n : 0;
+        sp += ds + c;
     }
 };
 
@@ -436,8 +444,8 @@ tc_fprop_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
 
     const int bw = 1 << p.bw_log2, bh = 1 << p.bh_log2;
     const int m_tiles = p.tiles_q * p.tiles_p * p.tiles_n;
-    const int total_tiles = m_tiles * p.tiles_k;
-    const int kiters = p.R * p.S * p.cblocks;
+    const int total_tiles = m_tiles * p.tiles_k * p.ksplit;
+    const int kiters = p.ksplit > 1 ? p.kps : p.R * p.S * p.cblocks;       // k-steps of one tile
 
     if (warp == 0) {
         // ------------------------------------------------------------ producer
@@ -502,9 +510,17 @@ tc_fprop_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                         }
                     }
                 } else {
-                    // k-step order: r, then s, then channel block
+                    // k-step order: r, then s, then channel block; a reduction split starts kps k-steps further
                     int c0 = 0, s = 0, tap = 0;
                     int cq = q0 - p.pad_w, cp = p0 - p.pad_h;
+                    if (p.ksplit > 1) {
+                        const int kit0 = it.sp * kiters;
+                        tap = kit0 / p.cblocks;
+                        c0 = (kit0 - tap * p.cblocks) * kBlockC;
+                        const int r0 = tap / p.S;
+                        s = tap - r0 * p.S;
+                        cq += s; cp += r0;
+                    }
                     for (int kit = 0; kit < kiters; kit += p.KS) {
                         if (!bounded_wait_addr(empty_a, phase ^ 1u, &abort_flag, p.status, WAIT_PRODUCER_EMPTY)) {
                             ok = false;
@@ -725,10 +741,11 @@ tc_fprop_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                 // (l>>3) + 4*i.  Bias, activation and the ReLU mask are applied on the way out.
                 size_t roff[8];
                 uint32_t vmask = 0;
+                const size_t sp_off = static_cast<size_t>(it.sp) * p.split_stride;      // (0 unless the reduction is split)
 #pragma unroll
                 for (int i = 0; i < 8; ++i) {
                     const int src = (lane >> 3) + 4 * i;
-                    roff[i] = __shfl_sync(0xffffffffu, static_cast<unsigned long long>(pix * p.Kout), src);
+                    roff[i] = __shfl_sync(0xffffffffu, static_cast<unsigned long long>(pix * p.Kout + sp_off), src);
                     vmask |= (__shfl_sync(0xffffffffu, static_cast<int>(valid), src) ? 1u : 0u) << i;
                 }
                 const uint32_t stg = smem_u32(epi_stage + epi * 4096);
@@ -836,7 +853,7 @@ tc_fprop_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                     if (!kPool && kEpi == kEpiWarps && p.split_acc) add_second_accumulator(t_row + t_second + ch * 32, v);
                     const int col0 = kt * p.BN + ch * 32;
                     if (valid && col0 < p.Kout) {
-                        float* dst = p.out + pix * p.Kout + col0;
+                        float* dst = p.out + static_cast<size_t>(it.sp) * p.split_stride + pix * p.Kout + col0;
                         const float* msk = kMask ? p.mask_src + pix * p.Kout + col0 : nullptr;
 #pragma unroll
                         for (int j = 0; j < 32; ++j) {
@@ -1069,6 +1086,46 @@ long tc_fprop_colsum_rows(const TcFpropArgs& a) {
     return rows;
 }
 
+namespace {
+// Reduction splits for a launch with few tiles and a long reduction (plain tiling, no fused mask / sums / pooling):
+// as many as fill the SMs, each an equal whole number of pipeline slots (at least two).
+int choose_ksplit(const TcFpropArgs& a, const TileCfg& cfg, int cblocks, int sm_count) {
+    if (cfg.halo || a.mask_src || a.colsum_rows || a.pool_out || !a.out || a.Kout % 4 != 0) return 1;
+    const int hook = env_int("PCL_KSPLIT", 0);              // test hook: 1 = never, n = n splits where they divide
+    if (hook == 1) return 1;
+    const long tiles = long(cfg.tiles_q) * cfg.tiles_p * cfg.tiles_n * cfg.tiles_k;        // CTAs (a pair is two)
+    const int kiters = a.R * a.S * cblocks;
+    if (kiters % cfg.KS != 0) return 1;
+    const int slots = kiters / cfg.KS;
+    long want = hook > 1 ? hook : sm_count / tiles;
+    if (want > 32) want = 32;
+    // measured (B200, minibatch 256): the second pass costs ~5 us, which splitting repays from ~32 slots on
+    // (C = 2048) when each split keeps at least 8
+    if (hook <= 1 && (tiles * 2 > sm_count || slots < 32)) return 1;
+    const int min_slots = hook > 1 ? 2 : 8;
+    for (int k = int(want); k >= 2; --k)
+        if (slots % k == 0 && slots / k >= min_slots) return k;
+    return 1;
+}
+}  // namespace
+
+size_t tc_fprop_split_ws_bytes(const TcFpropArgs& a) {
+    int sm = g_sm_count;
+    if (sm == 0) {
+        int dev = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess ||
+            cudaDeviceGetAttribute(&sm, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sm <= 0)
+            sm = 148;
+    }
+    if (!tc_fprop_eligible(a)) return 0;
+    const TileCfg cfg = select_cfg(a, sm);
+    if (!cfg.ok) return 0;
+    TcFpropArgs b = a;
+    if (!b.out) b.out = reinterpret_cast<float*>(16);       // (sizing query: only "an output exists" matters)
+    const int k = choose_ksplit(b, cfg, (a.Cin + kBlockC - 1) / kBlockC, sm);
+    return k > 1 ? size_t(k) * a.N * a.P * a.Q * a.Kout * 4 : 0;
+}
+
 int launch_tc_fprop(const TcFpropArgs& a, cudaStream_t st) {
     if (!tc_fprop_eligible(a)) return PCL_ERR_UNSUPPORTED_SHAPE;
     static bool attr_set = false;
@@ -1114,6 +1171,17 @@ int launch_tc_fprop(const TcFpropArgs& a, cudaStream_t st) {
     p.tmem_cols = 32;
     while (p.tmem_cols < (p.split_acc ? 4 : 2) * p.MT * p.BN) p.tmem_cols *= 2;
     p.bias = a.bias; p.mask_src = a.mask_src; p.out = a.out;
+    // split reduction: raw partial tiles to the caller's scratch, bias and activation after the splits are added
+    p.ksplit = 1; p.kps = 0; p.split_stride = 0;
+    if (a.split_ws) {
+        int k = choose_ksplit(a, cfg, p.cblocks, g_sm_count);
+        const size_t per = size_t(a.N) * a.P * a.Q * a.Kout * 4;
+        while (k > 1 && (size_t(k) * per > a.split_ws_bytes || (a.R * a.S * p.cblocks / cfg.KS) % k != 0)) --k;
+        if (k > 1 && m_tiles * p.tiles_k * k <= 0x7fffffffL) {
+            p.ksplit = k; p.kps = a.R * a.S * p.cblocks / k; p.split_stride = per / 4;
+            p.out = a.split_ws; p.bias = nullptr; p.act = PCL_ACT_NONE;
+        }
+    }
     if (a.pool_out && !tc_fprop_can_pool(a)) return PCL_ERR_UNSUPPORTED_SHAPE;
     p.pool_out = a.pool_out;
     p.pool_idx = a.pool_out ? a.pool_idx : nullptr;
@@ -1177,7 +1245,9 @@ int launch_tc_fprop(const TcFpropArgs& a, cudaStream_t st) {
     // Output map for the TMA-store epilogue: a warp stores the 32 consecutive box pixels it owns, 32 maps at a time.
     CUtensorMap tmOut = tmA;        // (a valid map is passed in any case; unused unless p.tma_store)
     p.tma_store = 0;
-    if (!a.out) {
+    if (p.ksplit > 1) {
+        // (split partials go out through the per-lane path: plain stores at out + split * split_stride)
+    } else if (!a.out) {
         // pooled output only: the epilogue stages each chunk as for a TMA store, takes the maxima from the staging
         // tile and stores nothing at full resolution
         if (!a.pool_out || a.colsum_rows) return PCL_ERR_BAD_ARG;
@@ -1207,7 +1277,7 @@ int launch_tc_fprop(const TcFpropArgs& a, cudaStream_t st) {
             if (fixed + stages * slot <= kSmemBudget) { p.stages = stages; wide_epi = true; }
         }
     }
-    const long total = m_tiles * p.tiles_k;
+    const long total = m_tiles * p.tiles_k * p.ksplit;
     const size_t smem = (p.halo ? size_t(p.NA) * p.a_buf_bytes + size_t(p.stages) * p.KS * (cfg.pair ? p.BN * 64 : p.BN * 128)
                                 : size_t(p.stages) * p.KS * (kABytes + (cfg.pair ? p.BN * 64 : p.BN * 128))) +
                         (wide_epi ? kEpiStageBytesWide : kEpiStageBytes) + 1024;
@@ -1228,7 +1298,7 @@ int launch_tc_fprop(const TcFpropArgs& a, cudaStream_t st) {
             cached_clusters = n < g_sm_count / 2 ? n : g_sm_count / 2;
             cached_smem = smem;
         }
-        const long pair_tiles = long(p.tiles_q) * p.tiles_p * p.tiles_n * p.tiles_k;
+        const long pair_tiles = long(p.tiles_q) * p.tiles_p * p.tiles_n * p.tiles_k * p.ksplit;
         long nclus = pair_tiles < cached_clusters ? pair_tiles : cached_clusters;
         lc.gridDim = dim3(unsigned(2 * nclus));
         LaunchScope scope(KID_TC_FPROP, 2.0 * a.N * a.P * a.Q * double(a.Kout) * a.Cin * a.R * a.S, st);
@@ -1245,7 +1315,10 @@ int launch_tc_fprop(const TcFpropArgs& a, cudaStream_t st) {
         else if (p.mask_src) tc_fprop_kernel<false, false, true><<<grid, kThreads, smem, st>>>(tmA, tmB, tmOut, p);
         else tc_fprop_kernel<false, false, false><<<grid, kThreads, smem, st>>>(tmA, tmB, tmOut, p);
     }
-    return cudaGetLastError() == cudaSuccess ? PCL_OK : PCL_ERR_CUDA;
+    if (cudaGetLastError() != cudaSuccess) return PCL_ERR_CUDA;
+    if (p.ksplit > 1)
+        return launch_reduce_splits_bias_act(a.split_ws, a.out, a.bias, a.act, size_t(a.N) * a.P * a.Q, a.Kout, p.ksplit, st);
+    return PCL_OK;
 }
 
 }  // namespace pcl

@@ -199,7 +199,7 @@ class VggA(_HostFeed):
                      B.conv_workspace_bytes(L.desc, B.PASS_BWD_WEIGHTS), B.conv_bwd_data_colsum_workspace_bytes(L.desc),
                      B.maxpool2x2_bwd_colsum_workspace_bytes(N, L.H, L.W, L.K))
         for C, K in fc:
-            ws = max(ws, B.fc_workspace_bytes(N, C, K, B.PASS_BWD_DATA))
+            ws = max(ws, B.fc_workspace_bytes(N, C, K, B.PASS_BWD_DATA), B.fc_workspace_bytes(N, C, K, B.PASS_FWD))
         self.ws = torch.empty(max(ws, 256), dtype=torch.uint8, device=dev)
         self.conv_flops_fwd = [2 * N * L.K * L.H * L.W * L.C * 9 for L in self.convs]
         self.fc_flops_fwd = [2 * N * C * K for C, K in fc]
@@ -231,7 +231,7 @@ class VggA(_HostFeed):
         a = self.pooled[-1].view(self.N, self.flat)
         for j, (C, K) in enumerate(self.fcs):
             act = B.ACT_RELU if j + 1 < len(self.fcs) else B.ACT_NONE
-            B.fc_fwd(self.N, C, K, a, self.fc_w(j), self.fc_b(j), self.fc_out[j], act)
+            B.fc_fwd(self.N, C, K, a, self.fc_w(j), self.fc_b(j), self.fc_out[j], act, self.ws)
             a = self.fc_out[j]
         B.softmax_xent(self.N, self.classes, self.fc_out[-1], self.labels, self.loss, self.fc_dout[-1])
 
@@ -297,7 +297,8 @@ class Dnn(_HostFeed):
         self.labels = torch.zeros(N, dtype=torch.int32, device=dev)
         self._feed_init()
         self.loss = torch.zeros(1, device=dev)
-        ws = max(B.fc_workspace_bytes(N, C, K, B.PASS_BWD_DATA) for C, K in self.layers)
+        ws = max(max(B.fc_workspace_bytes(N, C, K, B.PASS_BWD_DATA), B.fc_workspace_bytes(N, C, K, B.PASS_FWD))
+                 for C, K in self.layers)
         self.ws = torch.empty(max(ws, 256), dtype=torch.uint8, device=dev)
         self.fc_flops_fwd = [2 * N * C * K for C, K in self.layers]
 
@@ -311,7 +312,7 @@ class Dnn(_HostFeed):
         n = len(self.layers)
         for j, (C, K) in enumerate(self.layers):
             act = B.ACT_SIGMOID if j + 1 < n else B.ACT_NONE
-            B.fc_fwd(self.N, C, K, a, self.w(j), self.b(j), self.out[j], act)
+            B.fc_fwd(self.N, C, K, a, self.w(j), self.b(j), self.out[j], act, self.ws)
             a = self.out[j]
         B.softmax_xent(self.N, self.dims[-1], self.out[-1], self.labels, self.loss, self.dout[-1])
 

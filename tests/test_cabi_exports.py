@@ -47,7 +47,11 @@ def test_host_side_checks(built_lib):
                           null, 0, null) == B.ERR_BAD_ARG
     # a pass that needs workspace refuses a missing one before touching the device
     big = B.conv_desc(8, 64, 64, 28, 28, 3, 3, 1, 1)
-    assert B.conv_workspace_bytes(big, B.PASS_BWD_DATA) == 64 * 64 * 9 * 4
+    # (room for the transposed weights, plus scratch for a split reduction where the layer has few tiles)
+    assert B.conv_workspace_bytes(big, B.PASS_BWD_DATA) >= 64 * 64 * 9 * 4
+    wide = B.conv_desc(256, 256, 256, 56, 56, 3, 3, 1, 1)      # thousands of tiles: no split, the weights' room only
+    assert B.conv_workspace_bytes(wide, B.PASS_BWD_DATA) == 256 * 256 * 9 * 4
+    assert B.conv_workspace_bytes(wide, B.PASS_FWD) == 0
     assert L.pcl_conv_bwd_data(ctypes.byref(big), ctypes.c_void_p(16), ctypes.c_void_p(16), null, ctypes.c_void_p(16),
                                null, 0, null) == B.ERR_WORKSPACE
     assert L.pcl_maxpool2x2_fwd(1, 3, 4, 4, ctypes.c_void_p(16), ctypes.c_void_p(16), null) == B.ERR_UNSUPPORTED_SHAPE

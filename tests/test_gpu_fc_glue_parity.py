@@ -10,6 +10,8 @@ pytestmark = pytest.mark.gpu
 
 FC_CASES = [
     # N, C, K, act            (ragged in every dimension; K > 256 spans several column tiles)
+    (96, 960, 264, "relu"),      # 30 channel blocks: reduction splits of 3 and 5 divide the slots
+    (256, 1920, 128, "sigmoid"),
     (130, 440, 200, "sigmoid"),
     (64, 96, 520, "relu"),
     (257, 36, 1000, "none"),
@@ -50,6 +52,16 @@ def test_fc_fwd_bwd(N, C, K, act, path, path_guard, monkeypatch):
     B.check_device_status()
     y = yt.cpu().numpy()
     G.assert_parity(y, oracle.fc_fwd(x, w, b, code), "fc fwd")
+    # with scratch the launcher may split the reduction over more CTAs (few tiles, long reduction); PCL_KSPLIT pins
+    # the number of splits where it divides the reduction's pipeline slots
+    for ks in ("0", "2", "3", "5"):
+        monkeypatch.setenv("PCL_KSPLIT", ks)
+        ws_f = G.workspace(B.fc_workspace_bytes(N, C, K, B.PASS_FWD))
+        yt2 = torch.full((N, K), float("nan"), device="cuda")
+        B.fc_fwd(N, C, K, xt, wt, bt, yt2, code, ws_f)
+        B.check_device_status()
+        G.assert_parity(yt2.cpu().numpy(), oracle.fc_fwd(x, w, b, code), f"fc fwd, PCL_KSPLIT={ks}")
+    monkeypatch.delenv("PCL_KSPLIT")
     # backward is checked on the GPU's own forward output (per-call parity)
     dyt = G.dev(dy)
     dxt = torch.full((N, C), float("nan"), device="cuda")
