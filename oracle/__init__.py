@@ -26,8 +26,10 @@ maximum in row-major window order.
 
 Pins (see ``tests/test_oracle_*.py``): literal scatter-form transcription in the
 paper's index order on tiny layers, adjoint identities, finite differences,
-matmul / shift / all-ones special cases, torch.float64 conv2d and autograd.
-Parity unpinned: nothing in this file.
+matmul / shift / all-ones special cases, torch.float64 conv2d and autograd;
+the chained steps of ``networks.py`` against torch.float64 networks with
+autograd and finite differences of their loss.
+Parity unpinned: nothing in this package.
 """
 from __future__ import annotations
 
@@ -227,10 +229,12 @@ def act_grad(y, dy, act) -> np.ndarray:
     raise ValueError(act)
 
 
-def fc_bwd(x, w, y, dy, act=ACT_NONE, dz_dtype=np.float32):
-    """Returns (dz, dx, dw, db).  dz = dy * act'(y) is rounded to ``dz_dtype``
-    (fp32 by default: the product path stores dz in fp32 and feeds that to both
-    contractions) before dx = dz w, dw = dz^T x, db = sum_n dz."""
+def fc_bwd(x, w, y, dy, act=ACT_NONE, dz_dtype=np.float64):
+    """Returns (dz, dx, dw, db): dz = dy * act'(y), dx = dz w, dw = dz^T x,
+    db = sum_n dz (the 1x1 case of the two update rules of Sec. 2.1), all in
+    float64.  A caller that compares against an implementation which stores dz
+    in fp32 between the two contractions passes ``dz_dtype=np.float32``: dz is
+    then rounded once before it is used."""
     N, C = x.shape
     K = w.shape[0]
     dz = act_grad(y, dy, act).astype(dz_dtype)

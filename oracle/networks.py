@@ -1,7 +1,9 @@
 """TEST INFRASTRUCTURE: fp64 oracle of one full training step of the two
 topologies (VGG-A CNN, fully-connected DNN), chaining the per-layer oracle
 functions in float64 with no intermediate rounding.  Used by the chained parity
-tests and by the benchmark's CPU-baseline leg only."""
+tests and by the benchmark's CPU-baseline leg only.  Pinned by
+``tests/test_oracle_network_pins.py`` (torch float64 library networks with
+autograd; finite differences of the loss)."""
 from __future__ import annotations
 
 import numpy as np

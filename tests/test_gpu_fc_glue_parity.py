@@ -70,7 +70,7 @@ def test_fc_fwd_bwd(N, C, K, act, path, path_guard, monkeypatch):
     ws = G.workspace(B.fc_workspace_bytes(N, C, K, B.PASS_BWD_DATA))
     B.fc_bwd(N, C, K, xt, wt, yt, code, dyt, dxt, dwt, dbt, ws)
     B.check_device_status()
-    dz_ref, dx_ref, dw_ref, db_ref = oracle.fc_bwd(x, w, y, dy, code)
+    dz_ref, dx_ref, dw_ref, db_ref = oracle.fc_bwd(x, w, y, dy, code, dz_dtype=np.float32)
     np.testing.assert_allclose(dyt.cpu().numpy(), dz_ref, rtol=1e-5, atol=1e-7)     # dz written back into dy
     dz_gpu = dyt.cpu().numpy()
     # contractions are checked against the oracle fed the GPU's own dz
