@@ -392,6 +392,7 @@ def run_ours(args):
     if status != B.OK:
         raise SystemExit(f"device status {status}: {B.status_string(status)}")
     value = replicas.whole_job_throughput(wl.units_per_step, args.steps, world, ms)
+    unit, h2d, d2h = wl.unit, wl.h2d, wl.d2h
 
     if args.kernels_only:      # for profiler captures: just the steps, one short line
         if rank == 0:
@@ -404,7 +405,8 @@ def run_ours(args):
     ms_e2e, _, _ = timed(wl.e2e_step, e2e_steps, 1)
     e2e_value = replicas.whole_job_throughput(wl.units_per_step, e2e_steps, world, ms_e2e)
 
-    # instrumented repeat of the same steps: CUDA events around every kernel launch on the launching stream
+    # instrumented repeat of the same steps: CUDA events around every kernel launch on the launching stream,
+    # tagged with the pass (ABI call) the launch belongs to
     prof_steps = max(1, min(args.steps, 5))
     barrier()
     B.profile_begin()
@@ -412,24 +414,120 @@ def run_ours(args):
         wl.step_eager()       # (a graph replay does not pass through the library's per-launch events)
     stats = B.profile_end()
     barrier()
-    total_ms = sum(s["total_ms"] for s in stats.values())
+    report = summarise_profile(stats, prof_steps, peaks, clocks, ms / args.steps, args.workload)
+
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        r = time_oracle(args.workload, 1, 0, min_seconds=12.0)
+        cpu = dict(value=r["value"], unit=wl.unit, cores=r["cores"], kind="oracle", sample=r["sample"],
+                   seconds=r["seconds"])
+
+    config = {"workload": wl.name, "l2": "inputs larger than L2 (activations are GBs per step)"
+              if args.workload != "dnn" else "weights+activations 0.3 GB per step, larger than L2",
+              "parallelism": "replicas only" if world > 1 else "single GPU", "cuda_graph": bool(use_graph),
+              **wl.describe()}
+    legs = None
+    if world == 1 and args.workload == "vgga" and not args.no_legs:
+        # the other configurations, a few repetitions each, so that one record carries them; and the TF32 stick
+        del wl
+        torch.cuda.empty_cache()
+        legs = run_legs(torch, B)
+        stick = measure_tf32_stick(torch, local_rank)
+        report["roofline"].update(stick)
+        if stick.get("peak_measured_tf32_burst"):
+            report["roofline"]["frac_of_measured_tf32_burst"] = report["roofline"]["achieved"] / stick["peak_measured_tf32_burst"]
+            report["roofline"]["frac_of_measured_tf32_sustained"] = report["roofline"]["achieved"] / stick["peak_measured_tf32_sustained"]
+
+    if rank == 0:
+        line = {
+            "metric": METRIC, "value": value, "unit": unit, "n_gpus": world, "steps": args.steps,
+            "warmup": max(args.warmup, 3), "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "tf32", "data": "synthetic",
+            "config": config,
+            "clocks": clocks,
+            "e2e": {"value": e2e_value, "unit": unit, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                    "ms_per_step": ms_e2e / e2e_steps, "steps": e2e_steps},
+            "gpu_launches": launches,
+            "cpu_baseline": cpu,
+            **report,
+        }
+        if legs is not None:
+            line["legs"] = legs
+        print(json.dumps(line), flush=True)
+    replicas.shutdown()
+
+
+CONTRACTIONS = ("tc_fprop_kernel", "tc_wgrad_kernel", "generic_fwd", "generic_bwd_data", "generic_bwd_weights")
+NOMINAL_TF32_TFLOPS = 1100.0
+
+
+def summarise_profile(stats, prof_steps, peaks, clocks, ms_per_step, workload):
+    """stats: {"<pass>/<kernel>": dict(launches, total_ms, work)} over prof_steps steps."""
+    by_kernel, by_pass = {}, {}
+    for name, s in stats.items():
+        ps, k = name.split("/", 1)
+        a = by_kernel.setdefault(k, dict(launches=0, total_ms=0.0, work=0.0))
+        for f in ("launches", "total_ms", "work"):
+            a[f] += s[f]
+        b = by_pass.setdefault(ps, dict(ms=0.0, contraction_ms=0.0, flop=0.0, launches=0))
+        b["ms"] += s["total_ms"]
+        b["launches"] += s["launches"]
+        if k in CONTRACTIONS:
+            b["contraction_ms"] += s["total_ms"]
+            b["flop"] += s["work"]
+    total_ms = sum(s["total_ms"] for s in by_kernel.values())
     kernels = {k: dict(launches=s["launches"] // prof_steps, ms_per_step=s["total_ms"] / prof_steps,
-                       share=s["total_ms"] / total_ms if total_ms else 0.0,
-                       work_per_step=s["work"] / prof_steps) for k, s in stats.items()}
-    dom = max(stats.items(), key=lambda kv: kv[1]["total_ms"])[0]
-    ds = stats[dom]
-    contraction = dom in ("tc_fprop_kernel", "tc_wgrad_kernel", "generic_fwd", "generic_bwd_data", "generic_bwd_weights")
-    if contraction:
+                       share=s["total_ms"] / total_ms if total_ms else 0.0, work_per_step=s["work"] / prof_steps)
+               for k, s in by_kernel.items()}
+
+    def rate(flop, ms_):
+        return flop / (ms_ / 1e3) / 1e12 if ms_ > 0 else None
+
+    # burst figure: the timed region is a fraction of a second (the sustained figure belongs to seconds-long loops
+    # at the power cap; MEASURED_PEAKS took it at a median 1305 MHz, this step runs at 1.7-1.96 GHz)
+    peak_burst = peaks["bf16_burst"] * TF32_OVER_BF16_NOMINAL
+    peak_sust = peaks["bf16_sustained"] * TF32_OVER_BF16_NOMINAL
+    out = {"kernels": kernels}
+    passes = {}
+    for ps, key in (("conv_fwd", "fwd"), ("conv_bwd_data", "bwd_data"), ("conv_bwd_weights", "bwd_weights")):
+        if ps in by_pass and by_pass[ps]["flop"] > 0:
+            b = by_pass[ps]
+            passes[key] = dict(tflops=rate(b["flop"], b["ms"]), ms=b["ms"] / prof_steps,
+                               contraction_kernel_tflops=rate(b["flop"], b["contraction_ms"]),
+                               contraction_kernel_ms=b["contraction_ms"] / prof_steps,
+                               flop=b["flop"] / prof_steps, launches=b["launches"] // prof_steps)
+    if passes:
+        out["conv_passes"] = passes
+        flop = sum(by_pass[ps]["flop"] for ps in ("conv_fwd", "conv_bwd_data", "conv_bwd_weights") if ps in by_pass)
+        ms_all = sum(by_pass[ps]["ms"] for ps in ("conv_fwd", "conv_bwd_data", "conv_bwd_weights") if ps in by_pass)
+        t = rate(flop, ms_all)
+        out["conv_layers"] = dict(tflops=t, ms=ms_all / prof_steps, flop=flop / prof_steps,
+                                  frac_of_nominal_1100=t / NOMINAL_TF32_TFLOPS, frac_of_measured=t / peak_burst,
+                                  note="every launch of the three conv passes (staging, split reductions and "
+                                       "transposes included) over the layers' own 2*N*K*P*Q*C*R*S")
+    fcs = [by_pass[ps] for ps in ("fc_fwd", "fc_bwd") if ps in by_pass and by_pass[ps]["flop"] > 0]
+    if fcs:
+        flop = sum(b["flop"] for b in fcs); ms_all = sum(b["ms"] for b in fcs)
+        out["fc_layers"] = dict(tflops=rate(flop, ms_all), ms=ms_all / prof_steps, flop=flop / prof_steps)
+    tc = [s for k, s in by_kernel.items() if k in CONTRACTIONS]
+    if tc:
+        t = rate(sum(s["work"] for s in tc), sum(s["total_ms"] for s in tc))
+        out["all_contractions"] = dict(tflops=t, frac_of_measured=t / peak_burst, frac_of_nominal_1100=t / NOMINAL_TF32_TFLOPS,
+                                       flop_over_step_time_tflops=rate(sum(s["work"] for s in tc) / prof_steps, ms_per_step))
+    if "sgd_kernel" in by_kernel:
+        s = by_kernel["sgd_kernel"]
+        out["sgd_update_gbs"] = s["work"] / (s["total_ms"] / 1e3) / 1e9
+
+    dom = max(by_kernel.items(), key=lambda kv: kv[1]["total_ms"])[0]
+    ds = by_kernel[dom]
+    if dom in CONTRACTIONS:
         achieved = ds["work"] / (ds["total_ms"] / 1e3) / 1e12
-        # the sustained figure for a kernel timed inside a long, power-capped step; the burst figure when the timed
-        # region never met the power cap (short steps: the clock sampler saw no sw_power_cap)
-        capped = bool(clocks and "sw_power_cap" in (clocks.get("reasons") or []))
-        which = "sustained" if capped or not clocks else "burst"
-        peak = peaks["bf16_" + which] * TF32_OVER_BF16_NOMINAL
-        roofline = dict(bound="tensor", kernel=dom, achieved=achieved, peak=peak, unit="TFLOP/s", frac=achieved / peak,
-                        traffic=None,
-                        peak_source=f"{peaks['source']} bf16 {which} {peaks['bf16_' + which]:.1f} TFLOP/s x nominal "
-                                    f"TF32/bf16 ratio {TF32_OVER_BF16_NOMINAL:.4f}",
+        roofline = dict(bound="tensor", kernel=dom, achieved=achieved, peak=peak_burst, unit="TFLOP/s",
+                        frac=achieved / peak_burst, traffic=None,
+                        peak_source=f"{peaks['source']} bf16 burst {peaks['bf16_burst']:.1f} TFLOP/s x nominal TF32/bf16 "
+                                    f"ratio {TF32_OVER_BF16_NOMINAL:.4f} (of {peaks['source']})",
+                        frac_of_sustained_derived=achieved / peak_sust, peak_sustained_derived=peak_sust,
+                        frac_of_nominal_1100=achieved / NOMINAL_TF32_TFLOPS,
                         launches_per_step=ds["launches"] // prof_steps,
                         flop_per_launch_avg=ds["work"] / ds["launches"], ms_per_launch_avg=ds["total_ms"] / ds["launches"],
                         timed_in="instrumented repeat of the timed steps (events on the launching stream)")
@@ -438,49 +536,111 @@ def run_ours(args):
         roofline = dict(bound="hbm", kernel=dom, achieved=achieved, peak=peaks["hbm_gbs"], unit="GB/s",
                         frac=achieved / peaks["hbm_gbs"], traffic=None, peak_source=f"{peaks['source']} copy bandwidth",
                         launches_per_step=ds["launches"] // prof_steps)
-    roofline["traffic"] = NCU_DRAM_BYTES_PER_LAUNCH.get(args.workload, {}).get(dom)
+    roofline["traffic"] = NCU_DRAM_BYTES_PER_LAUNCH.get(workload, {}).get(dom)
+    roofline["traffic_source"] = "ncu capture summarised under profiles/ (a constant of this script, not measured by this run)"
+    out["roofline"] = roofline
+    return out
 
-    extra = {}
-    tc = [stats[k] for k in ("tc_fprop_kernel", "tc_wgrad_kernel") if k in stats]
-    if tc:
-        tflops = sum(s["work"] for s in tc) / (sum(s["total_ms"] for s in tc) / 1e3) / 1e12
-        peak_s = peaks["bf16_sustained"] * TF32_OVER_BF16_NOMINAL
-        extra["tensor_core_kernels"] = dict(tflops=tflops, frac_of_measured_sustained_tf32=tflops / peak_s,
-                                            frac_of_nominal_1100=tflops / 1100.0)
-    allc = [s for k, s in stats.items() if k in ("tc_fprop_kernel", "tc_wgrad_kernel", "generic_fwd",
-                                                 "generic_bwd_data", "generic_bwd_weights")]
-    if allc:
-        extra["all_contractions_tflops"] = sum(s["work"] for s in allc) / (sum(s["total_ms"] for s in allc) / 1e3) / 1e12
-    if "sgd_kernel" in stats:
-        s = stats["sgd_kernel"]
-        extra["sgd_update_gbs"] = s["work"] / (s["total_ms"] / 1e3) / 1e9
 
-    cpu = None
-    if rank == 0 and world == 1 and not args.no_cpu_baseline:
-        r = time_oracle(args.workload, 1, 0, min_seconds=12.0)
-        cpu = dict(value=r["value"], unit=wl.unit, cores=r["cores"], kind="oracle", sample=r["sample"],
-                   seconds=r["seconds"])
+def measure_tf32_stick(torch, gpu_index):
+    """A TF32 measuring stick outside the product path and outside every timed region: torch.matmul 8192^3 with
+    allow_tf32 (cuBLAS), best of 10 (burst) and back to back for ~3 s (sustained), clocks sampled meanwhile."""
+    try:
+        old = torch.backends.cuda.matmul.allow_tf32
+        torch.backends.cuda.matmul.allow_tf32 = True
+        n = 8192
+        a = torch.randn(n, n, device="cuda"); b = torch.randn(n, n, device="cuda"); c = torch.empty(n, n, device="cuda")
+        flop = 2.0 * n ** 3
+        for _ in range(3):
+            torch.matmul(a, b, out=c)
+        torch.cuda.synchronize()
+        best = 1e30
+        for _ in range(10):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(); torch.matmul(a, b, out=c); e1.record(); e1.synchronize()
+            best = min(best, e0.elapsed_time(e1))
+        sampler = ClockSampler(gpu_index); sampler.start()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        reps = max(10, int(3000.0 / best))
+        e0.record()
+        for _ in range(reps):
+            torch.matmul(a, b, out=c)
+        e1.record(); e1.synchronize()
+        clk = sampler.stop()
+        torch.backends.cuda.matmul.allow_tf32 = old
+        return dict(peak_measured_tf32_burst=flop / (best / 1e3) / 1e12,
+                    peak_measured_tf32_sustained=flop * reps / (e0.elapsed_time(e1) / 1e3) / 1e12,
+                    peak_measured_tf32_how="torch.matmul fp32 8192^3 with allow_tf32 (a library GEMM, measuring stick only): "
+                                           "best of 10, and back to back for ~3 s",
+                    peak_measured_tf32_clocks=clk)
+    except Exception as e:          # the stick is context; the bench line must not depend on it
+        return dict(peak_measured_tf32_burst=None, peak_measured_tf32_sustained=None, peak_measured_tf32_how=f"failed: {e}")
 
-    if rank == 0:
-        line = {
-            "metric": METRIC, "value": value, "unit": wl.unit, "n_gpus": world, "steps": args.steps,
-            "warmup": max(args.warmup, 3), "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak",
-            "vs_baseline": None, "dtype": "tf32", "data": "synthetic",
-            "config": {"workload": wl.name, "l2": "inputs larger than L2 (activations are GBs per step)"
-                       if args.workload != "dnn" else "weights+activations 0.3 GB per step, larger than L2",
-                       "parallelism": "replicas only" if world > 1 else "single GPU", "cuda_graph": bool(use_graph),
-                       **wl.describe()},
-            "clocks": clocks,
-            "e2e": {"value": e2e_value, "unit": wl.unit, "h2d_bytes_per_step": wl.h2d, "d2h_bytes_per_step": wl.d2h,
-                    "ms_per_step": ms_e2e / e2e_steps, "steps": e2e_steps},
-            "gpu_launches": launches,
-            "roofline": roofline,
-            "cpu_baseline": cpu,
-            "kernels": kernels,
-            **extra,
-        }
-        print(json.dumps(line), flush=True)
-    replicas.shutdown()
+
+def run_legs(torch, B):
+    """Short legs for the other configurations: the three passes of the mid VGG-A layer (configs[1]) and of each
+    OverFeat-FAST-shaped layer (configs[2]), and the DNN step (configs[3]).  Device-side seeded inputs with the
+    recipe's distributions; L2 is flushed before every timed repetition (a 256 MB buffer is overwritten)."""
+    gen = torch.Generator(device="cuda"); gen.manual_seed(160206709)
+    flush = torch.empty(64 * 1024 * 1024, device="cuda")
+
+    def time_call(fn, reps=5, warm=3):
+        for _ in range(warm):
+            fn()
+        best, tot = 1e30, 0.0
+        for _ in range(reps):
+            flush.zero_()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(); fn(); e1.record(); e1.synchronize()
+            t = e0.elapsed_time(e1); best = min(best, t); tot += t
+        return tot / reps, best
+
+    def conv_leg(N, C, K, H, R, stride, pad):
+        d = B.conv_desc(N, C, K, H, H, R, R, stride, pad)
+        P = (H + 2 * pad - R) // stride + 1
+        x = torch.rand(N, H, H, C, device="cuda", generator=gen)
+        w = torch.randn(K, R, R, C, device="cuda", generator=gen) * (2.0 / (R * R * C)) ** 0.5
+        dy = torch.randn(N, P, P, K, device="cuda", generator=gen) * 1e-3
+        bias = torch.zeros(K, device="cuda")
+        y = torch.empty_like(dy); dx = torch.empty_like(x); dw = torch.empty_like(w)
+        ws = torch.empty(max(256, max(B.conv_workspace_bytes(d, i) for i in range(3))), dtype=torch.uint8, device="cuda")
+        flop = 2.0 * N * K * P * P * C * R * R
+        out = {"shape": f"N={N} C={C} K={K} H=W={H} {R}x{R} stride {stride} pad {pad}", "flop_per_pass": flop}
+        for key, fn in (("fwd", lambda: B.conv_fwd(d, x, w, bias, y, B.ACT_RELU, ws)),
+                        ("bwd_data", lambda: B.conv_bwd_data(d, dy, w, None, dx, ws)),
+                        ("bwd_weights", lambda: B.conv_bwd_weights(d, x, dy, dw, None, True, ws))):
+            mean, best = time_call(fn)
+            out[key] = dict(ms=mean, best_ms=best, tflops=flop / (mean / 1e3) / 1e12,
+                            frac_of_nominal_1100=flop / (mean / 1e3) / 1e12 / NOMINAL_TF32_TFLOPS)
+        return out
+
+    legs = {"timing": "CUDA events per call, mean of 5 after 3 warm-ups, L2 flushed before each; whole ABI call "
+                      "(staging, transposes and split reductions included)"}
+    legs["cfg2_vgg_mid_layer"] = conv_leg(256, 256, 256, 56, 3, 1, 1)
+    cfg3 = {}
+    for name, (C, H, K, R, st, pad) in (("C1", (3, 231, 96, 11, 4, 0)), ("C2", (96, 24, 256, 5, 1, 0)),
+                                        ("C3", (256, 12, 512, 3, 1, 1)), ("C4", (512, 12, 1024, 3, 1, 1)),
+                                        ("C5", (1024, 12, 1024, 3, 1, 1))):
+        cfg3[name] = conv_leg(256, C, K, H, R, st, pad)
+        torch.cuda.empty_cache()
+    legs["cfg3_overfeat_fast"] = cfg3
+    dnn = DnnWorkload(0)
+    dnn.use_graph()
+    for _ in range(3):
+        dnn.step()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(20):
+        dnn.step()
+    e1.record(); e1.synchronize()
+    ms_dnn = e0.elapsed_time(e1) / 20
+    fl = 3 * sum(dnn.net.fc_flops_fwd) - dnn.net.fc_flops_fwd[0]       # the first layer has no backpropagation
+    legs["cfg4_dnn_step"] = dict(ms_per_step=ms_dnn, frames_per_s=dnn.N / (ms_dnn / 1e3), tflops=fl / (ms_dnn / 1e3) / 1e12,
+                                 flop_per_step=fl, cuda_graph=True, steps=20)
+    status = B.last_device_status()
+    if status != B.OK:
+        raise SystemExit(f"device status {status} after the legs: {B.status_string(status)}")
+    return legs
 
 
 def main():
@@ -491,6 +651,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="vgga", choices=sorted(WORKLOADS))
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-legs", action="store_true", help="skip the short legs for the other configurations")
     ap.add_argument("--graph", default="auto", choices=["auto", "0", "1"],
                     help="replay the step from a CUDA graph of its launches (auto: the DNN step only)")
     ap.add_argument("--minibatch", type=int, default=0, help="override the workload's minibatch (profiling only)")

@@ -54,7 +54,8 @@ enum {
     PCL_ERR_WORKSPACE = 4,         /* workspace smaller than pcl_*_workspace_bytes()  */
     PCL_ERR_CUDA = 5,              /* a CUDA runtime/driver call failed               */
     PCL_ERR_DEVICE_TIMEOUT = 6,    /* a bounded device-side wait ran out              */
-    PCL_ERR_SCRATCH_LIMIT = 7      /* problem larger than the built-in scratch array  */
+    PCL_ERR_SCRATCH_LIMIT = 7,     /* problem larger than the built-in scratch array  */
+    PCL_ERR_BAD_LABEL = 8          /* pcl_softmax_xent met a label outside [0, K)     */
 };
 
 enum { PCL_PASS_FWD = 0, PCL_PASS_BWD_DATA = 1, PCL_PASS_BWD_WEIGHTS = 2 };
@@ -81,7 +82,7 @@ size_t pcl_fc_workspace_bytes(int N, int C, int K, int pass);
  *                                            q*stride_w + s - pad_w, c] * w[k,r,s,c])
  * with zero contribution outside the image (cross-correlation, no kernel
  * flip).  x: NHWC in, w: KRSC in, bias: [K] in or NULL, y: NPQK out.
- * act: PCL_ACT_NONE or PCL_ACT_RELU (fused into the epilogue). */
+ * act: PCL_ACT_NONE, PCL_ACT_RELU or PCL_ACT_SIGMOID (fused into the epilogue). */
 int pcl_conv_fwd(const pcl_conv_desc* d, const float* x, const float* w, const float* bias,
                  float* y, int act, void* ws, size_t ws_bytes, void* cuda_stream);
 
@@ -114,8 +115,9 @@ int pcl_conv_fwd_pool(const pcl_conv_desc* d, const float* x, const float* w, co
  * tap reaches get 0).  relu_mask_src: NULL, or an NHWC tensor of dx's shape
  * (the layer's input, i.e. a ReLU output): dx is zeroed where it is <= 0.
  * Workspace: pcl_conv_workspace_bytes(d, PCL_PASS_BWD_DATA) (room for a flipped,
- * transposed copy of w, the "transpose-weights" of Sec. 2.3; the tensor-core path
- * reads w in place instead when C is a multiple of 32, the workspace must still be given). */
+ * transposed copy of w, the "transpose-weights" of Sec. 2.3, plus optional room for
+ * a split reduction; the tensor-core path reads w in place instead when C is a
+ * multiple of 32, and a smaller or absent workspace then only forgoes the split). */
 int pcl_conv_bwd_data(const pcl_conv_desc* d, const float* dy, const float* w,
                       const float* relu_mask_src, float* dx,
                       void* ws, size_t ws_bytes, void* cuda_stream);
@@ -217,12 +219,16 @@ int pcl_maxpool2x2_bwd_codes(int N, int H, int W, int C, const unsigned char* co
                              int relu_mask, float* dx, float* dx_colsum,
                              void* ws, size_t ws_bytes, void* cuda_stream);
 /* loss = -(1/N) sum_n log softmax(logits[n,:])[labels[n]]  (device scalar, overwritten)
- * dlogits = (softmax(logits) - onehot(labels)) / N.  labels: device int32 [N]. */
+ * dlogits = (softmax(logits) - onehot(labels)) / N.  labels: device int32 [N].
+ * A label outside [0, K) is never used as an index: that row gets no target (its gradient is
+ * softmax/N) and no loss term, and the next pcl_last_device_status() returns PCL_ERR_BAD_LABEL.
+ * dlogits is bitwise reproducible; the loss scalar is summed over the rows with fp32 atomics, so
+ * its last bits may differ from run to run. */
 int pcl_softmax_xent(int N, int K, const float* logits, const int* labels,
                      float* loss, float* dlogits, void* cuda_stream);
 
 /* Synchronises the stream, then reads and clears the device status word of the
- * current device.  PCL_OK, PCL_ERR_DEVICE_TIMEOUT or PCL_ERR_CUDA. */
+ * current device.  PCL_OK, PCL_ERR_DEVICE_TIMEOUT, PCL_ERR_BAD_LABEL or PCL_ERR_CUDA. */
 int pcl_last_device_status(void* cuda_stream);
 /* Which wait gave up when pcl_last_device_status() last returned PCL_ERR_DEVICE_TIMEOUT (0 if it never did):
  * 0x101 producer waiting for a free slot, 0x102 MMA issuer waiting for operands, 0x103 MMA issuer waiting for a
@@ -242,8 +248,13 @@ unsigned long long pcl_launch_count(void);
  * else's pool, any place where cudaMalloc is off limits.  The call itself makes
  * no cudaMalloc / cudaFree and uses no allocating library routine.
  *
- *  - Capacity: pcl_noalloc_scratch_bytes() = 16 MiB, i.e. K*R*S*C <= 4 194 304
- *    weights.  Larger layers get PCL_ERR_SCRATCH_LIMIT and nothing is launched.
+ *  - Capacity: pcl_noalloc_scratch_bytes() = 16 MiB.  What has to fit is the
+ *    transposed copy, which only layers with C % 32 != 0 need: for those
+ *    K*R*S*C <= 4 194 304 weights, else PCL_ERR_SCRATCH_LIMIT and nothing is
+ *    launched.  Layers with C % 32 == 0 are read in place and accepted at any size.
+ *    (Where the regular call would also use scratch to split a long reduction, this
+ *    one splits only as far as the array's remaining room allows: same result up to
+ *    the order of the fp32 additions when the split count differs.)
  *    Every GPU that loads the library holds these 16 MiB until the process ends.
  *  - The first call on each device looks up the array's device address (one
  *    runtime query, no allocation); make that first call before any stream
@@ -264,10 +275,14 @@ size_t pcl_noalloc_scratch_bytes(void);
  * pcl_profile_end() waits for those events, stops the bracketing and returns, per
  * kernel family that ran, the number of launches, the summed event time and the
  * summed algorithmic work (flops for the contraction kernels, bytes for the
- * memory-bound ones).  stats: HOST array of max_stats entries; *n_stats entries
- * are filled.  Event objects are created on first use and reused. */
+ * memory-bound ones), separately for each pass the launches belonged to: `name` is
+ * "<pass>/<kernel>" with pass one of conv_fwd, conv_bwd_data, conv_bwd_weights, fc_fwd,
+ * fc_bwd, other (the ABI call that made the launch).  A contraction launch counts the
+ * layer's own 2*N*K*P*Q*C*R*S (Comp of Sec. 3.1 per pass), also where the kernel runs on
+ * a zero-padded view of the layer.  stats: HOST array of max_stats entries; *n_stats
+ * entries are filled.  Event objects are created on first use and reused. */
 typedef struct {
-    char name[32];
+    char name[64];
     unsigned long long launches;
     double total_ms;
     double work;

@@ -20,6 +20,7 @@ PATH_AUTO, PATH_TENSOR, PATH_GENERIC = 0, 1, 2
 OK = 0
 ERR_BAD_ARG, ERR_UNSUPPORTED_SHAPE, ERR_MISALIGNED, ERR_WORKSPACE, ERR_CUDA, ERR_DEVICE_TIMEOUT = 1, 2, 3, 4, 5, 6
 ERR_SCRATCH_LIMIT = 7
+ERR_BAD_LABEL = 8
 
 EXPORTS = [
     "pcl_set_path", "pcl_conv_out_dims", "pcl_conv_workspace_bytes", "pcl_fc_workspace_bytes",
@@ -40,7 +41,7 @@ class PclError(RuntimeError):
 
 
 class KernelStat(ctypes.Structure):
-    _fields_ = [("name", ctypes.c_char * 32), ("launches", ctypes.c_ulonglong), ("total_ms", ctypes.c_double),
+    _fields_ = [("name", ctypes.c_char * 64), ("launches", ctypes.c_ulonglong), ("total_ms", ctypes.c_double),
                 ("work", ctypes.c_double)]
 
 
@@ -291,9 +292,9 @@ def profile_begin():
 
 
 def profile_end():
-    """Returns {kernel name: dict(launches, total_ms, work)} for the kernels that ran since profile_begin()."""
-    arr = (KernelStat * 32)()
+    """Returns {"<pass>/<kernel>": dict(launches, total_ms, work)} for the launches since profile_begin()."""
+    arr = (KernelStat * 128)()
     n = ctypes.c_int(0)
-    _check(lib().pcl_profile_end(arr, 32, ctypes.byref(n)), "pcl_profile_end")
+    _check(lib().pcl_profile_end(arr, 128, ctypes.byref(n)), "pcl_profile_end")
     return {arr[i].name.decode(): dict(launches=int(arr[i].launches), total_ms=float(arr[i].total_ms),
                                        work=float(arr[i].work)) for i in range(n.value)}

@@ -338,7 +338,8 @@ __global__ void __launch_bounds__(256) maxpool_bwd_idx_kernel(const unsigned cha
 // One CTA per row: max, sum of exponentials, loss term, gradient.
 __global__ void __launch_bounds__(256) softmax_xent_kernel(const float* __restrict__ logits,
                                                            const int* __restrict__ labels, float* __restrict__ loss,
-                                                           float* __restrict__ dlogits, int N, int K) {
+                                                           float* __restrict__ dlogits, int N, int K,
+                                                           unsigned int* __restrict__ status) {
     __shared__ float red[32];
     __shared__ float bcast;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -369,14 +370,20 @@ __global__ void __launch_bounds__(256) softmax_xent_kernel(const float* __restri
         }
         __syncthreads();
         sum = bcast;
-        const int lab = labels[n];
+        // a label outside [0, K) names no class: the row gets no target and no loss term (nothing is read through
+        // it), and the device status word records it
+        int lab = labels[n];
+        if (lab < 0 || lab >= K) {
+            if (threadIdx.x == 0) atomicCAS(status, 0u, static_cast<unsigned int>(kStatusBadLabel));
+            lab = -1;
+        }
         const float inv_n = 1.f / float(N);
         const float inv_sum = 1.f / sum;
         for (int k = threadIdx.x; k < K; k += blockDim.x) {
             const float pk = expf(z[k] - mx) * inv_sum;
             dlogits[size_t(n) * K + k] = (pk - (k == lab ? 1.f : 0.f)) * inv_n;
         }
-        if (threadIdx.x == 0) atomicAdd(loss, -(z[lab] - mx - logf(sum)) * inv_n);
+        if (threadIdx.x == 0 && lab >= 0) atomicAdd(loss, -(z[lab] - mx - logf(sum)) * inv_n);
         __syncthreads();
     }
 }
@@ -651,7 +658,9 @@ int launch_softmax_xent(int N, int K, const float* logits, const int* labels, fl
     if (rc != PCL_OK) return rc;
     {
         LaunchScope scope(KID_SOFTMAX_XENT, 8.0 * double(N) * K, st);
-        softmax_xent_kernel<<<N < 1184 ? N : 1184, 256, 0, st>>>(logits, labels, loss, dlogits, N, K);
+        unsigned int* status = device_status_ptr();
+        if (!status) return PCL_ERR_CUDA;
+        softmax_xent_kernel<<<N < 1184 ? N : 1184, 256, 0, st>>>(logits, labels, loss, dlogits, N, K, status);
     }
     return PCL_CHECK_LAUNCH();
 }

@@ -14,8 +14,10 @@
 
 namespace {
 
-// Capacity of the built-in scratch: 4 Mi floats = 16 MiB.  It holds K*R*S*C
-// weights, so layers up to e.g. 512 x 512 x 3 x 3 (2.36 M weights) fit.
+// Capacity of the built-in scratch: 4 Mi floats = 16 MiB.  What must fit is the
+// transposed copy of the K*R*S*C weights, and only for layers that need one
+// (C not a multiple of 32); layers whose weights are read in place need no
+// scratch and are accepted at any size.
 constexpr size_t kScratchFloats = size_t(4) << 20;
 
 // File-scope device array.  In host code this name is only a handle for the
@@ -46,15 +48,17 @@ float* scratch_address(int* rc) {
 extern "C" int pcl_conv_bwd_data_noalloc(const pcl_conv_desc* d, const float* dy, const float* w,
                                          const float* relu_mask_src, float* dx, void* cuda_stream) {
     if (!d) return PCL_ERR_BAD_ARG;
-    const size_t need = pcl_conv_workspace_bytes(d, PCL_PASS_BWD_DATA);
+    int P = 0, Q = 0;
+    int rc = pcl_conv_out_dims(d, &P, &Q);
+    if (rc != PCL_OK) return rc;
+    // Only the transposed weight copy is mandatory.  The regular entry point also uses scratch, when it has some,
+    // to split long reductions over more thread blocks; here it splits as far as the rest of the array allows.
+    const size_t need = pcl::bwd_data_transposed_bytes(*d);
     if (need > kScratchFloats * sizeof(float)) return PCL_ERR_SCRATCH_LIMIT;
-    if (need == 0)   // this shape runs on a kernel that needs no scratch
-        return pcl_conv_bwd_data(d, dy, w, relu_mask_src, dx, nullptr, 0, cuda_stream);
-    int rc = PCL_OK;
     float* scratch = scratch_address(&rc);
     if (rc != PCL_OK) return rc;
-    // The transposed weights are written in full before they are read, so nothing has to be cleared
-    // between calls; what the previous call left in the array is simply overwritten.
+    // The transposed weights (and any split partials) are written in full before they are read, so nothing
+    // has to be cleared between calls; what the previous call left in the array is simply overwritten.
     return pcl_conv_bwd_data(d, dy, w, relu_mask_src, dx, scratch, kScratchFloats * sizeof(float), cuda_stream);
 }
 

@@ -3,6 +3,7 @@
 // the caller's stream.
 #include <atomic>
 #include <mutex>
+#include <stdio.h>
 #include <string.h>
 #include <vector>
 
@@ -31,7 +32,17 @@ unsigned int* device_status_ptr() {
 static std::atomic<unsigned long long> g_launches{0};
 
 namespace {
-struct ProfEntry { int kid; double work; cudaEvent_t e0, e1; };
+struct ProfEntry { int kid; int pass; double work; cudaEvent_t e0, e1; };
+// Which ABI call the launches of this thread belong to (outermost call wins), and, for its contraction launches,
+// the layer's own algorithmic work 2*N*K*P*Q*C*R*S: a launch that runs on a padded or staged view of the layer
+// (few-channel staging, phase-decomposed strides) must not count the zero padding as work.
+struct PassState { int pass = 0; int depth = 0; double flops = 0.0; };
+thread_local PassState t_pass;
+const char* const kPassNames[PROF_PASS_COUNT] = {"other", "conv_fwd", "conv_bwd_data", "conv_bwd_weights", "fc_fwd", "fc_bwd"};
+bool is_contraction(int kid) {
+    return kid == KID_TC_FPROP || kid == KID_TC_WGRAD || kid == KID_GENERIC_FWD || kid == KID_GENERIC_DGRAD ||
+           kid == KID_GENERIC_WGRAD;
+}
 std::mutex g_prof_mu;
 bool g_prof_on = false;
 std::vector<ProfEntry> g_prof_entries;       // entries of the current profiling window
@@ -57,7 +68,8 @@ LaunchScope::LaunchScope(int kid, double work, cudaStream_t stream) : slot(-1), 
     g_launches.fetch_add(1, std::memory_order_relaxed);
     std::lock_guard<std::mutex> lock(g_prof_mu);
     if (!g_prof_on) return;
-    ProfEntry e{kid, work, prof_event(), prof_event()};
+    if (t_pass.depth > 0 && t_pass.flops > 0.0 && is_contraction(kid)) work = t_pass.flops;
+    ProfEntry e{kid, t_pass.depth > 0 ? t_pass.pass : PROF_PASS_OTHER, work, prof_event(), prof_event()};
     if (!e.e0 || !e.e1) return;
     cudaEventRecord(e.e0, st);
     slot = int(g_prof_entries.size());
@@ -68,6 +80,16 @@ LaunchScope::~LaunchScope() {
     if (slot < 0) return;
     std::lock_guard<std::mutex> lock(g_prof_mu);
     if (slot < int(g_prof_entries.size())) cudaEventRecord(g_prof_entries[slot].e1, st);
+}
+
+PassScope::PassScope(int pass, double flops) {
+    if (t_pass.depth++ == 0) { t_pass.pass = pass; t_pass.flops = flops; }
+}
+PassScope::~PassScope() {
+    if (--t_pass.depth == 0) { t_pass.pass = PROF_PASS_OTHER; t_pass.flops = 0.0; }
+}
+double conv_pass_flops(const pcl_conv_desc& d, int P, int Q) {
+    return 2.0 * d.N * double(d.K) * P * Q * double(d.C) * d.R * d.S;
 }
 
 static std::atomic<int> g_path{PCL_PATH_AUTO};
@@ -122,6 +144,18 @@ bool weights_read_in_place(const pcl_conv_desc& d) {
     return d.C % 32 == 0 && !(v && v[0] == '0');
 }
 
+size_t dw_bytes(const pcl_conv_desc& d);
+}  // namespace
+
+// Bytes of the flipped, transposed weight copy backward-data makes on the tensor-core path (0 where the weights
+// are read in place or another kernel family runs): the part of the backward-data workspace that is mandatory.
+size_t bwd_data_transposed_bytes(const pcl_conv_desc& d) {
+    if (g_path.load() == PCL_PATH_GENERIC || d.stride_h != 1 || d.stride_w != 1) return 0;
+    if (!(d.K % 4 == 0 && d.pad_h <= d.R - 1 && d.pad_w <= d.S - 1)) return 0;
+    return weights_read_in_place(d) ? 0 : dw_bytes(d);
+}
+
+namespace {
 int check_desc(const pcl_conv_desc* d, int* P, int* Q) {
     if (!d) return PCL_ERR_BAD_ARG;
     if (d->N <= 0 || d->C <= 0 || d->K <= 0 || d->H <= 0 || d->W <= 0 || d->R <= 0 || d->S <= 0 || d->stride_h <= 0 ||
@@ -278,6 +312,7 @@ static int conv_fwd_impl(const pcl_conv_desc* d, const float* x, const float* w,
     int rc = check_desc(d, &P, &Q);
     if (rc != PCL_OK) return rc;
     if (!x || !w || (!y && !y_pool)) return PCL_ERR_BAD_ARG;
+    PassScope pass_scope(PROF_PASS_CONV_FWD, conv_pass_flops(*d, P, Q));
     if (act != PCL_ACT_NONE && act != PCL_ACT_RELU && act != PCL_ACT_SIGMOID) return PCL_ERR_BAD_ARG;
     if (!aligned16(x) || !aligned16(w) || !aligned16(y) || !aligned16(bias) || !aligned16(y_pool)) return PCL_ERR_MISALIGNED;
     // without y only the one-kernel form can run (the separate pooling kernel reads y)
@@ -345,17 +380,21 @@ int pcl_conv_bwd_data(const pcl_conv_desc* d, const float* dy, const float* w, c
     int rc = check_desc(d, &P, &Q);
     if (rc != PCL_OK) return rc;
     if (!dy || !w || !dx) return PCL_ERR_BAD_ARG;
+    PassScope pass_scope(PROF_PASS_CONV_BWD_DATA, conv_pass_flops(*d, P, Q));
     if (!aligned16(dy) || !aligned16(w) || !aligned16(dx) || !aligned16(relu_mask_src)) return PCL_ERR_MISALIGNED;
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
     if (tensor_path_for(*d, PCL_PASS_BWD_DATA)) {
-        const size_t need = dw_bytes(*d);
-        if (!ws || ws_bytes < need) return PCL_ERR_WORKSPACE;
-        if (reinterpret_cast<uintptr_t>(ws) & 255) return PCL_ERR_MISALIGNED;
+        // mandatory: room for the transposed copy where one is made; whatever follows it is optional scratch for
+        // a split reduction (the launcher splits as far as that room allows, or not at all)
+        const size_t need = bwd_data_transposed_bytes(*d);
+        if (need > 0 && (!ws || ws_bytes < need)) return PCL_ERR_WORKSPACE;
+        if (ws && (reinterpret_cast<uintptr_t>(ws) & 255)) return PCL_ERR_MISALIGNED;
         // dx = "forward" convolution of dy with the flipped, transposed weights, pad' = R-1-pad
         TcFpropArgs a{dy, w, nullptr, relu_mask_src, dx, d->N, P, Q, d->K, d->C, d->R, d->S,
                       d->R - 1 - d->pad_h, d->S - 1 - d->pad_w, d->H, d->W, PCL_ACT_NONE};
-        // what follows the transposed-weights area is scratch for a split reduction
-        a.split_ws = reinterpret_cast<float*>(static_cast<char*>(ws) + need); a.split_ws_bytes = ws_bytes - need;
+        if (ws && ws_bytes > need) {
+            a.split_ws = reinterpret_cast<float*>(static_cast<char*>(ws) + need); a.split_ws_bytes = ws_bytes - need;
+        }
         if (weights_read_in_place(*d)) {
             // the kernel reads w itself as an MN-major operand (taps flipped by index): no transposed copy
             a.wt_mn_major = 1; a.flip_taps = 1;
@@ -407,6 +446,7 @@ int pcl_conv_bwd_data_colsum(const pcl_conv_desc* d, const float* dy, const floa
     int rc = check_desc(d, &P, &Q);
     if (rc != PCL_OK) return rc;
     if (!dy || !w || !dx || !dx_colsum) return PCL_ERR_BAD_ARG;
+    PassScope pass_scope(PROF_PASS_CONV_BWD_DATA, conv_pass_flops(*d, P, Q));
     if (!aligned16(dy) || !aligned16(w) || !aligned16(dx) || !aligned16(relu_mask_src) || !aligned16(dx_colsum))
         return PCL_ERR_MISALIGNED;
     const size_t need = pcl_conv_bwd_data_colsum_workspace_bytes(d);
@@ -547,6 +587,7 @@ int pcl_conv_bwd_weights_pooled(const pcl_conv_desc* d, const float* x, const fl
     int rc = check_desc(d, &P, &Q);
     if (rc != PCL_OK) return rc;
     if (!x || !dy_pool || !pool_codes || !dw) return PCL_ERR_BAD_ARG;
+    PassScope pass_scope(PROF_PASS_CONV_BWD_WEIGHTS, conv_pass_flops(*d, P, Q));
     if (!aligned16(x) || !aligned16(dy_pool) || !aligned16(pool_codes) || !aligned16(dw) || !aligned16(dbias))
         return PCL_ERR_MISALIGNED;
     const PooledWgradPlan pl = plan_pooled_wgrad(*d, P, Q);
@@ -583,6 +624,7 @@ int pcl_conv_bwd_weights(const pcl_conv_desc* d, const float* x, const float* dy
     int rc = check_desc(d, &P, &Q);
     if (rc != PCL_OK) return rc;
     if (!x || !dy || !dw) return PCL_ERR_BAD_ARG;
+    PassScope pass_scope(PROF_PASS_CONV_BWD_WEIGHTS, conv_pass_flops(*d, P, Q));
     if (!aligned16(x) || !aligned16(dy) || !aligned16(dw) || !aligned16(dbias)) return PCL_ERR_MISALIGNED;
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
     const WgradPlan pl = plan_wgrad(*d, P, Q);
@@ -635,6 +677,7 @@ int pcl_conv_bwd_weights(const pcl_conv_desc* d, const float* x, const float* dy
 int pcl_fc_fwd(int N, int C, int K, const float* x, const float* w, const float* bias, float* y, int act, void* ws,
                size_t ws_bytes, void* cuda_stream) {
     const pcl_conv_desc d{N, C, K, 1, 1, 1, 1, 1, 1, 0, 0};
+    PassScope pass_scope(PROF_PASS_FC_FWD, 2.0 * N * double(C) * K);
     return pcl_conv_fwd(&d, x, w, bias, y, act, ws, ws_bytes, cuda_stream);
 }
 
@@ -649,6 +692,7 @@ int pcl_fc_bwd(int N, int C, int K, const float* x, const float* w, const float*
         return PCL_ERR_MISALIGNED;
     const pcl_conv_desc d{N, C, K, 1, 1, 1, 1, 1, 1, 0, 0};
     const bool dw_fwd = fc_dw_as_forward(N, C, K);
+    PassScope pass_scope(PROF_PASS_FC_BWD, 2.0 * N * double(C) * K);
     const size_t colsum_bytes = plan_wgrad(d, 1, 1).colsum_bytes;
     const size_t need_w = dw_fwd ? fc_dzt_bytes(N, K) + colsum_bytes : pcl_conv_workspace_bytes(&d, PCL_PASS_BWD_WEIGHTS);
     const size_t need_d = dx ? pcl_conv_workspace_bytes(&d, PCL_PASS_BWD_DATA) : 0;
@@ -714,7 +758,7 @@ int pcl_last_device_status(void* cuda_stream) {
         g_last_wait_code.store(v);
         const unsigned int zero = 0;
         if (cudaMemcpyToSymbol(g_device_status, &zero, sizeof(zero)) != cudaSuccess) return PCL_ERR_CUDA;
-        return PCL_ERR_DEVICE_TIMEOUT;
+        return v == kStatusBadLabel ? PCL_ERR_BAD_LABEL : PCL_ERR_DEVICE_TIMEOUT;
     }
     return PCL_OK;
 }
@@ -735,7 +779,7 @@ int pcl_profile_end(pcl_kernel_stat* stats, int max_stats, int* n_stats) {
     if (!stats || !n_stats || max_stats < 0) return PCL_ERR_BAD_ARG;
     std::lock_guard<std::mutex> lock(g_prof_mu);
     g_prof_on = false;
-    pcl_kernel_stat agg[KID_COUNT];
+    static pcl_kernel_stat agg[PROF_PASS_COUNT * KID_COUNT];
     memset(agg, 0, sizeof(agg));
     int rc = PCL_OK;
     for (const ProfEntry& e : g_prof_entries) {
@@ -744,16 +788,17 @@ int pcl_profile_end(pcl_kernel_stat* stats, int max_stats, int* n_stats) {
             rc = PCL_ERR_CUDA;
             break;
         }
-        agg[e.kid].launches += 1;
-        agg[e.kid].total_ms += ms;
-        agg[e.kid].work += e.work;
+        pcl_kernel_stat& a = agg[e.pass * KID_COUNT + e.kid];
+        a.launches += 1;
+        a.total_ms += ms;
+        a.work += e.work;
     }
     g_prof_entries.clear();
     g_prof_pool_used = 0;
     int n = 0;
-    for (int k = 0; k < KID_COUNT && n < max_stats; ++k) {
+    for (int k = 0; k < PROF_PASS_COUNT * KID_COUNT && n < max_stats; ++k) {
         if (agg[k].launches == 0) continue;
-        strncpy(agg[k].name, kKernelNames[k], sizeof(agg[k].name) - 1);
+        snprintf(agg[k].name, sizeof(agg[k].name), "%s/%s", kPassNames[k / KID_COUNT], kKernelNames[k % KID_COUNT]);
         stats[n++] = agg[k];
     }
     *n_stats = n;
@@ -770,6 +815,7 @@ const char* pcl_status_string(int status) {
         case PCL_ERR_CUDA: return "CUDA call failed";
         case PCL_ERR_DEVICE_TIMEOUT: return "device-side wait timed out";
         case PCL_ERR_SCRATCH_LIMIT: return "problem exceeds the capacity of the built-in scratch array";
+        case PCL_ERR_BAD_LABEL: return "a class label lies outside [0, K)";
     }
     return "unknown status";
 }

@@ -29,6 +29,23 @@ struct LaunchScope {
     cudaStream_t st;
 };
 
+// Tags the launches an ABI call makes with the pass they belong to (for the per-pass timing of pcl_profile_end) and
+// carries the layer's own algorithmic flops for its contraction launches.  Nested calls keep the outermost tag.
+enum ProfPass { PROF_PASS_OTHER = 0, PROF_PASS_CONV_FWD, PROF_PASS_CONV_BWD_DATA, PROF_PASS_CONV_BWD_WEIGHTS,
+                PROF_PASS_FC_FWD, PROF_PASS_FC_BWD, PROF_PASS_COUNT };
+struct PassScope {
+    PassScope(int pass, double flops);
+    ~PassScope();
+    PassScope(const PassScope&) = delete;
+    PassScope& operator=(const PassScope&) = delete;
+};
+double conv_pass_flops(const pcl_conv_desc& d, int P, int Q);
+// Mandatory part of the backward-data workspace: bytes of the transposed weight copy, 0 where none is made.
+size_t bwd_data_transposed_bytes(const pcl_conv_desc& d);
+
+// Device status word values that are not wait codes (those are 0x1xx, see pcl_ptx.cuh).
+constexpr unsigned int kStatusBadLabel = 0x201;     // pcl_softmax_xent met a label outside [0, K)
+
 // Address of the current device's status word (0 = fine, else the code of the
 // first bounded wait that ran out).  nullptr if the address cannot be obtained.
 unsigned int* device_status_ptr();

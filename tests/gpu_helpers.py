@@ -72,10 +72,27 @@ def run_conv_bwd_weights(s, x, dy, want_db, deterministic=True):
 # wrote.  `samples` > 0 checks that many randomly chosen output elements per
 # tensor (for sizes where the full oracle would take too long); 0 checks all.
 # ---------------------------------------------------------------------------
+def sample_indices(shape, samples, rng, edge=6):
+    """Flat indices of `samples` uniformly random elements plus stratified ones: for every dimension, `edge`
+    elements whose coordinate in that dimension lies in its last min(32, d) entries (the last image, the last tile
+    row / column, the last 32 output maps, the last k tile) and `edge` in its first min(8, d), the other
+    coordinates random -- a defect confined to a boundary tile cannot hide from these at any tensor size."""
+    shape = tuple(int(d) for d in shape)
+    size = int(np.prod(shape))
+    idx = [rng.choice(size, size=min(samples, size), replace=False).astype(np.int64)]
+    for j, dj in enumerate(shape):
+        for lo, hi in ((max(0, dj - 32), dj), (0, min(8, dj))):
+            coords = [rng.integers(0, d, size=edge) for d in shape]
+            coords[j] = rng.integers(lo, hi, size=edge)
+            idx.append(np.ravel_multi_index(coords, shape).astype(np.int64))
+    return np.unique(np.concatenate(idx))
+
+
 def _cmp(got_t, ref_fn, size, samples, rng, what, report):
     got = got_t.detach().cpu().numpy().reshape(-1)
     if samples and size > samples:
-        idx = np.sort(rng.choice(size, size=samples, replace=False)).astype(np.int64)
+        idx = sample_indices(got_t.shape, samples, rng) if got_t.numel() == size else \
+            np.sort(rng.choice(size, size=samples, replace=False)).astype(np.int64)
         ref = ref_fn(idx)
         g = got[idx]
     else:
@@ -96,7 +113,7 @@ def _check_pooled_only(net, i, s, xin, w, b, samples, rng, report):
     size = N * (P // 2) * (Q // 2) * K
     got_p = net.pooled[i].detach().cpu().numpy().reshape(-1)
     codes = net.pool_codes[i].detach().cpu().numpy().reshape(-1)
-    idx = (np.sort(rng.choice(size, size=samples, replace=False)).astype(np.int64) if samples and size > samples
+    idx = (sample_indices((N, P // 2, Q // 2, K), samples, rng) if samples and size > samples
            else np.arange(size, dtype=np.int64))
     k = idx % K; q2 = (idx // K) % (Q // 2); p2 = (idx // (K * (Q // 2))) % (P // 2); n = idx // (K * (Q // 2) * (P // 2))
     win = np.stack([((n * P + 2 * p2 + e // 2) * Q + 2 * q2 + e % 2) * K + k for e in range(4)], axis=1)   # [len][4]

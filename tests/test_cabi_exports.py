@@ -46,9 +46,10 @@ def test_host_side_checks(built_lib):
     assert L.pcl_conv_fwd(ctypes.byref(d), ctypes.c_void_p(16), ctypes.c_void_p(16), null, ctypes.c_void_p(16), 7,
                           null, 0, null) == B.ERR_BAD_ARG
     # a pass that needs workspace refuses a missing one before touching the device
-    big = B.conv_desc(8, 64, 64, 28, 28, 3, 3, 1, 1)
+    # (C % 32 != 0: backward-data makes a transposed copy of the weights, whose room is mandatory)
+    big = B.conv_desc(8, 40, 64, 28, 28, 3, 3, 1, 1)
     # (room for the transposed weights, plus scratch for a split reduction where the layer has few tiles)
-    assert B.conv_workspace_bytes(big, B.PASS_BWD_DATA) >= 64 * 64 * 9 * 4
+    assert B.conv_workspace_bytes(big, B.PASS_BWD_DATA) >= 40 * 64 * 9 * 4
     wide = B.conv_desc(256, 256, 256, 56, 56, 3, 3, 1, 1)      # thousands of tiles: no split, the weights' room only
     assert B.conv_workspace_bytes(wide, B.PASS_BWD_DATA) == 256 * 256 * 9 * 4
     assert B.conv_workspace_bytes(wide, B.PASS_FWD) == 0

@@ -148,6 +148,32 @@ def test_softmax_xent(N, K):
     np.testing.assert_allclose(dz.cpu().numpy(), dz_ref, rtol=1e-4, atol=1e-8)
 
 
+def test_softmax_xent_label_outside_the_classes_is_reported_and_never_used_as_an_index():
+    """A label outside [0, K) must not become an address: the row gets no target and no loss term, and the status
+    call reports it once."""
+    import gpu_helpers as G
+    from paper_1602_06709_b200 import binding as B
+    from paper_1602_06709_b200 import inputs
+    N, K = 6, 40
+    z = inputs.normal(inputs.tensor_id("xent_bad", N, K, "z"), (N, K), 2.0)
+    lab = np.array([3, -1, K, 17, K + 1000, 0], dtype=np.int32)
+    good = (lab >= 0) & (lab < K)
+    zt = G.dev(z); lt = torch.from_numpy(lab).cuda()
+    loss = torch.full((1,), float("nan"), device="cuda")
+    dz = torch.full((N, K), float("nan"), device="cuda")
+    assert B.last_device_status() == B.OK
+    B.softmax_xent(N, K, zt, lt, loss, dz)
+    assert B.last_device_status() == B.ERR_BAD_LABEL
+    assert B.last_device_status() == B.OK                      # reported once, then cleared
+    loss_ref, dz_ref = oracle.softmax_xent(z, np.where(good, lab, 0))
+    zs = z.astype(np.float64) - z.max(axis=1, keepdims=True)
+    sm = np.exp(zs) / np.exp(zs).sum(axis=1, keepdims=True)
+    dz_ref[~good] = sm[~good] / N                              # no one-hot on the rows without a target
+    terms = -(zs[np.arange(N), np.where(good, lab, 0)] - np.log(np.exp(zs).sum(axis=1)))
+    np.testing.assert_allclose(dz.cpu().numpy(), dz_ref, rtol=1e-4, atol=1e-8)
+    assert abs(loss.item() - terms[good].sum() / N) <= 1e-5
+
+
 @pytest.mark.parametrize("N,H,W,C", [(2, 8, 6, 8), (3, 14, 14, 20), (2, 28, 28, 64), (1, 4, 4, 1024)])
 def test_maxpool_bwd_with_fused_column_sums(N, H, W, C):
     import gpu_helpers as G

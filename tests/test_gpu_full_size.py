@@ -1,7 +1,9 @@
 """GPU parity at the full workload sizes, in the launch configuration the
 benchmark times.  The oracle cannot produce whole tensors at these sizes in
-seconds, so each output tensor is checked on randomly sampled elements the
-oracle computes one by one, plus properties that hold at any size (bitwise
+seconds, so each output tensor is checked on sampled elements the oracle
+computes one by one (uniformly random ones plus, for every dimension, elements
+from its first and last entries: boundary tiles, the last image, the last
+output maps), plus properties that hold at any size (bitwise
 reproducibility of the two-pass weight gradient)."""
 import numpy as np
 import pytest
@@ -28,7 +30,7 @@ def _sampled_three_passes(s, cfg, layer, samples=SAMPLES, skip_bwd_data=False):
 
     def check(t, ref_fn, what):
         flat = t.reshape(-1)
-        idx = np.sort(rng.choice(flat.numel(), size=min(samples, flat.numel()), replace=False)).astype(np.int64)
+        idx = G.sample_indices(t.shape, samples, rng)       # random + first / last entries of every dimension
         got = flat[torch.from_numpy(idx).cuda()].cpu().numpy()
         G.assert_parity(got, ref_fn(idx), f"{layer} {what}")
 

@@ -39,11 +39,35 @@ def test_noalloc_matches_regular_entry_point_twice():
         G.assert_parity(ref.cpu().numpy(), oracle.conv_bwd_data(s, dy, w, x), "bwd_data (no-alloc)")
 
 
+def test_noalloc_capacity_counts_only_the_transposed_copy():
+    """What must fit the built-in array is the transposed weight copy.  A wide layer whose weights are read in
+    place (C % 32 == 0) needs none and runs although the regular call's full workspace (copy area + room to split
+    the reduction) would not fit; a layer with C % 32 != 0 just under the limit runs too.  Both bit-equal to the
+    regular entry point given exactly the same amount of scratch."""
+    import gpu_helpers as G
+    from paper_1602_06709_b200 import binding as B
+    B.set_path(B.PATH_AUTO)
+    cap = B.noalloc_scratch_bytes()
+    for s in (ConvShape(N=4, C=512, K=512, H=14, W=14, R=3, S=3, pad_h=1, pad_w=1),
+              ConvShape(N=2, C=904, K=512, H=6, W=6, R=3, S=3, pad_h=1, pad_w=1)):     # 4.17 M of 4.19 M weights
+        d = G.shape_to_desc(s)
+        x, w, dy, _ = G.make_inputs(s, f"noalloc_cap{s.C}")
+        dyt, wt = G.dev(dy), G.dev(w)
+        ref = torch.full((s.N, s.H, s.W, s.C), float("nan"), device="cuda")
+        B.conv_bwd_data(d, dyt, wt, None, ref, torch.empty(cap, dtype=torch.uint8, device="cuda"))
+        for rep in range(2):
+            got = torch.full_like(ref, float("nan"))
+            B.conv_bwd_data_noalloc(d, dyt, wt, None, got)
+            B.check_device_status()
+            assert torch.equal(got, ref), f"C={s.C} call {rep}: differs from pcl_conv_bwd_data with the same scratch"
+        G.assert_parity(ref.cpu().numpy(), oracle.conv_bwd_data(s, dy, w), f"bwd_data (no-alloc, C={s.C})")
+
+
 def test_noalloc_rejects_layers_beyond_its_capacity():
     import ctypes
     from paper_1602_06709_b200 import binding as B
     assert B.noalloc_scratch_bytes() == 16 << 20
-    big = B.conv_desc(1, 2048, 2048, 4, 4, 3, 3, 1, 1)       # 37.7 M weights > 4 Mi floats
+    big = B.conv_desc(1, 2040, 2048, 4, 4, 3, 3, 1, 1)       # C % 32 != 0: needs a copy of 37.6 M weights > 4 Mi floats
     assert B.conv_workspace_bytes(big, B.PASS_BWD_DATA) > B.noalloc_scratch_bytes()
     null = ctypes.c_void_p(0)
     rc = B.lib().pcl_conv_bwd_data_noalloc(ctypes.byref(big), ctypes.c_void_p(256), ctypes.c_void_p(256), null,
