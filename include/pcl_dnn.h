@@ -68,6 +68,18 @@ enum { PCL_PASS_FWD = 0, PCL_PASS_BWD_DATA = 1, PCL_PASS_BWD_WEIGHTS = 2 };
 enum { PCL_PATH_AUTO = 0, PCL_PATH_TENSOR = 1, PCL_PATH_GENERIC = 2 };
 int pcl_set_path(int path);
 
+/* Test and tuning knobs (the paper has no counterpart).  Every choice the launchers make -- tiling,
+ * tile width, k-steps per pipeline slot, CTA pairs, issuing threads, epilogue form, reduction splits --
+ * has a named knob with which the tests pin each kernel variant and the alternatives were measured:
+ * TILING (0 plain, 1-3 haloed layouts), BN, KS, KS_HALO, KS_WGRAD, PAIR, PAIR_HALO, PAIR_WGRAD, GRP,
+ * ISSUERS, SPLIT_ACC, PIX_WGRAD, XHALO_WGRAD, TMA_STORE, WEIGHTS_IN_PLACE, EPI_WARPS, FC_DW_FORWARD,
+ * KSPLIT, WAIT_LIMIT_US (limit of the bounded device-side waits, microseconds), FAULT_INJECT (test
+ * only, see pcl_last_device_status).  value INT_MIN unsets a knob; pcl_reset_tuning() unsets all.
+ * Unset knobs take the launchers' own rules.  Process-wide; nothing is ever read from the environment.
+ * Returns PCL_ERR_BAD_ARG for an unknown name. */
+int pcl_set_tuning(const char* name, int value);
+int pcl_reset_tuning(void);
+
 /* Output spatial size of a convolution.  Returns PCL_ERR_BAD_ARG if the
  * kernel does not fit in the padded input. */
 int pcl_conv_out_dims(const pcl_conv_desc* d, int* P, int* Q);

@@ -30,7 +30,7 @@ EXPORTS = [
     "pcl_conv_bwd_data_colsum_workspace_bytes", "pcl_conv_bwd_data_colsum",
     "pcl_maxpool2x2_bwd_colsum_workspace_bytes", "pcl_maxpool2x2_bwd_colsum", "pcl_conv_fwd_pool", "pcl_conv_fwd_pool_is_fused",
     "pcl_conv_bwd_weights_pooled", "pcl_conv_bwd_weights_pooled_is_fused", "pcl_conv_bwd_weights_pooled_workspace_bytes",
-    "pcl_maxpool2x2_fwd_codes", "pcl_maxpool2x2_bwd_codes", "pcl_last_wait_code",
+    "pcl_maxpool2x2_fwd_codes", "pcl_maxpool2x2_bwd_codes", "pcl_last_wait_code", "pcl_set_tuning", "pcl_reset_tuning",
 ]
 
 
@@ -64,6 +64,7 @@ def lib() -> ctypes.CDLL:
         vp, sz, ci, cf = ctypes.c_void_p, ctypes.c_size_t, ctypes.c_int, ctypes.c_float
         dp = ctypes.POINTER(ConvDesc)
         L.pcl_set_path.argtypes = [ci]
+        L.pcl_set_tuning.argtypes = [ctypes.c_char_p, ci]
         L.pcl_conv_out_dims.argtypes = [dp, ctypes.POINTER(ci), ctypes.POINTER(ci)]
         L.pcl_conv_workspace_bytes.argtypes = [dp, ci]
         L.pcl_conv_workspace_bytes.restype = sz
@@ -128,6 +129,24 @@ def _stream(stream=None):
 def conv_desc(N, C, K, H, W, R, S, stride=1, pad=0, stride_w=None, pad_w=None) -> ConvDesc:
     return ConvDesc(N, C, K, H, W, R, S, stride, stride if stride_w is None else stride_w,
                     pad, pad if pad_w is None else pad_w)
+
+
+TILINGS = {"plain": 0, "halo0": 1, "halo1": 2, "halo2": 3}
+UNSET = -2 ** 31
+
+
+def set_tuning(name: str, value):
+    """Pins one of the launchers' choices (see pcl_set_tuning in the header).  value None unsets the knob; the
+    TILING knob also takes the names plain / halo0 / halo1 / halo2."""
+    if value is None:
+        value = UNSET
+    elif name == "TILING" and isinstance(value, str):
+        value = TILINGS[value]
+    _check(lib().pcl_set_tuning(name.encode(), int(value)), f"pcl_set_tuning({name})")
+
+
+def reset_tuning():
+    _check(lib().pcl_reset_tuning(), "pcl_reset_tuning")
 
 
 def set_path(path: int):

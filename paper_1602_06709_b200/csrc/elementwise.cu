@@ -12,7 +12,7 @@ namespace {
 
 int grid_for(size_t work_items, int block, int per_sm = 8) {
     size_t blocks = (work_items + block - 1) / block;
-    const size_t cap = size_t(148) * per_sm;
+    const size_t cap = size_t(device_sm_count()) * per_sm;
     if (blocks > cap) blocks = cap;
     if (blocks < 1) blocks = 1;
     return int(blocks);
@@ -660,7 +660,7 @@ int launch_softmax_xent(int N, int K, const float* logits, const int* labels, fl
         LaunchScope scope(KID_SOFTMAX_XENT, 8.0 * double(N) * K, st);
         unsigned int* status = device_status_ptr();
         if (!status) return PCL_ERR_CUDA;
-        softmax_xent_kernel<<<N < 1184 ? N : 1184, 256, 0, st>>>(logits, labels, loss, dlogits, N, K, status);
+        softmax_xent_kernel<<<N < 8 * device_sm_count() ? N : 8 * device_sm_count(), 256, 0, st>>>(logits, labels, loss, dlogits, N, K, status);
     }
     return PCL_CHECK_LAUNCH();
 }

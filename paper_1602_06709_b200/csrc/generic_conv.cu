@@ -179,7 +179,7 @@ int launch_generic_bwd_data(const pcl_conv_desc& d, int P, int Q, const float* d
 int generic_wgrad_splits(const pcl_conv_desc& d, int P, int Q) {
     const long tiles = long((d.K + BM - 1) / BM) * ((long(d.R) * d.S * d.C + BN - 1) / BN);
     const long depth = long(d.N) * P * Q;
-    long splits = (4 * 148 + tiles - 1) / tiles;
+    long splits = (4 * device_sm_count() + tiles - 1) / tiles;
     const long max_by_depth = (depth + 255) / 256;
     if (splits > max_by_depth) splits = max_by_depth;
     if (splits > 256) splits = 256;

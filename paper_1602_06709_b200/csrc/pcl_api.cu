@@ -3,6 +3,7 @@
 // the caller's stream.
 #include <atomic>
 #include <mutex>
+#include <limits.h>
 #include <stdio.h>
 #include <string.h>
 #include <vector>
@@ -30,6 +31,33 @@ unsigned int* device_status_ptr() {
 }
 
 static std::atomic<unsigned long long> g_launches{0};
+
+namespace {
+struct TuneSlot { std::atomic<int> set{0}; std::atomic<int> value{0}; };
+TuneSlot g_tune[TUNE_COUNT];
+std::atomic<unsigned> g_tune_gen{0};
+const char* const kTuneNames[TUNE_COUNT] = {
+    "TILING", "BN", "KS", "KS_HALO", "KS_WGRAD", "PAIR", "PAIR_HALO", "PAIR_WGRAD", "GRP", "ISSUERS", "SPLIT_ACC",
+    "PIX_WGRAD", "XHALO_WGRAD", "TMA_STORE", "WEIGHTS_IN_PLACE", "EPI_WARPS", "FC_DW_FORWARD", "KSPLIT",
+    "WAIT_LIMIT_US", "FAULT_INJECT"};
+}  // namespace
+
+int tune(int id, int dflt) {
+    return g_tune[id].set.load(std::memory_order_relaxed) ? g_tune[id].value.load(std::memory_order_relaxed) : dflt;
+}
+bool tune_is_set(int id) { return g_tune[id].set.load(std::memory_order_relaxed) != 0; }
+unsigned tune_generation() { return g_tune_gen.load(std::memory_order_relaxed); }
+
+int device_sm_count() {
+    static std::atomic<int> cache[64] = {};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 148;
+    int n = cache[dev].load(std::memory_order_relaxed);
+    if (n > 0) return n;
+    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) return 148;
+    cache[dev].store(n, std::memory_order_relaxed);
+    return n;
+}
 
 namespace {
 struct ProfEntry { int kid; int pass; double work; cudaEvent_t e0, e1; };
@@ -138,11 +166,8 @@ bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 
 
 // Backward-data on the tensor-core path reads the KRSC weights in place (as an MN-major operand) when the layer's
 // input-map count is a multiple of 32; otherwise it goes through a flipped, transposed copy in the workspace.
-// PCL_WEIGHTS_IN_PLACE=0 forces the copy (test hook).
-bool weights_read_in_place(const pcl_conv_desc& d) {
-    const char* v = getenv("PCL_WEIGHTS_IN_PLACE");
-    return d.C % 32 == 0 && !(v && v[0] == '0');
-}
+// The WEIGHTS_IN_PLACE knob set to 0 forces the copy (test hook).
+bool weights_read_in_place(const pcl_conv_desc& d) { return d.C % 32 == 0 && tune(TUNE_WEIGHTS_IN_PLACE, 1) != 0; }
 
 size_t dw_bytes(const pcl_conv_desc& d);
 }  // namespace
@@ -237,7 +262,7 @@ WgradPlan plan_wgrad(const pcl_conv_desc& d, int P, int Q) {
 bool fc_dw_as_forward(int N, int C, int K) {
     if (g_path.load() == PCL_PATH_GENERIC) return false;
     if (N % 4 != 0 || C % 32 != 0 || K % 4 != 0) return false;
-    if (const char* v = getenv("PCL_FC_DW_FORWARD")) return atoi(v) != 0;      // test / tuning hook
+    if (tune_is_set(TUNE_FC_DW_FORWARD)) return tune(TUNE_FC_DW_FORWARD, 0) != 0;      // test / tuning hook
     // measured (B200): it pays for a short reduction and a large dw (VGG-A FC1: 0.26 -> 0.13 ms, FC2: 0.052 -> 0.039
     // with the transpose); at minibatch 1024 (the DNN layers) and for small dw the weight-gradient kernel is as fast
     return N <= 512 && size_t(K) * C >= (size_t(1) << 23);
@@ -250,6 +275,24 @@ size_t fc_dzt_bytes(int N, int K) { return align_up(size_t(N) * K * 4, 256); }
 using namespace pcl;
 
 extern "C" {
+
+int pcl_set_tuning(const char* name, int value) {
+    if (!name) return PCL_ERR_BAD_ARG;
+    for (int i = 0; i < TUNE_COUNT; ++i)
+        if (strcmp(name, kTuneNames[i]) == 0) {
+            g_tune[i].value.store(value);
+            g_tune[i].set.store(value == INT_MIN ? 0 : 1);
+            g_tune_gen.fetch_add(1);
+            return PCL_OK;
+        }
+    return PCL_ERR_BAD_ARG;
+}
+
+int pcl_reset_tuning(void) {
+    for (int i = 0; i < TUNE_COUNT; ++i) g_tune[i].set.store(0);
+    g_tune_gen.fetch_add(1);
+    return PCL_OK;
+}
 
 int pcl_set_path(int path) {
     if (path != PCL_PATH_AUTO && path != PCL_PATH_TENSOR && path != PCL_PATH_GENERIC) return PCL_ERR_BAD_ARG;

@@ -5,6 +5,9 @@
 #include <stddef.h>
 #include <stdint.h>
 
+#include <atomic>
+#include <mutex>
+
 #include "../../include/pcl_dnn.h"
 
 namespace pcl {
@@ -42,6 +45,42 @@ struct PassScope {
 double conv_pass_flops(const pcl_conv_desc& d, int P, int Q);
 // Mandatory part of the backward-data workspace: bytes of the transposed weight copy, 0 where none is made.
 size_t bwd_data_transposed_bytes(const pcl_conv_desc& d);
+
+// Test / tuning knobs: every choice the launchers make has one, so that the tests can pin each pipeline variant and
+// the alternatives can be measured.  They are set through pcl_set_tuning() only (never read from the environment:
+// a stray variable must not change which kernel a production call runs); tune() returns the knob's value, or
+// `dflt` while it is unset.
+enum TuneId {
+    TUNE_TILING = 0,        // forward-type kernel: 0 plain, 1-3 haloed layouts 0-2
+    TUNE_BN, TUNE_KS, TUNE_KS_HALO, TUNE_KS_WGRAD, TUNE_PAIR, TUNE_PAIR_HALO, TUNE_PAIR_WGRAD, TUNE_GRP, TUNE_ISSUERS,
+    TUNE_SPLIT_ACC, TUNE_PIX_WGRAD, TUNE_XHALO_WGRAD, TUNE_TMA_STORE, TUNE_WEIGHTS_IN_PLACE, TUNE_EPI_WARPS,
+    TUNE_FC_DW_FORWARD, TUNE_KSPLIT, TUNE_WAIT_LIMIT_US, TUNE_FAULT_INJECT, TUNE_COUNT
+};
+int tune(int id, int dflt);
+bool tune_is_set(int id);
+unsigned tune_generation();      // bumped by every pcl_set_tuning / pcl_reset_tuning (cached launch plans key on it)
+
+// SM count of the current device (cached per device, thread-safe).  Without a usable device (a sizing query on a
+// machine that has none) the B200's 148 is returned: a launch would fail there anyway.
+int device_sm_count();
+// Runs `setup` once per device (thread-safe) and remembers its success; used for cudaFuncSetAttribute, which
+// applies to the current device only.
+struct PerDeviceOnce {
+    template <class F>
+    int run(F&& setup) {
+        int dev = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return PCL_ERR_CUDA;
+        if (done_[dev].load(std::memory_order_acquire)) return PCL_OK;
+        std::lock_guard<std::mutex> lock(mu_);
+        if (done_[dev].load(std::memory_order_relaxed)) return PCL_OK;
+        const int rc = setup();
+        if (rc == PCL_OK) done_[dev].store(true, std::memory_order_release);
+        return rc;
+    }
+  private:
+    std::mutex mu_;
+    std::atomic<bool> done_[64] = {};
+};
 
 // Device status word values that are not wait codes (those are 0x1xx, see pcl_ptx.cuh).
 constexpr unsigned int kStatusBadLabel = 0x201;     // pcl_softmax_xent met a label outside [0, K)

@@ -908,8 +908,8 @@ void choose_box(int P, int Q, int N, bool pool, int* bw_log2, int* bh_log2) {
 }
 
 int choose_bn(int Kout, long m_tiles, int sm_count) {
-    if (const char* v = getenv("PCL_BN")) {          // tuning hook: a multiple of 32 in [32, 256]
-        const int bn = atoi(v);
+    if (tune_is_set(TUNE_BN)) {          // tuning hook: a multiple of 32 in [32, 256]
+        const int bn = tune(TUNE_BN, 0);
         if (bn >= 32 && bn <= 256 && bn % 32 == 0) return bn;
     }
     // Score = (fraction of SM-slots the tiles fill, counting whole waves) x (tensor efficiency of the width):
@@ -935,8 +935,6 @@ int choose_bn(int Kout, long m_tiles, int sm_count) {
     return best;
 }
 
-int g_sm_count = 0;
-
 }  // namespace
 
 bool tc_fprop_can_pool(const TcFpropArgs& a) {
@@ -955,10 +953,6 @@ namespace {
 
 // One way of tiling a layer: plain (a box of 128 pixels, one TMA box per tap) or halo (MT boxes of 8 x 16
 // pixels cut from one haloed patch per channel block).
-int env_int(const char* name, int dflt) {       // test / tuning hook
-    const char* v = getenv(name);
-    return v ? atoi(v) : dflt;
-}
 
 struct TileCfg {
     bool ok = false;
@@ -981,15 +975,15 @@ TileCfg plain_cfg(const TcFpropArgs& a, int cblocks, int sm_count) {
     // narrow tiles: several k-steps per slot (see the kernel), as long as 4 slots still fit
     // pairs pay where operand traffic or the issue rate of wide MMAs bounds the tile; narrow tiles are bound by
     // the issuing thread and run as single CTAs with two issuers instead
-    c.pair = env_int("PCL_PAIR", 1) && c.BN >= 128 && c.tiles_n >= 2 && sm_count >= 2 &&
+    c.pair = tune(TUNE_PAIR, 1) && c.BN >= 128 && c.tiles_n >= 2 && sm_count >= 2 &&
              (!a.wt_mn_major || c.BN % 64 == 0);        // MN-major weights are fetched in whole 32-map groups per CTA
     const int step_bytes = kABytes + (c.pair ? c.BN * 64 : c.BN * 128);
-    c.KS = env_int("PCL_KS", 2);
+    c.KS = tune(TUNE_KS, 2);
     const int kiters = a.R * a.S * cblocks;
     if (c.KS > kiters) c.KS = kiters;
     while (c.KS > 1 && (kSmemBudget - kEpiStageBytes) / (c.KS * step_bytes) < 3) --c.KS;
     c.stages = (kSmemBudget - kEpiStageBytes) / (c.KS * step_bytes);
-    c.grp = env_int("PCL_GRP", 1) && c.KS > 1 && a.Cin % kBlockC == 0 && cblocks % c.KS == 0 && a.in_inner == 0;
+    c.grp = tune(TUNE_GRP, 1) && c.KS > 1 && a.Cin % kBlockC == 0 && cblocks % c.KS == 0 && a.in_inner == 0;
     if (c.stages > kMaxStages) c.stages = kMaxStages;
     c.ok = c.stages >= 2;
     return c;
@@ -1013,14 +1007,14 @@ TileCfg halo_cfg(const TcFpropArgs& a, int cblocks, int sm_count, int layout) {
     c.BN = choose_bn(a.Kout, m_tiles, sm_count);
     if (2 * c.MT * c.BN > 512) return c;          // two accumulator sets must fit the 512 TMEM columns
     c.tiles_k = (a.Kout + c.BN - 1) / c.BN;
-    c.pair = env_int("PCL_PAIR_HALO", 0) && c.tiles_n >= 2 && sm_count >= 2;      // pairs of images (no gain measured)
+    c.pair = tune(TUNE_PAIR_HALO, 0) && c.tiles_n >= 2 && sm_count >= 2;      // pairs of images (no gain measured)
     const int b_bytes = c.pair ? c.BN * 64 : c.BN * 128;
     const int room = kSmemBudget - kEpiStageBytes;
     c.NA = 2;
-    c.KS = env_int("PCL_KS_HALO", c.BN <= 64 ? 3 : (c.BN <= 128 ? 2 : 1));
+    c.KS = tune(TUNE_KS_HALO, c.BN <= 64 ? 3 : (c.BN <= 128 ? 2 : 1));
     if (c.KS > a.R * a.S) c.KS = a.R * a.S;
     while (c.KS > 1 && (room - c.NA * c.a_buf_bytes) / (c.KS * b_bytes) < 3) --c.KS;
-    c.grp = env_int("PCL_GRP", 1) && c.KS > 1 && !a.wt_mn_major;      // (MN-major weights: one copy per tap)
+    c.grp = tune(TUNE_GRP, 1) && c.KS > 1 && !a.wt_mn_major;      // (MN-major weights: one copy per tap)
     const int slot = c.KS * b_bytes;
     c.stages = (room - c.NA * c.a_buf_bytes) / slot;
     if (c.stages >= 9 && (room - 3 * c.a_buf_bytes) / slot >= 6) {
@@ -1038,9 +1032,9 @@ TileCfg select_cfg(const TcFpropArgs& a, int sm_count) {
     const int cblocks = (a.Cin + kBlockC - 1) / kBlockC;
     TileCfg cfg = plain_cfg(a, cblocks, sm_count);
     if (!cfg.ok) return cfg;
-    // Test hook: PCL_TILING = plain | halo0 | halo1 | halo2 pins the tiling (when that tiling is possible).
-    const char* pin = getenv("PCL_TILING");
-    const int pinned = !pin ? -2 : (pin[0] == 'p' ? -1 : (pin[0] == 'h' && pin[4] >= '0' && pin[4] <= '2' ? pin[4] - '0' : -2));
+    // Test hook: the TILING knob pins the tiling (when that tiling is possible).
+    const int pin = tune(TUNE_TILING, -1);       // unset: the rule below; 0: plain; 1-3: haloed layout 0-2
+    const int pinned = pin < 0 || pin > 3 ? -2 : pin - 1;
     for (int layout = 0; layout < 3; ++layout) {
         const TileCfg h = halo_cfg(a, cblocks, sm_count, layout);
         if (!h.ok) continue;
@@ -1055,23 +1049,8 @@ TileCfg select_cfg(const TcFpropArgs& a, int sm_count) {
 
 }  // namespace
 
-static int ensure_device_setup() {
-    if (g_sm_count == 0) {
-        int dev = 0;
-        if (cudaGetDevice(&dev) != cudaSuccess) return PCL_ERR_CUDA;
-        if (cudaDeviceGetAttribute(&g_sm_count, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return PCL_ERR_CUDA;
-    }
-    return PCL_OK;
-}
-
 long tc_fprop_colsum_rows(const TcFpropArgs& a) {
-    int sm = g_sm_count;
-    if (sm == 0) {      // sizing query before any launch (possibly without a device): use the B200 SM count
-        int dev = 0;
-        if (cudaGetDevice(&dev) != cudaSuccess ||
-            cudaDeviceGetAttribute(&sm, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sm <= 0)
-            sm = 148;
-    }
+    const int sm = device_sm_count();
     if (a.Kout % 4 != 0) return 0;
     // rows are independent of BN, but the haloed / plain choice depends on it: take the larger of all tilings
     long rows = 0;
@@ -1091,7 +1070,7 @@ namespace {
 // as many as fill the SMs, each an equal whole number of pipeline slots (at least two).
 int choose_ksplit(const TcFpropArgs& a, const TileCfg& cfg, int cblocks, int sm_count) {
     if (cfg.halo || a.mask_src || a.colsum_rows || a.pool_out || !a.out || a.Kout % 4 != 0) return 1;
-    const int hook = env_int("PCL_KSPLIT", 0);              // test hook: 1 = never, n = n splits where they divide
+    const int hook = tune(TUNE_KSPLIT, 0);              // test hook: 1 = never, n = n splits where they divide
     if (hook == 1) return 1;
     const long tiles = long(cfg.tiles_q) * cfg.tiles_p * cfg.tiles_n * cfg.tiles_k;        // CTAs (a pair is two)
     const int kiters = a.R * a.S * cblocks;
@@ -1110,13 +1089,7 @@ int choose_ksplit(const TcFpropArgs& a, const TileCfg& cfg, int cblocks, int sm_
 }  // namespace
 
 size_t tc_fprop_split_ws_bytes(const TcFpropArgs& a) {
-    int sm = g_sm_count;
-    if (sm == 0) {
-        int dev = 0;
-        if (cudaGetDevice(&dev) != cudaSuccess ||
-            cudaDeviceGetAttribute(&sm, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sm <= 0)
-            sm = 148;
-    }
+    const int sm = device_sm_count();
     if (!tc_fprop_eligible(a)) return 0;
     const TileCfg cfg = select_cfg(a, sm);
     if (!cfg.ok) return 0;
@@ -1128,9 +1101,8 @@ size_t tc_fprop_split_ws_bytes(const TcFpropArgs& a) {
 
 int launch_tc_fprop(const TcFpropArgs& a, cudaStream_t st) {
     if (!tc_fprop_eligible(a)) return PCL_ERR_UNSUPPORTED_SHAPE;
-    static bool attr_set = false;
-    if (!attr_set) {
-        if (ensure_device_setup() != PCL_OK) return PCL_ERR_CUDA;
+    static PerDeviceOnce attr_once;       // (the attribute applies to the current device only)
+    const int setup_rc = attr_once.run([]() -> int {
         const void* kernels[8] = {
             (const void*)tc_fprop_kernel<false, false, false>, (const void*)tc_fprop_kernel<false, true, false>,
             (const void*)tc_fprop_kernel<false, false, true>,  (const void*)tc_fprop_kernel<true, false, false>,
@@ -1140,8 +1112,10 @@ int launch_tc_fprop(const TcFpropArgs& a, cudaStream_t st) {
         for (const void* k : kernels)
             if (cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget + 1024) != cudaSuccess)
                 return PCL_ERR_CUDA;
-        attr_set = true;
-    }
+        return PCL_OK;
+    });
+    if (setup_rc != PCL_OK) return setup_rc;
+    const int g_sm_count = device_sm_count();
     FpropParams p{};
     p.cblocks = (a.Cin + kBlockC - 1) / kBlockC;
     const TileCfg cfg = select_cfg(a, g_sm_count);
@@ -1159,7 +1133,7 @@ int launch_tc_fprop(const TcFpropArgs& a, cudaStream_t st) {
     // tiles of a few k-steps (the few-channel first layer: 3).
     const int slots_per_tile = cfg.halo ? p.cblocks * ((a.R * a.S + cfg.KS - 1) / cfg.KS)
                                         : (a.R * a.S * p.cblocks + cfg.KS - 1) / cfg.KS;
-    p.issuers = (!cfg.pair && slots_per_tile >= 8 && env_int("PCL_ISSUERS", 2) >= 2) ? 2 : 1;
+    p.issuers = (!cfg.pair && slots_per_tile >= 8 && tune(TUNE_ISSUERS, 2) >= 2) ? 2 : 1;
     const int bw = 1 << p.bw_log2, bh = 1 << p.bh_log2, bn = kTileM / (bw * bh);
     const long m_tiles = long(p.tiles_q) * p.tiles_p * p.tiles_n;
     if (m_tiles * p.tiles_k > 0x7fffffffL) return PCL_ERR_UNSUPPORTED_SHAPE;
@@ -1167,7 +1141,7 @@ int launch_tc_fprop(const TcFpropArgs& a, cudaStream_t st) {
     p.N = a.N; p.P = a.P; p.Q = a.Q; p.Kout = a.Kout;
     p.act = a.act;
     // (not in the pooling instantiation: its epilogue has no registers to spare)
-    p.split_acc = (p.issuers == 2 && 4 * p.MT * p.BN <= 512 && !a.pool_out && env_int("PCL_SPLIT_ACC", 1)) ? 1 : 0;
+    p.split_acc = (p.issuers == 2 && 4 * p.MT * p.BN <= 512 && !a.pool_out && tune(TUNE_SPLIT_ACC, 1)) ? 1 : 0;
     p.tmem_cols = 32;
     while (p.tmem_cols < (p.split_acc ? 4 : 2) * p.MT * p.BN) p.tmem_cols *= 2;
     p.bias = a.bias; p.mask_src = a.mask_src; p.out = a.out;
@@ -1252,7 +1226,7 @@ int launch_tc_fprop(const TcFpropArgs& a, cudaStream_t st) {
         // tile and stores nothing at full resolution
         if (!a.pool_out || a.colsum_rows) return PCL_ERR_BAD_ARG;
         p.tma_store = 1;
-    } else if (env_int("PCL_TMA_STORE", 1) && !a.mask_src && !a.colsum_rows && a.Kout % 4 == 0 &&
+    } else if (tune(TUNE_TMA_STORE, 1) && !a.mask_src && !a.colsum_rows && a.Kout % 4 == 0 &&
         (reinterpret_cast<uintptr_t>(a.out) & 15) == 0) {
         const uint32_t bx = bw < 32 ? bw : 32, by = uint32_t(bh) < 32 / bx ? uint32_t(bh) : 32 / bx, bnn = 32 / (bx * by);
         const uint64_t dims[4] = {uint64_t(a.Kout), uint64_t(a.Q), uint64_t(a.P), uint64_t(a.N)};
@@ -1265,7 +1239,7 @@ int launch_tc_fprop(const TcFpropArgs& a, cudaStream_t st) {
     // BN <= 64 columns takes ~50 cycles, wider ones BN/2) against ~1600 cycles per 32-column chunk and warp.  Their
     // staging tiles take 32 KB more; the ring gives up slots for them as long as three remain.
     bool wide_epi = false;
-    const int epi_hook = env_int("PCL_EPI_WARPS", 16);      // test hook: 8 = never, 32 = wherever the variant can run
+    const int epi_hook = tune(TUNE_EPI_WARPS, 16);      // test hook: 8 = never, 32 = wherever the variant can run
     if (!cfg.pair && p.tma_store && !p.split_acc && epi_hook >= 16) {
         const long mma_clk = long(a.R) * a.S * p.cblocks * 4 * (p.BN <= 64 ? 50 : p.BN / 2);
         const long epi_clk = long(p.BN / 32) * 1600 / 2;
@@ -1289,14 +1263,19 @@ int launch_tc_fprop(const TcFpropArgs& a, cudaStream_t st) {
         lc.blockDim = dim3(kThreads); lc.dynamicSmemBytes = smem; lc.stream = st;
         lc.attrs = attr; lc.numAttrs = 1;
         // how many pairs the device holds at once with this much shared memory (cached per size)
+        static std::mutex cache_mu;
         static size_t cached_smem = 0;
-        static int cached_clusters = 0;
-        if (cached_smem != smem) {
+        static int cached_clusters = 0, cached_dev = -1;
+        int cur_dev = 0;
+        if (cudaGetDevice(&cur_dev) != cudaSuccess) return PCL_ERR_CUDA;
+        std::lock_guard<std::mutex> cache_lock(cache_mu);
+        if (cached_smem != smem || cached_dev != cur_dev) {
             lc.gridDim = dim3(unsigned(g_sm_count / 2 * 2));
             int n = 0;
             if (cudaOccupancyMaxActiveClusters(&n, tc_fprop_kernel<true, false, false>, &lc) != cudaSuccess || n <= 0) return PCL_ERR_CUDA;
             cached_clusters = n < g_sm_count / 2 ? n : g_sm_count / 2;
             cached_smem = smem;
+            cached_dev = cur_dev;
         }
         const long pair_tiles = long(p.tiles_q) * p.tiles_p * p.tiles_n * p.tiles_k * p.ksplit;
         long nclus = pair_tiles < cached_clusters ? pair_tiles : cached_clusters;

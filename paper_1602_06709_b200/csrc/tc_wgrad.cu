@@ -571,11 +571,6 @@ void choose_pixel_box(int pix, int P, int Q, int N, int* bw_log2, int* bh_log2, 
     *bh_log2 = best_h;
 }
 
-int env_int(const char* name, int dflt) {       // test / tuning hook
-    const char* v = getenv(name);
-    return v ? atoi(v) : dflt;
-}
-
 // How a layer is cut into work items and k-steps.
 struct WgradPlan {
     int grouped, L, runs_per_tap, total_runs, rpi, run_blocks;
@@ -592,7 +587,7 @@ WgradPlan plan_wgrad(int N, int P, int Q, int C, int K, int R, int S, int tap_gr
     const int cgroups = (C + 31) / 32;
     const int k_tiles = (K + 127) / 128;
     r.grouped = (!tap_groups && C % 32 == 0 && K % 32 == 0) ? 1 : 0;
-    r.pair = env_int("PCL_PAIR_WGRAD", 1) && r.grouped && k_tiles % 2 == 0 && !pooled_dy;
+    r.pair = tune(TUNE_PAIR_WGRAD, 1) && r.grouped && k_tiles % 2 == 0 && !pooled_dy;
     r.L = 1;
     if (r.grouped)
         for (int l = r.pair ? 4 : 8; l >= 1; --l)        // pair: each CTA loads whole runs, half of the item's
@@ -610,8 +605,8 @@ WgradPlan plan_wgrad(int N, int P, int Q, int C, int K, int R, int S, int tap_gr
     r.run_blocks = (r.total_runs + r.rpi - 1) / r.rpi;
     // Haloed x boxes for single-CTA items of layers with few input maps (all taps of a kernel row fit one
     // accumulator): the pixel box must hold whole 8-pixel runs in w.
-    if (r.grouped && !r.pair && !pooled_dy && S >= 2 && cgroups * S * 32 <= 256 && Q >= 8 && env_int("PCL_XHALO_WGRAD", 1)) {
-        for (int pix = env_int("PCL_PIX_WGRAD", 64) == 64 ? 64 : 32; pix >= 32 && !r.xhalo; pix >>= 1) {
+    if (r.grouped && !r.pair && !pooled_dy && S >= 2 && cgroups * S * 32 <= 256 && Q >= 8 && tune(TUNE_XHALO_WGRAD, 1)) {
+        for (int pix = tune(TUNE_PIX_WGRAD, 64) == 64 ? 64 : 32; pix >= 32 && !r.xhalo; pix >>= 1) {
             int lw, lh;
             choose_pixel_box(pix, P, Q, N, &lw, &lh, 0, 3);
             const long bw = 1L << lw, bh = 1L << lh, bn = pix / (bw * bh);
@@ -630,7 +625,7 @@ WgradPlan plan_wgrad(int N, int P, int Q, int C, int K, int R, int S, int tap_gr
     }
     // 64-pixel k-steps halve the copies and commits per MMA; taken when three pipeline slots still fit
     const int cta_groups = 4 + (r.pair ? r.rpi / 2 : r.rpi) * r.L;      // 32-map groups a CTA loads per k-step
-    r.pix = env_int("PCL_PIX_WGRAD", 64);
+    r.pix = tune(TUNE_PIX_WGRAD, 64);
     if (r.pix != 64 || kSmemBudget / (cta_groups * 64 * 128) < 3) r.pix = 32;
     r.step_bytes = cta_groups * r.pix * 128;
     // A k-step of a narrow column block is a few short MMAs; such blocks get several k-steps per slot (one
@@ -638,7 +633,7 @@ WgradPlan plan_wgrad(int N, int P, int Q, int C, int K, int R, int S, int tap_gr
     const int max_groups = r.rpi * r.L;
     const int mma_clk = (r.pix / 8) * (max_groups * 16 > 52 ? max_groups * 16 : 52);
     r.KS = (600 + mma_clk - 1) / mma_clk;
-    r.KS = env_int("PCL_KS_WGRAD", r.KS);
+    r.KS = tune(TUNE_KS_WGRAD, r.KS);
     while (r.KS > 1 && kSmemBudget / (r.KS * r.step_bytes) < 3) --r.KS;
     if (r.KS < 1) r.KS = 1;
     r.stages = kSmemBudget / (r.KS * r.step_bytes);
@@ -649,17 +644,7 @@ WgradPlan plan_wgrad(int N, int P, int Q, int C, int K, int R, int S, int tap_gr
     return r;
 }
 
-int g_sm_count = 0;
-int sm_count() {
-    if (g_sm_count == 0) {
-        int dev = 0;
-        if (cudaGetDevice(&dev) != cudaSuccess ||
-            cudaDeviceGetAttribute(&g_sm_count, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || g_sm_count <= 0)
-            g_sm_count = 148;   // sizing only; a launch would fail anyway without a device
-    }
-    return g_sm_count;
-}
-bool g_attr_set = false;
+int sm_count() { return device_sm_count(); }
 
 }  // namespace
 
@@ -692,14 +677,16 @@ int tc_wgrad_splits(int N, int P, int Q, int C, int K, int R, int S, int tap_gro
 
 int launch_tc_wgrad(const TcWgradArgs& a, cudaStream_t st) {
     if (!tc_wgrad_eligible(a)) return PCL_ERR_UNSUPPORTED_SHAPE;
-    if (!g_attr_set) {
+    static PerDeviceOnce attr_once;       // (the attribute applies to the current device only)
+    const int setup_rc = attr_once.run([]() -> int {
         if (cudaFuncSetAttribute(tc_wgrad_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  kSmemBudget + 1024) != cudaSuccess ||
             cudaFuncSetAttribute(tc_wgrad_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  kSmemBudget + 1024) != cudaSuccess)
             return PCL_ERR_CUDA;
-        g_attr_set = true;
-    }
+        return PCL_OK;
+    });
+    if (setup_rc != PCL_OK) return setup_rc;
     WgradParams p{};
     const int pooled = a.dy_pool ? 1 : 0;
     if (pooled && (!a.codes || !tc_wgrad_can_take_pooled_dy(a.N, a.P, a.Q, a.C, a.K, a.R, a.S, a.tap_groups)))

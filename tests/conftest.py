@@ -24,3 +24,12 @@ def pytest_collection_modifyitems(config, items):
     for item in items:
         if "gpu" in item.keywords:
             item.add_marker(skip)
+
+
+@pytest.fixture(autouse=True)
+def _tuning_knobs_do_not_leak():
+    """A test that pins a launcher choice (binding.set_tuning) must not change what the next test runs."""
+    yield
+    from paper_1602_06709_b200 import binding as B
+    if B._lib is not None:
+        B.reset_tuning()

@@ -59,3 +59,6 @@ def test_host_side_checks(built_lib):
     assert L.pcl_sgd_update(null, null, 0, 0.1, null) == B.OK
     assert B.status_string(B.ERR_DEVICE_TIMEOUT) == "device-side wait timed out"
     assert L.pcl_set_path(9) == B.ERR_BAD_ARG
+    # launcher choices are pinned through the ABI only; an unknown knob is refused
+    assert L.pcl_set_tuning(b"TILING", 1) == B.OK and L.pcl_set_tuning(b"NO_SUCH_KNOB", 1) == B.ERR_BAD_ARG
+    assert L.pcl_set_tuning(None, 1) == B.ERR_BAD_ARG and L.pcl_reset_tuning() == B.OK

@@ -123,10 +123,10 @@ HALO_SHAPES = {
 @pytest.mark.parametrize("tag", sorted(HALO_SHAPES))
 def test_forward_type_kernel_every_tiling(tag, tiling, path_guard, monkeypatch):
     """The forward-type kernel has a plain tiling and three haloed ones (taps as row-shifted views of one
-    input patch); PCL_TILING pins one.  All must agree with the oracle for forward and backward-data."""
+    input patch); the TILING knob pins one.  All must agree with the oracle for forward and backward-data."""
     import gpu_helpers as G
     from paper_1602_06709_b200 import binding as B
-    monkeypatch.setenv("PCL_TILING", tiling)
+    B.set_tuning("TILING", tiling)
     B.set_path(B.PATH_TENSOR)
     s = HALO_SHAPES[tag]
     x, w, dy, bias = G.make_inputs(s, "halo_" + tag)
@@ -154,13 +154,13 @@ def test_forward_type_kernel_pipeline_variants(tag, variant, path_guard, monkeyp
     bias gradient path left to the network tests)."""
     import gpu_helpers as G
     from paper_1602_06709_b200 import binding as B
-    env = {"pair0": dict(PCL_PAIR="0", PCL_KS="1"), "pair1_ks1": dict(PCL_PAIR="1", PCL_KS="1"),
-           "pair1_ks2_nogroup": dict(PCL_PAIR="1", PCL_KS="2", PCL_GRP="0"),
-           "pair1_ks2_group": dict(PCL_PAIR="1", PCL_KS="2", PCL_GRP="1"),
-           "pair0_ks2_group": dict(PCL_PAIR="0", PCL_KS="2", PCL_GRP="1")}[variant]
+    env = {"pair0": dict(PAIR="0", KS="1"), "pair1_ks1": dict(PAIR="1", KS="1"),
+           "pair1_ks2_nogroup": dict(PAIR="1", KS="2", GRP="0"),
+           "pair1_ks2_group": dict(PAIR="1", KS="2", GRP="1"),
+           "pair0_ks2_group": dict(PAIR="0", KS="2", GRP="1")}[variant]
     for k, v in env.items():
-        monkeypatch.setenv(k, v)
-    monkeypatch.setenv("PCL_TILING", "plain")
+        B.set_tuning(k, v)
+    B.set_tuning("TILING", "plain")
     B.set_path(B.PATH_TENSOR)
     s = PIPELINE_SHAPES[tag]
     x, w, dy, bias = G.make_inputs(s, "pipe_" + tag)
@@ -175,19 +175,19 @@ def test_forward_type_kernel_pipeline_variants(tag, variant, path_guard, monkeyp
 @pytest.mark.parametrize("tag", sorted(PIPELINE_SHAPES))
 def test_forward_with_sixteen_epilogue_warps(tag, tiling, path_guard, monkeypatch):
     """Launches with a very short reduction run sixteen epilogue warps instead of eight (four per TMEM lane
-    quarter share a tile's 32-column chunks).  PCL_EPI_WARPS=32 forces that variant wherever it can run: the
+    quarter share a tile's 32-column chunks).  the EPI_WARPS knob = 32 forces that variant wherever it can run: the
     result must equal the eight-warp variant's bit for bit (same accumulators, same epilogue arithmetic)."""
     import gpu_helpers as G
     from paper_1602_06709_b200 import binding as B
-    monkeypatch.setenv("PCL_TILING", tiling)
-    monkeypatch.setenv("PCL_PAIR", "0")
-    monkeypatch.setenv("PCL_SPLIT_ACC", "0")
+    B.set_tuning("TILING", tiling)
+    B.set_tuning("PAIR", "0")
+    B.set_tuning("SPLIT_ACC", "0")
     B.set_path(B.PATH_TENSOR)
     s = PIPELINE_SHAPES[tag]
     x, w, dy, bias = G.make_inputs(s, "epi16_" + tag)
     res = {}
     for warps in ("8", "32"):
-        monkeypatch.setenv("PCL_EPI_WARPS", warps)
+        B.set_tuning("EPI_WARPS", warps)
         res[warps] = G.run_conv_fwd(s, x, w, bias, B.ACT_RELU)
     G.assert_parity(res["32"], oracle.conv_fwd(s, x, w, bias, oracle.ACT_RELU), f"fwd {tiling}")
     assert np.array_equal(res["8"], res["32"])
@@ -210,17 +210,17 @@ XHALO_SHAPES = {
 @pytest.mark.parametrize("tag", sorted(XHALO_SHAPES))
 def test_weight_gradient_with_haloed_input_boxes(tag, pix, path_guard, monkeypatch):
     """Layers with few input maps fetch one haloed input box per k-step and take the S taps of a kernel row as
-    row-shifted views of it (one MMA over 32*S columns); PCL_XHALO_WGRAD=0 keeps one box per tap.  Both must agree
+    row-shifted views of it (one MMA over 32*S columns); the XHALO_WGRAD knob = 0 keeps one box per tap.  Both must agree
     with the oracle; the two-pass result must repeat bit for bit."""
     import gpu_helpers as G
     from paper_1602_06709_b200 import binding as B
     B.set_path(B.PATH_TENSOR)
-    monkeypatch.setenv("PCL_PIX_WGRAD", pix)
+    B.set_tuning("PIX_WGRAD", pix)
     s = XHALO_SHAPES[tag]
     x, w, dy, _ = G.make_inputs(s, "xhalo_" + tag)
     dw_ref, db_ref = oracle.conv_bwd_weights(s, x, dy, want_db=True)
     for mode in ("1", "0"):
-        monkeypatch.setenv("PCL_XHALO_WGRAD", mode)
+        B.set_tuning("XHALO_WGRAD", mode)
         dw, db = G.run_conv_bwd_weights(s, x, dy, True, deterministic=True)
         G.assert_parity(dw, dw_ref, f"bwd_weights xhalo={mode}")
         G.assert_parity(db, db_ref, "dbias")
@@ -235,17 +235,17 @@ def test_weight_gradient_with_haloed_input_boxes(tag, pix, path_guard, monkeypat
 @pytest.mark.parametrize("tag", ["odd_groups", "even_groups_wide", "fc_like"])
 def test_backward_data_reads_weights_in_place(tag, tiling, path_guard, monkeypatch):
     """Backward-data takes the KRSC weights as an MN-major operand (taps flipped by index) when the layer's
-    input-map count is a multiple of 32; PCL_WEIGHTS_IN_PLACE=0 forces the flipped, transposed copy.  Same
+    input-map count is a multiple of 32; the WEIGHTS_IN_PLACE knob = 0 forces the flipped, transposed copy.  Same
     products, same order of additions: the two must agree bit for bit, and with the oracle."""
     import gpu_helpers as G
     from paper_1602_06709_b200 import binding as B
-    monkeypatch.setenv("PCL_TILING", tiling)
+    B.set_tuning("TILING", tiling)
     B.set_path(B.PATH_TENSOR)
     s = PIPELINE_SHAPES[tag]
     x, w, dy, _ = G.make_inputs(s, "inplace_" + tag)
-    monkeypatch.setenv("PCL_WEIGHTS_IN_PLACE", "1")
+    B.set_tuning("WEIGHTS_IN_PLACE", "1")
     dx1 = G.run_conv_bwd_data(s, dy, w, x)
-    monkeypatch.setenv("PCL_WEIGHTS_IN_PLACE", "0")
+    B.set_tuning("WEIGHTS_IN_PLACE", "0")
     dx0 = G.run_conv_bwd_data(s, dy, w, x)
     G.assert_parity(dx1, oracle.conv_bwd_data(s, dy, w, x), "bwd_data in place")
     assert np.array_equal(dx0, dx1)
@@ -261,17 +261,17 @@ def test_two_issuers_keep_results_reproducible(tag, mode, path_guard, monkeypatc
     bit for bit; the ordered mode must equal the single issuer exactly."""
     import gpu_helpers as G
     from paper_1602_06709_b200 import binding as B
-    env = {"solo": dict(PCL_ISSUERS="1"), "ordered": dict(PCL_ISSUERS="2", PCL_SPLIT_ACC="0"),
-           "split": dict(PCL_ISSUERS="2", PCL_SPLIT_ACC="1")}
+    env = {"solo": dict(ISSUERS="1"), "ordered": dict(ISSUERS="2", SPLIT_ACC="0"),
+           "split": dict(ISSUERS="2", SPLIT_ACC="1")}
     B.set_path(B.PATH_TENSOR)
     s = HALO_SHAPES[tag]
     x, w, dy, bias = G.make_inputs(s, "issuers_" + tag)
 
     def run(m):
-        for k in ("PCL_ISSUERS", "PCL_SPLIT_ACC"):
-            monkeypatch.delenv(k, raising=False)
+        for k in ("ISSUERS", "SPLIT_ACC"):
+            B.set_tuning(k, None)
         for k, v in env[m].items():
-            monkeypatch.setenv(k, v)
+            B.set_tuning(k, v)
         return G.run_conv_fwd(s, x, w, bias, B.ACT_RELU), G.run_conv_bwd_data(s, dy, w, x)
 
     y, dx = run(mode)

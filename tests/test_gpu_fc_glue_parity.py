@@ -33,12 +33,12 @@ def path_guard():
 def test_fc_fwd_bwd(N, C, K, act, path, path_guard, monkeypatch):
     """The FC weight gradient has two forms on the tensor path: the weight-gradient kernel, or (short reductions,
     C % 32 == 0) the forward-type kernel over dz^T with x read in place as an MN-major operand;
-    PCL_FC_DW_FORWARD pins one."""
+    the FC_DW_FORWARD knob pins one."""
     import gpu_helpers as G
     from paper_1602_06709_b200 import binding as B
     from paper_1602_06709_b200 import inputs
     if path.startswith("tensor_dw"):
-        monkeypatch.setenv("PCL_FC_DW_FORWARD", "1" if "forward" in path else "0")
+        B.set_tuning("FC_DW_FORWARD", "1" if "forward" in path else "0")
     B.set_path(B.PATH_GENERIC if path == "generic" else B.PATH_TENSOR)
     code = {"none": B.ACT_NONE, "relu": B.ACT_RELU, "sigmoid": B.ACT_SIGMOID}[act]
     tid = lambda r: inputs.tensor_id("fc", N, C, K, r)
@@ -52,16 +52,16 @@ def test_fc_fwd_bwd(N, C, K, act, path, path_guard, monkeypatch):
     B.check_device_status()
     y = yt.cpu().numpy()
     G.assert_parity(y, oracle.fc_fwd(x, w, b, code), "fc fwd")
-    # with scratch the launcher may split the reduction over more CTAs (few tiles, long reduction); PCL_KSPLIT pins
+    # with scratch the launcher may split the reduction over more CTAs (few tiles, long reduction); the KSPLIT knob pins
     # the number of splits where it divides the reduction's pipeline slots
     for ks in ("0", "2", "3", "5"):
-        monkeypatch.setenv("PCL_KSPLIT", ks)
+        B.set_tuning("KSPLIT", ks)
         ws_f = G.workspace(B.fc_workspace_bytes(N, C, K, B.PASS_FWD))
         yt2 = torch.full((N, K), float("nan"), device="cuda")
         B.fc_fwd(N, C, K, xt, wt, bt, yt2, code, ws_f)
         B.check_device_status()
-        G.assert_parity(yt2.cpu().numpy(), oracle.fc_fwd(x, w, b, code), f"fc fwd, PCL_KSPLIT={ks}")
-    monkeypatch.delenv("PCL_KSPLIT")
+        G.assert_parity(yt2.cpu().numpy(), oracle.fc_fwd(x, w, b, code), f"fc fwd, KSPLIT={ks}")
+    B.set_tuning("KSPLIT", None)
     # backward is checked on the GPU's own forward output (per-call parity)
     dyt = G.dev(dy)
     dxt = torch.full((N, C), float("nan"), device="cuda")
@@ -201,7 +201,7 @@ def test_conv_bwd_data_with_fused_column_sums(shape, tiling, monkeypatch):
     from oracle import ConvShape
     from paper_1602_06709_b200 import binding as B
     if tiling != "auto":
-        monkeypatch.setenv("PCL_TILING", tiling)
+        B.set_tuning("TILING", tiling)
     N, C, K, H, W = shape
     s = ConvShape(N=N, C=C, K=K, H=H, W=W, R=3, S=3, pad_h=1, pad_w=1)
     x, w, dy, _ = G.make_inputs(s, f"dgradcs{C}")
@@ -242,13 +242,13 @@ def test_conv_fwd_with_fused_maxpool(shape, tiling, store, monkeypatch):
     from oracle import ConvShape
     from paper_1602_06709_b200 import binding as B
     if tiling != "auto":
-        monkeypatch.setenv("PCL_TILING", tiling)
+        B.set_tuning("TILING", tiling)
     # the epilogue writes y either with TMA stores from its staging tiles or with per-lane coalesced stores
-    monkeypatch.setenv("PCL_TMA_STORE", "0" if store == "direct" else "1")
+    B.set_tuning("TMA_STORE", "0" if store == "direct" else "1")
     # the kernel variant with sixteen epilogue warps (chosen by itself only for very short reductions), single CTAs
-    monkeypatch.setenv("PCL_EPI_WARPS", "32" if store == "tma_16_epilogue_warps" else "8")
+    B.set_tuning("EPI_WARPS", "32" if store == "tma_16_epilogue_warps" else "8")
     if store == "tma_16_epilogue_warps":
-        monkeypatch.setenv("PCL_PAIR", "0")
+        B.set_tuning("PAIR", "0")
     N, C, K, H, W = shape
     s = ConvShape(N=N, C=C, K=K, H=H, W=W, R=3, S=3, pad_h=1, pad_w=1)
     x, w, _, bias = G.make_inputs(s, f"fwdpool{C}_{K}")
