@@ -390,13 +390,13 @@ __global__ void __launch_bounds__(256) softmax_xent_kernel(const float* __restri
 
 // xs[n][hh][ww][0..3]: channel-padded copy of x with a zero halo of (pad_h, pad_w).  One block per padded image row
 // (no per-pixel index divisions: the kernel is otherwise bound by them, not by memory); the block after the last
-// row writes the 8 trailing zero pixels (windows are read 32 floats wide).
+// row writes the trailing zero pixels (windows are read 32 floats wide, so the last ones reach past the last row).
 __global__ void __launch_bounds__(256) stage_pad_c4_kernel(const float* __restrict__ x, float4* __restrict__ xs, int N,
-                                                           int H, int W, int C, int pad_h, int pad_w) {
+                                                           int H, int W, int C, int pad_h, int pad_w, int slack) {
     const int Hp = H + 2 * pad_h, Wp = W + 2 * pad_w;
     const size_t row = blockIdx.x;                       // n * Hp + hh + pad_h
     if (row == size_t(N) * Hp) {
-        if (threadIdx.x < 8) xs[row * Wp + threadIdx.x] = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (int(threadIdx.x) < slack) xs[row * Wp + threadIdx.x] = make_float4(0.f, 0.f, 0.f, 0.f);
         return;
     }
     const size_t n = row / Hp;
@@ -416,28 +416,45 @@ __global__ void __launch_bounds__(256) stage_pad_c4_kernel(const float* __restri
     }
 }
 
-// w32[k*R + r][s*4 + c] = w[k][r][s][c] for c < C, s < S; every other element of the 32-float row is zero
+// w32[k*R + r][s*4 + c] = w[k][r][s][c] for c < C, s < S; every other element of the row_floats-long row is zero
 __global__ void __launch_bounds__(256) stage_w4_kernel(const float* __restrict__ w, float* __restrict__ w32,
-                                                       size_t rows, int S, int C) {
-    const size_t total = rows * 32;
+                                                       size_t rows, int S, int C, int row_floats) {
+    const size_t total = rows * row_floats;
     const size_t stride = size_t(gridDim.x) * blockDim.x;
     for (size_t i = size_t(blockIdx.x) * blockDim.x + threadIdx.x; i < total; i += stride) {
-        const int j = int(i & 31); const size_t row = i >> 5;
+        const size_t row = i / row_floats; const int j = int(i - row * row_floats);
         const int s = j >> 2, c = j & 3;
         w32[i] = (s < S && c < C) ? w[(row * S + s) * C + c] : 0.f;
     }
 }
 
-// dw[tap][c] = sum_s dw4[s][tap][c], c < C  (fixed order)
+// dw[row][s][c] = sum over splits of dw4[split][row][s*4 + c], c < C, s < S  (fixed order)
 __global__ void __launch_bounds__(256) unpad_reduce_kernel(const float* __restrict__ dw4, float* __restrict__ dw,
-                                                           size_t taps, int C, int splits, size_t split_stride) {
-    const size_t total = taps * C;
+                                                           size_t rows, int S, int C, int row_floats, int splits,
+                                                           size_t split_stride) {
+    const size_t total = rows * S * C;
     const size_t stride = size_t(gridDim.x) * blockDim.x;
     for (size_t i = size_t(blockIdx.x) * blockDim.x + threadIdx.x; i < total; i += stride) {
         const size_t tap = i / C; const int c = int(i % C);
+        const size_t row = tap / S; const int s = int(tap - row * S);
         float acc = 0.f;
-        for (int s = 0; s < splits; ++s) acc += dw4[size_t(s) * split_stride + tap * 4 + c];
+        for (int sp = 0; sp < splits; ++sp) acc += dw4[size_t(sp) * split_stride + row * row_floats + s * 4 + c];
         dw[i] = acc;
+    }
+}
+
+// One phase of a strided backward-data pass: out[c][Ra-1-i][Sb-1-j][k] = w[k][a + i*sh][b + j*sw][c].
+__global__ void __launch_bounds__(256) phase_weights_kernel(const float* __restrict__ w, float* __restrict__ out, int K,
+                                                            int R, int S, int C, int a, int b, int sh, int sw, int Ra,
+                                                            int Sb) {
+    const size_t total = size_t(C) * Ra * Sb * K;
+    const size_t stride = size_t(gridDim.x) * blockDim.x;
+    for (size_t o = size_t(blockIdx.x) * blockDim.x + threadIdx.x; o < total; o += stride) {
+        const int k = int(o % K); size_t t = o / K;
+        const int jj = int(t % Sb); t /= Sb;
+        const int ii = int(t % Ra); const int c = int(t / Ra);
+        const int r = a + (Ra - 1 - ii) * sh, s = b + (Sb - 1 - jj) * sw;
+        out[o] = w[((size_t(k) * R + r) * S + s) * C + c];
     }
 }
 
@@ -523,30 +540,45 @@ int launch_transpose_flip(const float* w, float* wt_t, int K, int R, int S, int 
     return PCL_CHECK_LAUNCH();
 }
 
-int launch_stage_pad_c4(const float* x, float* xs, int N, int H, int W, int C, int pad_h, int pad_w, cudaStream_t st) {
-    const size_t total = size_t(N) * (H + 2 * pad_h) * (W + 2 * pad_w) + 8;
+int launch_phase_weights(const float* w, float* wt_t, int K, int R, int S, int C, int a, int b, int stride_h,
+                         int stride_w, int Ra, int Sb, cudaStream_t st) {
+    const size_t total = size_t(C) * Ra * Sb * K;
+    if (total == 0) return PCL_OK;
+    {
+        LaunchScope scope(KID_TRANSPOSE_FLIP, 8.0 * double(total), st);
+        phase_weights_kernel<<<grid_for(total, 256), 256, 0, st>>>(w, wt_t, K, R, S, C, a, b, stride_h, stride_w, Ra, Sb);
+    }
+    return PCL_CHECK_LAUNCH();
+}
+
+int launch_stage_pad_c4(const float* x, float* xs, int N, int H, int W, int C, int pad_h, int pad_w, int slack_pixels,
+                        cudaStream_t st) {
+    if (slack_pixels < 0 || slack_pixels > 256) return PCL_ERR_UNSUPPORTED_SHAPE;
+    const size_t total = size_t(N) * (H + 2 * pad_h) * (W + 2 * pad_w) + slack_pixels;
     {
         LaunchScope scope(KID_STAGE_PAD_C4, 4.0 * double(N) * H * W * C + 16.0 * double(total), st);
         const size_t rows = size_t(N) * (H + 2 * pad_h) + 1;        // + the block that writes the trailing zero pixels
         if (rows > 0x7fffffffu) return PCL_ERR_UNSUPPORTED_SHAPE;
-        stage_pad_c4_kernel<<<unsigned(rows), 256, 0, st>>>(x, reinterpret_cast<float4*>(xs), N, H, W, C, pad_h, pad_w);
+        stage_pad_c4_kernel<<<unsigned(rows), 256, 0, st>>>(x, reinterpret_cast<float4*>(xs), N, H, W, C, pad_h, pad_w,
+                                                            slack_pixels);
     }
     return PCL_CHECK_LAUNCH();
 }
 
-int launch_stage_w4(const float* w, float* w32, size_t rows, int S, int C, cudaStream_t st) {
+int launch_stage_w4(const float* w, float* w32, size_t rows, int S, int C, int row_floats, cudaStream_t st) {
     {
-        LaunchScope scope(KID_STAGE_W4, double(rows) * (4.0 * S * C + 128.0), st);
-        stage_w4_kernel<<<grid_for(rows * 32, 256), 256, 0, st>>>(w, w32, rows, S, C);
+        LaunchScope scope(KID_STAGE_W4, double(rows) * (4.0 * S * C + 4.0 * row_floats), st);
+        stage_w4_kernel<<<grid_for(rows * row_floats, 256), 256, 0, st>>>(w, w32, rows, S, C, row_floats);
     }
     return PCL_CHECK_LAUNCH();
 }
 
-int launch_unpad_reduce(const float* dw4, float* dw, size_t taps, int C, int splits, size_t split_stride,
-                        cudaStream_t st) {
+int launch_unpad_reduce(const float* dw4, float* dw, size_t rows, int S, int C, int row_floats, int splits,
+                        size_t split_stride, cudaStream_t st) {
     {
-        LaunchScope scope(KID_UNPAD_REDUCE, 4.0 * double(taps) * C * (splits + 1), st);
-        unpad_reduce_kernel<<<grid_for(taps * C, 256), 256, 0, st>>>(dw4, dw, taps, C, splits, split_stride);
+        LaunchScope scope(KID_UNPAD_REDUCE, 4.0 * double(rows) * S * C * (splits + 1), st);
+        unpad_reduce_kernel<<<grid_for(rows * S * C, 256), 256, 0, st>>>(dw4, dw, rows, S, C, row_floats, splits,
+                                                                          split_stride);
     }
     return PCL_CHECK_LAUNCH();
 }

@@ -64,7 +64,7 @@ struct ProfEntry { int kid; int pass; double work; cudaEvent_t e0, e1; };
 // Which ABI call the launches of this thread belong to (outermost call wins), and, for its contraction launches,
 // the layer's own algorithmic work 2*N*K*P*Q*C*R*S: a launch that runs on a padded or staged view of the layer
 // (few-channel staging, phase-decomposed strides) must not count the zero padding as work.
-struct PassState { int pass = 0; int depth = 0; double flops = 0.0; };
+struct PassState { int pass = 0; int depth = 0; double flops = 0.0; int counted = 0; };
 thread_local PassState t_pass;
 const char* const kPassNames[PROF_PASS_COUNT] = {"other", "conv_fwd", "conv_bwd_data", "conv_bwd_weights", "fc_fwd", "fc_bwd"};
 bool is_contraction(int kid) {
@@ -96,7 +96,12 @@ LaunchScope::LaunchScope(int kid, double work, cudaStream_t stream) : slot(-1), 
     g_launches.fetch_add(1, std::memory_order_relaxed);
     std::lock_guard<std::mutex> lock(g_prof_mu);
     if (!g_prof_on) return;
-    if (t_pass.depth > 0 && t_pass.flops > 0.0 && is_contraction(kid)) work = t_pass.flops;
+    if (t_pass.depth > 0 && t_pass.flops > 0.0 && is_contraction(kid)) {
+        // the first `counted` contraction launches of the call carry the layer's flops; a call that cuts one pass
+        // into several launches (the phases of a strided backward-data pass) counts it once
+        work = t_pass.counted > 0 ? t_pass.flops : 0.0;
+        if (t_pass.counted > 0) --t_pass.counted;
+    }
     ProfEntry e{kid, t_pass.depth > 0 ? t_pass.pass : PROF_PASS_OTHER, work, prof_event(), prof_event()};
     if (!e.e0 || !e.e1) return;
     cudaEventRecord(e.e0, st);
@@ -110,8 +115,8 @@ LaunchScope::~LaunchScope() {
     if (slot < int(g_prof_entries.size())) cudaEventRecord(g_prof_entries[slot].e1, st);
 }
 
-PassScope::PassScope(int pass, double flops) {
-    if (t_pass.depth++ == 0) { t_pass.pass = pass; t_pass.flops = flops; }
+PassScope::PassScope(int pass, double flops, int contraction_launches) {
+    if (t_pass.depth++ == 0) { t_pass.pass = pass; t_pass.flops = flops; t_pass.counted = contraction_launches; }
 }
 PassScope::~PassScope() {
     if (--t_pass.depth == 0) { t_pass.pass = PROF_PASS_OTHER; t_pass.flops = 0.0; }
@@ -136,7 +141,7 @@ encode_tiled_fn get_encode_tiled() {
 }
 
 int make_tmap(CUtensorMap* out, const void* base, int rank, const uint64_t* dims, const uint64_t* strides_bytes,
-              const uint32_t* box, bool atom32, bool plain_f32) {
+              const uint32_t* box, bool atom32, bool plain_f32, const uint32_t* elem_strides) {
     encode_tiled_fn enc = get_encode_tiled();
     if (!enc) return PCL_ERR_CUDA;
     cuuint64_t gdim[5];
@@ -145,8 +150,8 @@ int make_tmap(CUtensorMap* out, const void* base, int rank, const uint64_t* dims
     for (int i = 0; i < rank; ++i) {
         gdim[i] = dims[i];
         gbox[i] = box[i];
-        estr[i] = 1;
-        if (box[i] == 0 || box[i] > 256) return PCL_ERR_UNSUPPORTED_SHAPE;
+        estr[i] = elem_strides ? elem_strides[i] : 1;
+        if (box[i] == 0 || box[i] > 256 || estr[i] == 0 || estr[i] > 8) return PCL_ERR_UNSUPPORTED_SHAPE;
     }
     for (int i = 0; i + 1 < rank; ++i) {
         gstr[i] = strides_bytes[i];
@@ -175,8 +180,10 @@ size_t dw_bytes(const pcl_conv_desc& d);
 // Bytes of the flipped, transposed weight copy backward-data makes on the tensor-core path (0 where the weights
 // are read in place or another kernel family runs): the part of the backward-data workspace that is mandatory.
 size_t bwd_data_transposed_bytes(const pcl_conv_desc& d) {
-    if (g_path.load() == PCL_PATH_GENERIC || d.stride_h != 1 || d.stride_w != 1) return 0;
-    if (!(d.K % 4 == 0 && d.pad_h <= d.R - 1 && d.pad_w <= d.S - 1)) return 0;
+    if (g_path.load() == PCL_PATH_GENERIC || d.K % 4 != 0) return 0;
+    if (d.stride_h != 1 || d.stride_w != 1)       // one flipped, transposed sub-kernel per phase, each 256-byte aligned
+        return d.stride_h <= 8 && d.stride_w <= 8 ? dw_bytes(d) + size_t(256) * d.stride_h * d.stride_w : 0;
+    if (!(d.pad_h <= d.R - 1 && d.pad_w <= d.S - 1)) return 0;
     return weights_read_in_place(d) ? 0 : dw_bytes(d);
 }
 
@@ -202,30 +209,47 @@ bool unit_stride(const pcl_conv_desc& d) { return d.stride_h == 1 && d.stride_w 
 // checked separately; all pointers are required to be 16-byte aligned anyway).
 bool tensor_path_for(const pcl_conv_desc& d, int pass) {
     if (g_path.load() == PCL_PATH_GENERIC) return false;
-    if (!unit_stride(d)) return false;
+    if (d.stride_h > 8 || d.stride_w > 8) return false;
     switch (pass) {
         case PCL_PASS_FWD: return d.C % 4 == 0;
-        case PCL_PASS_BWD_DATA: return d.K % 4 == 0 && d.pad_h <= d.R - 1 && d.pad_w <= d.S - 1;
+        // (a strided layer runs one stride-1 sub-convolution per phase of the input grid, see conv_bwd_data_phases)
+        case PCL_PASS_BWD_DATA: return d.K % 4 == 0 && (!unit_stride(d) || (d.pad_h <= d.R - 1 && d.pad_w <= d.S - 1));
         case PCL_PASS_BWD_WEIGHTS: return d.C % 4 == 0 && d.K % 4 == 0;
     }
     return false;
 }
 
-// Few-channel first layers (C < 4, stride 1): the input is staged once as a
-// 4-channel, halo-padded copy; a row of S taps x 4 channels is then contiguous
-// (S*4 <= 32 floats), so the tensor-core kernels see a layer with S*4 "channels",
-// an R x 1 kernel and no padding, read through overlapping TMA windows.
+// Few-channel first layers (C < 4): the input is staged once as a 4-channel, halo-padded copy; a window of 8 pixels
+// x 4 channels is then 32 contiguous floats, read through overlapping TMA windows (pixel stride 16 bytes, times the
+// layer's stride).  The tensor-core kernels see a layer with 32 "channels" per tap, an R x S' kernel whose S' =
+// ceil(S / 8) taps of a row lie 8 pixels apart (tap s' covers kernel columns 8s' .. 8s'+7; columns past S and the
+// fourth channel meet zero weights), and no padding.
+int few_sblocks(const pcl_conv_desc& d) { return (d.S + 7) / 8; }
 bool few_channel_path_for(const pcl_conv_desc& d, int pass) {
     if (g_path.load() == PCL_PATH_GENERIC) return false;
-    if (!unit_stride(d) || d.C >= 4 || d.S * 4 > 32 || d.R > 8) return false;
+    if (d.C >= 4 || d.S > 32 || d.stride_h > 8 || d.stride_w > 8) return false;
     if (pass == PCL_PASS_FWD) return true;
     if (pass == PCL_PASS_BWD_WEIGHTS) return d.K % 4 == 0;
     return false;
 }
-size_t staged_x_bytes(const pcl_conv_desc& d) {   // + 8 zero pixels of slack: windows are read 32 floats wide
-    return align_up((size_t(d.N) * (d.H + 2 * d.pad_h) * (d.W + 2 * d.pad_w) + 8) * 16, 256);
+// The weight gradient of stride-1 few-channel layers with one window per kernel row and at most 8 rows takes all
+// tap rows of a k tile in one work item (TcWgradArgs::tap_groups); other few-channel layers run the general form.
+bool few_taprows_form(const pcl_conv_desc& d) { return unit_stride(d) && d.S <= 8 && d.R <= 8; }
+int few_slack_pixels(const pcl_conv_desc& d) { return 8 * few_sblocks(d); }   // the last windows reach past the last row
+size_t staged_x_bytes(const pcl_conv_desc& d) {
+    return align_up((size_t(d.N) * (d.H + 2 * d.pad_h) * (d.W + 2 * d.pad_w) + few_slack_pixels(d)) * 16, 256);
 }
-size_t staged_w_bytes(const pcl_conv_desc& d) { return align_up(size_t(d.K) * d.R * 128, 256); }
+size_t staged_w_bytes(const pcl_conv_desc& d) { return align_up(size_t(d.K) * d.R * few_sblocks(d) * 128, 256); }
+// The staged layer as the forward-type kernel sees it.
+TcFpropArgs few_fwd_args(const pcl_conv_desc& d, int P, int Q, const float* xs, const float* w4, const float* bias,
+                         float* y, int act) {
+    const int Hp = d.H + 2 * d.pad_h, Wp = d.W + 2 * d.pad_w, Sb = few_sblocks(d);
+    // declared width: one window start per reachable pixel, (Q-1)*stride_w + 8*(S'-1) being the last
+    TcFpropArgs a{xs, w4, bias, nullptr, y, d.N, Hp, (Q - 1) * d.stride_w + 8 * (Sb - 1) + 1, 32, d.K, d.R, Sb, 0, 0, P, Q, act};
+    a.in_stride_w = 4; a.in_stride_h = long(Wp) * 4; a.in_stride_n = long(Hp) * Wp * 4;
+    a.stride_h = d.stride_h; a.stride_w = d.stride_w; a.dil_w = 8;
+    return a;
+}
 
 size_t dw_bytes(const pcl_conv_desc& d) { return align_up(size_t(d.K) * d.R * d.S * d.C * 4, 256); }
 
@@ -242,11 +266,13 @@ WgradPlan plan_wgrad(const pcl_conv_desc& d, int P, int Q) {
     pl.few = few_channel_path_for(d, PCL_PASS_BWD_WEIGHTS);
     pl.tensor = pl.few || tensor_path_for(d, PCL_PASS_BWD_WEIGHTS);
     if (pl.few) {
-        pl.splits = tc_wgrad_splits(d.N, P, Q, d.S * 4, d.K, d.R, 1, 1);
+        pl.splits = few_taprows_form(d) ? tc_wgrad_splits(d.N, P, Q, d.S * 4, d.K, d.R, 1, 1)
+                                        : tc_wgrad_splits(d.N, P, Q, 32, d.K, d.R, few_sblocks(d), 0, 0, 1);
         // staged x + per-split dw4 tiles (always two-pass: the un-padding pass is needed anyway)
         pl.partial_bytes = staged_x_bytes(d) + size_t(pl.splits) * staged_w_bytes(d);
     } else {
-        pl.splits = pl.tensor ? tc_wgrad_splits(d.N, P, Q, d.C, d.K, d.R, d.S) : generic_wgrad_splits(d, P, Q);
+        pl.splits = pl.tensor ? tc_wgrad_splits(d.N, P, Q, d.C, d.K, d.R, d.S, 0, 0, unit_stride(d) ? 0 : 1)
+                              : generic_wgrad_splits(d, P, Q);
         pl.partial_bytes = pl.splits > 1 ? size_t(pl.splits) * dw_bytes(d) : 0;
     }
     const int cs = colsum_splits(size_t(d.N) * P * Q);
@@ -310,9 +336,11 @@ int pcl_conv_out_dims(const pcl_conv_desc* d, int* P, int* Q) {
 static size_t fwd_split_bytes(const pcl_conv_desc& d, int P, int Q) {
     TcFpropArgs a{nullptr, nullptr, nullptr, nullptr, nullptr, d.N, d.H, d.W, d.C, d.K, d.R, d.S, d.pad_h, d.pad_w, P, Q,
                   PCL_ACT_NONE};
+    a.stride_h = d.stride_h; a.stride_w = d.stride_w;
     return align_up(tc_fprop_split_ws_bytes(a), 256);
 }
 static size_t bwd_data_split_bytes(const pcl_conv_desc& d, int P, int Q) {
+    if (d.stride_h != 1 || d.stride_w != 1) return 0;
     TcFpropArgs a{nullptr, nullptr, nullptr, nullptr, nullptr, d.N, P, Q, d.K, d.C, d.R, d.S,
                   d.R - 1 - d.pad_h, d.S - 1 - d.pad_w, d.H, d.W, PCL_ACT_NONE};
     if (d.C % 32 == 0) a.wt_mn_major = 1;       // (either form of the weights gives the same tiling)
@@ -326,7 +354,10 @@ size_t pcl_conv_workspace_bytes(const pcl_conv_desc* d, int pass) {
         case PCL_PASS_FWD:
             if (few_channel_path_for(*d, pass)) return staged_x_bytes(*d) + staged_w_bytes(*d);
             return tensor_path_for(*d, pass) ? fwd_split_bytes(*d, P, Q) : 0;
-        case PCL_PASS_BWD_DATA: return tensor_path_for(*d, pass) ? dw_bytes(*d) + bwd_data_split_bytes(*d, P, Q) : 0;
+        case PCL_PASS_BWD_DATA:
+            if (!tensor_path_for(*d, pass)) return 0;
+            if (!unit_stride(*d)) return bwd_data_transposed_bytes(*d);
+            return dw_bytes(*d) + bwd_data_split_bytes(*d, P, Q);
         case PCL_PASS_BWD_WEIGHTS: {
             const WgradPlan pl = plan_wgrad(*d, P, Q);
             return pl.partial_bytes + pl.colsum_bytes;
@@ -369,18 +400,17 @@ static int conv_fwd_impl(const pcl_conv_desc* d, const float* x, const float* w,
         if (reinterpret_cast<uintptr_t>(ws) & 255) return PCL_ERR_MISALIGNED;
         float* xs = static_cast<float*>(ws);
         float* w4 = reinterpret_cast<float*>(static_cast<char*>(ws) + xs_bytes);
-        rc = launch_stage_pad_c4(x, xs, d->N, d->H, d->W, d->C, d->pad_h, d->pad_w, st);
+        rc = launch_stage_pad_c4(x, xs, d->N, d->H, d->W, d->C, d->pad_h, d->pad_w, few_slack_pixels(*d), st);
         if (rc != PCL_OK) return rc;
-        rc = launch_stage_w4(w, w4, size_t(d->K) * d->R, d->S, d->C, st);
+        rc = launch_stage_w4(w, w4, size_t(d->K) * d->R, d->S, d->C, few_sblocks(*d) * 32, st);
         if (rc != PCL_OK) return rc;
-        const int Hp = d->H + 2 * d->pad_h, Wp = d->W + 2 * d->pad_w;
-        // the staged layer: 32 "channels" per pixel window (S*4 carry weight, the rest meets zero weights)
-        TcFpropArgs a{xs, w4, bias, nullptr, y, d->N, Hp, Q, 32, d->K, d->R, 1, 0, 0, P, Q, act};
-        a.in_stride_w = 4; a.in_stride_h = long(Wp) * 4; a.in_stride_n = long(Hp) * Wp * 4;
+        // the staged layer: 32 "channels" per pixel window (the taps' channels carry weight, the rest meets zero weights)
+        TcFpropArgs a = few_fwd_args(*d, P, Q, xs, w4, bias, y, act);
         if (y_pool && tc_fprop_can_pool(a)) { a.pool_out = y_pool; a.pool_idx = pool_codes; y_pool = nullptr; }
         rc = launch_tc_fprop(a, st);
     } else if (tensor_path_for(*d, PCL_PASS_FWD)) {
         TcFpropArgs a{x, w, bias, nullptr, y, d->N, d->H, d->W, d->C, d->K, d->R, d->S, d->pad_h, d->pad_w, P, Q, act};
+        a.stride_h = d->stride_h; a.stride_w = d->stride_w;
         if (y_pool && tc_fprop_can_pool(a)) { a.pool_out = y_pool; a.pool_idx = pool_codes; y_pool = nullptr; }
         if (ws && (reinterpret_cast<uintptr_t>(ws) & 255) == 0) {      // scratch for a split reduction, if the caller gave some
             a.split_ws = static_cast<float*>(ws); a.split_ws_bytes = ws_bytes;
@@ -417,6 +447,47 @@ int pcl_conv_fwd_pool(const pcl_conv_desc* d, const float* x, const float* w, co
     return conv_fwd_impl(d, x, w, bias, y, y_pool, pool_codes, act, ws, ws_bytes, cuda_stream);
 }
 
+namespace {
+// Backward-data of a strided layer on the tensor-core path.  Input pixel h belongs to phase a = (h + pad_h) mod
+// stride_h (likewise b in w); only the taps r = a + i*stride_h reach it, from output rows p = (h + pad_h - a) /
+// stride_h - i.  So every phase (a, b) is a stride-1 convolution of dy with the flipped sub-kernel
+// w[k][a + i*stride_h][b + j*stride_w][c], written to every stride-th pixel of dx: stride_h * stride_w launches of
+// the forward-type kernel, each with its own transposed sub-kernel in the workspace.  Pixels of phases without taps
+// (a stride larger than the kernel) are zeroed first.
+int conv_bwd_data_phases(const pcl_conv_desc& d, int P, int Q, const float* dy, const float* w, const float* mask,
+                         float* dx, char* ws, cudaStream_t st) {
+    const int sh = d.stride_h, sw = d.stride_w;
+    if (sh > d.R || sw > d.S) {
+        const int rc = launch_zero(dx, size_t(d.N) * d.H * d.W * d.C, st);
+        if (rc != PCL_OK) return rc;
+    }
+    size_t off = 0;
+    for (int a = 0; a < sh; ++a)
+        for (int b = 0; b < sw; ++b) {
+            const int Ra = a < d.R ? (d.R - a + sh - 1) / sh : 0, Sb = b < d.S ? (d.S - b + sw - 1) / sw : 0;
+            if (Ra == 0 || Sb == 0) continue;
+            // pixels of the phase: h + pad_h = u*stride_h + a with 0 <= h < H, i.e. u0 <= u <= u1
+            const int u0 = d.pad_h > a ? (d.pad_h - a + sh - 1) / sh : 0, v0 = d.pad_w > b ? (d.pad_w - b + sw - 1) / sw : 0;
+            const int top_h = d.H - 1 + d.pad_h - a, top_w = d.W - 1 + d.pad_w - b;
+            if (top_h < 0 || top_w < 0) continue;
+            const int Hph = top_h / sh - u0 + 1, Wph = top_w / sw - v0 + 1;
+            if (Hph <= 0 || Wph <= 0) continue;
+            float* wt = reinterpret_cast<float*>(ws + off);
+            off += align_up(size_t(d.C) * Ra * Sb * d.K * 4, 256);
+            int rc = launch_phase_weights(w, wt, d.K, d.R, d.S, d.C, a, b, sh, sw, Ra, Sb, st);
+            if (rc != PCL_OK) return rc;
+            const size_t first = (size_t(u0 * sh + a - d.pad_h) * d.W + size_t(v0 * sw + b - d.pad_w)) * d.C;
+            // out[n, u', v', c] = sum_{r', s', k} dy[n, u' + r' - (Ra-1-u0), v' + s' - (Sb-1-v0), k] * wt[c][r'][s'][k]
+            TcFpropArgs t{dy, wt, nullptr, mask ? mask + first : nullptr, dx + first, d.N, P, Q, d.K, d.C, Ra, Sb,
+                          Ra - 1 - u0, Sb - 1 - v0, Hph, Wph, PCL_ACT_NONE};
+            t.out_stride_w = long(sw) * d.C; t.out_stride_h = long(sh) * d.W * d.C; t.out_stride_n = long(d.H) * d.W * d.C;
+            rc = launch_tc_fprop(t, st);
+            if (rc != PCL_OK) return rc;
+        }
+    return PCL_OK;
+}
+}  // namespace
+
 int pcl_conv_bwd_data(const pcl_conv_desc* d, const float* dy, const float* w, const float* relu_mask_src, float* dx,
                       void* ws, size_t ws_bytes, void* cuda_stream) {
     int P, Q;
@@ -432,6 +503,7 @@ int pcl_conv_bwd_data(const pcl_conv_desc* d, const float* dy, const float* w, c
         const size_t need = bwd_data_transposed_bytes(*d);
         if (need > 0 && (!ws || ws_bytes < need)) return PCL_ERR_WORKSPACE;
         if (ws && (reinterpret_cast<uintptr_t>(ws) & 255)) return PCL_ERR_MISALIGNED;
+        if (!unit_stride(*d)) return conv_bwd_data_phases(*d, P, Q, dy, w, relu_mask_src, dx, static_cast<char*>(ws), st);
         // dx = "forward" convolution of dy with the flipped, transposed weights, pad' = R-1-pad
         TcFpropArgs a{dy, w, nullptr, relu_mask_src, dx, d->N, P, Q, d->K, d->C, d->R, d->S,
                       d->R - 1 - d->pad_h, d->S - 1 - d->pad_w, d->H, d->W, PCL_ACT_NONE};
@@ -476,7 +548,7 @@ size_t pcl_conv_bwd_data_colsum_workspace_bytes(const pcl_conv_desc* d) {
     if (check_desc(d, &P, &Q) != PCL_OK) return 0;
     const size_t base = pcl_conv_workspace_bytes(d, PCL_PASS_BWD_DATA);
     long rows = 0;
-    if (tensor_path_for(*d, PCL_PASS_BWD_DATA) && d->C % 4 == 0)
+    if (tensor_path_for(*d, PCL_PASS_BWD_DATA) && d->C % 4 == 0 && unit_stride(*d))
         rows = tc_fprop_colsum_rows(bwd_data_args(*d, P, Q, nullptr, nullptr, nullptr, nullptr));
     if (rows > 0) return base + colsum_stage_bytes(rows, d->C);
     const int cs = colsum_splits(size_t(d->N) * d->H * d->W);          // unfused: column sum of dx itself
@@ -501,7 +573,7 @@ int pcl_conv_bwd_data_colsum(const pcl_conv_desc* d, const float* dy, const floa
     const size_t base = pcl_conv_workspace_bytes(d, PCL_PASS_BWD_DATA);
     char* extra = static_cast<char*>(ws) + base;
     long rows = 0;
-    if (tensor_path_for(*d, PCL_PASS_BWD_DATA) && d->C % 4 == 0)
+    if (tensor_path_for(*d, PCL_PASS_BWD_DATA) && d->C % 4 == 0 && unit_stride(*d))
         rows = tc_fprop_colsum_rows(bwd_data_args(*d, P, Q, nullptr, nullptr, nullptr, nullptr));
     if (rows > 0) {
         TcFpropArgs a = bwd_data_args(*d, P, Q, dy, w, relu_mask_src, dx);
@@ -598,7 +670,7 @@ namespace {
 struct PooledWgradPlan { bool ok; int splits; size_t tiles_off, rows_off, cs_off, total; };
 PooledWgradPlan plan_pooled_wgrad(const pcl_conv_desc& d, int P, int Q) {
     PooledWgradPlan pl{};
-    if (!few_channel_path_for(d, PCL_PASS_BWD_WEIGHTS)) return pl;
+    if (!few_channel_path_for(d, PCL_PASS_BWD_WEIGHTS) || !few_taprows_form(d)) return pl;
     if (!tc_wgrad_can_take_pooled_dy(d.N, P, Q, d.S * 4, d.K, d.R, 1, 1)) return pl;
     pl.ok = true;
     pl.splits = tc_wgrad_splits(d.N, P, Q, d.S * 4, d.K, d.R, 1, 1, 1);
@@ -642,7 +714,7 @@ int pcl_conv_bwd_weights_pooled(const pcl_conv_desc* d, const float* x, const fl
     float* dw4 = reinterpret_cast<float*>(static_cast<char*>(ws) + pl.tiles_off);
     float* rows = reinterpret_cast<float*>(static_cast<char*>(ws) + pl.rows_off);
     float* cs = reinterpret_cast<float*>(static_cast<char*>(ws) + pl.cs_off);
-    rc = launch_stage_pad_c4(x, xs, d->N, d->H, d->W, d->C, d->pad_h, d->pad_w, st);
+    rc = launch_stage_pad_c4(x, xs, d->N, d->H, d->W, d->C, d->pad_h, d->pad_w, few_slack_pixels(*d), st);
     if (rc != PCL_OK) return rc;
     const int Hp = d->H + 2 * d->pad_h, Wp = d->W + 2 * d->pad_w;
     const size_t taps = size_t(d->K) * d->R * d->S;
@@ -655,7 +727,7 @@ int pcl_conv_bwd_weights_pooled(const pcl_conv_desc* d, const float* x, const fl
     a.dy_pool = dy_pool; a.codes = pool_codes; a.relu_mask = relu_mask ? 1 : 0; a.db_rows = dbias ? rows : nullptr;
     rc = launch_tc_wgrad(a, st);
     if (rc != PCL_OK) return rc;
-    rc = launch_unpad_reduce(dw4, dw, taps, d->C, pl.splits, taps * 4, st);
+    rc = launch_unpad_reduce(dw4, dw, size_t(d->K) * d->R, d->S, d->C, d->S * 4, pl.splits, taps * 4, st);
     if (rc != PCL_OK) return rc;
     if (dbias) rc = launch_colsum(rows, size_t(pl.splits) * 8, d->K, cs, dbias, st);       // adds the rows, fixed order
     return rc;
@@ -680,20 +752,36 @@ int pcl_conv_bwd_weights(const pcl_conv_desc* d, const float* x, const float* dy
         float* xs = static_cast<float*>(ws);
         float* dw4 = reinterpret_cast<float*>(static_cast<char*>(ws) + xs_bytes);
         float* cs = reinterpret_cast<float*>(static_cast<char*>(ws) + pl.partial_bytes);
-        rc = launch_stage_pad_c4(x, xs, d->N, d->H, d->W, d->C, d->pad_h, d->pad_w, st);
+        rc = launch_stage_pad_c4(x, xs, d->N, d->H, d->W, d->C, d->pad_h, d->pad_w, few_slack_pixels(*d), st);
         if (rc != PCL_OK) return rc;
         const int Hp = d->H + 2 * d->pad_h, Wp = d->W + 2 * d->pad_w;
         const size_t taps = size_t(d->K) * d->R * d->S;
-        // partial tiles always go to the workspace (splits == 1 included): dw4 is [split][K][R][S*4]
-        TcWgradArgs a{xs, dy, dw4, pl.splits > 1 ? dw4 : nullptr, d->N, Hp, Q, d->S * 4, d->K, d->R, 1, 0, 0, P, Q,
-                      pl.splits};
-        a.x_stride_w = 4; a.x_stride_h = long(Wp) * 4; a.x_stride_n = long(Hp) * Wp * 4;
-        a.x_inner = 32;
-        a.tap_groups = 1;
-        a.skip_reduce = 1;
-        rc = launch_tc_wgrad(a, st);
-        if (rc != PCL_OK) return rc;
-        rc = launch_unpad_reduce(dw4, dw, taps, d->C, pl.splits, taps * 4, st);
+        if (few_taprows_form(*d)) {
+            // partial tiles always go to the workspace (splits == 1 included): dw4 is [split][K][R][S*4]
+            TcWgradArgs a{xs, dy, dw4, pl.splits > 1 ? dw4 : nullptr, d->N, Hp, Q, d->S * 4, d->K, d->R, 1, 0, 0, P, Q,
+                          pl.splits};
+            a.x_stride_w = 4; a.x_stride_h = long(Wp) * 4; a.x_stride_n = long(Hp) * Wp * 4;
+            a.x_inner = 32;
+            a.tap_groups = 1;
+            a.skip_reduce = 1;
+            rc = launch_tc_wgrad(a, st);
+            if (rc != PCL_OK) return rc;
+            rc = launch_unpad_reduce(dw4, dw, size_t(d->K) * d->R, d->S, d->C, d->S * 4, pl.splits, taps * 4, st);
+        } else {
+            // general form: a layer with 32 "channels" per tap and an R x S' kernel whose taps lie 8 pixels apart;
+            // dw4 is [split][K][R][S'][32]
+            const int Sb = few_sblocks(*d);
+            const size_t tile = size_t(d->K) * d->R * Sb * 32;
+            TcWgradArgs a{xs, dy, dw4, pl.splits > 1 ? dw4 : nullptr, d->N, Hp, (Q - 1) * d->stride_w + 8 * (Sb - 1) + 1, 32,
+                          d->K, d->R, Sb, 0, 0, P, Q, pl.splits};
+            a.x_stride_w = 4; a.x_stride_h = long(Wp) * 4; a.x_stride_n = long(Hp) * Wp * 4;
+            a.x_inner = 32;
+            a.stride_h = d->stride_h; a.stride_w = d->stride_w; a.dil_w = 8;
+            a.skip_reduce = 1;
+            rc = launch_tc_wgrad(a, st);
+            if (rc != PCL_OK) return rc;
+            rc = launch_unpad_reduce(dw4, dw, size_t(d->K) * d->R, d->S, d->C, Sb * 32, pl.splits, tile, st);
+        }
         if (rc != PCL_OK) return rc;
         if (dbias) rc = launch_colsum(dy, size_t(d->N) * P * Q, d->K, cs, dbias, st);
         return rc;
@@ -708,6 +796,7 @@ int pcl_conv_bwd_weights(const pcl_conv_desc* d, const float* x, const float* dy
     float* cs_partial = reinterpret_cast<float*>(static_cast<char*>(ws) + (need_partial ? pl.partial_bytes : 0));
     if (pl.tensor) {
         TcWgradArgs a{x, dy, dw, partial, d->N, d->H, d->W, d->C, d->K, d->R, d->S, d->pad_h, d->pad_w, P, Q, pl.splits};
+        a.stride_h = d->stride_h; a.stride_w = d->stride_w;
         rc = launch_tc_wgrad(a, st);
     } else {
         rc = launch_generic_bwd_weights(*d, P, Q, x, dy, dw, partial, pl.splits, st);
@@ -735,7 +824,7 @@ int pcl_fc_bwd(int N, int C, int K, const float* x, const float* w, const float*
         return PCL_ERR_MISALIGNED;
     const pcl_conv_desc d{N, C, K, 1, 1, 1, 1, 1, 1, 0, 0};
     const bool dw_fwd = fc_dw_as_forward(N, C, K);
-    PassScope pass_scope(PROF_PASS_FC_BWD, 2.0 * N * double(C) * K);
+    PassScope pass_scope(PROF_PASS_FC_BWD, 2.0 * N * double(C) * K, dx ? 2 : 1);
     const size_t colsum_bytes = plan_wgrad(d, 1, 1).colsum_bytes;
     const size_t need_w = dw_fwd ? fc_dzt_bytes(N, K) + colsum_bytes : pcl_conv_workspace_bytes(&d, PCL_PASS_BWD_WEIGHTS);
     const size_t need_d = dx ? pcl_conv_workspace_bytes(&d, PCL_PASS_BWD_DATA) : 0;

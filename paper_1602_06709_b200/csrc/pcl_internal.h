@@ -37,7 +37,7 @@ struct LaunchScope {
 enum ProfPass { PROF_PASS_OTHER = 0, PROF_PASS_CONV_FWD, PROF_PASS_CONV_BWD_DATA, PROF_PASS_CONV_BWD_WEIGHTS,
                 PROF_PASS_FC_FWD, PROF_PASS_FC_BWD, PROF_PASS_COUNT };
 struct PassScope {
-    PassScope(int pass, double flops);
+    PassScope(int pass, double flops, int contraction_launches = 1);
     ~PassScope();
     PassScope(const PassScope&) = delete;
     PassScope& operator=(const PassScope&) = delete;
@@ -100,11 +100,13 @@ encode_tiled_fn get_encode_tiled();
 // (K-major operands) or, if atom32, in 32-byte chunks (MN-major operands).
 // dims/box innermost first; strides_bytes has rank-1 entries (dims 1..rank-1).
 // The element type is TFLOAT32 (TMA rounds fp32 to tf32, nearest-even, on load) unless plain_f32 (maps used for stores).
+// elem_strides (optional, rank entries): traversal stride per dimension; a dimension with stride t > 1 takes every
+// t-th element, and its box entry counts elements of the tensor (box / t elements land in shared memory).
 int make_tmap(CUtensorMap* out, const void* base, int rank, const uint64_t* dims, const uint64_t* strides_bytes,
-              const uint32_t* box, bool atom32, bool plain_f32 = false);
+              const uint32_t* box, bool atom32, bool plain_f32 = false, const uint32_t* elem_strides = nullptr);
 
-// ---- forward-type implicit GEMM on tcgen05 (stride-1 convolution) ----------
-// out[n,p,q,k] = epi( sum_{r,s,c} in[n, p + r - pad_h, q + s - pad_w, c] * wt[k, r*S+s, c] )
+// ---- forward-type implicit GEMM on tcgen05 -----------------------------------
+// out[n,p,q,k] = epi( sum_{r,s,c} in[n, p*stride_h + r - pad_h, q*stride_w + s*dil_w - pad_w, c] * wt[k, r*S+s, c] )
 // epi: + bias[k], activation, optional zeroing where mask_src[n,p,q,k] <= 0.
 struct TcFpropArgs {
     const float* in;   // [N][H][W][Cin]
@@ -141,6 +143,14 @@ struct TcFpropArgs {
     // reads B as an MN-major operand and no transposed copy is needed.  Needs Kout % 32 == 0.
     // flip_taps != 0: tap t of the loop reads tap R*S-1-t of `wt` (the spatial flip of backward-data).
     int wt_mn_major = 0, flip_taps = 0;
+    // Strides of the convolution (fetched by TMA with a traversal stride: only the pixels a tile needs are read) and
+    // the distance in pixels between consecutive taps of a kernel row (8 on the few-channel path when a kernel row
+    // is wider than one 32-float window: tap s' then covers kernel columns 8s' .. 8s'+7).  pad_h / pad_w may be
+    // negative (the phases of a strided backward-data pass).
+    int stride_h = 1, stride_w = 1, dil_w = 1;
+    // Element strides of `out` (and of mask_src) between adjacent q, p and n positions; 0 = packed NPQK.  A strided
+    // backward-data pass writes each of its phases to every stride-th pixel of dx.
+    long out_stride_w = 0, out_stride_h = 0, out_stride_n = 0;
 };
 bool tc_fprop_can_pool(const TcFpropArgs& a);
 // bytes of split_ws with which launch_tc_fprop(a) would split the reduction (0: it would not)
@@ -149,8 +159,8 @@ bool tc_fprop_eligible(const TcFpropArgs& a);
 long tc_fprop_colsum_rows(const TcFpropArgs& a);
 int launch_tc_fprop(const TcFpropArgs& a, cudaStream_t st);
 
-// ---- weight-gradient-type GEMM on tcgen05 (stride-1 convolution) -----------
-// dw[k, r, s, c] = sum_{n,p,q} dy[n,p,q,k] * x[n, p + r - pad_h, q + s - pad_w, c]
+// ---- weight-gradient-type GEMM on tcgen05 ------------------------------------
+// dw[k, r, s, c] = sum_{n,p,q} dy[n,p,q,k] * x[n, p*stride_h + r - pad_h, q*stride_w + s*dil_w - pad_w, c]
 struct TcWgradArgs {
     const float* x;   // [N][H][W][C]
     const float* dy;  // [N][P][Q][K]
@@ -176,10 +186,12 @@ struct TcWgradArgs {
     const unsigned char* codes = nullptr;
     int relu_mask = 0;
     float* db_rows = nullptr;
+    int stride_h = 1, stride_w = 1, dil_w = 1;      // as in TcFpropArgs
 };
 bool tc_wgrad_eligible(const TcWgradArgs& a);
 bool tc_wgrad_can_take_pooled_dy(int N, int P, int Q, int C, int K, int R, int S, int tap_groups);
-int tc_wgrad_splits(int N, int P, int Q, int C, int K, int R, int S, int tap_groups = 0, int pooled_dy = 0);
+int tc_wgrad_splits(int N, int P, int Q, int C, int K, int R, int S, int tap_groups = 0, int pooled_dy = 0,
+                    int strided = 0);
 int launch_tc_wgrad(const TcWgradArgs& a, cudaStream_t st);
 
 // ---- generic CUDA-core kernels (any stride / pad / channel count) ----------
@@ -200,13 +212,19 @@ int launch_reduce_splits_bias_act(const float* partial, float* out, const float*
 int launch_zero(float* p, size_t n, cudaStream_t st);
 // wt_t[c][R-1-r][S-1-s][k] = w[k][r][s][c]
 int launch_transpose_flip(const float* w, float* wt_t, int K, int R, int S, int C, cudaStream_t st);
+// One phase of a strided backward-data pass: wt_t[c][Ra-1-i][Sb-1-j][k] = w[k][a + i*stride_h][b + j*stride_w][c],
+// i < Ra, j < Sb (the taps that reach input pixels of phase (a, b), flipped and transposed).
+int launch_phase_weights(const float* w, float* wt_t, int K, int R, int S, int C, int a, int b, int stride_h,
+                         int stride_w, int Ra, int Sb, cudaStream_t st);
 // Few-channel staging (C < 4): xs[n][h+pad_h][w+pad_w][0..3] = x[n][h][w][0..C-1] padded with zeros (channel
-// padding and a spatial halo of pad_h / pad_w); w32[k][r][s*4 + c] = w[k][r][s][c] in zero-padded 32-float rows;
-// dw[k][r][s][c] = sum over splits of dw4[split][k][r][s*4 + c].
-int launch_stage_pad_c4(const float* x, float* xs, int N, int H, int W, int C, int pad_h, int pad_w, cudaStream_t st);
-int launch_stage_w4(const float* w, float* w32, size_t rows, int S, int C, cudaStream_t st);
-int launch_unpad_reduce(const float* dw4, float* dw, size_t taps, int C, int splits, size_t split_stride,
+// padding and a spatial halo of pad_h / pad_w), followed by `slack_pixels` zero pixels; w32[row][s*4 + c] =
+// w[row][s][c] (row = k*R + r) in zero-padded rows of row_floats (a multiple of 32) floats;
+// dw[row][s][c] = sum over splits of dw4[split][row][s*4 + c] with rows of row_floats floats.
+int launch_stage_pad_c4(const float* x, float* xs, int N, int H, int W, int C, int pad_h, int pad_w, int slack_pixels,
                         cudaStream_t st);
+int launch_stage_w4(const float* w, float* w32, size_t rows, int S, int C, int row_floats, cudaStream_t st);
+int launch_unpad_reduce(const float* dw4, float* dw, size_t rows, int S, int C, int row_floats, int splits,
+                        size_t split_stride, cudaStream_t st);
 // dz = dy * act'(y), in place on dy
 int launch_act_grad(float* dy, const float* y, size_t n, int act, cudaStream_t st);
 // out[k] = sum_rows m[row][k]; partial: [colsum_splits(rows)][K] workspace

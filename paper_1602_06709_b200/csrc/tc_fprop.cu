@@ -56,6 +56,8 @@ struct FpropParams {
     int tiles_q, tiles_p, tiles_n, tiles_k;
     int BN;                     // output maps per tile, multiple of 32, <= 256
     int R, S, pad_h, pad_w, cblocks;
+    int stride_h, stride_w, dil_w;      // convolution strides; pixels between consecutive taps of a kernel row
+    long long o_sw, o_sh, o_sn;         // element strides of `out` / `mask_src` between adjacent q, p, n
     int N, P, Q, Kout;
     int act;
     int stages;
@@ -512,14 +514,17 @@ tc_fprop_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                 } else {
                     // k-step order: r, then s, then channel block; a reduction split starts kps k-steps further
                     int c0 = 0, s = 0, tap = 0;
-                    int cq = q0 - p.pad_w, cp = p0 - p.pad_h;
+                    // (input coordinates of the tile's first pixel for tap (0, 0); a strided layer's box takes every
+                    // stride-th pixel from there)
+                    int cq = q0 * p.stride_w - p.pad_w, cp = p0 * p.stride_h - p.pad_h;
+                    const int dil = p.dil_w, row_back = p.S * p.dil_w;
                     if (p.ksplit > 1) {
                         const int kit0 = it.sp * kiters;
                         tap = kit0 / p.cblocks;
                         c0 = (kit0 - tap * p.cblocks) * kBlockC;
                         const int r0 = tap / p.S;
                         s = tap - r0 * p.S;
-                        cq += s; cp += r0;
+                        cq += s * dil; cp += r0;
                     }
                     for (int kit = 0; kit < kiters; kit += p.KS) {
                         if (!bounded_wait_addr(empty_a, phase ^ 1u, &abort_flag, p.status, WAIT_PRODUCER_EMPTY)) {
@@ -538,8 +543,8 @@ tc_fprop_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                             else tma_load_4d_addr<kPair>(dst + p.KS * kABytes, &tmB, full_dst, 0, kcol, c0 >> 5, tap);
                             c0 += p.KS * kBlockC;
                             if (c0 == c_end) {
-                                c0 = 0; ++tap; ++cq;
-                                if (++s == p.S) { s = 0; cq -= p.S; ++cp; }
+                                c0 = 0; ++tap; cq += dil;
+                                if (++s == p.S) { s = 0; cq -= row_back; ++cp; }
                             }
                         } else
                         for (int j = 0; j < nst; ++j, dst += step_bytes) {
@@ -548,8 +553,8 @@ tc_fprop_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                             else tma_load_3d_addr<kPair>(dst + kABytes, &tmB, full_dst, c0, tap, kcol);
                             c0 += kBlockC;
                             if (c0 == c_end) {
-                                c0 = 0; ++tap; ++cq;
-                                if (++s == p.S) { s = 0; cq -= p.S; ++cp; }
+                                c0 = 0; ++tap; cq += dil;
+                                if (++s == p.S) { s = 0; cq -= row_back; ++cp; }
                             }
                         }
                         ++issued;
@@ -621,7 +626,8 @@ tc_fprop_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
             const int pp = it.pi * p.th + ih + h * p.half_dp;
             const int n = ni * p.tn + in_;
             const bool valid = (q < p.Q) && (pp < p.P) && (n < p.N);
-            const size_t pix = (static_cast<size_t>(n) * p.P + pp) * p.Q + q;
+            // element offset of the pixel's row in `out` (packed NPQK, or every stride-th pixel of a larger tensor)
+            const size_t pix_off = static_cast<size_t>(n) * p.o_sn + static_cast<size_t>(pp) * p.o_sh + static_cast<size_t>(q) * p.o_sw;
             const uint32_t t_row = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) +
                                    ((p.split_acc ? 2 * acc : acc) * p.MT + h) * p.BN;
             const uint32_t t_second = p.MT * p.BN;      // split accumulators: the second issuer's copy of this box
@@ -745,7 +751,7 @@ tc_fprop_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
 #pragma unroll
                 for (int i = 0; i < 8; ++i) {
                     const int src = (lane >> 3) + 4 * i;
-                    roff[i] = __shfl_sync(0xffffffffu, static_cast<unsigned long long>(pix * p.Kout + sp_off), src);
+                    roff[i] = __shfl_sync(0xffffffffu, static_cast<unsigned long long>(pix_off + sp_off), src);
                     vmask |= (__shfl_sync(0xffffffffu, static_cast<int>(valid), src) ? 1u : 0u) << i;
                 }
                 const uint32_t stg = smem_u32(epi_stage + epi * 4096);
@@ -853,8 +859,8 @@ tc_fprop_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                     if (!kPool && kEpi == kEpiWarps && p.split_acc) add_second_accumulator(t_row + t_second + ch * 32, v);
                     const int col0 = kt * p.BN + ch * 32;
                     if (valid && col0 < p.Kout) {
-                        float* dst = p.out + static_cast<size_t>(it.sp) * p.split_stride + pix * p.Kout + col0;
-                        const float* msk = kMask ? p.mask_src + pix * p.Kout + col0 : nullptr;
+                        float* dst = p.out + static_cast<size_t>(it.sp) * p.split_stride + pix_off + col0;
+                        const float* msk = kMask ? p.mask_src + pix_off + col0 : nullptr;
 #pragma unroll
                         for (int j = 0; j < 32; ++j) {
                             if (col0 + j < p.Kout) {
@@ -893,12 +899,14 @@ tc_fprop_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
 // Pick the 128-pixel box bw x bh x bn (powers of two) that wastes the least
 // work on ragged edges; ties go to the widest box.
 // pool: the box must hold whole 2x2 windows inside each 32-pixel quarter (2 <= bw <= 16, bh >= 2).
-void choose_box(int P, int Q, int N, bool pool, int* bw_log2, int* bh_log2) {
+// stride_w / stride_h: a TMA box spans bw * stride_w x bh * stride_h input pixels, at most 256 each.
+void choose_box(int P, int Q, int N, bool pool, int* bw_log2, int* bh_log2, int stride_w = 1, int stride_h = 1) {
     double best = 1e300;
     int best_w = pool ? 1 : 0, best_h = pool ? 1 : 0;
     for (int lw = pool ? 4 : 7; lw >= (pool ? 1 : 0); --lw)
         for (int lh = 7 - lw; lh >= (pool ? 1 : 0); --lh) {
             const long bw = 1L << lw, bh = 1L << lh, bn = 128 / (bw * bh);
+            if (bw * stride_w > 256 || bh * stride_h > 256) continue;
             const double covered = double((Q + bw - 1) / bw * bw) * double((P + bh - 1) / bh * bh) *
                                    double((N + bn - 1) / bn * bn);
             if (covered < best) { best = covered; best_w = lw; best_h = lh; }
@@ -946,6 +954,8 @@ bool tc_fprop_eligible(const TcFpropArgs& a) {
     if (a.Cin % 4 != 0) return false;                       // TMA strides are multiples of 16 bytes
     if ((reinterpret_cast<uintptr_t>(a.in) | reinterpret_cast<uintptr_t>(a.wt)) & 15) return false;
     if (a.R * a.S > 65535) return false;
+    if (a.stride_h < 1 || a.stride_w < 1 || a.stride_h > 8 || a.stride_w > 8 || a.dil_w < 1) return false;
+    if ((a.out_stride_w | a.out_stride_h | a.out_stride_n) != 0 && (a.pool_out || a.split_ws)) return false;
     return true;
 }
 
@@ -966,7 +976,7 @@ struct TileCfg {
 
 TileCfg plain_cfg(const TcFpropArgs& a, int cblocks, int sm_count) {
     TileCfg c;
-    choose_box(a.P, a.Q, a.N, a.pool_out != nullptr, &c.bw_log2, &c.bh_log2);
+    choose_box(a.P, a.Q, a.N, a.pool_out != nullptr, &c.bw_log2, &c.bh_log2, a.stride_w, a.stride_h);
     c.tw = 1 << c.bw_log2; c.th = 1 << c.bh_log2; c.tn = kTileM / (c.tw * c.th);
     c.tiles_q = (a.Q + c.tw - 1) / c.tw; c.tiles_p = (a.P + c.th - 1) / c.th; c.tiles_n = (a.N + c.tn - 1) / c.tn;
     const long m_tiles = long(c.tiles_q) * c.tiles_p * c.tiles_n;
@@ -999,6 +1009,7 @@ TileCfg halo_cfg(const TcFpropArgs& a, int cblocks, int sm_count, int layout) {
     c.PW = c.tw + a.S - 1;
     const int PH = c.th + a.R - 1;
     if (a.R * a.S <= 1 || c.PW > 256 || PH > 256) return c;
+    if (a.stride_h != 1 || a.stride_w != 1 || a.dil_w != 1) return c;      // taps as shifted views need unit steps
     c.patch_bytes = c.PW * PH * 128;
     c.a_buf_bytes = (c.patch_bytes + 1023) / 1024 * 1024;
     c.half_off_bytes = layout == 1 ? 8 * 128 : (layout == 2 ? 16 * c.PW * 128 : 0);
@@ -1138,7 +1149,12 @@ int launch_tc_fprop(const TcFpropArgs& a, cudaStream_t st) {
     const long m_tiles = long(p.tiles_q) * p.tiles_p * p.tiles_n;
     if (m_tiles * p.tiles_k > 0x7fffffffL) return PCL_ERR_UNSUPPORTED_SHAPE;
     p.R = a.R; p.S = a.S; p.pad_h = a.pad_h; p.pad_w = a.pad_w;
+    p.stride_h = a.stride_h; p.stride_w = a.stride_w; p.dil_w = a.dil_w;
     p.N = a.N; p.P = a.P; p.Q = a.Q; p.Kout = a.Kout;
+    const bool out_strided = (a.out_stride_w | a.out_stride_h | a.out_stride_n) != 0;
+    p.o_sw = out_strided ? a.out_stride_w : a.Kout;
+    p.o_sh = out_strided ? a.out_stride_h : (long long)a.Q * a.Kout;
+    p.o_sn = out_strided ? a.out_stride_n : (long long)a.P * a.Q * a.Kout;
     p.act = a.act;
     // (not in the pooling instantiation: its epilogue has no registers to spare)
     p.split_acc = (p.issuers == 2 && 4 * p.MT * p.BN <= 512 && !a.pool_out && tune(TUNE_SPLIT_ACC, 1)) ? 1 : 0;
@@ -1172,17 +1188,18 @@ int launch_tc_fprop(const TcFpropArgs& a, cudaStream_t st) {
         const uint64_t sh = a.in_stride_h ? uint64_t(a.in_stride_h) : uint64_t(a.W) * a.Cin;
         const uint64_t sn = a.in_stride_n ? uint64_t(a.in_stride_n) : uint64_t(a.H) * a.W * a.Cin;
         const uint64_t strides[3] = {sw * 4, sh * 4, sn * 4};
-        const uint32_t box_plain[4] = {kBlockC, uint32_t(bw), uint32_t(bh), uint32_t(bn)};
+        const uint32_t box_plain[4] = {kBlockC, uint32_t(bw * a.stride_w), uint32_t(bh * a.stride_h), uint32_t(bn)};
+        const uint32_t estr[5] = {1, uint32_t(a.stride_w), uint32_t(a.stride_h), 1, 1};
         const uint32_t box_halo[4] = {kBlockC, uint32_t(p.PW), uint32_t(p.th + a.R - 1), 1};
         int rc;
         if (cfg.grp && !cfg.halo) {
             // channel blocks as a fifth dimension (128 bytes apart), so that one box spans KS of them
             const uint64_t dims5[5] = {kBlockC, uint64_t(a.W), uint64_t(a.H), uint64_t(a.N), uint64_t(p.cblocks)};
             const uint64_t strides5[4] = {sw * 4, sh * 4, sn * 4, kBlockC * 4};
-            const uint32_t box5[5] = {kBlockC, uint32_t(bw), uint32_t(bh), uint32_t(bn), uint32_t(p.KS)};
-            rc = make_tmap(&tmA, a.in, 5, dims5, strides5, box5, false);
+            const uint32_t box5[5] = {kBlockC, uint32_t(bw * a.stride_w), uint32_t(bh * a.stride_h), uint32_t(bn), uint32_t(p.KS)};
+            rc = make_tmap(&tmA, a.in, 5, dims5, strides5, box5, false, false, estr);
         } else {
-            rc = make_tmap(&tmA, a.in, 4, dims, strides, p.halo ? box_halo : box_plain, false);
+            rc = make_tmap(&tmA, a.in, 4, dims, strides, p.halo ? box_halo : box_plain, false, false, p.halo ? nullptr : estr);
         }
         if (rc != PCL_OK) return rc;
     }
@@ -1226,7 +1243,7 @@ int launch_tc_fprop(const TcFpropArgs& a, cudaStream_t st) {
         // tile and stores nothing at full resolution
         if (!a.pool_out || a.colsum_rows) return PCL_ERR_BAD_ARG;
         p.tma_store = 1;
-    } else if (tune(TUNE_TMA_STORE, 1) && !a.mask_src && !a.colsum_rows && a.Kout % 4 == 0 &&
+    } else if (tune(TUNE_TMA_STORE, 1) && !out_strided && !a.mask_src && !a.colsum_rows && a.Kout % 4 == 0 &&
         (reinterpret_cast<uintptr_t>(a.out) & 15) == 0) {
         const uint32_t bx = bw < 32 ? bw : 32, by = uint32_t(bh) < 32 / bx ? uint32_t(bh) : 32 / bx, bnn = 32 / (bx * by);
         const uint64_t dims[4] = {uint64_t(a.Kout), uint64_t(a.Q), uint64_t(a.P), uint64_t(a.N)};

@@ -71,6 +71,7 @@ struct WgradParams {
     int rpi;                  // runs per work item (rpi*L <= 8); even in pair mode
     int run_blocks;           // ceil(total_runs / rpi)
     int R, S, pad_h, pad_w;
+    int stride_h, stride_w, dil_w;   // convolution strides; pixels between consecutive taps of a kernel row
     int K, C;
     int splits, boxes_per_split;
     int stages, tmem_cols;
@@ -186,7 +187,7 @@ tc_wgrad_kernel(const __grid_constant__ CUtensorMap tmDy, const __grid_constant_
                     const int tap = run / p.runs_per_tap;
                     const int cg0 = (run - tap * p.runs_per_tap) * p.L;
                     const int r = tap / p.S, s = tap - r * p.S;
-                    run_dw[j] = s - p.pad_w;
+                    run_dw[j] = s * p.dil_w - p.pad_w;
                     run_dh[j] = r - p.pad_h;
                     run_c[j] = p.grouped ? cg0 : cg0 * 32;
                 } else {
@@ -204,6 +205,7 @@ tc_wgrad_kernel(const __grid_constant__ CUtensorMap tmDy, const __grid_constant_
             uint32_t dst = ring0;
             int sub = 0;                                         // position of the k-step inside its slot
             int q0 = qi * bw, p0 = pi * bh, n0 = ni * bn;
+            const int xsw = p.stride_w, xsh = p.stride_h;      // x coordinates of a box: the dy box's times the stride
             for (int b = box_begin; b < box_end; ++b) {
                 if (sub == 0) {
                     if (!bounded_wait_addr(empty_a, phase ^ 1u, &abort_flag, p.status, WAIT_PRODUCER_EMPTY)) { ok = false; break; }
@@ -232,14 +234,14 @@ tc_wgrad_kernel(const __grid_constant__ CUtensorMap tmDy, const __grid_constant_
 #pragma unroll
                     for (int j = 0; j < 8; ++j)
                         if (j < my_runs)
-                            tma_load_5d_addr<kPair>(xdst + j * run_bytes, &tmX, full_dst, 0, q0 + run_dw[j], p0 + run_dh[j],
-                                                    n0, run_c[j]);
+                            tma_load_5d_addr<kPair>(xdst + j * run_bytes, &tmX, full_dst, 0, q0 * xsw + run_dw[j],
+                                                    p0 * xsh + run_dh[j], n0, run_c[j]);
                 } else {
 #pragma unroll
                     for (int j = 0; j < 8; ++j)
                         if (j < my_runs)
-                            tma_load_4d_addr<kPair>(xdst + j * run_bytes, &tmX, full_dst, run_c[j], q0 + run_dw[j],
-                                                    p0 + run_dh[j], n0);
+                            tma_load_4d_addr<kPair>(xdst + j * run_bytes, &tmX, full_dst, run_c[j], q0 * xsw + run_dw[j],
+                                                    p0 * xsh + run_dh[j], n0);
                 }
                 // next pixel box
                 q0 += bw;
@@ -555,7 +557,9 @@ tc_wgrad_kernel(const __grid_constant__ CUtensorMap tmDy, const __grid_constant_
 
 // min_l: smallest log2 of the box width and height (1 for pooled dy: the box must hold whole 2x2 windows)
 // min_lw: smallest log2 of the box width alone (3 for haloed x: a box row must hold whole 8-pixel MMA steps)
-void choose_pixel_box(int pix, int P, int Q, int N, int* bw_log2, int* bh_log2, int min_l = 0, int min_lw = 0) {
+// stride_w / stride_h: the x box spans bw * stride_w x bh * stride_h input pixels, at most 256 each
+void choose_pixel_box(int pix, int P, int Q, int N, int* bw_log2, int* bh_log2, int min_l = 0, int min_lw = 0,
+                      int stride_w = 1, int stride_h = 1) {
     const int lp = pix == 64 ? 6 : 5;
     double best = 1e300;
     if (min_lw < min_l) min_lw = min_l;
@@ -563,6 +567,7 @@ void choose_pixel_box(int pix, int P, int Q, int N, int* bw_log2, int* bh_log2, 
     for (int lw = lp - min_l; lw >= min_lw; --lw)
         for (int lh = lp - lw; lh >= min_l; --lh) {
             const long bw = 1L << lw, bh = 1L << lh, bn = pix / (bw * bh);
+            if (bw * stride_w > 256 || bh * stride_h > 256) continue;
             const double covered = double((Q + bw - 1) / bw * bw) * double((P + bh - 1) / bh * bh) *
                                    double((N + bn - 1) / bn * bn);
             if (covered < best) { best = covered; best_w = lw; best_h = lh; }
@@ -582,7 +587,9 @@ struct WgradPlan {
     int xhalo, x_group_bytes;     // haloed x boxes (see the header): item = (k tile, kernel row, split)
 };
 
-WgradPlan plan_wgrad(int N, int P, int Q, int C, int K, int R, int S, int tap_groups, int pooled_dy = 0) {
+WgradPlan plan_wgrad(int N, int P, int Q, int C, int K, int R, int S, int tap_groups, int pooled_dy = 0,
+                     int stride_w = 1, int stride_h = 1, int dil_w = 1) {
+    const bool strided = stride_w != 1 || stride_h != 1 || dil_w != 1;
     WgradPlan r{};
     const int cgroups = (C + 31) / 32;
     const int k_tiles = (K + 127) / 128;
@@ -605,7 +612,7 @@ WgradPlan plan_wgrad(int N, int P, int Q, int C, int K, int R, int S, int tap_gr
     r.run_blocks = (r.total_runs + r.rpi - 1) / r.rpi;
     // Haloed x boxes for single-CTA items of layers with few input maps (all taps of a kernel row fit one
     // accumulator): the pixel box must hold whole 8-pixel runs in w.
-    if (r.grouped && !r.pair && !pooled_dy && S >= 2 && cgroups * S * 32 <= 256 && Q >= 8 && tune(TUNE_XHALO_WGRAD, 1)) {
+    if (r.grouped && !r.pair && !pooled_dy && !strided && S >= 2 && cgroups * S * 32 <= 256 && Q >= 8 && tune(TUNE_XHALO_WGRAD, 1)) {
         for (int pix = tune(TUNE_PIX_WGRAD, 64) == 64 ? 64 : 32; pix >= 32 && !r.xhalo; pix >>= 1) {
             int lw, lh;
             choose_pixel_box(pix, P, Q, N, &lw, &lh, 0, 3);
@@ -638,7 +645,7 @@ WgradPlan plan_wgrad(int N, int P, int Q, int C, int K, int R, int S, int tap_gr
     if (r.KS < 1) r.KS = 1;
     r.stages = kSmemBudget / (r.KS * r.step_bytes);
     if (r.stages > kMaxStages) r.stages = kMaxStages;
-    choose_pixel_box(r.pix, P, Q, N, &r.bw_log2, &r.bh_log2, pooled_dy ? 1 : 0);
+    choose_pixel_box(r.pix, P, Q, N, &r.bw_log2, &r.bh_log2, pooled_dy ? 1 : 0, 0, stride_w, stride_h);
     const long bw = 1L << r.bw_log2, bh = 1L << r.bh_log2, bn = r.pix / (bw * bh);
     r.boxes = ((Q + bw - 1) / bw) * ((P + bh - 1) / bh) * ((N + bn - 1) / bn);
     return r;
@@ -651,6 +658,8 @@ int sm_count() { return device_sm_count(); }
 bool tc_wgrad_eligible(const TcWgradArgs& a) {
     if (a.C % 4 != 0 || a.K % 4 != 0) return false;
     if (a.tap_groups && (a.S != 1 || a.C > 32 || a.R * 32 > 256)) return false;
+    if (a.stride_h < 1 || a.stride_w < 1 || a.stride_h > 8 || a.stride_w > 8 || a.dil_w < 1) return false;
+    if ((a.stride_h != 1 || a.stride_w != 1 || a.dil_w != 1) && (a.tap_groups || a.dy_pool)) return false;
     if ((reinterpret_cast<uintptr_t>(a.x) | reinterpret_cast<uintptr_t>(a.dy)) & 15) return false;
     return true;
 }
@@ -662,8 +671,10 @@ bool tc_wgrad_can_take_pooled_dy(int N, int P, int Q, int C, int K, int R, int S
     return !rp.pair && rp.stages * rp.KS * rp.step_bytes >= 40960;
 }
 
-int tc_wgrad_splits(int N, int P, int Q, int C, int K, int R, int S, int tap_groups, int pooled_dy) {
-    const WgradPlan rp = plan_wgrad(N, P, Q, C, K, R, S, tap_groups, pooled_dy);
+int tc_wgrad_splits(int N, int P, int Q, int C, int K, int R, int S, int tap_groups, int pooled_dy, int strided) {
+    // (the number of work items and pixel boxes does not depend on the stride values, only on whether the haloed-x
+    // form, which needs unit strides, is open)
+    const WgradPlan rp = plan_wgrad(N, P, Q, C, K, R, S, tap_groups, pooled_dy, strided ? 2 : 1, strided ? 2 : 1);
     const long items = long((K + 127) / 128) * rp.run_blocks;
     long splits = sm_count() / items;
     if (splits < 1) splits = 1;
@@ -691,7 +702,7 @@ int launch_tc_wgrad(const TcWgradArgs& a, cudaStream_t st) {
     const int pooled = a.dy_pool ? 1 : 0;
     if (pooled && (!a.codes || !tc_wgrad_can_take_pooled_dy(a.N, a.P, a.Q, a.C, a.K, a.R, a.S, a.tap_groups)))
         return PCL_ERR_UNSUPPORTED_SHAPE;
-    const WgradPlan rp = plan_wgrad(a.N, a.P, a.Q, a.C, a.K, a.R, a.S, a.tap_groups, pooled);
+    const WgradPlan rp = plan_wgrad(a.N, a.P, a.Q, a.C, a.K, a.R, a.S, a.tap_groups, pooled, a.stride_w, a.stride_h, a.dil_w);
     p.dy_pool = a.dy_pool; p.codes = a.codes; p.relu_mask = a.relu_mask; p.db_rows = pooled ? a.db_rows : nullptr;
     p.N = a.N; p.P = a.P; p.Q = a.Q;
     p.pix = rp.pix; p.bw_log2 = rp.bw_log2; p.bh_log2 = rp.bh_log2;
@@ -706,6 +717,7 @@ int launch_tc_wgrad(const TcWgradArgs& a, cudaStream_t st) {
     p.rpi = rp.rpi; p.run_blocks = rp.run_blocks;
     p.k_tiles = (a.K + 127) / 128;
     p.R = a.R; p.S = a.S; p.pad_h = a.pad_h; p.pad_w = a.pad_w;
+    p.stride_h = a.stride_h; p.stride_w = a.stride_w; p.dil_w = a.dil_w;
     p.K = a.K; p.C = a.C;
     p.splits = a.splits;
     if (p.splits < 1) return PCL_ERR_BAD_ARG;
@@ -772,15 +784,17 @@ int launch_tc_wgrad(const TcWgradArgs& a, cudaStream_t st) {
         } else if (p.grouped) {
             const uint64_t dims[5] = {32, uint64_t(a.W), uint64_t(a.H), uint64_t(a.N), uint64_t(a.C / 32)};
             const uint64_t strides[4] = {sw * 4, sh * 4, sn * 4, 128};
-            const uint32_t box[5] = {32, uint32_t(bw), uint32_t(bh), uint32_t(bn), uint32_t(p.L)};
-            int rc = make_tmap(&tmX, a.x, 5, dims, strides, box, true);
+            const uint32_t box[5] = {32, uint32_t(bw * a.stride_w), uint32_t(bh * a.stride_h), uint32_t(bn), uint32_t(p.L)};
+            const uint32_t estr[5] = {1, uint32_t(a.stride_w), uint32_t(a.stride_h), 1, 1};
+            int rc = make_tmap(&tmX, a.x, 5, dims, strides, box, true, false, estr);
             if (rc != PCL_OK) return rc;
         } else {
             const uint64_t dims[4] = {uint64_t(a.x_inner ? a.x_inner : a.C), uint64_t(a.W), uint64_t(a.H),
                                       uint64_t(a.N)};
             const uint64_t strides[3] = {sw * 4, sh * 4, sn * 4};
-            const uint32_t box[4] = {32, uint32_t(bw), uint32_t(bh), uint32_t(bn)};
-            int rc = make_tmap(&tmX, a.x, 4, dims, strides, box, true);
+            const uint32_t box[4] = {32, uint32_t(bw * a.stride_w), uint32_t(bh * a.stride_h), uint32_t(bn)};
+            const uint32_t estr[4] = {1, uint32_t(a.stride_w), uint32_t(a.stride_h), 1};
+            int rc = make_tmap(&tmX, a.x, 4, dims, strides, box, true, false, estr);
             if (rc != PCL_OK) return rc;
         }
     }

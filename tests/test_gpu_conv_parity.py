@@ -27,11 +27,23 @@ FEW_CHANNEL_SHAPES = {   # C < 4, stride 1: staged 4-channel copy + overlapping 
     "two_ch_nopad": ConvShape(N=2, C=2, K=36, H=12, W=15, R=3, S=2),
     "rgb_7x7_pad": ConvShape(N=1, C=3, K=8, H=14, W=14, R=7, S=7, pad_h=3, pad_w=1),
 }
-GENERIC_SHAPES = {
+# Strided layers on the tensor cores: forward and weight gradient fetch every stride-th pixel by TMA, backward-data
+# runs one stride-1 sub-convolution per phase of the input grid; few-channel layers with kernel rows wider than one
+# 32-float window (S > 8) take taps 8 pixels apart.
+STRIDED_SHAPES = {
     "rgb_stride4": ConvShape(N=2, C=3, K=24, H=47, W=47, R=11, S=11, stride_h=4, stride_w=4),
     "stride2": ConvShape(N=3, C=20, K=36, H=15, W=18, R=3, S=3, stride_h=2, stride_w=2, pad_h=1, pad_w=1),
-    "odd_channels": ConvShape(N=2, C=7, K=9, H=11, W=13, R=3, S=3, pad_h=1, pad_w=1),
     "mixed_stride": ConvShape(N=2, C=8, K=12, H=16, W=16, R=3, S=5, stride_h=1, stride_w=2, pad_h=0, pad_w=2),
+    "stride2_wide": ConvShape(N=4, C=64, K=96, H=30, W=34, R=3, S=3, stride_h=2, stride_w=2, pad_h=1, pad_w=1),
+    "stride3_k2": ConvShape(N=2, C=16, K=32, H=20, W=23, R=2, S=2, stride_h=3, stride_w=3),   # pixels no tap reaches
+    "stride4_k5_pad2": ConvShape(N=2, C=32, K=64, H=33, W=29, R=5, S=5, stride_h=4, stride_w=4, pad_h=2, pad_w=2),
+    "stride2x3_k3x4": ConvShape(N=2, C=24, K=40, H=26, W=31, R=3, S=4, stride_h=2, stride_w=3, pad_h=1, pad_w=2),
+    "rgb_11x11_s1": ConvShape(N=1, C=3, K=16, H=24, W=26, R=11, S=11),
+    "gray_s2": ConvShape(N=2, C=1, K=20, H=21, W=22, R=3, S=3, stride_h=2, stride_w=2, pad_h=1, pad_w=1),
+    "rgb_9x17_s2": ConvShape(N=2, C=3, K=12, H=40, W=45, R=9, S=17, stride_h=2, stride_w=2, pad_h=4, pad_w=8),
+}
+GENERIC_SHAPES = {
+    "odd_channels": ConvShape(N=2, C=7, K=9, H=11, W=13, R=3, S=3, pad_h=1, pad_w=1),
 }
 
 
@@ -43,6 +55,9 @@ def _cases():
         out.append(pytest.param(tag, s, B.PATH_GENERIC, id=f"generic-{tag}"))
     for tag, s in FEW_CHANNEL_SHAPES.items():
         out.append(pytest.param(tag, s, B.PATH_AUTO, id=f"few-{tag}"))
+        out.append(pytest.param(tag, s, B.PATH_GENERIC, id=f"generic-{tag}"))
+    for tag, s in STRIDED_SHAPES.items():
+        out.append(pytest.param(tag, s, B.PATH_TENSOR, id=f"tensor-{tag}"))     # (forced: a fallback would be refused)
         out.append(pytest.param(tag, s, B.PATH_GENERIC, id=f"generic-{tag}"))
     for tag, s in GENERIC_SHAPES.items():
         out.append(pytest.param(tag, s, B.PATH_AUTO, id=f"auto-{tag}"))
