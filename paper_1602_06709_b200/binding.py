@@ -131,13 +131,13 @@ def conv_desc(N, C, K, H, W, R, S, stride=1, pad=0, stride_w=None, pad_w=None) -
                     pad, pad if pad_w is None else pad_w)
 
 
-TILINGS = {"plain": 0, "halo0": 1, "halo1": 2, "halo2": 3}
 UNSET = -2 ** 31
+TILINGS = {"plain": 0, "halo0": 1, "halo1": 2, "halo2": 3, "auto": UNSET}      # auto: the launcher's own rule
 
 
 def set_tuning(name: str, value):
     """Pins one of the launchers' choices (see pcl_set_tuning in the header).  value None unsets the knob; the
-    TILING knob also takes the names plain / halo0 / halo1 / halo2."""
+    TILING knob also takes the names plain / halo0 / halo1 / halo2 / auto."""
     if value is None:
         value = UNSET
     elif name == "TILING" and isinstance(value, str):

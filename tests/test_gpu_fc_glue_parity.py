@@ -5,6 +5,7 @@ import pytest
 import torch
 
 import oracle
+from oracle import ConvShape
 
 pytestmark = pytest.mark.gpu
 
@@ -283,6 +284,36 @@ def test_conv_fwd_with_fused_maxpool(shape, tiling, store, monkeypatch):
             assert torch.equal(yp3, yp)
 
 
+@pytest.mark.parametrize("shape", [
+    ConvShape(N=3, C=16, K=32, H=24, W=40, R=3, S=3, stride_h=2, stride_w=2, pad_h=1, pad_w=1),
+    ConvShape(N=2, C=3, K=24, H=47, W=55, R=11, S=11, stride_h=4, stride_w=4),      # few-channel, two windows per row
+])
+def test_strided_conv_fwd_with_fused_maxpool(shape):
+    """A strided layer followed by the 2x2 pool, as one call: y against the oracle, the pooled tensor and the codes
+    bit for bit the maxima / positions of that y, with and without storing y."""
+    import gpu_helpers as G
+    from paper_1602_06709_b200 import binding as B
+    s = shape
+    assert s.P % 2 == 0 and s.Q % 2 == 0
+    x, w, _, bias = G.make_inputs(s, f"fwdpool_strided{s.C}")
+    d = G.shape_to_desc(s)
+    assert B.conv_fwd_pool_is_fused(d)
+    ws = G.workspace(B.conv_workspace_bytes(d, B.PASS_FWD))
+    y = torch.full((s.N, s.P, s.Q, s.K), float("nan"), device="cuda")
+    yp = torch.full((s.N, s.P // 2, s.Q // 2, s.K), float("nan"), device="cuda")
+    codes = torch.full((s.N, s.P // 2, s.Q // 2, s.K), 255, dtype=torch.uint8, device="cuda")
+    B.conv_fwd_pool(d, G.dev(x), G.dev(w), G.dev(bias), y, yp, B.ACT_RELU, ws, pool_codes=codes)
+    B.check_device_status()
+    G.assert_parity(y.cpu().numpy(), oracle.conv_fwd(s, x, w, bias, oracle.ACT_RELU), "y")
+    yh = y.cpu().numpy()
+    assert np.array_equal(yp.cpu().numpy(), oracle.maxpool2x2_fwd(yh.astype(np.float64)).astype(np.float32))
+    assert np.array_equal(codes.cpu().numpy(), oracle.maxpool2x2_codes(yh))
+    yp2 = torch.full_like(yp, float("nan")); codes2 = torch.full_like(codes, 255)
+    B.conv_fwd_pool(d, G.dev(x), G.dev(w), G.dev(bias), None, yp2, B.ACT_RELU, ws, pool_codes=codes2)
+    B.check_device_status()
+    assert torch.equal(yp2, yp) and torch.equal(codes2, codes)
+
+
 def test_conv_fwd_pool_rejects_odd_output():
     import gpu_helpers as G
     from oracle import ConvShape
@@ -296,15 +327,18 @@ def test_conv_fwd_pool_rejects_odd_output():
 
 
 def test_conv_fwd_pool_without_y_only_where_fused():
-    """A strided layer runs the generic convolution and a separate pooling kernel, which reads y: y is required."""
+    """A layer whose channel count is not a multiple of 4 runs the generic convolution and a separate pooling kernel,
+    which reads y: y is required.  (Strided layers are on the tensor-core path and fuse the pooling.)"""
     import gpu_helpers as G
     from oracle import ConvShape
     from paper_1602_06709_b200 import binding as B
-    s = ConvShape(N=1, C=8, K=8, H=16, W=16, R=3, S=3, stride_h=2, stride_w=2, pad_h=1, pad_w=1)
+    s = ConvShape(N=1, C=7, K=8, H=16, W=16, R=3, S=3, pad_h=1, pad_w=1)
     d = G.shape_to_desc(s)
     assert not B.conv_fwd_pool_is_fused(d)
-    x = torch.zeros(1, 16, 16, 8, device="cuda"); w = torch.zeros(8, 3, 3, 8, device="cuda")
-    yp = torch.zeros(1, 4, 4, 8, device="cuda")
+    x = torch.zeros(1, 16, 16, 7, device="cuda"); w = torch.zeros(8, 3, 3, 7, device="cuda")
+    yp = torch.zeros(1, 8, 8, 8, device="cuda")
+    s2 = ConvShape(N=1, C=8, K=8, H=16, W=16, R=3, S=3, stride_h=2, stride_w=2, pad_h=1, pad_w=1)
+    assert B.conv_fwd_pool_is_fused(G.shape_to_desc(s2))
     with pytest.raises(B.PclError) as e:
         B.conv_fwd_pool(d, x, w, None, None, yp, B.ACT_RELU, None)
     assert e.value.code == B.ERR_UNSUPPORTED_SHAPE
