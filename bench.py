@@ -159,11 +159,12 @@ class ConvWorkload:
     name = "configs[1]: VGG-A mid conv layer 3x3 s1 p1, N=256 C=K=256 56x56: fwd + bwd_data + bwd_weights + SGD update"
     unit = "TFLOP/s"
 
-    def __init__(self, rank: int, minibatch: int = 0, layer=None):
+    def __init__(self, rank: int, minibatch: int = 0, layer=None, pooled=False):
         import torch
         from paper_1602_06709_b200 import binding as B
         from paper_1602_06709_b200 import inputs
         self.torch, self.B = torch, B
+        self.pooled = pooled
         c = dict(inputs.CFG2)
         if minibatch:
             c["N"] = minibatch
@@ -182,6 +183,14 @@ class ConvWorkload:
         self.bias = torch.zeros(c["K"], device="cuda")
         self.y = torch.empty_like(self.dy); self.dx = torch.empty_like(self.x); self.dw = torch.empty_like(self.w)
         ws = max(B.conv_workspace_bytes(self.d, i) for i in range(3))
+        if pooled:      # the layer as a pooled first layer of a step: conv + ReLU + 2x2 pool in one call (y not stored),
+            # weight gradient straight from the pooled gradient and the position codes
+            assert B.conv_fwd_pool_is_fused(self.d) and B.conv_bwd_weights_pooled_is_fused(self.d)
+            ws = max(ws, B.conv_bwd_weights_pooled_workspace_bytes(self.d))
+            self.yp = torch.empty(c["N"], c["H"] // 2, c["W"] // 2, c["K"], device="cuda")
+            self.codes = torch.empty(c["N"], c["H"] // 2, c["W"] // 2, c["K"], dtype=torch.uint8, device="cuda")
+            self.dyp = self.dy[:, ::2, ::2, :].contiguous()
+            self.db = torch.empty(c["K"], device="cuda")
         self.ws = torch.empty(max(ws, 256), dtype=torch.uint8, device="cuda")
         self.flops_pass = 2 * c["N"] * c["K"] * c["H"] * c["W"] * c["C"] * 9
         self.units_per_step = 3 * self.flops_pass / 1e12      # TFLOP per step
@@ -191,6 +200,10 @@ class ConvWorkload:
 
     def step(self):
         B = self.B
+        if self.pooled:
+            B.conv_fwd_pool(self.d, self.x, self.w, self.bias, None, self.yp, B.ACT_RELU, self.ws, pool_codes=self.codes)
+            B.conv_bwd_weights_pooled(self.d, self.x, self.dyp, self.codes, True, self.dw, self.db, self.ws)
+            return
         B.conv_fwd(self.d, self.x, self.w, self.bias, self.y, B.ACT_RELU, self.ws)
         B.conv_bwd_weights(self.d, self.x, self.dy, self.dw, None, True, self.ws)
         B.conv_bwd_data(self.d, self.dy, self.w, self.x, self.dx, self.ws)
@@ -357,7 +370,7 @@ def run_ours(args):
     if args.layer and not (args.kernels_only and args.workload == "conv"):
         raise SystemExit("--layer changes the workload: only allowed with --workload conv --kernels-only")
     if args.layer:
-        wl = ConvWorkload(rank, args.minibatch, tuple(int(v) for v in args.layer.split(",")))
+        wl = ConvWorkload(rank, args.minibatch, tuple(int(v) for v in args.layer.split(",")), pooled=args.pooled)
     else:
         wl = WORKLOADS[args.workload](rank, args.minibatch)
     peaks = load_peaks()
@@ -656,6 +669,9 @@ def main():
                     help="replay the step from a CUDA graph of its launches (auto: the DNN step only)")
     ap.add_argument("--minibatch", type=int, default=0, help="override the workload's minibatch (profiling only)")
     ap.add_argument("--layer", default="", help="C,K,H of another 3x3 pad-1 layer for --workload conv (profiling only)")
+    ap.add_argument("--pooled", action="store_true",
+                    help="with --layer: run the layer as a pooled first layer (conv+pool in one call, weight gradient "
+                         "from the pooled gradient); profiling only")
     ap.add_argument("--kernels-only", action="store_true",
                     help="run warm-up + timed steps only and print a short line (for profiler captures)")
     args = ap.parse_args()

@@ -388,7 +388,7 @@ __global__ void __launch_bounds__(256) softmax_xent_kernel(const float* __restri
     }
 }
 
-// xs[n][hh][ww][0..3]: channel-padded copy of x with a zero halo of (pad_h, pad_w).  One block per padded image row
+// xs[n][hh][ww][0..3]: channel-padded, TF32-rounded copy of x with a zero halo of (pad_h, pad_w).  One block per padded image row
 // (no per-pixel index divisions: the kernel is otherwise bound by them, not by memory); the block after the last
 // row writes the trailing zero pixels (windows are read 32 floats wide, so the last ones reach past the last row).
 __global__ void __launch_bounds__(256) stage_pad_c4_kernel(const float* __restrict__ x, float4* __restrict__ xs, int N,
@@ -411,7 +411,13 @@ __global__ void __launch_bounds__(256) stage_pad_c4_kernel(const float* __restri
         const int ww = i - pad_w;
         float v[4] = {0.f, 0.f, 0.f, 0.f};
         if (ww >= 0 && ww < W)
-            for (int c = 0; c < C; ++c) v[c] = __ldg(src + size_t(ww) * C + c);
+            for (int c = 0; c < C; ++c) {
+                // rounded to TF32 (nearest even) here, once: what a TMA load through a TFLOAT32 tensor map would do to
+                // every element it fetches; the tensor-core kernels may then also copy the staged data with plain loads
+                uint32_t r;
+                asm("cvt.rn.tf32.f32 %0, %1;" : "=r"(r) : "f"(__ldg(src + size_t(ww) * C + c)));
+                v[c] = __uint_as_float(r);
+            }
         dst[i] = make_float4(v[0], v[1], v[2], v[3]);
     }
 }

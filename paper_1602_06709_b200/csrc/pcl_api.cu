@@ -39,7 +39,7 @@ std::atomic<unsigned> g_tune_gen{0};
 const char* const kTuneNames[TUNE_COUNT] = {
     "TILING", "BN", "KS", "KS_HALO", "KS_WGRAD", "PAIR", "PAIR_HALO", "PAIR_WGRAD", "GRP", "ISSUERS", "SPLIT_ACC",
     "PIX_WGRAD", "XHALO_WGRAD", "TMA_STORE", "WEIGHTS_IN_PLACE", "EPI_WARPS", "FC_DW_FORWARD", "KSPLIT",
-    "WAIT_LIMIT_US", "FAULT_INJECT"};
+    "WAIT_LIMIT_US", "FAULT_INJECT", "RESIDENT_B", "KSLICES"};
 }  // namespace
 
 int tune(int id, int dflt) {
@@ -247,7 +247,8 @@ TcFpropArgs few_fwd_args(const pcl_conv_desc& d, int P, int Q, const float* xs, 
     // declared width: one window start per reachable pixel, (Q-1)*stride_w + 8*(S'-1) being the last
     TcFpropArgs a{xs, w4, bias, nullptr, y, d.N, Hp, (Q - 1) * d.stride_w + 8 * (Sb - 1) + 1, 32, d.K, d.R, Sb, 0, 0, P, Q, act};
     a.in_stride_w = 4; a.in_stride_h = long(Wp) * 4; a.in_stride_n = long(Hp) * Wp * 4;
-    a.stride_h = d.stride_h; a.stride_w = d.stride_w; a.dil_w = 8;
+    a.stride_h = d.stride_h; a.stride_w = d.stride_w; a.dil_w = Sb > 1 ? 8 : 1;     // (one window per row: no step between taps)
+    a.k_live = Sb > 1 ? 0 : d.S * 4;      // one window per kernel row: only the first S*4 floats of it meet weights
     return a;
 }
 
@@ -776,7 +777,7 @@ int pcl_conv_bwd_weights(const pcl_conv_desc* d, const float* x, const float* dy
                           d->K, d->R, Sb, 0, 0, P, Q, pl.splits};
             a.x_stride_w = 4; a.x_stride_h = long(Wp) * 4; a.x_stride_n = long(Hp) * Wp * 4;
             a.x_inner = 32;
-            a.stride_h = d->stride_h; a.stride_w = d->stride_w; a.dil_w = 8;
+            a.stride_h = d->stride_h; a.stride_w = d->stride_w; a.dil_w = Sb > 1 ? 8 : 1;
             a.skip_reduce = 1;
             rc = launch_tc_wgrad(a, st);
             if (rc != PCL_OK) return rc;

@@ -54,7 +54,7 @@ enum TuneId {
     TUNE_TILING = 0,        // forward-type kernel: 0 plain, 1-3 haloed layouts 0-2
     TUNE_BN, TUNE_KS, TUNE_KS_HALO, TUNE_KS_WGRAD, TUNE_PAIR, TUNE_PAIR_HALO, TUNE_PAIR_WGRAD, TUNE_GRP, TUNE_ISSUERS,
     TUNE_SPLIT_ACC, TUNE_PIX_WGRAD, TUNE_XHALO_WGRAD, TUNE_TMA_STORE, TUNE_WEIGHTS_IN_PLACE, TUNE_EPI_WARPS,
-    TUNE_FC_DW_FORWARD, TUNE_KSPLIT, TUNE_WAIT_LIMIT_US, TUNE_FAULT_INJECT, TUNE_COUNT
+    TUNE_FC_DW_FORWARD, TUNE_KSPLIT, TUNE_WAIT_LIMIT_US, TUNE_FAULT_INJECT, TUNE_RESIDENT_B, TUNE_KSLICES, TUNE_COUNT
 };
 int tune(int id, int dflt);
 bool tune_is_set(int id);
@@ -119,6 +119,10 @@ struct TcFpropArgs {
     // NHWC (Cin, W*Cin, H*W*Cin).  A w stride smaller than Cin gives overlapping
     // windows (used by the few-channel first-layer path).
     long in_stride_w = 0, in_stride_h = 0, in_stride_n = 0;
+    // k_live (0 = all): how many leading elements of every 32-element channel block can be non-zero in `wt` (the
+    // few-channel path packs S taps x 4 channels into a block and zero-fills the rest): MMAs over all-zero K = 8
+    // slices are skipped.
+    int k_live = 0;
     // Innermost extent the tensor map declares (0 = Cin).  The few-channel path declares 32 although only Cin
     // elements carry weight: the rest of the window is real neighbouring data that meets zero weights, which
     // avoids TMA's slower partial-row zero fill.

@@ -437,24 +437,29 @@ __device__ __forceinline__ void umma_kstep_tf32(uint32_t d_tmem, uint32_t a_lo, 
 }
 #undef PCL_UMMA_KSTEP_BODY
 // The same with a K-major A (k-block = 2 units) and the k-block stride of B in a register (2: K-major, 64: MN-major).
+// `nsl` (1..4): how many of the four K = 8 slices are issued; the rest are known to multiply zeros only (few-channel
+// layers pack fewer than 32 live reduction elements into a block) and are skipped by a guard predicate.
 #define PCL_UMMA_KSTEP_BODY_BS(CG)                                                                                \
     asm volatile(                                                                                                 \
-        "{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\t.reg .b32 al, bl;\n\t"                                        \
+        "{\n\t.reg .pred p, q2, q3, q4;\n\t.reg .b64 da, db;\n\t.reg .b32 al, bl;\n\t"                            \
         "setp.ne.b32 p, %6, 0;\n\t"                                                                               \
+        "setp.gt.u32 q2, %8, 1;\n\tsetp.gt.u32 q3, %8, 2;\n\tsetp.gt.u32 q4, %8, 3;\n\t"                          \
         "mov.b64 da, {%1, %3};\n\tmov.b64 db, {%2, %4};\n\t"                                                      \
         "tcgen05.mma.cta_group::" CG ".kind::tf32 [%0], da, db, %5, p;\n\t"                                        \
         "setp.ne.b32 p, 1, 0;\n\t"                                                                                \
         "add.u32 al, %1, 2;\n\tadd.u32 bl, %2, %7;\n\tmov.b64 da, {al, %3};\n\tmov.b64 db, {bl, %4};\n\t"           \
-        "tcgen05.mma.cta_group::" CG ".kind::tf32 [%0], da, db, %5, p;\n\t"                                        \
+        "@q2 tcgen05.mma.cta_group::" CG ".kind::tf32 [%0], da, db, %5, p;\n\t"                                    \
         "add.u32 al, al, 2;\n\tadd.u32 bl, bl, %7;\n\tmov.b64 da, {al, %3};\n\tmov.b64 db, {bl, %4};\n\t"           \
-        "tcgen05.mma.cta_group::" CG ".kind::tf32 [%0], da, db, %5, p;\n\t"                                        \
+        "@q3 tcgen05.mma.cta_group::" CG ".kind::tf32 [%0], da, db, %5, p;\n\t"                                    \
         "add.u32 al, al, 2;\n\tadd.u32 bl, bl, %7;\n\tmov.b64 da, {al, %3};\n\tmov.b64 db, {bl, %4};\n\t"           \
-        "tcgen05.mma.cta_group::" CG ".kind::tf32 [%0], da, db, %5, p;\n\t}"                                       \
-        ::"r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(a_hi), "r"(b_hi), "r"(idesc), "r"(acc_first), "r"(b_step)        \
+        "@q4 tcgen05.mma.cta_group::" CG ".kind::tf32 [%0], da, db, %5, p;\n\t}"                                   \
+        ::"r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(a_hi), "r"(b_hi), "r"(idesc), "r"(acc_first), "r"(b_step),       \
+        "r"(nsl)                                                                                                  \
         : "memory")
 template <bool kPair>
 __device__ __forceinline__ void umma_kstep_tf32_bs(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t a_hi,
-                                                   uint32_t b_hi, uint32_t idesc, uint32_t acc_first, uint32_t b_step) {
+                                                   uint32_t b_hi, uint32_t idesc, uint32_t acc_first, uint32_t b_step,
+                                                   uint32_t nsl) {
     if constexpr (kPair) PCL_UMMA_KSTEP_BODY_BS("2");
     else PCL_UMMA_KSTEP_BODY_BS("1");
 }

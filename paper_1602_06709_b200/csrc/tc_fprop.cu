@@ -88,6 +88,13 @@ struct FpropParams {
     // out + split * split_stride (the caller adds the splits, then bias and activation).  Plain tiling only.
     int ksplit, kps;
     size_t split_stride;
+    // resident_b (haloed tiling, one k tile, few taps): the CTA's weight tiles are loaded once and stay in the ring
+    // for every tile.
+    int resident_b;
+    // K = 8 slices of a 32-element channel block that hold anything but zeros (4 unless the few-channel path packs
+    // fewer live taps x channels into a block: the MMAs of all-zero slices are not issued)
+    int kslices;
+    int bias_in_smem;           // the CTA keeps bias[0 .. BN) in shared memory (tiles_k == 1: every tile has the same columns)
     unsigned char* pool_idx;    // optional, with pool_out: per pooled element the position of the maximum (bits 0-1) and bit 2
                                 // if that maximum is <= 0
     float* pool_out;            // optional [N][P/2][Q/2][Kout]: 2x2 window maxima of the output
@@ -191,11 +198,11 @@ __device__ __forceinline__ void add_second_accumulator(uint32_t taddr, uint32_t 
 template <bool kPair, int kTaps, int kMT>
 __device__ __forceinline__ void halo_taps(uint32_t d_tmem, uint32_t BN, uint32_t& a_lo, uint32_t b_lo, int& s, int S,
                                           uint32_t row16, uint32_t half_off16, uint32_t b16, uint32_t a_hi,
-                                          uint32_t b_hi, uint32_t idesc, uint32_t& accum, uint32_t bks) {
+                                          uint32_t b_hi, uint32_t idesc, uint32_t& accum, uint32_t bks, uint32_t nsl) {
 #pragma unroll
     for (int j = 0; j < kTaps; ++j) {
-        umma_kstep_tf32_bs<kPair>(d_tmem, a_lo, b_lo, a_hi, b_hi, idesc, accum, bks);
-        if (kMT == 2) umma_kstep_tf32_bs<kPair>(d_tmem + BN, a_lo + half_off16, b_lo, a_hi, b_hi, idesc, accum, bks);
+        umma_kstep_tf32_bs<kPair>(d_tmem, a_lo, b_lo, a_hi, b_hi, idesc, accum, bks, nsl);
+        if (kMT == 2) umma_kstep_tf32_bs<kPair>(d_tmem + BN, a_lo + half_off16, b_lo, a_hi, b_hi, idesc, accum, bks, nsl);
         accum = 1;
         b_lo += b16;
         const bool wrap = ++s == S;     // the tap (r, s): next pixel of the patch, or the start of the next patch row
@@ -234,6 +241,8 @@ __device__ __noinline__ void mma_issuer(const FpropParams& p, const IssuerCtx& c
     // other (no turn at all) gave, rarely, wrong sums and lost slot releases on a 96-wide plain tiling with three
     // stages; cause not found, ordered starts are clean (40 x 40 repetitions, bit-identical).
     const bool split = kDuo && p.split_acc;
+    const bool resident = p.resident_b != 0;
+    const uint32_t nsl = uint32_t(p.kslices);      // (single issuer, haloed tiling: every tile reads the same weight slots)
     const int bmn = p.bmn;
     const uint32_t idesc = make_idesc_tf32(BN, false, bmn != 0, kPair ? 256u : 128u);
     const uint32_t bks = bmn ? 64u : 2u;         // k-block stride of B inside a k-step (16-byte units)
@@ -269,13 +278,14 @@ __device__ __noinline__ void mma_issuer(const FpropParams& p, const IssuerCtx& c
     bool mine = true;                                                                                             \
     if (kDuo) { mine = turn == issuer; turn ^= 1u; }
 #define PCL_SLOT_ACQUIRE()                                                                                        \
-    if (!bounded_wait_addr(full_a, phase, abort_flag, status, WAIT_MMA_FULL)) { ok = false; break; }             \
+    if (!(resident && tile_cnt > 0) &&                                                                            \
+        !bounded_wait_addr(full_a, phase, abort_flag, status, WAIT_MMA_FULL)) { ok = false; break; }             \
     if (kDuo && !wait_issue_turn(issue_seq, seq, abort_flag, status)) { ok = false; break; }                     \
     if (kDuo && split) *issue_seq = seq + 1;     /* split: only the slot STARTS are ordered (see below) */        \
     tc_fence_after();
 #define PCL_SLOT_RELEASE()                                                                                        \
     if (kDuo && !split) *issue_seq = seq + 1;                                                                     \
-    umma_commit_addr<kPair>(empty_a);
+    if (!resident) umma_commit_addr<kPair>(empty_a);
 #define PCL_SLOT_END()                                                                                            \
     if (kDuo) ++seq;                                                                                              \
     if (!split || mine) accum = 1;      /* split: an issuer's own first slot overwrites its own accumulator */    \
@@ -289,6 +299,7 @@ __device__ __noinline__ void mma_issuer(const FpropParams& p, const IssuerCtx& c
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + (split ? (2 * acc + issuer) * MT * BN : acc * MT * BN);
         uint32_t accum = 0;         // the tile's first MMA (whoever issues it) overwrites the accumulator
+        if (resident) { stage = 0; phase = 0; full_a = full0; empty_a = empty0; slot_lo = ring_lo0; }
         if (halo) {
             const uint64_t a_desc0 = make_smem_desc(0, 16, PW * 128, kSwizzle128B);   // 8-pixel groups are one patch row apart
             const uint32_t a_hi = uint32_t(a_desc0 >> 32);
@@ -304,20 +315,20 @@ __device__ __noinline__ void mma_issuer(const FpropParams& p, const IssuerCtx& c
                     if (mine) {
                         PCL_SLOT_ACQUIRE()
                         if (MT == 2) {
-                            if (nst == 3) halo_taps<kPair, 3, 2>(d_tmem, BN, a_lo, slot_lo, s, S, row16, half_off16, b16, a_hi, b_hi, idesc, accum, bks);
-                            else if (nst == 2) halo_taps<kPair, 2, 2>(d_tmem, BN, a_lo, slot_lo, s, S, row16, half_off16, b16, a_hi, b_hi, idesc, accum, bks);
+                            if (nst == 3) halo_taps<kPair, 3, 2>(d_tmem, BN, a_lo, slot_lo, s, S, row16, half_off16, b16, a_hi, b_hi, idesc, accum, bks, nsl);
+                            else if (nst == 2) halo_taps<kPair, 2, 2>(d_tmem, BN, a_lo, slot_lo, s, S, row16, half_off16, b16, a_hi, b_hi, idesc, accum, bks, nsl);
                             else {
                                 uint32_t b_lo = slot_lo;
                                 for (int j = 0; j < nst; ++j, b_lo += b16)
-                                    halo_taps<kPair, 1, 2>(d_tmem, BN, a_lo, b_lo, s, S, row16, half_off16, b16, a_hi, b_hi, idesc, accum, bks);
+                                    halo_taps<kPair, 1, 2>(d_tmem, BN, a_lo, b_lo, s, S, row16, half_off16, b16, a_hi, b_hi, idesc, accum, bks, nsl);
                             }
                         } else {
-                            if (nst == 3) halo_taps<kPair, 3, 1>(d_tmem, BN, a_lo, slot_lo, s, S, row16, half_off16, b16, a_hi, b_hi, idesc, accum, bks);
-                            else if (nst == 2) halo_taps<kPair, 2, 1>(d_tmem, BN, a_lo, slot_lo, s, S, row16, half_off16, b16, a_hi, b_hi, idesc, accum, bks);
+                            if (nst == 3) halo_taps<kPair, 3, 1>(d_tmem, BN, a_lo, slot_lo, s, S, row16, half_off16, b16, a_hi, b_hi, idesc, accum, bks, nsl);
+                            else if (nst == 2) halo_taps<kPair, 2, 1>(d_tmem, BN, a_lo, slot_lo, s, S, row16, half_off16, b16, a_hi, b_hi, idesc, accum, bks, nsl);
                             else {
                                 uint32_t b_lo = slot_lo;
                                 for (int j = 0; j < nst; ++j, b_lo += b16)
-                                    halo_taps<kPair, 1, 1>(d_tmem, BN, a_lo, b_lo, s, S, row16, half_off16, b16, a_hi, b_hi, idesc, accum, bks);
+                                    halo_taps<kPair, 1, 1>(d_tmem, BN, a_lo, b_lo, s, S, row16, half_off16, b16, a_hi, b_hi, idesc, accum, bks, nsl);
                             }
                         }
                         PCL_SLOT_RELEASE()
@@ -339,8 +350,8 @@ __device__ __noinline__ void mma_issuer(const FpropParams& p, const IssuerCtx& c
                 PCL_SLOT_BEGIN()
                 if (mine) {
                     PCL_SLOT_ACQUIRE()
-                    umma_kstep_tf32_bs<kPair>(d_tmem, slot_lo, slot_lo + b_off16, a_hi_plain, b_hi, idesc, accum, bks);
-                    umma_kstep_tf32_bs<kPair>(d_tmem, slot_lo + a_step16, slot_lo + b_off16 + b_step16, a_hi_plain, b_hi, idesc, 1, bks);
+                    umma_kstep_tf32_bs<kPair>(d_tmem, slot_lo, slot_lo + b_off16, a_hi_plain, b_hi, idesc, accum, bks, nsl);
+                    umma_kstep_tf32_bs<kPair>(d_tmem, slot_lo + a_step16, slot_lo + b_off16 + b_step16, a_hi_plain, b_hi, idesc, 1, bks, nsl);
                     PCL_SLOT_RELEASE()
                 }
                 PCL_SLOT_END()
@@ -353,7 +364,7 @@ __device__ __noinline__ void mma_issuer(const FpropParams& p, const IssuerCtx& c
                     PCL_SLOT_ACQUIRE()
                     uint32_t a_lo = slot_lo, b_lo = slot_lo + b_off16;
                     for (int j = 0; j < nst; ++j, a_lo += a_step16, b_lo += b_step16) {
-                        umma_kstep_tf32_bs<kPair>(d_tmem, a_lo, b_lo, a_hi_plain, b_hi, idesc, accum, bks);
+                        umma_kstep_tf32_bs<kPair>(d_tmem, a_lo, b_lo, a_hi_plain, b_hi, idesc, accum, bks, nsl);
                         accum = 1;
                     }
                     PCL_SLOT_RELEASE()
@@ -391,6 +402,7 @@ tc_fprop_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
     __shared__ uint32_t tmem_base_slot;
     __shared__ uint32_t abort_flag;
     __shared__ volatile uint32_t issue_seq;      // two issuers: number of slots whose MMAs have been issued
+    __shared__ __align__(16) float bias_s[256];  // the tile's bias values (launches whose tiles all have the same columns)
 
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
@@ -438,6 +450,8 @@ tc_fprop_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
         if constexpr (kPair) { tmem_alloc_pair(&tmem_base_slot, p.tmem_cols); tmem_relinquish_pair(); }
         else { tmem_alloc(&tmem_base_slot, p.tmem_cols); tmem_relinquish(); }
     }
+    if (kPool && p.bias_in_smem)
+        for (int i = threadIdx.x; i < 256; i += blockDim.x) bias_s[i] = (p.bias && i < p.Kout) ? __ldg(p.bias + i) : 0.f;
     tc_fence_before();
     __syncthreads();
     if constexpr (kPair) cluster_sync_all();     // the peer's barriers exist before anything signals them
@@ -485,6 +499,7 @@ tc_fprop_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                         ++issuedA;
                         if (++a_slot == p.NA) { a_slot = 0; phaseA ^= 1u; }
                         for (int tap = 0; tap < taps; tap += p.KS) {
+                            if (p.resident_b && it.t != first_tile) break;      // (loaded for the first tile, never released)
                             if (!bounded_wait_addr(empty_a, phase ^ 1u, &abort_flag, p.status, WAIT_PRODUCER_EMPTY)) {
                                 ok = false;
                                 break;
@@ -644,6 +659,88 @@ tc_fprop_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                 // consecutive pixels of the box, i.e. a sub-box whose first pixel is (sq, sp, sn).
                 const uint32_t stg = smem_u32(epi_stage + epi * 4096);
                 const int srow = quarter * 32;
+                if (kPool && !p.out && p.act != PCL_ACT_SIGMOID) {
+                    // Pooled output only (the step never reads the full-resolution output of a pooled layer).  The raw
+                    // accumulators are staged, each lane takes two windows of its four columns, adds the bias to the
+                    // four values s_e of a window, takes their maximum m and applies the activation to m alone: max
+                    // commutes with the (monotone) bias add and ReLU, so the stored maximum is bit for bit the maximum
+                    // of the finished values.  Position code: the first e with act(s_e) == act(m), i.e. with s_e == m,
+                    // except that under ReLU a window with m <= 0 holds four zeros, whose first maximum is e = 0.
+                    const int lb = p.bw_log2;
+                    const uint32_t my_row = stg + lane * 128, my_x = (lane & 7) * 16;
+                    uint32_t ld_a[2][4];
+                    size_t po_base[2];
+                    bool w_ok[2];
+#pragma unroll
+                    for (int half = 0; half < 2; ++half) {
+                        const int wdx = (lane >> 3) + 4 * half;
+                        const int r0 = ((wdx & ((1 << (lb - 1)) - 1)) << 1) | ((wdx >> (lb - 1)) << (lb + 1));
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) {
+                            const int rr = r0 | (e & 1) | ((e >> 1) << lb);
+                            ld_a[half][e] = stg + rr * 128 + (((lane & 7) ^ (rr & 7)) * 16);
+                        }
+                        const int wrow = srow + r0;
+                        const int wq = it.qi * p.tw + (wrow & (bw - 1)) + h * p.half_dq;
+                        const int wp = it.pi * p.th + ((wrow >> p.bw_log2) & (bh - 1)) + h * p.half_dp;
+                        const int wn = ni * p.tn + (wrow >> (p.bw_log2 + p.bh_log2));
+                        w_ok[half] = wq < p.Q && wp < p.P && wn < p.N;
+                        po_base[half] = ((static_cast<size_t>(wn) * (p.P >> 1) + (wp >> 1)) * (p.Q >> 1) + (wq >> 1)) * p.Kout +
+                                        kt * p.BN + (lane & 7) * 4;
+                    }
+                    const bool relu = p.act == PCL_ACT_RELU;
+                    for (int ch = ch0; ch < cpb; ch += kSub) {
+                        const int col = kt * p.BN + ch * 32 + (lane & 7) * 4;
+                        float4 b = make_float4(0.f, 0.f, 0.f, 0.f);
+                        if (p.bias_in_smem) b = *reinterpret_cast<const float4*>(bias_s + ch * 32 + (lane & 7) * 4);
+                        else if (p.bias && col < p.Kout) b = __ldg(reinterpret_cast<const float4*>(p.bias + col));
+                        if constexpr (kEpi == kEpiWarps) {
+                            uint32_t v[32];
+                            tmem_ld_32x32(t_row + ch * 32, v);
+                            tmem_ld_wait();
+                            if (p.split_acc) add_second_accumulator(t_row + t_second + ch * 32, v);
+#pragma unroll
+                            for (int j = 0; j < 8; ++j)
+                                st_shared_v4(my_row + ((j * 16) ^ my_x), __uint_as_float(v[4 * j]), __uint_as_float(v[4 * j + 1]),
+                                             __uint_as_float(v[4 * j + 2]), __uint_as_float(v[4 * j + 3]));
+                        } else {
+#pragma unroll
+                            for (int hh = 0; hh < 2; ++hh) {
+                                uint32_t v[16];
+                                tmem_ld_32x16(t_row + ch * 32 + hh * 16, v);
+                                tmem_ld_wait();
+#pragma unroll
+                                for (int jj = 0; jj < 4; ++jj)
+                                    st_shared_v4(my_row + (((hh * 4 + jj) * 16) ^ my_x), __uint_as_float(v[4 * jj]),
+                                                 __uint_as_float(v[4 * jj + 1]), __uint_as_float(v[4 * jj + 2]),
+                                                 __uint_as_float(v[4 * jj + 3]));
+                            }
+                        }
+                        __syncwarp();
+#pragma unroll
+                        for (int half = 0; half < 2; ++half) {
+                            float4 s0 = ld_shared_v4(ld_a[half][0]), s1 = ld_shared_v4(ld_a[half][1]);
+                            float4 s2 = ld_shared_v4(ld_a[half][2]), s3 = ld_shared_v4(ld_a[half][3]);
+                            auto one = [&](float a0, float a1, float a2, float a3, float bb, float& mo) -> uint32_t {
+                                a0 += bb; a1 += bb; a2 += bb; a3 += bb;
+                                const float m = fmaxf(fmaxf(a0, a1), fmaxf(a2, a3));
+                                uint32_t pos = a0 == m ? 0u : (a1 == m ? 1u : (a2 == m ? 2u : 3u));
+                                const bool nonpos = !(m > 0.f);
+                                if (relu) { mo = fmaxf(m, 0.f); pos = nonpos ? 0u : pos; } else { mo = m; }
+                                return pos | (nonpos ? 4u : 0u);
+                            };
+                            float4 m;
+                            const uint32_t c0 = one(s0.x, s1.x, s2.x, s3.x, b.x, m.x), c1 = one(s0.y, s1.y, s2.y, s3.y, b.y, m.y);
+                            const uint32_t c2 = one(s0.z, s1.z, s2.z, s3.z, b.z, m.z), c3 = one(s0.w, s1.w, s2.w, s3.w, b.w, m.w);
+                            if (w_ok[half] && col < p.Kout) {
+                                const size_t po = po_base[half] + ch * 32;
+                                *reinterpret_cast<float4*>(p.pool_out + po) = m;
+                                if (p.pool_idx) *reinterpret_cast<uint32_t*>(p.pool_idx + po) = c0 | (c1 << 8) | (c2 << 16) | (c3 << 24);
+                            }
+                        }
+                        __syncwarp();       // the staging tile is free for the next chunk
+                    }
+                } else
                 for (int ch = ch0; ch < cpb; ch += kSub) {
                     const int col0 = kt * p.BN + ch * 32;
                     // (the 8-warp variant fetches the chunk's bias ahead of the accumulator, eight vectors per lane;
@@ -1175,6 +1272,13 @@ int launch_tc_fprop(const TcFpropArgs& a, cudaStream_t st) {
     if (a.pool_out && !tc_fprop_can_pool(a)) return PCL_ERR_UNSUPPORTED_SHAPE;
     p.pool_out = a.pool_out;
     p.pool_idx = a.pool_out ? a.pool_idx : nullptr;
+    p.bias_in_smem = (a.pool_out && p.tiles_k == 1 && p.BN <= 256) ? 1 : 0;
+    {
+        const int slots = p.cblocks * ((a.R * a.S + cfg.KS - 1) / cfg.KS);
+        p.resident_b = (cfg.halo && !cfg.pair && p.issuers == 1 && p.tiles_k == 1 && !p.bmn && slots <= 3 && slots <= cfg.stages &&      // (a launch keeps at least three slots)
+                        tune(TUNE_RESIDENT_B, 1)) ? 1 : 0;
+        p.kslices = (a.k_live > 0 && a.k_live < 32 && tune(TUNE_KSLICES, 1)) ? (a.k_live + 7) / 8 : 4;
+    }
     p.colsum_rows = (a.Kout % 4 == 0) ? a.colsum_rows : nullptr;
     if (a.colsum_rows && !p.colsum_rows) return PCL_ERR_UNSUPPORTED_SHAPE;
     p.status = device_status_ptr();
