@@ -73,8 +73,11 @@ int pcl_set_path(int path);
  * has a named knob with which the tests pin each kernel variant and the alternatives were measured:
  * TILING (0 plain, 1-3 haloed layouts), BN, KS, KS_HALO, KS_WGRAD, PAIR, PAIR_HALO, PAIR_WGRAD, GRP,
  * ISSUERS, SPLIT_ACC, PIX_WGRAD, XHALO_WGRAD, TMA_STORE, WEIGHTS_IN_PLACE, EPI_WARPS, FC_DW_FORWARD,
- * KSPLIT, RESIDENT_B, KSLICES, WAIT_LIMIT_US (limit of the bounded device-side waits, microseconds), FAULT_INJECT (test
- * only, see pcl_last_device_status).  value INT_MIN unsets a knob; pcl_reset_tuning() unsets all.
+ * KSPLIT, RESIDENT_B, KSLICES, WAIT_LIMIT_US (limit of the bounded device-side waits in microseconds,
+ * default 2 s; applies to the current device), FAULT_INJECT (test only: 1 / 2 make the next forward-type /
+ * weight-gradient launch that runs as single CTAs arm its first pipeline slot for 16 bytes more than it copies,
+ * so that the waits on that slot run out, the kernel gives up and returns, and pcl_last_device_status()
+ * reports PCL_ERR_DEVICE_TIMEOUT; nothing faults and the context stays usable).  value INT_MIN unsets a knob; pcl_reset_tuning() unsets all.
  * Unset knobs take the launchers' own rules.  Process-wide; nothing is ever read from the environment.
  * Returns PCL_ERR_BAD_ARG for an unknown name. */
 int pcl_set_tuning(const char* name, int value);

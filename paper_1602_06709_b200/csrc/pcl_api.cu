@@ -13,7 +13,9 @@
 
 namespace pcl {
 
-__device__ unsigned int g_device_status = 0;
+// [0]: status word (0 = fine, else the code of the first bounded wait that ran out, or kStatusBadLabel);
+// [1]: limit of the bounded device-side waits in microseconds
+__device__ unsigned int g_device_status[2] = {0u, 2000000u};
 
 unsigned int* device_status_ptr() {
     // one copy of the symbol per device: look the address up per device, once
@@ -310,14 +312,23 @@ int pcl_set_tuning(const char* name, int value) {
             g_tune[i].value.store(value);
             g_tune[i].set.store(value == INT_MIN ? 0 : 1);
             g_tune_gen.fetch_add(1);
+            if (i == TUNE_WAIT_LIMIT_US) {       // lives in device memory next to the status word (current device)
+                const unsigned int us = (value == INT_MIN || value <= 0) ? 2000000u : static_cast<unsigned int>(value);
+                if (cudaMemcpyToSymbol(g_device_status, &us, sizeof(us), sizeof(unsigned int)) != cudaSuccess) return PCL_ERR_CUDA;
+            }
             return PCL_OK;
         }
     return PCL_ERR_BAD_ARG;
 }
 
 int pcl_reset_tuning(void) {
+    const bool had_limit = g_tune[TUNE_WAIT_LIMIT_US].set.load() != 0;
     for (int i = 0; i < TUNE_COUNT; ++i) g_tune[i].set.store(0);
     g_tune_gen.fetch_add(1);
+    if (had_limit) {
+        const unsigned int us = 2000000u;
+        if (cudaMemcpyToSymbol(g_device_status, &us, sizeof(us), sizeof(unsigned int)) != cudaSuccess) return PCL_ERR_CUDA;
+    }
     return PCL_OK;
 }
 
@@ -886,7 +897,7 @@ static std::atomic<unsigned int> g_last_wait_code{0};
 int pcl_last_device_status(void* cuda_stream) {
     if (cudaStreamSynchronize(static_cast<cudaStream_t>(cuda_stream)) != cudaSuccess) return PCL_ERR_CUDA;
     unsigned int v = 0;
-    if (cudaMemcpyFromSymbol(&v, g_device_status, sizeof(v)) != cudaSuccess) return PCL_ERR_CUDA;
+    if (cudaMemcpyFromSymbol(&v, g_device_status, sizeof(v)) != cudaSuccess) return PCL_ERR_CUDA;      // word [0]
     if (v != 0) {
         g_last_wait_code.store(v);
         const unsigned int zero = 0;

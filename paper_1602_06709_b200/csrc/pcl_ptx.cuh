@@ -38,13 +38,18 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
 }
 
 // Every wait in this library goes through here.  It polls the barrier until it
-// completes, for at most kWaitNanos of wall time (checked every 64 polls), and
+// completes, for at most the wait limit of wall time (checked every 64 polls), and
 // gives up at once if another role of the CTA has already given up.  On expiry
 // it records `code` in the device status word (0 = fine; read and cleared by
 // pcl_last_device_status()), raises the CTA's abort flag and returns false;
 // callers then leave their loops and fall through to the common teardown, so the
 // kernel always terminates.
-constexpr unsigned long long kWaitNanos = 2000000000ull;   // 2 s; real waits last micro- to milliseconds
+// The limit lives next to the status word (status_word[1], in microseconds; 2 s unless a test shortens it): it is
+// read only on the slow path, when a wait has already polled 64 times without success.
+constexpr unsigned int kDefaultWaitMicros = 2000000u;      // 2 s; real waits last micro- to milliseconds
+__device__ __forceinline__ unsigned long long wait_limit_nanos(const unsigned int* status_word) {
+    return 1000ull * *reinterpret_cast<const volatile unsigned int*>(status_word + 1);
+}
 
 __device__ __forceinline__ unsigned long long global_nanos() {
     unsigned long long t;
@@ -54,14 +59,14 @@ __device__ __forceinline__ unsigned long long global_nanos() {
 
 __device__ __forceinline__ bool bounded_wait(uint64_t* bar, uint32_t parity, volatile uint32_t* abort_flag,
                                              unsigned int* status_word, uint32_t code) {
-    unsigned long long t0 = 0;
+    unsigned long long t0 = 0, limit = 0;
     for (uint32_t spin = 0;; ++spin) {
         if (mbar_try_wait(bar, parity)) return true;
         if ((spin & 63u) == 63u) {
             if (*abort_flag) return false;
             const unsigned long long now = global_nanos();
-            if (t0 == 0) t0 = now;
-            else if (now - t0 > kWaitNanos) break;
+            if (t0 == 0) { t0 = now; limit = wait_limit_nanos(status_word); }
+            else if (now - t0 > limit) break;
             __nanosleep(64);
         }
     }
@@ -86,7 +91,7 @@ __device__ __forceinline__ bool bounded_wait_warp_relaxed(uint64_t* bar, uint32_
                                                           unsigned int* status_word, uint32_t code) {
     int ok = 1;
     if ((threadIdx.x & 31) == 0) {
-        unsigned long long t0 = 0;
+        unsigned long long t0 = 0, limit = 0;
         ok = 0;
         for (uint32_t spin = 0;; ++spin) {
             if (mbar_try_wait(bar, parity)) { ok = 1; break; }
@@ -94,8 +99,8 @@ __device__ __forceinline__ bool bounded_wait_warp_relaxed(uint64_t* bar, uint32_
             if ((spin & 15u) == 15u) {
                 if (*abort_flag) break;
                 const unsigned long long now = global_nanos();
-                if (t0 == 0) t0 = now;
-                else if (now - t0 > kWaitNanos) {
+                if (t0 == 0) { t0 = now; limit = wait_limit_nanos(status_word); }
+                else if (now - t0 > limit) {
                     *abort_flag = 1u;
                     atomicCAS(status_word, 0u, code);
                     break;
@@ -339,14 +344,14 @@ __device__ __forceinline__ bool mbar_try_wait_addr(uint32_t bar_addr, uint32_t p
 }
 static __device__ __noinline__ bool bounded_wait_slow(uint32_t bar_addr, uint32_t parity, volatile uint32_t* abort_flag,
                                                unsigned int* status_word, uint32_t code) {
-    unsigned long long t0 = 0;
+    unsigned long long t0 = 0, limit = 0;
     for (uint32_t spin = 0;; ++spin) {
         if (mbar_try_wait_addr(bar_addr, parity)) return true;
         if ((spin & 63u) == 63u) {
             if (*abort_flag) return false;
             const unsigned long long now = global_nanos();
-            if (t0 == 0) t0 = now;
-            else if (now - t0 > kWaitNanos) break;
+            if (t0 == 0) { t0 = now; limit = wait_limit_nanos(status_word); }
+            else if (now - t0 > limit) break;
             __nanosleep(64);
         }
     }

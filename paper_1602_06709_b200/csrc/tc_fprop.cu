@@ -99,7 +99,9 @@ struct FpropParams {
                                 // if that maximum is <= 0
     float* pool_out;            // optional [N][P/2][Q/2][Kout]: 2x2 window maxima of the output
     float* colsum_rows;         // optional [m_tiles * MT * 4][Kout] per-(box, quarter) column sums of the output
-    unsigned int* status;       // device status word
+    int inject_short_copy;      // test mode: the first slot is armed for 16 bytes more than are copied, so that the
+                                // waits on it run out (exercises the give-up path; single-CTA launches only)
+    unsigned int* status;       // device status word (status[1]: limit of the bounded waits in microseconds)
 };
 
 // Walks the persistent tile sequence t = blockIdx.x, blockIdx.x + gridDim.x, ... and keeps the tile's
@@ -136,14 +138,14 @@ struct TileIter {
 __device__ __forceinline__ bool wait_issue_turn(volatile uint32_t* issue_seq, uint32_t seq, volatile uint32_t* abort_flag,
                                                 unsigned int* status_word) {
     if (*issue_seq == seq) return true;
-    unsigned long long t0 = 0;
+    unsigned long long t0 = 0, limit = 0;
     for (uint32_t spin = 0;; ++spin) {
         if (*issue_seq == seq) return true;
         if ((spin & 255u) == 255u) {
             if (*abort_flag) return false;
             const unsigned long long now = global_nanos();
-            if (t0 == 0) t0 = now;
-            else if (now - t0 > kWaitNanos) break;
+            if (t0 == 0) { t0 = now; limit = wait_limit_nanos(status_word); }
+            else if (now - t0 > limit) break;
         }
     }
     *abort_flag = 1u;
@@ -548,7 +550,7 @@ tc_fprop_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                         }
                         const int nst = kiters - kit < p.KS ? kiters - kit : p.KS;
                         // pair: both CTAs' copies complete on the leader's barrier, which its producer arms
-                        if (!kPair) mbar_expect_tx_addr(full_a, nst * step_bytes);
+                        if (!kPair) mbar_expect_tx_addr(full_a, nst * step_bytes + (p.inject_short_copy && issued == 0 ? 16 : 0));
                         else if (pair_rank == 0) mbar_expect_tx_addr(full_a, 2 * nst * step_bytes);
                         uint32_t dst = slot_a;
                         if (p.grp) {
@@ -1283,6 +1285,8 @@ int launch_tc_fprop(const TcFpropArgs& a, cudaStream_t st) {
     if (a.colsum_rows && !p.colsum_rows) return PCL_ERR_UNSUPPORTED_SHAPE;
     p.status = device_status_ptr();
     if (!p.status) return PCL_ERR_CUDA;
+    // test mode (FAULT_INJECT knob = 1): only a non-pair launch in the plain tiling takes it
+    p.inject_short_copy = (tune(TUNE_FAULT_INJECT, 0) == 1 && !cfg.pair && !cfg.halo) ? 1 : 0;
 
     CUtensorMap tmA, tmB;
     {

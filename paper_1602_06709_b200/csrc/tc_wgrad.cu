@@ -93,7 +93,8 @@ struct WgradParams {
     int N, P, Q;              // output size (for the pooled tile's bounds)
     float* out;               // dw, or the partial-sum workspace [splits][K*R*S*C]
     size_t split_stride;      // K*R*S*C (0 when writing straight to dw)
-    unsigned int* status;     // device status word
+    int inject_short_copy;    // test mode: the first slot is armed for 16 bytes more than are copied (see the forward kernel)
+    unsigned int* status;     // device status word (status[1]: limit of the bounded waits in microseconds)
 };
 
 // One box row of a haloed-x k-step: kSteps MMA steps of 8 pixels, each one MMA per map group (kCg of them) over the
@@ -211,7 +212,7 @@ tc_wgrad_kernel(const __grid_constant__ CUtensorMap tmDy, const __grid_constant_
                     if (!bounded_wait_addr(empty_a, phase ^ 1u, &abort_flag, p.status, WAIT_PRODUCER_EMPTY)) { ok = false; break; }
                     const int nst = box_end - b < p.KS ? box_end - b : p.KS;
                     // pair: both CTAs' copies complete on the leader's barrier, which its producer arms
-                    if (!kPair) mbar_expect_tx_addr(full_a, nst * tx_bytes);
+                    if (!kPair) mbar_expect_tx_addr(full_a, nst * tx_bytes + (p.inject_short_copy && issued == 0 ? 16 : 0));
                     else if (pair_rank == 0) mbar_expect_tx_addr(full_a, 2 * nst * tx_bytes);
                     dst = slot_a;
                 }
@@ -729,6 +730,7 @@ int launch_tc_wgrad(const TcWgradArgs& a, cudaStream_t st) {
     while (p.tmem_cols < max_groups * 32) p.tmem_cols *= 2;
     p.status = device_status_ptr();
     if (!p.status) return PCL_ERR_CUDA;
+    p.inject_short_copy = (tune(TUNE_FAULT_INJECT, 0) == 2 && !rp.pair && !pooled) ? 1 : 0;      // test mode
     const size_t dw_elems = size_t(a.K) * a.R * a.S * a.C;
     if (p.splits == 1) {
         p.out = a.dw; p.split_stride = 0; p.use_atomics = 0;

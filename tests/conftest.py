@@ -33,3 +33,14 @@ def _tuning_knobs_do_not_leak():
     from paper_1602_06709_b200 import binding as B
     if B._lib is not None:
         B.reset_tuning()
+
+
+@pytest.fixture(autouse=True)
+def _guard_bands_intact():
+    """Outputs and workspaces allocated through gpu_helpers sit between pattern-filled bands: no kernel of the test
+    may have written outside its buffers."""
+    yield
+    import sys
+    G = sys.modules.get("gpu_helpers")
+    if G is not None and G._guards:
+        G.check_guards(clear=True)

@@ -23,8 +23,37 @@ def assert_parity(got, ref, what):
     return rel, mx
 
 
+# Guard bands: every output and workspace these helpers allocate sits between two 4 KB bands filled with a byte
+# pattern; check_guards() (called by the helpers after each call and by an autouse fixture at the end of every
+# test) asserts that no kernel wrote past either end of its buffer.
+GUARD_BYTES = 4096
+GUARD_BYTE = 0xA5
+_guards = []
+
+
+def guarded(shape, dtype=torch.float32, fill=float("nan")):
+    """A tensor of `shape` in the middle of a pattern-filled allocation (256-byte aligned)."""
+    n = int(np.prod(shape)) * torch.empty((), dtype=dtype).element_size()
+    raw = torch.full((GUARD_BYTES + n + GUARD_BYTES,), GUARD_BYTE, dtype=torch.uint8, device="cuda")
+    t = raw[GUARD_BYTES:GUARD_BYTES + n].view(dtype).view(*shape)
+    if fill is not None:
+        t.fill_(fill)
+    _guards.append((raw, n))
+    return t
+
+
+def check_guards(clear=False):
+    torch.cuda.synchronize()
+    for raw, n in _guards:
+        lo, hi = raw[:GUARD_BYTES], raw[GUARD_BYTES + n:]
+        assert bool((lo == GUARD_BYTE).all()), "a kernel wrote in front of its buffer"
+        assert bool((hi == GUARD_BYTE).all()), "a kernel wrote past the end of its buffer"
+    if clear:
+        _guards.clear()
+
+
 def workspace(nbytes):
-    return torch.empty(max(nbytes, 256), dtype=torch.uint8, device="cuda") if nbytes else None
+    return guarded((max(nbytes, 256),), torch.uint8, fill=None) if nbytes else None
 
 
 def shape_to_desc(s: ConvShape):
@@ -39,29 +68,32 @@ def make_inputs(s: ConvShape, tag, kind="unit"):
 
 def run_conv_fwd(s, x, w, bias, act):
     d = shape_to_desc(s)
-    y = torch.full((s.N, s.P, s.Q, s.K), float("nan"), device="cuda")
+    y = guarded((s.N, s.P, s.Q, s.K))
     B.conv_fwd(d, dev(x), dev(w), None if bias is None else dev(bias), y, act,
                workspace(B.conv_workspace_bytes(d, B.PASS_FWD)))
     B.check_device_status()
+    check_guards()
     return y.cpu().numpy()
 
 
 def run_conv_bwd_data(s, dy, w, mask):
     d = shape_to_desc(s)
-    dx = torch.full((s.N, s.H, s.W, s.C), float("nan"), device="cuda")
+    dx = guarded((s.N, s.H, s.W, s.C))
     B.conv_bwd_data(d, dev(dy), dev(w), None if mask is None else dev(mask), dx,
                     workspace(B.conv_workspace_bytes(d, B.PASS_BWD_DATA)))
     B.check_device_status()
+    check_guards()
     return dx.cpu().numpy()
 
 
 def run_conv_bwd_weights(s, x, dy, want_db, deterministic=True):
     d = shape_to_desc(s)
-    dw = torch.full((s.K, s.R, s.S, s.C), float("nan"), device="cuda")
-    db = torch.full((s.K,), float("nan"), device="cuda") if want_db else None
+    dw = guarded((s.K, s.R, s.S, s.C))
+    db = guarded((s.K,)) if want_db else None
     B.conv_bwd_weights(d, dev(x), dev(dy), dw, db, deterministic,
                        workspace(B.conv_workspace_bytes(d, B.PASS_BWD_WEIGHTS)))
     B.check_device_status()
+    check_guards()
     return dw.cpu().numpy(), (db.cpu().numpy() if want_db else None)
 
 

@@ -5,6 +5,7 @@ import numpy as np
 import pytest
 import torch
 
+import gpu_helpers as G
 import oracle
 from oracle import ConvShape
 
@@ -358,8 +359,8 @@ def test_weight_gradient_from_pooled_gradient(tag, relu, path_guard):
     ws = G.workspace(B.conv_bwd_weights_pooled_workspace_bytes(d))
     outs = []
     for _ in range(2):
-        dw = torch.full((s.K, s.R, s.S, s.C), float("nan"), device="cuda")
-        db = torch.full((s.K,), float("nan"), device="cuda")
+        dw = G.guarded((s.K, s.R, s.S, s.C))
+        db = G.guarded((s.K,))
         B.conv_bwd_weights_pooled(d, G.dev(x), G.dev(dyp), torch.from_numpy(codes).cuda(), relu, dw, db, ws)
         B.check_device_status()
         outs.append((dw.cpu().numpy(), db.cpu().numpy()))
@@ -367,7 +368,7 @@ def test_weight_gradient_from_pooled_gradient(tag, relu, path_guard):
     G.assert_parity(outs[0][1], db_ref, "db from pooled dy")
     assert np.array_equal(outs[0][0], outs[1][0]) and np.array_equal(outs[0][1], outs[1][1])
     # without the bias gradient
-    dw2 = torch.full((s.K, s.R, s.S, s.C), float("nan"), device="cuda")
+    dw2 = G.guarded((s.K, s.R, s.S, s.C))
     B.conv_bwd_weights_pooled(d, G.dev(x), G.dev(dyp), torch.from_numpy(codes).cuda(), relu, dw2, None, ws)
     B.check_device_status()
     assert np.array_equal(dw2.cpu().numpy(), outs[0][0])

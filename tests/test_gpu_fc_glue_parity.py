@@ -4,6 +4,7 @@ import numpy as np
 import pytest
 import torch
 
+import gpu_helpers as G
 import oracle
 from oracle import ConvShape
 
@@ -48,7 +49,7 @@ def test_fc_fwd_bwd(N, C, K, act, path, path_guard, monkeypatch):
     b = inputs.uniform(tid("b"), (K,), -0.5, 0.5)
     dy = inputs.normal(tid("dy"), (N, K), 1.0)
     xt, wt, bt = G.dev(x), G.dev(w), G.dev(b)
-    yt = torch.full((N, K), float("nan"), device="cuda")
+    yt = G.guarded((N, K))
     B.fc_fwd(N, C, K, xt, wt, bt, yt, code)
     B.check_device_status()
     y = yt.cpu().numpy()
@@ -58,16 +59,16 @@ def test_fc_fwd_bwd(N, C, K, act, path, path_guard, monkeypatch):
     for ks in ("0", "2", "3", "5"):
         B.set_tuning("KSPLIT", ks)
         ws_f = G.workspace(B.fc_workspace_bytes(N, C, K, B.PASS_FWD))
-        yt2 = torch.full((N, K), float("nan"), device="cuda")
+        yt2 = G.guarded((N, K))
         B.fc_fwd(N, C, K, xt, wt, bt, yt2, code, ws_f)
         B.check_device_status()
         G.assert_parity(yt2.cpu().numpy(), oracle.fc_fwd(x, w, b, code), f"fc fwd, KSPLIT={ks}")
     B.set_tuning("KSPLIT", None)
     # backward is checked on the GPU's own forward output (per-call parity)
     dyt = G.dev(dy)
-    dxt = torch.full((N, C), float("nan"), device="cuda")
-    dwt = torch.full((K, C), float("nan"), device="cuda")
-    dbt = torch.full((K,), float("nan"), device="cuda")
+    dxt = G.guarded((N, C))
+    dwt = G.guarded((K, C))
+    dbt = G.guarded((K,))
     ws = G.workspace(B.fc_workspace_bytes(N, C, K, B.PASS_BWD_DATA))
     B.fc_bwd(N, C, K, xt, wt, yt, code, dyt, dxt, dwt, dbt, ws)
     B.check_device_status()
@@ -122,10 +123,10 @@ def test_maxpool(N, H, W, C):
     x = np.maximum(inputs.normal(inputs.tensor_id("pool", N, H, W, C, "x"), (N, H, W, C), 1.0), 0.0)  # post-ReLU: has ties at 0
     dy = inputs.normal(inputs.tensor_id("pool", N, H, W, C, "dy"), (N, H // 2, W // 2, C), 1.0)
     xt, dyt = G.dev(x), G.dev(dy)
-    yt = torch.full((N, H // 2, W // 2, C), float("nan"), device="cuda")
+    yt = G.guarded((N, H // 2, W // 2, C))
     B.maxpool2x2_fwd(N, H, W, C, xt, yt)
     assert np.array_equal(yt.cpu().numpy(), oracle.maxpool2x2_fwd(x).astype(np.float32))
-    dxt = torch.full((N, H, W, C), float("nan"), device="cuda")
+    dxt = G.guarded((N, H, W, C))
     B.maxpool2x2_bwd(N, H, W, C, xt, dyt, None, dxt)
     assert np.array_equal(dxt.cpu().numpy(), oracle.maxpool2x2_bwd(x, dy).astype(np.float32))
     B.maxpool2x2_bwd(N, H, W, C, xt, dyt, xt, dxt)
@@ -140,8 +141,8 @@ def test_softmax_xent(N, K):
     z = inputs.normal(inputs.tensor_id("xent", N, K, "z"), (N, K), 3.0)
     lab = inputs.labels(inputs.tensor_id("xent", N, K, "lab"), N, K)
     zt = G.dev(z); lt = torch.from_numpy(lab).cuda()
-    loss = torch.full((1,), float("nan"), device="cuda")
-    dz = torch.full((N, K), float("nan"), device="cuda")
+    loss = G.guarded((1,))
+    dz = G.guarded((N, K))
     B.softmax_xent(N, K, zt, lt, loss, dz)
     loss_ref, dz_ref = oracle.softmax_xent(z, lab)
     assert abs(loss.item() - loss_ref) <= 1e-5 * max(1.0, abs(loss_ref))
@@ -160,8 +161,8 @@ def test_softmax_xent_label_outside_the_classes_is_reported_and_never_used_as_an
     lab = np.array([3, -1, K, 17, K + 1000, 0], dtype=np.int32)
     good = (lab >= 0) & (lab < K)
     zt = G.dev(z); lt = torch.from_numpy(lab).cuda()
-    loss = torch.full((1,), float("nan"), device="cuda")
-    dz = torch.full((N, K), float("nan"), device="cuda")
+    loss = G.guarded((1,))
+    dz = G.guarded((N, K))
     assert B.last_device_status() == B.OK
     B.softmax_xent(N, K, zt, lt, loss, dz)
     assert B.last_device_status() == B.ERR_BAD_LABEL
@@ -183,8 +184,8 @@ def test_maxpool_bwd_with_fused_column_sums(N, H, W, C):
     x = np.maximum(inputs.normal(inputs.tensor_id("poolcs", N, H, W, C, "x"), (N, H, W, C), 1.0), 0.0)
     dy = inputs.normal(inputs.tensor_id("poolcs", N, H, W, C, "dy"), (N, H // 2, W // 2, C), 1.0)
     xt, dyt = G.dev(x), G.dev(dy)
-    dxt = torch.full((N, H, W, C), float("nan"), device="cuda")
-    cs = torch.full((C,), float("nan"), device="cuda")
+    dxt = G.guarded((N, H, W, C))
+    cs = G.guarded((C,))
     ws = G.workspace(B.maxpool2x2_bwd_colsum_workspace_bytes(N, H, W, C))
     B.maxpool2x2_bwd_colsum(N, H, W, C, xt, dyt, xt, dxt, cs, ws)
     ref = oracle.maxpool2x2_bwd(x, dy, x)
@@ -207,8 +208,8 @@ def test_conv_bwd_data_with_fused_column_sums(shape, tiling, monkeypatch):
     s = ConvShape(N=N, C=C, K=K, H=H, W=W, R=3, S=3, pad_h=1, pad_w=1)
     x, w, dy, _ = G.make_inputs(s, f"dgradcs{C}")
     d = G.shape_to_desc(s)
-    dx = torch.full((N, H, W, C), float("nan"), device="cuda")
-    cs = torch.full((C,), float("nan"), device="cuda")
+    dx = G.guarded((N, H, W, C))
+    cs = G.guarded((C,))
     ws = G.workspace(B.conv_bwd_data_colsum_workspace_bytes(d))
     B.conv_bwd_data_colsum(d, G.dev(dy), G.dev(w), G.dev(x), dx, cs, ws)
     B.check_device_status()
@@ -255,10 +256,10 @@ def test_conv_fwd_with_fused_maxpool(shape, tiling, store, monkeypatch):
     x, w, _, bias = G.make_inputs(s, f"fwdpool{C}_{K}")
     d = G.shape_to_desc(s)
     for act, oact in ((B.ACT_RELU, oracle.ACT_RELU), (B.ACT_NONE, oracle.ACT_NONE)):
-        y = torch.full((N, H, W, K), float("nan"), device="cuda")
-        yp = torch.full((N, H // 2, W // 2, K), float("nan"), device="cuda")
+        y = G.guarded((N, H, W, K))
+        yp = G.guarded((N, H // 2, W // 2, K))
         ws = G.workspace(B.conv_workspace_bytes(d, B.PASS_FWD))
-        codes = torch.full((N, H // 2, W // 2, K), 255, dtype=torch.uint8, device="cuda")
+        codes = G.guarded((N, H // 2, W // 2, K), torch.uint8, fill=255)
         B.conv_fwd_pool(d, G.dev(x), G.dev(w), G.dev(bias), y, yp, act, ws, pool_codes=codes)
         B.check_device_status()
         G.assert_parity(y.cpu().numpy(), oracle.conv_fwd(s, x, w, bias, oact), "y")
@@ -267,7 +268,7 @@ def test_conv_fwd_with_fused_maxpool(shape, tiling, store, monkeypatch):
         # the position codes route a gradient exactly as the pooling backward pass does from the y this call wrote
         g = inputs_normal(("fwdpool_g", N, H, W, K), (N, H // 2, W // 2, K))
         for relu in (False, True):
-            dx = torch.full((N, H, W, K), float("nan"), device="cuda")
+            dx = G.guarded((N, H, W, K))
             B.maxpool2x2_bwd_codes(N, H, W, K, codes, G.dev(g), relu, dx)
             ref = oracle.maxpool2x2_bwd(yh, g, yh if relu else None)
             assert np.array_equal(dx.cpu().numpy(), ref.astype(np.float32))
@@ -299,9 +300,9 @@ def test_strided_conv_fwd_with_fused_maxpool(shape):
     d = G.shape_to_desc(s)
     assert B.conv_fwd_pool_is_fused(d)
     ws = G.workspace(B.conv_workspace_bytes(d, B.PASS_FWD))
-    y = torch.full((s.N, s.P, s.Q, s.K), float("nan"), device="cuda")
-    yp = torch.full((s.N, s.P // 2, s.Q // 2, s.K), float("nan"), device="cuda")
-    codes = torch.full((s.N, s.P // 2, s.Q // 2, s.K), 255, dtype=torch.uint8, device="cuda")
+    y = G.guarded((s.N, s.P, s.Q, s.K))
+    yp = G.guarded((s.N, s.P // 2, s.Q // 2, s.K))
+    codes = G.guarded((s.N, s.P // 2, s.Q // 2, s.K), torch.uint8, fill=255)
     B.conv_fwd_pool(d, G.dev(x), G.dev(w), G.dev(bias), y, yp, B.ACT_RELU, ws, pool_codes=codes)
     B.check_device_status()
     G.assert_parity(y.cpu().numpy(), oracle.conv_fwd(s, x, w, bias, oracle.ACT_RELU), "y")
@@ -357,19 +358,19 @@ def test_maxpool_with_position_codes(N, H, W, C):
     x = np.maximum(inputs.normal(inputs.tensor_id("poolcodes", N, H, W, C, "x"), (N, H, W, C), 1.0), 0.0)  # ties at 0
     dy = inputs.normal(inputs.tensor_id("poolcodes", N, H, W, C, "dy"), (N, H // 2, W // 2, C), 1.0)
     xt, dyt = G.dev(x), G.dev(dy)
-    yt = torch.full((N, H // 2, W // 2, C), float("nan"), device="cuda")
-    codes = torch.full((N, H // 2, W // 2, C), 255, dtype=torch.uint8, device="cuda")
+    yt = G.guarded((N, H // 2, W // 2, C))
+    codes = G.guarded((N, H // 2, W // 2, C), torch.uint8, fill=255)
     B.maxpool2x2_fwd_codes(N, H, W, C, xt, yt, codes)
     assert np.array_equal(yt.cpu().numpy(), oracle.maxpool2x2_fwd(x).astype(np.float32))
     assert int(codes.max()) <= 7
     for relu in (False, True):
-        dxt = torch.full((N, H, W, C), float("nan"), device="cuda")
+        dxt = G.guarded((N, H, W, C))
         B.maxpool2x2_bwd_codes(N, H, W, C, codes, dyt, relu, dxt)
         ref = oracle.maxpool2x2_bwd(x, dy, x if relu else None)
         assert np.array_equal(dxt.cpu().numpy(), ref.astype(np.float32))
-    cs = torch.full((C,), float("nan"), device="cuda")
+    cs = G.guarded((C,))
     ws = G.workspace(B.maxpool2x2_bwd_colsum_workspace_bytes(N, H, W, C))
-    dxt = torch.full((N, H, W, C), float("nan"), device="cuda")
+    dxt = G.guarded((N, H, W, C))
     B.maxpool2x2_bwd_codes(N, H, W, C, codes, dyt, True, dxt, cs, ws)
     ref = oracle.maxpool2x2_bwd(x, dy, x)
     assert np.array_equal(dxt.cpu().numpy(), ref.astype(np.float32))

@@ -5,6 +5,8 @@ failure, so each shape is launched several times and compared with itself."""
 import pytest
 import torch
 
+import gpu_helpers as G
+
 pytestmark = pytest.mark.gpu
 
 SHAPES = [
@@ -59,8 +61,8 @@ def test_forward_with_pool_repeats_bit_for_bit(name, N, C, K, H):
     ws = torch.empty(max(256, B.conv_workspace_bytes(d, B.PASS_FWD)), dtype=torch.uint8, device="cuda")
     ref = None
     for i in range(8):
-        yp = torch.full((N, H // 2, H // 2, K), float("nan"), device="cuda")
-        codes = torch.full((N, H // 2, H // 2, K), 255, dtype=torch.uint8, device="cuda")
+        yp = G.guarded((N, H // 2, H // 2, K))
+        codes = G.guarded((N, H // 2, H // 2, K), torch.uint8, fill=255)
         y = torch.empty(N, H, H, K, device="cuda") if i % 2 else None
         B.conv_fwd_pool(d, x, w, b, y, yp, B.ACT_RELU, ws, pool_codes=codes)
         B.check_device_status()
@@ -85,8 +87,8 @@ def test_first_layer_weight_gradient_from_pooled_gradient_repeats_bit_for_bit():
     ws = torch.empty(max(256, B.conv_bwd_weights_pooled_workspace_bytes(d)), dtype=torch.uint8, device="cuda")
     ref = None
     for _ in range(10):
-        dw = torch.full((K, 3, 3, C), float("nan"), device="cuda")
-        db = torch.full((K,), float("nan"), device="cuda")
+        dw = G.guarded((K, 3, 3, C))
+        db = G.guarded((K,))
         B.conv_bwd_weights_pooled(d, x, dyp, codes, True, dw, db, ws)
         B.check_device_status()
         if ref is None:

@@ -12,6 +12,7 @@ import numpy as np
 import pytest
 import torch
 
+import gpu_helpers as G
 import oracle
 from oracle import ConvShape
 
@@ -29,7 +30,7 @@ def test_noalloc_matches_regular_entry_point_twice():
         assert B.conv_workspace_bytes(d, B.PASS_BWD_DATA) > 0, "the case must be one that needs scratch"
         x, w, dy, _ = G.make_inputs(s, f"noalloc{call}")
         dyt, wt, xt = G.dev(dy), G.dev(w), G.dev(x)
-        ref = torch.full((s.N, s.H, s.W, s.C), float("nan"), device="cuda")
+        ref = G.guarded((s.N, s.H, s.W, s.C))
         B.conv_bwd_data(d, dyt, wt, xt, ref, G.workspace(B.conv_workspace_bytes(d, B.PASS_BWD_DATA)))
         for rep in range(2):                                 # two calls in a row share the built-in array
             got = torch.full_like(ref, float("nan"))
@@ -53,7 +54,7 @@ def test_noalloc_capacity_counts_only_the_transposed_copy():
         d = G.shape_to_desc(s)
         x, w, dy, _ = G.make_inputs(s, f"noalloc_cap{s.C}")
         dyt, wt = G.dev(dy), G.dev(w)
-        ref = torch.full((s.N, s.H, s.W, s.C), float("nan"), device="cuda")
+        ref = G.guarded((s.N, s.H, s.W, s.C))
         B.conv_bwd_data(d, dyt, wt, None, ref, torch.empty(cap, dtype=torch.uint8, device="cuda"))
         for rep in range(2):
             got = torch.full_like(ref, float("nan"))
