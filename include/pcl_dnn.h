@@ -203,6 +203,17 @@ int pcl_fc_bwd(int N, int C, int K, const float* x, const float* w, const float*
                float* dy, float* dx, float* dw, float* dbias,
                void* ws, size_t ws_bytes, void* cuda_stream);
 
+/* pcl_fc_bwd() with the layer below's share of the work folded into the backpropagation kernel's epilogue
+ * (the paper has no counterpart; same update rules, Sec. 2.1):
+ *   dx[n,c]      = (sum_k dz[n,k] * w[k,c]) * x_act'(x[n,c])   x_act = the activation that produced x (NONE, RELU:
+ *                  [x > 0], SIGMOID: x(1-x)): dx is then the gradient w.r.t. the pre-activation of the layer
+ *                  below, i.e. the dz that layer's own call would otherwise form with a pass of its own;
+ *   dx_colsum[c] = sum_n dx[n,c]   (NULL to skip): with x_act set, the bias gradient of the layer below.
+ * The layer below is then called with act = PCL_ACT_NONE and dbias = NULL.  Deterministic.  Workspace as pcl_fc_bwd(). */
+int pcl_fc_bwd_fused(int N, int C, int K, const float* x, const float* w, const float* y, int act,
+                     float* dy, float* dx, int x_act, float* dx_colsum, float* dw, float* dbias,
+                     void* ws, size_t ws_bytes, void* cuda_stream);
+
 /* Vanilla SGD (Sec. 1: algorithm and hyper-parameters untouched):
  *   w[i] <- w[i] - lr * dw[i],  i < n.   w, dw only need 4-byte alignment. */
 int pcl_sgd_update(float* w, const float* dw, size_t n, float lr, void* cuda_stream);

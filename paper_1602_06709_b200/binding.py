@@ -30,7 +30,7 @@ EXPORTS = [
     "pcl_conv_bwd_data_colsum_workspace_bytes", "pcl_conv_bwd_data_colsum",
     "pcl_maxpool2x2_bwd_colsum_workspace_bytes", "pcl_maxpool2x2_bwd_colsum", "pcl_conv_fwd_pool", "pcl_conv_fwd_pool_is_fused",
     "pcl_conv_bwd_weights_pooled", "pcl_conv_bwd_weights_pooled_is_fused", "pcl_conv_bwd_weights_pooled_workspace_bytes",
-    "pcl_maxpool2x2_fwd_codes", "pcl_maxpool2x2_bwd_codes", "pcl_last_wait_code", "pcl_set_tuning", "pcl_reset_tuning",
+    "pcl_maxpool2x2_fwd_codes", "pcl_maxpool2x2_bwd_codes", "pcl_last_wait_code", "pcl_set_tuning", "pcl_reset_tuning", "pcl_fc_bwd_fused",
 ]
 
 
@@ -83,6 +83,7 @@ def lib() -> ctypes.CDLL:
         L.pcl_conv_bwd_weights.argtypes = [dp, vp, vp, vp, vp, ci, vp, sz, vp]
         L.pcl_fc_fwd.argtypes = [ci, ci, ci, vp, vp, vp, vp, ci, vp, sz, vp]
         L.pcl_fc_bwd.argtypes = [ci, ci, ci, vp, vp, vp, ci, vp, vp, vp, vp, vp, sz, vp]
+        L.pcl_fc_bwd_fused.argtypes = [ci, ci, ci, vp, vp, vp, ci, vp, vp, ci, vp, vp, vp, vp, sz, vp]
         L.pcl_sgd_update.argtypes = [vp, vp, sz, cf, vp]
         L.pcl_maxpool2x2_fwd.argtypes = [ci, ci, ci, ci, vp, vp, vp]
         L.pcl_maxpool2x2_bwd.argtypes = [ci, ci, ci, ci, vp, vp, vp, vp, vp]
@@ -273,6 +274,14 @@ def fc_bwd(N, C, K, x, w, y, act, dy, dx, dw, dbias, ws=None, stream=None):
     wp, wb = _ws(ws)
     _check(lib().pcl_fc_bwd(N, C, K, _ptr(x), _ptr(w), _ptr(y), act, _ptr(dy), _ptr(dx), _ptr(dw), _ptr(dbias),
                             wp, wb, _stream(stream)), "pcl_fc_bwd")
+
+
+def fc_bwd_fused(N, C, K, x, w, y, act, dy, dx, x_act, dx_colsum, dw, dbias, ws=None, stream=None):
+    """fc_bwd with the gradient of the activation that produced x (x_act) and the column sums of dx (the bias
+    gradient of the layer below) formed in the backpropagation kernel's epilogue."""
+    wp, wb = _ws(ws)
+    _check(lib().pcl_fc_bwd_fused(N, C, K, _ptr(x), _ptr(w), _ptr(y), act, _ptr(dy), _ptr(dx), x_act, _ptr(dx_colsum),
+                                  _ptr(dw), _ptr(dbias), wp, wb, _stream(stream)), "pcl_fc_bwd_fused")
 
 
 def sgd_update(w, dw, lr, stream=None):

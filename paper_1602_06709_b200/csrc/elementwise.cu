@@ -388,6 +388,73 @@ __global__ void __launch_bounds__(256) softmax_xent_kernel(const float* __restri
     }
 }
 
+// The same for rows of at most 256 * kPer values: the row is read once and kept in registers (the three passes of the
+// kernel above re-read it from L1/L2), thread t holding elements t, t + 256, ...
+template <int kPer>
+__global__ void __launch_bounds__(256) softmax_xent_regs_kernel(const float* __restrict__ logits,
+                                                                const int* __restrict__ labels, float* __restrict__ loss,
+                                                                float* __restrict__ dlogits, int N, int K,
+                                                                unsigned int* __restrict__ status) {
+    __shared__ float red[8];
+    __shared__ float bcast;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    for (int n = blockIdx.x; n < N; n += gridDim.x) {
+        const float* z = logits + size_t(n) * K;
+        float v[kPer];
+        float mx = -INFINITY;
+#pragma unroll
+        for (int i = 0; i < kPer; ++i) {
+            const int k = i * 256 + threadIdx.x;
+            v[i] = k < K ? __ldg(z + k) : -INFINITY;
+            mx = fmaxf(mx, v[i]);
+        }
+        for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+        if (lane == 0) red[warp] = mx;
+        __syncthreads();
+        if (warp == 0) {
+            float t = lane < 8 ? red[lane] : -INFINITY;
+            for (int o = 4; o > 0; o >>= 1) t = fmaxf(t, __shfl_xor_sync(0xffffffffu, t, o));
+            if (lane == 0) bcast = t;
+        }
+        __syncthreads();
+        mx = bcast;
+        int lab = labels[n];
+        if (lab < 0 || lab >= K) {
+            if (threadIdx.x == 0) atomicCAS(status, 0u, static_cast<unsigned int>(kStatusBadLabel));
+            lab = -1;
+        }
+        float sum = 0.f, zlab = 0.f;
+#pragma unroll
+        for (int i = 0; i < kPer; ++i) {
+            const int k = i * 256 + threadIdx.x;
+            if (k == lab) zlab = v[i];
+            v[i] = k < K ? expf(v[i] - mx) : 0.f;
+            sum += v[i];
+        }
+        for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
+        __syncthreads();
+        if (lane == 0) red[warp] = sum;
+        __syncthreads();
+        if (warp == 0) {
+            float t = lane < 8 ? red[lane] : 0.f;
+            for (int o = 4; o > 0; o >>= 1) t += __shfl_xor_sync(0xffffffffu, t, o);
+            if (lane == 0) bcast = t;
+        }
+        __syncthreads();
+        sum = bcast;
+        const float inv_n = 1.f / float(N), inv_sum = 1.f / sum;
+        float* out = dlogits + size_t(n) * K;
+#pragma unroll
+        for (int i = 0; i < kPer; ++i) {
+            const int k = i * 256 + threadIdx.x;
+            if (k < K) out[k] = (v[i] * inv_sum - (k == lab ? 1.f : 0.f)) * inv_n;
+        }
+        // (the thread that holds the labelled element adds the row's loss term)
+        if (lab >= 0 && (lab & 255) == int(threadIdx.x)) atomicAdd(loss, -(zlab - mx - logf(sum)) * inv_n);
+        __syncthreads();
+    }
+}
+
 // xs[n][hh][ww][0..3]: channel-padded, TF32-rounded copy of x with a zero halo of (pad_h, pad_w).  One block per padded image row
 // (no per-pixel index divisions: the kernel is otherwise bound by them, not by memory); the block after the last
 // row writes the trailing zero pixels (windows are read 32 floats wide, so the last ones reach past the last row).
@@ -698,7 +765,10 @@ int launch_softmax_xent(int N, int K, const float* logits, const int* labels, fl
         LaunchScope scope(KID_SOFTMAX_XENT, 8.0 * double(N) * K, st);
         unsigned int* status = device_status_ptr();
         if (!status) return PCL_ERR_CUDA;
-        softmax_xent_kernel<<<N < 8 * device_sm_count() ? N : 8 * device_sm_count(), 256, 0, st>>>(logits, labels, loss, dlogits, N, K, status);
+        const int grid = N < 8 * device_sm_count() ? N : 8 * device_sm_count();
+        if (K <= 256 * 8) softmax_xent_regs_kernel<8><<<grid, 256, 0, st>>>(logits, labels, loss, dlogits, N, K, status);
+        else if (K <= 256 * 32) softmax_xent_regs_kernel<32><<<grid, 256, 0, st>>>(logits, labels, loss, dlogits, N, K, status);
+        else softmax_xent_kernel<<<grid, 256, 0, st>>>(logits, labels, loss, dlogits, N, K, status);
     }
     return PCL_CHECK_LAUNCH();
 }

@@ -386,7 +386,8 @@ size_t pcl_fc_workspace_bytes(int N, int C, int K, int pass) {
     // sized for either of its two forms)
     const size_t wgrad_form = pcl_conv_workspace_bytes(&d, PCL_PASS_BWD_WEIGHTS);
     const size_t fwd_form = fc_dzt_bytes(N, K) + plan_wgrad(d, 1, 1).colsum_bytes;
-    return pcl_conv_workspace_bytes(&d, PCL_PASS_BWD_DATA) + (wgrad_form > fwd_form ? wgrad_form : fwd_form);
+    // (backward-data sized for its form with fused column sums, which contains the plain form)
+    return pcl_conv_bwd_data_colsum_workspace_bytes(&d) + (wgrad_form > fwd_form ? wgrad_form : fwd_form);
 }
 
 // Forward pass; y_pool != nullptr: also the 2x2 window maxima of y, fused into the tensor-core epilogue where
@@ -567,6 +568,65 @@ size_t pcl_conv_bwd_data_colsum_workspace_bytes(const pcl_conv_desc* d) {
     return base + (cs > 1 ? align_up(size_t(cs) * d->C * 4, 256) : 0);
 }
 
+namespace {
+// Backward-data with the gradient of the activation that produced `mask` folded into the epilogue (mask_mode 0: ReLU,
+// 1: sigmoid) and, if dx_colsum != nullptr, the per-map sums of what was written.  Workspace layout as
+// pcl_conv_bwd_data_colsum_workspace_bytes() describes.
+int bwd_data_masked_colsum(const pcl_conv_desc* d, int P, int Q, const float* dy, const float* w, const float* mask,
+                           int mask_mode, float* dx, float* dx_colsum, void* ws, size_t ws_bytes, void* cuda_stream) {
+    const size_t need = dx_colsum ? pcl_conv_bwd_data_colsum_workspace_bytes(d) : bwd_data_transposed_bytes(*d);
+    if (need > 0) {
+        if (!ws || ws_bytes < need) return PCL_ERR_WORKSPACE;
+        if (reinterpret_cast<uintptr_t>(ws) & 255) return PCL_ERR_MISALIGNED;
+    }
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    const size_t base = pcl_conv_workspace_bytes(d, PCL_PASS_BWD_DATA);
+    const bool tensor = tensor_path_for(*d, PCL_PASS_BWD_DATA) && unit_stride(*d);
+    int rc;
+    if (tensor) {
+        long rows = 0;
+        if (dx_colsum && d->C % 4 == 0) rows = tc_fprop_colsum_rows(bwd_data_args(*d, P, Q, nullptr, nullptr, nullptr, nullptr));
+        TcFpropArgs a = bwd_data_args(*d, P, Q, dy, w, mask, dx);
+        a.mask_mode = mask_mode;
+        if (!a.wt_mn_major) {
+            float* wt_t = static_cast<float*>(ws);
+            rc = launch_transpose_flip(w, wt_t, d->K, d->R, d->S, d->C, st);
+            if (rc != PCL_OK) return rc;
+            a.wt = wt_t;
+        }
+        if (rows > 0) {
+            char* extra = static_cast<char*>(ws) + base;
+            float* sum_rows = reinterpret_cast<float*>(extra);
+            a.colsum_rows = sum_rows;
+            // rows the chosen tiling does not write must not contribute: the sizing took the largest tiling
+            rc = launch_zero(sum_rows, size_t(rows) * d->C, st);
+            if (rc != PCL_OK) return rc;
+            rc = launch_tc_fprop(a, st);
+            if (rc != PCL_OK) return rc;
+            float* partial = reinterpret_cast<float*>(extra + align_up(size_t(rows) * d->C * 4, 256));
+            return launch_colsum(sum_rows, size_t(rows), d->C, partial, dx_colsum, st);
+        }
+        if (!dx_colsum && !mask && ws && ws_bytes > bwd_data_transposed_bytes(*d)) {      // room to split a long reduction
+            const size_t t = bwd_data_transposed_bytes(*d);
+            a.split_ws = reinterpret_cast<float*>(static_cast<char*>(ws) + t); a.split_ws_bytes = ws_bytes - t;
+        }
+        rc = launch_tc_fprop(a, st);
+        if (rc != PCL_OK) return rc;
+    } else {
+        // other kernel families: backward-data with the ReLU mask they know, any other gradient as a pass over dx
+        rc = pcl_conv_bwd_data(d, dy, w, mask_mode == 0 ? mask : nullptr, dx, ws, base, cuda_stream);
+        if (rc != PCL_OK) return rc;
+        if (mask && mask_mode == 1) {
+            rc = launch_act_grad(dx, mask, size_t(d->N) * d->H * d->W * d->C, PCL_ACT_SIGMOID, st);
+            if (rc != PCL_OK) return rc;
+        }
+    }
+    if (!dx_colsum) return PCL_OK;
+    char* extra = static_cast<char*>(ws) + base;
+    return launch_colsum(dx, size_t(d->N) * d->H * d->W, d->C, reinterpret_cast<float*>(extra), dx_colsum, st);
+}
+}  // namespace
+
 int pcl_conv_bwd_data_colsum(const pcl_conv_desc* d, const float* dy, const float* w, const float* relu_mask_src,
                              float* dx, float* dx_colsum, void* ws, size_t ws_bytes, void* cuda_stream) {
     int P, Q;
@@ -576,38 +636,7 @@ int pcl_conv_bwd_data_colsum(const pcl_conv_desc* d, const float* dy, const floa
     PassScope pass_scope(PROF_PASS_CONV_BWD_DATA, conv_pass_flops(*d, P, Q));
     if (!aligned16(dy) || !aligned16(w) || !aligned16(dx) || !aligned16(relu_mask_src) || !aligned16(dx_colsum))
         return PCL_ERR_MISALIGNED;
-    const size_t need = pcl_conv_bwd_data_colsum_workspace_bytes(d);
-    if (need > 0) {
-        if (!ws || ws_bytes < need) return PCL_ERR_WORKSPACE;
-        if (reinterpret_cast<uintptr_t>(ws) & 255) return PCL_ERR_MISALIGNED;
-    }
-    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
-    const size_t base = pcl_conv_workspace_bytes(d, PCL_PASS_BWD_DATA);
-    char* extra = static_cast<char*>(ws) + base;
-    long rows = 0;
-    if (tensor_path_for(*d, PCL_PASS_BWD_DATA) && d->C % 4 == 0 && unit_stride(*d))
-        rows = tc_fprop_colsum_rows(bwd_data_args(*d, P, Q, nullptr, nullptr, nullptr, nullptr));
-    if (rows > 0) {
-        TcFpropArgs a = bwd_data_args(*d, P, Q, dy, w, relu_mask_src, dx);
-        if (!a.wt_mn_major) {
-            float* wt_t = static_cast<float*>(ws);
-            rc = launch_transpose_flip(w, wt_t, d->K, d->R, d->S, d->C, st);
-            if (rc != PCL_OK) return rc;
-            a.wt = wt_t;
-        }
-        float* sum_rows = reinterpret_cast<float*>(extra);
-        a.colsum_rows = sum_rows;
-        // rows the chosen tiling does not write must not contribute: the sizing took the largest tiling
-        rc = launch_zero(sum_rows, size_t(rows) * d->C, st);
-        if (rc != PCL_OK) return rc;
-        rc = launch_tc_fprop(a, st);
-        if (rc != PCL_OK) return rc;
-        float* partial = reinterpret_cast<float*>(extra + align_up(size_t(rows) * d->C * 4, 256));
-        return launch_colsum(sum_rows, size_t(rows), d->C, partial, dx_colsum, st);
-    }
-    rc = pcl_conv_bwd_data(d, dy, w, relu_mask_src, dx, ws, base, cuda_stream);
-    if (rc != PCL_OK) return rc;
-    return launch_colsum(dx, size_t(d->N) * d->H * d->W, d->C, reinterpret_cast<float*>(extra), dx_colsum, st);
+    return bwd_data_masked_colsum(d, P, Q, dy, w, relu_mask_src, 0, dx, dx_colsum, ws, ws_bytes, cuda_stream);
 }
 
 size_t pcl_maxpool2x2_bwd_colsum_workspace_bytes(int N, int H, int W, int C) {
@@ -825,21 +854,27 @@ int pcl_fc_fwd(int N, int C, int K, const float* x, const float* w, const float*
     return pcl_conv_fwd(&d, x, w, bias, y, act, ws, ws_bytes, cuda_stream);
 }
 
-int pcl_fc_bwd(int N, int C, int K, const float* x, const float* w, const float* y, int act, float* dy, float* dx,
-               float* dw, float* dbias, void* ws, size_t ws_bytes, void* cuda_stream) {
+namespace {
+bool known_act(int act) { return act == PCL_ACT_NONE || act == PCL_ACT_RELU || act == PCL_ACT_SIGMOID; }
+
+int fc_bwd_impl(int N, int C, int K, const float* x, const float* w, const float* y, int act, float* dy, float* dx,
+                int x_act, float* dx_colsum, float* dw, float* dbias, void* ws, size_t ws_bytes, void* cuda_stream) {
     if (N <= 0 || C <= 0 || K <= 0) return PCL_ERR_BAD_ARG;
     if (!x || !w || !dy || !dw) return PCL_ERR_BAD_ARG;
-    if (act != PCL_ACT_NONE && act != PCL_ACT_RELU && act != PCL_ACT_SIGMOID) return PCL_ERR_BAD_ARG;
+    if (!known_act(act) || !known_act(x_act)) return PCL_ERR_BAD_ARG;
     if (act != PCL_ACT_NONE && !y) return PCL_ERR_BAD_ARG;
+    if (!dx && dx_colsum) return PCL_ERR_BAD_ARG;
     if (!aligned16(x) || !aligned16(w) || !aligned16(y) || !aligned16(dy) || !aligned16(dx) || !aligned16(dw) ||
-        !aligned16(dbias))
+        !aligned16(dbias) || !aligned16(dx_colsum))
         return PCL_ERR_MISALIGNED;
     const pcl_conv_desc d{N, C, K, 1, 1, 1, 1, 1, 1, 0, 0};
     const bool dw_fwd = fc_dw_as_forward(N, C, K);
     PassScope pass_scope(PROF_PASS_FC_BWD, 2.0 * N * double(C) * K, dx ? 2 : 1);
     const size_t colsum_bytes = plan_wgrad(d, 1, 1).colsum_bytes;
     const size_t need_w = dw_fwd ? fc_dzt_bytes(N, K) + colsum_bytes : pcl_conv_workspace_bytes(&d, PCL_PASS_BWD_WEIGHTS);
-    const size_t need_d = dx ? pcl_conv_workspace_bytes(&d, PCL_PASS_BWD_DATA) : 0;
+    const bool fused_dx = dx && (x_act != PCL_ACT_NONE || dx_colsum);
+    const size_t need_d = !dx ? 0 : (dx_colsum ? pcl_conv_bwd_data_colsum_workspace_bytes(&d)
+                                               : pcl_conv_workspace_bytes(&d, PCL_PASS_BWD_DATA));
     if (need_w + need_d > 0) {
         if (!ws || ws_bytes < need_w + need_d) return PCL_ERR_WORKSPACE;
         if (reinterpret_cast<uintptr_t>(ws) & 255) return PCL_ERR_MISALIGNED;
@@ -861,8 +896,24 @@ int pcl_fc_bwd(int N, int C, int K, const float* x, const float* w, const float*
         rc = pcl_conv_bwd_weights(&d, x, dy, dw, dbias, 1, ws, need_w, cuda_stream);
     }
     if (rc != PCL_OK) return rc;
-    if (dx) rc = pcl_conv_bwd_data(&d, dy, w, nullptr, dx, static_cast<char*>(ws) + need_w, need_d, cuda_stream);
-    return rc;
+    if (!dx) return PCL_OK;
+    char* ws_d = static_cast<char*>(ws) + need_w;
+    if (!fused_dx) return pcl_conv_bwd_data(&d, dy, w, nullptr, dx, ws_d, need_d, cuda_stream);
+    // dx = (dz w) times the gradient of the activation that produced x: what the layer below needs as its dz
+    return bwd_data_masked_colsum(&d, 1, 1, dy, w, x_act == PCL_ACT_NONE ? nullptr : x, x_act == PCL_ACT_SIGMOID ? 1 : 0, dx,
+                                  dx_colsum, ws_d, need_d, cuda_stream);
+}
+}  // namespace
+
+int pcl_fc_bwd(int N, int C, int K, const float* x, const float* w, const float* y, int act, float* dy, float* dx,
+               float* dw, float* dbias, void* ws, size_t ws_bytes, void* cuda_stream) {
+    return fc_bwd_impl(N, C, K, x, w, y, act, dy, dx, PCL_ACT_NONE, nullptr, dw, dbias, ws, ws_bytes, cuda_stream);
+}
+
+int pcl_fc_bwd_fused(int N, int C, int K, const float* x, const float* w, const float* y, int act, float* dy, float* dx,
+                     int x_act, float* dx_colsum, float* dw, float* dbias, void* ws, size_t ws_bytes,
+                     void* cuda_stream) {
+    return fc_bwd_impl(N, C, K, x, w, y, act, dy, dx, x_act, dx_colsum, dw, dbias, ws, ws_bytes, cuda_stream);
 }
 
 int pcl_sgd_update(float* w, const float* dw, size_t n, float lr, void* cuda_stream) {

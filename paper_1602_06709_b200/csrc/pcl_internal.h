@@ -112,13 +112,16 @@ struct TcFpropArgs {
     const float* in;   // [N][H][W][Cin]
     const float* wt;   // [Kout][R*S][Cin]
     const float* bias; // [Kout] or null
-    const float* mask_src; // [N][P][Q][Kout] or null
+    const float* mask_src; // [N][P][Q][Kout] or null (see mask_mode)
     float* out;        // [N][P][Q][Kout]; may be null with pool_out (nothing is stored at full resolution)
     int N, H, W, Cin, Kout, R, S, pad_h, pad_w, P, Q, act;
     // Element strides of `in` between adjacent w, h and n positions; 0 = packed
     // NHWC (Cin, W*Cin, H*W*Cin).  A w stride smaller than Cin gives overlapping
     // windows (used by the few-channel first-layer path).
     long in_stride_w = 0, in_stride_h = 0, in_stride_n = 0;
+    // What mask_src does: 0 = the output is zeroed where mask_src <= 0 (gradient of the ReLU that produced mask_src);
+    // 1 = the output is multiplied by mask_src * (1 - mask_src) (gradient of the sigmoid that produced mask_src).
+    int mask_mode = 0;
     // k_live (0 = all): how many leading elements of every 32-element channel block can be non-zero in `wt` (the
     // few-channel path packs S taps x 4 channels into a block and zero-fills the rest): MMAs over all-zero K = 8
     // slices are skipped.

@@ -81,6 +81,8 @@ struct FpropParams {
     int half_dq, half_dp;       // pixel offset of the second box inside the tile
     const float* bias;
     const float* mask_src;
+    int mask_mode;              // what mask_src does to the output: 0 zero where mask_src <= 0 (ReLU gradient),
+                                // 1 multiply by mask_src * (1 - mask_src) (sigmoid gradient, mask_src being the sigmoid's output)
     float* out;
     int tma_store;              // the epilogue writes `out` with TMA stores from the staging tiles (tmOut is valid)
     // Split reduction (few tiles, long reduction: the FC layers at small minibatch): ksplit > 1 cuts the k-steps of
@@ -902,8 +904,13 @@ tc_fprop_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                                     o.z = 1.f / (1.f + __expf(-o.z)); o.w = 1.f / (1.f + __expf(-o.w));
                                 }
                                 if (kMask) {
-                                    o.x = mk[i].x > 0.f ? o.x : 0.f; o.y = mk[i].y > 0.f ? o.y : 0.f;
-                                    o.z = mk[i].z > 0.f ? o.z : 0.f; o.w = mk[i].w > 0.f ? o.w : 0.f;
+                                    if (p.mask_mode == 0) {
+                                        o.x = mk[i].x > 0.f ? o.x : 0.f; o.y = mk[i].y > 0.f ? o.y : 0.f;
+                                        o.z = mk[i].z > 0.f ? o.z : 0.f; o.w = mk[i].w > 0.f ? o.w : 0.f;
+                                    } else {
+                                        o.x *= mk[i].x * (1.f - mk[i].x); o.y *= mk[i].y * (1.f - mk[i].y);
+                                        o.z *= mk[i].z * (1.f - mk[i].z); o.w *= mk[i].w * (1.f - mk[i].w);
+                                    }
                                 }
                                 *reinterpret_cast<float4*>(p.out + roff[i] + col) = o;
                                 csum.x += o.x; csum.y += o.y; csum.z += o.z; csum.w += o.w;
@@ -967,7 +974,10 @@ tc_fprop_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                                 if (p.bias) o += __ldg(p.bias + col0 + j);
                                 if (p.act == PCL_ACT_RELU) o = fmaxf(o, 0.f);
                                 else if (p.act == PCL_ACT_SIGMOID) o = 1.f / (1.f + __expf(-o));
-                                if (msk && !(__ldg(msk + j) > 0.f)) o = 0.f;
+                                if (msk) {
+                                    const float m = __ldg(msk + j);
+                                    o = p.mask_mode == 0 ? (m > 0.f ? o : 0.f) : o * (m * (1.f - m));
+                                }
                                 dst[j] = o;
                             }
                         }
@@ -1260,6 +1270,7 @@ int launch_tc_fprop(const TcFpropArgs& a, cudaStream_t st) {
     p.tmem_cols = 32;
     while (p.tmem_cols < (p.split_acc ? 4 : 2) * p.MT * p.BN) p.tmem_cols *= 2;
     p.bias = a.bias; p.mask_src = a.mask_src; p.out = a.out;
+    p.mask_mode = a.mask_mode;
     // split reduction: raw partial tiles to the caller's scratch, bias and activation after the splits are added
     p.ksplit = 1; p.kps = 0; p.split_stride = 0;
     if (a.split_ws) {

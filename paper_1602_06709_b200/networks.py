@@ -241,9 +241,11 @@ class VggA(_HostFeed):
             C, K = self.fcs[j]
             a = self.fc_out[j - 1] if j > 0 else self.pooled[-1].view(self.N, self.flat)
             dx = self.fc_dout[j - 1] if j > 0 else self.dpooled[-1].view(self.N, self.flat)
-            act = B.ACT_RELU if j + 1 < nfc else B.ACT_NONE
-            B.fc_bwd(self.N, C, K, a, self.fc_w(j), self.fc_out[j], act, self.fc_dout[j], dx, self.fc_dw(j),
-                     self.fc_db(j), self.ws)
+            # fc_dout[j] already is dz_j: the softmax gradient for the last layer, and for the others the layer above
+            # folded this layer's ReLU gradient and bias gradient into its backpropagation kernel
+            B.fc_bwd_fused(self.N, C, K, a, self.fc_w(j), None, B.ACT_NONE, self.fc_dout[j], dx,
+                           B.ACT_RELU if j > 0 else B.ACT_NONE, self.fc_db(j - 1) if j > 0 else None, self.fc_dw(j),
+                           self.fc_db(j) if j + 1 == nfc else None, self.ws)
         for i in reversed(range(len(self.convs))):
             L = self.convs[i]
             # The bias gradient of layer i is the per-map sum of dy[i]; it is formed by whichever kernel writes
@@ -322,8 +324,10 @@ class Dnn(_HostFeed):
             C, K = self.layers[j]
             a = self.out[j - 1] if j > 0 else self.x
             dx = self.dout[j - 1] if j > 0 else None          # first layer: no backpropagation
-            act = B.ACT_SIGMOID if j + 1 < n else B.ACT_NONE
-            B.fc_bwd(self.N, C, K, a, self.w(j), self.out[j], act, self.dout[j], dx, self.dw(j), self.db(j), self.ws)
+            # dout[j] already is dz_j (the softmax gradient, or formed by the layer above together with db_j)
+            B.fc_bwd_fused(self.N, C, K, a, self.w(j), None, B.ACT_NONE, self.dout[j], dx,
+                           B.ACT_SIGMOID if j > 0 else B.ACT_NONE, self.db(j - 1) if j > 0 else None, self.dw(j),
+                           self.db(j) if j + 1 == n else None, self.ws)
 
     def update(self):
         B.sgd_update(self.store.params, self.store.grads, self.lr)

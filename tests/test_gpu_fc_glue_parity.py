@@ -133,7 +133,7 @@ def test_maxpool(N, H, W, C):
     assert np.array_equal(dxt.cpu().numpy(), oracle.maxpool2x2_bwd(x, dy, x).astype(np.float32))
 
 
-@pytest.mark.parametrize("N,K", [(4, 10), (37, 1000), (256, 1000), (64, 8192), (1, 3)])
+@pytest.mark.parametrize("N,K", [(4, 10), (37, 1000), (256, 1000), (64, 8192), (1, 3), (5, 2048), (5, 2049), (3, 9000)])
 def test_softmax_xent(N, K):
     import gpu_helpers as G
     from paper_1602_06709_b200 import binding as B
@@ -148,6 +148,41 @@ def test_softmax_xent(N, K):
     assert abs(loss.item() - loss_ref) <= 1e-5 * max(1.0, abs(loss_ref))
     G.assert_parity(dz.cpu().numpy(), dz_ref, "dlogits")
     np.testing.assert_allclose(dz.cpu().numpy(), dz_ref, rtol=1e-4, atol=1e-8)
+
+
+@pytest.mark.parametrize("x_act", ["none", "relu", "sigmoid"])
+@pytest.mark.parametrize("N,C,K", [(96, 960, 264), (130, 440, 200), (64, 96, 520), (256, 2048, 2048), (33, 36, 40), (8, 30, 12)])
+def test_fc_bwd_fused_epilogue(N, C, K, x_act, path_guard):
+    """pcl_fc_bwd_fused: backpropagation with the gradient of the activation that produced x and the column sums of dx
+    (the layer below's dz and bias gradient) formed in the kernel's epilogue, against the oracle's chain rule."""
+    from paper_1602_06709_b200 import binding as B
+    from paper_1602_06709_b200 import inputs
+    code = {"none": B.ACT_NONE, "relu": B.ACT_RELU, "sigmoid": B.ACT_SIGMOID}[x_act]
+    pre = inputs.normal(inputs.tensor_id("fcf", N, C, K, "pre"), (N, C), 1.0).astype(np.float64)
+    x = {"none": pre, "relu": np.maximum(pre, 0.0), "sigmoid": 1.0 / (1.0 + np.exp(-pre))}[x_act].astype(np.float32)
+    w = inputs.normal(inputs.tensor_id("fcf", N, C, K, "w"), (K, C), (1.0 / C) ** 0.5)
+    dz = inputs.normal(inputs.tensor_id("fcf", N, C, K, "dz"), (N, K), 1.0)
+    xt, wt = G.dev(x), G.dev(w)
+    for want_cs in (True, False):
+        dzt = G.dev(dz)
+        dx = G.guarded((N, C)); dw = G.guarded((K, C)); db = G.guarded((K,))
+        cs = G.guarded((C,)) if want_cs else None
+        ws = G.workspace(B.fc_workspace_bytes(N, C, K, B.PASS_BWD_DATA))
+        B.fc_bwd_fused(N, C, K, xt, wt, None, B.ACT_NONE, dzt, dx, code, cs, dw, db, ws)
+        B.check_device_status()
+        G.check_guards()
+        _, dx_ref, dw_ref, db_ref = oracle.fc_bwd(x, w, None, dz, oracle.ACT_NONE, dz_dtype=np.float32)
+        xd = x.astype(np.float64)
+        g = {"none": 1.0, "relu": (xd > 0).astype(np.float64), "sigmoid": xd * (1.0 - xd)}[x_act]
+        G.assert_parity(dx.cpu().numpy(), dx_ref * g, f"dx times {x_act}'")
+        G.assert_parity(dw.cpu().numpy(), dw_ref, "dw")
+        G.assert_parity(db.cpu().numpy(), db_ref, "db")
+        if want_cs:
+            # the sums are of the values the kernel wrote (per-call parity of the reduction itself)
+            G.assert_parity(cs.cpu().numpy(), dx.cpu().numpy().astype(np.float64).sum(axis=0), "column sums of dx")
+            cs2 = G.guarded((C,)); dx2 = G.guarded((N, C))
+            B.fc_bwd_fused(N, C, K, xt, wt, None, B.ACT_NONE, G.dev(dz), dx2, code, cs2, dw, db, ws)
+            assert torch.equal(cs, cs2) and torch.equal(dx, dx2), "fused sums must be bitwise reproducible"
 
 
 def test_softmax_xent_label_outside_the_classes_is_reported_and_never_used_as_an_index():
