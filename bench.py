@@ -373,10 +373,20 @@ def run_ours(args):
         wl = ConvWorkload(rank, args.minibatch, tuple(int(v) for v in args.layer.split(",")), pooled=args.pooled)
     else:
         wl = WORKLOADS[args.workload](rank, args.minibatch)
+    if args.data_parallel:
+        # Sec. 3.1 / 3.4: the ranks share one model; every rank's step() exchanges the weight gradients layer by layer
+        if not hasattr(wl, "net"):
+            raise SystemExit("--data-parallel needs a network workload (vgga or dnn)")
+        from paper_1602_06709_b200 import data_parallel
+        dp = data_parallel.DataParallelStep(wl.net)
+        wl.step = dp.step
+        wl.step_eager = dp.step
+        wl.e2e_step = None
     peaks = load_peaks()
     # The DNN step is ~45 short kernels and bound by the host's launch rate when issued one by one: by default it is
     # replayed from a CUDA graph of exactly those launches.  The VGG-A step keeps the GPU busy either way.
-    use_graph = hasattr(wl, "use_graph") and (args.graph == "1" or (args.graph == "auto" and args.workload == "dnn"))
+    use_graph = hasattr(wl, "use_graph") and not args.data_parallel and \
+        (args.graph == "1" or (args.graph == "auto" and args.workload == "dnn"))
     graph_launches = wl.use_graph() if use_graph else 0
 
     def timed(fn, steps, warmup, sample_clocks=False):
@@ -415,8 +425,11 @@ def run_ours(args):
 
     # end to end through the user-level call: pinned host minibatch in, result out, every step
     e2e_steps = max(3, min(args.steps, 10))
-    ms_e2e, _, _ = timed(wl.e2e_step, e2e_steps, 1)
-    e2e_value = replicas.whole_job_throughput(wl.units_per_step, e2e_steps, world, ms_e2e)
+    if wl.e2e_step is not None:
+        ms_e2e, _, _ = timed(wl.e2e_step, e2e_steps, 1)
+        e2e_value = replicas.whole_job_throughput(wl.units_per_step, e2e_steps, world, ms_e2e)
+    else:       # (the data-parallel job is timed with resident inputs only)
+        ms_e2e, e2e_value = float("nan"), None
 
     # instrumented repeat of the same steps: CUDA events around every kernel launch on the launching stream,
     # tagged with the pass (ABI call) the launch belongs to
@@ -437,7 +450,8 @@ def run_ours(args):
 
     config = {"workload": wl.name, "l2": "inputs larger than L2 (activations are GBs per step)"
               if args.workload != "dnn" else "weights+activations 0.3 GB per step, larger than L2",
-              "parallelism": "replicas only" if world > 1 else "single GPU", "cuda_graph": bool(use_graph),
+              "parallelism": ("data-parallel: per-layer reduce-scatter / owned-strip SGD / all-gather" if args.data_parallel
+                              else "replicas only" if world > 1 else "single GPU"), "cuda_graph": bool(use_graph),
               **wl.describe()}
     legs = None
     if world == 1 and args.workload == "vgga" and not args.no_legs:
@@ -669,6 +683,11 @@ def main():
                     help="replay the step from a CUDA graph of its launches (auto: the DNN step only)")
     ap.add_argument("--minibatch", type=int, default=0, help="override the workload's minibatch (profiling only)")
     ap.add_argument("--layer", default="", help="C,K,H of another 3x3 pad-1 layer for --workload conv (profiling only)")
+    ap.add_argument("--data-parallel", action="store_true",
+                    help="vgga / dnn with --gpus N > 1: one data-parallel job (per-layer reduce-scatter of the weight "
+                         "gradients, SGD on the owned strip, all-gather of the weights, overlapped with the backward "
+                         "pass) instead of N independent replicas; every rank keeps the workload's minibatch "
+                         "(the global minibatch grows with N: weak scaling)")
     ap.add_argument("--pooled", action="store_true",
                     help="with --layer: run the layer as a pooled first layer (conv+pool in one call, weight gradient "
                          "from the pooled gradient); profiling only")

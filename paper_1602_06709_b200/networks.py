@@ -26,7 +26,7 @@ def _align(n: int, a: int = 64) -> int:
 class _ParamStore:
     """Flat fp32 parameter and gradient buffers with 256-byte aligned views."""
 
-    def __init__(self, shapes: List[tuple]):
+    def __init__(self, shapes: List[tuple], device="cuda"):
         self.offsets = []
         off = 0
         for shp in shapes:
@@ -34,8 +34,8 @@ class _ParamStore:
             off += _align(int(np.prod(shp)))
         self.total = off
         self.shapes = shapes
-        self.params = torch.zeros(off, device="cuda")
-        self.grads = torch.zeros(off, device="cuda")
+        self.params = torch.zeros(off, device=device)
+        self.grads = torch.zeros(off, device=device)
 
     def view(self, buf, i):
         n = int(np.prod(self.shapes[i]))
@@ -49,6 +49,15 @@ class _ParamStore:
 
     def n_real(self) -> int:
         return sum(int(np.prod(s)) for s in self.shapes)
+
+    def layer_buckets(self):
+        """(offset, length) of every (weights, bias) pair: the unit of the data-parallel gradient exchange.  Every
+        tensor starts on a 64-element boundary, so a bucket divides into 2, 4, 8 or 16 equal 16-byte aligned strips."""
+        out = []
+        for i in range(0, len(self.shapes), 2):
+            end = self.offsets[i + 2] if i + 2 < len(self.shapes) else self.total
+            out.append((self.offsets[i], end - self.offsets[i]))
+        return out
 
 
 @dataclass
@@ -221,8 +230,14 @@ class VggA(_HostFeed):
         return self.pooled[i - 1] if prev.pool else self.y[i - 1]
 
     # -- one training step --------------------------------------------------
-    def forward(self):
+    def param_buckets(self):
+        return self.store.layer_buckets()        # conv layers first, then the FC layers: the order of forward()
+
+    def forward(self, before_layer=None):
+        """before_layer(j), if given, is called before layer j (convolutions, then FC layers) reads its weights."""
         for i, L in enumerate(self.convs):
+            if before_layer:
+                before_layer(i)
             if L.pool:      # conv -> ReLU -> 2x2 pool, the maxima taken in the convolution's epilogue
                 B.conv_fwd_pool(L.desc, self.layer_input(i), self.conv_w(i), self.conv_b(i), self.y[i], self.pooled[i],
                                 B.ACT_RELU, self.ws, pool_codes=self.pool_codes[i])
@@ -230,12 +245,17 @@ class VggA(_HostFeed):
                 B.conv_fwd(L.desc, self.layer_input(i), self.conv_w(i), self.conv_b(i), self.y[i], B.ACT_RELU, self.ws)
         a = self.pooled[-1].view(self.N, self.flat)
         for j, (C, K) in enumerate(self.fcs):
+            if before_layer:
+                before_layer(len(self.convs) + j)
             act = B.ACT_RELU if j + 1 < len(self.fcs) else B.ACT_NONE
             B.fc_fwd(self.N, C, K, a, self.fc_w(j), self.fc_b(j), self.fc_out[j], act, self.ws)
             a = self.fc_out[j]
         B.softmax_xent(self.N, self.classes, self.fc_out[-1], self.labels, self.loss, self.fc_dout[-1])
 
-    def backward(self):
+    def backward(self, after_layer=None, after_backprop=None):
+        """after_layer(j), if given, is called once the weight and bias gradients of layer j are complete (its bias
+        gradient comes out of the layer above's call, so it is complete by then too); after_backprop(j) once the
+        layer's backpropagation, the last reader of its weights in this step, has been issued."""
         nfc = len(self.fcs)
         for j in reversed(range(nfc)):
             C, K = self.fcs[j]
@@ -246,6 +266,10 @@ class VggA(_HostFeed):
             B.fc_bwd_fused(self.N, C, K, a, self.fc_w(j), None, B.ACT_NONE, self.fc_dout[j], dx,
                            B.ACT_RELU if j > 0 else B.ACT_NONE, self.fc_db(j - 1) if j > 0 else None, self.fc_dw(j),
                            self.fc_db(j) if j + 1 == nfc else None, self.ws)
+            if after_layer:
+                after_layer(len(self.convs) + j)
+            if after_backprop:
+                after_backprop(len(self.convs) + j)
         for i in reversed(range(len(self.convs))):
             L = self.convs[i]
             # The bias gradient of layer i is the per-map sum of dy[i]; it is formed by whichever kernel writes
@@ -254,11 +278,17 @@ class VggA(_HostFeed):
                 # pooling backward, ReLU mask, bias gradient and weight gradient in one pass over the pooled gradient
                 B.conv_bwd_weights_pooled(L.desc, self.layer_input(0), self.dpooled[0], self.pool_codes[0], True,
                                           self.conv_dw(0), self.conv_db(0), self.ws)
+                if after_layer:
+                    after_layer(0)
+                if after_backprop:
+                    after_backprop(0)
                 continue
             if L.pool:   # gradient through the pool, then through the ReLU (fused mask), routed by the position codes
                 B.maxpool2x2_bwd_codes(self.N, L.H, L.W, L.K, self.pool_codes[i], self.dpooled[i], True, self.dy[i],
                                        self.conv_db(i), self.ws)
             B.conv_bwd_weights(L.desc, self.layer_input(i), self.dy[i], self.conv_dw(i), None, True, self.ws)
+            if after_layer:
+                after_layer(i)
             if i > 0:
                 prev = self.convs[i - 1]
                 if prev.pool:
@@ -266,6 +296,8 @@ class VggA(_HostFeed):
                 else:   # the layer's input is the previous ReLU output: fuse its mask (and its bias gradient)
                     B.conv_bwd_data_colsum(L.desc, self.dy[i], self.conv_w(i), self.y[i - 1], self.dy[i - 1],
                                            self.conv_db(i - 1), self.ws)
+            if after_backprop:
+                after_backprop(i)
 
     def update(self):
         B.sgd_update(self.store.params, self.store.grads, self.lr)
@@ -309,16 +341,21 @@ class Dnn(_HostFeed):
     def dw(self, j): return self.store.g(2 * j)
     def db(self, j): return self.store.g(2 * j + 1)
 
-    def forward(self):
+    def param_buckets(self):
+        return self.store.layer_buckets()
+
+    def forward(self, before_layer=None):
         a = self.x
         n = len(self.layers)
         for j, (C, K) in enumerate(self.layers):
+            if before_layer:
+                before_layer(j)
             act = B.ACT_SIGMOID if j + 1 < n else B.ACT_NONE
             B.fc_fwd(self.N, C, K, a, self.w(j), self.b(j), self.out[j], act, self.ws)
             a = self.out[j]
         B.softmax_xent(self.N, self.dims[-1], self.out[-1], self.labels, self.loss, self.dout[-1])
 
-    def backward(self):
+    def backward(self, after_layer=None, after_backprop=None):
         n = len(self.layers)
         for j in reversed(range(n)):
             C, K = self.layers[j]
@@ -328,6 +365,10 @@ class Dnn(_HostFeed):
             B.fc_bwd_fused(self.N, C, K, a, self.w(j), None, B.ACT_NONE, self.dout[j], dx,
                            B.ACT_SIGMOID if j > 0 else B.ACT_NONE, self.db(j - 1) if j > 0 else None, self.dw(j),
                            self.db(j) if j + 1 == n else None, self.ws)
+            if after_layer:
+                after_layer(j)
+            if after_backprop:
+                after_backprop(j)
 
     def update(self):
         B.sgd_update(self.store.params, self.store.grads, self.lr)

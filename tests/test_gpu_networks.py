@@ -176,3 +176,35 @@ def test_captured_step_graph_equals_eager_steps(kind):
         assert np.allclose(l0, l1, rtol=1e-5, atol=0)       # (the scalar loss is summed with atomics)
         assert np.array_equal(p0, p1)
     assert len(set(l0)) > 1
+
+
+@pytest.mark.parametrize("kind", ["vgg", "dnn"])
+def test_data_parallel_step_on_one_rank_equals_the_plain_step(kind):
+    """The data-parallel step (per-layer hooks, exchange stream, update of each layer as soon as its backpropagation
+    has been issued) with a single rank must leave bit-identical parameters to the plain step: same kernels, the
+    update only moves from one launch over the whole store to one per layer on the second stream."""
+    from paper_1602_06709_b200 import binding as B
+    from paper_1602_06709_b200 import data_parallel, inputs, networks
+
+    def make():
+        if kind == "vgg":
+            return _small_vgg()[0]
+        net = networks.Dnn(64, dims=[40, 96, 96, 32], cfg="small_dnn")
+        _randomise_biases(net)
+        net.x.copy_(torch.from_numpy(inputs.normal(inputs.tensor_id("small_dnn", "x"), (64, 40), 1.0)))
+        net.labels.copy_(torch.from_numpy(inputs.labels(inputs.tensor_id("small_dnn", "labels"), 64, 32)))
+        return net
+    plain, dp_net = make(), make()
+    assert torch.equal(plain.store.params, dp_net.store.params)
+    dp = data_parallel.DataParallelStep(dp_net)
+    for _ in range(3):
+        plain.step()
+        dp.step()
+    dp.finish()
+    torch.cuda.synchronize()
+    B.check_device_status()
+    assert torch.equal(plain.store.params, dp_net.store.params)
+    assert torch.equal(plain.loss, dp_net.loss)
+    buckets = dp_net.param_buckets()
+    assert len(buckets) == len(dp_net.store.shapes) // 2
+    assert sum(length for _, length in buckets) == dp_net.store.total and all(length % 64 == 0 for _, length in buckets)
