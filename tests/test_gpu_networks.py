@@ -204,7 +204,32 @@ def test_data_parallel_step_on_one_rank_equals_the_plain_step(kind):
     torch.cuda.synchronize()
     B.check_device_status()
     assert torch.equal(plain.store.params, dp_net.store.params)
-    assert torch.equal(plain.loss, dp_net.loss)
+    assert torch.allclose(plain.loss, dp_net.loss, rtol=1e-5)        # (the loss scalar is summed with atomics)
     buckets = dp_net.param_buckets()
     assert len(buckets) == len(dp_net.store.shapes) // 2
     assert sum(length for _, length in buckets) == dp_net.store.total and all(length % 64 == 0 for _, length in buckets)
+
+
+def test_hybrid_fc_layer_with_library_kernels_single_rank():
+    """hybrid.HybridFc with the library's FC kernels as its contractions (one rank: one group of one): forward,
+    backward and update against the oracle's fully-connected passes."""
+    import gpu_helpers as G
+    from paper_1602_06709_b200 import hybrid, inputs
+    N, C, K, lr = 96, 256, 128, 0.05
+    x = inputs.normal(inputs.tensor_id("hyb", "x"), (N, C), 1.0)
+    w = inputs.normal(inputs.tensor_id("hyb", "w"), (K, C), (1.0 / C) ** 0.5)
+    b = inputs.uniform(inputs.tensor_id("hyb", "b"), (K,), -0.5, 0.5)
+    dy = inputs.normal(inputs.tensor_id("hyb", "dy"), (N, K), 1.0)
+    L = hybrid.HybridFc(C, K, 1, "relu", lr, ops=hybrid.LibraryOps(), w_full=torch.from_numpy(w), b_full=torch.from_numpy(b),
+                        device="cuda")
+    y = L.forward(G.dev(x))
+    y_ref = oracle.fc_fwd(x, w, b, oracle.ACT_RELU)
+    G.assert_parity(y.cpu().numpy(), y_ref, "hybrid fc forward")
+    dx = L.backward(G.dev(dy))
+    _, dx_ref, dw_ref, db_ref = oracle.fc_bwd(x, w, y.cpu().numpy(), dy, oracle.ACT_RELU, dz_dtype=np.float32)
+    G.assert_parity(dx.cpu().numpy(), dx_ref, "hybrid fc dx")
+    G.assert_parity(L.dw.cpu().numpy(), dw_ref, "hybrid fc dw")
+    G.assert_parity(L.db.cpu().numpy(), db_ref, "hybrid fc db")
+    dw_gpu = L.dw.cpu().numpy().copy()
+    L.update()
+    np.testing.assert_allclose(L.w.cpu().numpy(), oracle.sgd_update(w, dw_gpu, lr), rtol=0, atol=1e-6)
