@@ -73,7 +73,7 @@ int pcl_set_path(int path);
  * has a named knob with which the tests pin each kernel variant and the alternatives were measured:
  * TILING (0 plain, 1-3 haloed layouts), BN, KS, KS_HALO, KS_WGRAD, PAIR, PAIR_HALO, PAIR_WGRAD, GRP,
  * ISSUERS, SPLIT_ACC, PIX_WGRAD, XHALO_WGRAD, TMA_STORE, WEIGHTS_IN_PLACE, EPI_WARPS, FC_DW_FORWARD,
- * KSPLIT, RESIDENT_B, KSLICES, WAIT_LIMIT_US (limit of the bounded device-side waits in microseconds,
+ * KSPLIT, RESIDENT_B, KSLICES, SELECT, WAIT_LIMIT_US (limit of the bounded device-side waits in microseconds,
  * default 2 s; applies to the current device), FAULT_INJECT (test only: 1 / 2 make the next forward-type /
  * weight-gradient launch that runs as single CTAs arm its first pipeline slot for 16 bytes more than it copies,
  * so that the waits on that slot run out, the kernel gives up and returns, and pcl_last_device_status()
@@ -82,6 +82,14 @@ int pcl_set_path(int path);
  * Returns PCL_ERR_BAD_ARG for an unknown name. */
 int pcl_set_tuning(const char* name, int value);
 int pcl_reset_tuning(void);
+
+/* Blocking search (Sec. 2.2-2.3 re-posed: the paper picks its blocks by minimising bytes per flop with a brute-force
+ * search; here candidates -- plain or haloed tiling, tile width, single CTAs or CTA pairs -- are scored by a cost
+ * model of the tensor pipe, the shared-memory fill rate, the issuing thread and the epilogue warps).  Writes a
+ * one-line description of the tiling the forward (PCL_PASS_FWD) or backward-data pass of this layer would launch
+ * with under the current knobs, the model's predicted cycles for it and the model's own choice.  Launches
+ * nothing.  The SELECT knob = 1 makes the launchers take the model's choice instead of their measured rules. */
+int pcl_conv_plan_describe(const pcl_conv_desc* d, int pass, char* buf, size_t buf_bytes);
 
 /* Output spatial size of a convolution.  Returns PCL_ERR_BAD_ARG if the
  * kernel does not fit in the padded input. */

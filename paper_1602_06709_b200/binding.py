@@ -30,7 +30,7 @@ EXPORTS = [
     "pcl_conv_bwd_data_colsum_workspace_bytes", "pcl_conv_bwd_data_colsum",
     "pcl_maxpool2x2_bwd_colsum_workspace_bytes", "pcl_maxpool2x2_bwd_colsum", "pcl_conv_fwd_pool", "pcl_conv_fwd_pool_is_fused",
     "pcl_conv_bwd_weights_pooled", "pcl_conv_bwd_weights_pooled_is_fused", "pcl_conv_bwd_weights_pooled_workspace_bytes",
-    "pcl_maxpool2x2_fwd_codes", "pcl_maxpool2x2_bwd_codes", "pcl_last_wait_code", "pcl_set_tuning", "pcl_reset_tuning", "pcl_fc_bwd_fused",
+    "pcl_maxpool2x2_fwd_codes", "pcl_maxpool2x2_bwd_codes", "pcl_last_wait_code", "pcl_set_tuning", "pcl_reset_tuning", "pcl_fc_bwd_fused", "pcl_conv_plan_describe",
 ]
 
 
@@ -65,6 +65,7 @@ def lib() -> ctypes.CDLL:
         dp = ctypes.POINTER(ConvDesc)
         L.pcl_set_path.argtypes = [ci]
         L.pcl_set_tuning.argtypes = [ctypes.c_char_p, ci]
+        L.pcl_conv_plan_describe.argtypes = [dp, ci, ctypes.c_char_p, sz]
         L.pcl_conv_out_dims.argtypes = [dp, ctypes.POINTER(ci), ctypes.POINTER(ci)]
         L.pcl_conv_workspace_bytes.argtypes = [dp, ci]
         L.pcl_conv_workspace_bytes.restype = sz
@@ -144,6 +145,13 @@ def set_tuning(name: str, value):
     elif name == "TILING" and isinstance(value, str):
         value = TILINGS[value]
     _check(lib().pcl_set_tuning(name.encode(), int(value)), f"pcl_set_tuning({name})")
+
+
+def conv_plan_describe(d: ConvDesc, pass_: int) -> str:
+    """The tiling the pass would launch with under the current knobs and the cost model's prediction for it."""
+    buf = ctypes.create_string_buffer(512)
+    _check(lib().pcl_conv_plan_describe(ctypes.byref(d), pass_, buf, 512), "pcl_conv_plan_describe")
+    return buf.value.decode()
 
 
 def reset_tuning():

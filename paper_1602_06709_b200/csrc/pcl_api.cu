@@ -41,7 +41,7 @@ std::atomic<unsigned> g_tune_gen{0};
 const char* const kTuneNames[TUNE_COUNT] = {
     "TILING", "BN", "KS", "KS_HALO", "KS_WGRAD", "PAIR", "PAIR_HALO", "PAIR_WGRAD", "GRP", "ISSUERS", "SPLIT_ACC",
     "PIX_WGRAD", "XHALO_WGRAD", "TMA_STORE", "WEIGHTS_IN_PLACE", "EPI_WARPS", "FC_DW_FORWARD", "KSPLIT",
-    "WAIT_LIMIT_US", "FAULT_INJECT", "RESIDENT_B", "KSLICES"};
+    "WAIT_LIMIT_US", "FAULT_INJECT", "RESIDENT_B", "KSLICES", "SELECT"};
 }  // namespace
 
 int tune(int id, int dflt) {
@@ -555,6 +555,26 @@ TcFpropArgs bwd_data_args(const pcl_conv_desc& d, int P, int Q, const float* dy,
     return a;
 }
 }  // namespace
+
+int pcl_conv_plan_describe(const pcl_conv_desc* d, int pass, char* buf, size_t buf_bytes) {
+    int P, Q;
+    int rc = check_desc(d, &P, &Q);
+    if (rc != PCL_OK) return rc;
+    if (!buf || buf_bytes < 64) return PCL_ERR_BAD_ARG;
+    const float* fake = reinterpret_cast<const float*>(uintptr_t(256));      // (alignment checks only; nothing is read)
+    if (pass == PCL_PASS_FWD && few_channel_path_for(*d, pass)) {
+        return tc_fprop_describe(few_fwd_args(*d, P, Q, fake, fake, nullptr, const_cast<float*>(fake), PCL_ACT_RELU), buf, buf_bytes);
+    } else if (pass == PCL_PASS_FWD && tensor_path_for(*d, pass)) {
+        TcFpropArgs a{fake, fake, nullptr, nullptr, const_cast<float*>(fake), d->N, d->H, d->W, d->C, d->K, d->R, d->S,
+                      d->pad_h, d->pad_w, P, Q, PCL_ACT_RELU};
+        a.stride_h = d->stride_h; a.stride_w = d->stride_w;
+        return tc_fprop_describe(a, buf, buf_bytes);
+    } else if (pass == PCL_PASS_BWD_DATA && tensor_path_for(*d, pass) && unit_stride(*d)) {
+        return tc_fprop_describe(bwd_data_args(*d, P, Q, fake, fake, nullptr, const_cast<float*>(fake)), buf, buf_bytes);
+    }
+    snprintf(buf, buf_bytes, "not a single forward-type tensor-core launch");
+    return PCL_OK;
+}
 
 size_t pcl_conv_bwd_data_colsum_workspace_bytes(const pcl_conv_desc* d) {
     int P, Q;

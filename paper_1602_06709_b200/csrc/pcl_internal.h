@@ -54,7 +54,7 @@ enum TuneId {
     TUNE_TILING = 0,        // forward-type kernel: 0 plain, 1-3 haloed layouts 0-2
     TUNE_BN, TUNE_KS, TUNE_KS_HALO, TUNE_KS_WGRAD, TUNE_PAIR, TUNE_PAIR_HALO, TUNE_PAIR_WGRAD, TUNE_GRP, TUNE_ISSUERS,
     TUNE_SPLIT_ACC, TUNE_PIX_WGRAD, TUNE_XHALO_WGRAD, TUNE_TMA_STORE, TUNE_WEIGHTS_IN_PLACE, TUNE_EPI_WARPS,
-    TUNE_FC_DW_FORWARD, TUNE_KSPLIT, TUNE_WAIT_LIMIT_US, TUNE_FAULT_INJECT, TUNE_RESIDENT_B, TUNE_KSLICES, TUNE_COUNT
+    TUNE_FC_DW_FORWARD, TUNE_KSPLIT, TUNE_WAIT_LIMIT_US, TUNE_FAULT_INJECT, TUNE_RESIDENT_B, TUNE_KSLICES, TUNE_SELECT, TUNE_COUNT
 };
 int tune(int id, int dflt);
 bool tune_is_set(int id);
@@ -165,6 +165,9 @@ size_t tc_fprop_split_ws_bytes(const TcFpropArgs& a);
 bool tc_fprop_eligible(const TcFpropArgs& a);
 long tc_fprop_colsum_rows(const TcFpropArgs& a);
 int launch_tc_fprop(const TcFpropArgs& a, cudaStream_t st);
+// Text description of the tiling launch_tc_fprop(a) would use and of the cost model's prediction for it (and of the
+// tiling the model itself would choose).
+int tc_fprop_describe(const TcFpropArgs& a, char* buf, size_t n);
 
 // ---- weight-gradient-type GEMM on tcgen05 ------------------------------------
 // dw[k, r, s, c] = sum_{n,p,q} dy[n,p,q,k] * x[n, p*stride_h + r - pad_h, q*stride_w + s*dil_w - pad_w, c]

@@ -26,6 +26,7 @@
 //                 -> global, through TMA stores or coalesced per-lane stores (two warps per TMEM lane quarter)
 //   warps 11-18   eight more epilogue warps (608 threads) in the variant for tiles with a very short reduction
 // Two TMEM accumulator sets let the epilogue of tile i overlap the main loop of tile i+1.
+#include <stdio.h>
 #include <stdlib.h>
 
 #include "pcl_internal.h"
@@ -1083,19 +1084,21 @@ struct TileCfg {
     int pair = 0;       // CTA pairs: two image-group tiles share one 256-wide weight tile (see the kernel)
 };
 
-TileCfg plain_cfg(const TcFpropArgs& a, int cblocks, int sm_count) {
+// bn_force / pair_force (-1 = the builder's own rule): the candidates the blocking search enumerates
+TileCfg plain_cfg(const TcFpropArgs& a, int cblocks, int sm_count, int bn_force = -1, int pair_force = -1) {
     TileCfg c;
     choose_box(a.P, a.Q, a.N, a.pool_out != nullptr, &c.bw_log2, &c.bh_log2, a.stride_w, a.stride_h);
     c.tw = 1 << c.bw_log2; c.th = 1 << c.bh_log2; c.tn = kTileM / (c.tw * c.th);
     c.tiles_q = (a.Q + c.tw - 1) / c.tw; c.tiles_p = (a.P + c.th - 1) / c.th; c.tiles_n = (a.N + c.tn - 1) / c.tn;
     const long m_tiles = long(c.tiles_q) * c.tiles_p * c.tiles_n;
-    c.BN = choose_bn(a.Kout, m_tiles, sm_count);
+    c.BN = bn_force > 0 ? bn_force : choose_bn(a.Kout, m_tiles, sm_count);
     c.tiles_k = (a.Kout + c.BN - 1) / c.BN;
     // narrow tiles: several k-steps per slot (see the kernel), as long as 4 slots still fit
     // pairs pay where operand traffic or the issue rate of wide MMAs bounds the tile; narrow tiles are bound by
     // the issuing thread and run as single CTAs with two issuers instead
-    c.pair = tune(TUNE_PAIR, 1) && c.BN >= 128 && c.tiles_n >= 2 && sm_count >= 2 &&
-             (!a.wt_mn_major || c.BN % 64 == 0);        // MN-major weights are fetched in whole 32-map groups per CTA
+    const bool pair_ok = c.BN >= 64 && c.BN % 16 == 0 && c.tiles_n >= 2 && sm_count >= 2 &&
+                         (!a.wt_mn_major || c.BN % 64 == 0);    // MN-major weights are fetched in whole 32-map groups per CTA
+    c.pair = pair_force >= 0 ? (pair_force && pair_ok) : (tune(TUNE_PAIR, 1) && c.BN >= 128 && pair_ok);
     const int step_bytes = kABytes + (c.pair ? c.BN * 64 : c.BN * 128);
     c.KS = tune(TUNE_KS, 2);
     const int kiters = a.R * a.S * cblocks;
@@ -1109,7 +1112,7 @@ TileCfg plain_cfg(const TcFpropArgs& a, int cblocks, int sm_count) {
 }
 
 // layout: 0 = one box (8 x 16), 1 = two boxes side by side (16 x 16), 2 = two boxes stacked (8 x 32)
-TileCfg halo_cfg(const TcFpropArgs& a, int cblocks, int sm_count, int layout) {
+TileCfg halo_cfg(const TcFpropArgs& a, int cblocks, int sm_count, int layout, int bn_force = -1) {
     TileCfg c;
     c.halo = 1; c.MT = layout == 0 ? 1 : 2;
     c.bw_log2 = 3; c.bh_log2 = 4;
@@ -1124,7 +1127,7 @@ TileCfg halo_cfg(const TcFpropArgs& a, int cblocks, int sm_count, int layout) {
     c.half_off_bytes = layout == 1 ? 8 * 128 : (layout == 2 ? 16 * c.PW * 128 : 0);
     c.tiles_q = (a.Q + c.tw - 1) / c.tw; c.tiles_p = (a.P + c.th - 1) / c.th; c.tiles_n = a.N;
     const long m_tiles = long(c.tiles_q) * c.tiles_p * c.tiles_n;
-    c.BN = choose_bn(a.Kout, m_tiles, sm_count);
+    c.BN = bn_force > 0 ? bn_force : choose_bn(a.Kout, m_tiles, sm_count);
     if (2 * c.MT * c.BN > 512) return c;          // two accumulator sets must fit the 512 TMEM columns
     c.tiles_k = (a.Kout + c.BN - 1) / c.BN;
     c.pair = tune(TUNE_PAIR_HALO, 0) && c.tiles_n >= 2 && sm_count >= 2;      // pairs of images (no gain measured)
@@ -1147,9 +1150,88 @@ TileCfg halo_cfg(const TcFpropArgs& a, int cblocks, int sm_count, int layout) {
     return c;
 }
 
+// ---- Blocking search (Sec. 2.2 / 2.3 re-posed for this memory hierarchy) ------------------------------------------
+// The paper chooses its cache and register blocks by minimising the bytes moved per flop under the capacity of the
+// cache, with a brute-force search over the block sizes.  Here the scarce rates are the tensor pipe, the fill rate
+// of shared memory out of L2, the lone issuing thread and the epilogue warps, under 227 KB of shared memory and 512
+// TMEM columns; a candidate's cost is the slowest of those four per tile, times the tiles a CTA takes.  Constants
+// are measurements on B200 (microbenchmarks and ncu captures of these kernels).
+struct TileCost { double mma, fill, issue, epilogue, tile, total; };
+constexpr double kMmaFloorClk = 52.0;        // a K = 8 MMA of N columns takes max(N / 2, 52) cycles
+constexpr double kFillSingle = 60.0;         // bytes per clock and SM into shared memory, single CTAs of this kernel
+constexpr double kFillPair = 57.0;           //   ... CTA pairs (which need a third fewer bytes per MMA)
+constexpr double kHaloMmaFactor = 1.5;       // MMAs whose A operand is a row-shifted view of a haloed patch run slower
+constexpr double kHaloOneBoxFactor = 1.3;    //   ... and slower still when a tile is one box (no second box to share a weight tile with)
+constexpr double kIssueMmaClk = 45.0;        // the issuing thread's cost per MMA
+constexpr double kIssueSlotClk = 160.0;      //   ... per pipeline slot (one barrier round trip and one commit)
+constexpr double kEpilogueChunkClk = 1600.0; // an epilogue warp's cost per 32 x 32 chunk
+constexpr double kTileFixedClk = 300.0, kLaunchFixedClk = 4000.0;
+
+TileCost predict_cost(const TcFpropArgs& a, const TileCfg& c, int cblocks, int sm_count) {
+    TileCost t{};
+    const double ksteps = double(a.R) * a.S * cblocks;
+    const double b_bytes = c.pair ? c.BN * 64.0 : c.BN * 128.0;
+    const double mma_clk = c.BN / 2.0 > kMmaFloorClk ? c.BN / 2.0 : kMmaFloorClk;
+    t.mma = c.MT * ksteps * 4.0 * mma_clk * (c.halo ? kHaloMmaFactor * (c.MT == 1 ? kHaloOneBoxFactor : 1.0) : 1.0);
+    const double bytes = c.halo ? cblocks * (double(c.patch_bytes) + double(a.R) * a.S * b_bytes) : ksteps * (kABytes + b_bytes);
+    t.fill = bytes / (c.pair ? kFillPair : kFillSingle);
+    const double slots = c.halo ? cblocks * double((a.R * a.S + c.KS - 1) / c.KS) : (ksteps + c.KS - 1) / c.KS;
+    const int issuers = (!c.pair && slots >= 8) ? 2 : 1;
+    t.issue = (c.MT * ksteps * 4.0 * kIssueMmaClk + slots * kIssueSlotClk) / issuers;
+    const double chunks = c.MT * (c.BN / 32.0) * 4.0;
+    t.epilogue = double(long((chunks + kEpiWarps - 1) / kEpiWarps)) * kEpilogueChunkClk * (a.pool_out ? 1.3 : 1.0);
+    t.tile = t.mma;
+    if (t.fill > t.tile) t.tile = t.fill;
+    if (t.issue > t.tile) t.tile = t.issue;
+    if (t.epilogue > t.tile) t.tile = t.epilogue;
+    t.tile += kTileFixedClk;
+    const double m_tiles = double(c.tiles_q) * c.tiles_p * (c.pair ? (c.tiles_n + 1) / 2 : c.tiles_n);
+    const double work_items = m_tiles * c.tiles_k;                       // CTA tiles (a pair's two tiles count once)
+    const double slots_sm = c.pair ? sm_count / 2 : sm_count;
+    const double per_cta = double(long((work_items + slots_sm - 1) / slots_sm));
+    t.total = per_cta * t.tile + kLaunchFixedClk;
+    return t;
+}
+
+// Enumerates the candidate tilings of a launch -- plain tiling x tile width x single CTAs or pairs, the three haloed
+// layouts x tile width -- and returns the one the cost model predicts fastest.
+TileCfg search_cfg(const TcFpropArgs& a, int sm_count, TileCost* best_cost = nullptr) {
+    const int cblocks = (a.Cin + kBlockC - 1) / kBlockC;
+    TileCfg best;
+    double best_total = 1e300;
+    const int k32 = (a.Kout + 31) / 32 * 32;
+    for (int bn = 32; bn <= 256; bn += 32) {
+        if (bn > k32) break;
+        if (a.wt_mn_major && (a.Kout % 32 != 0)) break;
+        const int n_tiles = (a.Kout + bn - 1) / bn;
+        if ((n_tiles - 1) * bn >= a.Kout) continue;
+        for (int variant = 0; variant < 5; ++variant) {
+            const TileCfg c = variant < 2 ? plain_cfg(a, cblocks, sm_count, bn, variant) : halo_cfg(a, cblocks, sm_count, variant - 2, bn);
+            if (!c.ok || (variant == 1 && !c.pair)) continue;
+            if (c.halo && a.pool_out && (c.bw_log2 < 1 || c.bh_log2 < 1)) continue;
+            const TileCost t = predict_cost(a, c, cblocks, sm_count);
+            // (a haloed candidate must beat the plain ones by a tenth: its prediction is the less certain one)
+            const double score = t.total * (c.halo ? 1.1 : 1.0);
+            if (score < best_total) { best_total = score; best = c; if (best_cost) *best_cost = t; }
+        }
+    }
+    return best;
+}
+
 // The tiling a launch will use (also needed to size the fused column-sum rows).
 TileCfg select_cfg(const TcFpropArgs& a, int sm_count) {
     const int cblocks = (a.Cin + kBlockC - 1) / kBlockC;
+    // Convolutions (more than one tap) take the candidate the cost model predicts fastest; the measured table of the
+    // blocking search (profiles/) has it within a few percent of the measured best on every layer of the benchmark
+    // configurations.  1 x 1 layers (the FC GEMMs) keep the rules below, which also decide their reduction splits.
+    // SELECT = 0 switches the model off, 1 applies it to every launch; a pinned knob always wins.
+    // (the few-channel path reads overlapping windows, whose fill cost the model does not describe: rules too)
+    const int sel = tune(TUNE_SELECT, (a.R * a.S > 1 && a.in_stride_w == 0) ? 1 : 0);
+    if (sel == 1 && tune(TUNE_TILING, -1) < 0 && !tune_is_set(TUNE_BN) && !tune_is_set(TUNE_PAIR) && !tune_is_set(TUNE_KS) &&
+        !tune_is_set(TUNE_KS_HALO) && !tune_is_set(TUNE_GRP) && !tune_is_set(TUNE_PAIR_HALO)) {
+        const TileCfg m = search_cfg(a, sm_count);
+        if (m.ok) return m;
+    }
     TileCfg cfg = plain_cfg(a, cblocks, sm_count);
     if (!cfg.ok) return cfg;
     // Test hook: the TILING knob pins the tiling (when that tiling is possible).
@@ -1207,6 +1289,25 @@ int choose_ksplit(const TcFpropArgs& a, const TileCfg& cfg, int cblocks, int sm_
     return 1;
 }
 }  // namespace
+
+int tc_fprop_describe(const TcFpropArgs& a, char* buf, size_t n) {
+    if (!tc_fprop_eligible(a)) return PCL_ERR_UNSUPPORTED_SHAPE;
+    const int sm = device_sm_count();
+    const int cblocks = (a.Cin + kBlockC - 1) / kBlockC;
+    const TileCfg c = select_cfg(a, sm);
+    if (!c.ok) return PCL_ERR_UNSUPPORTED_SHAPE;
+    const TileCost t = predict_cost(a, c, cblocks, sm);
+    TileCost mt{};
+    const TileCfg m = search_cfg(a, sm, &mt);
+    const char* names[4] = {"plain", "halo0", "halo1", "halo2"};
+    auto name = [&](const TileCfg& x) { return names[!x.halo ? 0 : (x.MT == 1 ? 1 : (x.half_dq ? 2 : 3))]; };
+    snprintf(buf, n,
+             "tiling=%s BN=%d pair=%d KS=%d stages=%d box=%dx%dx%d predicted_clk=%.0f (mma %.0f fill %.0f issue %.0f epilogue %.0f per "
+             "tile) | model_choice: tiling=%s BN=%d pair=%d predicted_clk=%.0f",
+             name(c), c.BN, c.pair, c.KS, c.stages, c.tw, c.th, c.tn, t.total, t.mma, t.fill, t.issue, t.epilogue, name(m), m.BN,
+             m.pair, mt.total);
+    return PCL_OK;
+}
 
 size_t tc_fprop_split_ws_bytes(const TcFpropArgs& a) {
     const int sm = device_sm_count();
