@@ -188,6 +188,17 @@ int pcl_conv_bwd_weights_pooled(const pcl_conv_desc* d, const float* x, const fl
                                 const unsigned char* pool_codes, int relu_mask, float* dw, float* dbias,
                                 void* ws, size_t ws_bytes, void* cuda_stream);
 
+/* The same from the staged input the layer's forward call left behind (the paper has no counterpart).  On the
+ * few-channel path pcl_conv_fwd() / pcl_conv_fwd_pool() first write a 4-channel, halo-padded, TF32-rounded copy of x
+ * to the first pcl_conv_staged_input_bytes(d) bytes of their workspace; a caller that keeps that workspace untouched
+ * until the backward pass hands its address to this call as x_staged (256-byte aligned) and saves staging x a second
+ * time.  Same result as pcl_conv_bwd_weights_pooled(), bit for bit.  pcl_conv_staged_input_bytes() is 0 for layers
+ * that stage nothing. */
+size_t pcl_conv_staged_input_bytes(const pcl_conv_desc* d);
+int pcl_conv_bwd_weights_pooled_staged(const pcl_conv_desc* d, const float* x_staged, const float* dy_pool,
+                                       const unsigned char* pool_codes, int relu_mask, float* dw, float* dbias,
+                                       void* ws, size_t ws_bytes, void* cuda_stream);
+
 /* Fully-connected forward: the k_h = k_w = out_h = out_w = 1 case of Algorithm 1
  * (Sec. 2.1):  y[n,k] = act(bias[k] + sum_c x[n,c] * w[k,c]).
  * x: [N][C], w: [K][C], bias: [K] or NULL, y: [N][K].

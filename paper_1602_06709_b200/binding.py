@@ -30,7 +30,8 @@ EXPORTS = [
     "pcl_conv_bwd_data_colsum_workspace_bytes", "pcl_conv_bwd_data_colsum",
     "pcl_maxpool2x2_bwd_colsum_workspace_bytes", "pcl_maxpool2x2_bwd_colsum", "pcl_conv_fwd_pool", "pcl_conv_fwd_pool_is_fused",
     "pcl_conv_bwd_weights_pooled", "pcl_conv_bwd_weights_pooled_is_fused", "pcl_conv_bwd_weights_pooled_workspace_bytes",
-    "pcl_maxpool2x2_fwd_codes", "pcl_maxpool2x2_bwd_codes", "pcl_last_wait_code", "pcl_set_tuning", "pcl_reset_tuning", "pcl_fc_bwd_fused", "pcl_conv_plan_describe",
+    "pcl_maxpool2x2_fwd_codes", "pcl_maxpool2x2_bwd_codes", "pcl_last_wait_code", "pcl_set_tuning", "pcl_reset_tuning", "pcl_fc_bwd_fused", "pcl_conv_plan_describe", "pcl_conv_staged_input_bytes",
+    "pcl_conv_bwd_weights_pooled_staged",
 ]
 
 
@@ -79,6 +80,9 @@ def lib() -> ctypes.CDLL:
         L.pcl_conv_bwd_weights_pooled_workspace_bytes.argtypes = [dp]
         L.pcl_conv_bwd_weights_pooled_workspace_bytes.restype = sz
         L.pcl_conv_bwd_weights_pooled.argtypes = [dp, vp, vp, vp, ci, vp, vp, vp, sz, vp]
+        L.pcl_conv_bwd_weights_pooled_staged.argtypes = [dp, vp, vp, vp, ci, vp, vp, vp, sz, vp]
+        L.pcl_conv_staged_input_bytes.argtypes = [dp]
+        L.pcl_conv_staged_input_bytes.restype = sz
         L.pcl_maxpool2x2_fwd_codes.argtypes = [ci, ci, ci, ci, vp, vp, vp, vp]
         L.pcl_maxpool2x2_bwd_codes.argtypes = [ci, ci, ci, ci, vp, vp, ci, vp, vp, vp, sz, vp]
         L.pcl_conv_bwd_weights.argtypes = [dp, vp, vp, vp, vp, ci, vp, sz, vp]
@@ -212,6 +216,19 @@ def conv_bwd_weights_pooled(d, x, dy_pool, pool_codes, relu_mask, dw, dbias=None
     _check(lib().pcl_conv_bwd_weights_pooled(ctypes.byref(d), _ptr(x), _ptr(dy_pool), _ptr(pool_codes),
                                              int(bool(relu_mask)), _ptr(dw), _ptr(dbias), wp, wb, _stream(stream)),
            "pcl_conv_bwd_weights_pooled")
+
+
+def conv_staged_input_bytes(d) -> int:
+    return int(lib().pcl_conv_staged_input_bytes(ctypes.byref(d)))
+
+
+def conv_bwd_weights_pooled_staged(d, x_staged, dy_pool, pool_codes, relu_mask, dw, dbias=None, ws=None, stream=None):
+    """conv_bwd_weights_pooled from the staged input that the layer's forward call left at the start of its workspace
+    (x_staged: that workspace tensor, kept untouched since)."""
+    wp, wb = _ws(ws)
+    _check(lib().pcl_conv_bwd_weights_pooled_staged(ctypes.byref(d), _ptr(x_staged), _ptr(dy_pool), _ptr(pool_codes),
+                                                    int(bool(relu_mask)), _ptr(dw), _ptr(dbias), wp, wb, _stream(stream)),
+           "pcl_conv_bwd_weights_pooled_staged")
 
 
 def maxpool2x2_fwd_codes(N, H, W, C, x, y, codes, stream=None):

@@ -756,13 +756,20 @@ size_t pcl_conv_bwd_weights_pooled_workspace_bytes(const pcl_conv_desc* d) {
     return plan_pooled_wgrad(*d, P, Q).total;
 }
 
-int pcl_conv_bwd_weights_pooled(const pcl_conv_desc* d, const float* x, const float* dy_pool,
-                                const unsigned char* pool_codes, int relu_mask, float* dw, float* dbias, void* ws,
-                                size_t ws_bytes, void* cuda_stream) {
+size_t pcl_conv_staged_input_bytes(const pcl_conv_desc* d) {
+    int P, Q;
+    if (check_desc(d, &P, &Q) != PCL_OK) return 0;
+    return few_channel_path_for(*d, PCL_PASS_FWD) ? staged_x_bytes(*d) : 0;
+}
+
+static int conv_bwd_weights_pooled_impl(const pcl_conv_desc* d, const float* x, const float* x_staged, const float* dy_pool,
+                                        const unsigned char* pool_codes, int relu_mask, float* dw, float* dbias, void* ws,
+                                        size_t ws_bytes, void* cuda_stream) {
     int P, Q;
     int rc = check_desc(d, &P, &Q);
     if (rc != PCL_OK) return rc;
-    if (!x || !dy_pool || !pool_codes || !dw) return PCL_ERR_BAD_ARG;
+    if ((!x && !x_staged) || !dy_pool || !pool_codes || !dw) return PCL_ERR_BAD_ARG;
+    if (x_staged && (reinterpret_cast<uintptr_t>(x_staged) & 255)) return PCL_ERR_MISALIGNED;
     PassScope pass_scope(PROF_PASS_CONV_BWD_WEIGHTS, conv_pass_flops(*d, P, Q));
     if (!aligned16(x) || !aligned16(dy_pool) || !aligned16(pool_codes) || !aligned16(dw) || !aligned16(dbias))
         return PCL_ERR_MISALIGNED;
@@ -771,12 +778,15 @@ int pcl_conv_bwd_weights_pooled(const pcl_conv_desc* d, const float* x, const fl
     if (!ws || ws_bytes < pl.total) return PCL_ERR_WORKSPACE;
     if (reinterpret_cast<uintptr_t>(ws) & 255) return PCL_ERR_MISALIGNED;
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
-    float* xs = static_cast<float*>(ws);
+    // the staged copy: the caller's (left by this layer's forward call at the start of its workspace), or made here
+    const float* xs = x_staged ? x_staged : static_cast<const float*>(ws);
     float* dw4 = reinterpret_cast<float*>(static_cast<char*>(ws) + pl.tiles_off);
     float* rows = reinterpret_cast<float*>(static_cast<char*>(ws) + pl.rows_off);
     float* cs = reinterpret_cast<float*>(static_cast<char*>(ws) + pl.cs_off);
-    rc = launch_stage_pad_c4(x, xs, d->N, d->H, d->W, d->C, d->pad_h, d->pad_w, few_slack_pixels(*d), st);
-    if (rc != PCL_OK) return rc;
+    if (!x_staged) {
+        rc = launch_stage_pad_c4(x, static_cast<float*>(ws), d->N, d->H, d->W, d->C, d->pad_h, d->pad_w, few_slack_pixels(*d), st);
+        if (rc != PCL_OK) return rc;
+    }
     const int Hp = d->H + 2 * d->pad_h, Wp = d->W + 2 * d->pad_w;
     const size_t taps = size_t(d->K) * d->R * d->S;
     TcWgradArgs a{xs, nullptr, dw4, pl.splits > 1 ? dw4 : nullptr, d->N, Hp, Q, d->S * 4, d->K, d->R, 1, 0, 0, P, Q,
@@ -792,6 +802,20 @@ int pcl_conv_bwd_weights_pooled(const pcl_conv_desc* d, const float* x, const fl
     if (rc != PCL_OK) return rc;
     if (dbias) rc = launch_colsum(rows, size_t(pl.splits) * 8, d->K, cs, dbias, st);       // adds the rows, fixed order
     return rc;
+}
+
+int pcl_conv_bwd_weights_pooled(const pcl_conv_desc* d, const float* x, const float* dy_pool,
+                                const unsigned char* pool_codes, int relu_mask, float* dw, float* dbias, void* ws,
+                                size_t ws_bytes, void* cuda_stream) {
+    if (!x) return PCL_ERR_BAD_ARG;
+    return conv_bwd_weights_pooled_impl(d, x, nullptr, dy_pool, pool_codes, relu_mask, dw, dbias, ws, ws_bytes, cuda_stream);
+}
+
+int pcl_conv_bwd_weights_pooled_staged(const pcl_conv_desc* d, const float* x_staged, const float* dy_pool,
+                                       const unsigned char* pool_codes, int relu_mask, float* dw, float* dbias, void* ws,
+                                       size_t ws_bytes, void* cuda_stream) {
+    if (!x_staged) return PCL_ERR_BAD_ARG;
+    return conv_bwd_weights_pooled_impl(d, nullptr, x_staged, dy_pool, pool_codes, relu_mask, dw, dbias, ws, ws_bytes, cuda_stream);
 }
 
 int pcl_conv_bwd_weights(const pcl_conv_desc* d, const float* x, const float* dy, float* dw, float* dbias,

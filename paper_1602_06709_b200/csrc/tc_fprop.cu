@@ -289,7 +289,9 @@ __device__ __noinline__ void mma_issuer(const FpropParams& p, const IssuerCtx& c
     if (kDuo && split) *issue_seq = seq + 1;     /* split: only the slot STARTS are ordered (see below) */        \
     tc_fence_after();
 #define PCL_SLOT_RELEASE()                                                                                        \
-    if (kDuo && !split) *issue_seq = seq + 1;                                                                     \
+    /* ordered hand-over: this thread's MMAs are fenced before the turn is published (the other issuer fences  */ \
+    /* after reading it), so that MMAs of consecutive slots into one accumulator are ordered across the threads */ \
+    if (kDuo && !split) { tc_fence_before(); *issue_seq = seq + 1; }                                              \
     if (!resident) umma_commit_addr<kPair>(empty_a);
 #define PCL_SLOT_END()                                                                                            \
     if (kDuo) ++seq;                                                                                              \

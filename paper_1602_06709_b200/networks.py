@@ -210,6 +210,12 @@ class VggA(_HostFeed):
         for C, K in fc:
             ws = max(ws, B.fc_workspace_bytes(N, C, K, B.PASS_BWD_DATA), B.fc_workspace_bytes(N, C, K, B.PASS_FWD))
         self.ws = torch.empty(max(ws, 256), dtype=torch.uint8, device=dev)
+        # The first layer's forward call stages its few-channel input at the start of its workspace; with a workspace
+        # of its own, kept until the backward pass, its weight gradient reads that copy instead of staging x again.
+        self.ws_first = None
+        if self.first_from_pooled and B.conv_staged_input_bytes(self.convs[0].desc) > 0:
+            self.ws_first = torch.empty(max(256, B.conv_workspace_bytes(self.convs[0].desc, B.PASS_FWD)), dtype=torch.uint8,
+                                        device=dev)
         self.conv_flops_fwd = [2 * N * L.K * L.H * L.W * L.C * 9 for L in self.convs]
         self.fc_flops_fwd = [2 * N * C * K for C, K in fc]
 
@@ -240,7 +246,8 @@ class VggA(_HostFeed):
                 before_layer(i)
             if L.pool:      # conv -> ReLU -> 2x2 pool, the maxima taken in the convolution's epilogue
                 B.conv_fwd_pool(L.desc, self.layer_input(i), self.conv_w(i), self.conv_b(i), self.y[i], self.pooled[i],
-                                B.ACT_RELU, self.ws, pool_codes=self.pool_codes[i])
+                                B.ACT_RELU, self.ws_first if (i == 0 and self.ws_first is not None) else self.ws,
+                                pool_codes=self.pool_codes[i])
             else:
                 B.conv_fwd(L.desc, self.layer_input(i), self.conv_w(i), self.conv_b(i), self.y[i], B.ACT_RELU, self.ws)
         a = self.pooled[-1].view(self.N, self.flat)
@@ -276,8 +283,12 @@ class VggA(_HostFeed):
             # dy[i] (the pool backward here, or the backward-data pass of layer i+1 below), not by a separate pass.
             if i == 0 and self.first_from_pooled:
                 # pooling backward, ReLU mask, bias gradient and weight gradient in one pass over the pooled gradient
-                B.conv_bwd_weights_pooled(L.desc, self.layer_input(0), self.dpooled[0], self.pool_codes[0], True,
-                                          self.conv_dw(0), self.conv_db(0), self.ws)
+                if self.ws_first is not None:
+                    B.conv_bwd_weights_pooled_staged(L.desc, self.ws_first, self.dpooled[0], self.pool_codes[0], True,
+                                                     self.conv_dw(0), self.conv_db(0), self.ws)
+                else:
+                    B.conv_bwd_weights_pooled(L.desc, self.layer_input(0), self.dpooled[0], self.pool_codes[0], True,
+                                              self.conv_dw(0), self.conv_db(0), self.ws)
                 if after_layer:
                     after_layer(0)
                 if after_backprop:

@@ -372,6 +372,17 @@ def test_weight_gradient_from_pooled_gradient(tag, relu, path_guard):
     B.conv_bwd_weights_pooled(d, G.dev(x), G.dev(dyp), torch.from_numpy(codes).cuda(), relu, dw2, None, ws)
     B.check_device_status()
     assert np.array_equal(dw2.cpu().numpy(), outs[0][0])
+    # from the staged input that the layer's forward call leaves at the start of its workspace: bit for bit the same
+    n_staged = B.conv_staged_input_bytes(d)
+    assert n_staged > 0
+    ws_f = G.workspace(B.conv_workspace_bytes(d, B.PASS_FWD))
+    assert ws_f.numel() >= n_staged
+    w = inputs.normal(inputs.tensor_id("pooled_wgrad", tag, "w"), (s.K, s.R, s.S, s.C), 0.3)
+    B.conv_fwd(d, G.dev(x), G.dev(w), None, G.guarded((s.N, s.P, s.Q, s.K)), B.ACT_RELU, ws_f)
+    dw3 = G.guarded((s.K, s.R, s.S, s.C)); db3 = G.guarded((s.K,))
+    B.conv_bwd_weights_pooled_staged(d, ws_f, G.dev(dyp), torch.from_numpy(codes).cuda(), relu, dw3, db3, ws)
+    B.check_device_status()
+    assert np.array_equal(dw3.cpu().numpy(), outs[0][0]) and np.array_equal(db3.cpu().numpy(), outs[0][1])
 
 
 def test_weight_gradient_from_pooled_gradient_only_where_fused():
