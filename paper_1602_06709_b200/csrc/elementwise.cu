@@ -613,6 +613,70 @@ int launch_transpose_flip(const float* w, float* wt_t, int K, int R, int S, int 
     return PCL_CHECK_LAUNCH();
 }
 
+// Phase-packed backward-data of strided layers with few input maps (see conv_bwd_data_packed in pcl_api.cu).
+// wpk[col][i'][j'][k], col = (a*sw + b)*C + c: w[k][a + sh*(Rm-1-i')][b + sw*(Sm-1-j')][c] where that tap exists, else 0;
+// columns >= sh*sw*C (padding to a multiple of 4) are zero.
+__global__ void __launch_bounds__(256) phase_pack_weights_kernel(const float* __restrict__ w, float* __restrict__ wpk, int K,
+                                                                 int R, int S, int C, int sh, int sw, int Rm, int Sm,
+                                                                 int cols4) {
+    const size_t total = size_t(cols4) * Rm * Sm * K;
+    const size_t stride = size_t(gridDim.x) * blockDim.x;
+    for (size_t o = size_t(blockIdx.x) * blockDim.x + threadIdx.x; o < total; o += stride) {
+        const int k = int(o % K); size_t t = o / K;
+        const int jj = int(t % Sm); t /= Sm;
+        const int ii = int(t % Rm); const int col = int(t / Rm);
+        float v = 0.f;
+        if (col < sh * sw * C) {
+            const int c = col % C, ab = col / C, b = ab % sw, a = ab / sw;
+            const int r = a + sh * (Rm - 1 - ii), s2 = b + sw * (Sm - 1 - jj);
+            if (r < R && s2 < S) v = w[((size_t(k) * R + r) * S + s2) * C + c];
+        }
+        wpk[o] = v;
+    }
+}
+// dx[n][h][w][c] = t[n][u][v][(a*sw + b)*C + c] with h + pad_h = u*sh + a, w + pad_w = v*sw + b (zeroed where mask <= 0).
+// One block per image row of dx: the row's (u, a) are block constants and the per-element index arithmetic is 32-bit.
+__global__ void __launch_bounds__(256) phase_unpack_kernel(const float* __restrict__ t, const float* __restrict__ mask,
+                                                           float* __restrict__ dx, int H, int W, int C, int sh, int sw,
+                                                           int pad_h, int pad_w, int U, int V, int cols4) {
+    const size_t row = blockIdx.x;                       // n * H + h
+    const size_t n = row / H;
+    const int hh = int(row - n * H);
+    const int u = (hh + pad_h) / sh, a = (hh + pad_h) - u * sh;
+    const float* trow = t + ((n * U + u) * V) * size_t(cols4) + a * sw * C;
+    const size_t o0 = row * size_t(W) * C;
+    const int row_elems = W * C;
+    for (int e = threadIdx.x; e < row_elems; e += blockDim.x) {
+        const int ww = e / C, c = e - ww * C;
+        const int v = (ww + pad_w) / sw, b = (ww + pad_w) - v * sw;
+        float val = __ldg(trow + v * cols4 + b * C + c);
+        if (mask && !(__ldg(mask + o0 + e) > 0.f)) val = 0.f;
+        dx[o0 + e] = val;
+    }
+}
+
+int launch_phase_pack_weights(const float* w, float* wpk, int K, int R, int S, int C, int sh, int sw, int Rm, int Sm,
+                              int cols4, cudaStream_t st) {
+    const size_t total = size_t(cols4) * Rm * Sm * K;
+    {
+        LaunchScope scope(KID_TRANSPOSE_FLIP, 8.0 * double(total), st);
+        phase_pack_weights_kernel<<<grid_for(total, 256), 256, 0, st>>>(w, wpk, K, R, S, C, sh, sw, Rm, Sm, cols4);
+    }
+    return PCL_CHECK_LAUNCH();
+}
+
+int launch_phase_unpack(const float* t, const float* mask, float* dx, int N, int H, int W, int C, int sh, int sw, int pad_h,
+                        int pad_w, int U, int V, int cols4, cudaStream_t st) {
+    const size_t total = size_t(N) * H * W * C;
+    {
+        LaunchScope scope(KID_UNPAD_REDUCE, (mask ? 12.0 : 8.0) * double(total), st);
+        const size_t rows = size_t(N) * H;
+        if (rows > 0x7fffffffu) return PCL_ERR_UNSUPPORTED_SHAPE;
+        phase_unpack_kernel<<<unsigned(rows), 256, 0, st>>>(t, mask, dx, H, W, C, sh, sw, pad_h, pad_w, U, V, cols4);
+    }
+    return PCL_CHECK_LAUNCH();
+}
+
 int launch_phase_weights(const float* w, float* wt_t, int K, int R, int S, int C, int a, int b, int stride_h,
                          int stride_w, int Ra, int Sb, cudaStream_t st) {
     const size_t total = size_t(C) * Ra * Sb * K;

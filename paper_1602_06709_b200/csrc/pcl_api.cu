@@ -41,7 +41,7 @@ std::atomic<unsigned> g_tune_gen{0};
 const char* const kTuneNames[TUNE_COUNT] = {
     "TILING", "BN", "KS", "KS_HALO", "KS_WGRAD", "PAIR", "PAIR_HALO", "PAIR_WGRAD", "GRP", "ISSUERS", "SPLIT_ACC",
     "PIX_WGRAD", "XHALO_WGRAD", "TMA_STORE", "WEIGHTS_IN_PLACE", "EPI_WARPS", "FC_DW_FORWARD", "KSPLIT",
-    "WAIT_LIMIT_US", "FAULT_INJECT", "RESIDENT_B", "KSLICES", "SELECT"};
+    "WAIT_LIMIT_US", "FAULT_INJECT", "RESIDENT_B", "KSLICES", "SELECT", "PACKED_BWD"};
 }  // namespace
 
 int tune(int id, int dflt) {
@@ -177,14 +177,34 @@ bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 
 bool weights_read_in_place(const pcl_conv_desc& d) { return d.C % 32 == 0 && tune(TUNE_WEIGHTS_IN_PLACE, 1) != 0; }
 
 size_t dw_bytes(const pcl_conv_desc& d);
+// Backward-data of a strided layer whose stride_h * stride_w * C fits one tile width runs as ONE stride-1 convolution
+// whose output maps are (phase, input map) pairs, plus a scatter of that output to dx; wider layers run one launch per
+// phase (conv_bwd_data_phases).
+struct StridedBwdPlan { bool packed; int Rm, Sm, U, V, cols4; size_t wpk_bytes, temp_bytes; };
+StridedBwdPlan strided_bwd_plan(const pcl_conv_desc& d) {
+    StridedBwdPlan p{};
+    const int cols = d.stride_h * d.stride_w * d.C;
+    p.cols4 = (cols + 3) / 4 * 4;
+    p.Rm = (d.R + d.stride_h - 1) / d.stride_h; p.Sm = (d.S + d.stride_w - 1) / d.stride_w;
+    p.U = (d.H - 1 + d.pad_h) / d.stride_h + 1; p.V = (d.W - 1 + d.pad_w) / d.stride_w + 1;
+    p.packed = p.cols4 <= 256 && d.K % 4 == 0;
+    p.wpk_bytes = align_up(size_t(p.cols4) * p.Rm * p.Sm * d.K * 4, 256);
+    p.temp_bytes = align_up(size_t(d.N) * p.U * p.V * p.cols4 * 4, 256);
+    return p;
+}
 }  // namespace
 
 // Bytes of the flipped, transposed weight copy backward-data makes on the tensor-core path (0 where the weights
 // are read in place or another kernel family runs): the part of the backward-data workspace that is mandatory.
 size_t bwd_data_transposed_bytes(const pcl_conv_desc& d) {
     if (g_path.load() == PCL_PATH_GENERIC || d.K % 4 != 0) return 0;
-    if (d.stride_h != 1 || d.stride_w != 1)       // one flipped, transposed sub-kernel per phase, each 256-byte aligned
-        return d.stride_h <= 8 && d.stride_w <= 8 ? dw_bytes(d) + size_t(256) * d.stride_h * d.stride_w : 0;
+    if (d.stride_h != 1 || d.stride_w != 1) {
+        if (d.stride_h > 8 || d.stride_w > 8) return 0;
+        const StridedBwdPlan sp = strided_bwd_plan(d);
+        const size_t phases = dw_bytes(d) + size_t(256) * d.stride_h * d.stride_w;    // one flipped, transposed sub-kernel per phase, 256-byte aligned
+        const size_t packed = sp.wpk_bytes + sp.temp_bytes;
+        return sp.packed && packed > phases ? packed : phases;
+    }
     if (!(d.pad_h <= d.R - 1 && d.pad_w <= d.S - 1)) return 0;
     return weights_read_in_place(d) ? 0 : dw_bytes(d);
 }
@@ -467,6 +487,24 @@ namespace {
 // w[k][a + i*stride_h][b + j*stride_w][c], written to every stride-th pixel of dx: stride_h * stride_w launches of
 // the forward-type kernel, each with its own transposed sub-kernel in the workspace.  Pixels of phases without taps
 // (a stride larger than the kernel) are zeroed first.
+// Few input maps: all phases at once.  With h + pad_h = u*stride_h + a the rule reads
+//   dx[n, h, w, c] = sum_{k, i, j} dy[n, u - i, v - j, k] * w[k, a + i*stride_h, b + j*stride_w, c],
+// a stride-1 convolution of dy with a ceil(R/stride_h) x ceil(S/stride_w) kernel whose output map index is (a, b, c)
+// (taps a phase does not have are zero weights); its output is scattered to dx by a bandwidth-bound pass.
+int conv_bwd_data_packed(const pcl_conv_desc& d, const StridedBwdPlan& sp, int P, int Q, const float* dy, const float* w,
+                         const float* mask, float* dx, char* ws, cudaStream_t st) {
+    float* wpk = reinterpret_cast<float*>(ws);
+    float* temp = reinterpret_cast<float*>(ws + sp.wpk_bytes);
+    int rc = launch_phase_pack_weights(w, wpk, d.K, d.R, d.S, d.C, d.stride_h, d.stride_w, sp.Rm, sp.Sm, sp.cols4, st);
+    if (rc != PCL_OK) return rc;
+    TcFpropArgs t{dy, wpk, nullptr, nullptr, temp, d.N, P, Q, d.K, sp.cols4, sp.Rm, sp.Sm, sp.Rm - 1, sp.Sm - 1, sp.U, sp.V,
+                  PCL_ACT_NONE};
+    rc = launch_tc_fprop(t, st);
+    if (rc != PCL_OK) return rc;
+    return launch_phase_unpack(temp, mask, dx, d.N, d.H, d.W, d.C, d.stride_h, d.stride_w, d.pad_h, d.pad_w, sp.U, sp.V,
+                               sp.cols4, st);
+}
+
 int conv_bwd_data_phases(const pcl_conv_desc& d, int P, int Q, const float* dy, const float* w, const float* mask,
                          float* dx, char* ws, cudaStream_t st) {
     const int sh = d.stride_h, sw = d.stride_w;
@@ -516,7 +554,13 @@ int pcl_conv_bwd_data(const pcl_conv_desc* d, const float* dy, const float* w, c
         const size_t need = bwd_data_transposed_bytes(*d);
         if (need > 0 && (!ws || ws_bytes < need)) return PCL_ERR_WORKSPACE;
         if (ws && (reinterpret_cast<uintptr_t>(ws) & 255)) return PCL_ERR_MISALIGNED;
-        if (!unit_stride(*d)) return conv_bwd_data_phases(*d, P, Q, dy, w, relu_mask_src, dx, static_cast<char*>(ws), st);
+        if (!unit_stride(*d)) {
+            const StridedBwdPlan sp = strided_bwd_plan(*d);
+            if (sp.packed && tune(TUNE_PACKED_BWD, 1))
+                return conv_bwd_data_packed(*d, sp, P, Q, dy, w, relu_mask_src, dx, static_cast<char*>(ws), st);
+            if (ws_bytes < dw_bytes(*d) + size_t(256) * d->stride_h * d->stride_w) return PCL_ERR_WORKSPACE;
+            return conv_bwd_data_phases(*d, P, Q, dy, w, relu_mask_src, dx, static_cast<char*>(ws), st);
+        }
         // dx = "forward" convolution of dy with the flipped, transposed weights, pad' = R-1-pad
         TcFpropArgs a{dy, w, nullptr, relu_mask_src, dx, d->N, P, Q, d->K, d->C, d->R, d->S,
                       d->R - 1 - d->pad_h, d->S - 1 - d->pad_w, d->H, d->W, PCL_ACT_NONE};

@@ -54,7 +54,7 @@ enum TuneId {
     TUNE_TILING = 0,        // forward-type kernel: 0 plain, 1-3 haloed layouts 0-2
     TUNE_BN, TUNE_KS, TUNE_KS_HALO, TUNE_KS_WGRAD, TUNE_PAIR, TUNE_PAIR_HALO, TUNE_PAIR_WGRAD, TUNE_GRP, TUNE_ISSUERS,
     TUNE_SPLIT_ACC, TUNE_PIX_WGRAD, TUNE_XHALO_WGRAD, TUNE_TMA_STORE, TUNE_WEIGHTS_IN_PLACE, TUNE_EPI_WARPS,
-    TUNE_FC_DW_FORWARD, TUNE_KSPLIT, TUNE_WAIT_LIMIT_US, TUNE_FAULT_INJECT, TUNE_RESIDENT_B, TUNE_KSLICES, TUNE_SELECT, TUNE_COUNT
+    TUNE_FC_DW_FORWARD, TUNE_KSPLIT, TUNE_WAIT_LIMIT_US, TUNE_FAULT_INJECT, TUNE_RESIDENT_B, TUNE_KSLICES, TUNE_SELECT, TUNE_PACKED_BWD, TUNE_COUNT
 };
 int tune(int id, int dflt);
 bool tune_is_set(int id);
@@ -226,6 +226,13 @@ int launch_transpose_flip(const float* w, float* wt_t, int K, int R, int S, int 
 // i < Ra, j < Sb (the taps that reach input pixels of phase (a, b), flipped and transposed).
 int launch_phase_weights(const float* w, float* wt_t, int K, int R, int S, int C, int a, int b, int stride_h,
                          int stride_w, int Ra, int Sb, cudaStream_t st);
+// Phase-packed backward-data (strided layers with stride_h * stride_w * C <= 256): the sub-kernels of all phases as the
+// output maps of ONE stride-1 convolution (wpk[col][Rm][Sm][K], col = (a*sw + b)*C + c, zero where a phase has no such
+// tap), and the scatter of its output t[N][U][V][cols4] to dx (optionally zeroed where mask <= 0).
+int launch_phase_pack_weights(const float* w, float* wpk, int K, int R, int S, int C, int sh, int sw, int Rm, int Sm,
+                              int cols4, cudaStream_t st);
+int launch_phase_unpack(const float* t, const float* mask, float* dx, int N, int H, int W, int C, int sh, int sw, int pad_h,
+                        int pad_w, int U, int V, int cols4, cudaStream_t st);
 // Few-channel staging (C < 4): xs[n][h+pad_h][w+pad_w][0..3] = x[n][h][w][0..C-1] padded with zeros (channel
 // padding and a spatial halo of pad_h / pad_w), followed by `slack_pixels` zero pixels; w32[row][s*4 + c] =
 // w[row][s][c] (row = k*R + r) in zero-padded rows of row_floats (a multiple of 32) floats;

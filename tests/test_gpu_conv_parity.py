@@ -396,3 +396,20 @@ def test_weight_gradient_from_pooled_gradient_only_where_fused():
         B.conv_bwd_weights_pooled(d, z(2, 8, 8, 32), z(2, 4, 4, 32), torch.zeros(2, 4, 4, 32, dtype=torch.uint8, device="cuda"),
                                   True, z(32, 3, 3, 32), None, G.workspace(1 << 20))
     assert e.value.code == B.ERR_UNSUPPORTED_SHAPE
+
+
+@pytest.mark.parametrize("form", ["packed", "phases"])
+@pytest.mark.parametrize("tag", sorted(STRIDED_SHAPES))
+def test_strided_backward_data_both_forms(tag, form, path_guard):
+    """Backward-data of a strided layer runs either as one stride-1 convolution whose output maps are (phase, input
+    map) pairs followed by a scatter (layers with stride_h * stride_w * C <= 256), or as one launch per phase
+    (the PACKED_BWD knob = 0 forces that form): both against the oracle, with and without the ReLU mask."""
+    from paper_1602_06709_b200 import binding as B
+    s = STRIDED_SHAPES[tag]
+    if s.stride_h == 1 and s.stride_w == 1:
+        pytest.skip("stride-1 layer")
+    B.set_path(B.PATH_TENSOR)
+    B.set_tuning("PACKED_BWD", 1 if form == "packed" else 0)
+    x, w, dy, _ = G.make_inputs(s, "strided_bwd_" + tag)
+    G.assert_parity(G.run_conv_bwd_data(s, dy, w, None), oracle.conv_bwd_data(s, dy, w), f"bwd_data {form}")
+    G.assert_parity(G.run_conv_bwd_data(s, dy, w, x), oracle.conv_bwd_data(s, dy, w, x), f"bwd_data {form} masked")
