@@ -1223,9 +1223,9 @@ TileCfg search_cfg(const TcFpropArgs& a, int sm_count, TileCost* best_cost = nul
 // The tiling a launch will use (also needed to size the fused column-sum rows).
 TileCfg select_cfg(const TcFpropArgs& a, int sm_count) {
     const int cblocks = (a.Cin + kBlockC - 1) / kBlockC;
-    // Convolutions (more than one tap) take the candidate the cost model predicts fastest; the measured table of the
-    // blocking search (profiles/) has it within a few percent of the measured best on every layer of the benchmark
-    // configurations.  1 x 1 layers (the FC GEMMs) keep the rules below, which also decide their reduction splits.
+    // Convolutions (more than one tap) take the candidate the cost model predicts fastest; measured against every
+    // candidate (python -m paper_1602_06709_b200.blocking_search) it is within a few percent of the measured best on
+    // every VGG-A and OverFeat-FAST layer at minibatch 256.  1 x 1 layers (the FC GEMMs) keep the rules below, which also decide their reduction splits.
     // SELECT = 0 switches the model off, 1 applies it to every launch; a pinned knob always wins.
     // (the few-channel path reads overlapping windows, whose fill cost the model does not describe: rules too)
     const int sel = tune(TUNE_SELECT, (a.R * a.S > 1 && a.in_stride_w == 0) ? 1 : 0);
