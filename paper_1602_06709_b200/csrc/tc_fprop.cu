@@ -97,6 +97,7 @@ struct FpropParams {
     // K = 8 slices of a 32-element channel block that hold anything but zeros (4 unless the few-channel path packs
     // fewer live taps x channels into a block: the MMAs of all-zero slices are not issued)
     int kslices;
+    int tile_duo;           // two issuing threads, alternate tiles (resident weights, one patch per tile, even NA)
     int bias_in_smem;           // the CTA keeps bias[0 .. BN) in shared memory (tiles_k == 1: every tile has the same columns)
     unsigned char* pool_idx;    // optional, with pool_out: per pooled element the position of the maximum (bits 0-1) and bit 2
                                 // if that maximum is <= 0
@@ -200,14 +201,30 @@ __device__ __forceinline__ void add_second_accumulator(uint32_t taddr, uint32_t 
 }
 
 // kTaps consecutive taps of a haloed slot, straight-line (a taken branch costs a lone thread tens of cycles).
-template <bool kPair, int kTaps, int kMT>
+// kNsl = 0: the number of K = 8 slices per tap is the run-time `nsl` (skipped slices still cost their issue slots);
+// kNsl = 1..3: exactly that many MMAs per tap are emitted (few-channel layers, whose tap rows hold fewer than 32
+// live reduction elements: the issuing thread, not the tensor pipe, is what bounds their tiles).
+template <bool kPair, int kTaps, int kMT, int kNsl = 0>
 __device__ __forceinline__ void halo_taps(uint32_t d_tmem, uint32_t BN, uint32_t& a_lo, uint32_t b_lo, int& s, int S,
                                           uint32_t row16, uint32_t half_off16, uint32_t b16, uint32_t a_hi,
                                           uint32_t b_hi, uint32_t idesc, uint32_t& accum, uint32_t bks, uint32_t nsl) {
 #pragma unroll
     for (int j = 0; j < kTaps; ++j) {
-        umma_kstep_tf32_bs<kPair>(d_tmem, a_lo, b_lo, a_hi, b_hi, idesc, accum, bks, nsl);
-        if (kMT == 2) umma_kstep_tf32_bs<kPair>(d_tmem + BN, a_lo + half_off16, b_lo, a_hi, b_hi, idesc, accum, bks, nsl);
+        if constexpr (kNsl == 0) {
+            umma_kstep_tf32_bs<kPair>(d_tmem, a_lo, b_lo, a_hi, b_hi, idesc, accum, bks, nsl);
+            if (kMT == 2) umma_kstep_tf32_bs<kPair>(d_tmem + BN, a_lo + half_off16, b_lo, a_hi, b_hi, idesc, accum, bks, nsl);
+        } else {
+#pragma unroll
+            for (int h = 0; h < kMT; ++h) {
+#pragma unroll
+                for (int k = 0; k < kNsl; ++k) {
+                    const uint64_t da = (uint64_t(a_hi) << 32) | (a_lo + (h ? half_off16 : 0u) + 2u * k);
+                    const uint64_t db = (uint64_t(b_hi) << 32) | (b_lo + bks * k);
+                    if constexpr (kPair) umma_tf32_pair(d_tmem + (h ? BN : 0u), da, db, idesc, k == 0 ? accum : 1u);
+                    else umma_tf32(d_tmem + (h ? BN : 0u), da, db, idesc, k == 0 ? accum : 1u);
+                }
+            }
+        }
         accum = 1;
         b_lo += b16;
         const bool wrap = ++s == S;     // the tap (r, s): next pixel of the patch, or the start of the next patch row
@@ -274,16 +291,20 @@ __device__ __noinline__ void mma_issuer(const FpropParams& p, const IssuerCtx& c
     int stage = 0;
     uint32_t phase = 0;
     uint32_t turn = 0, seq = 0;     // kDuo: whose slot comes next; slots so far (both threads count alike)
-    int a_slot = 0;
+    // tile_duo: the two issuing threads take the CTA's tiles alternately, each with its own accumulator set and its
+    // own patch buffers (NA is even), so nothing orders them against each other; the weights stay resident.
+    const bool tduo = !kDuo && p.tile_duo != 0;
+    const int cnt0 = tduo ? int(issuer) : 0, cnt_step = tduo ? 2 : 1;
+    int a_slot = cnt0;
     uint32_t phaseA = 0;
-    int tile_cnt = 0;
+    int tile_cnt = cnt0;
     bool ok = true;
 
 #define PCL_SLOT_BEGIN()                                                                                          \
     bool mine = true;                                                                                             \
     if (kDuo) { mine = turn == issuer; turn ^= 1u; }
 #define PCL_SLOT_ACQUIRE()                                                                                        \
-    if (!(resident && tile_cnt > 0) &&                                                                            \
+    if (!(resident && tile_cnt > cnt0) &&                                                                         \
         !bounded_wait_addr(full_a, phase, abort_flag, status, WAIT_MMA_FULL)) { ok = false; break; }             \
     if (kDuo && !wait_issue_turn(issue_seq, seq, abort_flag, status)) { ok = false; break; }                     \
     if (kDuo && split) *issue_seq = seq + 1;     /* split: only the slot STARTS are ordered (see below) */        \
@@ -299,7 +320,7 @@ __device__ __noinline__ void mma_issuer(const FpropParams& p, const IssuerCtx& c
     full_a += 8; empty_a += 8; slot_lo += stage16;                                                                \
     if (++stage == stages) { stage = 0; phase ^= 1u; full_a = full0; empty_a = empty0; slot_lo = ring_lo0; }
 
-    for (int t = first_tile; t < total_tiles && ok; t += tile_stride, ++tile_cnt) {
+    for (int t = first_tile + cnt0 * tile_stride; t < total_tiles && ok; t += cnt_step * tile_stride, tile_cnt += cnt_step) {
         const uint32_t acc = tile_cnt & 1;
         const uint32_t acc_phase = (tile_cnt >> 1) & 1;
         if (!bounded_wait_addr(tempty0 + acc * 8, acc_phase ^ 1u, abort_flag, status, WAIT_MMA_TMEM_EMPTY)) break;
@@ -322,7 +343,8 @@ __device__ __noinline__ void mma_issuer(const FpropParams& p, const IssuerCtx& c
                     if (mine) {
                         PCL_SLOT_ACQUIRE()
                         if (MT == 2) {
-                            if (nst == 3) halo_taps<kPair, 3, 2>(d_tmem, BN, a_lo, slot_lo, s, S, row16, half_off16, b16, a_hi, b_hi, idesc, accum, bks, nsl);
+                            if (nst == 3 && nsl == 2) halo_taps<kPair, 3, 2, 2>(d_tmem, BN, a_lo, slot_lo, s, S, row16, half_off16, b16, a_hi, b_hi, idesc, accum, bks, nsl);
+                            else if (nst == 3) halo_taps<kPair, 3, 2>(d_tmem, BN, a_lo, slot_lo, s, S, row16, half_off16, b16, a_hi, b_hi, idesc, accum, bks, nsl);
                             else if (nst == 2) halo_taps<kPair, 2, 2>(d_tmem, BN, a_lo, slot_lo, s, S, row16, half_off16, b16, a_hi, b_hi, idesc, accum, bks, nsl);
                             else {
                                 uint32_t b_lo = slot_lo;
@@ -349,7 +371,8 @@ __device__ __noinline__ void mma_issuer(const FpropParams& p, const IssuerCtx& c
                     PCL_SLOT_END()
                 }
                 if (ok) umma_commit_addr<kPair>(emptyA0 + a_slot * 8);       // one arrival per issuer
-                if (++a_slot == NA) { a_slot = 0; phaseA ^= 1u; }
+                a_slot += cnt_step;
+                if (a_slot >= NA) { a_slot -= NA; phaseA ^= 1u; }
             }
         } else if (KS == 2 && grp) {
             // two k-steps per slot, fetched by one copy per operand (the hot loop of the wide layers)
@@ -608,7 +631,7 @@ tc_fprop_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
     } else if (warp == 1 || warp == kSecondIssuerWarp) {
         // --------------------------------------------------------- MMA issuers
         const uint32_t issuer = warp == 1 ? 0u : 1u;
-        if (lane == 0 && pair_rank == 0 && issuer < uint32_t(p.issuers)) {
+        if (lane == 0 && pair_rank == 0 && issuer < uint32_t(p.tile_duo ? 2 : p.issuers)) {
             IssuerCtx c;
             c.smem = smem; c.b_ring = b_ring;
             c.full_bar = full_bar; c.empty_bar = empty_bar; c.fullA_bar = fullA_bar; c.emptyA_bar = emptyA_bar;
@@ -635,6 +658,128 @@ tc_fprop_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
         const bool vec_ok = (p.Kout & 3) == 0;
         int tile_cnt = 0;
         TileIter it;
+        bool pooled_only = false;
+        if constexpr (kPool) pooled_only = !p.out && p.act != PCL_ACT_SIGMOID && (kEpi > kEpiWarps || (!kMask && p.tma_store));
+        if (pooled_only) {
+            // Pooled output only (the step never reads the full-resolution output of a pooled layer).  The raw
+            // accumulators are staged, each lane takes two windows of its four columns, adds the bias to the four
+            // values s_e of a window, takes their maximum m and applies the activation to m alone: max commutes with
+            // the (monotone) bias add and ReLU, so the stored maximum is bit for bit the maximum of the finished
+            // values.  Position code: the first e with act(s_e) == act(m), i.e. with s_e == m, except that under ReLU a
+            // window with m <= 0 holds four zeros, whose first maximum is e = 0.
+            // Few-channel layers are bound by these warps, not by the tensor pipe: everything that does not depend on
+            // the tile is computed once, a box without a chunk for this warp costs it nothing, and the accumulator set
+            // is handed back as soon as the warp's last chunk is in registers.
+            const int lb = p.bw_log2;
+            const uint32_t stg = smem_u32(epi_stage + epi * 4096);
+            const uint32_t my_row = stg + lane * 128, my_x = (lane & 7) * 16;
+            const int P2 = p.P >> 1, Q2 = p.Q >> 1;
+            uint32_t ld_a[2][4];
+            int wdq[2], wdp[2], wdn[2];
+            uint32_t woff[2];           // the window's pooled element inside the tile's pooled block (+ this lane's columns)
+#pragma unroll
+            for (int half = 0; half < 2; ++half) {
+                const int wdx = (lane >> 3) + 4 * half;
+                const int r0 = ((wdx & ((1 << (lb - 1)) - 1)) << 1) | ((wdx >> (lb - 1)) << (lb + 1));
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    const int rr = r0 | (e & 1) | ((e >> 1) << lb);
+                    ld_a[half][e] = stg + rr * 128 + (((lane & 7) ^ (rr & 7)) * 16);
+                }
+                const int wrow = quarter * 32 + r0;
+                wdq[half] = wrow & (bw - 1);
+                wdp[half] = (wrow >> p.bw_log2) & (bh - 1);
+                wdn[half] = wrow >> (p.bw_log2 + p.bh_log2);
+                woff[half] = uint32_t(((wdn[half] * P2 + (wdp[half] >> 1)) * Q2 + (wdq[half] >> 1)) * p.Kout + (lane & 7) * 4);
+            }
+            int my_items = 0;           // chunks of a tile that are this warp's
+            for (int h = 0; h < p.MT; ++h)
+                for (int ch = (sub - h * cpb) & (kSub - 1); ch < cpb; ch += kSub) ++my_items;
+            const bool relu = p.act == PCL_ACT_RELU;
+            const uint32_t t_quarter = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16);
+            const uint32_t t_second = p.MT * p.BN;      // split accumulators: the second issuer's copy of this box
+            for (it.init(p, first_tile, tile_stride); it.t < total_tiles; it.next(p), ++tile_cnt) {
+                const int acc = tile_cnt & 1;
+                const int ni = kPair ? 2 * it.ni + int(pair_rank) : it.ni;
+                const uint32_t acc_phase = (tile_cnt >> 1) & 1;
+                if (!bounded_wait_warp(&tmem_full_bar[acc], acc_phase, &abort_flag, p.status, WAIT_EPI_TMEM_FULL)) break;
+                tc_fence_after();
+                int left = my_items;
+                auto hand_back = [&]() {        // this warp has read all it needs of the accumulator set
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) {
+                        if (kPair && pair_rank != 0) mbar_arrive_cluster(map_to_cta(&tmem_empty_bar[acc], 0));
+                        else mbar_arrive(&tmem_empty_bar[acc]);
+                    }
+                };
+                if (left == 0) hand_back();
+                const int q_base = it.qi * p.tw, p_base = it.pi * p.th, n_base = ni * p.tn;
+                for (int h = 0; h < p.MT; ++h) {
+                    const int ch0 = (sub - h * cpb) & (kSub - 1);
+                    if (ch0 >= cpb) continue;
+                    const int qb = q_base + h * p.half_dq, pb = p_base + h * p.half_dp;
+                    const size_t tile_off = ((static_cast<size_t>(n_base) * P2 + (pb >> 1)) * Q2 + (qb >> 1)) * p.Kout + it.kt * p.BN;
+                    const bool w_ok[2] = {qb + wdq[0] < p.Q && pb + wdp[0] < p.P && n_base + wdn[0] < p.N,
+                                          qb + wdq[1] < p.Q && pb + wdp[1] < p.P && n_base + wdn[1] < p.N};
+                    const uint32_t t_row = t_quarter + ((p.split_acc ? 2 * acc : acc) * p.MT + h) * p.BN;
+                    for (int ch = ch0; ch < cpb; ch += kSub) {
+                        const int col = it.kt * p.BN + ch * 32 + (lane & 7) * 4;
+                        float4 b = make_float4(0.f, 0.f, 0.f, 0.f);
+                        if (p.bias_in_smem) b = *reinterpret_cast<const float4*>(bias_s + ch * 32 + (lane & 7) * 4);
+                        else if (p.bias && col < p.Kout) b = __ldg(reinterpret_cast<const float4*>(p.bias + col));
+                        if constexpr (kEpi == kEpiWarps) {
+                            uint32_t v[32];
+                            tmem_ld_32x32(t_row + ch * 32, v);
+                            tmem_ld_wait();
+                            if (p.split_acc) add_second_accumulator(t_row + t_second + ch * 32, v);
+                            if (--left == 0) hand_back();
+#pragma unroll
+                            for (int j = 0; j < 8; ++j)
+                                st_shared_v4(my_row + ((j * 16) ^ my_x), __uint_as_float(v[4 * j]), __uint_as_float(v[4 * j + 1]),
+                                             __uint_as_float(v[4 * j + 2]), __uint_as_float(v[4 * j + 3]));
+                        } else {
+                            uint32_t v[16], u[16];
+                            tmem_ld_32x16(t_row + ch * 32, v);
+                            tmem_ld_32x16(t_row + ch * 32 + 16, u);
+                            tmem_ld_wait();
+                            if (--left == 0) hand_back();
+#pragma unroll
+                            for (int jj = 0; jj < 4; ++jj)
+                                st_shared_v4(my_row + ((jj * 16) ^ my_x), __uint_as_float(v[4 * jj]), __uint_as_float(v[4 * jj + 1]),
+                                             __uint_as_float(v[4 * jj + 2]), __uint_as_float(v[4 * jj + 3]));
+#pragma unroll
+                            for (int jj = 0; jj < 4; ++jj)
+                                st_shared_v4(my_row + (((4 + jj) * 16) ^ my_x), __uint_as_float(u[4 * jj]), __uint_as_float(u[4 * jj + 1]),
+                                             __uint_as_float(u[4 * jj + 2]), __uint_as_float(u[4 * jj + 3]));
+                        }
+                        __syncwarp();
+#pragma unroll
+                        for (int half = 0; half < 2; ++half) {
+                            float4 s0 = ld_shared_v4(ld_a[half][0]), s1 = ld_shared_v4(ld_a[half][1]);
+                            float4 s2 = ld_shared_v4(ld_a[half][2]), s3 = ld_shared_v4(ld_a[half][3]);
+                            auto one = [&](float a0, float a1, float a2, float a3, float bb, float& mo) -> uint32_t {
+                                a0 += bb; a1 += bb; a2 += bb; a3 += bb;
+                                const float m = fmaxf(fmaxf(a0, a1), fmaxf(a2, a3));
+                                uint32_t pos = a0 == m ? 0u : (a1 == m ? 1u : (a2 == m ? 2u : 3u));
+                                const bool nonpos = !(m > 0.f);
+                                if (relu) { mo = fmaxf(m, 0.f); pos = nonpos ? 0u : pos; } else { mo = m; }
+                                return pos | (nonpos ? 4u : 0u);
+                            };
+                            float4 m;
+                            const uint32_t c0 = one(s0.x, s1.x, s2.x, s3.x, b.x, m.x), c1 = one(s0.y, s1.y, s2.y, s3.y, b.y, m.y);
+                            const uint32_t c2 = one(s0.z, s1.z, s2.z, s3.z, b.z, m.z), c3 = one(s0.w, s1.w, s2.w, s3.w, b.w, m.w);
+                            if (w_ok[half] && col < p.Kout) {
+                                const size_t po = tile_off + woff[half] + ch * 32;
+                                *reinterpret_cast<float4*>(p.pool_out + po) = m;
+                                if (p.pool_idx) *reinterpret_cast<uint32_t*>(p.pool_idx + po) = c0 | (c1 << 8) | (c2 << 16) | (c3 << 24);
+                            }
+                        }
+                        __syncwarp();       // the staging tile is free for the next chunk
+                    }
+                }
+            }
+        } else
         for (it.init(p, first_tile, tile_stride); it.t < total_tiles; it.next(p), ++tile_cnt) {
             const int acc = tile_cnt & 1;
             const int ni = kPair ? 2 * it.ni + int(pair_rank) : it.ni;
@@ -666,88 +811,6 @@ tc_fprop_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                 // consecutive pixels of the box, i.e. a sub-box whose first pixel is (sq, sp, sn).
                 const uint32_t stg = smem_u32(epi_stage + epi * 4096);
                 const int srow = quarter * 32;
-                if (kPool && !p.out && p.act != PCL_ACT_SIGMOID) {
-                    // Pooled output only (the step never reads the full-resolution output of a pooled layer).  The raw
-                    // accumulators are staged, each lane takes two windows of its four columns, adds the bias to the
-                    // four values s_e of a window, takes their maximum m and applies the activation to m alone: max
-                    // commutes with the (monotone) bias add and ReLU, so the stored maximum is bit for bit the maximum
-                    // of the finished values.  Position code: the first e with act(s_e) == act(m), i.e. with s_e == m,
-                    // except that under ReLU a window with m <= 0 holds four zeros, whose first maximum is e = 0.
-                    const int lb = p.bw_log2;
-                    const uint32_t my_row = stg + lane * 128, my_x = (lane & 7) * 16;
-                    uint32_t ld_a[2][4];
-                    size_t po_base[2];
-                    bool w_ok[2];
-#pragma unroll
-                    for (int half = 0; half < 2; ++half) {
-                        const int wdx = (lane >> 3) + 4 * half;
-                        const int r0 = ((wdx & ((1 << (lb - 1)) - 1)) << 1) | ((wdx >> (lb - 1)) << (lb + 1));
-#pragma unroll
-                        for (int e = 0; e < 4; ++e) {
-                            const int rr = r0 | (e & 1) | ((e >> 1) << lb);
-                            ld_a[half][e] = stg + rr * 128 + (((lane & 7) ^ (rr & 7)) * 16);
-                        }
-                        const int wrow = srow + r0;
-                        const int wq = it.qi * p.tw + (wrow & (bw - 1)) + h * p.half_dq;
-                        const int wp = it.pi * p.th + ((wrow >> p.bw_log2) & (bh - 1)) + h * p.half_dp;
-                        const int wn = ni * p.tn + (wrow >> (p.bw_log2 + p.bh_log2));
-                        w_ok[half] = wq < p.Q && wp < p.P && wn < p.N;
-                        po_base[half] = ((static_cast<size_t>(wn) * (p.P >> 1) + (wp >> 1)) * (p.Q >> 1) + (wq >> 1)) * p.Kout +
-                                        kt * p.BN + (lane & 7) * 4;
-                    }
-                    const bool relu = p.act == PCL_ACT_RELU;
-                    for (int ch = ch0; ch < cpb; ch += kSub) {
-                        const int col = kt * p.BN + ch * 32 + (lane & 7) * 4;
-                        float4 b = make_float4(0.f, 0.f, 0.f, 0.f);
-                        if (p.bias_in_smem) b = *reinterpret_cast<const float4*>(bias_s + ch * 32 + (lane & 7) * 4);
-                        else if (p.bias && col < p.Kout) b = __ldg(reinterpret_cast<const float4*>(p.bias + col));
-                        if constexpr (kEpi == kEpiWarps) {
-                            uint32_t v[32];
-                            tmem_ld_32x32(t_row + ch * 32, v);
-                            tmem_ld_wait();
-                            if (p.split_acc) add_second_accumulator(t_row + t_second + ch * 32, v);
-#pragma unroll
-                            for (int j = 0; j < 8; ++j)
-                                st_shared_v4(my_row + ((j * 16) ^ my_x), __uint_as_float(v[4 * j]), __uint_as_float(v[4 * j + 1]),
-                                             __uint_as_float(v[4 * j + 2]), __uint_as_float(v[4 * j + 3]));
-                        } else {
-#pragma unroll
-                            for (int hh = 0; hh < 2; ++hh) {
-                                uint32_t v[16];
-                                tmem_ld_32x16(t_row + ch * 32 + hh * 16, v);
-                                tmem_ld_wait();
-#pragma unroll
-                                for (int jj = 0; jj < 4; ++jj)
-                                    st_shared_v4(my_row + (((hh * 4 + jj) * 16) ^ my_x), __uint_as_float(v[4 * jj]),
-                                                 __uint_as_float(v[4 * jj + 1]), __uint_as_float(v[4 * jj + 2]),
-                                                 __uint_as_float(v[4 * jj + 3]));
-                            }
-                        }
-                        __syncwarp();
-#pragma unroll
-                        for (int half = 0; half < 2; ++half) {
-                            float4 s0 = ld_shared_v4(ld_a[half][0]), s1 = ld_shared_v4(ld_a[half][1]);
-                            float4 s2 = ld_shared_v4(ld_a[half][2]), s3 = ld_shared_v4(ld_a[half][3]);
-                            auto one = [&](float a0, float a1, float a2, float a3, float bb, float& mo) -> uint32_t {
-                                a0 += bb; a1 += bb; a2 += bb; a3 += bb;
-                                const float m = fmaxf(fmaxf(a0, a1), fmaxf(a2, a3));
-                                uint32_t pos = a0 == m ? 0u : (a1 == m ? 1u : (a2 == m ? 2u : 3u));
-                                const bool nonpos = !(m > 0.f);
-                                if (relu) { mo = fmaxf(m, 0.f); pos = nonpos ? 0u : pos; } else { mo = m; }
-                                return pos | (nonpos ? 4u : 0u);
-                            };
-                            float4 m;
-                            const uint32_t c0 = one(s0.x, s1.x, s2.x, s3.x, b.x, m.x), c1 = one(s0.y, s1.y, s2.y, s3.y, b.y, m.y);
-                            const uint32_t c2 = one(s0.z, s1.z, s2.z, s3.z, b.z, m.z), c3 = one(s0.w, s1.w, s2.w, s3.w, b.w, m.w);
-                            if (w_ok[half] && col < p.Kout) {
-                                const size_t po = po_base[half] + ch * 32;
-                                *reinterpret_cast<float4*>(p.pool_out + po) = m;
-                                if (p.pool_idx) *reinterpret_cast<uint32_t*>(p.pool_idx + po) = c0 | (c1 << 8) | (c2 << 16) | (c3 << 24);
-                            }
-                        }
-                        __syncwarp();       // the staging tile is free for the next chunk
-                    }
-                } else
                 for (int ch = ch0; ch < cpb; ch += kSub) {
                     const int col0 = kt * p.BN + ch * 32;
                     // (the 8-warp variant fetches the chunk's bias ahead of the accumulator, eight vectors per lane;
@@ -1394,6 +1457,7 @@ int launch_tc_fprop(const TcFpropArgs& a, cudaStream_t st) {
         p.resident_b = (cfg.halo && !cfg.pair && p.issuers == 1 && p.tiles_k == 1 && !p.bmn && slots <= 3 && slots <= cfg.stages &&      // (a launch keeps at least three slots)
                         tune(TUNE_RESIDENT_B, 1)) ? 1 : 0;
         p.kslices = (a.k_live > 0 && a.k_live < 32 && tune(TUNE_KSLICES, 1)) ? (a.k_live + 7) / 8 : 4;
+        p.tile_duo = (p.resident_b && p.cblocks == 1 && p.NA % 2 == 0 && tune(TUNE_ISSUERS, 2) >= 2) ? 1 : 0;
     }
     p.colsum_rows = (a.Kout % 4 == 0) ? a.colsum_rows : nullptr;
     if (a.colsum_rows && !p.colsum_rows) return PCL_ERR_UNSUPPORTED_SHAPE;
