@@ -781,8 +781,8 @@ PooledWgradPlan plan_pooled_wgrad(const pcl_conv_desc& d, int P, int Q) {
     pl.splits = tc_wgrad_splits(d.N, P, Q, d.S * 4, d.K, d.R, 1, 1, 1);
     pl.tiles_off = staged_x_bytes(d);
     pl.rows_off = pl.tiles_off + size_t(pl.splits) * staged_w_bytes(d);
-    pl.cs_off = pl.rows_off + align_up(size_t(pl.splits) * 8 * d.K * 4, 256);      // one row per (split, epilogue warp)
-    const int cs = colsum_splits(size_t(pl.splits) * 8);
+    pl.cs_off = pl.rows_off + align_up(size_t(pl.splits) * kPooledDbRows * d.K * 4, 256);      // one row per (split, builder warp)
+    const int cs = colsum_splits(size_t(pl.splits) * kPooledDbRows);
     pl.total = pl.cs_off + (cs > 1 ? align_up(size_t(cs) * d.K * 4, 256) : 0);
     return pl;
 }
@@ -844,7 +844,7 @@ static int conv_bwd_weights_pooled_impl(const pcl_conv_desc* d, const float* x, 
     if (rc != PCL_OK) return rc;
     rc = launch_unpad_reduce(dw4, dw, size_t(d->K) * d->R, d->S, d->C, d->S * 4, pl.splits, taps * 4, st);
     if (rc != PCL_OK) return rc;
-    if (dbias) rc = launch_colsum(rows, size_t(pl.splits) * 8, d->K, cs, dbias, st);       // adds the rows, fixed order
+    if (dbias) rc = launch_colsum(rows, size_t(pl.splits) * kPooledDbRows, d->K, cs, dbias, st);       // adds the rows, fixed order
     return rc;
 }
 

@@ -189,7 +189,7 @@ struct TcWgradArgs {
     int skip_reduce = 0;
     // Pooled dy: `dy` is null and the kernel builds its dy tiles from dy_pool [N][P/2][Q/2][K] and the pooling
     // windows' position codes (same shape, bytes): the coded position of each window gets the gradient, the other
-    // three zero; relu_mask: windows whose code has bit 2 set get nothing.  db_rows (optional, [splits * 8][K]) gets
+    // three zero; relu_mask: windows whose code has bit 2 set get nothing.  db_rows (optional, [splits * kPooledDbRows][K]) gets
     // per-(split, epilogue warp) sums of the scattered gradient, i.e. the bias gradient before the rows are added.
     // Needs even P and Q, K % 4 == 0, single-CTA items (tc_wgrad_can_take_pooled_dy()).
     const float* dy_pool = nullptr;
@@ -199,6 +199,7 @@ struct TcWgradArgs {
     int stride_h = 1, stride_w = 1, dil_w = 1;      // as in TcFpropArgs
 };
 bool tc_wgrad_eligible(const TcWgradArgs& a);
+constexpr int kPooledDbRows = 16;       // bias-gradient rows per pixel split that a pooled-dy launch writes
 bool tc_wgrad_can_take_pooled_dy(int N, int P, int Q, int C, int K, int R, int S, int tap_groups);
 int tc_wgrad_splits(int N, int P, int Q, int C, int K, int R, int S, int tap_groups = 0, int pooled_dy = 0,
                     int strided = 0);

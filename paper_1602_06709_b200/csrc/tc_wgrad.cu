@@ -56,7 +56,9 @@ namespace pcl {
 namespace {
 
 constexpr int kMaxStages = 8;
-constexpr int kWgradThreads = 320;     // warp 0 producer, warp 1 MMA issuer, warps 2-9 epilogue (two per TMEM lane quarter)
+constexpr int kWgradThreads = 352;     // warp 0 producer, warps 1 and 10 MMA issuers, warps 2-9 epilogue (two per TMEM lane quarter)
+constexpr int kSecondIssuerWarp = 10;
+constexpr int kWgradThreadsWide = 608; // pooled-dy launches with two issuers: warps 11-18 are a second group of dy builders
 constexpr int kSmemBudget = 224 * 1024;
 constexpr int kExpanderWarps = 8;      // the epilogue warps, which build the dy tiles of pooled-dy launches during the main loop
 
@@ -93,6 +95,12 @@ struct WgradParams {
     int N, P, Q;              // output size (for the pooled tile's bounds)
     float* out;               // dw, or the partial-sum workspace [splits][K*R*S*C]
     size_t split_stride;      // K*R*S*C (0 when writing straight to dw)
+    // duo: two issuing threads take the pipeline slots alternately (the number of slots is even, so a slot always
+    // belongs to the same thread), each into an accumulator of its own, acc_cols columns apart; the epilogue adds
+    // the two in a fixed order.  What bounds a single-CTA item is the issuing thread (~100-140 cycles per MMA,
+    // whatever its width), not the tensor pipe.
+    int duo, acc_cols;
+    int dy_groups;            // 32-map groups of a k-step's dy tile (4, fewer for pooled dy with K < 128)
     int inject_short_copy;    // test mode: the first slot is armed for 16 bytes more than are copied (see the forward kernel)
     unsigned int* status;     // device status word (status[1]: limit of the bounded waits in microseconds)
 };
@@ -112,8 +120,11 @@ __device__ __forceinline__ void xhalo_row(uint32_t d_tmem, uint32_t xn, uint32_t
 
 // kPair: see the header.  Pair mode needs grouped x and dy maps; every item then has rpi runs (runs past the
 // last tap read zeros through the out-of-bounds fill and are not stored).
-template <bool kPair>
-__global__ void __launch_bounds__(kWgradThreads, 1)
+// kWide (pooled dy with two issuers): sixteen warps build the dy tiles, in two groups that take the pipeline slots
+// alternately like the issuing threads do -- a builder warp is a chain of dependent instructions per k-step, and two
+// warps per scheduler cannot hide it.
+template <bool kPair, bool kWide = false>
+__global__ void __launch_bounds__(kWide ? kWgradThreadsWide : kWgradThreads, 1)
 tc_wgrad_kernel(const __grid_constant__ CUtensorMap tmDy, const __grid_constant__ CUtensorMap tmX, WgradParams p) {
     extern __shared__ uint8_t smem_raw[];
     __shared__ uint64_t full_bar[kMaxStages];
@@ -138,7 +149,10 @@ tc_wgrad_kernel(const __grid_constant__ CUtensorMap tmDy, const __grid_constant_
     const int my_runs = kPair ? nruns >> 1 : nruns;   // runs this CTA loads (pair: its half of the columns)
     const int my_run0 = run0 + int(pair_rank) * my_runs;
     const uint32_t group_bytes = p.pix * 128;         // one {32 maps x pix pixels} box
-    const uint32_t a_bytes = 4 * group_bytes;         // 128 output maps
+    // 128 output maps; pooled-dy launches of layers with K < 128 build only the groups that exist, and the MMAs' rows
+    // beyond them read the x tile behind (finite numbers into accumulator rows that are never stored; the slot
+    // holds at least four groups, so the operand stays inside it)
+    const uint32_t a_bytes = p.dy_groups * group_bytes;
     const uint32_t step_bytes = p.xhalo ? uint32_t(p.x_step_bytes)
                                         : a_bytes + (kPair ? (p.rpi >> 1) : p.rpi) * p.L * group_bytes;   // one k-step (same for every item)
     const uint32_t stage_bytes = p.KS * step_bytes;                     // a slot holds KS k-steps
@@ -149,7 +163,7 @@ tc_wgrad_kernel(const __grid_constant__ CUtensorMap tmDy, const __grid_constant_
             mbar_init(&full_bar[s], p.dy_pool ? 1 + kExpanderWarps : 1);     // + one arrival per warp that builds dy
             mbar_init(&empty_bar[s], 1);
         }
-        mbar_init(&tmem_full_bar, 1);
+        mbar_init(&tmem_full_bar, p.duo ? 2 : 1);
         abort_flag = 0;
         mbar_fence_init();
         prefetch_tmap(&tmDy);
@@ -271,16 +285,19 @@ tc_wgrad_kernel(const __grid_constant__ CUtensorMap tmDy, const __grid_constant_
                 }
             }
         }
-    } else if (warp == 1) {
-        if (lane == 0 && pair_rank == 0) {     // one thread runs the whole issue loop, waits included
+    } else if (warp == 1 || warp == kSecondIssuerWarp) {
+        const uint32_t issuer = warp == 1 ? 0u : 1u;
+        const uint32_t nis = p.duo ? 2u : 1u;
+        if (lane == 0 && pair_rank == 0 && issuer < nis) {     // one thread runs a whole issue loop, waits included
+        const uint32_t d_tmem = tmem_base + issuer * uint32_t(p.acc_cols);
         const uint32_t idesc = make_idesc_tf32(n_groups * 32, true, true, kPair ? 256u : 128u);
         // 8 pixels per MMA = two 512-byte groups of 4 rows (1 KB, 64 sixteen-byte units, per MMA); descriptors differ
         // only in the address field of their low word
         const uint64_t desc0 = make_smem_desc(smem_u32(smem), group_bytes, 512, kSwizzle128B_Atom32B);
         const uint32_t hi = uint32_t(desc0 >> 32), ring_lo0 = uint32_t(desc0);
         const uint32_t full0 = smem_u32(&full_bar[0]), empty0 = smem_u32(&empty_bar[0]);
-        uint32_t full_a = full0, empty_a = empty0, slot_lo = ring_lo0;
         const uint32_t stage16 = stage_bytes >> 4, step16 = step_bytes >> 4, a16 = a_bytes >> 4;
+        uint32_t full_a = full0 + 8u * issuer, empty_a = empty0 + 8u * issuer, slot_lo = ring_lo0 + issuer * stage16;
         const bool wide = p.pix == 64;
         // xhalo: N = 32*S per MMA, B's leading-dimension offset one 128-byte row (8 sixteen-byte units, bits 16-29 of
         // the low word) = one tap; a box row of bw pixels is bw/8 MMA steps per map group, the next box row starts
@@ -290,32 +307,38 @@ tc_wgrad_kernel(const __grid_constant__ CUtensorMap tmDy, const __grid_constant_
         const uint32_t xlbo = (8u << 16) - (ring_lo0 & 0x3FFF0000u);      // replaces dy's offset field by 8
         const int xrows = p.pix >> p.bw_log2, xsteps = bw >> 3;
         const uint32_t xrow16 = uint32_t(bw + p.S - 1) * 8u;
-        int stage = 0;
+        int stage = int(issuer);
         uint32_t phase = 0, accum = 0;
         bool ok = true;
+        auto next_slot = [&]() {        // this thread's next slot: nis slots further round the ring
+            stage += int(nis); full_a += 8u * nis; empty_a += 8u * nis; slot_lo += nis * stage16;
+            if (stage >= p.stages) {
+                stage -= p.stages; phase ^= 1u;
+                full_a = full0 + 8u * stage; empty_a = empty0 + 8u * stage; slot_lo = ring_lo0 + uint32_t(stage) * stage16;
+            }
+        };
         // haloed x: one k-step per slot (KS = 1); the whole k-step is straight-line for the common box shapes
         auto xhalo_loop = [&](auto rows_c, auto steps_c, auto cg_c) {
             constexpr int kRows = decltype(rows_c)::value, kSteps = decltype(steps_c)::value, kCg = decltype(cg_c)::value;
             const int rows = kRows ? kRows : xrows, steps = kSteps ? kSteps : xsteps, cgs = kCg ? kCg : p.cg;
-            for (int kit = 0; kit < kiters; ++kit) {
+            for (int kit = int(issuer); kit < kiters; kit += int(nis)) {
                 if (!bounded_wait_addr(full_a, phase, &abort_flag, p.status, WAIT_MMA_FULL)) { ok = false; break; }
                 tc_fence_after();
                 uint32_t ar = slot_lo, br = slot_lo + a16 + xlbo;
                 if constexpr (kRows != 0) {
 #pragma unroll
                     for (int r = 0; r < kRows; ++r, ar += 64u * kSteps, br += xrow16)
-                        xhalo_row<kSteps, kCg>(tmem_base, xn, ar, br, hi, idesc_x, r == 0 ? accum : 1u, xg16);
+                        xhalo_row<kSteps, kCg>(d_tmem, xn, ar, br, hi, idesc_x, r == 0 ? accum : 1u, xg16);
                 } else {
                     for (int r = 0; r < rows; ++r, ar += 64u * steps, br += xrow16)
                         for (int m = 0; m < steps; ++m)
                             for (int g = 0; g < cgs; ++g)
-                                umma_tf32(tmem_base + g * xn, (uint64_t(hi) << 32) | (ar + 64u * m),
+                                umma_tf32(d_tmem + g * xn, (uint64_t(hi) << 32) | (ar + 64u * m),
                                           (uint64_t(hi) << 32) | (br + 64u * m + g * xg16), idesc_x, (accum | r | m) ? 1u : 0u);
                 }
                 accum = 1;
                 umma_commit_addr<kPair>(empty_a);
-                full_a += 8; empty_a += 8; slot_lo += stage16;
-                if (++stage == p.stages) { stage = 0; phase ^= 1u; full_a = full0; empty_a = empty0; slot_lo = ring_lo0; }
+                next_slot();
             }
         };
         using std::integral_constant;
@@ -328,19 +351,18 @@ tc_wgrad_kernel(const __grid_constant__ CUtensorMap tmDy, const __grid_constant_
             else if (key == 222) xhalo_loop(integral_constant<int, 2>{}, integral_constant<int, 2>{}, integral_constant<int, 2>{});
             else xhalo_loop(integral_constant<int, 0>{}, integral_constant<int, 0>{}, integral_constant<int, 0>{});
         } else
-        for (int kit = 0; kit < kiters; kit += p.KS) {
+        for (int kit = int(issuer) * p.KS; kit < kiters; kit += int(nis) * p.KS) {
             if (!bounded_wait_addr(full_a, phase, &abort_flag, p.status, WAIT_MMA_FULL)) { ok = false; break; }
             tc_fence_after();
             const int nst = kiters - kit < p.KS ? kiters - kit : p.KS;
             uint32_t a_lo = slot_lo;
             for (int j = 0; j < nst; ++j, a_lo += step16) {
-                umma_kstep_tf32<kPair, 64, 64>(tmem_base, a_lo, a_lo + a16, hi, hi, idesc, accum);
+                umma_kstep_tf32<kPair, 64, 64>(d_tmem, a_lo, a_lo + a16, hi, hi, idesc, accum);
                 accum = 1;
-                if (wide) umma_kstep_tf32<kPair, 64, 64>(tmem_base, a_lo + 256, a_lo + a16 + 256, hi, hi, idesc, 1);
+                if (wide) umma_kstep_tf32<kPair, 64, 64>(d_tmem, a_lo + 256, a_lo + a16 + 256, hi, hi, idesc, 1);
             }
             umma_commit_addr<kPair>(empty_a);
-            full_a += 8; empty_a += 8; slot_lo += stage16;
-            if (++stage == p.stages) { stage = 0; phase ^= 1u; full_a = full0; empty_a = empty0; slot_lo = ring_lo0; }
+            next_slot();
         }
         if (ok) umma_commit_addr<kPair>(smem_u32(&tmem_full_bar));
         }
@@ -351,7 +373,10 @@ tc_wgrad_kernel(const __grid_constant__ CUtensorMap tmDy, const __grid_constant_
         const bool valid = k < p.K;
         const bool vec_ok = (p.C & 3) == 0;
         float4 db_acc[2] = {make_float4(0.f, 0.f, 0.f, 0.f), make_float4(0.f, 0.f, 0.f, 0.f)};
-        const int t = int(threadIdx.x) - 64;                 // 0 .. 255 among the epilogue warps
+        const int bgroup = (kWide && warp > kSecondIssuerWarp) ? 1 : 0;       // builder group (the second has no epilogue)
+        const int bwarp = bgroup ? warp - (kSecondIssuerWarp + 1) : warp - 2;  // 0 .. 7 inside the group
+        constexpr int kGroups = kWide ? 2 : 1;
+        const int t = bwarp * 32 + lane;                     // 0 .. 255 among the group's warps
         int maps_here = p.K - kt * 128;                      // output maps of this k tile
         if (maps_here > 128) maps_here = 128;
         const int units = maps_here >> 2;                    // 4-map units of the tile (K % 4 == 0)
@@ -362,11 +387,14 @@ tc_wgrad_kernel(const __grid_constant__ CUtensorMap tmDy, const __grid_constant_
             const int items = ppix * units;                   // (pooled pixel, 4-map unit) items per k-step: <= 512
             const int P2 = p.P >> 1, Q2 = p.Q >> 1;
             const uint32_t ring0 = smem_u32(smem);
-            int stage = 0, sub = 0;
+            int stage = bgroup, sub = 0;
             uint32_t phase = 0, dstA = ring0;
-            int qi = box_begin % p.boxes_q;
-            int pi = (box_begin / p.boxes_q) % p.boxes_p;
-            int ni = box_begin / (p.boxes_q * p.boxes_p);
+            // the group's k-steps: slots bgroup, bgroup + kGroups, ... of KS boxes each; (qi, pi, ni) walks two k-steps
+            // ahead of the k-step being written (the fetch cursor)
+            int fb = box_begin + bgroup * p.KS, fsub = 0;
+            int qi = fb % p.boxes_q;
+            int pi = (fb / p.boxes_q) % p.boxes_p;
+            int ni = fb / (p.boxes_q * p.boxes_p);
             bool ok = true;
             // this thread's (at most two) items: pooled pixel j of the box and 4-map unit u, the same in every k-step
             int item_w[2], item_h[2], item_n[2];
@@ -408,18 +436,22 @@ tc_wgrad_kernel(const __grid_constant__ CUtensorMap tmDy, const __grid_constant_
             };
             float4 v[2], vn[2], vnn[2];
             uint32_t c[2], cn[2], cnn[2];
-            auto next_box = [&]() {             // the producer's walk over the pixel boxes
-                if (++qi == p.boxes_q) {
-                    qi = 0;
-                    if (++pi == p.boxes_p) { pi = 0; ++ni; }
-                }
+            auto next_box = [&]() {             // the fetch cursor's next k-step of this group
+                int step = 1;
+                if (++fsub == p.KS) { fsub = 0; step += (kGroups - 1) * p.KS; }
+                fb += step;
+                for (int i = 0; i < step; ++i)
+                    if (++qi == p.boxes_q) {
+                        qi = 0;
+                        if (++pi == p.boxes_p) { pi = 0; ++ni; }
+                    }
             };
-            if (box_begin < box_end) { fetch(qi, pi, ni, vn, cn); next_box(); }
-            if (box_begin + 1 < box_end) { fetch(qi, pi, ni, vnn, cnn); next_box(); }
-            for (int b = box_begin; b < box_end && ok; ++b) {
+            if (fb < box_end) { fetch(qi, pi, ni, vn, cn); next_box(); }
+            if (fb < box_end) { fetch(qi, pi, ni, vnn, cnn); next_box(); }
+            for (int b = box_begin + bgroup * p.KS; b < box_end && ok;) {
 #pragma unroll
                 for (int i = 0; i < 2; ++i) { v[i] = vn[i]; c[i] = cn[i]; vn[i] = vnn[i]; cn[i] = cnn[i]; }
-                if (b + 2 < box_end) { fetch(qi, pi, ni, vnn, cnn); next_box(); }
+                if (fb < box_end) { fetch(qi, pi, ni, vnn, cnn); next_box(); }
                 if (sub == 0) {
                     if (!bounded_wait_warp(&empty_bar[stage], phase ^ 1u, &abort_flag, p.status, WAIT_PRODUCER_EMPTY)) { ok = false; break; }
                     dstA = ring0 + stage * stage_bytes;
@@ -450,7 +482,11 @@ tc_wgrad_kernel(const __grid_constant__ CUtensorMap tmDy, const __grid_constant_
                     fence_proxy_async_shared();          // the tensor core reads the tile through the async proxy
                     __syncwarp();
                     if (lane == 0) mbar_arrive(&full_bar[stage]);
-                    if (++stage == p.stages) { stage = 0; phase ^= 1u; }
+                    stage += kGroups;
+                    if (stage >= p.stages) { stage -= p.stages; phase ^= 1u; }
+                    b += 1 + (kGroups - 1) * p.KS;       // over the other group's slot
+                } else {
+                    ++b;
                 }
             }
         }
@@ -461,24 +497,26 @@ tc_wgrad_kernel(const __grid_constant__ CUtensorMap tmDy, const __grid_constant_
                 // scattered, and writes one row [K] per (split, warp); the caller adds the rows.  (Warp-local on
                 // purpose: no barrier between warps that a timed-out warp could leave the others waiting at.  The
                 // pipeline's shared memory is idle by now; the 1 KB slots lie behind the epilogue's staging tiles.)
-                float4* scratch = reinterpret_cast<float4*>(smem + 32768) + (warp - 2) * 64;
+                float4* scratch = reinterpret_cast<float4*>(smem + 32768) + (bgroup * 8 + bwarp) * 64;
                 scratch[lane] = db_acc[0];
                 scratch[32 + lane] = db_acc[1];
                 __syncwarp();
                 if (lane < units) {
                     float4 sum = make_float4(0.f, 0.f, 0.f, 0.f);
                     for (int e = 0; e < 64; ++e) {
-                        const int item = (e < 32 ? 0 : 256 - 32) + (warp - 2) * 32 + e;      // lane e (e - 32) of this warp, slot 0 (1)
+                        const int item = (e < 32 ? 0 : 256 - 32) + bwarp * 32 + e;      // lane e (e - 32) of this warp, slot 0 (1)
                         if (item % units == lane) {
                             const float4 a = scratch[e];
                             sum.x += a.x; sum.y += a.y; sum.z += a.z; sum.w += a.w;
                         }
                     }
-                    *reinterpret_cast<float4*>(p.db_rows + (static_cast<size_t>(split) * kExpanderWarps + (warp - 2)) * p.K +
-                                               kt * 128 + lane * 4) = sum;
+                    float* row = p.db_rows + (static_cast<size_t>(split) * kPooledDbRows + bgroup * 8 + bwarp) * p.K + kt * 128 + lane * 4;
+                    *reinterpret_cast<float4*>(row) = sum;
+                    if (!kWide) *reinterpret_cast<float4*>(row + 8 * static_cast<size_t>(p.K)) = make_float4(0.f, 0.f, 0.f, 0.f);
                 }
                 __syncwarp();
             }
+            if (bgroup == 0) {
             const uint32_t t_row = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16);
             const size_t krow = static_cast<size_t>(valid ? k : 0) * p.R * p.S;
             // Each lane owns one output-map row of the accumulator, but 32 columns of a row are 128 contiguous
@@ -502,6 +540,13 @@ tc_wgrad_kernel(const __grid_constant__ CUtensorMap tmDy, const __grid_constant_
                 if (kiters > 0) {
                     tmem_ld_32x32(t_row + ch * 32, v);
                     tmem_ld_wait();
+                    if (p.duo && kiters > p.KS) {      // the second issuer had at least one slot
+                        uint32_t u[32];
+                        tmem_ld_32x32(t_row + p.acc_cols + ch * 32, u);
+                        tmem_ld_wait();
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) v[j] = __float_as_uint(__uint_as_float(v[j]) + __uint_as_float(u[j]));
+                    }
                 } else {
 #pragma unroll
                     for (int j = 0; j < 32; ++j) v[j] = 0u;
@@ -542,6 +587,7 @@ tc_wgrad_kernel(const __grid_constant__ CUtensorMap tmDy, const __grid_constant_
                             if (c0 + j < p.C) dst[j] = __uint_as_float(v[j]);
                     }
                 }
+            }
             }
         }
     }
@@ -586,6 +632,7 @@ struct WgradPlan {
     int bw_log2, bh_log2;
     long boxes;
     int xhalo, x_group_bytes;     // haloed x boxes (see the header): item = (k tile, kernel row, split)
+    int dy_groups;                // 32-map groups of the dy tile
 };
 
 WgradPlan plan_wgrad(int N, int P, int Q, int C, int K, int R, int S, int tap_groups, int pooled_dy = 0,
@@ -621,7 +668,7 @@ WgradPlan plan_wgrad(int N, int P, int Q, int C, int K, int R, int S, int tap_gr
             const int xg = int((bw + S - 1) * bh * bn * 128);
             const int step = (4 * pix * 128 + cgroups * xg + 1023) / 1024 * 1024;
             if (kSmemBudget / step < 3) continue;
-            r.xhalo = 1; r.x_group_bytes = xg; r.pix = pix; r.step_bytes = step;
+            r.xhalo = 1; r.x_group_bytes = xg; r.pix = pix; r.step_bytes = step; r.dy_groups = 4;
             r.bw_log2 = lw; r.bh_log2 = lh;
             r.run_blocks = R;
             r.KS = 1;
@@ -632,7 +679,10 @@ WgradPlan plan_wgrad(int N, int P, int Q, int C, int K, int R, int S, int tap_gr
         if (r.xhalo) return r;
     }
     // 64-pixel k-steps halve the copies and commits per MMA; taken when three pipeline slots still fit
-    const int cta_groups = 4 + (r.pair ? r.rpi / 2 : r.rpi) * r.L;      // 32-map groups a CTA loads per k-step
+    const int x_groups = (r.pair ? r.rpi / 2 : r.rpi) * r.L;
+    r.dy_groups = 4;
+    if (pooled_dy && K < 128 && (K + 31) / 32 + x_groups >= 4) r.dy_groups = (K + 31) / 32;
+    const int cta_groups = r.dy_groups + x_groups;      // 32-map groups a CTA loads per k-step
     r.pix = tune(TUNE_PIX_WGRAD, 64);
     if (r.pix != 64 || kSmemBudget / (cta_groups * 64 * 128) < 3) r.pix = 32;
     r.step_bytes = cta_groups * r.pix * 128;
@@ -668,8 +718,8 @@ bool tc_wgrad_eligible(const TcWgradArgs& a) {
 bool tc_wgrad_can_take_pooled_dy(int N, int P, int Q, int C, int K, int R, int S, int tap_groups) {
     if (P % 2 != 0 || Q % 2 != 0 || K % 4 != 0 || N <= 0) return false;
     const WgradPlan rp = plan_wgrad(N, P, Q, C, K, R, S, tap_groups, 1);
-    // the bias-gradient scratch (8 KB behind the epilogue's 32 KB of staging tiles) lies in the pipeline's memory
-    return !rp.pair && rp.stages * rp.KS * rp.step_bytes >= 40960;
+    // the bias-gradient scratch (16 KB behind the epilogue's 32 KB of staging tiles) lies in the pipeline's memory
+    return !rp.pair && (rp.stages & ~1) * rp.KS * rp.step_bytes >= 49152;
 }
 
 int tc_wgrad_splits(int N, int P, int Q, int C, int K, int R, int S, int tap_groups, int pooled_dy, int strided) {
@@ -694,6 +744,8 @@ int launch_tc_wgrad(const TcWgradArgs& a, cudaStream_t st) {
         if (cudaFuncSetAttribute(tc_wgrad_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  kSmemBudget + 1024) != cudaSuccess ||
             cudaFuncSetAttribute(tc_wgrad_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 kSmemBudget + 1024) != cudaSuccess ||
+            cudaFuncSetAttribute(tc_wgrad_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  kSmemBudget + 1024) != cudaSuccess)
             return PCL_ERR_CUDA;
         return PCL_OK;
@@ -726,8 +778,12 @@ int launch_tc_wgrad(const TcWgradArgs& a, cudaStream_t st) {
     const int max_groups = p.xhalo ? p.cg * a.S : p.rpi * p.L;
     p.KS = rp.KS; p.stages = rp.stages;
     const int stage_bytes = p.KS * rp.step_bytes;
+    p.dy_groups = rp.dy_groups;
+    p.acc_cols = max_groups * 32;
+    p.duo = (!rp.pair && p.stages >= 4 && 2 * p.acc_cols <= 512 && tune(TUNE_ISSUERS, 2) >= 2) ? 1 : 0;
+    if (p.duo) p.stages &= ~1;      // an even ring: every slot stays with one issuing thread
     p.tmem_cols = 32;
-    while (p.tmem_cols < max_groups * 32) p.tmem_cols *= 2;
+    while (p.tmem_cols < (p.duo ? 2 : 1) * p.acc_cols) p.tmem_cols *= 2;
     p.status = device_status_ptr();
     if (!p.status) return PCL_ERR_CUDA;
     p.inject_short_copy = (tune(TUNE_FAULT_INJECT, 0) == 2 && !rp.pair && !pooled) ? 1 : 0;      // test mode
@@ -814,6 +870,8 @@ int launch_tc_wgrad(const TcWgradArgs& a, cudaStream_t st) {
             lc.gridDim = dim3(unsigned(items)); lc.blockDim = dim3(kWgradThreads); lc.dynamicSmemBytes = smem; lc.stream = st;
             lc.attrs = attr; lc.numAttrs = 1;
             if (cudaLaunchKernelEx(&lc, tc_wgrad_kernel<true>, tmDy, tmX, p) != cudaSuccess) return PCL_ERR_CUDA;
+        } else if (pooled && p.duo) {
+            tc_wgrad_kernel<false, true><<<int(items), kWgradThreadsWide, smem, st>>>(tmDy, tmX, p);
         } else {
             tc_wgrad_kernel<false><<<int(items), kWgradThreads, smem, st>>>(tmDy, tmX, p);
         }
