@@ -572,8 +572,8 @@ __global__ void __launch_bounds__(256) reduce_splits_bias_act_kernel(const float
         if (act == PCL_ACT_RELU) {
             acc.x = fmaxf(acc.x, 0.f); acc.y = fmaxf(acc.y, 0.f); acc.z = fmaxf(acc.z, 0.f); acc.w = fmaxf(acc.w, 0.f);
         } else if (act == PCL_ACT_SIGMOID) {
-            acc.x = 1.f / (1.f + __expf(-acc.x)); acc.y = 1.f / (1.f + __expf(-acc.y));
-            acc.z = 1.f / (1.f + __expf(-acc.z)); acc.w = 1.f / (1.f + __expf(-acc.w));
+            acc.x = sigmoid_fast(acc.x); acc.y = sigmoid_fast(acc.y);
+            acc.z = sigmoid_fast(acc.z); acc.w = sigmoid_fast(acc.w);
         }
         out[i] = acc;
     }

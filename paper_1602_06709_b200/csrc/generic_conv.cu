@@ -41,7 +41,7 @@ struct FwdProblem {
     __device__ void store(long m, long col, float v, int) const {
         if (bias) v += __ldg(bias + col);
         if (act == PCL_ACT_RELU) v = fmaxf(v, 0.f);
-        else if (act == PCL_ACT_SIGMOID) v = 1.f / (1.f + __expf(-v));
+        else if (act == PCL_ACT_SIGMOID) v = sigmoid_fast(v);
         y[m * g.K + col] = v;
     }
 };

@@ -12,6 +12,12 @@
 
 namespace pcl {
 
+#ifdef __CUDACC__
+// Logistic function from the two approximate special-function instructions (ex2 and rcp, each within 2 ulp): an
+// IEEE division per element costs a one-tile GEMM's epilogue several microseconds.
+__device__ __forceinline__ float sigmoid_fast(float x) { return __fdividef(1.f, 1.f + __expf(-x)); }
+#endif
+
 // Kernel families, for launch counting and the optional per-kernel timing.
 enum KernelId {
     KID_TC_FPROP = 0, KID_TC_WGRAD, KID_GENERIC_FWD, KID_GENERIC_DGRAD, KID_GENERIC_WGRAD, KID_SGD, KID_REDUCE_SPLITS,

@@ -185,8 +185,8 @@ __device__ __forceinline__ float4 finish4(float4 o, const float4 b, const int ac
     if (act == PCL_ACT_RELU) {
         o.x = fmaxf(o.x, 0.f); o.y = fmaxf(o.y, 0.f); o.z = fmaxf(o.z, 0.f); o.w = fmaxf(o.w, 0.f);
     } else if (act == PCL_ACT_SIGMOID) {
-        o.x = 1.f / (1.f + __expf(-o.x)); o.y = 1.f / (1.f + __expf(-o.y));
-        o.z = 1.f / (1.f + __expf(-o.z)); o.w = 1.f / (1.f + __expf(-o.w));
+        o.x = sigmoid_fast(o.x); o.y = sigmoid_fast(o.y);
+        o.z = sigmoid_fast(o.z); o.w = sigmoid_fast(o.w);
     }
     return o;
 }
@@ -836,8 +836,8 @@ tc_fprop_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                         if (p.act == PCL_ACT_RELU) {
                             o.x = fmaxf(o.x, 0.f); o.y = fmaxf(o.y, 0.f); o.z = fmaxf(o.z, 0.f); o.w = fmaxf(o.w, 0.f);
                         } else if (p.act == PCL_ACT_SIGMOID) {
-                            o.x = 1.f / (1.f + __expf(-o.x)); o.y = 1.f / (1.f + __expf(-o.y));
-                            o.z = 1.f / (1.f + __expf(-o.z)); o.w = 1.f / (1.f + __expf(-o.w));
+                            o.x = sigmoid_fast(o.x); o.y = sigmoid_fast(o.y);
+                            o.z = sigmoid_fast(o.z); o.w = sigmoid_fast(o.w);
                         }
                         st_shared_v4(stg + lane * 128 + ((j ^ (lane & 7)) * 16), o.x, o.y, o.z, o.w);
                     };
@@ -966,8 +966,8 @@ tc_fprop_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                                     o.x = fmaxf(o.x, 0.f); o.y = fmaxf(o.y, 0.f);
                                     o.z = fmaxf(o.z, 0.f); o.w = fmaxf(o.w, 0.f);
                                 } else if (p.act == PCL_ACT_SIGMOID) {
-                                    o.x = 1.f / (1.f + __expf(-o.x)); o.y = 1.f / (1.f + __expf(-o.y));
-                                    o.z = 1.f / (1.f + __expf(-o.z)); o.w = 1.f / (1.f + __expf(-o.w));
+                                    o.x = sigmoid_fast(o.x); o.y = sigmoid_fast(o.y);
+                                    o.z = sigmoid_fast(o.z); o.w = sigmoid_fast(o.w);
                                 }
                                 if (kMask) {
                                     if (p.mask_mode == 0) {
@@ -1039,7 +1039,7 @@ tc_fprop_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                                 float o = __uint_as_float(v[j]);
                                 if (p.bias) o += __ldg(p.bias + col0 + j);
                                 if (p.act == PCL_ACT_RELU) o = fmaxf(o, 0.f);
-                                else if (p.act == PCL_ACT_SIGMOID) o = 1.f / (1.f + __expf(-o));
+                                else if (p.act == PCL_ACT_SIGMOID) o = sigmoid_fast(o);
                                 if (msk) {
                                     const float m = __ldg(msk + j);
                                     o = p.mask_mode == 0 ? (m > 0.f ? o : 0.f) : o * (m * (1.f - m));
