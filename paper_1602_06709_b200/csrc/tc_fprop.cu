@@ -233,8 +233,10 @@ __device__ __forceinline__ void halo_taps(uint32_t d_tmem, uint32_t BN, uint32_t
     }
 }
 
-// The MMA-issuing role, one thread per issuing warp (waits included), kept out of line and free of anything the
-// loops do not need.  A lone thread executes an instruction every several cycles; a barrier poll or a commit costs
+// The MMA-issuing role, one warp per issuer (waits included), kept out of line and free of anything the loops do not
+// need.  The WHOLE warp runs it, every lane with the same values, and the MMA and commit forms elect one lane to issue:
+// run by lane 0 alone the same loops are divergent code whose descriptors the compiler moves into uniform registers
+// word by word, at twice the cycles per MMA.  A lone thread executes an instruction every several cycles; a barrier poll or a commit costs
 // it ~80 cycles and every MMA ~45, so per slot it spends 300-400 cycles outside the MMAs, which the MMA queue (4-5
 // deep) hides only behind wide MMAs (N = 256).  kDuo: two issuers take the slots alternately, so that one thread's
 // bookkeeping overlaps the other's MMAs.  MMAs of both accumulate into the same tile (the pipe executes them one
@@ -293,6 +295,7 @@ __device__ __noinline__ void mma_issuer(const FpropParams& p, const IssuerCtx& c
     uint32_t turn = 0, seq = 0;     // kDuo: whose slot comes next; slots so far (both threads count alike)
     // tile_duo: the two issuing threads take the CTA's tiles alternately, each with its own accumulator set and its
     // own patch buffers (NA is even), so nothing orders them against each other; the weights stay resident.
+    const bool leader = elected_lane();       // the lane that issues; it alone publishes the turn
     const bool tduo = !kDuo && p.tile_duo != 0;
     const int cnt0 = tduo ? int(issuer) : 0, cnt_step = tduo ? 2 : 1;
     int a_slot = cnt0;
@@ -305,14 +308,15 @@ __device__ __noinline__ void mma_issuer(const FpropParams& p, const IssuerCtx& c
     if (kDuo) { mine = turn == issuer; turn ^= 1u; }
 #define PCL_SLOT_ACQUIRE()                                                                                        \
     if (!(resident && tile_cnt > cnt0) &&                                                                         \
-        !bounded_wait_addr(full_a, phase, abort_flag, status, WAIT_MMA_FULL)) { ok = false; break; }             \
-    if (kDuo && !wait_issue_turn(issue_seq, seq, abort_flag, status)) { ok = false; break; }                     \
-    if (kDuo && split) *issue_seq = seq + 1;     /* split: only the slot STARTS are ordered (see below) */        \
+        !bounded_wait_addr_warp(full_a, phase, abort_flag, status, WAIT_MMA_FULL)) { ok = false; break; }        \
+    if (kDuo && !__all_sync(0xffffffffu, wait_issue_turn(issue_seq, seq, abort_flag, status))) { ok = false; break; } \
+    if (kDuo && split && leader) *issue_seq = seq + 1;     /* split: only the slot STARTS are ordered (see below) */ \
+    __syncwarp();                                                                                                 \
     tc_fence_after();
 #define PCL_SLOT_RELEASE()                                                                                        \
     /* ordered hand-over: this thread's MMAs are fenced before the turn is published (the other issuer fences  */ \
     /* after reading it), so that MMAs of consecutive slots into one accumulator are ordered across the threads */ \
-    if (kDuo && !split) { tc_fence_before(); *issue_seq = seq + 1; }                                              \
+    if (kDuo && !split) { tc_fence_before(); if (leader) *issue_seq = seq + 1; __syncwarp(); }                    \
     if (!resident) umma_commit_addr<kPair>(empty_a);
 #define PCL_SLOT_END()                                                                                            \
     if (kDuo) ++seq;                                                                                              \
@@ -323,7 +327,7 @@ __device__ __noinline__ void mma_issuer(const FpropParams& p, const IssuerCtx& c
     for (int t = first_tile + cnt0 * tile_stride; t < total_tiles && ok; t += cnt_step * tile_stride, tile_cnt += cnt_step) {
         const uint32_t acc = tile_cnt & 1;
         const uint32_t acc_phase = (tile_cnt >> 1) & 1;
-        if (!bounded_wait_addr(tempty0 + acc * 8, acc_phase ^ 1u, abort_flag, status, WAIT_MMA_TMEM_EMPTY)) break;
+        if (!bounded_wait_addr_warp(tempty0 + acc * 8, acc_phase ^ 1u, abort_flag, status, WAIT_MMA_TMEM_EMPTY)) break;
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + (split ? (2 * acc + issuer) * MT * BN : acc * MT * BN);
         uint32_t accum = 0;         // the tile's first MMA (whoever issues it) overwrites the accumulator
@@ -333,7 +337,7 @@ __device__ __noinline__ void mma_issuer(const FpropParams& p, const IssuerCtx& c
             const uint32_t a_hi = uint32_t(a_desc0 >> 32);
             const uint32_t row16 = (PW - S) * 8;        // from the end of a tap row to the start of the next
             for (int cb = 0; cb < cblocks && ok; ++cb) {
-                if (!bounded_wait_addr(fullA0 + a_slot * 8, phaseA, abort_flag, status, WAIT_MMA_FULL)) { ok = false; break; }
+                if (!bounded_wait_addr_warp(fullA0 + a_slot * 8, phaseA, abort_flag, status, WAIT_MMA_FULL)) { ok = false; break; }
                 // the tap (r, s) = a shift by (r * PW + s) pixels of 128 bytes inside the patch
                 uint32_t a_lo = uint32_t(a_desc0) + ((smem_u32(smem + a_slot * a_buf_bytes) & 0x3FFFFu) >> 4);
                 int s = 0;
@@ -444,14 +448,6 @@ tc_fprop_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
     const uint32_t pair_rank = kPair ? cluster_ctarank() : 0u;
     const int first_tile = kPair ? int(cluster_id_x()) : int(blockIdx.x);
     const int tile_stride = kPair ? int(nclusters_x()) : int(gridDim.x);
-    auto issue_mma = [](uint32_t d, uint64_t da, uint64_t db, uint32_t idesc, uint32_t accumulate) {
-        if constexpr (kPair) umma_tf32_pair(d, da, db, idesc, accumulate);
-        else umma_tf32(d, da, db, idesc, accumulate);
-    };
-    auto commit = [](uint64_t* bar) {
-        if constexpr (kPair) umma_commit_pair(bar);
-        else umma_commit(bar);
-    };
     const uint32_t step_bytes = p.halo ? b_bytes : kABytes + b_bytes;
     const uint32_t stage_bytes = p.KS * step_bytes;
     uint8_t* b_ring = smem + (p.halo ? p.NA * p.a_buf_bytes : kABytes);
@@ -631,7 +627,7 @@ tc_fprop_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
     } else if (warp == 1 || warp == kSecondIssuerWarp) {
         // --------------------------------------------------------- MMA issuers
         const uint32_t issuer = warp == 1 ? 0u : 1u;
-        if (lane == 0 && pair_rank == 0 && issuer < uint32_t(p.tile_duo ? 2 : p.issuers)) {
+        if (pair_rank == 0 && issuer < uint32_t(p.tile_duo ? 2 : p.issuers)) {     // the whole warp (see mma_issuer)
             IssuerCtx c;
             c.smem = smem; c.b_ring = b_ring;
             c.full_bar = full_bar; c.empty_bar = empty_bar; c.fullA_bar = fullA_bar; c.emptyA_bar = emptyA_bar;

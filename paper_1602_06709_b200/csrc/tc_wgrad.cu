@@ -288,7 +288,7 @@ tc_wgrad_kernel(const __grid_constant__ CUtensorMap tmDy, const __grid_constant_
     } else if (warp == 1 || warp == kSecondIssuerWarp) {
         const uint32_t issuer = warp == 1 ? 0u : 1u;
         const uint32_t nis = p.duo ? 2u : 1u;
-        if (lane == 0 && pair_rank == 0 && issuer < nis) {     // one thread runs a whole issue loop, waits included
+        if (pair_rank == 0 && issuer < nis) {     // the whole warp runs the issue loop, waits included; an elected lane issues
         const uint32_t d_tmem = tmem_base + issuer * uint32_t(p.acc_cols);
         const uint32_t idesc = make_idesc_tf32(n_groups * 32, true, true, kPair ? 256u : 128u);
         // 8 pixels per MMA = two 512-byte groups of 4 rows (1 KB, 64 sixteen-byte units, per MMA); descriptors differ
@@ -322,7 +322,7 @@ tc_wgrad_kernel(const __grid_constant__ CUtensorMap tmDy, const __grid_constant_
             constexpr int kRows = decltype(rows_c)::value, kSteps = decltype(steps_c)::value, kCg = decltype(cg_c)::value;
             const int rows = kRows ? kRows : xrows, steps = kSteps ? kSteps : xsteps, cgs = kCg ? kCg : p.cg;
             for (int kit = int(issuer); kit < kiters; kit += int(nis)) {
-                if (!bounded_wait_addr(full_a, phase, &abort_flag, p.status, WAIT_MMA_FULL)) { ok = false; break; }
+                if (!bounded_wait_addr_warp(full_a, phase, &abort_flag, p.status, WAIT_MMA_FULL)) { ok = false; break; }
                 tc_fence_after();
                 uint32_t ar = slot_lo, br = slot_lo + a16 + xlbo;
                 if constexpr (kRows != 0) {
@@ -352,7 +352,7 @@ tc_wgrad_kernel(const __grid_constant__ CUtensorMap tmDy, const __grid_constant_
             else xhalo_loop(integral_constant<int, 0>{}, integral_constant<int, 0>{}, integral_constant<int, 0>{});
         } else
         for (int kit = int(issuer) * p.KS; kit < kiters; kit += int(nis) * p.KS) {
-            if (!bounded_wait_addr(full_a, phase, &abort_flag, p.status, WAIT_MMA_FULL)) { ok = false; break; }
+            if (!bounded_wait_addr_warp(full_a, phase, &abort_flag, p.status, WAIT_MMA_FULL)) { ok = false; break; }
             tc_fence_after();
             const int nst = kiters - kit < p.KS ? kiters - kit : p.KS;
             uint32_t a_lo = slot_lo;
