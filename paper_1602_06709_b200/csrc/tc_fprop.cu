@@ -491,9 +491,9 @@ tc_fprop_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
 
     if (warp == 0) {
         // ------------------------------------------------------------ producer
-        // One thread; its loop is kept to a few instructions per copy (addresses and coordinates advance by
-        // addition), because at one thread per warp every instruction costs cycles of the k-step budget.
-        if (lane == 0) {
+        // The whole warp runs the loop (every lane the same values) and an elected lane issues the copies and arms the
+        // barriers; the loop is kept to a few instructions per copy (addresses and coordinates advance by addition).
+        {
             int stage = 0, issued = 0;
             uint32_t phase = 0;
             int a_slot = 0, issuedA = 0;
@@ -513,7 +513,7 @@ tc_fprop_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                 const int kcol = it.kt * p.BN + (kPair ? int(pair_rank) * (p.BN >> 1) : 0);
                 if (p.halo) {
                     for (int c0 = 0; c0 < c_end && ok; c0 += kBlockC) {
-                        if (!bounded_wait(&emptyA_bar[a_slot], phaseA ^ 1u, &abort_flag, p.status, WAIT_PRODUCER_EMPTY)) {
+                        if (!bounded_wait_warp(&emptyA_bar[a_slot], phaseA ^ 1u, &abort_flag, p.status, WAIT_PRODUCER_EMPTY)) {
                             ok = false;
                             break;
                         }
@@ -526,7 +526,7 @@ tc_fprop_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                         if (++a_slot == p.NA) { a_slot = 0; phaseA ^= 1u; }
                         for (int tap = 0; tap < taps; tap += p.KS) {
                             if (p.resident_b && it.t != first_tile) break;      // (loaded for the first tile, never released)
-                            if (!bounded_wait_addr(empty_a, phase ^ 1u, &abort_flag, p.status, WAIT_PRODUCER_EMPTY)) {
+                            if (!bounded_wait_addr_warp(empty_a, phase ^ 1u, &abort_flag, p.status, WAIT_PRODUCER_EMPTY)) {
                                 ok = false;
                                 break;
                             }
@@ -568,7 +568,7 @@ tc_fprop_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                         cq += s * dil; cp += r0;
                     }
                     for (int kit = 0; kit < kiters; kit += p.KS) {
-                        if (!bounded_wait_addr(empty_a, phase ^ 1u, &abort_flag, p.status, WAIT_PRODUCER_EMPTY)) {
+                        if (!bounded_wait_addr_warp(empty_a, phase ^ 1u, &abort_flag, p.status, WAIT_PRODUCER_EMPTY)) {
                             ok = false;
                             break;
                         }

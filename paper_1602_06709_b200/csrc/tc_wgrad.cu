@@ -187,9 +187,9 @@ tc_wgrad_kernel(const __grid_constant__ CUtensorMap tmDy, const __grid_constant_
     const int bw = 1 << p.bw_log2, bh = 1 << p.bh_log2, bn = p.pix >> (p.bw_log2 + p.bh_log2);
 
     if (warp == 0) {
-        // One thread; the loop is kept to a few instructions per copy (every instruction of a lone thread
-        // costs cycles of the k-step budget): addresses advance by addition, run coordinates are decoded once.
-        if (lane == 0) {
+        // The whole warp runs the loop and an elected lane issues the copies; the loop is kept to a few instructions
+        // per copy: addresses advance by addition, run coordinates are decoded once.
+        {
             int stage = 0;
             uint32_t phase = 0;
             int issued = 0;
@@ -223,7 +223,7 @@ tc_wgrad_kernel(const __grid_constant__ CUtensorMap tmDy, const __grid_constant_
             const int xsw = p.stride_w, xsh = p.stride_h;      // x coordinates of a box: the dy box's times the stride
             for (int b = box_begin; b < box_end; ++b) {
                 if (sub == 0) {
-                    if (!bounded_wait_addr(empty_a, phase ^ 1u, &abort_flag, p.status, WAIT_PRODUCER_EMPTY)) { ok = false; break; }
+                    if (!bounded_wait_addr_warp(empty_a, phase ^ 1u, &abort_flag, p.status, WAIT_PRODUCER_EMPTY)) { ok = false; break; }
                     const int nst = box_end - b < p.KS ? box_end - b : p.KS;
                     // pair: both CTAs' copies complete on the leader's barrier, which its producer arms
                     if (!kPair) mbar_expect_tx_addr(full_a, nst * tx_bytes + (p.inject_short_copy && issued == 0 ? 16 : 0));
