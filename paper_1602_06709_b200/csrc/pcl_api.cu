@@ -662,13 +662,16 @@ int bwd_data_masked_colsum(const pcl_conv_desc* d, int P, int Q, const float* dy
             char* extra = static_cast<char*>(ws) + base;
             float* sum_rows = reinterpret_cast<float*>(extra);
             a.colsum_rows = sum_rows;
-            // rows the chosen tiling does not write must not contribute: the sizing took the largest tiling
-            rc = launch_zero(sum_rows, size_t(rows) * d->C, st);
+            // (the workspace is sized for the tiling with the most rows; this launch writes rows 0 .. written-1, of which a
+            // grid smaller than the device leaves some untouched: those must not contribute)
+            long written = tc_fprop_colsum_rows_written(a);
+            if (written <= 0 || written > rows) written = rows;
+            rc = launch_zero(sum_rows, size_t(written) * d->C, st);
             if (rc != PCL_OK) return rc;
             rc = launch_tc_fprop(a, st);
             if (rc != PCL_OK) return rc;
             float* partial = reinterpret_cast<float*>(extra + align_up(size_t(rows) * d->C * 4, 256));
-            return launch_colsum(sum_rows, size_t(rows), d->C, partial, dx_colsum, st);
+            return launch_colsum(sum_rows, size_t(written), d->C, partial, dx_colsum, st);
         }
         if (!dx_colsum && !mask && ws && ws_bytes > bwd_data_transposed_bytes(*d)) {      // room to split a long reduction
             const size_t t = bwd_data_transposed_bytes(*d);

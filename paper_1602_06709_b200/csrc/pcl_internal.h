@@ -136,9 +136,10 @@ struct TcFpropArgs {
     // elements carry weight: the rest of the window is real neighbouring data that meets zero weights, which
     // avoids TMA's slower partial-row zero fill.
     int in_inner = 0;
-    // Optional fused column sums of the output (after bias / activation / mask): every (tile box, 32-row
-    // quarter) writes one row of per-column sums to `colsum_rows` ([tc_fprop_colsum_rows(a)][Kout], fully
-    // written when Kout % 4 == 0); the caller adds the rows up in a fixed order.
+    // Optional fused column sums of the output (after bias / activation / mask), Kout % 4 == 0: rows of per-column
+    // sums go to `colsum_rows` -- one per (CTA, tile box, 32-row quarter) when all tiles have the same columns (the
+    // sums are kept over the CTA's tiles), else one per (tile, box, quarter); tc_fprop_colsum_rows_written(a) rows,
+    // of which a small grid may leave some untouched (zero them first); the caller adds the rows in a fixed order.
     float* colsum_rows = nullptr;
     // Optional fused 2x2 / stride-2 max pooling of the output: pool_out [N][P/2][Q/2][Kout] gets the window maxima
     // of `out` (after bias and activation).  Needs even P and Q and Kout % 4 == 0 (tc_fprop_can_pool()).
@@ -169,7 +170,8 @@ bool tc_fprop_can_pool(const TcFpropArgs& a);
 // bytes of split_ws with which launch_tc_fprop(a) would split the reduction (0: it would not)
 size_t tc_fprop_split_ws_bytes(const TcFpropArgs& a);
 bool tc_fprop_eligible(const TcFpropArgs& a);
-long tc_fprop_colsum_rows(const TcFpropArgs& a);
+long tc_fprop_colsum_rows(const TcFpropArgs& a);              // upper bound over all tilings (workspace sizing)
+long tc_fprop_colsum_rows_written(const TcFpropArgs& a);      // rows the launch for exactly these arguments writes
 int launch_tc_fprop(const TcFpropArgs& a, cudaStream_t st);
 // Text description of the tiling launch_tc_fprop(a) would use and of the cost model's prediction for it (and of the
 // tiling the model itself would choose).

@@ -97,6 +97,8 @@ struct FpropParams {
     // K = 8 slices of a 32-element channel block that hold anything but zeros (4 unless the few-channel path packs
     // fewer live taps x channels into a block: the MMAs of all-zero slices are not issued)
     int kslices;
+    int colsum_cta;         // column sums are kept per CTA over all its tiles (tiles_k == 1) and written once, one row
+                            // per (CTA, box, lane quarter), instead of one row per (tile, box, lane quarter)
     int tile_duo;           // two issuing threads, alternate tiles (resident weights, one patch per tile, even NA)
     int bias_in_smem;           // the CTA keeps bias[0 .. BN) in shared memory (tiles_k == 1: every tile has the same columns)
     unsigned char* pool_idx;    // optional, with pool_out: per pooled element the position of the maximum (bits 0-1) and bit 2
@@ -654,6 +656,8 @@ tc_fprop_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
         const bool vec_ok = (p.Kout & 3) == 0;
         int tile_cnt = 0;
         TileIter it;
+        // per-CTA column sums (colsum_cta): this lane's partial sums of the warp's (at most four) chunks of a tile
+        float4 cacc0 = make_float4(0.f, 0.f, 0.f, 0.f), cacc1 = cacc0, cacc2 = cacc0, cacc3 = cacc0;
         bool pooled_only = false;
         if constexpr (kPool) pooled_only = !p.out && p.act != PCL_ACT_SIGMOID && (kEpi > kEpiWarps || (!kMask && p.tma_store));
         if (pooled_only) {
@@ -783,6 +787,7 @@ tc_fprop_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
             const int kt = it.kt;
             if (!bounded_wait_warp(&tmem_full_bar[acc], acc_phase, &abort_flag, p.status, WAIT_EPI_TMEM_FULL)) break;
             tc_fence_after();
+            int cs_item = 0;        // running index of the warp's chunks in this tile (h-major), for the per-CTA sums
             for (int h = 0; h < p.MT; ++h) {
             const int ch0 = (sub - h * cpb) & (kSub - 1);       // first chunk of box h that is this warp's
             const int q = it.qi * p.tw + iw + h * p.half_dq;
@@ -795,7 +800,7 @@ tc_fprop_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                                    ((p.split_acc ? 2 * acc : acc) * p.MT + h) * p.BN;
             const uint32_t t_second = p.MT * p.BN;      // split accumulators: the second issuer's copy of this box
             float* cs_row = nullptr;
-            if (p.colsum_rows && ni * p.tn < p.N) {      // (an odd image-group count leaves the pair's last tile empty)
+            if (p.colsum_rows && !p.colsum_cta && ni * p.tn < p.N) {      // (an odd image-group count leaves the pair's last tile empty)
                 const size_t m_index = (static_cast<size_t>(ni) * p.tiles_p + it.pi) * p.tiles_q + it.qi;
                 cs_row = p.colsum_rows + ((m_index * p.MT + h) * 4 + quarter) * p.Kout;
             }
@@ -919,7 +924,7 @@ tc_fprop_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                 }
                 const uint32_t stg = smem_u32(epi_stage + epi * 4096);
                 const int cg = (lane & 7) * 4;
-                for (int ch = ch0; ch < cpb; ch += kSub) {
+                for (int ch = ch0; ch < cpb; ch += kSub, ++cs_item) {
                     const int col = kt * p.BN + ch * 32 + cg;
                     // (the bias is fetched before the accumulator so that its latency hides behind the staging)
                     float4 b = make_float4(0.f, 0.f, 0.f, 0.f);
@@ -978,7 +983,14 @@ tc_fprop_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                                 csum.x += o.x; csum.y += o.y; csum.z += o.z; csum.w += o.w;
                             }
                         }
-                        if (cs_row) {
+                        if (p.colsum_cta) {
+                            // (per-CTA sums: this lane's partial sums of the chunk are kept over the CTA's tiles, in
+                            // the order of the tiles; the lane groups are added once, at the end)
+                            if (cs_item == 0) { cacc0.x += csum.x; cacc0.y += csum.y; cacc0.z += csum.z; cacc0.w += csum.w; }
+                            else if (cs_item == 1) { cacc1.x += csum.x; cacc1.y += csum.y; cacc1.z += csum.z; cacc1.w += csum.w; }
+                            else if (cs_item == 2) { cacc2.x += csum.x; cacc2.y += csum.y; cacc2.z += csum.z; cacc2.w += csum.w; }
+                            else { cacc3.x += csum.x; cacc3.y += csum.y; cacc3.z += csum.z; cacc3.w += csum.w; }
+                        } else if (cs_row) {
                             // rows (lane>>3) + 4i were summed per lane; add the four lane groups in a fixed order
                             csum.x += __shfl_xor_sync(live, csum.x, 8);  csum.y += __shfl_xor_sync(live, csum.y, 8);
                             csum.z += __shfl_xor_sync(live, csum.z, 8);  csum.w += __shfl_xor_sync(live, csum.w, 8);
@@ -1055,6 +1067,21 @@ tc_fprop_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
             }
         }
         if (!kMask && p.tma_store && lane == 0) bulk_wait_group0();     // every store of this warp has completed
+        if (p.colsum_cta && p.colsum_rows) {
+            // one row per (CTA, box, lane quarter): the four lane groups of each chunk are added in a fixed order
+            int item = 0;
+            for (int h = 0; h < p.MT; ++h)
+                for (int ch = (sub - h * cpb) & (kSub - 1); ch < cpb; ch += kSub, ++item) {
+                    float4 c = item == 0 ? cacc0 : (item == 1 ? cacc1 : (item == 2 ? cacc2 : cacc3));
+                    c.x += __shfl_xor_sync(0xffffffffu, c.x, 8);  c.y += __shfl_xor_sync(0xffffffffu, c.y, 8);
+                    c.z += __shfl_xor_sync(0xffffffffu, c.z, 8);  c.w += __shfl_xor_sync(0xffffffffu, c.w, 8);
+                    c.x += __shfl_xor_sync(0xffffffffu, c.x, 16); c.y += __shfl_xor_sync(0xffffffffu, c.y, 16);
+                    c.z += __shfl_xor_sync(0xffffffffu, c.z, 16); c.w += __shfl_xor_sync(0xffffffffu, c.w, 16);
+                    const int col = ch * 32 + (lane & 7) * 4;      // (tiles_k == 1: every tile has these columns)
+                    if (lane < 8 && col < p.Kout)
+                        *reinterpret_cast<float4*>(p.colsum_rows + ((static_cast<size_t>(blockIdx.x) * p.MT + h) * 4 + quarter) * p.Kout + col) = c;
+                }
+        }
     }
 
     tc_fence_before();
@@ -1312,6 +1339,17 @@ TileCfg select_cfg(const TcFpropArgs& a, int sm_count) {
 
 }  // namespace
 
+// Rows of column sums the launch for `a` writes (rows 0 .. n-1 of its colsum_rows buffer): per CTA where every tile
+// has the same columns, else per tile.
+long tc_fprop_colsum_rows_written(const TcFpropArgs& a) {
+    const int sm = device_sm_count();
+    if (a.Kout % 4 != 0) return 0;
+    const TileCfg c = select_cfg(a, sm);
+    if (!c.ok) return 0;
+    if (c.tiles_k == 1) return long(sm) * c.MT * 4;
+    return long(c.tiles_q) * c.tiles_p * c.tiles_n * c.MT * 4;
+}
+
 long tc_fprop_colsum_rows(const TcFpropArgs& a) {
     const int sm = device_sm_count();
     if (a.Kout % 4 != 0) return 0;
@@ -1456,6 +1494,7 @@ int launch_tc_fprop(const TcFpropArgs& a, cudaStream_t st) {
         p.tile_duo = (p.resident_b && p.cblocks == 1 && p.NA % 2 == 0 && tune(TUNE_ISSUERS, 2) >= 2) ? 1 : 0;
     }
     p.colsum_rows = (a.Kout % 4 == 0) ? a.colsum_rows : nullptr;
+    p.colsum_cta = (p.colsum_rows && p.tiles_k == 1 && p.ksplit == 1) ? 1 : 0;
     if (a.colsum_rows && !p.colsum_rows) return PCL_ERR_UNSUPPORTED_SHAPE;
     p.status = device_status_ptr();
     if (!p.status) return PCL_ERR_CUDA;
