@@ -232,7 +232,10 @@ def test_maxpool_bwd_with_fused_column_sums(N, H, W, C):
 
 
 @pytest.mark.parametrize("tiling", ["auto", "plain", "halo1"])
-@pytest.mark.parametrize("shape", [(3, 40, 72, 19, 23), (2, 64, 64, 32, 32), (2, 128, 320, 12, 12), (2, 7, 9, 11, 13)])
+@pytest.mark.parametrize("shape", [(3, 40, 72, 19, 23), (2, 64, 64, 32, 32), (2, 128, 320, 12, 12), (2, 7, 9, 11, 13),
+                                   # more tiles than SMs (a CTA keeps its column sums over several tiles); dx wider than one
+                                   # tile (tiles differ in their columns: one row of sums per tile)
+                                   (16, 32, 48, 40, 40), (2, 320, 64, 12, 12)])
 def test_conv_bwd_data_with_fused_column_sums(shape, tiling, monkeypatch):
     import gpu_helpers as G
     from oracle import ConvShape
