@@ -3,7 +3,7 @@
 The paper picks the cache and register blocks of every layer with a brute-force
 search that minimises bytes moved per flop under the cache capacity.  Here the
 blocks are the kernel's tilings -- plain or haloed (three layouts), tile width
-BN, single CTAs or CTA pairs -- and the search does both things the paper's does:
+BN, single CTAs or CTA pairs (both tilings) -- and the search does both things the paper's does:
 
 * the library's cost model (tensor pipe, shared-memory fill rate, issuing
   thread, epilogue warps; ``pcl_conv_plan_describe``) predicts every candidate;
@@ -76,9 +76,10 @@ def search_layer(name, N, C, K, H, R, pad, reps, flush, gen):
             for bn in (64, 128, 256):
                 if bn > max(64, (K + 31) // 32 * 32 if pid == B.PASS_FWD else (C + 31) // 32 * 32):
                     continue
-                for pair in ((0, 1) if tiling == "plain" else (0,)):
+                for pair in (0, 1):
                     B.reset_tuning()
-                    B.set_tuning("TILING", tiling); B.set_tuning("BN", bn); B.set_tuning("PAIR", pair)
+                    B.set_tuning("TILING", tiling); B.set_tuning("BN", bn)
+                    B.set_tuning("PAIR" if tiling == "plain" else "PAIR_HALO", pair)
                     desc = B.conv_plan_describe(d, pid)
                     cfg = _cfg_of(desc)
                     if cfg in results:

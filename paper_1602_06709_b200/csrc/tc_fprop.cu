@@ -1200,7 +1200,7 @@ TileCfg plain_cfg(const TcFpropArgs& a, int cblocks, int sm_count, int bn_force 
 }
 
 // layout: 0 = one box (8 x 16), 1 = two boxes side by side (16 x 16), 2 = two boxes stacked (8 x 32)
-TileCfg halo_cfg(const TcFpropArgs& a, int cblocks, int sm_count, int layout, int bn_force = -1) {
+TileCfg halo_cfg(const TcFpropArgs& a, int cblocks, int sm_count, int layout, int bn_force = -1, int pair_force = -1) {
     TileCfg c;
     c.halo = 1; c.MT = layout == 0 ? 1 : 2;
     c.bw_log2 = 3; c.bh_log2 = 4;
@@ -1218,11 +1218,16 @@ TileCfg halo_cfg(const TcFpropArgs& a, int cblocks, int sm_count, int layout, in
     c.BN = bn_force > 0 ? bn_force : choose_bn(a.Kout, m_tiles, sm_count);
     if (2 * c.MT * c.BN > 512) return c;          // two accumulator sets must fit the 512 TMEM columns
     c.tiles_k = (a.Kout + c.BN - 1) / c.BN;
-    c.pair = tune(TUNE_PAIR_HALO, 0) && c.tiles_n >= 2 && sm_count >= 2;      // pairs of images (no gain measured)
+    // Pairs of images: the two CTAs of a cluster take the same tile of two consecutive images against the same weight
+    // tile, of which each loads half the rows (the conditions are the plain tiling's: whole 16-column MMA halves,
+    // MN-major weights in whole 32-map groups per CTA).  Halving the weight bytes per CTA doubles the depth of the
+    // weight ring, which is what a narrow layer's tiles wait for.
+    const bool pair_ok = c.BN >= 64 && c.BN % 16 == 0 && c.tiles_n >= 2 && sm_count >= 2 && (!a.wt_mn_major || c.BN % 64 == 0);
+    c.pair = (pair_force >= 0 ? pair_force != 0 : tune(TUNE_PAIR_HALO, 0) != 0) && pair_ok;
     const int b_bytes = c.pair ? c.BN * 64 : c.BN * 128;
     const int room = kSmemBudget - kEpiStageBytes;
     c.NA = 2;
-    c.KS = tune(TUNE_KS_HALO, c.BN <= 64 ? 3 : (c.BN <= 128 ? 2 : 1));
+    c.KS = tune(TUNE_KS_HALO, (c.BN <= 64 || (c.pair && c.BN <= 128)) ? 3 : (c.BN <= 128 ? 2 : 1));
     if (c.KS > a.R * a.S) c.KS = a.R * a.S;
     while (c.KS > 1 && (room - c.NA * c.a_buf_bytes) / (c.KS * b_bytes) < 3) --c.KS;
     c.grp = tune(TUNE_GRP, 1) && c.KS > 1 && !a.wt_mn_major;      // (MN-major weights: one copy per tap)
@@ -1248,7 +1253,8 @@ struct TileCost { double mma, fill, issue, epilogue, tile, total; };
 constexpr double kMmaFloorClk = 52.0;        // a K = 8 MMA of N columns takes max(N / 2, 52) cycles
 constexpr double kFillSingle = 60.0;         // bytes per clock and SM into shared memory, single CTAs of this kernel
 constexpr double kFillPair = 57.0;           //   ... CTA pairs (which need a third fewer bytes per MMA)
-constexpr double kHaloMmaFactor = 1.5;       // MMAs whose A operand is a row-shifted view of a haloed patch run slower
+constexpr double kHaloMmaFactor = 1.5;       // haloed tiles take this much longer than their MMAs (a fit: the pipe itself runs row-shifted views at full rate)
+constexpr double kHaloPairMmaFactor = 1.3;   //   ... as CTA pairs (half the weight bytes per CTA, a weight ring twice as deep)
 constexpr double kHaloOneBoxFactor = 1.3;    //   ... and slower still when a tile is one box (no second box to share a weight tile with)
 constexpr double kIssueMmaClk = 45.0;        // the issuing thread's cost per MMA
 constexpr double kIssueSlotClk = 160.0;      //   ... per pipeline slot (one barrier round trip and one commit)
@@ -1260,7 +1266,7 @@ TileCost predict_cost(const TcFpropArgs& a, const TileCfg& c, int cblocks, int s
     const double ksteps = double(a.R) * a.S * cblocks;
     const double b_bytes = c.pair ? c.BN * 64.0 : c.BN * 128.0;
     const double mma_clk = c.BN / 2.0 > kMmaFloorClk ? c.BN / 2.0 : kMmaFloorClk;
-    t.mma = c.MT * ksteps * 4.0 * mma_clk * (c.halo ? kHaloMmaFactor * (c.MT == 1 ? kHaloOneBoxFactor : 1.0) : 1.0);
+    t.mma = c.MT * ksteps * 4.0 * mma_clk * (c.halo ? (c.pair ? kHaloPairMmaFactor : kHaloMmaFactor) * (c.MT == 1 ? kHaloOneBoxFactor : 1.0) : 1.0);
     const double bytes = c.halo ? cblocks * (double(c.patch_bytes) + double(a.R) * a.S * b_bytes) : ksteps * (kABytes + b_bytes);
     t.fill = bytes / (c.pair ? kFillPair : kFillSingle);
     const double slots = c.halo ? cblocks * double((a.R * a.S + c.KS - 1) / c.KS) : (ksteps + c.KS - 1) / c.KS;
@@ -1293,13 +1299,18 @@ TileCfg search_cfg(const TcFpropArgs& a, int sm_count, TileCost* best_cost = nul
         if (a.wt_mn_major && (a.Kout % 32 != 0)) break;
         const int n_tiles = (a.Kout + bn - 1) / bn;
         if ((n_tiles - 1) * bn >= a.Kout) continue;
-        for (int variant = 0; variant < 5; ++variant) {
-            const TileCfg c = variant < 2 ? plain_cfg(a, cblocks, sm_count, bn, variant) : halo_cfg(a, cblocks, sm_count, variant - 2, bn);
-            if (!c.ok || (variant == 1 && !c.pair)) continue;
+        const int halo_pairs = tune(TUNE_PAIR_HALO, 1) ? 3 : 0;      // (PAIR_HALO = 0 takes the paired haloed candidates out)
+        for (int variant = 0; variant < 5 + halo_pairs; ++variant) {
+            const TileCfg c = variant < 2 ? plain_cfg(a, cblocks, sm_count, bn, variant)
+                              : variant < 5 ? halo_cfg(a, cblocks, sm_count, variant - 2, bn, 0)
+                                            : halo_cfg(a, cblocks, sm_count, variant - 5, bn, 1);
+            if (!c.ok || ((variant == 1 || variant >= 5) && !c.pair)) continue;
             if (c.halo && a.pool_out && (c.bw_log2 < 1 || c.bh_log2 < 1)) continue;
             const TileCost t = predict_cost(a, c, cblocks, sm_count);
             // (a haloed candidate must beat the plain ones by a tenth: its prediction is the less certain one)
-            const double score = t.total * (c.halo ? 1.1 : 1.0);
+            // (and between a haloed candidate and its paired form, which the model prices alike, the pair wins: it
+            // fetches half the weight bytes per CTA)
+            const double score = t.total * (c.halo ? (c.pair ? 1.099 : 1.1) : 1.0);
             if (score < best_total) { best_total = score; best = c; if (best_cost) *best_cost = t; }
         }
     }
@@ -1316,7 +1327,7 @@ TileCfg select_cfg(const TcFpropArgs& a, int sm_count) {
     // (the few-channel path reads overlapping windows, whose fill cost the model does not describe: rules too)
     const int sel = tune(TUNE_SELECT, (a.R * a.S > 1 && a.in_stride_w == 0) ? 1 : 0);
     if (sel == 1 && tune(TUNE_TILING, -1) < 0 && !tune_is_set(TUNE_BN) && !tune_is_set(TUNE_PAIR) && !tune_is_set(TUNE_KS) &&
-        !tune_is_set(TUNE_KS_HALO) && !tune_is_set(TUNE_GRP) && !tune_is_set(TUNE_PAIR_HALO)) {
+        !tune_is_set(TUNE_KS_HALO) && !tune_is_set(TUNE_GRP) && tune(TUNE_PAIR_HALO, 0) == 0) {
         const TileCfg m = search_cfg(a, sm_count);
         if (m.ok) return m;
     }

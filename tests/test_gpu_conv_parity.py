@@ -135,13 +135,18 @@ HALO_SHAPES = {
 }
 
 
-@pytest.mark.parametrize("tiling", ["plain", "halo0", "halo1", "halo2"])
+@pytest.mark.parametrize("tiling", ["plain", "halo0", "halo1", "halo2", "halo1_pair", "halo2_pair"])
 @pytest.mark.parametrize("tag", sorted(HALO_SHAPES))
 def test_forward_type_kernel_every_tiling(tag, tiling, path_guard, monkeypatch):
     """The forward-type kernel has a plain tiling and three haloed ones (taps as row-shifted views of one
-    input patch); the TILING knob pins one.  All must agree with the oracle for forward and backward-data."""
+    input patch), the haloed ones also as CTA pairs over two images; the TILING and PAIR_HALO knobs pin one.  All must
+    agree with the oracle for forward and backward-data (shapes whose tile width or weight layout does not allow a
+    pair run as single CTAs)."""
     import gpu_helpers as G
     from paper_1602_06709_b200 import binding as B
+    if tiling.endswith("_pair"):
+        tiling = tiling[:-5]
+        B.set_tuning("PAIR_HALO", 1)
     B.set_tuning("TILING", tiling)
     B.set_path(B.PATH_TENSOR)
     s = HALO_SHAPES[tag]
