@@ -1294,8 +1294,11 @@ TileCfg search_cfg(const TcFpropArgs& a, int sm_count, TileCost* best_cost = nul
     TileCfg best;
     double best_total = 1e300;
     const int k32 = (a.Kout + 31) / 32 * 32;
+    // (one tile width beyond the output's: a layer of 96 maps also tries 128-wide tiles, whose last 32 columns multiply
+    // zero fill and are not stored, because only multiples of 64 can run as CTA pairs)
+    const int k64 = (a.Kout + 63) / 64 * 64;
     for (int bn = 32; bn <= 256; bn += 32) {
-        if (bn > k32) break;
+        if (bn > k32 && bn != k64) break;
         if (a.wt_mn_major && (a.Kout % 32 != 0)) break;
         const int n_tiles = (a.Kout + bn - 1) / bn;
         if ((n_tiles - 1) * bn >= a.Kout) continue;
