@@ -118,12 +118,14 @@ class VggWorkload:
     name = "configs[4]: full VGG-A training step (fwd+bwd+SGD), N=256, 3x224x224, He-normal weights, 1000 classes"
     unit = "images/s"
 
-    def __init__(self, rank: int, minibatch: int = 0):
+    def __init__(self, rank: int, minibatch: int = 0, fused_update: bool = True):
         import torch
         from paper_1602_06709_b200 import inputs, networks
         self.torch = torch
         self.N = minibatch or 256
-        self.net = networks.VggA(self.N)
+        # (fused_update: each layer's SGD update is applied by its own weight-gradient call; the data-parallel step,
+        # which exchanges the gradients, keeps them and updates the owned strips)
+        self.net = networks.VggA(self.N, fused_update=fused_update)
         x = inputs.uniform(inputs.tensor_id("cfg5", "x", rank), (self.N, 224, 224, 3), 0.0, 1.0)
         lab = inputs.labels(inputs.tensor_id("cfg5", "labels", rank), self.N, 1000)
         self.x_host = torch.from_numpy(x).pin_memory()
@@ -226,12 +228,12 @@ class DnnWorkload:
     name = "configs[3]: 7-layer DNN 440-5x2048-8192, sigmoid, minibatch 1024: fwd + bwd + SGD update"
     unit = "frames/s"
 
-    def __init__(self, rank: int, minibatch: int = 0):
+    def __init__(self, rank: int, minibatch: int = 0, fused_update: bool = True):
         import torch
         from paper_1602_06709_b200 import inputs, networks
         self.torch = torch
         self.N = minibatch or inputs.CFG4_N
-        self.net = networks.Dnn(self.N)
+        self.net = networks.Dnn(self.N, fused_update=fused_update)
         x = inputs.normal(inputs.tensor_id("cfg4", "x", rank), (self.N, 440), 1.0)
         lab = inputs.labels(inputs.tensor_id("cfg4", "labels", rank), self.N, 8192)
         self.x_host = torch.from_numpy(x).pin_memory(); self.lab_host = torch.from_numpy(lab).pin_memory()
@@ -372,7 +374,8 @@ def run_ours(args):
     if args.layer:
         wl = ConvWorkload(rank, args.minibatch, tuple(int(v) for v in args.layer.split(",")), pooled=args.pooled)
     else:
-        wl = WORKLOADS[args.workload](rank, args.minibatch)
+        wl = (WORKLOADS[args.workload](rank, args.minibatch, fused_update=False)
+              if args.data_parallel and args.workload in ("vgga", "dnn") else WORKLOADS[args.workload](rank, args.minibatch))
     if args.data_parallel:
         # Sec. 3.1 / 3.4: the ranks share one model; every rank's step() exchanges the weight gradients layer by layer
         if not hasattr(wl, "net"):

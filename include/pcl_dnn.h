@@ -169,6 +169,18 @@ int pcl_conv_bwd_weights(const pcl_conv_desc* d, const float* x, const float* dy
                          float* dw, float* dbias, int deterministic,
                          void* ws, size_t ws_bytes, void* cuda_stream);
 
+/* Weight-gradient update with the SGD step applied by its own second pass (Sec. 3.1: a layer's new weights are
+ * only needed before its next forward pass, so the update need not wait for a pass of its own):
+ *   w[k,r,s,c] <- w[k,r,s,c] - lr * dw[k,r,s,c],   dw as in pcl_conv_bwd_weights(), never written to memory where the
+ * reduction over pixels is split (its second pass adds the partial sums in the fixed order and applies the update);
+ * otherwise dw goes to the workspace and the update follows.  Bit-identical to pcl_conv_bwd_weights() (deterministic)
+ * followed by pcl_sgd_update().  The caller must have issued every reader of the OLD weights (the layer's
+ * backpropagation) before this call.  w: KRSC in/out (device, 16-byte aligned); dbias: [K] out or NULL, as above.
+ * Workspace: pcl_conv_bwd_weights_sgd_workspace_bytes(d), 256-byte aligned.  Errors as pcl_conv_bwd_weights(). */
+size_t pcl_conv_bwd_weights_sgd_workspace_bytes(const pcl_conv_desc* d);
+int pcl_conv_bwd_weights_sgd(const pcl_conv_desc* d, const float* x, const float* dy, float* w, float lr,
+                             float* dbias, void* ws, size_t ws_bytes, void* cuda_stream);
+
 /* Weight-gradient update of a layer whose output went through the 2x2 / stride-2 max pool (the
  * conv -> ReLU -> pool blocks of the VGG-A topology, Sec. 5), taken straight from the POOLED gradient:
  *   dy[n,p,q,k] = dy_pool[n,p/2,q/2,k]  where (p%2)*2 + q%2 == pool_codes[n,p/2,q/2,k] & 3
@@ -232,6 +244,16 @@ int pcl_fc_bwd(int N, int C, int K, const float* x, const float* w, const float*
 int pcl_fc_bwd_fused(int N, int C, int K, const float* x, const float* w, const float* y, int act,
                      float* dy, float* dx, int x_act, float* dx_colsum, float* dw, float* dbias,
                      void* ws, size_t ws_bytes, void* cuda_stream);
+
+/* pcl_fc_bwd_fused() with the SGD step folded in: dx (and dx_colsum) are computed from the OLD weights first, then
+ *   w[k,c] <- w[k,c] - lr * dw[k,c]
+ * in place, without dw ever being stored (the weight-gradient GEMM's epilogue reads w and writes the updated value,
+ * or the second pass of its split reduction does).  dbias as in pcl_fc_bwd().  Bit-identical to pcl_fc_bwd_fused()
+ * followed by pcl_sgd_update() on w.  w: [K][C] in/out.  Workspace: pcl_fc_bwd_fused_sgd_workspace_bytes(N, C, K). */
+size_t pcl_fc_bwd_fused_sgd_workspace_bytes(int N, int C, int K);
+int pcl_fc_bwd_fused_sgd(int N, int C, int K, const float* x, float* w, const float* y, int act,
+                         float* dy, float* dx, int x_act, float* dx_colsum, float lr, float* dbias,
+                         void* ws, size_t ws_bytes, void* cuda_stream);
 
 /* Vanilla SGD (Sec. 1: algorithm and hyper-parameters untouched):
  *   w[i] <- w[i] - lr * dw[i],  i < n.   w, dw only need 4-byte alignment. */

@@ -31,7 +31,8 @@ EXPORTS = [
     "pcl_maxpool2x2_bwd_colsum_workspace_bytes", "pcl_maxpool2x2_bwd_colsum", "pcl_conv_fwd_pool", "pcl_conv_fwd_pool_is_fused",
     "pcl_conv_bwd_weights_pooled", "pcl_conv_bwd_weights_pooled_is_fused", "pcl_conv_bwd_weights_pooled_workspace_bytes",
     "pcl_maxpool2x2_fwd_codes", "pcl_maxpool2x2_bwd_codes", "pcl_last_wait_code", "pcl_set_tuning", "pcl_reset_tuning", "pcl_fc_bwd_fused", "pcl_conv_plan_describe", "pcl_conv_staged_input_bytes",
-    "pcl_conv_bwd_weights_pooled_staged",
+    "pcl_conv_bwd_weights_pooled_staged", "pcl_conv_bwd_weights_sgd", "pcl_conv_bwd_weights_sgd_workspace_bytes",
+    "pcl_fc_bwd_fused_sgd", "pcl_fc_bwd_fused_sgd_workspace_bytes",
 ]
 
 
@@ -90,6 +91,12 @@ def lib() -> ctypes.CDLL:
         L.pcl_fc_bwd.argtypes = [ci, ci, ci, vp, vp, vp, ci, vp, vp, vp, vp, vp, sz, vp]
         L.pcl_fc_bwd_fused.argtypes = [ci, ci, ci, vp, vp, vp, ci, vp, vp, ci, vp, vp, vp, vp, sz, vp]
         L.pcl_sgd_update.argtypes = [vp, vp, sz, cf, vp]
+        L.pcl_conv_bwd_weights_sgd_workspace_bytes.argtypes = [dp]
+        L.pcl_conv_bwd_weights_sgd_workspace_bytes.restype = sz
+        L.pcl_conv_bwd_weights_sgd.argtypes = [dp, vp, vp, vp, cf, vp, vp, sz, vp]
+        L.pcl_fc_bwd_fused_sgd_workspace_bytes.argtypes = [ci, ci, ci]
+        L.pcl_fc_bwd_fused_sgd_workspace_bytes.restype = sz
+        L.pcl_fc_bwd_fused_sgd.argtypes = [ci, ci, ci, vp, vp, vp, ci, vp, vp, ci, vp, cf, vp, vp, sz, vp]
         L.pcl_maxpool2x2_fwd.argtypes = [ci, ci, ci, ci, vp, vp, vp]
         L.pcl_maxpool2x2_bwd.argtypes = [ci, ci, ci, ci, vp, vp, vp, vp, vp]
         L.pcl_softmax_xent.argtypes = [ci, ci, vp, vp, vp, vp, vp]
@@ -307,6 +314,28 @@ def fc_bwd_fused(N, C, K, x, w, y, act, dy, dx, x_act, dx_colsum, dw, dbias, ws=
     wp, wb = _ws(ws)
     _check(lib().pcl_fc_bwd_fused(N, C, K, _ptr(x), _ptr(w), _ptr(y), act, _ptr(dy), _ptr(dx), x_act, _ptr(dx_colsum),
                                   _ptr(dw), _ptr(dbias), wp, wb, _stream(stream)), "pcl_fc_bwd_fused")
+
+
+def conv_bwd_weights_sgd_workspace_bytes(d) -> int:
+    return int(lib().pcl_conv_bwd_weights_sgd_workspace_bytes(ctypes.byref(d)))
+
+
+def conv_bwd_weights_sgd(d, x, dy, w, lr, dbias=None, ws=None, stream=None):
+    """w <- w - lr * dw(x, dy) in place, the update applied by the weight gradient's second pass (dw is not stored)."""
+    wp, wb = _ws(ws)
+    _check(lib().pcl_conv_bwd_weights_sgd(ctypes.byref(d), _ptr(x), _ptr(dy), _ptr(w), ctypes.c_float(lr), _ptr(dbias),
+                                          wp, wb, _stream(stream)), "pcl_conv_bwd_weights_sgd")
+
+
+def fc_bwd_fused_sgd_workspace_bytes(N, C, K) -> int:
+    return int(lib().pcl_fc_bwd_fused_sgd_workspace_bytes(N, C, K))
+
+
+def fc_bwd_fused_sgd(N, C, K, x, w, y, act, dy, dx, x_act, dx_colsum, lr, dbias, ws=None, stream=None):
+    """fc_bwd_fused with the SGD step folded in: dx from the old weights first, then w <- w - lr * dw in place."""
+    wp, wb = _ws(ws)
+    _check(lib().pcl_fc_bwd_fused_sgd(N, C, K, _ptr(x), _ptr(w), _ptr(y), act, _ptr(dy), _ptr(dx), x_act, _ptr(dx_colsum),
+                                      ctypes.c_float(lr), _ptr(dbias), wp, wb, _stream(stream)), "pcl_fc_bwd_fused_sgd")
 
 
 def sgd_update(w, dw, lr, stream=None):

@@ -56,6 +56,20 @@ __global__ void __launch_bounds__(256) reduce_splits_kernel(const float* __restr
     }
 }
 
+// w[i] <- w[i] - lr * (partial[0][i] + partial[1][i] + ...): the weight gradient's second pass applying the update itself
+// (Sec. 3.1: a layer's new weights are not needed before its next forward pass).  The sum is formed exactly as
+// reduce_splits_kernel forms it and applied exactly as sgd_kernel applies it, so the result equals the two-kernel form bit
+// for bit; dw itself is never written.
+__global__ void __launch_bounds__(256) reduce_splits_sgd_kernel(const float* __restrict__ partial, float* __restrict__ w,
+                                                                size_t n, int splits, float lr) {
+    const size_t stride = size_t(gridDim.x) * blockDim.x;
+    for (size_t i = size_t(blockIdx.x) * blockDim.x + threadIdx.x; i < n; i += stride) {
+        float acc = partial[i];
+        for (int s = 1; s < splits; ++s) acc += partial[size_t(s) * n + i];
+        w[i] = fmaf(-lr, acc, w[i]);
+    }
+}
+
 // wt_t[c][R-1-r][S-1-s][k] = w[k][r][s][c]: the "transpose-weights" copy the
 // backward-data pass contracts against (Sec. 2.3 keeps such a copy too).
 __global__ void __launch_bounds__(256) transpose_flip_kernel(const float* __restrict__ w, float* __restrict__ out,
@@ -598,6 +612,15 @@ int launch_reduce_splits(const float* partial, float* out, size_t n, int splits,
     {
         LaunchScope scope(KID_REDUCE_SPLITS, 4.0 * double(n) * (splits + 1), st);
         reduce_splits_kernel<<<grid_for(n, 256), 256, 0, st>>>(partial, out, n, splits);
+    }
+    return PCL_CHECK_LAUNCH();
+}
+
+int launch_reduce_splits_sgd(const float* partial, float* w, size_t n, int splits, float lr, cudaStream_t st) {
+    if (n == 0) return PCL_OK;
+    {
+        LaunchScope scope(KID_REDUCE_SPLITS, 4.0 * double(n) * (splits + 2), st);
+        reduce_splits_sgd_kernel<<<grid_for(n, 256), 256, 0, st>>>(partial, w, n, splits, lr);
     }
     return PCL_CHECK_LAUNCH();
 }

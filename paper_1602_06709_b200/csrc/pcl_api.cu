@@ -865,8 +865,54 @@ int pcl_conv_bwd_weights_pooled_staged(const pcl_conv_desc* d, const float* x_st
     return conv_bwd_weights_pooled_impl(d, nullptr, x_staged, dy_pool, pool_codes, relu_mask, dw, dbias, ws, ws_bytes, cuda_stream);
 }
 
+namespace {
+// Workspace of the fused-update form behind the plain form's: a dw-sized scratch, unless the update rides on the second
+// pass of a split reduction (tensor path, more than one pixel split), which never forms dw.
+bool sgd_rides_on_reduction(const pcl_conv_desc& d, int P, int Q) {
+    const WgradPlan pl = plan_wgrad(d, P, Q);
+    return pl.tensor && !pl.few;      // (more than one pixel split: the second pass; one: the kernel's epilogue)
+}
+int conv_bwd_weights_impl(const pcl_conv_desc* d, const float* x, const float* dy, float* dw, float* dbias, int deterministic,
+                          void* ws, size_t ws_bytes, void* cuda_stream, float* w_update, float lr);
+}  // namespace
+
 int pcl_conv_bwd_weights(const pcl_conv_desc* d, const float* x, const float* dy, float* dw, float* dbias,
                          int deterministic, void* ws, size_t ws_bytes, void* cuda_stream) {
+    return conv_bwd_weights_impl(d, x, dy, dw, dbias, deterministic, ws, ws_bytes, cuda_stream, nullptr, 0.f);
+}
+
+size_t pcl_conv_bwd_weights_sgd_workspace_bytes(const pcl_conv_desc* d) {
+    int P, Q;
+    if (check_desc(d, &P, &Q) != PCL_OK) return 0;
+    const size_t base = align_up(pcl_conv_workspace_bytes(d, PCL_PASS_BWD_WEIGHTS), 256);
+    return sgd_rides_on_reduction(*d, P, Q) ? base : base + align_up(dw_bytes(*d), 256);
+}
+
+int pcl_conv_bwd_weights_sgd(const pcl_conv_desc* d, const float* x, const float* dy, float* w, float lr, float* dbias,
+                             void* ws, size_t ws_bytes, void* cuda_stream) {
+    int P, Q;
+    int rc = check_desc(d, &P, &Q);
+    if (rc != PCL_OK) return rc;
+    if (!w) return PCL_ERR_BAD_ARG;
+    if (!aligned16(w)) return PCL_ERR_MISALIGNED;
+    const size_t need = pcl_conv_bwd_weights_sgd_workspace_bytes(d);
+    if (need > 0) {
+        if (!ws || ws_bytes < need) return PCL_ERR_WORKSPACE;
+        if (reinterpret_cast<uintptr_t>(ws) & 255) return PCL_ERR_MISALIGNED;
+    }
+    if (sgd_rides_on_reduction(*d, P, Q))
+        return conv_bwd_weights_impl(d, x, dy, w /* unused as dw */, dbias, 1, ws, ws_bytes, cuda_stream, w, lr);
+    // no split reduction to ride on: dw goes to the scratch behind the plain form's workspace, then the update
+    const size_t base = align_up(pcl_conv_workspace_bytes(d, PCL_PASS_BWD_WEIGHTS), 256);
+    float* dw = reinterpret_cast<float*>(static_cast<char*>(ws) + base);
+    rc = conv_bwd_weights_impl(d, x, dy, dw, dbias, 1, ws, base, cuda_stream, nullptr, 0.f);
+    if (rc != PCL_OK) return rc;
+    return launch_sgd(w, dw, size_t(d->K) * d->R * d->S * d->C, lr, static_cast<cudaStream_t>(cuda_stream));
+}
+
+namespace {
+int conv_bwd_weights_impl(const pcl_conv_desc* d, const float* x, const float* dy, float* dw, float* dbias, int deterministic,
+                          void* ws, size_t ws_bytes, void* cuda_stream, float* w_update, float lr) {
     int P, Q;
     int rc = check_desc(d, &P, &Q);
     if (rc != PCL_OK) return rc;
@@ -929,14 +975,24 @@ int pcl_conv_bwd_weights(const pcl_conv_desc* d, const float* x, const float* dy
     if (pl.tensor) {
         TcWgradArgs a{x, dy, dw, partial, d->N, d->H, d->W, d->C, d->K, d->R, d->S, d->pad_h, d->pad_w, P, Q, pl.splits};
         a.stride_h = d->stride_h; a.stride_w = d->stride_w;
+        if (w_update && pl.splits > 1) {      // the second pass of the split reduction applies the update
+            if (!partial) return PCL_ERR_BAD_ARG;
+            a.skip_reduce = 1;
+        } else if (w_update) {                // unsplit: the kernel's epilogue does
+            a.w_update = w_update; a.lr = lr;
+        }
         rc = launch_tc_wgrad(a, st);
+        if (rc == PCL_OK && w_update && pl.splits > 1)
+            rc = launch_reduce_splits_sgd(partial, w_update, size_t(d->K) * d->R * d->S * d->C, pl.splits, lr, st);
     } else {
+        if (w_update) return PCL_ERR_BAD_ARG;
         rc = launch_generic_bwd_weights(*d, P, Q, x, dy, dw, partial, pl.splits, st);
     }
     if (rc != PCL_OK) return rc;
     if (dbias) rc = launch_colsum(dy, size_t(d->N) * P * Q, d->K, cs_partial, dbias, st);
     return rc;
 }
+}  // namespace
 
 int pcl_fc_fwd(int N, int C, int K, const float* x, const float* w, const float* bias, float* y, int act, void* ws,
                size_t ws_bytes, void* cuda_stream) {
@@ -948,9 +1004,13 @@ int pcl_fc_fwd(int N, int C, int K, const float* x, const float* w, const float*
 namespace {
 bool known_act(int act) { return act == PCL_ACT_NONE || act == PCL_ACT_RELU || act == PCL_ACT_SIGMOID; }
 
+// w_update (with lr): the layer's weights are updated in place, w <- w - lr * dw, and dw is not stored (`dw` is ignored);
+// backpropagation, which reads the old weights, then runs first.
 int fc_bwd_impl(int N, int C, int K, const float* x, const float* w, const float* y, int act, float* dy, float* dx,
-                int x_act, float* dx_colsum, float* dw, float* dbias, void* ws, size_t ws_bytes, void* cuda_stream) {
+                int x_act, float* dx_colsum, float* dw, float* dbias, void* ws, size_t ws_bytes, void* cuda_stream,
+                float* w_update = nullptr, float lr = 0.f) {
     if (N <= 0 || C <= 0 || K <= 0) return PCL_ERR_BAD_ARG;
+    if (w_update) dw = w_update;      // (only its alignment is looked at below)
     if (!x || !w || !dy || !dw) return PCL_ERR_BAD_ARG;
     if (!known_act(act) || !known_act(x_act)) return PCL_ERR_BAD_ARG;
     if (act != PCL_ACT_NONE && !y) return PCL_ERR_BAD_ARG;
@@ -962,7 +1022,9 @@ int fc_bwd_impl(int N, int C, int K, const float* x, const float* w, const float
     const bool dw_fwd = fc_dw_as_forward(N, C, K);
     PassScope pass_scope(PROF_PASS_FC_BWD, 2.0 * N * double(C) * K, dx ? 2 : 1);
     const size_t colsum_bytes = plan_wgrad(d, 1, 1).colsum_bytes;
-    const size_t need_w = dw_fwd ? fc_dzt_bytes(N, K) + colsum_bytes : pcl_conv_workspace_bytes(&d, PCL_PASS_BWD_WEIGHTS);
+    const size_t need_w = dw_fwd ? fc_dzt_bytes(N, K) + colsum_bytes
+                                 : (w_update ? pcl_conv_bwd_weights_sgd_workspace_bytes(&d)
+                                             : pcl_conv_workspace_bytes(&d, PCL_PASS_BWD_WEIGHTS));
     const bool fused_dx = dx && (x_act != PCL_ACT_NONE || dx_colsum);
     const size_t need_d = !dx ? 0 : (dx_colsum ? pcl_conv_bwd_data_colsum_workspace_bytes(&d)
                                                : pcl_conv_workspace_bytes(&d, PCL_PASS_BWD_DATA));
@@ -973,6 +1035,18 @@ int fc_bwd_impl(int N, int C, int K, const float* x, const float* w, const float
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
     int rc = launch_act_grad(dy, y, size_t(N) * K, act, st);
     if (rc != PCL_OK) return rc;
+    char* ws_d = static_cast<char*>(ws) + need_w;
+    auto backprop = [&]() -> int {
+        if (!dx) return PCL_OK;
+        if (!fused_dx) return pcl_conv_bwd_data(&d, dy, w, nullptr, dx, ws_d, need_d, cuda_stream);
+        // dx = (dz w) times the gradient of the activation that produced x: what the layer below needs as its dz
+        return bwd_data_masked_colsum(&d, 1, 1, dy, w, x_act == PCL_ACT_NONE ? nullptr : x, x_act == PCL_ACT_SIGMOID ? 1 : 0, dx,
+                                      dx_colsum, ws_d, need_d, cuda_stream);
+    };
+    if (w_update) {       // in-place update: the old weights are read first
+        rc = backprop();
+        if (rc != PCL_OK) return rc;
+    }
     // weight gradient first, then backpropagation (the order Sec. 3.1 schedules them in)
     if (dw_fwd) {
         float* dzt = static_cast<float*>(ws);
@@ -981,18 +1055,16 @@ int fc_bwd_impl(int N, int C, int K, const float* x, const float* w, const float
         if (rc != PCL_OK) return rc;
         TcFpropArgs a{dzt, x, nullptr, nullptr, dw, K, 1, 1, N, C, 1, 1, 0, 0, 1, 1, PCL_ACT_NONE};
         a.wt_mn_major = 1;
+        if (w_update) { a.mask_src = w_update; a.mask_mode = 2; a.lr = lr; a.out = w_update; }     // w - lr * dw, in place
         rc = launch_tc_fprop(a, st);
         if (rc == PCL_OK && dbias) rc = launch_colsum(dy, size_t(N), K, cs, dbias, st);
+    } else if (w_update) {
+        rc = pcl_conv_bwd_weights_sgd(&d, x, dy, w_update, lr, dbias, ws, need_w, cuda_stream);
     } else {
         rc = pcl_conv_bwd_weights(&d, x, dy, dw, dbias, 1, ws, need_w, cuda_stream);
     }
     if (rc != PCL_OK) return rc;
-    if (!dx) return PCL_OK;
-    char* ws_d = static_cast<char*>(ws) + need_w;
-    if (!fused_dx) return pcl_conv_bwd_data(&d, dy, w, nullptr, dx, ws_d, need_d, cuda_stream);
-    // dx = (dz w) times the gradient of the activation that produced x: what the layer below needs as its dz
-    return bwd_data_masked_colsum(&d, 1, 1, dy, w, x_act == PCL_ACT_NONE ? nullptr : x, x_act == PCL_ACT_SIGMOID ? 1 : 0, dx,
-                                  dx_colsum, ws_d, need_d, cuda_stream);
+    return w_update ? PCL_OK : backprop();
 }
 }  // namespace
 
@@ -1005,6 +1077,22 @@ int pcl_fc_bwd_fused(int N, int C, int K, const float* x, const float* w, const 
                      int x_act, float* dx_colsum, float* dw, float* dbias, void* ws, size_t ws_bytes,
                      void* cuda_stream) {
     return fc_bwd_impl(N, C, K, x, w, y, act, dy, dx, x_act, dx_colsum, dw, dbias, ws, ws_bytes, cuda_stream);
+}
+
+int pcl_fc_bwd_fused_sgd(int N, int C, int K, const float* x, float* w, const float* y, int act, float* dy, float* dx,
+                         int x_act, float* dx_colsum, float lr, float* dbias, void* ws, size_t ws_bytes,
+                         void* cuda_stream) {
+    if (!w) return PCL_ERR_BAD_ARG;
+    return fc_bwd_impl(N, C, K, x, w, y, act, dy, dx, x_act, dx_colsum, nullptr, dbias, ws, ws_bytes, cuda_stream, w, lr);
+}
+
+size_t pcl_fc_bwd_fused_sgd_workspace_bytes(int N, int C, int K) {
+    if (N <= 0 || C <= 0 || K <= 0) return 0;
+    const pcl_conv_desc d{N, C, K, 1, 1, 1, 1, 1, 1, 0, 0};
+    // (sized for either form of the weight-gradient part, like pcl_fc_workspace_bytes)
+    const size_t wgrad_form = pcl_conv_bwd_weights_sgd_workspace_bytes(&d);
+    const size_t fwd_form = fc_dzt_bytes(N, K) + plan_wgrad(d, 1, 1).colsum_bytes;
+    return pcl_conv_bwd_data_colsum_workspace_bytes(&d) + align_up(wgrad_form > fwd_form ? wgrad_form : fwd_form, 256);
 }
 
 int pcl_sgd_update(float* w, const float* dw, size_t n, float lr, void* cuda_stream) {

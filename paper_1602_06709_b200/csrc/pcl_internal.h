@@ -128,6 +128,7 @@ struct TcFpropArgs {
     // What mask_src does: 0 = the output is zeroed where mask_src <= 0 (gradient of the ReLU that produced mask_src);
     // 1 = the output is multiplied by mask_src * (1 - mask_src) (gradient of the sigmoid that produced mask_src).
     int mask_mode = 0;
+    float lr = 0.f;         // mask_mode 2: out = mask_src - lr * (the contraction); out may be mask_src itself (SGD in place)
     // k_live (0 = all): how many leading elements of every 32-element channel block can be non-zero in `wt` (the
     // few-channel path packs S taps x 4 channels into a block and zero-fills the rest): MMAs over all-zero K = 8
     // slices are skipped.
@@ -205,6 +206,9 @@ struct TcWgradArgs {
     int relu_mask = 0;
     float* db_rows = nullptr;
     int stride_h = 1, stride_w = 1, dil_w = 1;      // as in TcFpropArgs
+    // unsplit launches (splits == 1): instead of storing dw the epilogue writes w_update[i] - lr * dw[i] in place
+    float* w_update = nullptr;
+    float lr = 0.f;
 };
 bool tc_wgrad_eligible(const TcWgradArgs& a);
 constexpr int kPooledDbRows = 16;       // bias-gradient rows per pixel split that a pooled-dy launch writes
@@ -225,6 +229,7 @@ int launch_generic_bwd_weights(const pcl_conv_desc& d, int P, int Q, const float
 // ---- HBM-bound helpers ------------------------------------------------------
 int launch_sgd(float* w, const float* dw, size_t n, float lr, cudaStream_t st);
 int launch_reduce_splits(const float* partial, float* out, size_t n, int splits, cudaStream_t st);
+int launch_reduce_splits_sgd(const float* partial, float* w, size_t n, int splits, float lr, cudaStream_t st);
 // out[r][k] = act(bias[k] + sum_s partial[s][r][k]), splits added in index order; K % 4 == 0
 int launch_reduce_splits_bias_act(const float* partial, float* out, const float* bias, int act, size_t rows, int K,
                                   int splits, cudaStream_t st);

@@ -83,7 +83,9 @@ struct FpropParams {
     const float* bias;
     const float* mask_src;
     int mask_mode;              // what mask_src does to the output: 0 zero where mask_src <= 0 (ReLU gradient),
-                                // 1 multiply by mask_src * (1 - mask_src) (sigmoid gradient, mask_src being the sigmoid's output)
+                                // 1 multiply by mask_src * (1 - mask_src) (sigmoid gradient, mask_src being the sigmoid's output),
+                                // 2 out = mask_src - lr * output (the SGD update of a weight gradient; out may be mask_src)
+    float lr;
     float* out;
     int tma_store;              // the epilogue writes `out` with TMA stores from the staging tiles (tmOut is valid)
     // Split reduction (few tiles, long reduction: the FC layers at small minibatch): ksplit > 1 cuts the k-steps of
@@ -954,9 +956,9 @@ tc_fprop_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                         if (kMask) {
 #pragma unroll
                             for (int i = 0; i < 8; ++i)
-                                mk[i] = ((vmask >> i) & 1u)
-                                            ? __ldg(reinterpret_cast<const float4*>(p.mask_src + roff[i] + col))
-                                            : make_float4(0.f, 0.f, 0.f, 0.f);
+                                mk[i] = !((vmask >> i) & 1u) ? make_float4(0.f, 0.f, 0.f, 0.f)
+                                        : p.mask_mode == 2 ? *reinterpret_cast<const float4*>(p.mask_src + roff[i] + col)   // (may be `out`)
+                                                           : __ldg(reinterpret_cast<const float4*>(p.mask_src + roff[i] + col));
                         }
 #pragma unroll
                         for (int i = 0; i < 8; ++i) {
@@ -974,6 +976,9 @@ tc_fprop_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                                     if (p.mask_mode == 0) {
                                         o.x = mk[i].x > 0.f ? o.x : 0.f; o.y = mk[i].y > 0.f ? o.y : 0.f;
                                         o.z = mk[i].z > 0.f ? o.z : 0.f; o.w = mk[i].w > 0.f ? o.w : 0.f;
+                                    } else if (p.mask_mode == 2) {
+                                        o.x = fmaf(-p.lr, o.x, mk[i].x); o.y = fmaf(-p.lr, o.y, mk[i].y);
+                                        o.z = fmaf(-p.lr, o.z, mk[i].z); o.w = fmaf(-p.lr, o.w, mk[i].w);
                                     } else {
                                         o.x *= mk[i].x * (1.f - mk[i].x); o.y *= mk[i].y * (1.f - mk[i].y);
                                         o.z *= mk[i].z * (1.f - mk[i].z); o.w *= mk[i].w * (1.f - mk[i].w);
@@ -1049,8 +1054,8 @@ tc_fprop_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                                 if (p.act == PCL_ACT_RELU) o = fmaxf(o, 0.f);
                                 else if (p.act == PCL_ACT_SIGMOID) o = sigmoid_fast(o);
                                 if (msk) {
-                                    const float m = __ldg(msk + j);
-                                    o = p.mask_mode == 0 ? (m > 0.f ? o : 0.f) : o * (m * (1.f - m));
+                                    const float m = p.mask_mode == 2 ? msk[j] : __ldg(msk + j);
+                                    o = p.mask_mode == 0 ? (m > 0.f ? o : 0.f) : (p.mask_mode == 2 ? fmaf(-p.lr, o, m) : o * (m * (1.f - m)));
                                 }
                                 dst[j] = o;
                             }
@@ -1484,7 +1489,7 @@ int launch_tc_fprop(const TcFpropArgs& a, cudaStream_t st) {
     p.tmem_cols = 32;
     while (p.tmem_cols < (p.split_acc ? 4 : 2) * p.MT * p.BN) p.tmem_cols *= 2;
     p.bias = a.bias; p.mask_src = a.mask_src; p.out = a.out;
-    p.mask_mode = a.mask_mode;
+    p.mask_mode = a.mask_mode; p.lr = a.lr;
     // split reduction: raw partial tiles to the caller's scratch, bias and activation after the splits are added
     p.ksplit = 1; p.kps = 0; p.split_stride = 0;
     if (a.split_ws) {

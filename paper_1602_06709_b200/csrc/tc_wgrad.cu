@@ -99,6 +99,8 @@ struct WgradParams {
     // belongs to the same thread), each into an accumulator of its own, acc_cols columns apart; the epilogue adds
     // the two in a fixed order.  What bounds a single-CTA item is the issuing thread (~100-140 cycles per MMA,
     // whatever its width), not the tensor pipe.
+    int sgd;                  // unsplit launch: the epilogue writes out[i] - lr * (the tile) instead of the tile (out = the weights)
+    float lr;
     int duo, acc_cols;
     int dy_groups;            // 32-map groups of a k-step's dy tile (4, fewer for pooled dy with K < 128)
     int inject_short_copy;    // test mode: the first slot is armed for 16 bytes more than are copied (see the forward kernel)
@@ -536,6 +538,18 @@ tc_wgrad_kernel(const __grid_constant__ CUtensorMap tmDy, const __grid_constant_
                     tap = run / p.runs_per_tap;
                     c0 = ((run - tap * p.runs_per_tap) * p.L + ch % p.L) * 32;
                 }
+                // (in-place update: the old weights of the chunk are fetched before the accumulator is read and staged, so
+                // that their latency does not fall between the stores)
+                const bool sgd = !kWide && p.sgd;      // (pooled-dy launches always have a second pass)
+                float4 wv[8];
+                if (sgd && vec_ok && c0 + cg < p.C) {
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) {
+                        const int kk = kt * 128 + quarter * 32 + (lane >> 3) + 4 * i;
+                        wv[i] = kk < p.K ? *reinterpret_cast<const float4*>(p.out + (static_cast<size_t>(kk) * p.R * p.S + tap) * p.C + c0 + cg)
+                                         : make_float4(0.f, 0.f, 0.f, 0.f);
+                    }
+                }
                 uint32_t v[32];
                 if (kiters > 0) {
                     tmem_ld_32x32(t_row + ch * 32, v);
@@ -568,6 +582,9 @@ tc_wgrad_kernel(const __grid_constant__ CUtensorMap tmDy, const __grid_constant_
                                              (static_cast<size_t>(kk) * p.R * p.S + tap) * p.C + c0 + cg;
                                 if (p.use_atomics) {
                                     atomicAdd(dst, o.x); atomicAdd(dst + 1, o.y); atomicAdd(dst + 2, o.z); atomicAdd(dst + 3, o.w);
+                                } else if (sgd) {
+                                    *reinterpret_cast<float4*>(dst) = make_float4(fmaf(-p.lr, o.x, wv[i].x), fmaf(-p.lr, o.y, wv[i].y),
+                                                                                  fmaf(-p.lr, o.z, wv[i].z), fmaf(-p.lr, o.w, wv[i].w));
                                 } else {
                                     *reinterpret_cast<float4*>(dst) = o;
                                 }
@@ -584,7 +601,7 @@ tc_wgrad_kernel(const __grid_constant__ CUtensorMap tmDy, const __grid_constant_
                     } else {
 #pragma unroll
                         for (int j = 0; j < 32; ++j)
-                            if (c0 + j < p.C) dst[j] = __uint_as_float(v[j]);
+                            if (c0 + j < p.C) dst[j] = sgd ? fmaf(-p.lr, __uint_as_float(v[j]), dst[j]) : __uint_as_float(v[j]);
                     }
                 }
             }
@@ -788,8 +805,10 @@ int launch_tc_wgrad(const TcWgradArgs& a, cudaStream_t st) {
     if (!p.status) return PCL_ERR_CUDA;
     p.inject_short_copy = (tune(TUNE_FAULT_INJECT, 0) == 2 && !rp.pair && !pooled) ? 1 : 0;      // test mode
     const size_t dw_elems = size_t(a.K) * a.R * a.S * a.C;
+    if (a.w_update && p.splits != 1) return PCL_ERR_BAD_ARG;      // (a split reduction updates in its second pass)
     if (p.splits == 1) {
-        p.out = a.dw; p.split_stride = 0; p.use_atomics = 0;
+        p.out = a.w_update ? a.w_update : a.dw; p.split_stride = 0; p.use_atomics = 0;
+        p.sgd = a.w_update ? 1 : 0; p.lr = a.lr;
     } else if (a.partial) {
         p.out = a.partial; p.split_stride = dw_elems; p.use_atomics = 0;
     } else {

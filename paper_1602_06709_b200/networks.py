@@ -26,14 +26,22 @@ def _align(n: int, a: int = 64) -> int:
 class _ParamStore:
     """Flat fp32 parameter and gradient buffers with 256-byte aligned views."""
 
-    def __init__(self, shapes: List[tuple], device="cuda"):
-        self.offsets = []
+    def __init__(self, shapes: List[tuple], device="cuda", tail=()):
+        """tail: indices of the tensors laid out behind all others (the fused-update steps keep there what still takes
+        the plain SGD launch: the biases and the first layer's few weights), in index order."""
+        self.offsets = [0] * len(shapes)
         off = 0
-        for shp in shapes:
-            self.offsets.append(off)
-            off += _align(int(np.prod(shp)))
+        tail = sorted(set(tail))
+        for i in [i for i in range(len(shapes)) if i not in tail] + tail:
+            if tail and i == tail[0]:
+                self.tail_offset = off
+            self.offsets[i] = off
+            off += _align(int(np.prod(shapes[i])))
+        if not tail:
+            self.tail_offset = off
         self.total = off
         self.shapes = shapes
+        self.in_order = not tail
         self.params = torch.zeros(off, device=device)
         self.grads = torch.zeros(off, device=device)
 
@@ -53,6 +61,7 @@ class _ParamStore:
     def layer_buckets(self):
         """(offset, length) of every (weights, bias) pair: the unit of the data-parallel gradient exchange.  Every
         tensor starts on a 64-element boundary, so a bucket divides into 2, 4, 8 or 16 equal 16-byte aligned strips."""
+        assert self.in_order, "the gradient exchange needs the (weights, bias) pairs side by side"
         out = []
         for i in range(0, len(self.shapes), 2):
             end = self.offsets[i + 2] if i + 2 < len(self.shapes) else self.total
@@ -147,10 +156,15 @@ class VggA(_HostFeed):
     FC 25088-4096-4096-1000 and softmax cross-entropy."""
 
     def __init__(self, N: int, hw: int = inputs.VGGA_HW, conv=None, fc=None, classes: int = inputs.VGGA_CLASSES,
-                 lr: float = 0.01, cfg: str = "cfg5", keep_unpooled: bool = False):
+                 lr: float = 0.01, cfg: str = "cfg5", keep_unpooled: bool = False, fused_update: bool = False):
         """keep_unpooled: also store the full-resolution output of the pooled layers (self.y[i]).  The step never
         reads it (pooling backward and the ReLU mask go by the position codes), so by default it is neither
         allocated nor written where the convolution and the pooling run as one kernel."""
+        # fused_update: every layer's weights but the first's are updated by the second pass (or epilogue) of their own
+        # weight-gradient call (Sec. 3.1), after the layer's backpropagation has read the old ones; their gradients are
+        # never stored, and update() is one small SGD launch over the biases and the first layer's weights.  Not for the
+        # data-parallel step, which exchanges the gradients.
+        self.fused_update = fused_update
         self.N, self.lr, self.classes = N, lr, classes
         conv = conv if conv is not None else inputs.VGGA_CONV
         self.convs: List[_ConvLayer] = []
@@ -171,7 +185,7 @@ class VggA(_HostFeed):
             shapes += [(L.K, 3, 3, L.C), (L.K,)]
         for C, K in fc:
             shapes += [(K, C), (K,)]
-        self.store = _ParamStore(shapes)
+        self.store = _ParamStore(shapes, tail=([0] + list(range(1, len(shapes), 2))) if fused_update else ())
         nconv = len(self.convs)
         for i, L in enumerate(self.convs):
             w = inputs.he_normal_conv(inputs.tensor_id(cfg, L.name, "w"), L.K, 3, 3, L.C)
@@ -209,6 +223,9 @@ class VggA(_HostFeed):
                      B.maxpool2x2_bwd_colsum_workspace_bytes(N, L.H, L.W, L.K))
         for C, K in fc:
             ws = max(ws, B.fc_workspace_bytes(N, C, K, B.PASS_BWD_DATA), B.fc_workspace_bytes(N, C, K, B.PASS_FWD))
+        if fused_update:
+            ws = max([ws] + [B.conv_bwd_weights_sgd_workspace_bytes(L.desc) for L in self.convs[1:]] +
+                     [B.fc_bwd_fused_sgd_workspace_bytes(N, C, K) for C, K in fc])
         self.ws = torch.empty(max(ws, 256), dtype=torch.uint8, device=dev)
         # The first layer's forward call stages its few-channel input at the start of its workspace; with a workspace
         # of its own, kept until the backward pass, its weight gradient reads that copy instead of staging x again.
@@ -270,9 +287,14 @@ class VggA(_HostFeed):
             dx = self.fc_dout[j - 1] if j > 0 else self.dpooled[-1].view(self.N, self.flat)
             # fc_dout[j] already is dz_j: the softmax gradient for the last layer, and for the others the layer above
             # folded this layer's ReLU gradient and bias gradient into its backpropagation kernel
-            B.fc_bwd_fused(self.N, C, K, a, self.fc_w(j), None, B.ACT_NONE, self.fc_dout[j], dx,
-                           B.ACT_RELU if j > 0 else B.ACT_NONE, self.fc_db(j - 1) if j > 0 else None, self.fc_dw(j),
-                           self.fc_db(j) if j + 1 == nfc else None, self.ws)
+            if self.fused_update:
+                B.fc_bwd_fused_sgd(self.N, C, K, a, self.fc_w(j), None, B.ACT_NONE, self.fc_dout[j], dx,
+                                   B.ACT_RELU if j > 0 else B.ACT_NONE, self.fc_db(j - 1) if j > 0 else None, self.lr,
+                                   self.fc_db(j) if j + 1 == nfc else None, self.ws)
+            else:
+                B.fc_bwd_fused(self.N, C, K, a, self.fc_w(j), None, B.ACT_NONE, self.fc_dout[j], dx,
+                               B.ACT_RELU if j > 0 else B.ACT_NONE, self.fc_db(j - 1) if j > 0 else None, self.fc_dw(j),
+                               self.fc_db(j) if j + 1 == nfc else None, self.ws)
             if after_layer:
                 after_layer(len(self.convs) + j)
             if after_backprop:
@@ -297,9 +319,10 @@ class VggA(_HostFeed):
             if L.pool:   # gradient through the pool, then through the ReLU (fused mask), routed by the position codes
                 B.maxpool2x2_bwd_codes(self.N, L.H, L.W, L.K, self.pool_codes[i], self.dpooled[i], True, self.dy[i],
                                        self.conv_db(i), self.ws)
-            B.conv_bwd_weights(L.desc, self.layer_input(i), self.dy[i], self.conv_dw(i), None, True, self.ws)
-            if after_layer:
-                after_layer(i)
+            if not self.fused_update:      # (Sec. 3.1: the weight gradient first, so that its exchange can start)
+                B.conv_bwd_weights(L.desc, self.layer_input(i), self.dy[i], self.conv_dw(i), None, True, self.ws)
+                if after_layer:
+                    after_layer(i)
             if i > 0:
                 prev = self.convs[i - 1]
                 if prev.pool:
@@ -307,11 +330,19 @@ class VggA(_HostFeed):
                 else:   # the layer's input is the previous ReLU output: fuse its mask (and its bias gradient)
                     B.conv_bwd_data_colsum(L.desc, self.dy[i], self.conv_w(i), self.y[i - 1], self.dy[i - 1],
                                            self.conv_db(i - 1), self.ws)
+            if self.fused_update:          # the old weights have been read: gradient and update in one call
+                if i > 0:
+                    B.conv_bwd_weights_sgd(L.desc, self.layer_input(i), self.dy[i], self.conv_w(i), self.lr, None, self.ws)
+                else:
+                    B.conv_bwd_weights(L.desc, self.layer_input(i), self.dy[i], self.conv_dw(i), None, True, self.ws)
+                if after_layer:
+                    after_layer(i)
             if after_backprop:
                 after_backprop(i)
 
     def update(self):
-        B.sgd_update(self.store.params, self.store.grads, self.lr)
+        t = self.store.tail_offset if self.fused_update else 0
+        B.sgd_update(self.store.params[t:], self.store.grads[t:], self.lr)
 
     def step(self):
         self.forward()
@@ -324,14 +355,15 @@ class Dnn(_HostFeed):
     """Fully-connected DNN: dims[0] inputs, sigmoid hidden layers, linear output
     layer with softmax cross-entropy (the 7-layer ASR network shape of Sec. 5.4)."""
 
-    def __init__(self, N: int, dims=None, lr: float = 0.01, cfg: str = "cfg4"):
+    def __init__(self, N: int, dims=None, lr: float = 0.01, cfg: str = "cfg4", fused_update: bool = False):
         dims = dims if dims is not None else inputs.CFG4_DIMS
         self.N, self.dims, self.lr = N, dims, lr
+        self.fused_update = fused_update      # (as in VggA: weights updated by their own weight-gradient call)
         self.layers = list(zip(dims[:-1], dims[1:]))
         shapes = []
         for C, K in self.layers:
             shapes += [(K, C), (K,)]
-        self.store = _ParamStore(shapes)
+        self.store = _ParamStore(shapes, tail=list(range(1, len(shapes), 2)) if fused_update else ())
         for j, (C, K) in enumerate(self.layers):
             w = inputs.xavier_uniform_fc(inputs.tensor_id(cfg, f"fc{j + 1}", "w"), K, C)
             self.store.p(2 * j).copy_(torch.from_numpy(w))
@@ -344,6 +376,8 @@ class Dnn(_HostFeed):
         self.loss = torch.zeros(1, device=dev)
         ws = max(max(B.fc_workspace_bytes(N, C, K, B.PASS_BWD_DATA), B.fc_workspace_bytes(N, C, K, B.PASS_FWD))
                  for C, K in self.layers)
+        if fused_update:
+            ws = max([ws] + [B.fc_bwd_fused_sgd_workspace_bytes(N, C, K) for C, K in self.layers])
         self.ws = torch.empty(max(ws, 256), dtype=torch.uint8, device=dev)
         self.fc_flops_fwd = [2 * N * C * K for C, K in self.layers]
 
@@ -373,16 +407,22 @@ class Dnn(_HostFeed):
             a = self.out[j - 1] if j > 0 else self.x
             dx = self.dout[j - 1] if j > 0 else None          # first layer: no backpropagation
             # dout[j] already is dz_j (the softmax gradient, or formed by the layer above together with db_j)
-            B.fc_bwd_fused(self.N, C, K, a, self.w(j), None, B.ACT_NONE, self.dout[j], dx,
-                           B.ACT_SIGMOID if j > 0 else B.ACT_NONE, self.db(j - 1) if j > 0 else None, self.dw(j),
-                           self.db(j) if j + 1 == n else None, self.ws)
+            if self.fused_update:
+                B.fc_bwd_fused_sgd(self.N, C, K, a, self.w(j), None, B.ACT_NONE, self.dout[j], dx,
+                                   B.ACT_SIGMOID if j > 0 else B.ACT_NONE, self.db(j - 1) if j > 0 else None, self.lr,
+                                   self.db(j) if j + 1 == n else None, self.ws)
+            else:
+                B.fc_bwd_fused(self.N, C, K, a, self.w(j), None, B.ACT_NONE, self.dout[j], dx,
+                               B.ACT_SIGMOID if j > 0 else B.ACT_NONE, self.db(j - 1) if j > 0 else None, self.dw(j),
+                               self.db(j) if j + 1 == n else None, self.ws)
             if after_layer:
                 after_layer(j)
             if after_backprop:
                 after_backprop(j)
 
     def update(self):
-        B.sgd_update(self.store.params, self.store.grads, self.lr)
+        t = self.store.tail_offset if self.fused_update else 0
+        B.sgd_update(self.store.params[t:], self.store.grads[t:], self.lr)
 
     def step(self):
         self.forward()

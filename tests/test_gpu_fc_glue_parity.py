@@ -416,3 +416,74 @@ def test_maxpool_with_position_codes(N, H, W, C):
     cs_x = torch.empty_like(cs)
     B.maxpool2x2_bwd_colsum(N, H, W, C, xt, dyt, xt, dxt, cs_x, ws)
     assert torch.equal(cs, cs_x)
+
+
+# ---- the SGD step applied by the weight gradient's own second pass / epilogue (Sec. 3.1) -----------------------------
+SGD_CONV_SHAPES = [
+    # N, C, K, H, W, R: a split pixel reduction (the update rides on its second pass); a reduction too short to split
+    # (dw goes through the scratch); the few-channel staged path; a strided layer
+    (8, 64, 96, 28, 28, 3), (2, 32, 32, 6, 6, 3), (4, 3, 16, 20, 20, 3), (4, 16, 24, 19, 19, 5),
+]
+
+
+@pytest.mark.parametrize("N,C,K,H,W,R", SGD_CONV_SHAPES)
+def test_conv_bwd_weights_sgd_equals_gradient_then_update(N, C, K, H, W, R):
+    """pcl_conv_bwd_weights_sgd: w - lr * dw with dw never stored must equal, bit for bit, the deterministic weight
+    gradient followed by pcl_sgd_update, and agree with the oracle's gradient and update."""
+    import gpu_helpers as G
+    from oracle import ConvShape
+    from paper_1602_06709_b200 import binding as B
+    stride = 2 if R == 5 else 1
+    s = ConvShape(N=N, C=C, K=K, H=H, W=W, R=R, S=R, pad_h=R // 2, pad_w=R // 2, stride_h=stride, stride_w=stride)
+    x, w, dy, _ = G.make_inputs(s, f"wsgd{C}_{K}")
+    d = G.shape_to_desc(s)
+    lr = 0.0625
+    xt, dyt = G.dev(x), G.dev(dy)
+    w_two = G.dev(w).clone(); dw = G.guarded(w.shape); db = G.guarded((K,))
+    ws = G.workspace(B.conv_workspace_bytes(d, B.PASS_BWD_WEIGHTS))
+    B.conv_bwd_weights(d, xt, dyt, dw, db, True, ws)
+    B.sgd_update(w_two, dw, lr)
+    w_one = G.guarded(w.shape); w_one.copy_(G.dev(w)); db2 = G.guarded((K,))
+    ws2 = G.workspace(B.conv_bwd_weights_sgd_workspace_bytes(d))
+    B.conv_bwd_weights_sgd(d, xt, dyt, w_one, lr, db2, ws2)
+    B.check_device_status()
+    G.check_guards()
+    assert torch.equal(w_one, w_two), "fused update differs from gradient + update"
+    assert torch.equal(db, db2)
+    dw_ref = oracle.conv_bwd_weights(s, x, dy)
+    G.assert_parity((G.dev(w) - w_one).cpu().numpy() / lr, dw_ref, "(w_old - w_new) / lr against the oracle's dw")
+
+
+@pytest.mark.parametrize("N,C,K", [(64, 4096, 2048), (256, 512, 384), (96, 440, 2048), (1024, 256, 256)])
+@pytest.mark.parametrize("x_act", ["none", "sigmoid"])
+def test_fc_bwd_fused_sgd_equals_backward_then_update(N, C, K, x_act):
+    """pcl_fc_bwd_fused_sgd (both forms of the FC weight gradient: the forward-type GEMM whose epilogue applies the
+    update, and the weight-gradient kernel with the update in its second pass or after its scratch): dx, column sums and
+    bias gradient as pcl_fc_bwd_fused on the OLD weights, the new weights bit-equal to the two-call form."""
+    import gpu_helpers as G
+    from paper_1602_06709_b200 import binding as B
+    from paper_1602_06709_b200 import inputs
+    code = {"none": B.ACT_NONE, "sigmoid": B.ACT_SIGMOID}[x_act]
+    pre = inputs.normal(inputs.tensor_id("fcsgd", N, C, K, "pre"), (N, C), 1.0).astype(np.float64)
+    x = {"none": pre, "sigmoid": 1.0 / (1.0 + np.exp(-pre))}[x_act].astype(np.float32)
+    w = inputs.normal(inputs.tensor_id("fcsgd", N, C, K, "w"), (K, C), (1.0 / C) ** 0.5)
+    dz = inputs.normal(inputs.tensor_id("fcsgd", N, C, K, "dz"), (N, K), 1.0)
+    lr = 0.03125
+    xt = G.dev(x)
+    # two calls
+    w_two = G.dev(w).clone()
+    dx = G.guarded((N, C)); dw = G.guarded((K, C)); db = G.guarded((K,)); cs = G.guarded((C,))
+    ws = G.workspace(B.fc_workspace_bytes(N, C, K, B.PASS_BWD_DATA))
+    B.fc_bwd_fused(N, C, K, xt, w_two, None, B.ACT_NONE, G.dev(dz), dx, code, cs, dw, db, ws)
+    B.sgd_update(w_two, dw, lr)
+    # one call
+    w_one = G.guarded((K, C)); w_one.copy_(G.dev(w))
+    dx1 = G.guarded((N, C)); db1 = G.guarded((K,)); cs1 = G.guarded((C,))
+    ws1 = G.workspace(B.fc_bwd_fused_sgd_workspace_bytes(N, C, K))
+    B.fc_bwd_fused_sgd(N, C, K, xt, w_one, None, B.ACT_NONE, G.dev(dz), dx1, code, cs1, lr, db1, ws1)
+    B.check_device_status()
+    G.check_guards()
+    assert torch.equal(dx, dx1) and torch.equal(cs, cs1) and torch.equal(db, db1)
+    assert torch.equal(w_one, w_two), "fused update differs from backward + update"
+    _, _, dw_ref, _ = oracle.fc_bwd(x, w, None, dz, oracle.ACT_NONE, dz_dtype=np.float32)
+    G.assert_parity((G.dev(w) - w_one).cpu().numpy() / lr, dw_ref, "(w_old - w_new) / lr against the oracle's dw")

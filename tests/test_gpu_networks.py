@@ -233,3 +233,39 @@ def test_hybrid_fc_layer_with_library_kernels_single_rank():
     dw_gpu = L.dw.cpu().numpy().copy()
     L.update()
     np.testing.assert_allclose(L.w.cpu().numpy(), oracle.sgd_update(w, dw_gpu, lr), rtol=0, atol=1e-6)
+
+
+@pytest.mark.parametrize("which", ["vgg", "dnn"])
+def test_fused_update_step_equals_plain_step(which):
+    """fused_update: every weight tensor but the first layer's is updated by its own weight-gradient call (second pass
+    of the split reduction, GEMM epilogue, or scratch + update), the backpropagation of the layer reading the old weights
+    first.  Two steps must leave every parameter tensor bit-identical to the plain step's (gradients stored, one SGD
+    launch), and the losses equal."""
+    from paper_1602_06709_b200 import binding as B
+    from paper_1602_06709_b200 import inputs, networks
+    nets = []
+    for fused in (False, True):
+        if which == "vgg":
+            N, hw = 4, 32
+            net = networks.VggA(N, hw=hw, conv=SMALL_CONV, fc=[(64, 128), (128, 128), (128, 10)], classes=10, cfg="small",
+                                fused_update=fused)
+            x = inputs.uniform(inputs.tensor_id("small", "x"), (N, hw, hw, 3), 0.0, 1.0)
+            lab = inputs.labels(inputs.tensor_id("small", "labels"), N, 10)
+        else:
+            N, dims = 96, [44, 160, 160, 72]
+            net = networks.Dnn(N, dims=dims, cfg="small_dnn", fused_update=fused)
+            x = inputs.normal(inputs.tensor_id("small_dnn", "x"), (N, dims[0]), 1.0)
+            lab = inputs.labels(inputs.tensor_id("small_dnn", "labels"), N, dims[-1])
+        _randomise_biases(net)
+        net.x.copy_(torch.from_numpy(x)); net.labels.copy_(torch.from_numpy(lab))
+        losses = []
+        for _ in range(2):
+            net.step()
+            losses.append(net.loss.item())
+        B.check_device_status()
+        nets.append((net, losses))
+    (plain, lp), (fused, lf) = nets
+    assert fused.store.tail_offset < fused.store.total and not fused.store.in_order
+    assert all(abs(a - b) <= 1e-5 * abs(a) for a, b in zip(lp, lf))       # (the loss is summed with atomics: last bits vary)
+    for i in range(len(plain.store.shapes)):
+        assert torch.equal(plain.store.p(i), fused.store.p(i)), f"parameter tensor {i} differs"
