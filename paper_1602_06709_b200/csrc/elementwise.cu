@@ -107,9 +107,9 @@ __global__ void __launch_bounds__(256) act_grad_kernel(float* __restrict__ dy, c
 constexpr int kColsumMinRows = 64;     // rows per split, at least; grown so that there are at most ~1200 splits
 template <int VEC>
 __global__ void __launch_bounds__(256) colsum_kernel(const float* __restrict__ m, size_t rows, int K,
-                                                     float* __restrict__ partial, size_t rows_per_split) {
+                                                     float* __restrict__ partial, size_t rows_per_split, int strip) {
     const int kv = K / VEC;                                  // column groups per row
-    const int strip = kv < 256 ? kv : 256;                   // column groups this block covers per row
+    // strip: column groups this block covers per row (see colsum_strip())
     const int lanes = 256 / strip;                           // rows handled concurrently
     const int cg = blockIdx.x * strip + threadIdx.x % strip; // this thread's column group
     const int rl = threadIdx.x / strip;
@@ -762,6 +762,17 @@ int colsum_splits(size_t rows) {
     return int((rows + per - 1) / per);
 }
 
+// Column groups per block: whole 256-group strips where there are many rows (each row is then read as one contiguous
+// run); narrower strips, i.e. more blocks with more rows in flight per block, where a few rows would leave the sum to a
+// handful of blocks reading them one after another (the 32 rows of per-tile sums of an FC layer: 9 -> 3 us).
+static int colsum_strip(int kv, size_t rows, int splits) {
+    int strip = kv < 256 ? kv : 256;
+    const size_t rows_in_split = (rows + splits - 1) / splits;
+    while (strip > 8 && strip % 2 == 0 && long((kv + strip - 1) / strip) * splits < 64 && size_t(256 / (strip / 2)) <= rows_in_split)
+        strip /= 2;
+    return strip;
+}
+
 int launch_colsum(const float* m, size_t rows, int K, float* partial, float* out, cudaStream_t st) {
     const int splits = colsum_splits(rows);
     const size_t per = colsum_rows_per_split(rows);
@@ -769,13 +780,13 @@ int launch_colsum(const float* m, size_t rows, int K, float* partial, float* out
     {
         LaunchScope scope(KID_COLSUM, 4.0 * double(rows) * K, st);
         if (K % 4 == 0 && (reinterpret_cast<uintptr_t>(m) & 15) == 0) {
-            const int kv = K / 4, strip = kv < 256 ? kv : 256;
+            const int kv = K / 4, strip = colsum_strip(kv, rows, splits);
             colsum_kernel<4><<<dim3((kv + strip - 1) / strip, splits), 256, 0, st>>>(m, rows, K,
-                                                                                     splits == 1 ? out : partial, per);
+                                                                                     splits == 1 ? out : partial, per, strip);
         } else {
-            const int strip = K < 256 ? K : 256;
+            const int strip = colsum_strip(K, rows, splits);
             colsum_kernel<1><<<dim3((K + strip - 1) / strip, splits), 256, 0, st>>>(m, rows, K,
-                                                                                    splits == 1 ? out : partial, per);
+                                                                                    splits == 1 ? out : partial, per, strip);
         }
     }
     if (cudaGetLastError() != cudaSuccess) return PCL_ERR_CUDA;

@@ -664,10 +664,13 @@ int bwd_data_masked_colsum(const pcl_conv_desc* d, int P, int Q, const float* dy
             a.colsum_rows = sum_rows;
             // (the workspace is sized for the tiling with the most rows; this launch writes rows 0 .. written-1, of which a
             // grid smaller than the device leaves some untouched: those must not contribute)
-            long written = tc_fprop_colsum_rows_written(a);
-            if (written <= 0 || written > rows) written = rows;
-            rc = launch_zero(sum_rows, size_t(written) * d->C, st);
-            if (rc != PCL_OK) return rc;
+            bool all_written = false;
+            long written = tc_fprop_colsum_rows_written(a, &all_written);
+            if (written <= 0 || written > rows) { written = rows; all_written = false; }
+            if (!all_written) {
+                rc = launch_zero(sum_rows, size_t(written) * d->C, st);
+                if (rc != PCL_OK) return rc;
+            }
             rc = launch_tc_fprop(a, st);
             if (rc != PCL_OK) return rc;
             float* partial = reinterpret_cast<float*>(extra + align_up(size_t(rows) * d->C * 4, 256));

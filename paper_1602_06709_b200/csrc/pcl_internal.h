@@ -172,7 +172,8 @@ bool tc_fprop_can_pool(const TcFpropArgs& a);
 size_t tc_fprop_split_ws_bytes(const TcFpropArgs& a);
 bool tc_fprop_eligible(const TcFpropArgs& a);
 long tc_fprop_colsum_rows(const TcFpropArgs& a);              // upper bound over all tilings (workspace sizing)
-long tc_fprop_colsum_rows_written(const TcFpropArgs& a);      // rows the launch for exactly these arguments writes
+// rows the launch for exactly these arguments writes (rows 0 .. n-1); *all_written: none of them is left untouched
+long tc_fprop_colsum_rows_written(const TcFpropArgs& a, bool* all_written = nullptr);
 int launch_tc_fprop(const TcFpropArgs& a, cudaStream_t st);
 // Text description of the tiling launch_tc_fprop(a) would use and of the cost model's prediction for it (and of the
 // tiling the model itself would choose).

@@ -1360,12 +1360,15 @@ TileCfg select_cfg(const TcFpropArgs& a, int sm_count) {
 
 // Rows of column sums the launch for `a` writes (rows 0 .. n-1 of its colsum_rows buffer): per CTA where every tile
 // has the same columns, else per tile.
-long tc_fprop_colsum_rows_written(const TcFpropArgs& a) {
+long tc_fprop_colsum_rows_written(const TcFpropArgs& a, bool* all_written) {
     const int sm = device_sm_count();
+    if (all_written) *all_written = false;
     if (a.Kout % 4 != 0) return 0;
     const TileCfg c = select_cfg(a, sm);
     if (!c.ok) return 0;
-    if (c.tiles_k == 1) return long(sm) * c.MT * 4;
+    if (c.tiles_k == 1) return long(sm) * c.MT * 4;       // (a grid smaller than the device leaves rows untouched)
+    // per tile: every row is written, unless a pair's last half is an image group that does not exist
+    if (all_written) *all_written = !(c.pair && (c.tiles_n & 1));
     return long(c.tiles_q) * c.tiles_p * c.tiles_n * c.MT * 4;
 }
 
