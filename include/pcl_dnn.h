@@ -73,7 +73,7 @@ int pcl_set_path(int path);
  * has a named knob with which the tests pin each kernel variant and the alternatives were measured:
  * TILING (0 plain, 1-3 haloed layouts), BN, KS, KS_HALO, KS_WGRAD, PAIR, PAIR_HALO, PAIR_WGRAD, GRP,
  * ISSUERS, SPLIT_ACC, PIX_WGRAD, XHALO_WGRAD, TMA_STORE, WEIGHTS_IN_PLACE, EPI_WARPS, FC_DW_FORWARD,
- * KSPLIT, RESIDENT_B, KSLICES, SELECT, PACKED_BWD, WAIT_LIMIT_US (limit of the bounded device-side waits in microseconds,
+ * KSPLIT, RESIDENT_B, KSLICES, SELECT, PACKED_BWD, PLAN_CACHE, WAIT_LIMIT_US (limit of the bounded device-side waits in microseconds,
  * default 2 s; applies to the current device), FAULT_INJECT (test only: 1 / 2 make the next forward-type /
  * weight-gradient launch that runs as single CTAs arm its first pipeline slot for 16 bytes more than it copies,
  * so that the waits on that slot run out, the kernel gives up and returns, and pcl_last_device_status()
@@ -254,6 +254,16 @@ size_t pcl_fc_bwd_fused_sgd_workspace_bytes(int N, int C, int K);
 int pcl_fc_bwd_fused_sgd(int N, int C, int K, const float* x, float* w, const float* y, int act,
                          float* dy, float* dx, int x_act, float* dx_colsum, float lr, float* dbias,
                          void* ws, size_t ws_bytes, void* cuda_stream);
+
+/* Launch plans.  What a tensor-core launch needs besides its data -- the tiling, the kernel's parameter block, its TMA
+ * tensor maps, the grid -- follows from the call's arguments alone, so it is built once per distinct argument set
+ * (descriptor, pointers, strides, options; per device; per setting of the tuning knobs) and kept in a host-side
+ * cache (a few hundred bytes per plan, at most 512 plans per kernel family, then the cache starts over).  A training
+ * step that calls with the same buffers every iteration selects tilings and encodes tensor maps once per layer and
+ * pass.  Thread-safe.  The PLAN_CACHE knob (pcl_set_tuning) set to 0 builds every launch's plan afresh.
+ * pcl_plan_cache_stats: launches served from the cache / launches that built a plan, since the library was loaded
+ * (host counters; either pointer may be NULL). */
+int pcl_plan_cache_stats(unsigned long long* hits, unsigned long long* misses);
 
 /* Vanilla SGD (Sec. 1: algorithm and hyper-parameters untouched):
  *   w[i] <- w[i] - lr * dw[i],  i < n.   w, dw only need 4-byte alignment. */

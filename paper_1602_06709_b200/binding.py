@@ -32,7 +32,7 @@ EXPORTS = [
     "pcl_conv_bwd_weights_pooled", "pcl_conv_bwd_weights_pooled_is_fused", "pcl_conv_bwd_weights_pooled_workspace_bytes",
     "pcl_maxpool2x2_fwd_codes", "pcl_maxpool2x2_bwd_codes", "pcl_last_wait_code", "pcl_set_tuning", "pcl_reset_tuning", "pcl_fc_bwd_fused", "pcl_conv_plan_describe", "pcl_conv_staged_input_bytes",
     "pcl_conv_bwd_weights_pooled_staged", "pcl_conv_bwd_weights_sgd", "pcl_conv_bwd_weights_sgd_workspace_bytes",
-    "pcl_fc_bwd_fused_sgd", "pcl_fc_bwd_fused_sgd_workspace_bytes",
+    "pcl_fc_bwd_fused_sgd", "pcl_fc_bwd_fused_sgd_workspace_bytes", "pcl_plan_cache_stats",
 ]
 
 
@@ -336,6 +336,13 @@ def fc_bwd_fused_sgd(N, C, K, x, w, y, act, dy, dx, x_act, dx_colsum, lr, dbias,
     wp, wb = _ws(ws)
     _check(lib().pcl_fc_bwd_fused_sgd(N, C, K, _ptr(x), _ptr(w), _ptr(y), act, _ptr(dy), _ptr(dx), x_act, _ptr(dx_colsum),
                                       ctypes.c_float(lr), _ptr(dbias), wp, wb, _stream(stream)), "pcl_fc_bwd_fused_sgd")
+
+
+def plan_cache_stats():
+    """(hits, misses): tensor-core launches served from the launch-plan cache / launches that built their plan."""
+    h, m = ctypes.c_ulonglong(0), ctypes.c_ulonglong(0)
+    _check(lib().pcl_plan_cache_stats(ctypes.byref(h), ctypes.byref(m)), "pcl_plan_cache_stats")
+    return int(h.value), int(m.value)
 
 
 def sgd_update(w, dw, lr, stream=None):

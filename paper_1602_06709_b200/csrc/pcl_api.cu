@@ -41,7 +41,7 @@ std::atomic<unsigned> g_tune_gen{0};
 const char* const kTuneNames[TUNE_COUNT] = {
     "TILING", "BN", "KS", "KS_HALO", "KS_WGRAD", "PAIR", "PAIR_HALO", "PAIR_WGRAD", "GRP", "ISSUERS", "SPLIT_ACC",
     "PIX_WGRAD", "XHALO_WGRAD", "TMA_STORE", "WEIGHTS_IN_PLACE", "EPI_WARPS", "FC_DW_FORWARD", "KSPLIT",
-    "WAIT_LIMIT_US", "FAULT_INJECT", "RESIDENT_B", "KSLICES", "SELECT", "PACKED_BWD"};
+    "WAIT_LIMIT_US", "FAULT_INJECT", "RESIDENT_B", "KSLICES", "SELECT", "PACKED_BWD", "PLAN_CACHE"};
 }  // namespace
 
 int tune(int id, int dflt) {
@@ -1096,6 +1096,11 @@ size_t pcl_fc_bwd_fused_sgd_workspace_bytes(int N, int C, int K) {
     const size_t wgrad_form = pcl_conv_bwd_weights_sgd_workspace_bytes(&d);
     const size_t fwd_form = fc_dzt_bytes(N, K) + plan_wgrad(d, 1, 1).colsum_bytes;
     return pcl_conv_bwd_data_colsum_workspace_bytes(&d) + align_up(wgrad_form > fwd_form ? wgrad_form : fwd_form, 256);
+}
+
+int pcl_plan_cache_stats(unsigned long long* hits, unsigned long long* misses) {
+    plan_cache_stats(hits, misses);
+    return PCL_OK;
 }
 
 int pcl_sgd_update(float* w, const float* dw, size_t n, float lr, void* cuda_stream) {

@@ -60,7 +60,7 @@ enum TuneId {
     TUNE_TILING = 0,        // forward-type kernel: 0 plain, 1-3 haloed layouts 0-2
     TUNE_BN, TUNE_KS, TUNE_KS_HALO, TUNE_KS_WGRAD, TUNE_PAIR, TUNE_PAIR_HALO, TUNE_PAIR_WGRAD, TUNE_GRP, TUNE_ISSUERS,
     TUNE_SPLIT_ACC, TUNE_PIX_WGRAD, TUNE_XHALO_WGRAD, TUNE_TMA_STORE, TUNE_WEIGHTS_IN_PLACE, TUNE_EPI_WARPS,
-    TUNE_FC_DW_FORWARD, TUNE_KSPLIT, TUNE_WAIT_LIMIT_US, TUNE_FAULT_INJECT, TUNE_RESIDENT_B, TUNE_KSLICES, TUNE_SELECT, TUNE_PACKED_BWD, TUNE_COUNT
+    TUNE_FC_DW_FORWARD, TUNE_KSPLIT, TUNE_WAIT_LIMIT_US, TUNE_FAULT_INJECT, TUNE_RESIDENT_B, TUNE_KSLICES, TUNE_SELECT, TUNE_PACKED_BWD, TUNE_PLAN_CACHE, TUNE_COUNT
 };
 int tune(int id, int dflt);
 bool tune_is_set(int id);
@@ -175,6 +175,9 @@ long tc_fprop_colsum_rows(const TcFpropArgs& a);              // upper bound ove
 // rows the launch for exactly these arguments writes (rows 0 .. n-1); *all_written: none of them is left untouched
 long tc_fprop_colsum_rows_written(const TcFpropArgs& a, bool* all_written = nullptr);
 int launch_tc_fprop(const TcFpropArgs& a, cudaStream_t st);
+// tensor-core launches whose plan (tiling, kernel parameters, tensor maps, grid) came out of / went into the plan caches
+void plan_cache_count(bool hit);
+void plan_cache_stats(unsigned long long* hits, unsigned long long* misses);
 // Text description of the tiling launch_tc_fprop(a) would use and of the cost model's prediction for it (and of the
 // tiling the model itself would choose).
 int tc_fprop_describe(const TcFpropArgs& a, char* buf, size_t n);

@@ -29,6 +29,11 @@
 #include <stdio.h>
 #include <stdlib.h>
 
+#include <atomic>
+#include <mutex>
+#include <string>
+#include <unordered_map>
+
 #include "pcl_internal.h"
 #include "pcl_ptx.cuh"
 
@@ -1441,7 +1446,83 @@ size_t tc_fprop_split_ws_bytes(const TcFpropArgs& a) {
     return k > 1 ? size_t(k) * a.N * a.P * a.Q * a.Kout * 4 : 0;
 }
 
+namespace {
+// Everything a launch needs that follows from its arguments alone (tiling, kernel parameters, tensor maps, grid):
+// built once per distinct argument set and kept (see launch_tc_fprop).
+struct FpropPlan {
+    FpropParams p;
+    CUtensorMap tmA, tmB, tmOut;
+    bool pair = false, wide_epi = false;
+    size_t smem = 0;
+    long total = 0;          // CTA tiles (pair: pair tiles)
+    int sm_count = 0, grid = 0;
+    double flops = 0.0;
+};
+int build_fprop_plan(const TcFpropArgs& a, FpropPlan* plan);
+int run_fprop_plan(const FpropPlan& plan, const TcFpropArgs& a, cudaStream_t st);
+
+// Plan cache.  The key is every field of the arguments (pointers included: they are in the tensor maps), the device and
+// the generation of the tuning knobs; a step driver that calls with the same buffers every step pays for tiling
+// selection and three cuTensorMapEncodeTiled calls once per layer and pass instead of once per call.
+void key_put(std::string& k, const void* v, size_t n) { k.append(static_cast<const char*>(v), n); }
+template <class T> void key_put(std::string& k, const T& v) { key_put(k, &v, sizeof(T)); }
+std::string fprop_plan_key(const TcFpropArgs& a, int device) {
+    std::string k;
+    k.reserve(320);
+    key_put(k, a.in); key_put(k, a.wt); key_put(k, a.bias); key_put(k, a.mask_src); key_put(k, a.out);
+    const int ints[] = {a.N, a.H, a.W, a.Cin, a.Kout, a.R, a.S, a.pad_h, a.pad_w, a.P, a.Q, a.act, a.mask_mode, a.k_live, a.in_inner,
+                        a.wt_mn_major, a.flip_taps, a.stride_h, a.stride_w, a.dil_w, device};
+    key_put(k, ints, sizeof(ints));
+    const long longs[] = {a.in_stride_w, a.in_stride_h, a.in_stride_n, a.out_stride_w, a.out_stride_h, a.out_stride_n};
+    key_put(k, longs, sizeof(longs));
+    key_put(k, a.lr); key_put(k, a.colsum_rows); key_put(k, a.pool_out); key_put(k, a.pool_idx); key_put(k, a.split_ws);
+    key_put(k, a.split_ws_bytes);
+    const unsigned long long gen = tune_generation();
+    key_put(k, gen);
+    return k;
+}
+std::mutex g_plan_mu;
+std::unordered_map<std::string, FpropPlan> g_plans;
+std::atomic<unsigned long long> g_plan_hits{0}, g_plan_misses{0};
+constexpr size_t kMaxPlans = 512;       // (a network has a few dozen distinct launches; beyond this the cache starts over)
+}  // namespace
+
+void plan_cache_count(bool hit) { if (hit) ++g_plan_hits; else ++g_plan_misses; }
+
+void plan_cache_stats(unsigned long long* hits, unsigned long long* misses) {
+    if (hits) *hits = g_plan_hits.load();
+    if (misses) *misses = g_plan_misses.load();
+}
+
 int launch_tc_fprop(const TcFpropArgs& a, cudaStream_t st) {
+    if (!tune(TUNE_PLAN_CACHE, 1)) {
+        FpropPlan plan;
+        const int rc = build_fprop_plan(a, &plan);
+        return rc != PCL_OK ? rc : run_fprop_plan(plan, a, st);
+    }
+    int device = 0;
+    if (cudaGetDevice(&device) != cudaSuccess) return PCL_ERR_CUDA;
+    const std::string key = fprop_plan_key(a, device);
+    FpropPlan plan;
+    bool hit = false;
+    {
+        std::lock_guard<std::mutex> lock(g_plan_mu);
+        auto it = g_plans.find(key);
+        if (it != g_plans.end()) { plan = it->second; hit = true; }
+    }
+    plan_cache_count(hit);
+    if (!hit) {
+        const int rc = build_fprop_plan(a, &plan);
+        if (rc != PCL_OK) return rc;
+        std::lock_guard<std::mutex> lock(g_plan_mu);
+        if (g_plans.size() >= kMaxPlans) g_plans.clear();
+        g_plans.emplace(key, plan);
+    }
+    return run_fprop_plan(plan, a, st);
+}
+
+namespace {
+int build_fprop_plan(const TcFpropArgs& a, FpropPlan* plan) {
     if (!tc_fprop_eligible(a)) return PCL_ERR_UNSUPPORTED_SHAPE;
     static PerDeviceOnce attr_once;       // (the attribute applies to the current device only)
     const int setup_rc = attr_once.run([]() -> int {
@@ -1615,14 +1696,18 @@ int launch_tc_fprop(const TcFpropArgs& a, cudaStream_t st) {
     const size_t smem = (p.halo ? size_t(p.NA) * p.a_buf_bytes + size_t(p.stages) * p.KS * (cfg.pair ? p.BN * 64 : p.BN * 128)
                                 : size_t(p.stages) * p.KS * (kABytes + (cfg.pair ? p.BN * 64 : p.BN * 128))) +
                         (wide_epi ? kEpiStageBytesWide : kEpiStageBytes) + 1024;
+    plan->p = p; plan->tmA = tmA; plan->tmB = tmB; plan->tmOut = tmOut;
+    plan->pair = cfg.pair != 0; plan->wide_epi = wide_epi; plan->smem = smem; plan->total = total; plan->sm_count = g_sm_count;
+    plan->flops = 2.0 * a.N * a.P * a.Q * double(a.Kout) * a.Cin * a.R * a.S;
+    plan->grid = int(total < g_sm_count ? total : g_sm_count);
     if (cfg.pair) {
+        // how many pairs the device holds at once with this much shared memory (cached per size)
         cudaLaunchAttribute attr[1];
         attr[0].id = cudaLaunchAttributeClusterDimension;
         attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
         cudaLaunchConfig_t lc{};
-        lc.blockDim = dim3(kThreads); lc.dynamicSmemBytes = smem; lc.stream = st;
+        lc.blockDim = dim3(kThreads); lc.dynamicSmemBytes = smem;
         lc.attrs = attr; lc.numAttrs = 1;
-        // how many pairs the device holds at once with this much shared memory (cached per size)
         static std::mutex cache_mu;
         static size_t cached_smem = 0;
         static int cached_clusters = 0, cached_dev = -1;
@@ -1637,17 +1722,35 @@ int launch_tc_fprop(const TcFpropArgs& a, cudaStream_t st) {
             cached_smem = smem;
             cached_dev = cur_dev;
         }
-        const long pair_tiles = long(p.tiles_q) * p.tiles_p * p.tiles_n * p.tiles_k * p.ksplit;
-        long nclus = pair_tiles < cached_clusters ? pair_tiles : cached_clusters;
-        lc.gridDim = dim3(unsigned(2 * nclus));
-        LaunchScope scope(KID_TC_FPROP, 2.0 * a.N * a.P * a.Q * double(a.Kout) * a.Cin * a.R * a.S, st);
+        const long nclus = total < cached_clusters ? total : cached_clusters;       // (total counts pair tiles here)
+        plan->grid = int(2 * nclus);
+    }
+    return PCL_OK;
+}
+
+int run_fprop_plan(const FpropPlan& plan, const TcFpropArgs& a, cudaStream_t st) {
+    const FpropParams& p = plan.p;
+    const CUtensorMap& tmA = plan.tmA;
+    const CUtensorMap& tmB = plan.tmB;
+    const CUtensorMap& tmOut = plan.tmOut;
+    const bool wide_epi = plan.wide_epi;
+    const size_t smem = plan.smem;
+    if (plan.pair) {
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeClusterDimension;
+        attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+        cudaLaunchConfig_t lc{};
+        lc.blockDim = dim3(kThreads); lc.dynamicSmemBytes = smem; lc.stream = st;
+        lc.attrs = attr; lc.numAttrs = 1;
+        lc.gridDim = dim3(unsigned(plan.grid));
+        LaunchScope scope(KID_TC_FPROP, plan.flops, st);
         const cudaError_t le = p.pool_out   ? cudaLaunchKernelEx(&lc, tc_fprop_kernel<true, true, false>, tmA, tmB, tmOut, p)
                                : p.mask_src ? cudaLaunchKernelEx(&lc, tc_fprop_kernel<true, false, true>, tmA, tmB, tmOut, p)
                                             : cudaLaunchKernelEx(&lc, tc_fprop_kernel<true, false, false>, tmA, tmB, tmOut, p);
         if (le != cudaSuccess) return PCL_ERR_CUDA;
     } else {
-        const int grid = int(total < g_sm_count ? total : g_sm_count);
-        LaunchScope scope(KID_TC_FPROP, 2.0 * a.N * a.P * a.Q * double(a.Kout) * a.Cin * a.R * a.S, st);
+        const int grid = plan.grid;
+        LaunchScope scope(KID_TC_FPROP, plan.flops, st);
         if (wide_epi && p.pool_out) tc_fprop_kernel<false, true, false, kEpiWarpsWide><<<grid, kThreadsWide, smem, st>>>(tmA, tmB, tmOut, p);
         else if (wide_epi) tc_fprop_kernel<false, false, false, kEpiWarpsWide><<<grid, kThreadsWide, smem, st>>>(tmA, tmB, tmOut, p);
         else if (p.pool_out) tc_fprop_kernel<false, true, false><<<grid, kThreads, smem, st>>>(tmA, tmB, tmOut, p);
@@ -1659,5 +1762,6 @@ int launch_tc_fprop(const TcFpropArgs& a, cudaStream_t st) {
         return launch_reduce_splits_bias_act(a.split_ws, a.out, a.bias, a.act, size_t(a.N) * a.P * a.Q, a.Kout, p.ksplit, st);
     return PCL_OK;
 }
+}  // namespace
 
 }  // namespace pcl

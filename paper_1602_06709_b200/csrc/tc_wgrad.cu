@@ -46,7 +46,10 @@
 // runs, and the even CTA issues M = 256 MMAs for both (cta_group::2).
 #include <stdlib.h>
 
+#include <mutex>
+#include <string>
 #include <type_traits>
+#include <unordered_map>
 
 #include "pcl_internal.h"
 #include "pcl_ptx.cuh"
@@ -754,7 +757,67 @@ int tc_wgrad_splits(int N, int P, int Q, int C, int K, int R, int S, int tap_gro
     return int(splits);
 }
 
+namespace {
+// What a launch needs that follows from its arguments alone; kept per distinct argument set like the forward-type
+// kernel's plans (same key discipline: every field, the device, the generation of the tuning knobs).
+struct WgradLaunchPlan {
+    WgradParams p;
+    CUtensorMap tmDy, tmX;
+    bool pair = false, wide = false, zero_first = false;
+    long items = 0;
+    size_t smem = 0, dw_elems = 0;
+    double flops = 0.0;
+};
+int build_wgrad_plan(const TcWgradArgs& a, WgradLaunchPlan* plan);
+int run_wgrad_plan(const WgradLaunchPlan& plan, const TcWgradArgs& a, cudaStream_t st);
+std::string wgrad_plan_key(const TcWgradArgs& a, int device) {
+    std::string k;
+    k.reserve(256);
+    auto put = [&k](const void* v, size_t n) { k.append(static_cast<const char*>(v), n); };
+    const void* ptrs[] = {a.x, a.dy, a.dw, a.partial, a.dy_pool, a.codes, a.db_rows, a.w_update};
+    put(ptrs, sizeof(ptrs));
+    const int ints[] = {a.N, a.H, a.W, a.C, a.K, a.R, a.S, a.pad_h, a.pad_w, a.P, a.Q, a.splits, a.x_inner, a.tap_groups, a.skip_reduce,
+                        a.relu_mask, a.stride_h, a.stride_w, a.dil_w, device};
+    put(ints, sizeof(ints));
+    const long longs[] = {a.x_stride_w, a.x_stride_h, a.x_stride_n};
+    put(longs, sizeof(longs));
+    put(&a.lr, sizeof(a.lr));
+    const unsigned gen = tune_generation();
+    put(&gen, sizeof(gen));
+    return k;
+}
+std::mutex g_wplan_mu;
+std::unordered_map<std::string, WgradLaunchPlan> g_wplans;
+}  // namespace
+
 int launch_tc_wgrad(const TcWgradArgs& a, cudaStream_t st) {
+    WgradLaunchPlan plan;
+    if (!tune(TUNE_PLAN_CACHE, 1)) {
+        const int rc = build_wgrad_plan(a, &plan);
+        return rc != PCL_OK ? rc : run_wgrad_plan(plan, a, st);
+    }
+    int device = 0;
+    if (cudaGetDevice(&device) != cudaSuccess) return PCL_ERR_CUDA;
+    const std::string key = wgrad_plan_key(a, device);
+    bool hit = false;
+    {
+        std::lock_guard<std::mutex> lock(g_wplan_mu);
+        auto it = g_wplans.find(key);
+        if (it != g_wplans.end()) { plan = it->second; hit = true; }
+    }
+    if (!hit) {
+        const int rc = build_wgrad_plan(a, &plan);
+        if (rc != PCL_OK) return rc;
+        std::lock_guard<std::mutex> lock(g_wplan_mu);
+        if (g_wplans.size() >= 512) g_wplans.clear();
+        g_wplans.emplace(key, plan);
+    }
+    plan_cache_count(hit);
+    return run_wgrad_plan(plan, a, st);
+}
+
+namespace {
+int build_wgrad_plan(const TcWgradArgs& a, WgradLaunchPlan* plan) {
     if (!tc_wgrad_eligible(a)) return PCL_ERR_UNSUPPORTED_SHAPE;
     static PerDeviceOnce attr_once;       // (the attribute applies to the current device only)
     const int setup_rc = attr_once.run([]() -> int {
@@ -805,6 +868,7 @@ int launch_tc_wgrad(const TcWgradArgs& a, cudaStream_t st) {
     if (!p.status) return PCL_ERR_CUDA;
     p.inject_short_copy = (tune(TUNE_FAULT_INJECT, 0) == 2 && !rp.pair && !pooled) ? 1 : 0;      // test mode
     const size_t dw_elems = size_t(a.K) * a.R * a.S * a.C;
+    bool zero_first = false;
     if (a.w_update && p.splits != 1) return PCL_ERR_BAD_ARG;      // (a split reduction updates in its second pass)
     if (p.splits == 1) {
         p.out = a.w_update ? a.w_update : a.dw; p.split_stride = 0; p.use_atomics = 0;
@@ -813,8 +877,7 @@ int launch_tc_wgrad(const TcWgradArgs& a, cudaStream_t st) {
         p.out = a.partial; p.split_stride = dw_elems; p.use_atomics = 0;
     } else {
         p.out = a.dw; p.split_stride = 0; p.use_atomics = 1;
-        int rc = launch_zero(a.dw, dw_elems, st);
-        if (rc != PCL_OK) return rc;
+        zero_first = true;
     }
 
     // When both map counts are multiples of 32, each tensor is viewed as 5-D {32 maps, w, h, n, group} (the
@@ -879,9 +942,26 @@ int launch_tc_wgrad(const TcWgradArgs& a, cudaStream_t st) {
     const long items = long(p.k_tiles) * p.run_blocks * p.splits;
     if (items > 0x7fffffffL) return PCL_ERR_UNSUPPORTED_SHAPE;
     const size_t smem = size_t(p.stages) * stage_bytes + 1024;
+    plan->p = p; plan->tmDy = tmDy; plan->tmX = tmX;
+    plan->pair = rp.pair != 0; plan->wide = pooled && p.duo; plan->zero_first = zero_first;
+    plan->items = items; plan->smem = smem; plan->dw_elems = dw_elems;
+    plan->flops = 2.0 * a.N * a.P * a.Q * double(a.K) * a.C * a.R * a.S;
+    return PCL_OK;
+}
+
+int run_wgrad_plan(const WgradLaunchPlan& plan, const TcWgradArgs& a, cudaStream_t st) {
+    const WgradParams& p = plan.p;
+    const CUtensorMap& tmDy = plan.tmDy;
+    const CUtensorMap& tmX = plan.tmX;
+    const long items = plan.items;
+    const size_t smem = plan.smem, dw_elems = plan.dw_elems;
+    if (plan.zero_first) {
+        const int rc = launch_zero(a.dw, dw_elems, st);
+        if (rc != PCL_OK) return rc;
+    }
     {
-        LaunchScope scope(KID_TC_WGRAD, 2.0 * a.N * a.P * a.Q * double(a.K) * a.C * a.R * a.S, st);
-        if (rp.pair) {
+        LaunchScope scope(KID_TC_WGRAD, plan.flops, st);
+        if (plan.pair) {
             cudaLaunchAttribute attr[1];
             attr[0].id = cudaLaunchAttributeClusterDimension;
             attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
@@ -889,7 +969,7 @@ int launch_tc_wgrad(const TcWgradArgs& a, cudaStream_t st) {
             lc.gridDim = dim3(unsigned(items)); lc.blockDim = dim3(kWgradThreads); lc.dynamicSmemBytes = smem; lc.stream = st;
             lc.attrs = attr; lc.numAttrs = 1;
             if (cudaLaunchKernelEx(&lc, tc_wgrad_kernel<true>, tmDy, tmX, p) != cudaSuccess) return PCL_ERR_CUDA;
-        } else if (pooled && p.duo) {
+        } else if (plan.wide) {
             tc_wgrad_kernel<false, true><<<int(items), kWgradThreadsWide, smem, st>>>(tmDy, tmX, p);
         } else {
             tc_wgrad_kernel<false><<<int(items), kWgradThreads, smem, st>>>(tmDy, tmX, p);
@@ -899,5 +979,6 @@ int launch_tc_wgrad(const TcWgradArgs& a, cudaStream_t st) {
     if (p.splits > 1 && a.partial && !a.skip_reduce) return launch_reduce_splits(a.partial, a.dw, dw_elems, p.splits, st);
     return PCL_OK;
 }
+}  // namespace
 
 }  // namespace pcl

@@ -269,3 +269,52 @@ def test_fused_update_step_equals_plain_step(which):
     assert all(abs(a - b) <= 1e-5 * abs(a) for a, b in zip(lp, lf))       # (the loss is summed with atomics: last bits vary)
     for i in range(len(plain.store.shapes)):
         assert torch.equal(plain.store.p(i), fused.store.p(i)), f"parameter tensor {i} differs"
+
+
+def test_launch_plans_are_cached_and_change_nothing():
+    """The second call with the same descriptor and buffers is served from the launch-plan cache (no tiling selection,
+    no tensor-map encoding); other buffers or a changed knob build a plan of their own; results are those of a build
+    with the cache switched off, bit for bit."""
+    import gpu_helpers as G
+    from paper_1602_06709_b200 import binding as B
+    N, C, K, H = 4, 64, 96, 24
+    d = B.conv_desc(N, C, K, H, H, 3, 3, 1, 1)
+    g = torch.Generator(device="cuda").manual_seed(42)
+    x = torch.rand(N, H, H, C, device="cuda", generator=g)
+    w = torch.randn(K, 3, 3, C, device="cuda", generator=g) * 0.05
+    dy = torch.randn(N, H, H, K, device="cuda", generator=g) * 1e-2
+    b = torch.zeros(K, device="cuda")
+    ws = G.workspace(max(B.conv_workspace_bytes(d, i) for i in range(3)))
+
+    def three_passes(xx):
+        y = torch.empty(N, H, H, K, device="cuda"); dx = torch.empty_like(xx); dw = torch.empty_like(w)
+        B.conv_fwd(d, xx, w, b, y, B.ACT_RELU, ws)
+        B.conv_bwd_data(d, dy, w, xx, dx, ws)
+        B.conv_bwd_weights(d, xx, dy, dw, None, True, ws)
+        return y, dx, dw
+
+    B.set_tuning("PLAN_CACHE", 0)
+    ref = three_passes(x)
+    h0, m0 = B.plan_cache_stats()
+    B.set_tuning("PLAN_CACHE", 1)
+    y1 = torch.empty(N, H, H, K, device="cuda")
+    B.conv_fwd(d, x, w, b, y1, B.ACT_RELU, ws)
+    h1, m1 = B.plan_cache_stats()
+    assert (h1, m1) == (h0, m0 + 1)                      # a new plan
+    B.conv_fwd(d, x, w, b, y1, B.ACT_RELU, ws)
+    h2, m2 = B.plan_cache_stats()
+    assert (h2, m2) == (h1 + 1, m1)                      # served from the cache
+    x2 = x.clone()
+    y2 = torch.empty(N, H, H, K, device="cuda")
+    B.conv_fwd(d, x2, w, b, y2, B.ACT_RELU, ws)          # other buffers: another plan
+    assert B.plan_cache_stats() == (h2, m2 + 1)
+    B.set_tuning("BN", 32)                               # a knob changed: another plan, and the knob is honoured
+    B.conv_fwd(d, x, w, b, y2, B.ACT_RELU, ws)
+    assert B.plan_cache_stats() == (h2, m2 + 2)
+    assert "BN=32" in B.conv_plan_describe(d, B.PASS_FWD)
+    B.set_tuning("BN", None)
+    for _ in range(2):                                   # cached plans of all three passes, twice: identical results
+        got = three_passes(x)
+        for a_, b_ in zip(ref, got):
+            assert torch.equal(a_, b_)
+    B.check_device_status()
