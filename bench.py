@@ -369,6 +369,11 @@ def run_ours(args):
     def max_over_ranks(v: float) -> float:
         return replicas.max_over_ranks(v, device="cuda")
 
+    for kv in args.tune:
+        if not args.kernels_only:
+            raise SystemExit("--tune changes which kernels run: only allowed with --kernels-only")
+        name, _, val = kv.partition("=")
+        B.set_tuning(name, val if name == "TILING" and not val.lstrip("-").isdigit() else int(val))
     if args.layer and not (args.kernels_only and args.workload == "conv"):
         raise SystemExit("--layer changes the workload: only allowed with --workload conv --kernels-only")
     if args.layer:
@@ -686,6 +691,8 @@ def main():
     ap.add_argument("--graph", default="auto", choices=["auto", "0", "1"],
                     help="replay the step from a CUDA graph of its launches (auto: the DNN step only)")
     ap.add_argument("--minibatch", type=int, default=0, help="override the workload's minibatch (profiling only)")
+    ap.add_argument("--tune", action="append", default=[], metavar="KNOB=VALUE",
+                    help="pin a launcher choice through pcl_set_tuning for this run (profiling only), e.g. XHALO_WGRAD=0")
     ap.add_argument("--layer", default="", help="C,K,H of another 3x3 pad-1 layer for --workload conv (profiling only)")
     ap.add_argument("--data-parallel", action="store_true",
                     help="vgga / dnn with --gpus N > 1: one data-parallel job (per-layer reduce-scatter of the weight "
