@@ -128,7 +128,9 @@ __device__ __forceinline__ void xhalo_row(uint32_t d_tmem, uint32_t xn, uint32_t
 // kWide (pooled dy with two issuers): sixteen warps build the dy tiles, in two groups that take the pipeline slots
 // alternately like the issuing threads do -- a builder warp is a chain of dependent instructions per k-step, and two
 // warps per scheduler cannot hide it.
-template <bool kPair, bool kWide = false>
+// kSgd: the epilogue of an unsplit launch applies the SGD update in place (an instantiation of its own: the prefetched old
+// weights would cost the plain epilogue registers and a branch per chunk).
+template <bool kPair, bool kWide = false, bool kSgd = false>
 __global__ void __launch_bounds__(kWide ? kWgradThreadsWide : kWgradThreads, 1)
 tc_wgrad_kernel(const __grid_constant__ CUtensorMap tmDy, const __grid_constant__ CUtensorMap tmX, WgradParams p) {
     extern __shared__ uint8_t smem_raw[];
@@ -543,7 +545,7 @@ tc_wgrad_kernel(const __grid_constant__ CUtensorMap tmDy, const __grid_constant_
                 }
                 // (in-place update: the old weights of the chunk are fetched before the accumulator is read and staged, so
                 // that their latency does not fall between the stores)
-                const bool sgd = !kWide && p.sgd;      // (pooled-dy launches always have a second pass)
+                constexpr bool sgd = kSgd;
                 float4 wv[8];
                 if (sgd && vec_ok && c0 + cg < p.C) {
 #pragma unroll
@@ -826,6 +828,10 @@ int build_wgrad_plan(const TcWgradArgs& a, WgradLaunchPlan* plan) {
             cudaFuncSetAttribute(tc_wgrad_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  kSmemBudget + 1024) != cudaSuccess ||
             cudaFuncSetAttribute(tc_wgrad_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 kSmemBudget + 1024) != cudaSuccess ||
+            cudaFuncSetAttribute(tc_wgrad_kernel<false, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 kSmemBudget + 1024) != cudaSuccess ||
+            cudaFuncSetAttribute(tc_wgrad_kernel<true, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  kSmemBudget + 1024) != cudaSuccess)
             return PCL_ERR_CUDA;
         return PCL_OK;
@@ -968,9 +974,13 @@ int run_wgrad_plan(const WgradLaunchPlan& plan, const TcWgradArgs& a, cudaStream
             cudaLaunchConfig_t lc{};
             lc.gridDim = dim3(unsigned(items)); lc.blockDim = dim3(kWgradThreads); lc.dynamicSmemBytes = smem; lc.stream = st;
             lc.attrs = attr; lc.numAttrs = 1;
-            if (cudaLaunchKernelEx(&lc, tc_wgrad_kernel<true>, tmDy, tmX, p) != cudaSuccess) return PCL_ERR_CUDA;
+            const cudaError_t le = p.sgd ? cudaLaunchKernelEx(&lc, tc_wgrad_kernel<true, false, true>, tmDy, tmX, p)
+                                         : cudaLaunchKernelEx(&lc, tc_wgrad_kernel<true>, tmDy, tmX, p);
+            if (le != cudaSuccess) return PCL_ERR_CUDA;
         } else if (plan.wide) {
             tc_wgrad_kernel<false, true><<<int(items), kWgradThreadsWide, smem, st>>>(tmDy, tmX, p);
+        } else if (p.sgd) {
+            tc_wgrad_kernel<false, false, true><<<int(items), kWgradThreads, smem, st>>>(tmDy, tmX, p);
         } else {
             tc_wgrad_kernel<false><<<int(items), kWgradThreads, smem, st>>>(tmDy, tmX, p);
         }
