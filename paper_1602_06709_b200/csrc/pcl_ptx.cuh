@@ -87,7 +87,7 @@ __device__ __forceinline__ bool bounded_wait_warp(uint64_t* bar, uint32_t parity
 }
 
 // Low-duty form for warps that wait long (an epilogue warp waits for a whole main loop): lane 0 polls and
-// sleeps between polls, so that the wait takes almost no issue slots from the single-thread pipeline loops
+// sleeps between polls, so that the wait takes almost no issue slots from the pipeline roles' loops
 // that share the warp scheduler; the result is broadcast.
 __device__ __forceinline__ bool bounded_wait_warp_relaxed(uint64_t* bar, uint32_t parity, volatile uint32_t* abort_flag,
                                                           unsigned int* status_word, uint32_t code) {
@@ -187,7 +187,7 @@ __device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t ncols) {
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 
-// D[tmem] (+)= A[smem] * B[smem], TF32 operands, fp32 accumulate; one thread issues.
+// D[tmem] (+)= A[smem] * B[smem], TF32 operands, fp32 accumulate.
 // Warp-collective (like every MMA, commit and k-step form below): the WHOLE warp executes it, converged, with the same
 // operands in every lane, and one elected lane issues the instruction.  A loop that runs in lane 0 alone is divergent
 // code to the compiler, which then moves every descriptor into the uniform registers the instruction takes, one word at
@@ -337,11 +337,12 @@ __device__ __forceinline__ void umma_commit_pair(uint64_t* bar) {
                  : "memory");
 }
 
-// ------------------------------------------------- lean forms for the single-thread pipeline loops
-// The producer and the MMA-issuing thread each run alone in their warp, so every instruction they execute costs
-// several cycles of the k-step budget (a 128 x 256 x 32 k-step is 512 tensor cycles; measured: a loop of ~100
-// instructions per k-step held the tensor pipe at 63 %).  These forms take shared-memory addresses as 32-bit
-// registers that the loops advance by addition, and issue the four K = 8 MMAs of a k-step from one asm block.
+// ------------------------------------------------- lean forms for the pipeline roles' loops
+// The producer and the MMA-issuing role are each one warp that executes a chain of dependent instructions (all lanes
+// the same values, one elected lane issuing), so every instruction costs several cycles of the k-step budget (a
+// 128 x 256 x 32 k-step is 512 tensor cycles; measured: a loop of ~100 instructions per k-step held the tensor pipe at
+// 63 %).  These forms take shared-memory addresses as 32-bit registers that the loops advance by addition, and issue the
+// four K = 8 MMAs of a k-step from one asm block.
 __device__ __forceinline__ bool mbar_try_wait_addr(uint32_t bar_addr, uint32_t parity) {
     uint32_t ok;
     asm volatile(

@@ -19,9 +19,10 @@
 //   CTA pairs       two CTAs of a cluster share a weight tile, the leader issues M = 256 MMAs (cta_group::2)
 //
 // Warp roles (352 threads, persistent over tiles):
-//   warp 0        TMA producer (one thread), fills the ring of slots
-//   warp 1        allocates TMEM; one thread issues tcgen05.mma kind::tf32 (mma_issuer())
-//   warp 10       second issuing thread for single-CTA tiles with many slots
+//   warp 0        TMA producer, fills the ring of slots (the warp runs its loop converged, an elected lane issues)
+//   warp 1        allocates TMEM; issues tcgen05.mma kind::tf32 (mma_issuer(); converged warp, elected lane)
+//   warp 10       second issuing warp: alternate slots of single-CTA tiles with many slots, or alternate tiles of the
+//                 few-channel first layer
 //   warps 2-9     epilogue: TMEM -> registers -> bias / activation / mask [/ column sums / 2x2 max pool]
 //                 -> global, through TMA stores or coalesced per-lane stores (two warps per TMEM lane quarter)
 //   warps 11-18   eight more epilogue warps (608 threads) in the variant for tiles with a very short reduction
@@ -209,7 +210,8 @@ __device__ __forceinline__ void add_second_accumulator(uint32_t taddr, uint32_t 
     for (int i = 0; i < 32; ++i) v[i] = __float_as_uint(__uint_as_float(v[i]) + __uint_as_float(w[i]));
 }
 
-// kTaps consecutive taps of a haloed slot, straight-line (a taken branch costs a lone thread tens of cycles).
+// kTaps consecutive taps of a haloed slot, straight-line (the issuing role is a chain of dependent instructions: a taken
+// branch costs it tens of cycles).
 // kNsl = 0: the number of K = 8 slices per tap is the run-time `nsl` (skipped slices still cost their issue slots);
 // kNsl = 1..3: exactly that many MMAs per tap are emitted (few-channel layers, whose tap rows hold fewer than 32
 // live reduction elements: the issuing thread, not the tensor pipe, is what bounds their tiles).
@@ -245,10 +247,9 @@ __device__ __forceinline__ void halo_taps(uint32_t d_tmem, uint32_t BN, uint32_t
 // The MMA-issuing role, one warp per issuer (waits included), kept out of line and free of anything the loops do not
 // need.  The WHOLE warp runs it, every lane with the same values, and the MMA and commit forms elect one lane to issue:
 // run by lane 0 alone the same loops are divergent code whose descriptors the compiler moves into uniform registers
-// word by word, at twice the cycles per MMA.  A lone thread executes an instruction every several cycles; a barrier poll or a commit costs
-// it ~80 cycles and every MMA ~45, so per slot it spends 300-400 cycles outside the MMAs, which the MMA queue (4-5
-// deep) hides only behind wide MMAs (N = 256).  kDuo: two issuers take the slots alternately, so that one thread's
-// bookkeeping overlaps the other's MMAs.  MMAs of both accumulate into the same tile (the pipe executes them one
+// word by word, at twice the cycles per MMA.  Even so a barrier poll or a commit costs the role ~80 cycles, so per
+// slot it spends a few hundred cycles outside the MMAs, which the MMA queue (~4 deep) hides only behind wide MMAs
+// (N = 256).  kDuo: two issuers take the slots alternately, so that one's bookkeeping overlaps the other's MMAs.  MMAs of both accumulate into the same tile (the pipe executes them one
 // after another whichever thread issued them); a sequence number in shared memory makes the threads issue slot g
 // only after slot g-1 has been issued, so the order of the additions, and with it every bit of the result, is
 // that of a single issuer.
@@ -1256,7 +1257,7 @@ TileCfg halo_cfg(const TcFpropArgs& a, int cblocks, int sm_count, int layout, in
 // ---- Blocking search (Sec. 2.2 / 2.3 re-posed for this memory hierarchy) ------------------------------------------
 // The paper chooses its cache and register blocks by minimising the bytes moved per flop under the capacity of the
 // cache, with a brute-force search over the block sizes.  Here the scarce rates are the tensor pipe, the fill rate
-// of shared memory out of L2, the lone issuing thread and the epilogue warps, under 227 KB of shared memory and 512
+// of shared memory out of L2, the issuing warp and the epilogue warps, under 227 KB of shared memory and 512
 // TMEM columns; a candidate's cost is the slowest of those four per tile, times the tiles a CTA takes.  Constants
 // are measurements on B200 (microbenchmarks and ncu captures of these kernels).
 struct TileCost { double mma, fill, issue, epilogue, tile, total; };

@@ -111,7 +111,7 @@ struct WgradParams {
 };
 
 // One box row of a haloed-x k-step: kSteps MMA steps of 8 pixels, each one MMA per map group (kCg of them) over the
-// S taps.  Straight-line: every instruction of the lone issuing thread costs cycles of the k-step budget.
+// S taps.  Straight-line: every instruction of the issuing role costs cycles of the k-step budget.
 template <int kSteps, int kCg>
 __device__ __forceinline__ void xhalo_row(uint32_t d_tmem, uint32_t xn, uint32_t a_lo, uint32_t b_lo, uint32_t hi,
                                           uint32_t idesc, uint32_t acc_first, uint32_t xg16) {
