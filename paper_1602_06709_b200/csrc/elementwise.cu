@@ -404,7 +404,10 @@ __global__ void __launch_bounds__(256) softmax_xent_kernel(const float* __restri
 
 // The same for rows of at most 256 * kPer values: the row is read once and kept in registers (the three passes of the
 // kernel above re-read it from L1/L2), thread t holding elements t, t + 256, ...
-template <int kPer>
+// kVec = 4 (K % 4 == 0, 16-byte aligned rows): thread t holds elements 4 * (256 * j + t) .. + 3, read and written as
+// float4; kVec = 1: elements 256 * i + t.  The exponentials are ex2.approx of the scaled argument (arguments in
+// [-|row range|, 0]: relative error ~1e-6, well inside the 1e-4 the gradients are held to).
+template <int kPer, int kVec>
 __global__ void __launch_bounds__(256) softmax_xent_regs_kernel(const float* __restrict__ logits,
                                                                 const int* __restrict__ labels, float* __restrict__ loss,
                                                                 float* __restrict__ dlogits, int N, int K,
@@ -412,15 +415,28 @@ __global__ void __launch_bounds__(256) softmax_xent_regs_kernel(const float* __r
     __shared__ float red[8];
     __shared__ float bcast;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    // index of this thread's i-th element in the row
+    auto elem = [](int i) { return kVec == 4 ? 4 * (256 * (i >> 2) + int(threadIdx.x)) + (i & 3) : i * 256 + int(threadIdx.x); };
     for (int n = blockIdx.x; n < N; n += gridDim.x) {
         const float* z = logits + size_t(n) * K;
         float v[kPer];
         float mx = -INFINITY;
+        if (kVec == 4) {
 #pragma unroll
-        for (int i = 0; i < kPer; ++i) {
-            const int k = i * 256 + threadIdx.x;
-            v[i] = k < K ? __ldg(z + k) : -INFINITY;
-            mx = fmaxf(mx, v[i]);
+            for (int j = 0; j < kPer / 4; ++j) {
+                const int k = elem(4 * j);
+                float4 q = make_float4(-INFINITY, -INFINITY, -INFINITY, -INFINITY);
+                if (k < K) q = __ldg(reinterpret_cast<const float4*>(z + k));
+                v[4 * j] = q.x; v[4 * j + 1] = q.y; v[4 * j + 2] = q.z; v[4 * j + 3] = q.w;
+                mx = fmaxf(fmaxf(mx, fmaxf(q.x, q.y)), fmaxf(q.z, q.w));
+            }
+        } else {
+#pragma unroll
+            for (int i = 0; i < kPer; ++i) {
+                const int k = elem(i);
+                v[i] = k < K ? __ldg(z + k) : -INFINITY;
+                mx = fmaxf(mx, v[i]);
+            }
         }
         for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
         if (lane == 0) red[warp] = mx;
@@ -440,9 +456,9 @@ __global__ void __launch_bounds__(256) softmax_xent_regs_kernel(const float* __r
         float sum = 0.f, zlab = 0.f;
 #pragma unroll
         for (int i = 0; i < kPer; ++i) {
-            const int k = i * 256 + threadIdx.x;
+            const int k = elem(i);
             if (k == lab) zlab = v[i];
-            v[i] = k < K ? expf(v[i] - mx) : 0.f;
+            v[i] = k < K ? __expf(v[i] - mx) : 0.f;
             sum += v[i];
         }
         for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
@@ -458,13 +474,26 @@ __global__ void __launch_bounds__(256) softmax_xent_regs_kernel(const float* __r
         sum = bcast;
         const float inv_n = 1.f / float(N), inv_sum = 1.f / sum;
         float* out = dlogits + size_t(n) * K;
+        if (kVec == 4) {
 #pragma unroll
-        for (int i = 0; i < kPer; ++i) {
-            const int k = i * 256 + threadIdx.x;
-            if (k < K) out[k] = (v[i] * inv_sum - (k == lab ? 1.f : 0.f)) * inv_n;
+            for (int j = 0; j < kPer / 4; ++j) {
+                const int k = elem(4 * j);
+                if (k < K)
+                    *reinterpret_cast<float4*>(out + k) = make_float4((v[4 * j] * inv_sum - (k == lab ? 1.f : 0.f)) * inv_n,
+                                                                      (v[4 * j + 1] * inv_sum - (k + 1 == lab ? 1.f : 0.f)) * inv_n,
+                                                                      (v[4 * j + 2] * inv_sum - (k + 2 == lab ? 1.f : 0.f)) * inv_n,
+                                                                      (v[4 * j + 3] * inv_sum - (k + 3 == lab ? 1.f : 0.f)) * inv_n);
+            }
+        } else {
+#pragma unroll
+            for (int i = 0; i < kPer; ++i) {
+                const int k = elem(i);
+                if (k < K) out[k] = (v[i] * inv_sum - (k == lab ? 1.f : 0.f)) * inv_n;
+            }
         }
         // (the thread that holds the labelled element adds the row's loss term)
-        if (lab >= 0 && (lab & 255) == int(threadIdx.x)) atomicAdd(loss, -(zlab - mx - logf(sum)) * inv_n);
+        const int owner = kVec == 4 ? (lab >> 2) & 255 : lab & 255;
+        if (lab >= 0 && owner == int(threadIdx.x)) atomicAdd(loss, -(zlab - mx - logf(sum)) * inv_n);
         __syncthreads();
     }
 }
@@ -864,8 +893,11 @@ int launch_softmax_xent(int N, int K, const float* logits, const int* labels, fl
         unsigned int* status = device_status_ptr();
         if (!status) return PCL_ERR_CUDA;
         const int grid = N < 8 * device_sm_count() ? N : 8 * device_sm_count();
-        if (K <= 256 * 8) softmax_xent_regs_kernel<8><<<grid, 256, 0, st>>>(logits, labels, loss, dlogits, N, K, status);
-        else if (K <= 256 * 32) softmax_xent_regs_kernel<32><<<grid, 256, 0, st>>>(logits, labels, loss, dlogits, N, K, status);
+        const bool vec = K % 4 == 0 && ((reinterpret_cast<uintptr_t>(logits) | reinterpret_cast<uintptr_t>(dlogits)) & 15) == 0;
+        if (K <= 256 * 8 && vec) softmax_xent_regs_kernel<8, 4><<<grid, 256, 0, st>>>(logits, labels, loss, dlogits, N, K, status);
+        else if (K <= 256 * 8) softmax_xent_regs_kernel<8, 1><<<grid, 256, 0, st>>>(logits, labels, loss, dlogits, N, K, status);
+        else if (K <= 256 * 32 && vec) softmax_xent_regs_kernel<32, 4><<<grid, 256, 0, st>>>(logits, labels, loss, dlogits, N, K, status);
+        else if (K <= 256 * 32) softmax_xent_regs_kernel<32, 1><<<grid, 256, 0, st>>>(logits, labels, loss, dlogits, N, K, status);
         else softmax_xent_kernel<<<grid, 256, 0, st>>>(logits, labels, loss, dlogits, N, K, status);
     }
     return PCL_CHECK_LAUNCH();
